@@ -1,0 +1,121 @@
+"""Architecture tables for the networks the paper evaluates (Section 3).
+
+An architecture is a dict::
+
+    {"name": str, "in_c": int, "in_h": int, "in_w": int, "n_classes": int,
+     "layers": [layer, ...]}
+
+and a layer is a dict with the keys
+
+    name      label used in reports
+    kind      "conv" (dense k x k), "dw" (depthwise k x k) or "fc"
+    cin, cout channel counts ("dw": cin == cout)
+    k, stride, pad
+    act       "none", "relu" or "relu6", applied after bias and residual add
+    input     index of the layer whose output feeds this one, -1 = network input
+    residual  index of the layer whose output is added before `act`, -1 = none
+    has_bn    True when the layer is followed by batch normalisation
+
+The list order is the order of the scheme vector q = (q_1 .. q_L) of Section 2.1:
+one bit-width per weight tensor.  An "fc" layer consumes the global average pool
+of its input layer's output.  Only shapes and wiring live here; no arithmetic.
+"""
+
+
+def _conv(name, cin, cout, k, stride, act, inp, residual=-1, kind="conv"):
+    return dict(name=name, kind=kind, cin=cin, cout=cout, k=k, stride=stride,
+                pad=k // 2, act=act, input=inp, residual=residual, has_bn=True)
+
+
+def _fc(name, cin, cout, inp):
+    return dict(name=name, kind="fc", cin=cin, cout=cout, k=1, stride=1, pad=0,
+                act="none", input=inp, residual=-1, has_bn=False)
+
+
+def resnet20(channels=(16, 32, 64), n_classes=10, in_hw=32, name="resnet20"):
+    """CIFAR ResNet-20 with 1x1 projection shortcuts where shape changes.
+
+    Stem conv3x3, three stages of three basic blocks, global average pool,
+    linear classifier.  Scheme order: stem; per block conv1, conv2, then the
+    block's projection (if any); classifier last.
+    """
+    layers = [_conv("stem", 3, channels[0], 3, 1, "relu", -1)]
+    prev = 0            # index of the layer producing the current block input
+    cin = channels[0]
+    for si, c in enumerate(channels):
+        for b in range(3):
+            stride = 2 if (si > 0 and b == 0) else 1
+            need_proj = stride != 1 or cin != c
+            i1 = len(layers)
+            i2 = i1 + 1
+            ip = i1 + 2
+            layers.append(_conv(f"s{si + 1}.b{b}.c1", cin, c, 3, stride, "relu", prev))
+            layers.append(_conv(f"s{si + 1}.b{b}.c2", c, c, 3, 1, "relu", i1,
+                                residual=ip if need_proj else prev))
+            if need_proj:
+                layers.append(_conv(f"s{si + 1}.b{b}.proj", cin, c, 1, stride, "none", prev))
+            prev = i2
+            cin = c
+    layers.append(_fc("fc", cin, n_classes, prev))
+    return dict(name=name, in_c=3, in_h=in_hw, in_w=in_hw, n_classes=n_classes, layers=layers)
+
+
+_MBV2_CFG = [(1, 16, 1), (6, 24, 2), (6, 32, 3), (6, 64, 4), (6, 96, 3), (6, 160, 3), (6, 320, 1)]
+
+
+def mobilenet_v2(variant="cifar"):
+    """MobileNetV2, width 1.0.
+
+    variant "cifar":    32x32 input, stem stride 1, stage strides (1,1,1,2,1,2,1), 10 classes.
+    variant "imagenet": 224x224 input, stem stride 2, stage strides (1,2,2,2,1,2,1), 1000 classes.
+    """
+    if variant == "cifar":
+        hw, stem_stride, strides, n_classes = 32, 1, (1, 1, 1, 2, 1, 2, 1), 10
+    elif variant == "imagenet":
+        hw, stem_stride, strides, n_classes = 224, 2, (1, 2, 2, 2, 1, 2, 1), 1000
+    else:
+        raise ValueError(variant)
+    layers = [_conv("stem", 3, 32, 3, stem_stride, "relu6", -1)]
+    prev, cin, bi = 0, 32, 0
+    for (t, c, n), s0 in zip(_MBV2_CFG, strides):
+        for i in range(n):
+            stride = s0 if i == 0 else 1
+            hid = cin * t
+            src = prev
+            if t != 1:
+                layers.append(_conv(f"b{bi}.expand", cin, hid, 1, 1, "relu6", src))
+                src = len(layers) - 1
+            layers.append(_conv(f"b{bi}.dw", hid, hid, 3, stride, "relu6", src, kind="dw"))
+            src = len(layers) - 1
+            use_res = stride == 1 and cin == c
+            layers.append(_conv(f"b{bi}.project", hid, c, 1, 1, "none", src,
+                                residual=prev if use_res else -1))
+            prev = len(layers) - 1
+            cin = c
+            bi += 1
+    layers.append(_conv("head", cin, 1280, 1, 1, "relu6", prev))
+    layers.append(_fc("fc", 1280, n_classes, len(layers) - 1))
+    return dict(name=f"mobilenet_v2_{variant}", in_c=3, in_h=hw, in_w=hw,
+                n_classes=n_classes, layers=layers)
+
+
+def tiny_net(in_c=3, hw=8, n_classes=5):
+    """A small network touching every layer kind and wiring form (test workload)."""
+    layers = [
+        _conv("stem", in_c, 8, 3, 1, "relu", -1),
+        _conv("b0.c1", 8, 16, 3, 2, "relu", 0),
+        _conv("b0.c2", 16, 16, 3, 1, "relu", 1, residual=3),
+        _conv("b0.proj", 8, 16, 1, 2, "none", 0),
+        _conv("b1.expand", 16, 48, 1, 1, "relu6", 2),
+        _conv("b1.dw", 48, 48, 3, 1, "relu6", 4, kind="dw"),
+        _conv("b1.project", 48, 16, 1, 1, "none", 5, residual=2),
+        _conv("b2.dw", 16, 16, 3, 2, "relu6", 6, kind="dw"),
+        _conv("b2.project", 16, 24, 1, 1, "none", 7),
+        _fc("fc", 24, n_classes, 8),
+    ]
+    return dict(name="tiny_net", in_c=in_c, in_h=hw, in_w=hw, n_classes=n_classes, layers=layers)
+
+
+def conv_layer_indices(arch):
+    """Indices of every layer that is not the classifier (the sweep candidates)."""
+    return [i for i, l in enumerate(arch["layers"]) if l["kind"] != "fc"]
