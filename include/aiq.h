@@ -1,0 +1,236 @@
+/*
+ * aiq.h - C ABI of the B200 (sm_100a) scheme evaluator for Arithmetic-Intensity-Aware
+ * Quantization (AIQ).
+ *
+ * The paper (Section 2.1) assigns every layer i of a trained CNN a bit-width q_i from a
+ * small set Q, forming a scheme q = (q_1 .. q_L), and scores a scheme by (i) its global
+ * arithmetic intensity AI(q), computed analytically, and (ii) its accuracy, measured by
+ * running the quantized model (Section 1).  Both search loops of Section 2.2 spend their
+ * time in (ii).  This library is that evaluation path:
+ *
+ *   aiq_fold_bn          fold batch-norm into the preceding convolution
+ *   aiq_quantize_layer   quantize + pack one layer's weights at 4 / 8 / 16 / 32 bits
+ *   aiq_qlinear          y = x * dequant(W)^T for a packed weight matrix (small batch)
+ *   aiq_model_create     fold, then build the L x {4,8,16,32} bank of packed weights
+ *   aiq_forward          logits of one scheme on one image batch
+ *   aiq_eval_schemes     top-1 agreement of many schemes on an image set
+ *   aiq_scheme_ai        AI(q), on the host
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
+ *     ordinary host memory.  The library never allocates or frees device memory: the
+ *     caller provides model memory and workspace and keeps them alive while they are used.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Every function returns an aiq_status_t (0 = AIQ_OK) unless stated; nothing throws.
+ *     aiq_last_error() gives a thread-local detail string for the last non-zero status.
+ *   - Bit-widths: 4 and 8 are symmetric integer codes with one float32 scale per output
+ *     channel; 16 is IEEE half; 32 is float32.  Anything else: AIQ_ERR_UNSUPPORTED_BITS.
+ *   - There is no CPU fallback: on a device that is not compute capability 10.x every
+ *     entry point that would launch a kernel returns AIQ_ERR_NOT_SM100.
+ */
+#ifndef AIQ_H_
+#define AIQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int aiq_status_t;
+enum {
+  AIQ_OK = 0,
+  AIQ_ERR_INVALID_ARG = 1,       /* null pointer, non-positive size, bad wiring              */
+  AIQ_ERR_UNSUPPORTED_BITS = 2,  /* bit-width outside {4, 8, 16, 32}                         */
+  AIQ_ERR_SHAPE = 3,             /* layer shapes inconsistent with the wiring                */
+  AIQ_ERR_WORKSPACE_TOO_SMALL = 4,
+  AIQ_ERR_CUDA = 5,              /* a CUDA runtime call failed; see aiq_last_error()         */
+  AIQ_ERR_NOT_SM100 = 6,
+  AIQ_ERR_NONFINITE = 7,         /* a weight was NaN or infinite                             */
+  AIQ_ERR_TIMEOUT = 8            /* a bounded device-side wait expired                       */
+};
+
+/* Static description of a status code. Never NULL. */
+const char* aiq_status_string(aiq_status_t status);
+/* Thread-local detail of the last failure on this thread ("" if none). */
+const char* aiq_last_error(void);
+
+/* ------------------------------------------------------------------------------------
+ * Batch-norm folding.  The paper evaluates a trained model as-is (Section 3); folding the
+ * inference batch-norm into the convolution before quantizing is this library's stated
+ * reading.  Per output channel n:
+ *     g = gamma[n] / sqrt(var[n] + eps);   Wf[n][k] = W[n][k] * g;   bf[n] = beta[n] - mean[n] * g
+ * float32, every operation rounded once (no fused multiply-add, IEEE division and sqrt).
+ * W, Wf: device [N][K] row-major (K = cin/groups * kh * kw in (c, r, t) order);
+ * gamma, beta, mean, var, bf: device [N].  Wf may alias W.  Asynchronous on `stream`.
+ */
+aiq_status_t aiq_fold_bn(const float* W, const float* gamma, const float* beta,
+                         const float* mean, const float* var, int N, int K, float eps,
+                         float* Wf, float* bf, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Quantize + pack (Section 2.1: layer i is stored at q_i bits; the paper prints no
+ * quantizer formula, so the rule is: symmetric, per output channel, max-abs scale, round
+ * half to even).  For row n of W [N][K]:
+ *   bits 4 / 8: qmax = 2^(bits-1) - 1; amax = max_k |W[n][k]|; s_n = amax / qmax (IEEE
+ *               float32 division; s_n = 1 when amax == 0);
+ *               code = clamp(rint(W[n][k] / s_n), -2^(bits-1), 2^(bits-1) - 1)
+ *   bits 16:    IEEE half, round to nearest even;  s_n = 1
+ *   bits 32:    bit copy;                          s_n = 1
+ * Packed layout: row-major, row stride aiq_packed_row_bytes(K, bits) = Kpad * bits / 8 with
+ * Kpad = K rounded up to a multiple of 32 elements; padding elements are zero.  At 4 bits
+ * byte j of a row holds element 2j in its low nibble and element 2j+1 in its high nibble,
+ * two's complement.  16- and 32-bit elements are little endian.
+ *
+ * W: device float32 [N][K].  packed_out: device, N * row_bytes, 16-byte aligned.
+ * scales_out: device float32 [N].  nonfinite_flag: optional device int32; set to 1 when a
+ * NaN or infinity is met (outputs are then unspecified); never cleared by the call.
+ * Asynchronous on `stream`.
+ */
+size_t aiq_packed_row_bytes(int K, int bits);   /* 0 for an unsupported bits or K <= 0 */
+aiq_status_t aiq_quantize_layer(const float* W, int N, int K, int bits, void* packed_out,
+                                float* scales_out, int32_t* nonfinite_flag, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Small-batch quantized linear layer - the memory-bound case the method targets
+ * (Abstract; Section 5, Roofline paragraph): weight bytes N*K*bits/8 dominate the traffic.
+ *     y[m][n] = s_n * sum_k code[n][k] * x[m][k] + bias[n]
+ * (16 / 32 bits: the stored element itself, s_n = 1).  float32 multiply-add, float32
+ * accumulation.  packed / scales: as written by aiq_quantize_layer (device).  bias: device
+ * [N] or NULL.  x: device float32 [M][K] row-major, 16-byte aligned; y: device float32
+ * [M][N].  M >= 1.  Asynchronous on `stream`.
+ */
+aiq_status_t aiq_qlinear(const void* packed, const float* scales, const float* bias, int N,
+                         int K, int bits, const float* x, int M, float* y, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Model description.  Layers are listed in scheme order: entry i of a scheme is the
+ * bit-width of layers[i] (Section 2.1).  A layer reads the output of layer `input`
+ * (-1 = the network input) and, before its activation, adds the output of layer
+ * `residual` (-1 = none).  `input` / `residual` may refer to a later entry (a block's
+ * projection shortcut is listed after the convolution that adds it); the wiring must be
+ * acyclic.  An AIQ_LAYER_FC layer consumes the global average pool of its input layer.
+ * The last layer produces the logits.
+ */
+enum { AIQ_LAYER_CONV = 0, AIQ_LAYER_DEPTHWISE = 1, AIQ_LAYER_FC = 2 };
+enum { AIQ_ACT_NONE = 0, AIQ_ACT_RELU = 1, AIQ_ACT_RELU6 = 2 };
+
+typedef struct aiq_layer_desc {
+  int32_t kind;      /* AIQ_LAYER_*                                        */
+  int32_t cin;       /* input channels (depthwise: == cout)                */
+  int32_t cout;      /* output channels / classes                          */
+  int32_t ksize;     /* square kernel: 1 or 3 (fc: 1)                      */
+  int32_t stride;    /* 1 or 2                                             */
+  int32_t pad;       /* zero padding on each side                          */
+  int32_t act;       /* AIQ_ACT_*, applied after bias and residual         */
+  int32_t input;     /* producing layer, -1 = network input                */
+  int32_t residual;  /* layer added before the activation, -1 = none       */
+  int32_t has_bn;    /* 1: gamma/beta/mean/var given and folded; 0: bias   */
+} aiq_layer_desc_t;
+
+typedef struct aiq_arch_desc {
+  int32_t n_layers;
+  int32_t in_c, in_h, in_w;        /* network input, NCHW                  */
+  const aiq_layer_desc_t* layers;  /* host [n_layers]                      */
+} aiq_arch_desc_t;
+
+/* Host pointers to one layer's trained float32 parameters.  W: [cout][cin/groups][k][k]
+ * (fc: [cout][cin]).  has_bn: gamma, beta, mean, var [cout], bias ignored.  Otherwise
+ * bias [cout] (NULL = zeros) and the batch-norm pointers are ignored. */
+typedef struct aiq_layer_weights {
+  const float* W;
+  const float* gamma;
+  const float* beta;
+  const float* mean;
+  const float* var;
+  const float* bias;
+} aiq_layer_weights_t;
+
+typedef struct aiq_model aiq_model_t;   /* opaque host object */
+
+/* Device bytes aiq_model_create needs for `arch` (folded weights, biases, the packed
+ * weight bank at all four bit-widths, scales).  0 on an invalid description. */
+size_t aiq_model_bytes(const aiq_arch_desc_t* arch);
+
+/* Uploads the weights, folds batch-norm (eps = 1e-5) and quantizes every layer at 4, 8,
+ * 16 and 32 bits into `dev_mem` (device, 256-byte aligned, >= aiq_model_bytes(arch)).
+ * A layer's quantized weights depend only on (layer, bits), so a scheme is an index vector
+ * into this bank.  Synchronises `stream` before returning.  The model refers to `dev_mem`
+ * until aiq_model_destroy; the arch and weight arrays are copied and may be freed.
+ * Errors: AIQ_ERR_INVALID_ARG / AIQ_ERR_SHAPE (wiring, shapes), AIQ_ERR_WORKSPACE_TOO_SMALL
+ * (dev_bytes), AIQ_ERR_NONFINITE, AIQ_ERR_NOT_SM100, AIQ_ERR_CUDA.  *out is NULL on error. */
+aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_layer_weights_t* weights,
+                              void* dev_mem, size_t dev_bytes, void* stream, aiq_model_t** out);
+/* Frees the host object only (device memory belongs to the caller). NULL is accepted. */
+void aiq_model_destroy(aiq_model_t* model);
+int aiq_model_num_layers(const aiq_model_t* model);   /* L, the scheme length; -1 if NULL */
+int aiq_model_num_classes(const aiq_model_t* model);  /* cout of the last layer           */
+
+/* Device views into the model memory, for inspection: folded weights Wf [cout][K] and bias
+ * [cout] of `layer`; packed rows and scales of (`layer`, `bits`) in the layout of
+ * aiq_quantize_layer.  Any output pointer may be NULL. */
+aiq_status_t aiq_model_layer_folded(const aiq_model_t* model, int layer, const float** Wf,
+                                    const float** bias, int* N, int* K);
+aiq_status_t aiq_model_layer_packed(const aiq_model_t* model, int layer, int bits,
+                                    const void** packed, const float** scales);
+
+/* Workspace bytes sufficient for aiq_forward with batch <= max_batch and for
+ * aiq_eval_schemes with n_schemes <= max_schemes processing max_batch images at a time. */
+size_t aiq_workspace_bytes(const aiq_model_t* model, int max_batch, int max_schemes);
+
+/* ------------------------------------------------------------------------------------
+ * One scheme, one batch (Section 1 (ii): the quantized model is run).  scheme_bits: host
+ * uint8 [L].  x: device float32 NCHW [batch][in_c][in_h][in_w].  logits: device float32
+ * [batch][n_classes].  Layer l uses the bank entry (l, scheme_bits[l]); weights are
+ * expanded from their packed form inside the kernels, products accumulate in float32, the
+ * per-channel scale multiplies the finished sum.  workspace: device, 256-byte aligned.
+ * Asynchronous on `stream` (the scheme is consumed before the call returns).
+ */
+aiq_status_t aiq_forward(const aiq_model_t* model, const uint8_t* scheme_bits, const float* x,
+                         int batch, float* logits, void* workspace, size_t workspace_bytes,
+                         void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Many candidate schemes, whole evaluation set - the inner loop of greedy search and
+ * coordinate descent (Section 2.2), which evaluates L(q; lambda) for every candidate move
+ * and so needs each candidate's accuracy on the validation images.
+ * schemes: host uint8 [n_schemes][L].  x: device float32 NCHW [n_images][...].  labels:
+ * device int32 [n_images].  acc: host float32 [n_schemes] = correct / n_images, where a
+ * prediction is the lowest index attaining the maximum logit.  correct_counts: optional
+ * host int32 [n_schemes].  preds: optional device int32 [n_schemes][n_images].
+ * Images are processed in chunks sized to the workspace; within a chunk, work shared by
+ * candidates (equal bit-widths on a common prefix of the network) is done once, which
+ * does not change any result.  Synchronises `stream` before returning.
+ */
+aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t* schemes, int n_schemes,
+                              const float* x, const int32_t* labels, int n_images, float* acc,
+                              int32_t* correct_counts, int32_t* preds, void* workspace,
+                              size_t workspace_bytes, void* stream);
+
+/* Evaluation knobs (process-wide, for experiments and tests; results never depend on
+ * them).  chunk: images per pass, 0 = choose from the workspace size.  share_prefix: 0
+ * evaluates every scheme independently. */
+void aiq_set_eval_options(int chunk, int share_prefix);
+
+/* Counters of the last aiq_forward / aiq_eval_schemes call on this thread: kernels
+ * launched, and layer evaluations executed vs. n_schemes * L * chunks without sharing. */
+void aiq_last_call_stats(int64_t* kernel_launches, int64_t* layer_evals, int64_t* layer_evals_unshared);
+
+/* ------------------------------------------------------------------------------------
+ * Analytic global arithmetic intensity (Section 1 (i); Section 2.2: "AI can be recomputed
+ * analytically").  The paper gives no formula; this one is used:
+ *     FLOPs_l = 2 * cout * K * Ho * Wo * ai_batch
+ *     Bytes_l = cout * K * q_l / 8 + 4 * ai_batch * (cin * Hi * Wi + cout * Ho * Wo)
+ *     AI(q)   = sum_l FLOPs_l / sum_l Bytes_l          [FLOP / byte]
+ * over every weight layer; biases, scales, activations functions, residual adds and
+ * pooling count for nothing.  Host only, no CUDA call.  ai, flops, bytes: host doubles
+ * (each may be NULL).
+ */
+aiq_status_t aiq_scheme_ai(const aiq_model_t* model, const uint8_t* scheme_bits, int ai_batch,
+                           double* ai, double* flops, double* bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AIQ_H_ */

@@ -1,0 +1,294 @@
+"""ctypes binding of libaiq.so: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (see include/aiq.h) and
+does nothing but convert arguments: torch tensors supply device pointers and the current
+stream, NumPy arrays supply host pointers.  All arithmetic runs inside the CUDA library;
+if the library is missing the import of this module fails.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libaiq.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED_BITS, ERR_SHAPE, ERR_WORKSPACE_TOO_SMALL = 1, 2, 3, 4
+ERR_CUDA, ERR_NOT_SM100, ERR_NONFINITE, ERR_TIMEOUT = 5, 6, 7, 8
+
+LAYER_KIND = {"conv": 0, "dw": 1, "fc": 2}
+ACT = {"none": 0, "relu": 1, "relu6": 2}
+
+EXPORTS = [
+    "aiq_status_string", "aiq_last_error", "aiq_fold_bn", "aiq_packed_row_bytes",
+    "aiq_quantize_layer", "aiq_qlinear", "aiq_model_bytes", "aiq_model_create",
+    "aiq_model_destroy", "aiq_model_num_layers", "aiq_model_num_classes",
+    "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
+    "aiq_eval_schemes", "aiq_set_eval_options", "aiq_last_call_stats", "aiq_scheme_ai",
+]
+
+
+class AiqError(RuntimeError):
+    def __init__(self, status, detail):
+        super().__init__(f"aiq status {status} ({status_string(status)}): {detail}")
+        self.status = status
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("kind", "cin", "cout", "ksize", "stride", "pad", "act",
+                                         "input", "residual", "has_bn")]
+
+
+class ArchDesc(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("in_c", C.c_int32), ("in_h", C.c_int32),
+                ("in_w", C.c_int32), ("layers", C.POINTER(LayerDesc))]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("W", "gamma", "beta", "mean", "var", "bias")]
+
+
+def _load():
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} is missing: build it with "
+                          "`python -m paper_2512_14090_b200.build` (there is no fallback path)")
+    lib = C.CDLL(_LIB_PATH)
+    vp, i32, f32, sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
+    lib.aiq_status_string.restype = C.c_char_p
+    lib.aiq_status_string.argtypes = [i32]
+    lib.aiq_last_error.restype = C.c_char_p
+    lib.aiq_last_error.argtypes = []
+    lib.aiq_fold_bn.restype = i32
+    lib.aiq_fold_bn.argtypes = [vp, vp, vp, vp, vp, i32, i32, f32, vp, vp, vp]
+    lib.aiq_packed_row_bytes.restype = sz
+    lib.aiq_packed_row_bytes.argtypes = [i32, i32]
+    lib.aiq_quantize_layer.restype = i32
+    lib.aiq_quantize_layer.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.aiq_qlinear.restype = i32
+    lib.aiq_qlinear.argtypes = [vp, vp, vp, i32, i32, i32, vp, i32, vp, vp]
+    lib.aiq_model_bytes.restype = sz
+    lib.aiq_model_bytes.argtypes = [C.POINTER(ArchDesc)]
+    lib.aiq_model_create.restype = i32
+    lib.aiq_model_create.argtypes = [C.POINTER(ArchDesc), C.POINTER(LayerWeights), vp, sz, vp,
+                                     C.POINTER(vp)]
+    lib.aiq_model_destroy.restype = None
+    lib.aiq_model_destroy.argtypes = [vp]
+    lib.aiq_model_num_layers.restype = i32
+    lib.aiq_model_num_layers.argtypes = [vp]
+    lib.aiq_model_num_classes.restype = i32
+    lib.aiq_model_num_classes.argtypes = [vp]
+    lib.aiq_model_layer_folded.restype = i32
+    lib.aiq_model_layer_folded.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(i32),
+                                           C.POINTER(i32)]
+    lib.aiq_model_layer_packed.restype = i32
+    lib.aiq_model_layer_packed.argtypes = [vp, i32, i32, C.POINTER(vp), C.POINTER(vp)]
+    lib.aiq_workspace_bytes.restype = sz
+    lib.aiq_workspace_bytes.argtypes = [vp, i32, i32]
+    lib.aiq_forward.restype = i32
+    lib.aiq_forward.argtypes = [vp, vp, vp, i32, vp, vp, sz, vp]
+    lib.aiq_eval_schemes.restype = i32
+    lib.aiq_eval_schemes.argtypes = [vp, vp, i32, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+    lib.aiq_set_eval_options.restype = None
+    lib.aiq_set_eval_options.argtypes = [i32, i32]
+    lib.aiq_last_call_stats.restype = None
+    lib.aiq_last_call_stats.argtypes = [C.POINTER(C.c_int64)] * 3
+    lib.aiq_scheme_ai.restype = i32
+    lib.aiq_scheme_ai.argtypes = [vp, vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                  C.POINTER(C.c_double)]
+    return lib
+
+
+lib = _load()
+
+
+def status_string(status):
+    return lib.aiq_status_string(int(status)).decode()
+
+
+def last_error():
+    return lib.aiq_last_error().decode()
+
+
+def _check(status):
+    if status != OK:
+        raise AiqError(status, last_error())
+
+
+def _dev(t):
+    """Device pointer of a contiguous CUDA tensor (None -> NULL)."""
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return C.c_void_p(t.data_ptr())
+
+
+def _host(a):
+    return C.c_void_p(a.ctypes.data) if a is not None else None
+
+
+def _stream(stream=None):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def arch_desc(arch):
+    """(ArchDesc, keep-alive list) from an architecture dict (kind/cin/cout/k/...)."""
+    layers = (LayerDesc * len(arch["layers"]))()
+    for d, l in zip(layers, arch["layers"]):
+        d.kind, d.cin, d.cout, d.ksize = LAYER_KIND[l["kind"]], l["cin"], l["cout"], l["k"]
+        d.stride, d.pad, d.act = l["stride"], l["pad"], ACT[l["act"]]
+        d.input, d.residual, d.has_bn = l["input"], l["residual"], int(bool(l["has_bn"]))
+    desc = ArchDesc(len(arch["layers"]), arch["in_c"], arch["in_h"], arch["in_w"], layers)
+    return desc, layers
+
+
+# ------------------------------------------------------------------------- plain calls
+def aiq_packed_row_bytes(K, bits):
+    return int(lib.aiq_packed_row_bytes(int(K), int(bits)))
+
+
+def aiq_fold_bn(W, gamma, beta, mean, var, Wf, bf, eps=1e-5, stream=None):
+    N = W.shape[0]
+    K = W.numel() // N
+    _check(lib.aiq_fold_bn(_dev(W), _dev(gamma), _dev(beta), _dev(mean), _dev(var), N, K,
+                           C.c_float(eps), _dev(Wf), _dev(bf), _stream(stream)))
+
+
+def aiq_quantize_layer(W, bits, packed_out, scales_out, nonfinite_flag=None, stream=None):
+    N, K = W.shape
+    _check(lib.aiq_quantize_layer(_dev(W), N, K, int(bits), _dev(packed_out), _dev(scales_out),
+                                  _dev(nonfinite_flag), _stream(stream)))
+
+
+def aiq_qlinear(packed, scales, bias, N, K, bits, x, y, stream=None):
+    M = x.shape[0]
+    _check(lib.aiq_qlinear(_dev(packed), _dev(scales), _dev(bias), int(N), int(K), int(bits),
+                           _dev(x), int(M), _dev(y), _stream(stream)))
+
+
+def aiq_set_eval_options(chunk=0, share_prefix=True):
+    lib.aiq_set_eval_options(int(chunk), int(bool(share_prefix)))
+
+
+def aiq_last_call_stats():
+    a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
+    lib.aiq_last_call_stats(C.byref(a), C.byref(b), C.byref(c))
+    return dict(kernel_launches=a.value, layer_evals=b.value, layer_evals_unshared=c.value)
+
+
+# ------------------------------------------------------------------------- model object
+class Model:
+    """Owns the device memory the C model lives in (a torch uint8 tensor) and the handle."""
+
+    def __init__(self, arch, params, device="cuda:0", stream=None):
+        import torch
+        self.arch = arch
+        self.device = torch.device(device)
+        desc, self._keep_layers = arch_desc(arch)
+        self._desc = desc
+        nbytes = int(lib.aiq_model_bytes(C.byref(desc)))
+        if nbytes == 0:
+            raise AiqError(ERR_INVALID_ARG, last_error())
+        self.mem = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        weights = (LayerWeights * len(params))()
+        keep = []
+        for w, p in zip(weights, params):
+            for name in ("W", "gamma", "beta", "mean", "var", "bias"):
+                if name in p and p[name] is not None:
+                    a = np.ascontiguousarray(p[name], dtype=np.float32)
+                    keep.append(a)
+                    setattr(w, name, a.ctypes.data)
+        handle = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(lib.aiq_model_create(C.byref(desc), weights, _dev(self.mem), nbytes,
+                                        _stream(stream), C.byref(handle)))
+        self.handle = handle
+        self.n_layers = int(lib.aiq_model_num_layers(handle))
+        self.n_classes = int(lib.aiq_model_num_classes(handle))
+        self._ws = None
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib.aiq_model_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
+
+    # views for inspection --------------------------------------------------------
+    def layer_folded(self, layer):
+        """(Wf [N][K], bias [N]) as torch views into the model memory."""
+        wf, b, n, k = C.c_void_p(), C.c_void_p(), C.c_int(), C.c_int()
+        _check(lib.aiq_model_layer_folded(self.handle, layer, C.byref(wf), C.byref(b), C.byref(n), C.byref(k)))
+        return (self._view(wf.value, n.value * k.value * 4).view(dtype=_f32()).view(n.value, k.value),
+                self._view(b.value, n.value * 4).view(dtype=_f32()))
+
+    def layer_packed(self, layer, bits):
+        wf, b, n, k = C.c_void_p(), C.c_void_p(), C.c_int(), C.c_int()
+        _check(lib.aiq_model_layer_folded(self.handle, layer, C.byref(wf), C.byref(b), C.byref(n), C.byref(k)))
+        p, s = C.c_void_p(), C.c_void_p()
+        _check(lib.aiq_model_layer_packed(self.handle, layer, int(bits), C.byref(p), C.byref(s)))
+        rb = aiq_packed_row_bytes(k.value, bits)
+        return (self._view(p.value, n.value * rb).view(n.value, rb),
+                self._view(s.value, n.value * 4).view(dtype=_f32()))
+
+    def _view(self, ptr, nbytes):
+        off = ptr - self.mem.data_ptr()
+        assert 0 <= off and off + nbytes <= self.mem.numel()
+        return self.mem[off:off + nbytes]
+
+    # workspace -------------------------------------------------------------------
+    def aiq_workspace_bytes(self, max_batch, max_schemes):
+        return int(lib.aiq_workspace_bytes(self.handle, int(max_batch), int(max_schemes)))
+
+    def workspace(self, max_batch, max_schemes):
+        import torch
+        need = self.aiq_workspace_bytes(max_batch, max_schemes)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = None
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    # the calls -------------------------------------------------------------------
+    def aiq_forward(self, scheme_bits, x, logits=None, workspace=None, stream=None):
+        import torch
+        scheme = np.ascontiguousarray(scheme_bits, dtype=np.uint8)
+        if scheme.shape != (self.n_layers,):
+            raise ValueError("scheme length must equal the number of layers")
+        B = x.shape[0]
+        if logits is None:
+            logits = torch.empty((B, self.n_classes), dtype=torch.float32, device=self.device)
+        ws = workspace if workspace is not None else self.workspace(B, 1)
+        _check(lib.aiq_forward(self.handle, _host(scheme), _dev(x), B, _dev(logits), _dev(ws),
+                               ws.numel(), _stream(stream)))
+        return logits
+
+    def aiq_eval_schemes(self, schemes, x, labels, preds=None, workspace=None, chunk=256,
+                         stream=None):
+        schemes = np.ascontiguousarray(schemes, dtype=np.uint8)
+        if schemes.ndim != 2 or schemes.shape[1] != self.n_layers:
+            raise ValueError("schemes must be [S][L]")
+        S, N = schemes.shape[0], x.shape[0]
+        acc = np.zeros(S, dtype=np.float32)
+        counts = np.zeros(S, dtype=np.int32)
+        ws = workspace if workspace is not None else self.workspace(min(chunk, N), S)
+        _check(lib.aiq_eval_schemes(self.handle, _host(schemes), S, _dev(x), _dev(labels), N,
+                                    _host(acc), _host(counts), _dev(preds), _dev(ws), ws.numel(),
+                                    _stream(stream)))
+        return acc, counts
+
+    def aiq_scheme_ai(self, scheme_bits, ai_batch=1):
+        scheme = np.ascontiguousarray(scheme_bits, dtype=np.uint8)
+        if scheme.shape != (self.n_layers,):
+            raise ValueError("scheme length must equal the number of layers")
+        ai, fl, by = C.c_double(), C.c_double(), C.c_double()
+        _check(lib.aiq_scheme_ai(self.handle, _host(scheme), int(ai_batch), C.byref(ai), C.byref(fl),
+                                 C.byref(by)))
+        return ai.value, fl.value, by.value
+
+
+def _f32():
+    import torch
+    return torch.float32

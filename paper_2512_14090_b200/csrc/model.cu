@@ -1,0 +1,690 @@
+// Host side of the library: status plumbing, the model object (folded weights + the
+// L x {4,8,16,32} bank of packed weights), the evaluation plan that shares work between
+// candidate schemes, aiq_forward / aiq_eval_schemes, and the analytic arithmetic intensity.
+#include "common.cuh"
+
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <tuple>
+#include <vector>
+
+namespace aiq {
+
+// ---------------------------------------------------------------------------------------
+// status plumbing
+// ---------------------------------------------------------------------------------------
+static thread_local char t_err[512] = "";
+static thread_local int64_t t_launches = 0, t_layer_evals = 0, t_layer_evals_unshared = 0;
+static int g_opt_chunk = 0;
+static int g_opt_share = 1;
+
+aiq_status_t set_error(aiq_status_t status, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(t_err, sizeof(t_err), fmt, ap);
+  va_end(ap);
+  return status;
+}
+
+void count_launch() { ++t_launches; }
+
+aiq_status_t check_device_sm100() {
+  static int cached[64];   // 0 unknown, 1 ok, 2 not sm_100
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return set_error(AIQ_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  if (dev >= 0 && dev < 64 && cached[dev]) {
+    if (cached[dev] == 1) return AIQ_OK;
+    return set_error(AIQ_ERR_NOT_SM100, "device %d is not compute capability 10.x", dev);
+  }
+  int major = 0;
+  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (e != cudaSuccess) return set_error(AIQ_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
+  if (dev >= 0 && dev < 64) cached[dev] = (major == 10) ? 1 : 2;
+  if (major != 10) return set_error(AIQ_ERR_NOT_SM100, "device %d is compute capability %d.x, need 10.x", dev, major);
+  return AIQ_OK;
+}
+
+static const int kBitsList[4] = {4, 8, 16, 32};
+static inline int bits_index(int bits) { return bits == 4 ? 0 : bits == 8 ? 1 : bits == 16 ? 2 : bits == 32 ? 3 : -1; }
+
+}  // namespace aiq
+
+// ---------------------------------------------------------------------------------------
+// model object
+// ---------------------------------------------------------------------------------------
+struct LayerInfo {
+  aiq_layer_desc_t d;
+  int K, Hi, Wi, Ho, Wo;
+  size_t out_elems;        // per image
+  float* Wf;
+  float* bias;
+  uint8_t* packed[4];
+  float* scales[4];
+  int slot;                // activation slot of the output (-1: fc)
+};
+
+struct aiq_model {
+  std::vector<LayerInfo> layers;
+  int in_c, in_h, in_w;
+  std::vector<int> order;            // execution order (every layer after its operands)
+  std::vector<size_t> slot_elems;    // per-image capacity of each activation slot
+  void* dev_mem;
+  size_t dev_bytes;
+};
+
+namespace aiq {
+
+static aiq_status_t infer_shapes(const aiq_arch_desc_t* arch, std::vector<LayerInfo>& L, std::vector<int>& order) {
+  if (!arch || !arch->layers || arch->n_layers <= 0 || arch->in_c <= 0 || arch->in_h <= 0 || arch->in_w <= 0)
+    return set_error(AIQ_ERR_INVALID_ARG, "architecture description is empty");
+  const int n = arch->n_layers;
+  L.assign(n, LayerInfo());
+  for (int i = 0; i < n; ++i) {
+    L[i].d = arch->layers[i];
+    const aiq_layer_desc_t& d = L[i].d;
+    if (d.kind < AIQ_LAYER_CONV || d.kind > AIQ_LAYER_FC) return set_error(AIQ_ERR_INVALID_ARG, "layer %d: kind %d", i, d.kind);
+    if (d.act < AIQ_ACT_NONE || d.act > AIQ_ACT_RELU6) return set_error(AIQ_ERR_INVALID_ARG, "layer %d: act %d", i, d.act);
+    if (d.input < -1 || d.input >= n || d.input == i) return set_error(AIQ_ERR_INVALID_ARG, "layer %d: input %d", i, d.input);
+    if (d.residual < -1 || d.residual >= n || d.residual == i) return set_error(AIQ_ERR_INVALID_ARG, "layer %d: residual %d", i, d.residual);
+    if (d.cin <= 0 || d.cout <= 0) return set_error(AIQ_ERR_SHAPE, "layer %d: cin %d cout %d", i, d.cin, d.cout);
+    if (d.kind == AIQ_LAYER_FC) {
+      if (i != n - 1) return set_error(AIQ_ERR_INVALID_ARG, "layer %d: the classifier must be the last layer", i);
+      if (d.input < 0 || d.residual >= 0) return set_error(AIQ_ERR_INVALID_ARG, "layer %d: classifier wiring", i);
+    } else {
+      if (d.ksize < 1 || d.ksize > 7 || d.stride < 1 || d.stride > 4 || d.pad < 0 || d.pad > 3)
+        return set_error(AIQ_ERR_SHAPE, "layer %d: ksize %d stride %d pad %d", i, d.ksize, d.stride, d.pad);
+      if (d.kind == AIQ_LAYER_DEPTHWISE && (d.ksize != 3 || d.pad != 1 || d.cin != d.cout || (d.cout & 3) || d.input < 0))
+        return set_error(AIQ_ERR_SHAPE, "layer %d: depthwise must be 3x3, pad 1, cin == cout, channels a multiple of 4", i);
+    }
+  }
+  if (L[n - 1].d.kind != AIQ_LAYER_FC) return set_error(AIQ_ERR_INVALID_ARG, "the last layer must be a classifier (fc)");
+
+  // execution order: depth-first over operands; a cycle shows up as a revisit of an open node
+  order.clear();
+  std::vector<int> state(n, 0);
+  struct Frame { int layer, stage; };
+  for (int root = 0; root < n; ++root) {
+    if (state[root]) continue;
+    std::vector<Frame> st;
+    st.push_back({root, 0});
+    state[root] = 1;
+    while (!st.empty()) {
+      Frame& f = st.back();
+      const int dep = f.stage == 0 ? L[f.layer].d.input : f.stage == 1 ? L[f.layer].d.residual : -2;
+      if (dep == -2) {
+        state[f.layer] = 2;
+        order.push_back(f.layer);
+        st.pop_back();
+        continue;
+      }
+      ++f.stage;
+      if (dep < 0 || state[dep] == 2) continue;
+      if (state[dep] == 1) return set_error(AIQ_ERR_INVALID_ARG, "wiring has a cycle through layer %d", dep);
+      state[dep] = 1;
+      st.push_back({dep, 0});
+    }
+  }
+
+  for (int i : order) {
+    LayerInfo& li = L[i];
+    const aiq_layer_desc_t& d = li.d;
+    int cin_avail, hi, wi;
+    if (d.input < 0) { cin_avail = arch->in_c; hi = arch->in_h; wi = arch->in_w; }
+    else {
+      if (L[d.input].d.kind == AIQ_LAYER_FC) return set_error(AIQ_ERR_INVALID_ARG, "layer %d reads the classifier", i);
+      cin_avail = L[d.input].d.cout; hi = L[d.input].Ho; wi = L[d.input].Wo;
+    }
+    if (cin_avail != d.cin) return set_error(AIQ_ERR_SHAPE, "layer %d: cin %d but its input has %d channels", i, d.cin, cin_avail);
+    li.Hi = hi; li.Wi = wi;
+    if (d.kind == AIQ_LAYER_FC) {
+      li.K = d.cin; li.Hi = 1; li.Wi = 1; li.Ho = 1; li.Wo = 1; li.out_elems = d.cout;   // reads the pooled vector
+      continue;
+    }
+    li.Ho = (hi + 2 * d.pad - d.ksize) / d.stride + 1;
+    li.Wo = (wi + 2 * d.pad - d.ksize) / d.stride + 1;
+    if (li.Ho <= 0 || li.Wo <= 0) return set_error(AIQ_ERR_SHAPE, "layer %d: empty output", i);
+    li.K = (d.kind == AIQ_LAYER_DEPTHWISE ? 1 : d.cin) * d.ksize * d.ksize;
+    li.out_elems = (size_t)d.cout * li.Ho * li.Wo;
+    if (d.residual >= 0) {
+      const LayerInfo& r = L[d.residual];
+      if (r.d.kind == AIQ_LAYER_FC || r.d.cout != d.cout || r.Ho != li.Ho || r.Wo != li.Wo)
+        return set_error(AIQ_ERR_SHAPE, "layer %d: residual from layer %d has another shape", i, d.residual);
+    }
+  }
+  return AIQ_OK;
+}
+
+static void assign_slots(aiq_model* m) {
+  const int n = (int)m->layers.size();
+  std::vector<int> pos(n), last_use(n, -1);
+  for (int i = 0; i < n; ++i) pos[m->order[i]] = i;
+  for (int l = 0; l < n; ++l) {
+    const aiq_layer_desc_t& d = m->layers[l].d;
+    if (d.input >= 0) last_use[d.input] = std::max(last_use[d.input], pos[l]);
+    if (d.residual >= 0) last_use[d.residual] = std::max(last_use[d.residual], pos[l]);
+  }
+  std::vector<int> owner;   // layer currently held by each slot, -1 = free
+  m->slot_elems.clear();
+  for (int i = 0; i < n; ++i) {
+    const int l = m->order[i];
+    LayerInfo& li = m->layers[l];
+    if (li.d.kind == AIQ_LAYER_FC) { li.slot = -1; }
+    else {
+      int s = -1;
+      for (size_t k = 0; k < owner.size(); ++k) if (owner[k] < 0) { s = (int)k; break; }
+      if (s < 0) { s = (int)owner.size(); owner.push_back(-1); m->slot_elems.push_back(0); }
+      owner[s] = l;
+      li.slot = s;
+      m->slot_elems[s] = std::max(m->slot_elems[s], li.out_elems);
+    }
+    for (size_t k = 0; k < owner.size(); ++k)
+      if (owner[k] >= 0 && last_use[owner[k]] <= i && owner[k] != l) owner[k] = -1;
+    if (li.slot >= 0 && last_use[l] < 0) owner[li.slot] = -1;   // never consumed
+  }
+}
+
+struct ModelLayout { size_t total, staging_off, flag_off; std::vector<size_t> wf, bias; std::vector<size_t> packed[4], scales[4]; };
+
+static ModelLayout model_layout(const std::vector<LayerInfo>& L) {
+  ModelLayout lay;
+  size_t off = 0, staging = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  lay.flag_off = take(256);
+  for (const LayerInfo& li : L) {
+    const size_t n = li.d.cout, k = li.K;
+    lay.wf.push_back(take(n * k * 4));
+    lay.bias.push_back(take(n * 4));
+    for (int b = 0; b < 4; ++b) {
+      lay.packed[b].push_back(take(n * row_bytes((int)k, kBitsList[b])));
+      lay.scales[b].push_back(take(n * 4));
+    }
+    staging = std::max(staging, align_up(n * k * 4, 256) + 5 * align_up(n * 4, 256));
+  }
+  lay.staging_off = take(staging);
+  lay.total = off;
+  return lay;
+}
+
+}  // namespace aiq
+
+extern "C" size_t aiq_model_bytes(const aiq_arch_desc_t* arch) {
+  std::vector<LayerInfo> L;
+  std::vector<int> order;
+  if (aiq::infer_shapes(arch, L, order) != AIQ_OK) return 0;
+  return aiq::model_layout(L).total;
+}
+
+extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_layer_weights_t* weights,
+                                         void* dev_mem, size_t dev_bytes, void* stream_, aiq_model_t** out) {
+  using namespace aiq;
+  if (out) *out = nullptr;
+  if (!arch || !weights || !dev_mem || !out) return set_error(AIQ_ERR_INVALID_ARG, "aiq_model_create: null pointer");
+  if (((uintptr_t)dev_mem) & 255) return set_error(AIQ_ERR_INVALID_ARG, "aiq_model_create: dev_mem not 256-byte aligned");
+  aiq_model* m = new (std::nothrow) aiq_model();
+  if (!m) return set_error(AIQ_ERR_INVALID_ARG, "out of host memory");
+  aiq_status_t st = infer_shapes(arch, m->layers, m->order);
+  if (st != AIQ_OK) { delete m; return st; }
+  for (int i = 0; i < arch->n_layers; ++i) {
+    const aiq_layer_weights_t& w = weights[i];
+    if (!w.W || (m->layers[i].d.has_bn && (!w.gamma || !w.beta || !w.mean || !w.var))) {
+      delete m;
+      return set_error(AIQ_ERR_INVALID_ARG, "layer %d: missing weight pointers", i);
+    }
+  }
+  const ModelLayout lay = model_layout(m->layers);
+  if (dev_bytes < lay.total) {
+    delete m;
+    return set_error(AIQ_ERR_WORKSPACE_TOO_SMALL, "model needs %zu device bytes, got %zu", lay.total, dev_bytes);
+  }
+  st = check_device_sm100();
+  if (st != AIQ_OK) { delete m; return st; }
+  m->in_c = arch->in_c; m->in_h = arch->in_h; m->in_w = arch->in_w;
+  m->dev_mem = dev_mem; m->dev_bytes = dev_bytes;
+  assign_slots(m);
+  cudaStream_t stream = (cudaStream_t)stream_;
+  uint8_t* base = static_cast<uint8_t*>(dev_mem);
+  int32_t* flag = reinterpret_cast<int32_t*>(base + lay.flag_off);
+
+  auto fail = [&](aiq_status_t s) { delete m; return s; };
+#define CREATE_TRY(expr)                                                                    \
+  do {                                                                                      \
+    cudaError_t e__ = (expr);                                                               \
+    if (e__ != cudaSuccess)                                                                 \
+      return fail(set_error(AIQ_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)));       \
+  } while (0)
+
+  CREATE_TRY(cudaMemsetAsync(flag, 0, 256, stream));
+  for (size_t i = 0; i < m->layers.size(); ++i) {
+    LayerInfo& li = m->layers[i];
+    const size_t n = li.d.cout, k = li.K;
+    li.Wf = reinterpret_cast<float*>(base + lay.wf[i]);
+    li.bias = reinterpret_cast<float*>(base + lay.bias[i]);
+    for (int b = 0; b < 4; ++b) {
+      li.packed[b] = base + lay.packed[b][i];
+      li.scales[b] = reinterpret_cast<float*>(base + lay.scales[b][i]);
+    }
+    const aiq_layer_weights_t& w = weights[i];
+    if (li.d.has_bn) {
+      float* sW = reinterpret_cast<float*>(base + lay.staging_off);
+      const size_t vec = align_up(n * 4, 256);
+      uint8_t* sv = base + lay.staging_off + align_up(n * k * 4, 256);
+      float* sG = reinterpret_cast<float*>(sv);
+      float* sB = reinterpret_cast<float*>(sv + vec);
+      float* sM = reinterpret_cast<float*>(sv + 2 * vec);
+      float* sV = reinterpret_cast<float*>(sv + 3 * vec);
+      CREATE_TRY(cudaMemcpyAsync(sW, w.W, n * k * 4, cudaMemcpyHostToDevice, stream));
+      CREATE_TRY(cudaMemcpyAsync(sG, w.gamma, n * 4, cudaMemcpyHostToDevice, stream));
+      CREATE_TRY(cudaMemcpyAsync(sB, w.beta, n * 4, cudaMemcpyHostToDevice, stream));
+      CREATE_TRY(cudaMemcpyAsync(sM, w.mean, n * 4, cudaMemcpyHostToDevice, stream));
+      CREATE_TRY(cudaMemcpyAsync(sV, w.var, n * 4, cudaMemcpyHostToDevice, stream));
+      st = launch_fold_bn(sW, sG, sB, sM, sV, (int)n, (int)k, 1e-5f, li.Wf, li.bias, stream);
+      if (st != AIQ_OK) return fail(st);
+    } else {
+      CREATE_TRY(cudaMemcpyAsync(li.Wf, w.W, n * k * 4, cudaMemcpyHostToDevice, stream));
+      if (w.bias) CREATE_TRY(cudaMemcpyAsync(li.bias, w.bias, n * 4, cudaMemcpyHostToDevice, stream));
+      else CREATE_TRY(cudaMemsetAsync(li.bias, 0, n * 4, stream));
+    }
+    for (int b = 0; b < 4; ++b) {
+      st = launch_quantize(li.Wf, (int)n, (int)k, kBitsList[b], li.packed[b], li.scales[b], flag, stream);
+      if (st != AIQ_OK) return fail(st);
+    }
+  }
+  int32_t host_flag = 0;
+  CREATE_TRY(cudaMemcpyAsync(&host_flag, flag, 4, cudaMemcpyDeviceToHost, stream));
+  CREATE_TRY(cudaStreamSynchronize(stream));
+#undef CREATE_TRY
+  if (host_flag) return fail(set_error(AIQ_ERR_NONFINITE, "a weight is NaN or infinite"));
+  *out = m;
+  return AIQ_OK;
+}
+
+extern "C" void aiq_model_destroy(aiq_model_t* model) { delete model; }
+extern "C" int aiq_model_num_layers(const aiq_model_t* model) { return model ? (int)model->layers.size() : -1; }
+extern "C" int aiq_model_num_classes(const aiq_model_t* model) { return model ? model->layers.back().d.cout : -1; }
+
+extern "C" aiq_status_t aiq_model_layer_folded(const aiq_model_t* model, int layer, const float** Wf,
+                                               const float** bias, int* N, int* K) {
+  if (!model || layer < 0 || layer >= (int)model->layers.size())
+    return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_model_layer_folded: layer %d", layer);
+  const LayerInfo& li = model->layers[layer];
+  if (Wf) *Wf = li.Wf;
+  if (bias) *bias = li.bias;
+  if (N) *N = li.d.cout;
+  if (K) *K = li.K;
+  return AIQ_OK;
+}
+
+extern "C" aiq_status_t aiq_model_layer_packed(const aiq_model_t* model, int layer, int bits,
+                                               const void** packed, const float** scales) {
+  if (!model || layer < 0 || layer >= (int)model->layers.size())
+    return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_model_layer_packed: layer %d", layer);
+  const int bi = aiq::bits_index(bits);
+  if (bi < 0) return aiq::set_error(AIQ_ERR_UNSUPPORTED_BITS, "aiq_model_layer_packed: bits=%d", bits);
+  if (packed) *packed = model->layers[layer].packed[bi];
+  if (scales) *scales = model->layers[layer].scales[bi];
+  return AIQ_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// evaluation plan
+// ---------------------------------------------------------------------------------------
+namespace aiq {
+
+// Workspace layout for a chunk of B images and up to S schemes:
+//   [ job records | counts | pooled S*B*C | logits S*B*classes | slot 0 | slot 1 | ... ]
+struct WsLayout {
+  size_t jobs_off, jobs_bytes, counts_off, pooled_off, logits_off, total;
+  std::vector<size_t> slot_off;
+};
+
+static size_t jobs_capacity(const aiq_model* m, int S) {
+  // every layer: up to S jobs; the head adds pool + argmax records
+  return ((size_t)m->layers.size() + 2) * (size_t)S;
+}
+
+static WsLayout ws_layout(const aiq_model* m, int B, int S) {
+  WsLayout w;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  w.jobs_bytes = jobs_capacity(m, S) * sizeof(LayerJob);
+  w.jobs_off = take(w.jobs_bytes);
+  w.counts_off = take((size_t)S * 4);
+  const LayerInfo& fc = m->layers.back();
+  w.pooled_off = take((size_t)S * B * fc.d.cin * 4);
+  w.logits_off = take((size_t)S * B * fc.d.cout * 4);
+  for (size_t e : m->slot_elems) w.slot_off.push_back(take((size_t)S * B * e * 4));
+  w.total = off;
+  return w;
+}
+
+struct LayerPlan {
+  int n_versions = 0;
+  size_t job_first = 0;                 // index of the first job record of this layer
+  // fc only
+  int n_pool = 0;
+  size_t pool_first = 0, argmax_first = 0;
+  std::vector<std::pair<int, int>> bit_groups;   // (first job, count) per bit-width for qlinear
+  std::vector<int> group_bits;
+};
+
+struct EvalPlan {
+  std::vector<LayerPlan> lp;            // per layer
+  std::vector<LayerJob> jobs;           // host image of all job records
+  std::vector<int> final_version;       // per scheme: version of the classifier output
+  int n_final = 0;
+  int64_t versions_total = 0;
+};
+
+// Builds the job records for `S` schemes over a chunk of B images.  With sharing on, a
+// (layer, version) is keyed by (bit-width, version of its input, version of its residual):
+// candidates that agree on a prefix of the network reuse its activations.
+static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S, int B, bool share,
+                               uint8_t* ws, const WsLayout& wl, float* user_logits, EvalPlan& plan) {
+  const int n = (int)m->layers.size();
+  for (int s = 0; s < S; ++s)
+    for (int l = 0; l < n; ++l)
+      if (!bits_ok(schemes[(size_t)s * n + l]))
+        return set_error(AIQ_ERR_UNSUPPORTED_BITS, "scheme %d, layer %d: bits=%d", s, l, (int)schemes[(size_t)s * n + l]);
+  plan.lp.assign(n, LayerPlan());
+  plan.jobs.clear();
+  std::vector<std::vector<int>> ver(n, std::vector<int>(S, 0));   // ver[l][s]
+  auto slot_ptr = [&](int layer, int version) -> float* {
+    const LayerInfo& li = m->layers[layer];
+    return reinterpret_cast<float*>(ws + wl.slot_off[li.slot]) + (size_t)version * B * li.out_elems;
+  };
+  for (int l : m->order) {
+    const LayerInfo& li = m->layers[l];
+    LayerPlan& lp = plan.lp[l];
+    std::map<std::tuple<int, int, int>, int> seen;
+    std::vector<std::tuple<int, int, int>> keys;   // per version
+    for (int s = 0; s < S; ++s) {
+      const int bits = schemes[(size_t)s * n + l];
+      const int vin = li.d.input >= 0 ? ver[li.d.input][s] : 0;
+      const int vres = li.d.residual >= 0 ? ver[li.d.residual][s] : 0;
+      if (share) {
+        auto key = std::make_tuple(bits, vin, vres);
+        auto it = seen.find(key);
+        if (it == seen.end()) {
+          it = seen.emplace(key, (int)keys.size()).first;
+          keys.push_back(key);
+        }
+        ver[l][s] = it->second;
+      } else {
+        ver[l][s] = s;
+        keys.push_back(std::make_tuple(bits, vin, vres));
+      }
+    }
+    lp.n_versions = (int)keys.size();
+    plan.versions_total += lp.n_versions;
+    if (li.d.kind != AIQ_LAYER_FC) {
+      lp.job_first = plan.jobs.size();
+      for (int v = 0; v < lp.n_versions; ++v) {
+        LayerJob j = {};
+        const int bits = std::get<0>(keys[v]);
+        const int bi = bits_index(bits);
+        j.in = li.d.input >= 0 ? slot_ptr(li.d.input, std::get<1>(keys[v])) : nullptr;
+        j.res = li.d.residual >= 0 ? slot_ptr(li.d.residual, std::get<2>(keys[v])) : nullptr;
+        j.out = slot_ptr(l, v);
+        j.w = li.packed[bi];
+        j.scale = li.scales[bi];
+        j.bias = li.bias;
+        j.bits = bits;
+        plan.jobs.push_back(j);
+      }
+      continue;
+    }
+    // classifier: pool every distinct input version once, then one linear job per version
+    // (grouped by bit-width), then arg-max per version
+    const LayerInfo& src = m->layers[li.d.input];
+    int n_in_versions = 0;
+    for (int s = 0; s < S; ++s) n_in_versions = std::max(n_in_versions, ver[li.d.input][s] + 1);
+    lp.n_pool = n_in_versions;
+    lp.pool_first = plan.jobs.size();
+    float* pooled = reinterpret_cast<float*>(ws + wl.pooled_off);
+    for (int v = 0; v < n_in_versions; ++v) {
+      LayerJob j = {};
+      j.in = slot_ptr(li.d.input, v);
+      j.out = pooled + (size_t)v * B * src.d.cout;
+      plan.jobs.push_back(j);
+    }
+    // order the linear jobs by bit-width so each launch is homogeneous
+    std::vector<int> vorder;
+    for (int b = 0; b < 4; ++b)
+      for (int v = 0; v < lp.n_versions; ++v)
+        if (std::get<0>(keys[v]) == kBitsList[b]) vorder.push_back(v);
+    float* logits = user_logits ? user_logits : reinterpret_cast<float*>(ws + wl.logits_off);
+    lp.job_first = plan.jobs.size();
+    for (size_t idx = 0; idx < vorder.size(); ++idx) {
+      const int v = vorder[idx];
+      const int bits = std::get<0>(keys[v]);
+      const int bi = bits_index(bits);
+      LayerJob j = {};
+      j.in = pooled + (size_t)std::get<1>(keys[v]) * B * src.d.cout;
+      j.out = logits + (size_t)v * B * li.d.cout;
+      j.w = li.packed[bi];
+      j.scale = li.scales[bi];
+      j.bias = li.bias;
+      j.bits = bits;
+      if (lp.group_bits.empty() || lp.group_bits.back() != bits) {
+        lp.group_bits.push_back(bits);
+        lp.bit_groups.push_back({(int)idx, 1});
+      } else {
+        lp.bit_groups.back().second++;
+      }
+      plan.jobs.push_back(j);
+    }
+    lp.argmax_first = plan.jobs.size();
+    for (int v = 0; v < lp.n_versions; ++v) {
+      LayerJob j = {};
+      j.in = logits + (size_t)v * B * li.d.cout;
+      j.label_slot = v;
+      plan.jobs.push_back(j);
+    }
+    plan.final_version.assign(S, 0);
+    for (int s = 0; s < S; ++s) plan.final_version[s] = ver[l][s];
+    plan.n_final = lp.n_versions;
+  }
+  if (plan.jobs.size() > jobs_capacity(m, S))
+    return set_error(AIQ_ERR_WORKSPACE_TOO_SMALL, "internal: job table overflow");
+  return AIQ_OK;
+}
+
+// Launches one pass over a chunk of `B` images (B <= the plan's chunk size).
+static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const LayerJob* jobs_dev, int B,
+                              const float* x_chunk, const int32_t* labels, int32_t* counts, int32_t* preds,
+                              long long preds_stride, long long img0, bool want_argmax, cudaStream_t stream) {
+  for (int l : m->order) {
+    const LayerInfo& li = m->layers[l];
+    const LayerPlan& lp = plan.lp[l];
+    aiq_status_t st;
+    if (li.d.kind == AIQ_LAYER_FC) {
+      const LayerInfo& src = m->layers[li.d.input];
+      st = launch_avgpool(jobs_dev + lp.pool_first, lp.n_pool, B, src.Ho * src.Wo, src.d.cout, stream);
+      if (st != AIQ_OK) return st;
+      for (size_t gi = 0; gi < lp.bit_groups.size(); ++gi) {
+        const size_t first = lp.job_first + lp.bit_groups[gi].first;
+        st = launch_qlinear(jobs_dev + first, &plan.jobs[first], lp.bit_groups[gi].second, li.d.cout, li.K, B, stream);
+        if (st != AIQ_OK) return st;
+      }
+      if (want_argmax) {
+        st = launch_argmax_count(jobs_dev + lp.argmax_first, lp.n_versions, B, li.d.cout, labels, counts, preds,
+                                 preds_stride, img0, stream);
+        if (st != AIQ_OK) return st;
+      }
+      continue;
+    }
+    ConvGeom g = {};
+    g.B = B; g.H = li.Hi; g.W = li.Wi; g.Cin = li.d.cin; g.Ho = li.Ho; g.Wo = li.Wo; g.Cout = li.d.cout;
+    g.ks = li.d.ksize; g.stride = li.d.stride; g.pad = li.d.pad; g.act = li.d.act; g.K = li.K;
+    if (li.d.input < 0) {          // network input: NCHW
+      g.in_sb = (long long)li.d.cin * li.Hi * li.Wi; g.in_sc = (long long)li.Hi * li.Wi; g.in_sy = li.Wi; g.in_sx = 1;
+    } else {                       // internal activations: NHWC
+      g.in_sb = (long long)li.Hi * li.Wi * li.d.cin; g.in_sy = (long long)li.Wi * li.d.cin; g.in_sx = li.d.cin; g.in_sc = 1;
+    }
+    if (li.d.kind == AIQ_LAYER_DEPTHWISE) st = launch_depthwise(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, stream);
+    else st = launch_conv(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, stream);
+    if (st != AIQ_OK) return st;
+  }
+  return AIQ_OK;
+}
+
+}  // namespace aiq
+
+extern "C" size_t aiq_workspace_bytes(const aiq_model_t* model, int max_batch, int max_schemes) {
+  if (!model || max_batch <= 0 || max_schemes <= 0) return 0;
+  return aiq::ws_layout(model, max_batch, max_schemes).total;
+}
+
+extern "C" void aiq_set_eval_options(int chunk, int share_prefix) {
+  aiq::g_opt_chunk = chunk > 0 ? chunk : 0;
+  aiq::g_opt_share = share_prefix ? 1 : 0;
+}
+
+extern "C" void aiq_last_call_stats(int64_t* kernel_launches, int64_t* layer_evals, int64_t* layer_evals_unshared) {
+  if (kernel_launches) *kernel_launches = aiq::t_launches;
+  if (layer_evals) *layer_evals = aiq::t_layer_evals;
+  if (layer_evals_unshared) *layer_evals_unshared = aiq::t_layer_evals_unshared;
+}
+
+extern "C" aiq_status_t aiq_forward(const aiq_model_t* model, const uint8_t* scheme_bits, const float* x,
+                                    int batch, float* logits, void* workspace, size_t workspace_bytes,
+                                    void* stream_) {
+  using namespace aiq;
+  if (!model || !scheme_bits || !x || !logits || !workspace) return set_error(AIQ_ERR_INVALID_ARG, "aiq_forward: null pointer");
+  if (batch <= 0) return set_error(AIQ_ERR_INVALID_ARG, "aiq_forward: batch=%d", batch);
+  if (((uintptr_t)workspace) & 255) return set_error(AIQ_ERR_INVALID_ARG, "aiq_forward: workspace not 256-byte aligned");
+  if ((((uintptr_t)x) & 15) || (((uintptr_t)logits) & 3)) return set_error(AIQ_ERR_INVALID_ARG, "aiq_forward: x must be 16-byte aligned");
+  const WsLayout wl = ws_layout(model, batch, 1);
+  if (workspace_bytes < wl.total)
+    return set_error(AIQ_ERR_WORKSPACE_TOO_SMALL, "aiq_forward: need %zu workspace bytes, got %zu", wl.total, workspace_bytes);
+  aiq_status_t st = check_device_sm100();
+  if (st != AIQ_OK) return st;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  t_launches = 0;
+  EvalPlan plan;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  st = build_plan(model, scheme_bits, 1, batch, true, ws, wl, logits, plan);
+  if (st != AIQ_OK) return st;
+  AIQ_CUDA_TRY(cudaMemcpyAsync(ws + wl.jobs_off, plan.jobs.data(), plan.jobs.size() * sizeof(LayerJob),
+                               cudaMemcpyHostToDevice, stream));
+  st = run_chunk(model, plan, reinterpret_cast<const LayerJob*>(ws + wl.jobs_off), batch, x, nullptr, nullptr,
+                 nullptr, 0, 0, false, stream);
+  t_layer_evals = plan.versions_total;
+  t_layer_evals_unshared = (int64_t)model->layers.size();
+  return st;
+}
+
+extern "C" aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t* schemes, int n_schemes,
+                                         const float* x, const int32_t* labels, int n_images, float* acc,
+                                         int32_t* correct_counts, int32_t* preds, void* workspace,
+                                         size_t workspace_bytes, void* stream_) {
+  using namespace aiq;
+  if (!model || !schemes || !x || !labels || !acc || !workspace)
+    return set_error(AIQ_ERR_INVALID_ARG, "aiq_eval_schemes: null pointer");
+  if (n_schemes <= 0 || n_images <= 0)
+    return set_error(AIQ_ERR_INVALID_ARG, "aiq_eval_schemes: n_schemes=%d n_images=%d", n_schemes, n_images);
+  if (((uintptr_t)workspace) & 255) return set_error(AIQ_ERR_INVALID_ARG, "aiq_eval_schemes: workspace not 256-byte aligned");
+  if (((uintptr_t)x) & 15) return set_error(AIQ_ERR_INVALID_ARG, "aiq_eval_schemes: x must be 16-byte aligned");
+  aiq_status_t st = check_device_sm100();
+  if (st != AIQ_OK) return st;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  t_launches = 0;
+
+  // chunk: the requested (or default) size, shrunk until the layout fits the workspace
+  int B = g_opt_chunk > 0 ? g_opt_chunk : 256;
+  if (B > n_images) B = n_images;
+  while (B > 1 && ws_layout(model, B, n_schemes).total > workspace_bytes) B = (B + 1) / 2;
+  const WsLayout wl = ws_layout(model, B, n_schemes);
+  if (wl.total > workspace_bytes)
+    return set_error(AIQ_ERR_WORKSPACE_TOO_SMALL, "aiq_eval_schemes: need %zu workspace bytes for one image, got %zu",
+                     wl.total, workspace_bytes);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  EvalPlan plan;
+  st = build_plan(model, schemes, n_schemes, B, g_opt_share != 0, ws, wl, nullptr, plan);
+  if (st != AIQ_OK) return st;
+  // Counts and predictions are indexed by a row in [0, n_schemes): the row of a final
+  // version is the first scheme that maps to it; duplicate schemes are filled in afterwards.
+  std::vector<int> first_scheme(plan.n_final, -1);
+  for (int s = 0; s < n_schemes; ++s)
+    if (first_scheme[plan.final_version[s]] < 0) first_scheme[plan.final_version[s]] = s;
+  const LayerPlan& fcp = plan.lp.back();
+  for (int v = 0; v < plan.n_final; ++v) plan.jobs[fcp.argmax_first + v].label_slot = first_scheme[v];
+
+  int32_t* counts_dev = reinterpret_cast<int32_t*>(ws + wl.counts_off);
+  AIQ_CUDA_TRY(cudaMemcpyAsync(ws + wl.jobs_off, plan.jobs.data(), plan.jobs.size() * sizeof(LayerJob),
+                               cudaMemcpyHostToDevice, stream));
+  AIQ_CUDA_TRY(cudaMemsetAsync(counts_dev, 0, (size_t)n_schemes * 4, stream));
+
+  const size_t img_elems = (size_t)model->in_c * model->in_h * model->in_w;
+  const LayerJob* jobs_dev = reinterpret_cast<const LayerJob*>(ws + wl.jobs_off);
+  int64_t chunks = 0;
+  for (long long img0 = 0; img0 < n_images; img0 += B, ++chunks) {
+    const int b = (int)std::min<long long>(B, n_images - img0);
+    st = run_chunk(model, plan, jobs_dev, b, x + img0 * img_elems, labels, counts_dev, preds, n_images, img0, true, stream);
+    if (st != AIQ_OK) return st;
+  }
+  std::vector<int32_t> counts(n_schemes, 0);
+  AIQ_CUDA_TRY(cudaMemcpyAsync(counts.data(), counts_dev, (size_t)n_schemes * 4, cudaMemcpyDeviceToHost, stream));
+  if (preds)
+    for (int s = 0; s < n_schemes; ++s) {
+      const int src = first_scheme[plan.final_version[s]];
+      if (src != s)
+        AIQ_CUDA_TRY(cudaMemcpyAsync(preds + (size_t)s * n_images, preds + (size_t)src * n_images,
+                                     (size_t)n_images * 4, cudaMemcpyDeviceToDevice, stream));
+    }
+  AIQ_CUDA_TRY(cudaStreamSynchronize(stream));
+  for (int s = 0; s < n_schemes; ++s) {
+    const int c = counts[first_scheme[plan.final_version[s]]];
+    acc[s] = (float)((double)c / (double)n_images);
+    if (correct_counts) correct_counts[s] = c;
+  }
+  t_layer_evals = plan.versions_total * chunks;
+  t_layer_evals_unshared = (int64_t)n_schemes * (int64_t)model->layers.size() * chunks;
+  return AIQ_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// analytic arithmetic intensity (host only)
+// ---------------------------------------------------------------------------------------
+extern "C" aiq_status_t aiq_scheme_ai(const aiq_model_t* model, const uint8_t* scheme_bits, int ai_batch,
+                                      double* ai, double* flops, double* bytes) {
+  using namespace aiq;
+  if (!model || !scheme_bits) return set_error(AIQ_ERR_INVALID_ARG, "aiq_scheme_ai: null pointer");
+  if (ai_batch <= 0) return set_error(AIQ_ERR_INVALID_ARG, "aiq_scheme_ai: ai_batch=%d", ai_batch);
+  double fl = 0.0, by = 0.0;
+  for (size_t l = 0; l < model->layers.size(); ++l) {
+    const LayerInfo& li = model->layers[l];
+    const int bits = scheme_bits[l];
+    if (!bits_ok(bits)) return set_error(AIQ_ERR_UNSUPPORTED_BITS, "aiq_scheme_ai: layer %zu bits=%d", l, bits);
+    const double weights = (double)li.d.cout * li.K;
+    fl += 2.0 * weights * li.Ho * li.Wo * ai_batch;
+    by += weights * bits / 8.0;
+    by += 4.0 * ai_batch * ((double)li.d.cin * li.Hi * li.Wi + (double)li.d.cout * li.Ho * li.Wo);
+  }
+  if (ai) *ai = fl / by;
+  if (flops) *flops = fl;
+  if (bytes) *bytes = by;
+  return AIQ_OK;
+}
+
+extern "C" const char* aiq_status_string(aiq_status_t status) {
+  switch (status) {
+    case AIQ_OK: return "ok";
+    case AIQ_ERR_INVALID_ARG: return "invalid argument";
+    case AIQ_ERR_UNSUPPORTED_BITS: return "unsupported bit-width";
+    case AIQ_ERR_SHAPE: return "shape mismatch";
+    case AIQ_ERR_WORKSPACE_TOO_SMALL: return "buffer too small";
+    case AIQ_ERR_CUDA: return "CUDA error";
+    case AIQ_ERR_NOT_SM100: return "device is not sm_100";
+    case AIQ_ERR_NONFINITE: return "non-finite weight";
+    case AIQ_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+extern "C" const char* aiq_last_error(void) { return aiq::t_err; }

@@ -1,0 +1,191 @@
+"""CUDA forward pass and scheme evaluator against the oracle (through the C ABI)."""
+import numpy as np
+import pytest
+
+from aiq_workloads import (resnet20, mobilenet_v2, tiny_net, gen_model, gen_images,
+                           gen_random_scheme, one_layer_lowered_schemes, coordinate_step_schemes,
+                           mixed_int4_int8_scheme, conv_layer_indices)
+from oracle import aiq_oracle as O
+from gpu_util import binding, to_dev, assert_logits_close, assert_preds_match
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_bank(arch, params, bits_set=(4, 8, 16, 32)):
+    folded = O.fold_model(arch, params)
+    return folded, O.build_weight_bank(folded, bits_set)
+
+
+def balance_classifier(arch, params, x):
+    """Random-init networks put almost every image in one class (a constant offset
+    dominates the logits).  Shift the classifier bias by the oracle's mean FP32 logits so
+    that predictions spread over the classes and margins become small: a much sharper test
+    of arg-max and counting.  The shift is computed by the oracle only."""
+    folded = O.fold_model(arch, params)
+    mean_logits = O.forward_fp32_unquantized(arch, folded, x).astype(np.float64).mean(axis=0)
+    params = [dict(p) for p in params]
+    params[-1]["bias"] = (params[-1]["bias"].astype(np.float64) - mean_logits).astype(np.float32)
+    return params
+
+
+@pytest.mark.parametrize("batch", [1, 3, 37])
+def test_tiny_net_random_schemes(batch):
+    aiq = binding()
+    arch = tiny_net()
+    params = gen_model(arch, 99)
+    model = aiq.Model(arch, params)
+    folded, bank = _oracle_bank(arch, params)
+    x = gen_images(batch, 3, 8, 8, 17 + batch)
+    for seed in range(6):
+        scheme = gen_random_scheme(model.n_layers, seed)
+        got = model.aiq_forward(scheme, to_dev(x)).cpu().numpy()
+        ref = O.forward_scheme(arch, bank, scheme, x)
+        assert_logits_close(got, ref, f"tiny batch={batch} seed={seed}")
+
+
+def test_resnet20_batch64_mixed_scheme():
+    """ResNet-20, batch 64, one bit-width per layer drawn from {32, 16, 8, 4}."""
+    aiq = binding()
+    arch = resnet20()
+    params = gen_model(arch, 1234)
+    model = aiq.Model(arch, params)
+    folded, bank = _oracle_bank(arch, params)
+    x = gen_images(64, 3, 32, 32, 5678)
+    scheme = gen_random_scheme(22, 42)
+    got = model.aiq_forward(scheme, to_dev(x)).cpu().numpy()
+    ref = O.forward_scheme(arch, bank, scheme, x)
+    assert_logits_close(got, ref, "resnet20 mixed")
+    assert_preds_match(O.predict(got), O.predict(ref), O.top2_margin(ref), "resnet20 mixed")
+    for bits in (32, 16, 8, 4):
+        got = model.aiq_forward([bits] * 22, to_dev(x[:9])).cpu().numpy()
+        assert_logits_close(got, O.forward_scheme(arch, bank, [bits] * 22, x[:9]), f"uniform {bits}")
+    # analytic AI equals the oracle's for this scheme and for the uniform ones
+    for s in (scheme, [32] * 22, [8] * 22, [4] * 22):
+        g, o = model.aiq_scheme_ai(s), O.scheme_ai(arch, s)
+        assert g[1] == o[1] and g[2] == o[2] and abs(g[0] - o[0]) <= 1e-12 * o[0]
+    g3, o3 = model.aiq_scheme_ai(scheme, 3), O.scheme_ai(arch, scheme, 3)
+    assert g3[1] == o3[1] and g3[2] == o3[2]
+
+
+@pytest.mark.parametrize("batch", [1, 24])
+def test_mobilenet_v2_cifar(batch):
+    aiq = binding()
+    arch = mobilenet_v2("cifar")
+    params = gen_model(arch, 2234)
+    model = aiq.Model(arch, params)
+    folded, bank = _oracle_bank(arch, params, (4, 8))
+    scheme = mixed_int4_int8_scheme(53, conv_layer_indices(arch), 10, 43)
+    assert (scheme == 4).sum() == 10 and scheme[-1] == 8
+    x = gen_images(batch, 3, 32, 32, 600 + batch)
+    got = model.aiq_forward(scheme, to_dev(x)).cpu().numpy()
+    ref = O.forward_scheme(arch, bank, scheme, x)
+    assert_logits_close(got, ref, f"mbv2 cifar batch={batch}")
+
+
+def test_mobilenet_v2_imagenet_shape():
+    aiq = binding()
+    arch = mobilenet_v2("imagenet")
+    params = gen_model(arch, 4234)
+    model = aiq.Model(arch, params)
+    folded, bank = _oracle_bank(arch, params, (4, 8, 16, 32))
+    x = gen_images(3, 3, 224, 224, 4235)
+    schemes = coordinate_step_schemes(53, conv_layer_indices(arch))
+    for j in (0, 1, 2, 30):
+        got = model.aiq_forward(schemes[j], to_dev(x)).cpu().numpy()
+        ref = O.forward_scheme(arch, bank, schemes[j], x)
+        assert got.shape == (3, 1000)
+        assert_logits_close(got, ref, f"mbv2 imagenet scheme {j}")
+
+
+def test_eval_schemes_greedy_step_resnet20():
+    """One greedy step: 21 candidates, each lowering one conv layer of an all-8 scheme to 4
+    bits.  Counts, predictions and accuracies against the oracle; sharing on/off and the
+    chunk size must not change a single count."""
+    import torch
+    aiq = binding()
+    arch = resnet20()
+    x = gen_images(176, 3, 32, 32, 5679)
+    params = balance_classifier(arch, gen_model(arch, 1234), x)
+    model = aiq.Model(arch, params)
+    folded, bank = _oracle_bank(arch, params, (4, 8))
+    labels = O.predict(O.forward_fp32_unquantized(arch, folded, x))
+    assert len(np.unique(labels)) >= 5                       # the balanced classifier spreads labels
+    schemes = one_layer_lowered_schemes(22, conv_layer_indices(arch))
+    assert schemes.shape == (21, 22)
+    oacc, ocounts, opreds, omargins = O.eval_schemes(arch, bank, schemes, x, labels)
+    assert len(set(ocounts.tolist())) > 1                    # the candidates really differ
+    xd, ld = to_dev(x), to_dev(labels)
+    results = []
+    for chunk, share in ((64, True), (64, False), (50, True), (176, True), (7, True)):
+        aiq.aiq_set_eval_options(chunk, share)
+        preds = torch.full((21, 176), -1, dtype=torch.int32, device="cuda")
+        acc, counts = model.aiq_eval_schemes(schemes, xd, ld, preds=preds, chunk=chunk)
+        stats = aiq.aiq_last_call_stats()
+        results.append((counts.copy(), preds.cpu().numpy(), stats))
+        assert np.allclose(acc, counts / 176.0)
+    aiq.aiq_set_eval_options(0, True)
+    counts0, preds0, stats0 = results[0]
+    for counts, preds, _ in results[1:]:
+        assert np.array_equal(counts, counts0)
+        assert np.array_equal(preds, preds0)
+    assert_preds_match(preds0, opreds, omargins, "greedy step")
+    slack = (omargins <= 1e-2).sum(axis=1)
+    assert np.all(np.abs(counts0 - ocounts) <= slack)
+    assert np.array_equal((preds0 == labels[None, :]).sum(axis=1), counts0)
+    # prefix sharing does strictly less work than 21 independent passes
+    assert stats0["layer_evals"] < results[1][2]["layer_evals"] == stats0["layer_evals_unshared"]
+    assert stats0["kernel_launches"] > 0
+
+
+def test_eval_schemes_duplicates_fc_candidates_and_tiny_net():
+    import torch
+    aiq = binding()
+    arch = tiny_net()
+    x = gen_images(45, 3, 8, 8, 71)
+    params = balance_classifier(arch, gen_model(arch, 99), x)
+    model = aiq.Model(arch, params)
+    folded, bank = _oracle_bank(arch, params)
+    labels = O.predict(O.forward_fp32_unquantized(arch, folded, x))
+    L = model.n_layers
+    schemes = np.concatenate([
+        one_layer_lowered_schemes(L, list(range(L))),                 # includes the classifier
+        coordinate_step_schemes(L, list(range(L))),
+        np.stack([gen_random_scheme(L, s) for s in range(5)]),
+        np.full((2, L), 32, np.uint8),                                # duplicates
+        one_layer_lowered_schemes(L, [3]),                            # duplicate of row 3
+    ])
+    oacc, ocounts, opreds, omargins = O.eval_schemes(arch, bank, schemes, x, labels)
+    preds = torch.full((len(schemes), 45), -1, dtype=torch.int32, device="cuda")
+    aiq.aiq_set_eval_options(16, True)
+    acc, counts = model.aiq_eval_schemes(schemes, to_dev(x), to_dev(labels), preds=preds, chunk=16)
+    aiq.aiq_set_eval_options(0, True)
+    p = preds.cpu().numpy()
+    assert_preds_match(p, opreds, omargins, "tiny eval")
+    assert np.all(np.abs(counts - ocounts) <= (omargins <= 1e-2).sum(axis=1))
+    assert np.array_equal(p[-1], p[3]) and np.array_equal(p[-2], p[-3])
+    assert counts[-2] == counts[-3] == 45                             # all-32 scheme agrees with itself
+    assert acc[-2] == 1.0
+
+
+def test_forward_and_eval_errors():
+    import torch
+    aiq = binding()
+    arch = tiny_net()
+    model = aiq.Model(arch, gen_model(arch, 1))
+    x = to_dev(gen_images(4, 3, 8, 8, 2))
+    bad = np.full(model.n_layers, 8, np.uint8)
+    bad[2] = 7
+    with pytest.raises(aiq.AiqError) as e:
+        model.aiq_forward(bad, x)
+    assert e.value.status == aiq.ERR_UNSUPPORTED_BITS
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(aiq.AiqError) as e:
+        model.aiq_forward(np.full(model.n_layers, 8, np.uint8), x, workspace=small)
+    assert e.value.status == aiq.ERR_WORKSPACE_TOO_SMALL
+    labels = torch.zeros(4, dtype=torch.int32, device="cuda")
+    with pytest.raises(aiq.AiqError) as e:
+        model.aiq_eval_schemes(bad[None, :], x, labels)
+    assert e.value.status == aiq.ERR_UNSUPPORTED_BITS
+    with pytest.raises(aiq.AiqError) as e:
+        model.aiq_eval_schemes(np.full((1, model.n_layers), 8, np.uint8), x, labels, workspace=small)
+    assert e.value.status == aiq.ERR_WORKSPACE_TOO_SMALL

@@ -1,0 +1,51 @@
+"""CUDA small-batch quantized linear layer against the oracle."""
+import numpy as np
+import pytest
+
+from aiq_workloads import gen_linear_case
+from oracle import aiq_oracle as O
+from gpu_util import binding, to_dev, assert_logits_close
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(aiq, W, x, bits, bias=None):
+    import torch
+    N, K = W.shape
+    rb = aiq.aiq_packed_row_bytes(K, bits)
+    packed = torch.empty((N, rb), dtype=torch.uint8, device="cuda")
+    scales = torch.empty(N, dtype=torch.float32, device="cuda")
+    aiq.aiq_quantize_layer(to_dev(W), bits, packed, scales)
+    y = torch.full((x.shape[0], N), float("nan"), dtype=torch.float32, device="cuda")
+    aiq.aiq_qlinear(packed, scales, to_dev(bias) if bias is not None else None, N, K, bits, to_dev(x), y)
+    torch.cuda.synchronize()
+    v, s = O.quantize_rows(W, bits)
+    return y.cpu().numpy(), O.qlinear(v, s, bias, bits, x)
+
+
+@pytest.mark.parametrize("bits", [4, 8, 16, 32])
+@pytest.mark.parametrize("N,K,M", [(1280, 320, 1), (1280, 320, 4), (1280, 320, 16), (10, 64, 64),
+                                   (1000, 1280, 5), (37, 100, 3), (5, 27, 2), (4096, 4096, 1),
+                                   (2048, 4096, 4), (300, 2052, 7), (1, 1, 1)])
+def test_qlinear_matches_oracle(bits, N, K, M):
+    aiq = binding()
+    W, x = gen_linear_case(N, K, M, seed=3234 + N + K + M)
+    bias = np.random.default_rng(N).standard_normal(N).astype(np.float32) if N % 2 == 0 else None
+    got, ref = _run(aiq, W, x, bits, bias)
+    assert_logits_close(got, ref, f"N={N} K={K} M={M} bits={bits}")
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_qlinear_exact_on_integers(bits):
+    """Integer weights and activations: every product and partial sum is exact in float32,
+    so the result must equal the integer answer exactly (s = 1)."""
+    aiq = binding()
+    rng = np.random.default_rng(1)
+    qmax = 2 ** (bits - 1) - 1
+    W = rng.integers(-qmax, qmax + 1, (96, 200)).astype(np.float32)
+    W[:, 0] = qmax
+    x = rng.integers(-8, 9, (4, 200)).astype(np.float32)
+    got, ref = _run(aiq, W, x, bits)
+    want = x.astype(np.int64) @ W.astype(np.int64).T
+    assert np.array_equal(got.astype(np.int64), want)
+    assert np.array_equal(ref.astype(np.int64), want)
