@@ -230,6 +230,35 @@ void aiq_last_call_stats(int64_t* kernel_launches, int64_t* layer_evals, int64_t
 aiq_status_t aiq_scheme_ai(const aiq_model_t* model, const uint8_t* scheme_bits, int ai_batch,
                            double* ai, double* flops, double* bytes);
 
+/* ------------------------------------------------------------------------------------
+ * Per-kernel timing.  The paper measures throughput by wall clock (Section 3, experiment
+ * 3); this is the device-side equivalent for the kernels of this library.  Between
+ * aiq_profile_start and aiq_profile_stop every kernel launch made by the calling thread is
+ * bracketed by CUDA events on its stream.  aiq_profile_stop synchronises those events and
+ * fills out[kind] with the number of launches, their summed duration in milliseconds, and
+ * the algorithmic work they were asked to do: floating-point operations (2 per
+ * multiply-add) and bytes (packed weights + scales once, input and output tensors once).
+ * Event records cost about a microsecond each on the host; leave profiling off otherwise.
+ */
+enum {
+  AIQ_KERNEL_FOLD = 0,
+  AIQ_KERNEL_QUANTIZE = 1,
+  AIQ_KERNEL_QLINEAR = 2,
+  AIQ_KERNEL_CONV = 3,
+  AIQ_KERNEL_DEPTHWISE = 4,
+  AIQ_KERNEL_POOL = 5,
+  AIQ_KERNEL_ARGMAX = 6,
+  AIQ_KERNEL_KINDS = 7
+};
+typedef struct aiq_kernel_profile {
+  int64_t launches;
+  double ms;
+  double flops;
+  double bytes;
+} aiq_kernel_profile_t;
+aiq_status_t aiq_profile_start(void);
+aiq_status_t aiq_profile_stop(aiq_kernel_profile_t* out /* host [AIQ_KERNEL_KINDS] */);
+
 #ifdef __cplusplus
 }
 #endif

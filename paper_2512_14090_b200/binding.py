@@ -25,7 +25,10 @@ EXPORTS = [
     "aiq_model_destroy", "aiq_model_num_layers", "aiq_model_num_classes",
     "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
     "aiq_eval_schemes", "aiq_set_eval_options", "aiq_last_call_stats", "aiq_scheme_ai",
+    "aiq_profile_start", "aiq_profile_stop",
 ]
+
+KERNEL_KINDS = ["fold", "quantize", "qlinear", "conv", "depthwise", "pool", "argmax"]
 
 
 class AiqError(RuntimeError):
@@ -42,6 +45,11 @@ class LayerDesc(C.Structure):
 class ArchDesc(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("in_c", C.c_int32), ("in_h", C.c_int32),
                 ("in_w", C.c_int32), ("layers", C.POINTER(LayerDesc))]
+
+
+class KernelProfile(C.Structure):
+    _fields_ = [("launches", C.c_int64), ("ms", C.c_double), ("flops", C.c_double),
+                ("bytes", C.c_double)]
 
 
 class LayerWeights(C.Structure):
@@ -95,6 +103,10 @@ def _load():
     lib.aiq_scheme_ai.restype = i32
     lib.aiq_scheme_ai.argtypes = [vp, vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double),
                                   C.POINTER(C.c_double)]
+    lib.aiq_profile_start.restype = i32
+    lib.aiq_profile_start.argtypes = []
+    lib.aiq_profile_stop.restype = i32
+    lib.aiq_profile_stop.argtypes = [C.POINTER(KernelProfile)]
     return lib
 
 
@@ -178,11 +190,25 @@ def aiq_last_call_stats():
     return dict(kernel_launches=a.value, layer_evals=b.value, layer_evals_unshared=c.value)
 
 
+def aiq_profile_start():
+    _check(lib.aiq_profile_start())
+
+
+def aiq_profile_stop():
+    """{kind: dict(launches, ms, flops, bytes)} for the launches since aiq_profile_start."""
+    out = (KernelProfile * len(KERNEL_KINDS))()
+    _check(lib.aiq_profile_stop(out))
+    return {k: dict(launches=o.launches, ms=o.ms, flops=o.flops, bytes=o.bytes)
+            for k, o in zip(KERNEL_KINDS, out)}
+
+
 # ------------------------------------------------------------------------- model object
 class Model:
     """Owns the device memory the C model lives in (a torch uint8 tensor) and the handle."""
 
-    def __init__(self, arch, params, device="cuda:0", stream=None):
+    def __init__(self, arch, params, device="cuda:0", stream=None, mem=None):
+        """Uploads `params` (host float32 arrays), folds and builds the weight bank.
+        `mem`: an existing uint8 CUDA tensor to build into (reused across rebuilds)."""
         import torch
         self.arch = arch
         self.device = torch.device(device)
@@ -191,7 +217,10 @@ class Model:
         nbytes = int(lib.aiq_model_bytes(C.byref(desc)))
         if nbytes == 0:
             raise AiqError(ERR_INVALID_ARG, last_error())
-        self.mem = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        if mem is not None and mem.numel() >= nbytes:
+            self.mem = mem
+        else:
+            self.mem = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
         weights = (LayerWeights * len(params))()
         keep = []
         for w, p in zip(weights, params):
@@ -202,7 +231,7 @@ class Model:
                     setattr(w, name, a.ctypes.data)
         handle = C.c_void_p()
         with torch.cuda.device(self.device):
-            _check(lib.aiq_model_create(C.byref(desc), weights, _dev(self.mem), nbytes,
+            _check(lib.aiq_model_create(C.byref(desc), weights, _dev(self.mem), self.mem.numel(),
                                         _stream(stream), C.byref(handle)))
         self.handle = handle
         self.n_layers = int(lib.aiq_model_num_layers(handle))

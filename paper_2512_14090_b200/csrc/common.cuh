@@ -30,6 +30,15 @@ void count_launch();                         // per-thread launch counter (aiq_l
     ::aiq::count_launch();                                                              \
   } while (0)
 
+// Brackets one kernel launch with CUDA events while profiling is on (see aiq_profile_start),
+// and adds the launch's algorithmic work to the per-kind totals.
+struct LaunchScope {
+  LaunchScope(int kind, cudaStream_t stream, double flops, double bytes);
+  ~LaunchScope();
+  int slot_;
+  cudaStream_t stream_;
+};
+
 inline bool bits_ok(int bits) { return bits == 4 || bits == 8 || bits == 16 || bits == 32; }
 inline int padded_k(int K) { return (K + 31) / 32 * 32; }
 inline size_t row_bytes(int K, int bits) { return (size_t)padded_k(K) * bits / 8; }
@@ -90,10 +99,11 @@ aiq_status_t launch_quantize(const float* W, int N, int K, int bits, void* packe
 // y[m][n] for every job: in = x [M][K], out = y [M][N]
 aiq_status_t launch_qlinear(const LayerJob* jobs_dev, const LayerJob* single_host, int n_jobs, int N,
                             int K, int M, cudaStream_t s);
+// weight_bytes: packed weights + scales + biases of all jobs (for the profile's byte count)
 aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
-                         const float* net_input, cudaStream_t s);
+                         const float* net_input, double weight_bytes, cudaStream_t s);
 aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
-                              const float* net_input, cudaStream_t s);
+                              const float* net_input, double weight_bytes, cudaStream_t s);
 // pooled[b][c] = mean over HW of in[b][hw][c], per job (in -> out)
 aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int HW, int C, cudaStream_t s);
 // pred = lowest index of the max logit; preds[slot][img0 + b] = pred; counts[slot] += (pred == label)

@@ -227,9 +227,11 @@ conv_igemm_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* __
 
 template <int BM, int BN, int TM, int TN>
 aiq_status_t launch_conv_tile(const ConvGeom& g, const LayerJob* jobs, int n_jobs, const float* net_input,
-                              bool vec, cudaStream_t s) {
+                              bool vec, double weight_bytes, cudaStream_t s) {
   const int M = g.B * g.Ho * g.Wo;
   dim3 grid((M + BM - 1) / BM, (g.Cout + BN - 1) / BN, n_jobs);
+  LaunchScope scope(AIQ_KERNEL_CONV, s, 2.0 * M * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
+                    weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W + (double)M * g.Cout));
   if (vec)
     conv_igemm_kernel<BM, BN, TM, TN, true><<<grid, kConvThreads, 0, s>>>(g, jobs, net_input);
   else
@@ -365,7 +367,7 @@ __global__ void argmax_count_kernel(const LayerJob* __restrict__ jobs, int B, in
 }  // namespace
 
 aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs, const float* net_input,
-                         cudaStream_t s) {
+                         double weight_bytes, cudaStream_t s) {
   // vector path: channel-contiguous (NHWC) input with a channel count that keeps float4
   // groups inside one tap
   const bool vec = (g.in_sc == 1) && (g.Cin % 4 == 0) && (g.in_sx % 4 == 0) && (g.in_sy % 4 == 0) &&
@@ -374,15 +376,17 @@ aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs
   int bn = 64;
   if (waste(32) < waste(bn)) bn = 32;
   if (waste(16) < waste(bn)) bn = 16;
-  if (bn == 64) return launch_conv_tile<128, 64, 8, 4>(g, jobs_dev, n_jobs, net_input, vec, s);
-  if (bn == 32) return launch_conv_tile<128, 32, 4, 4>(g, jobs_dev, n_jobs, net_input, vec, s);
-  return launch_conv_tile<256, 16, 4, 4>(g, jobs_dev, n_jobs, net_input, vec, s);
+  if (bn == 64) return launch_conv_tile<128, 64, 8, 4>(g, jobs_dev, n_jobs, net_input, vec, weight_bytes, s);
+  if (bn == 32) return launch_conv_tile<128, 32, 4, 4>(g, jobs_dev, n_jobs, net_input, vec, weight_bytes, s);
+  return launch_conv_tile<256, 16, 4, 4>(g, jobs_dev, n_jobs, net_input, vec, weight_bytes, s);
 }
 
 aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
-                              const float* /*net_input*/, cudaStream_t s) {
+                              const float* /*net_input*/, double weight_bytes, cudaStream_t s) {
   const int M = g.B * g.Ho * g.Wo;
   dim3 grid((M + kDwPixPerBlock - 1) / kDwPixPerBlock, (g.Cout + 127) / 128, n_jobs);
+  LaunchScope scope(AIQ_KERNEL_DEPTHWISE, s, 18.0 * M * g.Cout * n_jobs,
+                    weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W + (double)M * g.Cout));
   depthwise3x3_kernel<<<grid, 256, 0, s>>>(g, jobs_dev);
   AIQ_LAUNCH_CHECK("depthwise3x3");
   return AIQ_OK;
@@ -390,6 +394,7 @@ aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n
 
 aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int HW, int C, cudaStream_t s) {
   int threads = C >= 256 ? 256 : (C >= 128 ? 128 : 64);
+  LaunchScope scope(AIQ_KERNEL_POOL, s, (double)n_jobs * B * HW * C, 4.0 * n_jobs * B * ((double)HW * C + C));
   avgpool_kernel<<<dim3(B, 1, n_jobs), threads, 0, s>>>(jobs_dev, HW, C);
   AIQ_LAUNCH_CHECK("avgpool");
   return AIQ_OK;
@@ -399,6 +404,7 @@ aiq_status_t launch_argmax_count(const LayerJob* jobs_dev, int n_jobs, int B, in
                                  const int32_t* labels, int32_t* counts, int32_t* preds,
                                  long long preds_stride, long long img0, cudaStream_t s) {
   const int warps = 8;
+  LaunchScope scope(AIQ_KERNEL_ARGMAX, s, 0.0, 4.0 * n_jobs * B * ((double)n_classes + 2));
   argmax_count_kernel<<<dim3((B + warps - 1) / warps, 1, n_jobs), warps * 32, 0, s>>>(
       jobs_dev, B, n_classes, labels, counts, preds, preds_stride, img0);
   AIQ_LAUNCH_CHECK("argmax_count");

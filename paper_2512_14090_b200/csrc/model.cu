@@ -32,6 +32,40 @@ aiq_status_t set_error(aiq_status_t status, const char* fmt, ...) {
 
 void count_launch() { ++t_launches; }
 
+// ---- per-kernel event timing ---------------------------------------------------------
+struct ProfiledLaunch { int kind; cudaEvent_t start, stop; };
+static thread_local bool t_profiling = false;
+static thread_local std::vector<ProfiledLaunch>* t_prof = nullptr;     // launches of this session
+static thread_local std::vector<cudaEvent_t>* t_event_pool = nullptr;  // reusable events
+static thread_local aiq_kernel_profile_t t_work[AIQ_KERNEL_KINDS];
+
+static cudaEvent_t take_event() {
+  if (t_event_pool && !t_event_pool->empty()) {
+    cudaEvent_t e = t_event_pool->back();
+    t_event_pool->pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+  return e;
+}
+
+LaunchScope::LaunchScope(int kind, cudaStream_t stream, double flops, double bytes) : slot_(-1), stream_(stream) {
+  if (!t_profiling || kind < 0 || kind >= AIQ_KERNEL_KINDS) return;
+  ProfiledLaunch pl = {kind, take_event(), take_event()};
+  if (!pl.start || !pl.stop) return;
+  t_work[kind].launches += 1;
+  t_work[kind].flops += flops;
+  t_work[kind].bytes += bytes;
+  cudaEventRecord(pl.start, stream);
+  t_prof->push_back(pl);
+  slot_ = (int)t_prof->size() - 1;
+}
+
+LaunchScope::~LaunchScope() {
+  if (slot_ >= 0) cudaEventRecord((*t_prof)[slot_].stop, stream_);
+}
+
 aiq_status_t check_device_sm100() {
   static int cached[64];   // 0 unknown, 1 ok, 2 not sm_100
   int dev = 0;
@@ -364,6 +398,7 @@ static WsLayout ws_layout(const aiq_model* m, int B, int S) {
 
 struct LayerPlan {
   int n_versions = 0;
+  double weight_bytes = 0.0;            // packed weights + scales + biases over all jobs
   size_t job_first = 0;                 // index of the first job record of this layer
   // fc only
   int n_pool = 0;
@@ -435,6 +470,7 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
         j.bias = li.bias;
         j.bits = bits;
         plan.jobs.push_back(j);
+        lp.weight_bytes += (double)li.d.cout * (row_bytes(li.K, bits) + 8.0);
       }
       continue;
     }
@@ -526,8 +562,8 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
     } else {                       // internal activations: NHWC
       g.in_sb = (long long)li.Hi * li.Wi * li.d.cin; g.in_sy = (long long)li.Wi * li.d.cin; g.in_sx = li.d.cin; g.in_sc = 1;
     }
-    if (li.d.kind == AIQ_LAYER_DEPTHWISE) st = launch_depthwise(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, stream);
-    else st = launch_conv(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, stream);
+    if (li.d.kind == AIQ_LAYER_DEPTHWISE) st = launch_depthwise(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, lp.weight_bytes, stream);
+    else st = launch_conv(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, lp.weight_bytes, stream);
     if (st != AIQ_OK) return st;
   }
   return AIQ_OK;
@@ -669,6 +705,34 @@ extern "C" aiq_status_t aiq_scheme_ai(const aiq_model_t* model, const uint8_t* s
   if (ai) *ai = fl / by;
   if (flops) *flops = fl;
   if (bytes) *bytes = by;
+  return AIQ_OK;
+}
+
+extern "C" aiq_status_t aiq_profile_start(void) {
+  using namespace aiq;
+  if (!t_prof) t_prof = new std::vector<ProfiledLaunch>();
+  if (!t_event_pool) t_event_pool = new std::vector<cudaEvent_t>();
+  for (ProfiledLaunch& pl : *t_prof) { t_event_pool->push_back(pl.start); t_event_pool->push_back(pl.stop); }
+  t_prof->clear();
+  memset(t_work, 0, sizeof(t_work));
+  t_profiling = true;
+  return AIQ_OK;
+}
+
+extern "C" aiq_status_t aiq_profile_stop(aiq_kernel_profile_t* out) {
+  using namespace aiq;
+  if (!out) return set_error(AIQ_ERR_INVALID_ARG, "aiq_profile_stop: null pointer");
+  if (!t_profiling) return set_error(AIQ_ERR_INVALID_ARG, "aiq_profile_stop without aiq_profile_start");
+  t_profiling = false;
+  for (int k = 0; k < AIQ_KERNEL_KINDS; ++k) { out[k] = t_work[k]; out[k].ms = 0.0; }
+  for (ProfiledLaunch& pl : *t_prof) {
+    AIQ_CUDA_TRY(cudaEventSynchronize(pl.stop));
+    float ms = 0.f;
+    AIQ_CUDA_TRY(cudaEventElapsedTime(&ms, pl.start, pl.stop));
+    out[pl.kind].ms += ms;
+  }
+  for (ProfiledLaunch& pl : *t_prof) { t_event_pool->push_back(pl.start); t_event_pool->push_back(pl.stop); }
+  t_prof->clear();
   return AIQ_OK;
 }
 

@@ -143,6 +143,8 @@ template <int BITS>
 aiq_status_t launch_bits(const LayerJob* jobs_dev, const LayerJob& single, int n_jobs, int N, int K,
                          int M, cudaStream_t s) {
   const int gx = (N + kWarps * kRowsPerWarp - 1) / (kWarps * kRowsPerWarp);
+  LaunchScope scope(AIQ_KERNEL_QLINEAR, s, 2.0 * M * N * K * n_jobs,
+                    n_jobs * ((double)N * row_bytes(K, BITS) + 4.0 * N + 4.0 * M * ((double)K + N)));
   if (M == 1) {
     qlinear_kernel<BITS, 1><<<dim3(gx, 1, n_jobs), kWarps * 32, 0, s>>>(single, jobs_dev, N, K, M);
   } else if (M == 2) {

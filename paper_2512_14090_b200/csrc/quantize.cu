@@ -27,7 +27,10 @@ aiq_status_t launch_fold_bn(const float* W, const float* gamma, const float* bet
                             const float* var, int N, int K, float eps, float* Wf, float* bf,
                             cudaStream_t s) {
   int threads = K >= 256 ? 256 : (K >= 128 ? 128 : (K >= 64 ? 64 : 32));
-  fold_bn_kernel<<<N, threads, 0, s>>>(W, gamma, beta, mean, var, K, eps, Wf, bf);
+  {
+    LaunchScope scope(AIQ_KERNEL_FOLD, s, (double)N * K, 8.0 * N * K + 20.0 * N);
+    fold_bn_kernel<<<N, threads, 0, s>>>(W, gamma, beta, mean, var, K, eps, Wf, bf);
+  }
   AIQ_LAUNCH_CHECK("fold_bn");
   return AIQ_OK;
 }
@@ -174,10 +177,14 @@ aiq_status_t launch_quantize(const float* W, int N, int K, int bits, void* packe
   int threads = 32;
   while (threads < 256 && threads < n_gran) threads <<= 1;
   uint8_t* p = static_cast<uint8_t*>(packed);
-  if (n_gran <= threads) {
-    quantize_rows_kernel<1><<<N, threads, 0, s>>>(W, K, Kpad, bits, p, scales, nonfinite_flag);
-  } else {
-    quantize_rows_kernel<4><<<N, threads, 0, s>>>(W, K, Kpad, bits, p, scales, nonfinite_flag);
+  {
+    LaunchScope scope(AIQ_KERNEL_QUANTIZE, s, 2.0 * N * K,
+                      4.0 * N * K + (double)N * row_bytes(K, bits) + 4.0 * N);
+    if (n_gran <= threads) {
+      quantize_rows_kernel<1><<<N, threads, 0, s>>>(W, K, Kpad, bits, p, scales, nonfinite_flag);
+    } else {
+      quantize_rows_kernel<4><<<N, threads, 0, s>>>(W, K, Kpad, bits, p, scales, nonfinite_flag);
+    }
   }
   AIQ_LAUNCH_CHECK("quantize_rows");
   return AIQ_OK;
