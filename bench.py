@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the AIQ scheme-evaluation hot path on B200.
+
+One step = one greedy search step on CIFAR ResNet-20: build the model's weight bank (fold
+batch-norm, quantize + pack every layer at 4/8/16/32 bits), then score 21 candidate schemes
+(each lowers one conv layer of an all-8-bit scheme to 4 bits) on a 10,000-image evaluation
+set, and compute each candidate's analytic arithmetic intensity.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl native|reference]
+
+Prints one JSON line (rank 0).  `value` is scheme evaluations per second with the images
+resident in device memory; `e2e` repeats the measurement with the images in pinned host
+memory, copied to the device inside the timed region.  With N > 1 (torchrun) every rank
+scores the same candidates on its own 10,000-image shard and the per-scheme counts are
+summed over ranks (weak scaling).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+N_IMAGES = 10000
+SEED_MODEL, SEED_IMAGES = 1234, 5679
+WORKLOAD = "resnet20_cifar_greedy_step: 21 schemes (all-8, one conv layer -> 4 bits) x 10000 images"
+METRIC = "scheme evals/sec (ResNet-20, 10k imgs)"
+UNIT = "scheme-evals/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the
+# committed ncu summary under profiles/ (None until captured / after the kernel changed)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                    sm_max_mhz=p.get("sm_max_mhz", 1965.0), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0,
+                sm_max_mhz=1965.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clock and throttle reasons while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.gpu_index)], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    mx.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                    samples=len(sm))
+
+
+def oracle_sample_rate(n_sample_images, schemes, arch, params, x):
+    """Times the CPU oracle, as it stands, on `n_sample_images` images x all schemes and
+    scales linearly to the 10,000-image set.  Returns (scheme-evals/s, seconds, threads)."""
+    from oracle import aiq_oracle as O
+    threads = os.cpu_count() or 1
+    try:
+        from threadpoolctl import threadpool_info
+        nt = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if nt:
+            threads = max(nt)
+    except Exception:
+        pass
+    t0 = time.perf_counter()
+    folded = O.fold_model(arch, params)
+    bank = O.build_weight_bank(folded, bits_set=(4, 8))
+    xs = x[:n_sample_images]
+    labels = O.predict(O.forward_scheme(arch, bank, [8] * len(arch["layers"]), xs))
+    O.eval_schemes(arch, bank, schemes, xs, labels)
+    for s in schemes:
+        O.scheme_ai(arch, s)
+    dt = time.perf_counter() - t0
+    evals_per_s = len(schemes) / (dt * (N_IMAGES / float(n_sample_images)))
+    return evals_per_s, dt, threads
+
+
+def run_reference(args, rank, world):
+    """--impl reference: the CPU oracle on the host cores, rank 0 only."""
+    if rank != 0:
+        return
+    from aiq_workloads import resnet20, gen_model, gen_images, one_layer_lowered_schemes, conv_layer_indices
+    arch = resnet20()
+    params = gen_model(arch, SEED_MODEL)
+    schemes = one_layer_lowered_schemes(len(arch["layers"]), conv_layer_indices(arch))
+    n_sample = 16
+    x = gen_images(n_sample, 3, 32, 32, SEED_IMAGES)
+    for _ in range(args.warmup):
+        oracle_sample_rate(4, schemes, arch, params, x)
+    secs, threads = 0.0, 1
+    for _ in range(args.steps):
+        _, dt, threads = oracle_sample_rate(n_sample, schemes, arch, params, x)
+        secs += dt
+    value = len(schemes) * args.steps / (secs * (N_IMAGES / float(n_sample)))
+    sample = (f"each step: all 21 schemes on the first {n_sample} of the 10000 images (fold, bank, "
+              f"labels, forward, count, AI), scaled linearly by 10000/{n_sample}")
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=1000.0 * secs / args.steps * (N_IMAGES / float(n_sample)),
+                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=WORKLOAD, note="CPU oracle (NumPy float64), extrapolated from a sample"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=threads, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--chunk", type=int, default=0, help="images per evaluator pass (0 = library default)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import torch.distributed as dist
+    from paper_2512_14090_b200 import build
+    build.build()
+    from paper_2512_14090_b200 import binding as aiq          # fails loudly without libaiq.so
+    from paper_2512_14090_b200.sharding import reduce_counts
+    from aiq_workloads import resnet20, gen_model, gen_images, one_layer_lowered_schemes, conv_layer_indices
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    arch = resnet20()
+    params = gen_model(arch, SEED_MODEL)
+    L = len(arch["layers"])
+    schemes = one_layer_lowered_schemes(L, conv_layer_indices(arch))
+    S = len(schemes)
+    x_host = torch.from_numpy(gen_images(N_IMAGES, 3, 32, 32, SEED_IMAGES + rank)).pin_memory()
+    x_dev = x_host.to(dev)
+    model = aiq.Model(arch, params, device=dev)
+    chunk = args.chunk if args.chunk > 0 else 256
+    aiq.aiq_set_eval_options(args.chunk, True)
+    ws = torch.empty(model.aiq_workspace_bytes(chunk, S), dtype=torch.uint8, device=dev)
+
+    # labels = arg-max of the FP32 model (the all-32 scheme), computed once by the library
+    preds32 = torch.empty((1, N_IMAGES), dtype=torch.int32, device=dev)
+    model.aiq_eval_schemes(np.full((1, L), 32, np.uint8), x_dev, torch.zeros(N_IMAGES, dtype=torch.int32, device=dev),
+                           preds=preds32, workspace=ws)
+    labels_dev = preds32[0].contiguous()
+    labels_host = labels_dev.cpu().pin_memory()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # > L2 (126 MB)
+    mem = model.mem
+    launches = [0]
+    bank_launches = sum(1 for l in arch["layers"] if l["has_bn"]) + 4 * L   # fold + 4 quantize per layer
+    result = {}
+
+    def step(x, labels):
+        m = aiq.Model(arch, params, device=dev, mem=mem)                 # fold + quantize bank
+        acc, counts = m.aiq_eval_schemes(schemes, x, labels, workspace=ws)
+        launches[0] += aiq.aiq_last_call_stats()["kernel_launches"] + bank_launches
+        ai = [m.aiq_scheme_ai(s)[0] for s in schemes]
+        if world > 1:
+            counts, total, acc = reduce_counts(counts, N_IMAGES, device=dev)
+        result.update(acc=np.asarray(acc, dtype=np.float64), ai=ai)
+        m.close()
+
+    def step_e2e():
+        xd = x_dev_e2e.copy_(x_host, non_blocking=True)
+        ld = labels_dev_e2e.copy_(labels_host, non_blocking=True)
+        step(xd, ld)
+
+    def timed(fn, n):
+        total_ms = 0.0
+        for _ in range(n):
+            flush.zero_()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            total_ms += e0.elapsed_time(e1)
+        return total_ms
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return ms
+
+    # ---- device-resident measurement ----------------------------------------------------
+    for _ in range(args.warmup):
+        step(x_dev, labels_dev)
+    launches[0] = 0
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    aiq.aiq_profile_start()
+    total_ms = timed(lambda: step(x_dev, labels_dev), args.steps)
+    prof = aiq.aiq_profile_stop()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = max_over_ranks(total_ms)
+    gpu_launches = launches[0]
+    ms_per_step = total_ms / args.steps
+    value = world * S * args.steps / (total_ms / 1000.0)
+
+    # ---- end to end: images and labels start in pinned host memory ----------------------
+    x_dev_e2e = torch.empty_like(x_dev)
+    labels_dev_e2e = torch.empty_like(labels_dev)
+    for _ in range(2):
+        step_e2e()
+    barrier()
+    e2e_ms = max_over_ranks(timed(step_e2e, args.steps))
+    barrier()
+    weight_bytes = sum(int(np.asarray(v).nbytes) for p in params for v in p.values())
+    h2d = x_host.numel() * 4 + labels_host.numel() * 4 + weight_bytes + S * L
+    d2h = S * 4 + 4
+    e2e_value = world * S * args.steps / (e2e_ms / 1000.0)
+
+    # ---- roofline of the dominant kernel -------------------------------------------------
+    peaks = measured_peaks()
+    top = max(prof, key=lambda k: prof[k]["ms"])
+    p = prof[top]
+    avg_ms = p["ms"] / max(p["launches"], 1)
+    sm_mhz = clocks.get("sm_mhz") or peaks["sm_max_mhz"]
+    if top == "conv":
+        # float32 multiply-add path: 148 SMs x 128 lanes x 2 FLOP per clock
+        peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12
+        achieved = p["flops"] / (p["ms"] / 1000.0) / 1e12
+        roofline = dict(bound="alu", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
+                        traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH, kernel="conv_igemm_kernel (float32 FMA)",
+                        peak_source=f"148 SMs x 128 FP32 lanes x 2 x {sm_mhz:.0f} MHz (median SM clock sampled during the run)",
+                        launches=p["launches"], avg_launch_ms=avg_ms,
+                        algorithmic_flops_per_launch=p["flops"] / max(p["launches"], 1),
+                        algorithmic_bytes_per_launch=p["bytes"] / max(p["launches"], 1))
+    else:
+        achieved = p["bytes"] / (p["ms"] / 1000.0) / 1e9
+        roofline = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=achieved / peaks["hbm_gbs"], traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                        kernel=top, peak_source=f"HBM copy bandwidth, {peaks['source']}",
+                        launches=p["launches"], avg_launch_ms=avg_ms,
+                        algorithmic_bytes_per_launch=p["bytes"] / max(p["launches"], 1))
+    all_ms = max(sum(q["ms"] for q in prof.values()), 1e-9)
+    kernel_share = {k: round(v["ms"] / all_ms, 4) for k, v in prof.items() if v["launches"]}
+
+    # ---- CPU oracle beside it (rank 0, N = 1 only) ----------------------------------------
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_sample = 128
+        v, dt, threads = oracle_sample_rate(n_sample, schemes, arch, params, x_host[:n_sample].numpy())
+        cpu_baseline = dict(value=v, unit=UNIT, cores=threads, kind="oracle", seconds=dt,
+                            sample=f"all 21 schemes on the first {n_sample} of the 10000 images (fold, bank, "
+                                   f"labels, forward, count, AI), scaled linearly by 10000/{n_sample}")
+
+    if rank == 0:
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                    ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype="f32", data="synthetic",
+                    config=dict(workload=WORKLOAD, images_per_rank=N_IMAGES, schemes=S, layers=L,
+                                chunk=chunk, l2="flushed between timed steps (256 MiB write)",
+                                step="fold + quantize bank (4/8/16/32 bits) + eval 21 schemes + AI",
+                                labels="arg-max of the all-32-bit scheme, computed by the library",
+                                prefix_sharing=True),
+                    e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                             ms_per_step=e2e_ms / args.steps),
+                    gpu_launches=gpu_launches, clocks=clocks, roofline=roofline, cpu_baseline=cpu_baseline,
+                    kernel_time_share=kernel_share,
+                    images_per_s=world * S * N_IMAGES * args.steps / (total_ms / 1000.0),
+                    acc_min=float(result["acc"].min()), acc_max=float(result["acc"].max()),
+                    ai_min=float(min(result["ai"])), ai_max=float(max(result["ai"])))
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
