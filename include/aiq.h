@@ -192,6 +192,36 @@ aiq_status_t aiq_forward(const aiq_model_t* model, const uint8_t* scheme_bits, c
                          void* stream);
 
 /* ------------------------------------------------------------------------------------
+ * aiq_forward without a caller-provided workspace.  (The paper has no counterpart: this is
+ * a packaging variant of aiq_forward, not a step of the method.)
+ *
+ * Some callers cannot obtain device memory at the moment they need a forward pass: code
+ * that runs inside another framework's callback where cudaMalloc (which synchronises the
+ * whole device) is forbidden, services that received a fixed memory budget at start-up and
+ * have already handed all of it out, or plug-ins that are given input and output buffers
+ * and nothing else.  For them the library carries its own workspace: a fixed device array
+ * of AIQ_STATIC_WORKSPACE_BYTES that belongs to the library image.  Every GPU that loads
+ * the library holds that array until the process exits, whether or not this call is used.
+ *
+ * Same arguments, results and asynchrony as aiq_forward, minus the workspace.  The call
+ * makes no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   - Limit: if the model at this batch needs more than AIQ_STATIC_WORKSPACE_BYTES (see
+ *     aiq_workspace_bytes(model, batch, 1)) the call returns AIQ_ERR_WORKSPACE_TOO_SMALL
+ *     and launches nothing; lower the batch or use aiq_forward.  8 MiB fits, e.g.,
+ *     ResNet-20 up to batch 42.
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress with that device current).  Make that first call outside any
+ *     stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the previous call
+ *     left there.  A forward pass needs nothing zeroed, so nothing is cleared; but two calls
+ *     whose kernels overlap on the GPU (different streams, or different host threads) write
+ *     the same scratch and race.  Issue them on one stream, or order them yourself.
+ */
+#define AIQ_STATIC_WORKSPACE_BYTES (8u * 1024u * 1024u)
+aiq_status_t aiq_forward_static(const aiq_model_t* model, const uint8_t* scheme_bits,
+                                const float* x, int batch, float* logits, void* stream);
+
+/* ------------------------------------------------------------------------------------
  * Many candidate schemes, whole evaluation set - the inner loop of greedy search and
  * coordinate descent (Section 2.2), which evaluates L(q; lambda) for every candidate move
  * and so needs each candidate's accuracy on the validation images.

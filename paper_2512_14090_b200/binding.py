@@ -25,8 +25,10 @@ EXPORTS = [
     "aiq_model_destroy", "aiq_model_num_layers", "aiq_model_num_classes",
     "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
     "aiq_eval_schemes", "aiq_set_eval_options", "aiq_last_call_stats", "aiq_scheme_ai",
-    "aiq_profile_start", "aiq_profile_stop",
+    "aiq_profile_start", "aiq_profile_stop", "aiq_forward_static",
 ]
+
+STATIC_WORKSPACE_BYTES = 8 * 1024 * 1024
 
 KERNEL_KINDS = ["fold", "quantize", "qlinear", "conv", "depthwise", "pool", "argmax"]
 
@@ -103,6 +105,8 @@ def _load():
     lib.aiq_scheme_ai.restype = i32
     lib.aiq_scheme_ai.argtypes = [vp, vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double),
                                   C.POINTER(C.c_double)]
+    lib.aiq_forward_static.restype = i32
+    lib.aiq_forward_static.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.aiq_profile_start.restype = i32
     lib.aiq_profile_start.argtypes = []
     lib.aiq_profile_stop.restype = i32
@@ -292,6 +296,16 @@ class Model:
         ws = workspace if workspace is not None else self.workspace(B, 1)
         _check(lib.aiq_forward(self.handle, _host(scheme), _dev(x), B, _dev(logits), _dev(ws),
                                ws.numel(), _stream(stream)))
+        return logits
+
+    def aiq_forward_static(self, scheme_bits, x, logits, stream=None):
+        """aiq_forward on the library's built-in workspace.  `logits` must be provided by the
+        caller ([batch][n_classes] float32 CUDA tensor): this call allocates nothing."""
+        scheme = np.ascontiguousarray(scheme_bits, dtype=np.uint8)
+        if scheme.shape != (self.n_layers,):
+            raise ValueError("scheme length must equal the number of layers")
+        _check(lib.aiq_forward_static(self.handle, _host(scheme), _dev(x), int(x.shape[0]),
+                                      _dev(logits), _stream(stream)))
         return logits
 
     def aiq_eval_schemes(self, schemes, x, labels, preds=None, workspace=None, chunk=256,

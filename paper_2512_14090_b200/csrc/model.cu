@@ -685,6 +685,54 @@ extern "C" aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t
 }
 
 // ---------------------------------------------------------------------------------------
+// aiq_forward for callers that have no device memory to lend as workspace.
+//
+// The workspace of this variant is a fixed array that is part of the library image: every
+// GPU that loads the library keeps AIQ_STATIC_WORKSPACE_BYTES of it until the process ends.
+// In host code the array's name is only a handle for the runtime, not a device address, so
+// the address is looked up once per device with cudaGetSymbolAddress and that pointer is
+// what the kernels receive.
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_workspace[AIQ_STATIC_WORKSPACE_BYTES];
+
+namespace aiq {
+static void* g_static_ws_ptr[64];        // per device; nullptr until the first call on it
+static bool g_static_ws_ready[64];
+}  // namespace aiq
+
+extern "C" aiq_status_t aiq_forward_static(const aiq_model_t* model, const uint8_t* scheme_bits,
+                                           const float* x, int batch, float* logits, void* stream_) {
+  using namespace aiq;
+  if (!model || !scheme_bits || !x || !logits)
+    return set_error(AIQ_ERR_INVALID_ARG, "aiq_forward_static: null pointer");
+  if (batch <= 0) return set_error(AIQ_ERR_INVALID_ARG, "aiq_forward_static: batch=%d", batch);
+  const size_t need = ws_layout(model, batch, 1).total;
+  if (need > (size_t)AIQ_STATIC_WORKSPACE_BYTES)
+    return set_error(AIQ_ERR_WORKSPACE_TOO_SMALL,
+                     "aiq_forward_static: batch %d of this model needs %zu workspace bytes, the built-in "
+                     "workspace holds %zu; use a smaller batch or aiq_forward with your own workspace",
+                     batch, need, (size_t)AIQ_STATIC_WORKSPACE_BYTES);
+  aiq_status_t st = check_device_sm100();
+  if (st != AIQ_OK) return st;
+  int dev = 0;
+  AIQ_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return set_error(AIQ_ERR_INVALID_ARG, "aiq_forward_static: device %d", dev);
+  if (!g_static_ws_ready[dev]) {
+    // first call on this device (it is the current one): resolve the array's device address
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_workspace);
+    if (e != cudaSuccess || !ptr)
+      return set_error(AIQ_ERR_CUDA, "cudaGetSymbolAddress(static workspace): %s", cudaGetErrorString(e));
+    g_static_ws_ptr[dev] = ptr;
+    g_static_ws_ready[dev] = true;
+  }
+  // Nothing in the workspace has to start at zero for a forward pass: the job records are
+  // copied in, and every activation, pooled value and logit is written before it is read.
+  return aiq_forward(model, scheme_bits, x, batch, logits, g_static_ws_ptr[dev],
+                     (size_t)AIQ_STATIC_WORKSPACE_BYTES, stream_);
+}
+
+// ---------------------------------------------------------------------------------------
 // analytic arithmetic intensity (host only)
 // ---------------------------------------------------------------------------------------
 extern "C" aiq_status_t aiq_scheme_ai(const aiq_model_t* model, const uint8_t* scheme_bits, int ai_batch,
