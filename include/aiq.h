@@ -208,7 +208,7 @@ aiq_status_t aiq_forward(const aiq_model_t* model, const uint8_t* scheme_bits, c
  *   - Limit: if the model at this batch needs more than AIQ_STATIC_WORKSPACE_BYTES (see
  *     aiq_workspace_bytes(model, batch, 1)) the call returns AIQ_ERR_WORKSPACE_TOO_SMALL
  *     and launches nothing; lower the batch or use aiq_forward.  8 MiB fits, e.g.,
- *     ResNet-20 up to batch 42.
+ *     ResNet-20 up to batch 40.
  *   - The first call on each device looks up the array's device address (one
  *     cudaGetSymbolAddress with that device current).  Make that first call outside any
  *     stream capture.
@@ -242,6 +242,21 @@ aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t* schemes, 
  * them).  chunk: images per pass, 0 = choose from the workspace size.  share_prefix: 0
  * evaluates every scheme independently. */
 void aiq_set_eval_options(int chunk, int share_prefix);
+
+/* Compute path of models created after the call (process-wide; the paper has no kernels,
+ * Section 3 runs stock PyTorch, so this is an implementation choice, not a step of AIQ):
+ *   AIQ_PATH_FP32    every layer on float32 multiply-add kernels, activations stored as
+ *                    float32.  Logits agree with a float64 reference to ~1e-5 relative.
+ *   AIQ_PATH_TENSOR  dense 3x3 / 1x1 convolutions with 4- or 8-bit weights and 16/32/64
+ *                    channels run on the bf16 tensor cores (tcgen05, float32 accumulation
+ *                    in tensor memory); activations are stored as the sum of two bfloat16
+ *                    (17-18 significant bits).  Other layers use the float32 kernels on the
+ *                    same storage.
+ *   AIQ_PATH_AUTO    AIQ_PATH_TENSOR when the model has at least one layer the tensor
+ *                    kernels accept, else AIQ_PATH_FP32.  This is the default.
+ */
+enum { AIQ_PATH_AUTO = 0, AIQ_PATH_FP32 = 1, AIQ_PATH_TENSOR = 2 };
+void aiq_set_compute_path(int path);
 
 /* Counters of the last aiq_forward / aiq_eval_schemes call on this thread: kernels
  * launched, and layer evaluations executed vs. n_schemes * L * chunks without sharing. */

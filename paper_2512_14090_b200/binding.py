@@ -26,7 +26,10 @@ EXPORTS = [
     "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
     "aiq_eval_schemes", "aiq_set_eval_options", "aiq_last_call_stats", "aiq_scheme_ai",
     "aiq_profile_start", "aiq_profile_stop", "aiq_forward_static",
+    "aiq_set_compute_path",
 ]
+
+PATH_AUTO, PATH_FP32, PATH_TENSOR = 0, 1, 2
 
 STATIC_WORKSPACE_BYTES = 8 * 1024 * 1024
 
@@ -107,6 +110,8 @@ def _load():
                                   C.POINTER(C.c_double)]
     lib.aiq_forward_static.restype = i32
     lib.aiq_forward_static.argtypes = [vp, vp, vp, i32, vp, vp]
+    lib.aiq_set_compute_path.restype = None
+    lib.aiq_set_compute_path.argtypes = [i32]
     lib.aiq_profile_start.restype = i32
     lib.aiq_profile_start.argtypes = []
     lib.aiq_profile_stop.restype = i32
@@ -186,6 +191,10 @@ def aiq_qlinear(packed, scales, bias, N, K, bits, x, y, stream=None):
 
 def aiq_set_eval_options(chunk=0, share_prefix=True):
     lib.aiq_set_eval_options(int(chunk), int(bool(share_prefix)))
+
+
+def aiq_set_compute_path(path):
+    lib.aiq_set_compute_path(int(path))
 
 
 def aiq_last_call_stats():

@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_fp16.h>
+#include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
 
@@ -69,25 +70,50 @@ __device__ __forceinline__ float apply_act(float v, int act) {
   return v;
 }
 
+// ---- internal activation formats ----------------------------------------------------
+// Activation tensors between layers are [B][H+2][W][pixel] with Cs = channels rounded up to
+// a multiple of 16 and 4*Cs bytes per pixel.  Rows 0 and H+1 of every image are zero
+// (vertical padding stored physically, so that (image, row) is one uniform dimension);
+// channels >= C are zero.  Two pixel formats:
+//   ACT_F32   Cs floats.  Used when every layer of the model runs on the float32 path.
+//   ACT_SPLIT [hi(Cs) | lo(Cs)] bfloat16, value = float(hi) + float(lo) with
+//             hi = bf16_rn(v), lo = bf16_rn(v - hi): 16+ significant bits in the same bytes,
+//             in the form the bf16 tensor cores consume without conversion (the two halves
+//             are two K-slices of the GEMM).  Used when the model has tensor-core layers.
+enum { ACT_F32 = 0, ACT_SPLIT = 1 };
+inline int padded_channels(int C) { return (C + 15) / 16 * 16; }
+inline size_t split_image_bytes(int H, int W, int C) {
+  return (size_t)(H + 2) * W * 2 * padded_channels(C) * 2;
+}
+
+__device__ __forceinline__ void split_bf16(float v, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+  hi = __float2bfloat16_rn(v);
+  lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
 // ---- job records: one evaluation of one layer under one weight choice ---------------
 // Device-resident arrays of these let a single launch cover every distinct version of a
 // layer that a group of schemes needs (gridDim.z = number of jobs).
 struct LayerJob {
-  const float* in;      // activations NHWC (nullptr: the network input passed as a kernel argument)
-  const float* res;     // residual operand NHWC, or nullptr
-  float* out;           // NHWC
+  const void* in;       // split activations (nullptr: the float32 NCHW network input, a kernel argument);
+                        // head jobs: float32 pooled features / logits
+  const void* res;      // residual operand (split), or nullptr
+  void* out;            // split activations; head jobs: float32
   const uint8_t* w;     // packed rows (aiq_quantize_layer layout)
   const float* scale;   // [cout]
   const float* bias;    // [cout]
   int32_t bits;
   int32_t label_slot;   // head jobs: index of the count / prediction row
+  int32_t in_version;   // index of `in` along the version dimension of its slot
+  int32_t pad_;
 };
 
 struct ConvGeom {
   int B, H, W, Cin, Ho, Wo, Cout, ks, stride, pad, act;
-  int K;            // Cin/groups * ks * ks
-  int row_bytes;    // packed row stride at the job's bit-width is computed per job
-  long long in_sb, in_sy, in_sx, in_sc;   // element strides of the input tensor
+  int K;              // Cin/groups * ks * ks
+  int Cs_in, Cs_out;  // padded channel counts of the split tensors
+  int in_is_nchw;     // 1: the input is the float32 NCHW network input
+  int act_format;     // ACT_F32 or ACT_SPLIT, for input, residual and output alike
 };
 
 // ---- launchers (defined in the .cu files) --------------------------------------------
@@ -104,8 +130,9 @@ aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs
                          const float* net_input, double weight_bytes, cudaStream_t s);
 aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
                               const float* net_input, double weight_bytes, cudaStream_t s);
-// pooled[b][c] = mean over HW of in[b][hw][c], per job (in -> out)
-aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int HW, int C, cudaStream_t s);
+// pooled[b][c] = mean over the H x W interior of a split tensor, per job (in -> out float32 [B][C])
+aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int H, int W, int C, int act_format,
+                            cudaStream_t s);
 // pred = lowest index of the max logit; preds[slot][img0 + b] = pred; counts[slot] += (pred == label)
 aiq_status_t launch_argmax_count(const LayerJob* jobs_dev, int n_jobs, int B, int n_classes,
                                  const int32_t* labels, int32_t* counts, int32_t* preds,

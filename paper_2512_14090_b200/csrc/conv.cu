@@ -7,6 +7,7 @@
 // accuracy measurement).  Weights are read in their packed form and expanded while they
 // are staged; the per-channel scale multiplies the finished float32 sum; bias, residual
 // add and activation are applied before the single store of the output tensor.
+// Activations are read and written in the split bfloat16 format described in common.cuh.
 #include "common.cuh"
 
 namespace aiq {
@@ -16,22 +17,78 @@ namespace {
 constexpr int kConvThreads = 256;
 constexpr int BK = 16;
 
+enum { IN_NCHW = 0, IN_SPLIT_VEC = 1, IN_SPLIT_SCALAR = 2 };
+
+__device__ __forceinline__ float4 load_split4(const __nv_bfloat16* __restrict__ pix, int c, int Cs) {
+  // 4 consecutive channels of one pixel: hi and lo halves are 8-byte loads
+  const uint2 h = __ldg(reinterpret_cast<const uint2*>(pix + c));
+  const uint2 l = __ldg(reinterpret_cast<const uint2*>(pix + Cs + c));
+  const __nv_bfloat162 h0 = *reinterpret_cast<const __nv_bfloat162*>(&h.x);
+  const __nv_bfloat162 h1 = *reinterpret_cast<const __nv_bfloat162*>(&h.y);
+  const __nv_bfloat162 l0 = *reinterpret_cast<const __nv_bfloat162*>(&l.x);
+  const __nv_bfloat162 l1 = *reinterpret_cast<const __nv_bfloat162*>(&l.y);
+  const float2 a = __bfloat1622float2(h0), b = __bfloat1622float2(h1);
+  const float2 c0 = __bfloat1622float2(l0), c1 = __bfloat1622float2(l1);
+  return make_float4(a.x + c0.x, a.y + c0.y, b.x + c1.x, b.y + c1.y);
+}
+
+__device__ __forceinline__ void store_split4(__nv_bfloat16* __restrict__ pix, int c, int Cs, float4 v) {
+  __nv_bfloat16 h[4], l[4];
+  split_bf16(v.x, h[0], l[0]);
+  split_bf16(v.y, h[1], l[1]);
+  split_bf16(v.z, h[2], l[2]);
+  split_bf16(v.w, h[3], l[3]);
+  uint2 hv, lv;
+  hv.x = (uint32_t)__bfloat16_as_ushort(h[0]) | ((uint32_t)__bfloat16_as_ushort(h[1]) << 16);
+  hv.y = (uint32_t)__bfloat16_as_ushort(h[2]) | ((uint32_t)__bfloat16_as_ushort(h[3]) << 16);
+  lv.x = (uint32_t)__bfloat16_as_ushort(l[0]) | ((uint32_t)__bfloat16_as_ushort(l[1]) << 16);
+  lv.y = (uint32_t)__bfloat16_as_ushort(l[2]) | ((uint32_t)__bfloat16_as_ushort(l[3]) << 16);
+  *reinterpret_cast<uint2*>(pix + c) = hv;
+  *reinterpret_cast<uint2*>(pix + Cs + c) = lv;
+}
+
+// Element access of an activation tensor in either storage format.  A pixel is 4*Cs bytes
+// in both: Cs floats (ACT_F32) or [hi Cs | lo Cs] bfloat16 (ACT_SPLIT).
+template <int FMT>
+__device__ __forceinline__ float4 act_load4(const void* __restrict__ base, size_t pixel, int c, int Cs) {
+  if (FMT == ACT_SPLIT)
+    return load_split4(static_cast<const __nv_bfloat16*>(base) + pixel * 2 * Cs, c, Cs);
+  return __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(base) + pixel * Cs + c));
+}
+template <int FMT>
+__device__ __forceinline__ float act_load1(const void* __restrict__ base, size_t pixel, int c, int Cs) {
+  if (FMT == ACT_SPLIT) {
+    const __nv_bfloat16* px = static_cast<const __nv_bfloat16*>(base) + pixel * 2 * Cs;
+    return __bfloat162float(px[c]) + __bfloat162float(px[Cs + c]);
+  }
+  return __ldg(static_cast<const float*>(base) + pixel * Cs + c);
+}
+template <int FMT>
+__device__ __forceinline__ void act_store4(void* __restrict__ base, size_t pixel, int c, int Cs, float4 v) {
+  if (FMT == ACT_SPLIT)
+    store_split4(static_cast<__nv_bfloat16*>(base) + pixel * 2 * Cs, c, Cs, v);
+  else
+    *reinterpret_cast<float4*>(static_cast<float*>(base) + pixel * Cs + c) = v;
+}
+
 // Implicit GEMM:  out[p][n] = act( s_n * sum_k code[n][k] * patch[p][k] + b_n + res[p][n] )
-// p = (image, oy, ox) flattened, k = (tap, channel) with the channel fastest.
+// p runs over the *padded* output pixel space (image, row 0..Ho+1, column): border rows are
+// written as zeros.  k = (tap, channel) with the channel fastest.
 // Block tile BM pixels x BN channels, thread tile TM x TN, K consumed in slices of 16
 // through a double-buffered shared-memory stage.
 //   As[k][p ^ ((k >> 2) << 3)]   (XOR keeps groups of 4 pixels contiguous and makes the
 //                                 transposing stores of the vector path conflict-free)
 //   Bs[k][n]
-template <int BM, int BN, int TM, int TN, bool VEC>
+template <int BM, int BN, int TM, int TN, int IN_MODE, int FMT>
 __global__ void __launch_bounds__(kConvThreads)
 conv_igemm_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* __restrict__ net_input) {
   static_assert((BM / TM) * (BN / TN) == kConvThreads, "thread tile must cover the block tile");
   static_assert(TM % 4 == 0 && TN == 4, "thread tile shape");
+  constexpr bool VEC = IN_MODE == IN_SPLIT_VEC;
   const LayerJob job = jobs[blockIdx.z];
-  const float* __restrict__ in = job.in ? job.in : net_input;
   const int tid = threadIdx.x;
-  const int M = g.B * g.Ho * g.Wo;
+  const int rows_out = g.Ho + 2;
+  const int M = g.B * rows_out * g.Wo;            // padded output pixels
   const int p_base = blockIdx.x * BM;
   const int n_base = blockIdx.y * BN;
   const int Kt = g.ks * g.ks * g.Cin;
@@ -45,22 +102,21 @@ conv_igemm_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* __
   constexpr int A_VEC_PER_THREAD = BM * BK / 4 / kConvThreads;   // float4 fetches (VEC)
   constexpr int A_SCL_PER_THREAD = BM * BK / kConvThreads;       // scalar fetches (!VEC)
   constexpr int NPIX = VEC ? A_VEC_PER_THREAD : 1;
-  long long pix_off[NPIX];
-  int pix_iy0[NPIX], pix_ix0[NPIX];
+  int pix_b[NPIX], pix_iy0[NPIX], pix_ix0[NPIX];
   bool pix_ok[NPIX];
 #pragma unroll
   for (int i = 0; i < NPIX; ++i) {
     const int pl = VEC ? (tid >> 2) + i * (kConvThreads >> 2) : (tid % BM);
     const int p = p_base + pl;
-    pix_ok[i] = p < M;
-    const int pp = pix_ok[i] ? p : 0;
-    const int b = pp / (g.Ho * g.Wo);
-    const int rem = pp - b * (g.Ho * g.Wo);
-    const int oy = rem / g.Wo;
-    const int ox = rem - oy * g.Wo;
-    pix_iy0[i] = oy * g.stride - g.pad;
+    const int pp = p < M ? p : 0;
+    const int b = pp / (rows_out * g.Wo);
+    const int rem = pp - b * (rows_out * g.Wo);
+    const int oyp = rem / g.Wo;                     // padded row 0..Ho+1
+    const int ox = rem - oyp * g.Wo;
+    pix_ok[i] = p < M && oyp >= 1 && oyp <= g.Ho;
+    pix_b[i] = b;
+    pix_iy0[i] = (oyp - 1) * g.stride - g.pad;
     pix_ix0[i] = ox * g.stride - g.pad;
-    pix_off[i] = (long long)b * g.in_sb;
   }
 
   float a_reg[VEC ? A_VEC_PER_THREAD * 4 : A_SCL_PER_THREAD];
@@ -82,8 +138,7 @@ conv_igemm_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* __
         const int iy = pix_iy0[i] + r, ix = pix_ix0[i] + t;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (pix_ok[i] && kk < Kt && iy >= 0 && iy < g.H && ix >= 0 && ix < g.W)
-          v = __ldg(reinterpret_cast<const float4*>(in + pix_off[i] + (long long)iy * g.in_sy +
-                                                    (long long)ix * g.in_sx + c));
+          v = act_load4<FMT>(job.in, (size_t)(pix_b[i] * (g.H + 2) + iy + 1) * g.W + ix, c, g.Cs_in);
         a_reg[4 * i] = v.x; a_reg[4 * i + 1] = v.y; a_reg[4 * i + 2] = v.z; a_reg[4 * i + 3] = v.w;
       }
     } else {
@@ -97,9 +152,13 @@ conv_igemm_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* __
         const int t = tap - r * g.ks;
         const int iy = pix_iy0[0] + r, ix = pix_ix0[0] + t;
         float v = 0.f;
-        if (pix_ok[0] && kk < Kt && iy >= 0 && iy < g.H && ix >= 0 && ix < g.W)
-          v = __ldg(in + pix_off[0] + (long long)iy * g.in_sy + (long long)ix * g.in_sx +
-                    (long long)c * g.in_sc);
+        if (pix_ok[0] && kk < Kt && iy >= 0 && iy < g.H && ix >= 0 && ix < g.W) {
+          if (IN_MODE == IN_NCHW) {
+            v = __ldg(net_input + (((size_t)pix_b[0] * g.Cin + c) * g.H + iy) * g.W + ix);
+          } else {
+            v = act_load1<FMT>(job.in, (size_t)(pix_b[0] * (g.H + 2) + iy + 1) * g.W + ix, c, g.Cs_in);
+          }
+        }
         a_reg[i] = v;
       }
     }
@@ -184,68 +243,73 @@ conv_igemm_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* __
     }
   }
 
-  // ---- epilogue: scale, bias, residual, activation, one store
+  // ---- epilogue: scale, bias, residual, activation, split, one store.  Border rows and
+  // padded channels are written as zeros.
   const int n = n_base + tx * TN;
-  if (n >= g.Cout) return;
+  if (n >= g.Cs_out) return;
   float sc[TN], bi[TN];
+  bool ch_ok[TN];
 #pragma unroll
   for (int j = 0; j < TN; ++j) {
-    const bool ok = n + j < g.Cout;
-    sc[j] = ok ? job.scale[n + j] : 0.f;
-    bi[j] = ok ? job.bias[n + j] : 0.f;
+    ch_ok[j] = n + j < g.Cout;
+    sc[j] = ch_ok[j] ? job.scale[n + j] : 0.f;
+    bi[j] = ch_ok[j] ? job.bias[n + j] : 0.f;
   }
-  const bool full = (n + TN <= g.Cout) && ((g.Cout & 3) == 0);
 #pragma unroll
   for (int pg = 0; pg < PGROUPS; ++pg) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int p = p_base + pg * PG_STRIDE + ty * 4 + i;
       if (p >= M) continue;
-      float v[TN];
+      const int oyp = (p / g.Wo) % rows_out;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (oyp >= 1 && oyp <= g.Ho) {
+        float u[TN];
 #pragma unroll
-      for (int j = 0; j < TN; ++j) v[j] = fmaf(acc[4 * pg + i][j], sc[j], bi[j]);
-      float* o = job.out + (size_t)p * g.Cout + n;
-      if (full) {
+        for (int j = 0; j < TN; ++j) u[j] = fmaf(acc[4 * pg + i][j], sc[j], bi[j]);
         if (job.res) {
-          const float4 r = *reinterpret_cast<const float4*>(job.res + (size_t)p * g.Cout + n);
-          v[0] += r.x; v[1] += r.y; v[2] += r.z; v[3] += r.w;
+          const float4 r = act_load4<FMT>(job.res, (size_t)p, n, g.Cs_out);
+          u[0] += r.x; u[1] += r.y; u[2] += r.z; u[3] += r.w;
         }
-        *reinterpret_cast<float4*>(o) = make_float4(apply_act(v[0], g.act), apply_act(v[1], g.act),
-                                                    apply_act(v[2], g.act), apply_act(v[3], g.act));
-      } else {
-#pragma unroll
-        for (int j = 0; j < TN; ++j) {
-          if (n + j >= g.Cout) break;
-          float u = v[j];
-          if (job.res) u += job.res[(size_t)p * g.Cout + n + j];
-          o[j] = apply_act(u, g.act);
-        }
+        v = make_float4(ch_ok[0] ? apply_act(u[0], g.act) : 0.f, ch_ok[1] ? apply_act(u[1], g.act) : 0.f,
+                        ch_ok[2] ? apply_act(u[2], g.act) : 0.f, ch_ok[3] ? apply_act(u[3], g.act) : 0.f);
       }
+      act_store4<FMT>(job.out, (size_t)p, n, g.Cs_out, v);
     }
   }
 }
 
 template <int BM, int BN, int TM, int TN>
 aiq_status_t launch_conv_tile(const ConvGeom& g, const LayerJob* jobs, int n_jobs, const float* net_input,
-                              bool vec, double weight_bytes, cudaStream_t s) {
-  const int M = g.B * g.Ho * g.Wo;
-  dim3 grid((M + BM - 1) / BM, (g.Cout + BN - 1) / BN, n_jobs);
-  LaunchScope scope(AIQ_KERNEL_CONV, s, 2.0 * M * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
-                    weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W + (double)M * g.Cout));
-  if (vec)
-    conv_igemm_kernel<BM, BN, TM, TN, true><<<grid, kConvThreads, 0, s>>>(g, jobs, net_input);
-  else
-    conv_igemm_kernel<BM, BN, TM, TN, false><<<grid, kConvThreads, 0, s>>>(g, jobs, net_input);
+                              int in_mode, double weight_bytes, cudaStream_t s) {
+  const int M = g.B * (g.Ho + 2) * g.Wo;
+  dim3 grid((M + BM - 1) / BM, (g.Cs_out + BN - 1) / BN, n_jobs);
+  LaunchScope scope(AIQ_KERNEL_CONV, s,
+                    2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
+                    weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
+                                                   (double)g.B * g.Ho * g.Wo * g.Cout));
+#define AIQ_CONV_LAUNCH(MODE)                                                                        \
+  do {                                                                                              \
+    if (g.act_format == ACT_SPLIT)                                                                  \
+      conv_igemm_kernel<BM, BN, TM, TN, MODE, ACT_SPLIT><<<grid, kConvThreads, 0, s>>>(g, jobs, net_input); \
+    else                                                                                            \
+      conv_igemm_kernel<BM, BN, TM, TN, MODE, ACT_F32><<<grid, kConvThreads, 0, s>>>(g, jobs, net_input);   \
+  } while (0)
+  if (in_mode == IN_SPLIT_VEC) AIQ_CONV_LAUNCH(IN_SPLIT_VEC);
+  else if (in_mode == IN_SPLIT_SCALAR) AIQ_CONV_LAUNCH(IN_SPLIT_SCALAR);
+  else AIQ_CONV_LAUNCH(IN_NCHW);
+#undef AIQ_CONV_LAUNCH
   AIQ_LAUNCH_CHECK("conv_igemm");
   return AIQ_OK;
 }
 
 // ---------------------------------------------------------------------------------------
-// Depthwise 3x3 (NHWC).  A block owns a slice of up to 128 channels and a tile of pixels;
-// a lane owns 4 consecutive channels, so a warp reads 512 contiguous bytes per tap.
+// Depthwise 3x3 on split tensors.  A block owns a slice of up to 128 channels and a tile
+// of padded output pixels; a lane owns 4 consecutive channels.
 // ---------------------------------------------------------------------------------------
 constexpr int kDwPixPerBlock = 64;
 
+template <int FMT>
 __global__ void __launch_bounds__(256)
 depthwise3x3_kernel(ConvGeom g, const LayerJob* __restrict__ jobs) {
   const LayerJob job = jobs[blockIdx.z];
@@ -266,59 +330,65 @@ depthwise3x3_kernel(ConvGeom g, const LayerJob* __restrict__ jobs) {
   }
   __syncthreads();
   const int c = c_base + lane * 4;
-  if (c >= g.Cout) return;
-  const int M = g.B * g.Ho * g.Wo;
-  const int C = g.Cout;
+  if (c >= g.Cs_out) return;
+  const int rows_out = g.Ho + 2;
+  const int M = g.B * rows_out * g.Wo;
+  const int Cs = g.Cs_out;                              // == Cs_in
   const float4 sc = *reinterpret_cast<const float4*>(&ssm[lane * 4]);
   const float4 bi = *reinterpret_cast<const float4*>(&bsm[lane * 4]);
+  const bool ok0 = c < g.Cout, ok1 = c + 1 < g.Cout, ok2 = c + 2 < g.Cout, ok3 = c + 3 < g.Cout;
   for (int pi = warp; pi < kDwPixPerBlock; pi += 8) {
     const int p = blockIdx.x * kDwPixPerBlock + pi;
     if (p >= M) break;
-    const int b = p / (g.Ho * g.Wo);
-    const int rem = p - b * (g.Ho * g.Wo);
-    const int oy = rem / g.Wo, ox = rem - (rem / g.Wo) * g.Wo;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int b = p / (rows_out * g.Wo);
+    const int rem = p - b * (rows_out * g.Wo);
+    const int oyp = rem / g.Wo, ox = rem - (rem / g.Wo) * g.Wo;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (oyp >= 1 && oyp <= g.Ho) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int r = 0; r < 3; ++r) {
-      const int iy = oy * g.stride - 1 + r;
-      if (iy < 0 || iy >= g.H) continue;
+      for (int r = 0; r < 3; ++r) {
+        const int iy = (oyp - 1) * g.stride - 1 + r;
+        if (iy < 0 || iy >= g.H) continue;
 #pragma unroll
-      for (int t = 0; t < 3; ++t) {
-        const int ix = ox * g.stride - 1 + t;
-        if (ix < 0 || ix >= g.W) continue;
-        const float4 xv = __ldg(reinterpret_cast<const float4*>(
-            job.in + ((size_t)(b * g.H + iy) * g.W + ix) * C + c));
-        const float4 wv = *reinterpret_cast<const float4*>(&wsm[r * 3 + t][lane * 4]);
-        acc.x = fmaf(xv.x, wv.x, acc.x);
-        acc.y = fmaf(xv.y, wv.y, acc.y);
-        acc.z = fmaf(xv.z, wv.z, acc.z);
-        acc.w = fmaf(xv.w, wv.w, acc.w);
+        for (int t = 0; t < 3; ++t) {
+          const int ix = ox * g.stride - 1 + t;
+          if (ix < 0 || ix >= g.W) continue;
+          const float4 xv = act_load4<FMT>(job.in, (size_t)(b * (g.H + 2) + iy + 1) * g.W + ix, c, Cs);
+          const float4 wv = *reinterpret_cast<const float4*>(&wsm[r * 3 + t][lane * 4]);
+          acc.x = fmaf(xv.x, wv.x, acc.x);
+          acc.y = fmaf(xv.y, wv.y, acc.y);
+          acc.z = fmaf(xv.z, wv.z, acc.z);
+          acc.w = fmaf(xv.w, wv.w, acc.w);
+        }
       }
+      float4 u = make_float4(fmaf(acc.x, sc.x, bi.x), fmaf(acc.y, sc.y, bi.y), fmaf(acc.z, sc.z, bi.z),
+                             fmaf(acc.w, sc.w, bi.w));
+      if (job.res) {
+        const float4 rr = act_load4<FMT>(job.res, (size_t)p, c, Cs);
+        u.x += rr.x; u.y += rr.y; u.z += rr.z; u.w += rr.w;
+      }
+      v = make_float4(ok0 ? apply_act(u.x, g.act) : 0.f, ok1 ? apply_act(u.y, g.act) : 0.f,
+                      ok2 ? apply_act(u.z, g.act) : 0.f, ok3 ? apply_act(u.w, g.act) : 0.f);
     }
-    float4 v = make_float4(fmaf(acc.x, sc.x, bi.x), fmaf(acc.y, sc.y, bi.y), fmaf(acc.z, sc.z, bi.z),
-                           fmaf(acc.w, sc.w, bi.w));
-    if (job.res) {
-      const float4 rr = *reinterpret_cast<const float4*>(job.res + (size_t)p * C + c);
-      v.x += rr.x; v.y += rr.y; v.z += rr.z; v.w += rr.w;
-    }
-    *reinterpret_cast<float4*>(job.out + (size_t)p * C + c) =
-        make_float4(apply_act(v.x, g.act), apply_act(v.y, g.act), apply_act(v.z, g.act),
-                    apply_act(v.w, g.act));
+    act_store4<FMT>(job.out, (size_t)p, c, Cs, v);
   }
 }
 
 // ---------------------------------------------------------------------------------------
-// Global average pool: pooled[b][c] = (1/HW) * sum_hw in[b][hw][c]
+// Global average pool over the interior of a split tensor: pooled[b][c] float32
 // ---------------------------------------------------------------------------------------
-__global__ void avgpool_kernel(const LayerJob* __restrict__ jobs, int HW, int C) {
+template <int FMT>
+__global__ void avgpool_kernel(const LayerJob* __restrict__ jobs, int H, int W, int C, int Cs) {
   const LayerJob job = jobs[blockIdx.z];
   const int b = blockIdx.x;
-  const float inv = 1.0f / (float)HW;
+  const float inv = 1.0f / (float)(H * W);
+  float* __restrict__ out = static_cast<float*>(job.out);
+  const size_t p0 = ((size_t)b * (H + 2) + 1) * W;       // first interior pixel of image b
   for (int c = threadIdx.x; c < C; c += blockDim.x) {
-    const float* p = job.in + (size_t)b * HW * C + c;
     float s = 0.f;
-    for (int i = 0; i < HW; ++i) s += p[(size_t)i * C];
-    job.out[(size_t)b * C + c] = s * inv;
+    for (int i = 0; i < H * W; ++i) s += act_load1<FMT>(job.in, p0 + i, c, Cs);
+    out[(size_t)b * C + c] = s * inv;
   }
 }
 
@@ -333,7 +403,7 @@ __global__ void argmax_count_kernel(const LayerJob* __restrict__ jobs, int B, in
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   int correct = 0;
   if (b < B) {
-    const float* lg = job.in + (size_t)b * n_classes;
+    const float* lg = static_cast<const float*>(job.in) + (size_t)b * n_classes;
     float best = -INFINITY;
     int arg = 0x7fffffff;
     for (int j = lane; j < n_classes; j += 32) {
@@ -368,34 +438,38 @@ __global__ void argmax_count_kernel(const LayerJob* __restrict__ jobs, int B, in
 
 aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs, const float* net_input,
                          double weight_bytes, cudaStream_t s) {
-  // vector path: channel-contiguous (NHWC) input with a channel count that keeps float4
-  // groups inside one tap
-  const bool vec = (g.in_sc == 1) && (g.Cin % 4 == 0) && (g.in_sx % 4 == 0) && (g.in_sy % 4 == 0) &&
-                   (g.in_sb % 4 == 0);
-  auto waste = [&](int bn) { return (g.Cout + bn - 1) / bn * bn - g.Cout; };
+  const int in_mode = g.in_is_nchw ? IN_NCHW : ((g.Cin % 4 == 0) ? IN_SPLIT_VEC : IN_SPLIT_SCALAR);
+  auto waste = [&](int bn) { return (g.Cs_out + bn - 1) / bn * bn - g.Cs_out; };
   int bn = 64;
   if (waste(32) < waste(bn)) bn = 32;
   if (waste(16) < waste(bn)) bn = 16;
-  if (bn == 64) return launch_conv_tile<128, 64, 8, 4>(g, jobs_dev, n_jobs, net_input, vec, weight_bytes, s);
-  if (bn == 32) return launch_conv_tile<128, 32, 4, 4>(g, jobs_dev, n_jobs, net_input, vec, weight_bytes, s);
-  return launch_conv_tile<256, 16, 4, 4>(g, jobs_dev, n_jobs, net_input, vec, weight_bytes, s);
+  if (bn == 64) return launch_conv_tile<128, 64, 8, 4>(g, jobs_dev, n_jobs, net_input, in_mode, weight_bytes, s);
+  if (bn == 32) return launch_conv_tile<128, 32, 4, 4>(g, jobs_dev, n_jobs, net_input, in_mode, weight_bytes, s);
+  return launch_conv_tile<256, 16, 4, 4>(g, jobs_dev, n_jobs, net_input, in_mode, weight_bytes, s);
 }
 
 aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
                               const float* /*net_input*/, double weight_bytes, cudaStream_t s) {
-  const int M = g.B * g.Ho * g.Wo;
-  dim3 grid((M + kDwPixPerBlock - 1) / kDwPixPerBlock, (g.Cout + 127) / 128, n_jobs);
-  LaunchScope scope(AIQ_KERNEL_DEPTHWISE, s, 18.0 * M * g.Cout * n_jobs,
-                    weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W + (double)M * g.Cout));
-  depthwise3x3_kernel<<<grid, 256, 0, s>>>(g, jobs_dev);
+  const int M = g.B * (g.Ho + 2) * g.Wo;
+  dim3 grid((M + kDwPixPerBlock - 1) / kDwPixPerBlock, (g.Cs_out + 127) / 128, n_jobs);
+  LaunchScope scope(AIQ_KERNEL_DEPTHWISE, s, 18.0 * g.B * g.Ho * g.Wo * g.Cout * n_jobs,
+                    weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
+                                                   (double)g.B * g.Ho * g.Wo * g.Cout));
+  if (g.act_format == ACT_SPLIT) depthwise3x3_kernel<ACT_SPLIT><<<grid, 256, 0, s>>>(g, jobs_dev);
+  else depthwise3x3_kernel<ACT_F32><<<grid, 256, 0, s>>>(g, jobs_dev);
   AIQ_LAUNCH_CHECK("depthwise3x3");
   return AIQ_OK;
 }
 
-aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int HW, int C, cudaStream_t s) {
+aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int H, int W, int C, int act_format,
+                            cudaStream_t s) {
   int threads = C >= 256 ? 256 : (C >= 128 ? 128 : 64);
-  LaunchScope scope(AIQ_KERNEL_POOL, s, (double)n_jobs * B * HW * C, 4.0 * n_jobs * B * ((double)HW * C + C));
-  avgpool_kernel<<<dim3(B, 1, n_jobs), threads, 0, s>>>(jobs_dev, HW, C);
+  LaunchScope scope(AIQ_KERNEL_POOL, s, (double)n_jobs * B * H * W * C,
+                    4.0 * n_jobs * B * ((double)H * W * C + C));
+  if (act_format == ACT_SPLIT)
+    avgpool_kernel<ACT_SPLIT><<<dim3(B, 1, n_jobs), threads, 0, s>>>(jobs_dev, H, W, C, padded_channels(C));
+  else
+    avgpool_kernel<ACT_F32><<<dim3(B, 1, n_jobs), threads, 0, s>>>(jobs_dev, H, W, C, padded_channels(C));
   AIQ_LAUNCH_CHECK("avgpool");
   return AIQ_OK;
 }

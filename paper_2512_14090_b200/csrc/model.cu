@@ -21,6 +21,7 @@ static thread_local char t_err[512] = "";
 static thread_local int64_t t_launches = 0, t_layer_evals = 0, t_layer_evals_unshared = 0;
 static int g_opt_chunk = 0;
 static int g_opt_share = 1;
+static int g_opt_path = AIQ_PATH_AUTO;
 
 aiq_status_t set_error(aiq_status_t status, const char* fmt, ...) {
   va_list ap;
@@ -94,7 +95,7 @@ static inline int bits_index(int bits) { return bits == 4 ? 0 : bits == 8 ? 1 : 
 struct LayerInfo {
   aiq_layer_desc_t d;
   int K, Hi, Wi, Ho, Wo;
-  size_t out_elems;        // per image
+  size_t out_bytes;        // per image, split format (fc: float32 logits)
   float* Wf;
   float* bias;
   uint8_t* packed[4];
@@ -106,9 +107,10 @@ struct aiq_model {
   std::vector<LayerInfo> layers;
   int in_c, in_h, in_w;
   std::vector<int> order;            // execution order (every layer after its operands)
-  std::vector<size_t> slot_elems;    // per-image capacity of each activation slot
+  std::vector<size_t> slot_bytes;    // per-image capacity of each activation slot
   void* dev_mem;
   size_t dev_bytes;
+  int act_format;                    // ACT_F32 or ACT_SPLIT (see common.cuh)
 };
 
 namespace aiq {
@@ -176,14 +178,14 @@ static aiq_status_t infer_shapes(const aiq_arch_desc_t* arch, std::vector<LayerI
     if (cin_avail != d.cin) return set_error(AIQ_ERR_SHAPE, "layer %d: cin %d but its input has %d channels", i, d.cin, cin_avail);
     li.Hi = hi; li.Wi = wi;
     if (d.kind == AIQ_LAYER_FC) {
-      li.K = d.cin; li.Hi = 1; li.Wi = 1; li.Ho = 1; li.Wo = 1; li.out_elems = d.cout;   // reads the pooled vector
+      li.K = d.cin; li.Hi = 1; li.Wi = 1; li.Ho = 1; li.Wo = 1; li.out_bytes = (size_t)d.cout * 4;   // reads the pooled vector
       continue;
     }
     li.Ho = (hi + 2 * d.pad - d.ksize) / d.stride + 1;
     li.Wo = (wi + 2 * d.pad - d.ksize) / d.stride + 1;
     if (li.Ho <= 0 || li.Wo <= 0) return set_error(AIQ_ERR_SHAPE, "layer %d: empty output", i);
     li.K = (d.kind == AIQ_LAYER_DEPTHWISE ? 1 : d.cin) * d.ksize * d.ksize;
-    li.out_elems = (size_t)d.cout * li.Ho * li.Wo;
+    li.out_bytes = split_image_bytes(li.Ho, li.Wo, d.cout);
     if (d.residual >= 0) {
       const LayerInfo& r = L[d.residual];
       if (r.d.kind == AIQ_LAYER_FC || r.d.cout != d.cout || r.Ho != li.Ho || r.Wo != li.Wo)
@@ -203,7 +205,7 @@ static void assign_slots(aiq_model* m) {
     if (d.residual >= 0) last_use[d.residual] = std::max(last_use[d.residual], pos[l]);
   }
   std::vector<int> owner;   // layer currently held by each slot, -1 = free
-  m->slot_elems.clear();
+  m->slot_bytes.clear();
   for (int i = 0; i < n; ++i) {
     const int l = m->order[i];
     LayerInfo& li = m->layers[l];
@@ -211,10 +213,10 @@ static void assign_slots(aiq_model* m) {
     else {
       int s = -1;
       for (size_t k = 0; k < owner.size(); ++k) if (owner[k] < 0) { s = (int)k; break; }
-      if (s < 0) { s = (int)owner.size(); owner.push_back(-1); m->slot_elems.push_back(0); }
+      if (s < 0) { s = (int)owner.size(); owner.push_back(-1); m->slot_bytes.push_back(0); }
       owner[s] = l;
       li.slot = s;
-      m->slot_elems[s] = std::max(m->slot_elems[s], li.out_elems);
+      m->slot_bytes[s] = std::max(m->slot_bytes[s], li.out_bytes);
     }
     for (size_t k = 0; k < owner.size(); ++k)
       if (owner[k] >= 0 && last_use[owner[k]] <= i && owner[k] != l) owner[k] = -1;
@@ -279,6 +281,7 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
   if (st != AIQ_OK) { delete m; return st; }
   m->in_c = arch->in_c; m->in_h = arch->in_h; m->in_w = arch->in_w;
   m->dev_mem = dev_mem; m->dev_bytes = dev_bytes;
+  m->act_format = (g_opt_path == AIQ_PATH_TENSOR) ? ACT_SPLIT : ACT_F32;
   assign_slots(m);
   cudaStream_t stream = (cudaStream_t)stream_;
   uint8_t* base = static_cast<uint8_t*>(dev_mem);
@@ -391,7 +394,7 @@ static WsLayout ws_layout(const aiq_model* m, int B, int S) {
   const LayerInfo& fc = m->layers.back();
   w.pooled_off = take((size_t)S * B * fc.d.cin * 4);
   w.logits_off = take((size_t)S * B * fc.d.cout * 4);
-  for (size_t e : m->slot_elems) w.slot_off.push_back(take((size_t)S * B * e * 4));
+  for (size_t e : m->slot_bytes) w.slot_off.push_back(take((size_t)S * B * e));
   w.total = off;
   return w;
 }
@@ -428,9 +431,9 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
   plan.lp.assign(n, LayerPlan());
   plan.jobs.clear();
   std::vector<std::vector<int>> ver(n, std::vector<int>(S, 0));   // ver[l][s]
-  auto slot_ptr = [&](int layer, int version) -> float* {
+  auto slot_ptr = [&](int layer, int version) -> uint8_t* {
     const LayerInfo& li = m->layers[layer];
-    return reinterpret_cast<float*>(ws + wl.slot_off[li.slot]) + (size_t)version * B * li.out_elems;
+    return ws + wl.slot_off[li.slot] + (size_t)version * B * li.out_bytes;
   };
   for (int l : m->order) {
     const LayerInfo& li = m->layers[l];
@@ -465,6 +468,7 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
         j.in = li.d.input >= 0 ? slot_ptr(li.d.input, std::get<1>(keys[v])) : nullptr;
         j.res = li.d.residual >= 0 ? slot_ptr(li.d.residual, std::get<2>(keys[v])) : nullptr;
         j.out = slot_ptr(l, v);
+        j.in_version = li.d.input >= 0 ? std::get<1>(keys[v]) : 0;
         j.w = li.packed[bi];
         j.scale = li.scales[bi];
         j.bias = li.bias;
@@ -540,7 +544,7 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
     aiq_status_t st;
     if (li.d.kind == AIQ_LAYER_FC) {
       const LayerInfo& src = m->layers[li.d.input];
-      st = launch_avgpool(jobs_dev + lp.pool_first, lp.n_pool, B, src.Ho * src.Wo, src.d.cout, stream);
+      st = launch_avgpool(jobs_dev + lp.pool_first, lp.n_pool, B, src.Ho, src.Wo, src.d.cout, m->act_format, stream);
       if (st != AIQ_OK) return st;
       for (size_t gi = 0; gi < lp.bit_groups.size(); ++gi) {
         const size_t first = lp.job_first + lp.bit_groups[gi].first;
@@ -557,11 +561,9 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
     ConvGeom g = {};
     g.B = B; g.H = li.Hi; g.W = li.Wi; g.Cin = li.d.cin; g.Ho = li.Ho; g.Wo = li.Wo; g.Cout = li.d.cout;
     g.ks = li.d.ksize; g.stride = li.d.stride; g.pad = li.d.pad; g.act = li.d.act; g.K = li.K;
-    if (li.d.input < 0) {          // network input: NCHW
-      g.in_sb = (long long)li.d.cin * li.Hi * li.Wi; g.in_sc = (long long)li.Hi * li.Wi; g.in_sy = li.Wi; g.in_sx = 1;
-    } else {                       // internal activations: NHWC
-      g.in_sb = (long long)li.Hi * li.Wi * li.d.cin; g.in_sy = (long long)li.Wi * li.d.cin; g.in_sx = li.d.cin; g.in_sc = 1;
-    }
+    g.Cs_in = padded_channels(li.d.cin); g.Cs_out = padded_channels(li.d.cout);
+    g.in_is_nchw = li.d.input < 0 ? 1 : 0;          // the network input is float32 NCHW
+    g.act_format = m->act_format;
     if (li.d.kind == AIQ_LAYER_DEPTHWISE) st = launch_depthwise(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, lp.weight_bytes, stream);
     else st = launch_conv(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, lp.weight_bytes, stream);
     if (st != AIQ_OK) return st;
@@ -579,6 +581,10 @@ extern "C" size_t aiq_workspace_bytes(const aiq_model_t* model, int max_batch, i
 extern "C" void aiq_set_eval_options(int chunk, int share_prefix) {
   aiq::g_opt_chunk = chunk > 0 ? chunk : 0;
   aiq::g_opt_share = share_prefix ? 1 : 0;
+}
+
+extern "C" void aiq_set_compute_path(int path) {
+  aiq::g_opt_path = (path == AIQ_PATH_FP32 || path == AIQ_PATH_TENSOR) ? path : AIQ_PATH_AUTO;
 }
 
 extern "C" void aiq_last_call_stats(int64_t* kernel_launches, int64_t* layer_evals, int64_t* layer_evals_unshared) {

@@ -63,7 +63,7 @@ qlinear_kernel(LayerJob single, const LayerJob* __restrict__ jobs, int N, int K,
   const int Kpad = (K + 31) / 32 * 32;
   const size_t rb = (size_t)Kpad * BITS / 8;
   const int n_chunks = Kpad / E;
-  const float* __restrict__ x = job.in;
+  const float* __restrict__ x = static_cast<const float*>(job.in);
   const bool xvec = ((K & 3) == 0) && ((((uintptr_t)x) & 15) == 0);
 
   float acc[kRowsPerWarp][MT];
@@ -134,7 +134,7 @@ qlinear_kernel(LayerJob single, const LayerJob* __restrict__ jobs, int N, int K,
       const float b = job.bias ? job.bias[n] : 0.0f;
 #pragma unroll
       for (int m = 0; m < MT; ++m)
-        if (m0 + m < M) job.out[(size_t)(m0 + m) * N + n] = fmaf(acc[r][m], s, b);
+        if (m0 + m < M) static_cast<float*>(job.out)[(size_t)(m0 + m) * N + n] = fmaf(acc[r][m], s, b);
     }
   }
 }

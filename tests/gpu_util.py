@@ -30,3 +30,28 @@ def assert_preds_match(preds, opreds, omargins, what=""):
     decided = omargins > 1e-2
     bad = (preds != opreds) & decided
     assert not bad.any(), f"{what}: {bad.sum()} arg-max mismatches at decided margins"
+
+
+def assert_logits_close_tensor(got, ref, what=""):
+    """|delta| <= 2e-2 * max|logit|: the tolerance of a bf16 tensor-core path."""
+    assert np.all(np.isfinite(got)), what
+    err = np.abs(got.astype(np.float64) - ref.astype(np.float64)).max()
+    bound = 2e-2 * np.abs(ref.astype(np.float64)).max()
+    assert err <= bound, f"{what}: max abs error {err:.3e} > {bound:.3e}"
+    return err
+
+
+class compute_path:
+    """Context manager: models created inside use the given compute path."""
+
+    def __init__(self, name):
+        self.name = name
+
+    def __enter__(self):
+        b = binding()
+        b.aiq_set_compute_path({"auto": b.PATH_AUTO, "fp32": b.PATH_FP32, "tensor": b.PATH_TENSOR}[self.name])
+        return self
+
+    def __exit__(self, *exc):
+        binding().aiq_set_compute_path(binding().PATH_AUTO)
+        return False

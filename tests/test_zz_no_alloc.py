@@ -36,7 +36,7 @@ def test_static_workspace_matches_forward_on_two_calls_in_a_row():
     model = aiq.Model(arch, gen_model(arch, 1234))
     assert model.aiq_workspace_bytes(24, 1) <= aiq.STATIC_WORKSPACE_BYTES
     # the limit the header documents for this network
-    assert model.aiq_workspace_bytes(42, 1) <= aiq.STATIC_WORKSPACE_BYTES < model.aiq_workspace_bytes(43, 1)
+    assert model.aiq_workspace_bytes(40, 1) <= aiq.STATIC_WORKSPACE_BYTES < model.aiq_workspace_bytes(41, 1)
     cases = [(gen_random_scheme(model.n_layers, 42), gen_images(24, 3, 32, 32, 5678)),
              (gen_random_scheme(model.n_layers, 43), gen_images(7, 3, 32, 32, 5680))]
     _compare_two_calls(aiq, model, cases)
