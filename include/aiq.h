@@ -166,6 +166,10 @@ aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_layer_weigh
 void aiq_model_destroy(aiq_model_t* model);
 int aiq_model_num_layers(const aiq_model_t* model);   /* L, the scheme length; -1 if NULL */
 int aiq_model_num_classes(const aiq_model_t* model);  /* cout of the last layer           */
+/* Synchronises `stream` and reports a device-side failure recorded by an earlier
+ * asynchronous call on this model (AIQ_ERR_TIMEOUT: a bounded wait inside a kernel expired;
+ * the outputs of that call are then invalid).  AIQ_OK otherwise.  Clears the record. */
+aiq_status_t aiq_model_status(const aiq_model_t* model, void* stream);
 
 /* Device views into the model memory, for inspection: folded weights Wf [cout][K] and bias
  * [cout] of `layer`; packed rows and scales of (`layer`, `bits`) in the layout of
@@ -293,7 +297,8 @@ enum {
   AIQ_KERNEL_DEPTHWISE = 4,
   AIQ_KERNEL_POOL = 5,
   AIQ_KERNEL_ARGMAX = 6,
-  AIQ_KERNEL_KINDS = 7
+  AIQ_KERNEL_CONV_TC = 7,   /* tensor-core convolution */
+  AIQ_KERNEL_KINDS = 8
 };
 typedef struct aiq_kernel_profile {
   int64_t launches;

@@ -26,14 +26,14 @@ EXPORTS = [
     "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
     "aiq_eval_schemes", "aiq_set_eval_options", "aiq_last_call_stats", "aiq_scheme_ai",
     "aiq_profile_start", "aiq_profile_stop", "aiq_forward_static",
-    "aiq_set_compute_path",
+    "aiq_set_compute_path", "aiq_model_status",
 ]
 
 PATH_AUTO, PATH_FP32, PATH_TENSOR = 0, 1, 2
 
 STATIC_WORKSPACE_BYTES = 8 * 1024 * 1024
 
-KERNEL_KINDS = ["fold", "quantize", "qlinear", "conv", "depthwise", "pool", "argmax"]
+KERNEL_KINDS = ["fold", "quantize", "qlinear", "conv", "depthwise", "pool", "argmax", "conv_tc"]
 
 
 class AiqError(RuntimeError):
@@ -110,6 +110,8 @@ def _load():
                                   C.POINTER(C.c_double)]
     lib.aiq_forward_static.restype = i32
     lib.aiq_forward_static.argtypes = [vp, vp, vp, i32, vp, vp]
+    lib.aiq_model_status.restype = i32
+    lib.aiq_model_status.argtypes = [vp, vp]
     lib.aiq_set_compute_path.restype = None
     lib.aiq_set_compute_path.argtypes = [i32]
     lib.aiq_profile_start.restype = i32
@@ -252,7 +254,7 @@ class Model:
         self._ws = None
 
     def close(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and lib is not None:      # lib is None at interpreter exit
             lib.aiq_model_destroy(self.handle)
             self.handle = None
 
@@ -330,6 +332,9 @@ class Model:
                                     _host(acc), _host(counts), _dev(preds), _dev(ws), ws.numel(),
                                     _stream(stream)))
         return acc, counts
+
+    def aiq_model_status(self, stream=None):
+        _check(lib.aiq_model_status(self.handle, _stream(stream)))
 
     def aiq_scheme_ai(self, scheme_bits, ai_batch=1):
         scheme = np.ascontiguousarray(scheme_bits, dtype=np.uint8)

@@ -130,6 +130,13 @@ aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs
                          const float* net_input, double weight_bytes, cudaStream_t s);
 aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
                               const float* net_input, double weight_bytes, cudaStream_t s);
+// Tensor-core convolution (conv_tc.cu).  `map` points to a 128-byte CUtensorMap over the input
+// slot: dims (2*Cs, W, batch_capacity*(H+2), versions).  Jobs must have 4- or 8-bit weights.
+bool conv_tc_eligible(const ConvGeom& g);
+aiq_status_t conv_tc_encode_map(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
+                                void* map_out);
+aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
+                            int32_t* error_flag, double weight_bytes, cudaStream_t s);
 // pooled[b][c] = mean over the H x W interior of a split tensor, per job (in -> out float32 [B][C])
 aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int H, int W, int C, int act_format,
                             cudaStream_t s);

@@ -1,0 +1,554 @@
+// Dense 3x3 / 1x1 convolution on the 5th-generation tensor cores (tcgen05) of sm_100a.
+//
+//   out[p][n] = act( s_n * sum_{tap,c} code[n][c][tap] * x[p @ tap][c] + b_n + res[p][n] )
+//
+// The activations are stored as the sum of two bfloat16 per element (ACT_SPLIT), one pixel
+// = [hi(C) | lo(C)], rows padded physically (common.cuh).  The implicit GEMM has
+//   M = 128 output pixels  (a tile of 16 padded rows x 8 columns),
+//   N = Cout (16 / 32 / 64),
+//   K = taps x 2C: the hi and the lo half of a pixel are two K-slices that meet the same
+//       weights, so x = hi + lo costs two MMAs and loses nothing in the products
+//       (integer codes |q| <= 128 are exact in bfloat16; accumulation is float32 in TMEM).
+//
+// Data movement per tile: for each horizontal tap t the producer warp issues one TMA load of
+// an 18-row x 8-column x 2C box (rows j0-1 .. j0+16, columns c0+t-1 .. c0+t+6; out-of-range
+// columns and rows arrive as zeros = the convolution's padding).  The box lands as 18 groups
+// of 8 pixel rows in the canonical K-major swizzled layout, so the three vertical taps are
+// the same buffer addressed one group further down: 3 loads feed 9 taps.  Weights arrive
+// packed (4 or 8 bits) by one bulk copy per CTA and are expanded to bfloat16 in shared
+// memory, in the swizzled layout the MMA reads.  One thread issues the MMAs; four warps
+// drain the float32 accumulators from tensor memory, apply scale, bias, residual and
+// activation, split the result into two bfloat16 and store it.  Two accumulator buffers let
+// the epilogue of a tile overlap the MMAs of the next.  Stride-2 layers are computed at
+// input resolution and the epilogue keeps the even positions.
+//
+// Every wait is bounded: when a wait gives up the CTA raises an error word in global
+// memory, every role falls through, tensor memory is released and the kernel returns.
+#include "common.cuh"
+
+#include <cuda.h>
+
+namespace aiq {
+
+namespace {
+
+constexpr int kTcThreads = 192;            // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
+constexpr int kRowsPerTile = 16;           // padded rows per tile
+constexpr int kColsPerTile = 8;
+constexpr int kBoxRows = kRowsPerTile + 2;
+constexpr uint64_t kWaitLimitNs = 2000ull * 1000ull * 1000ull;   // every wait gives up after 2 s
+constexpr uint32_t kSpinLimit = 1u << 30;                         // and after this many polls at the latest
+
+struct TcParams {
+  int B, H, W;            // input geometry (output = input for stride 1, halved for stride 2)
+  int Ho, Wo;
+  int ks, stride, act;
+  int n_stages;
+  int K;                  // Cin * ks * ks (packed row length in elements)
+  int32_t* error_flag;    // device word, set to 1 when a bounded wait expired
+};
+
+// ---- PTX wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the abort flag) when the limit is hit or another
+// role has already aborted.
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* error_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 63u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) break;
+    }
+  }
+  *abort_flag = 1;
+  if (error_flag) atomicExch(error_flag, 1);
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, K-major, swizzled: rows of `swizzle bytes` pitch in groups
+// of 8; SBO = distance between groups.  layout: 2 = 128B, 4 = 64B, 6 = 32B swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t sbo_bytes, uint32_t layout) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+  d |= (uint64_t)1 << 16;                               // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;                               // descriptor version of sm_100
+  d |= (uint64_t)layout << 61;
+  return d;
+}
+
+// 16-byte-unit XOR swizzle of a byte offset inside a tile whose base is aligned to the pattern
+__device__ __forceinline__ uint32_t swizzle_off(uint32_t off, uint32_t mask) {
+  return off ^ (((off >> 7) & mask) << 4);
+}
+
+template <int CS, int N>
+struct TcLayout {
+  static constexpr int PIX_BYTES = 4 * CS;                       // [hi | lo] bfloat16
+  static constexpr int CW_BYTES = PIX_BYTES < 128 ? PIX_BYTES : 128;   // bytes per pixel row of one box
+  static constexpr int CHUNKS = PIX_BYTES / CW_BYTES;
+  static constexpr int GROUP_BYTES = 8 * CW_BYTES;
+  static constexpr int CHUNK_BYTES = kBoxRows * GROUP_BYTES;
+  static constexpr int STAGE_BYTES = CHUNKS * CHUNK_BYTES;
+  static constexpr uint32_t A_LAYOUT = CW_BYTES == 128 ? 2u : 4u;
+  static constexpr int W_ROW_BYTES = 2 * CS;                     // one weight row of one tap
+  static constexpr uint32_t W_LAYOUT = W_ROW_BYTES == 128 ? 2u : (W_ROW_BYTES == 64 ? 4u : 6u);
+  static constexpr uint32_t W_SWZ_MASK = W_ROW_BYTES == 128 ? 7u : (W_ROW_BYTES == 64 ? 3u : 1u);
+  static constexpr int W_TAP_BYTES = N * W_ROW_BYTES;
+  static constexpr int TMEM_COLS = 2 * N < 32 ? 32 : 2 * N;      // two accumulator buffers
+};
+
+// Offsets of the dynamic shared memory regions (base aligned to 1024 bytes)
+template <int CS, int N>
+struct TcSmem {
+  using L = TcLayout<CS, N>;
+  static __host__ __device__ constexpr int ring(int) { return 0; }
+  static __host__ __device__ constexpr int weights(int stages) { return stages * L::STAGE_BYTES; }
+  static __host__ __device__ constexpr int scale(int stages, int taps) { return weights(stages) + taps * L::W_TAP_BYTES; }
+  static __host__ __device__ constexpr int bias(int stages, int taps) { return scale(stages, taps) + N * 4; }
+  static __host__ __device__ constexpr int bars(int stages, int taps) { return bias(stages, taps) + N * 4; }
+  // barriers: full[stages], empty[stages], acc_full[2], acc_empty[2], wbar; then tmem ptr, abort flag
+  static __host__ __device__ constexpr int total(int stages, int taps) { return bars(stages, taps) + (2 * stages + 5) * 8 + 16; }
+};
+
+template <int CS, int N>
+__global__ void __launch_bounds__(kTcThreads, 1)
+conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const LayerJob* __restrict__ jobs) {
+  using L = TcLayout<CS, N>;
+  using S = TcSmem<CS, N>;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  // the runtime only promises 16-byte alignment of dynamic shared memory: align by hand
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const LayerJob job = jobs[blockIdx.y];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int taps = p.ks * p.ks;
+  const int stages = p.n_stages;
+
+  uint8_t* ring = smem;
+  uint8_t* wsm = smem + S::weights(stages);
+  float* s_scale = reinterpret_cast<float*>(smem + S::scale(stages, taps));
+  float* s_bias = reinterpret_cast<float*>(smem + S::bias(stages, taps));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::bars(stages, taps));
+  const uint32_t bar_full = smem_u32(bars);
+  const uint32_t bar_empty = bar_full + 8 * stages;
+  const uint32_t bar_acc_full = bar_empty + 8 * stages;
+  const uint32_t bar_acc_empty = bar_acc_full + 16;
+  const uint32_t bar_w = bar_acc_empty + 16;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * stages + 5);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  const int rows_total = p.B * (p.H + 2);
+  const int n_rb = (rows_total + kRowsPerTile - 1) / kRowsPerTile;
+  const int n_cb = p.W / kColsPerTile;
+  const int n_tiles = n_rb * n_cb;
+
+  // ---- set-up -----------------------------------------------------------------------------
+  if (tid == 0) {
+    for (int i = 0; i < stages; ++i) {
+      mbar_init(bar_full + 8 * i, 1);
+      mbar_init(bar_empty + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_acc_full + 8 * i, 1);
+      mbar_init(bar_acc_empty + 8 * i, 4);     // one arrival per epilogue warp
+    }
+    mbar_init(bar_w, 1);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tmem_alloc(smem_u32(s_tmem), L::TMEM_COLS);
+    tmem_relinquish();
+  }
+  // packed weights: one bulk copy into the (still unused) ring, then expansion to bfloat16
+  const int kpad = (p.K + 31) / 32 * 32;
+  const uint32_t wrow_bytes = (uint32_t)kpad * job.bits / 8;
+  const uint32_t packed_bytes = wrow_bytes * N;
+  if (tid == 0) {
+    mbar_expect_tx(bar_w, packed_bytes);
+    bulk_load(smem_u32(ring), job.w, packed_bytes, bar_w);
+  }
+  for (int i = tid; i < N; i += kTcThreads) {
+    s_scale[i] = job.scale[i];
+    s_bias[i] = job.bias[i];
+  }
+  bool alive = mbar_wait(bar_w, 0, s_abort, p.error_flag);
+  if (alive) {
+    const int units_per_row = CS / 8;                         // 16-byte units of one weight row
+    const int total_units = taps * N * units_per_row;
+    for (int u = tid; u < total_units; u += kTcThreads) {
+      const int c8 = u % units_per_row;
+      const int n = (u / units_per_row) % N;
+      const int tap = u / (units_per_row * N);
+      const uint8_t* row = ring + (size_t)n * wrow_bytes;
+      uint32_t packed[4];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int k = (c8 * 8 + j) * taps + tap;             // element index in the (c, r, t) ordered row
+        int code;
+        if (job.bits == 8) {
+          code = (int)(int8_t)row[k];
+        } else {
+          const int byte = row[k >> 1];
+          const int nib = (k & 1) ? (byte >> 4) : (byte & 0xF);
+          code = (nib ^ 8) - 8;
+        }
+        const uint32_t h = (uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code));
+        if (j & 1) packed[j >> 1] |= h << 16; else packed[j >> 1] = h;
+      }
+      const uint32_t off = swizzle_off((uint32_t)(n * L::W_ROW_BYTES + c8 * 16), L::W_SWZ_MASK);
+      *reinterpret_cast<uint4*>(wsm + (size_t)tap * L::W_TAP_BYTES + off) =
+          make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    }
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // expanded weights -> visible to the MMA
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  alive = alive && (*s_abort == 0);            // the same answer in every thread
+
+  // ---- roles ------------------------------------------------------------------------------
+  const int t_first = p.ks == 3 ? 0 : 1, t_last = p.ks == 3 ? 2 : 1;
+  if (warp == 0) {
+    if (lane == 0 && alive) {
+      uint32_t stage = 0, phase = 0;
+      uint32_t issued = 0, issued_phase = 0;       // per stage: a load was issued / parity of the last one
+      for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
+        const int rb = tile / n_cb, cb = tile - rb * n_cb;
+        for (int t = t_first; t <= t_last && alive; ++t) {
+          alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+          if (!alive) break;
+          issued |= 1u << stage;
+          issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
+          mbar_expect_tx(bar_full + 8 * stage, L::STAGE_BYTES);
+#pragma unroll
+          for (int ch = 0; ch < L::CHUNKS; ++ch)
+            tma_load_4d(smem_u32(ring) + stage * L::STAGE_BYTES + ch * L::CHUNK_BYTES, &in_map,
+                        bar_full + 8 * stage, ch * 64, cb * kColsPerTile + t - 1, rb * kRowsPerTile - 1,
+                        job.in_version);
+          if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      // copies in flight must land before the CTA exits: wait (bounded) for the last load
+      // of every stage.  On the normal path the consumer has seen them all and this returns
+      // at once; it matters when another role gave up.
+      for (int i = 0; i < stages; ++i)
+        if (issued & (1u << i)) {
+          const uint64_t t0 = global_timer_ns();
+          while (!mbar_try_wait(bar_full + 8 * i, (issued_phase >> i) & 1u) && global_timer_ns() - t0 < kWaitLimitNs) {}
+        }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && alive) {
+      // instruction descriptor: D float32, A and B bfloat16, both K-major, M = 128, N
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
+      uint32_t stage = 0, phase = 0;
+      int it = 0;
+      for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
+        const int buf = it & 1;
+        alive = mbar_wait(bar_acc_empty + 8 * buf, ((it >> 1) & 1) ^ 1u, s_abort, p.error_flag);
+        if (!alive) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * N);
+        uint32_t accumulate = 0;
+        for (int t = t_first; t <= t_last && alive; ++t) {
+          alive = mbar_wait(bar_full + 8 * stage, phase, s_abort, p.error_flag);
+          if (!alive) break;
+          tc_fence_after();
+          const uint32_t a_stage = smem_u32(ring) + stage * L::STAGE_BYTES;
+          for (int r = t_first; r <= t_last; ++r) {
+            const int tap = p.ks == 3 ? r * 3 + t : 0;
+            const uint32_t w_tap = smem_u32(wsm) + tap * L::W_TAP_BYTES;
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+#pragma unroll
+              for (int kk = 0; kk < CS / 16; ++kk) {
+                const int byte = (part * CS + kk * 16) * 2;              // offset inside the pixel
+                const uint32_t a_addr = a_stage + (byte / L::CW_BYTES) * L::CHUNK_BYTES + r * L::GROUP_BYTES +
+                                        (byte % L::CW_BYTES);
+                const uint64_t adesc = smem_desc(a_addr, L::GROUP_BYTES, L::A_LAYOUT);
+                const uint64_t bdesc = smem_desc(w_tap + kk * 32, 8 * L::W_ROW_BYTES, L::W_LAYOUT);
+                umma_bf16(d_tmem, adesc, bdesc, idesc, accumulate);
+                accumulate = 1;
+              }
+            }
+          }
+          umma_commit(bar_empty + 8 * stage);        // the stage is free once these MMAs retire
+          if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+        }
+        if (alive) umma_commit(bar_acc_full + 8 * buf);
+      }
+    }
+  } else {
+    // epilogue: warp q of the four owns TMEM lanes 32q .. 32q+31 (q = warp index mod 4)
+    const int q = warp & 3;
+    const int m = q * 32 + lane;                       // row of the tile: pixel (g, wl)
+    const int g = m >> 3, wl = m & 7;
+    int it = 0;
+    for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
+      const int buf = it & 1;
+      alive = mbar_wait(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);
+      alive = __all_sync(0xffffffffu, alive);     // the tensor-memory loads below need the whole warp
+      if (!alive) break;
+      tc_fence_after();
+      const int rb = tile / n_cb, cb = tile - rb * n_cb;
+      const int j = rb * kRowsPerTile + g;             // padded input row (image, y')
+      const int col = cb * kColsPerTile + wl;
+      const int b = j / (p.H + 2);
+      const int yp = j - b * (p.H + 2);
+      bool store = j < rows_total;
+      bool interior = yp >= 1 && yp <= p.H;
+      size_t out_pixel;
+      if (p.stride == 1) {
+        out_pixel = (size_t)j * p.W + col;
+      } else {
+        // keep even positions; padded border rows map to the output's border rows
+        int oyp;
+        if (yp == 0) oyp = 0;
+        else if (yp == p.H + 1) oyp = p.Ho + 1;
+        else { oyp = ((yp - 1) >> 1) + 1; store = store && (((yp - 1) & 1) == 0); }
+        store = store && ((col & 1) == 0);
+        out_pixel = ((size_t)b * (p.Ho + 2) + oyp) * p.Wo + (col >> 1);
+      }
+      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(job.out) + out_pixel * (2 * N);
+      const __nv_bfloat16* res = job.res ? static_cast<const __nv_bfloat16*>(job.res) + out_pixel * (2 * N) : nullptr;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * N);
+#pragma unroll
+      for (int c0 = 0; c0 < N; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(taddr + c0, v);
+        tmem_ld_wait();
+        if (store) {
+          uint32_t hi[8], lo[8];
+          uint32_t rh[8] = {0, 0, 0, 0, 0, 0, 0, 0}, rl[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+          if (res && interior) {
+            const uint4 a0 = __ldg(reinterpret_cast<const uint4*>(res + c0)), a1 = __ldg(reinterpret_cast<const uint4*>(res + c0) + 1);
+            const uint4 b0 = __ldg(reinterpret_cast<const uint4*>(res + N + c0)), b1 = __ldg(reinterpret_cast<const uint4*>(res + N + c0) + 1);
+            rh[0] = a0.x; rh[1] = a0.y; rh[2] = a0.z; rh[3] = a0.w; rh[4] = a1.x; rh[5] = a1.y; rh[6] = a1.z; rh[7] = a1.w;
+            rl[0] = b0.x; rl[1] = b0.y; rl[2] = b0.z; rl[3] = b0.w; rl[4] = b1.x; rl[5] = b1.y; rl[6] = b1.z; rl[7] = b1.w;
+          }
+#pragma unroll
+          for (int e = 0; e < 16; e += 2) {
+            float u0 = 0.f, u1 = 0.f;
+            if (interior) {
+              u0 = fmaf(__uint_as_float(v[e]), s_scale[c0 + e], s_bias[c0 + e]);
+              u1 = fmaf(__uint_as_float(v[e + 1]), s_scale[c0 + e + 1], s_bias[c0 + e + 1]);
+              // a bfloat16 is the upper half of a float: residual = hi + lo
+              u0 += __uint_as_float(rh[e >> 1] << 16) + __uint_as_float(rl[e >> 1] << 16);
+              u1 += __uint_as_float(rh[e >> 1] & 0xFFFF0000u) + __uint_as_float(rl[e >> 1] & 0xFFFF0000u);
+              u0 = apply_act(u0, p.act);
+              u1 = apply_act(u1, p.act);
+            }
+            __nv_bfloat16 h0, l0, h1, l1;
+            split_bf16(u0, h0, l0);
+            split_bf16(u1, h1, l1);
+            hi[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+            lo[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+          }
+          uint4* oh = reinterpret_cast<uint4*>(out + c0);
+          uint4* ol = reinterpret_cast<uint4*>(out + N + c0);
+          oh[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          oh[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+          ol[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          ol[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+    }
+  }
+
+  // ---- teardown -----------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, L::TMEM_COLS);
+  }
+}
+
+// ---- host side ------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* sym = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(sym);
+  return fn;
+}
+
+template <int CS, int N>
+aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob* jobs_dev, int n_jobs,
+                       int32_t* error_flag, double weight_bytes, cudaStream_t s) {
+  using L = TcLayout<CS, N>;
+  using S = TcSmem<CS, N>;
+  const int taps = g.ks * g.ks;
+  static int smem_limit = 0, n_sms = 0;
+  if (!smem_limit) {
+    int dev = 0;
+    AIQ_CUDA_TRY(cudaGetDevice(&dev));
+    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
+  }
+  // as many ring stages as fit (two tiles in flight = 6), never fewer than 3
+  int stages = 6;
+  while (stages > 3 && S::total(stages, taps) + 1024 > smem_limit) --stages;
+  const int smem_bytes = S::total(stages, taps) + 1024;
+  if (smem_bytes > smem_limit)
+    return set_error(AIQ_ERR_SHAPE, "conv_tc: %d bytes of shared memory needed, %d available", smem_bytes, smem_limit);
+  const int packed = N * (int)row_bytes(g.K, 8);
+  if (packed > stages * L::STAGE_BYTES)
+    return set_error(AIQ_ERR_SHAPE, "conv_tc: packed weights (%d bytes) exceed the staging ring", packed);
+  static bool attr_set = false;
+  if (!attr_set) {
+    AIQ_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<CS, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
+    attr_set = true;
+  }
+  TcParams p = {};
+  p.B = g.B; p.H = g.H; p.W = g.W; p.Ho = g.Ho; p.Wo = g.Wo; p.ks = g.ks; p.stride = g.stride; p.act = g.act;
+  p.n_stages = stages; p.K = g.K; p.error_flag = error_flag;
+  const int rows_total = g.B * (g.H + 2);
+  const int n_tiles = ((rows_total + kRowsPerTile - 1) / kRowsPerTile) * (g.W / kColsPerTile);
+  int ctas = (n_sms + n_jobs - 1) / n_jobs;
+  if (ctas > n_tiles) ctas = n_tiles;
+  if (ctas < 1) ctas = 1;
+  {
+    LaunchScope scope(AIQ_KERNEL_CONV_TC, s,
+                      2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
+                      weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
+                                                     (double)g.B * g.Ho * g.Wo * g.Cout));
+    conv_tc_kernel<CS, N><<<dim3(ctas, n_jobs), kTcThreads, smem_bytes, s>>>(map, p, jobs_dev);
+  }
+  AIQ_LAUNCH_CHECK("conv_tc");
+  return AIQ_OK;
+}
+
+}  // namespace
+
+bool conv_tc_eligible(const ConvGeom& g) {
+  if (g.in_is_nchw || g.act_format != ACT_SPLIT) return false;
+  if (!((g.ks == 3 && g.pad == 1) || (g.ks == 1 && g.pad == 0))) return false;
+  if (g.stride != 1 && g.stride != 2) return false;
+  if (g.Cin != 16 && g.Cin != 32 && g.Cin != 64) return false;
+  if (g.Cout != 16 && g.Cout != 32 && g.Cout != 64) return false;
+  if (g.W % kColsPerTile != 0) return false;
+  if (g.stride == 2 && ((g.H & 1) || (g.W & 1))) return false;
+  return true;
+}
+
+aiq_status_t conv_tc_encode_map(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
+                                void* map_out) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  const cuuint64_t pix_bytes = 4ull * g.Cs_in;
+  const cuuint64_t rows = (cuuint64_t)batch_capacity * (g.H + 2);
+  cuuint64_t dims[4] = {(cuuint64_t)2 * g.Cs_in, (cuuint64_t)g.W, rows, (cuuint64_t)n_versions};
+  cuuint64_t strides[3] = {pix_bytes, pix_bytes * g.W, pix_bytes * g.W * rows};
+  const cuuint32_t inner = pix_bytes < 128 ? (cuuint32_t)(2 * g.Cs_in) : 64u;
+  cuuint32_t box[4] = {inner, (cuuint32_t)kColsPerTile, (cuuint32_t)kBoxRows, 1u};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUtensorMapSwizzle swz = pix_bytes < 128 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
+  CUresult r = enc(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(slot_base),
+                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return AIQ_OK;
+}
+
+aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
+                            int32_t* error_flag, double weight_bytes, cudaStream_t s) {
+  const CUtensorMap& m = *static_cast<const CUtensorMap*>(map);
+#define AIQ_TC_CASE(CS_, N_) \
+  if (g.Cin == CS_ && g.Cout == N_) return launch_tc<CS_, N_>(g, m, jobs_dev, n_jobs, error_flag, weight_bytes, s);
+  AIQ_TC_CASE(16, 16) AIQ_TC_CASE(16, 32) AIQ_TC_CASE(16, 64)
+  AIQ_TC_CASE(32, 16) AIQ_TC_CASE(32, 32) AIQ_TC_CASE(32, 64)
+  AIQ_TC_CASE(64, 16) AIQ_TC_CASE(64, 32) AIQ_TC_CASE(64, 64)
+#undef AIQ_TC_CASE
+  return set_error(AIQ_ERR_SHAPE, "conv_tc: no kernel for Cin=%d Cout=%d", g.Cin, g.Cout);
+}
+
+}  // namespace aiq

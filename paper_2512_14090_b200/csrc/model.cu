@@ -111,6 +111,7 @@ struct aiq_model {
   void* dev_mem;
   size_t dev_bytes;
   int act_format;                    // ACT_F32 or ACT_SPLIT (see common.cuh)
+  int32_t* status_word;              // device word raised by a kernel whose bounded wait expired
 };
 
 namespace aiq {
@@ -193,6 +194,20 @@ static aiq_status_t infer_shapes(const aiq_arch_desc_t* arch, std::vector<LayerI
     }
   }
   return AIQ_OK;
+}
+
+static ConvGeom make_geom(const aiq_model* m, const LayerInfo& li, int B) {
+  ConvGeom g = {};
+  g.B = B; g.H = li.Hi; g.W = li.Wi; g.Cin = li.d.cin; g.Ho = li.Ho; g.Wo = li.Wo; g.Cout = li.d.cout;
+  g.ks = li.d.ksize; g.stride = li.d.stride; g.pad = li.d.pad; g.act = li.d.act; g.K = li.K;
+  g.Cs_in = padded_channels(li.d.cin); g.Cs_out = padded_channels(li.d.cout);
+  g.in_is_nchw = li.d.input < 0 ? 1 : 0;          // the network input is float32 NCHW
+  g.act_format = m->act_format;
+  return g;
+}
+
+static bool layer_on_tensor_cores(const aiq_model* m, const LayerInfo& li) {
+  return li.d.kind == AIQ_LAYER_CONV && conv_tc_eligible(make_geom(m, li, 1));
 }
 
 static void assign_slots(aiq_model* m) {
@@ -281,11 +296,15 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
   if (st != AIQ_OK) { delete m; return st; }
   m->in_c = arch->in_c; m->in_h = arch->in_h; m->in_w = arch->in_w;
   m->dev_mem = dev_mem; m->dev_bytes = dev_bytes;
-  m->act_format = (g_opt_path == AIQ_PATH_TENSOR) ? ACT_SPLIT : ACT_F32;
+  m->act_format = ACT_SPLIT;                      // tentatively, to ask which layers would qualify
+  bool any_tc = false;
+  for (const LayerInfo& li : m->layers) any_tc = any_tc || layer_on_tensor_cores(m, li);
+  m->act_format = (g_opt_path == AIQ_PATH_TENSOR || (g_opt_path == AIQ_PATH_AUTO && any_tc)) ? ACT_SPLIT : ACT_F32;
   assign_slots(m);
   cudaStream_t stream = (cudaStream_t)stream_;
   uint8_t* base = static_cast<uint8_t*>(dev_mem);
   int32_t* flag = reinterpret_cast<int32_t*>(base + lay.flag_off);
+  m->status_word = flag + 1;                      // zeroed with the flag region below
 
   auto fail = [&](aiq_status_t s) { delete m; return s; };
 #define CREATE_TRY(expr)                                                                    \
@@ -341,6 +360,20 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
 }
 
 extern "C" void aiq_model_destroy(aiq_model_t* model) { delete model; }
+extern "C" aiq_status_t aiq_model_status(const aiq_model_t* model, void* stream_) {
+  using namespace aiq;
+  if (!model) return set_error(AIQ_ERR_INVALID_ARG, "aiq_model_status: null model");
+  cudaStream_t stream = (cudaStream_t)stream_;
+  int32_t dev_status = 0;
+  AIQ_CUDA_TRY(cudaMemcpyAsync(&dev_status, model->status_word, 4, cudaMemcpyDeviceToHost, stream));
+  AIQ_CUDA_TRY(cudaStreamSynchronize(stream));
+  if (dev_status) {
+    AIQ_CUDA_TRY(cudaMemsetAsync(model->status_word, 0, 4, stream));
+    return set_error(AIQ_ERR_TIMEOUT, "a bounded wait inside a kernel expired; outputs of that call are invalid");
+  }
+  return AIQ_OK;
+}
+
 extern "C" int aiq_model_num_layers(const aiq_model_t* model) { return model ? (int)model->layers.size() : -1; }
 extern "C" int aiq_model_num_classes(const aiq_model_t* model) { return model ? model->layers.back().d.cout : -1; }
 
@@ -399,9 +432,14 @@ static WsLayout ws_layout(const aiq_model* m, int B, int S) {
   return w;
 }
 
+struct alignas(64) TensorMapBytes { uint8_t b[128]; };   // storage of one CUtensorMap
+
 struct LayerPlan {
   int n_versions = 0;
+  int n_tc = 0;                         // leading jobs that run on the tensor-core kernel
   double weight_bytes = 0.0;            // packed weights + scales + biases over all jobs
+  double weight_bytes_tc = 0.0;
+  TensorMapBytes in_map;                // over the input slot (tensor-core layers)
   size_t job_first = 0;                 // index of the first job record of this layer
   // fc only
   int n_pool = 0;
@@ -461,7 +499,21 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
     plan.versions_total += lp.n_versions;
     if (li.d.kind != AIQ_LAYER_FC) {
       lp.job_first = plan.jobs.size();
-      for (int v = 0; v < lp.n_versions; ++v) {
+      // job order: versions the tensor-core kernel takes (4- / 8-bit weights) first
+      const bool tc_layer = layer_on_tensor_cores(m, li);
+      std::vector<int> vorder;
+      for (int pass = 0; pass < 2; ++pass)
+        for (int v = 0; v < lp.n_versions; ++v) {
+          const bool tc = tc_layer && std::get<0>(keys[v]) <= 8;
+          if (tc == (pass == 0)) vorder.push_back(v);
+        }
+      if (tc_layer) {
+        const LayerInfo& src = m->layers[li.d.input];
+        aiq_status_t st = conv_tc_encode_map(make_geom(m, li, B), ws + wl.slot_off[src.slot], B,
+                                             plan.lp[li.d.input].n_versions, &lp.in_map);
+        if (st != AIQ_OK) return st;
+      }
+      for (int v : vorder) {
         LayerJob j = {};
         const int bits = std::get<0>(keys[v]);
         const int bi = bits_index(bits);
@@ -474,7 +526,9 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
         j.bias = li.bias;
         j.bits = bits;
         plan.jobs.push_back(j);
-        lp.weight_bytes += (double)li.d.cout * (row_bytes(li.K, bits) + 8.0);
+        const double wb = (double)li.d.cout * (row_bytes(li.K, bits) + 8.0);
+        if (tc_layer && bits <= 8) { lp.n_tc++; lp.weight_bytes_tc += wb; }
+        else lp.weight_bytes += wb;
       }
       continue;
     }
@@ -558,15 +612,20 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
       }
       continue;
     }
-    ConvGeom g = {};
-    g.B = B; g.H = li.Hi; g.W = li.Wi; g.Cin = li.d.cin; g.Ho = li.Ho; g.Wo = li.Wo; g.Cout = li.d.cout;
-    g.ks = li.d.ksize; g.stride = li.d.stride; g.pad = li.d.pad; g.act = li.d.act; g.K = li.K;
-    g.Cs_in = padded_channels(li.d.cin); g.Cs_out = padded_channels(li.d.cout);
-    g.in_is_nchw = li.d.input < 0 ? 1 : 0;          // the network input is float32 NCHW
-    g.act_format = m->act_format;
-    if (li.d.kind == AIQ_LAYER_DEPTHWISE) st = launch_depthwise(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, lp.weight_bytes, stream);
-    else st = launch_conv(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, lp.weight_bytes, stream);
-    if (st != AIQ_OK) return st;
+    const ConvGeom g = make_geom(m, li, B);
+    if (li.d.kind == AIQ_LAYER_DEPTHWISE) {
+      st = launch_depthwise(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, lp.weight_bytes, stream);
+      if (st != AIQ_OK) return st;
+      continue;
+    }
+    if (lp.n_tc > 0) {
+      st = launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, m->status_word, lp.weight_bytes_tc, stream);
+      if (st != AIQ_OK) return st;
+    }
+    if (lp.n_versions > lp.n_tc) {
+      st = launch_conv(g, jobs_dev + lp.job_first + lp.n_tc, lp.n_versions - lp.n_tc, x_chunk, lp.weight_bytes, stream);
+      if (st != AIQ_OK) return st;
+    }
   }
   return AIQ_OK;
 }
@@ -679,7 +738,13 @@ extern "C" aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t
         AIQ_CUDA_TRY(cudaMemcpyAsync(preds + (size_t)s * n_images, preds + (size_t)src * n_images,
                                      (size_t)n_images * 4, cudaMemcpyDeviceToDevice, stream));
     }
+  int32_t dev_status = 0;
+  AIQ_CUDA_TRY(cudaMemcpyAsync(&dev_status, model->status_word, 4, cudaMemcpyDeviceToHost, stream));
   AIQ_CUDA_TRY(cudaStreamSynchronize(stream));
+  if (dev_status) {
+    AIQ_CUDA_TRY(cudaMemsetAsync(model->status_word, 0, 4, stream));
+    return set_error(AIQ_ERR_TIMEOUT, "aiq_eval_schemes: a bounded wait inside a kernel expired; results are invalid");
+  }
   for (int s = 0; s < n_schemes; ++s) {
     const int c = counts[first_scheme[plan.final_version[s]]];
     acc[s] = (float)((double)c / (double)n_images);
