@@ -202,7 +202,7 @@ def main():
     x_host = torch.from_numpy(gen_images(N_IMAGES, 3, 32, 32, SEED_IMAGES + rank)).pin_memory()
     x_dev = x_host.to(dev)
     model = aiq.Model(arch, params, device=dev)
-    chunk = args.chunk if args.chunk > 0 else 256
+    chunk = args.chunk if args.chunk > 0 else 1024
     aiq.aiq_set_eval_options(args.chunk, True)
     ws = torch.empty(model.aiq_workspace_bytes(chunk, S), dtype=torch.uint8, device=dev)
 

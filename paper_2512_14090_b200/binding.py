@@ -319,7 +319,7 @@ class Model:
                                       _dev(logits), _stream(stream)))
         return logits
 
-    def aiq_eval_schemes(self, schemes, x, labels, preds=None, workspace=None, chunk=256,
+    def aiq_eval_schemes(self, schemes, x, labels, preds=None, workspace=None, chunk=1024,
                          stream=None):
         schemes = np.ascontiguousarray(schemes, dtype=np.uint8)
         if schemes.ndim != 2 or schemes.shape[1] != self.n_layers:

@@ -36,7 +36,7 @@ constexpr int kTcThreads = 192;            // warp 0: TMA producer, warp 1: MMA 
 constexpr int kRowsPerTile = 16;           // padded rows per tile
 constexpr int kColsPerTile = 8;
 constexpr int kBoxRows = kRowsPerTile + 2;
-constexpr uint64_t kWaitLimitNs = 2000ull * 1000ull * 1000ull;   // every wait gives up after 2 s
+constexpr long long kWaitLimitCycles = 4000ll * 1000ll * 1000ll;  // every wait gives up after ~2 s of SM clocks
 constexpr uint32_t kSpinLimit = 1u << 30;                         // and after this many polls at the latest
 
 struct TcParams {
@@ -73,20 +73,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (and raises the abort flag) when the limit is hit or another
 // role has already aborted.
-__device__ __forceinline__ uint64_t global_timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int32_t* error_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63u) == 63u) {
+    if ((i & 255u) == 255u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) break;
+      if (clock64() - t0 > kWaitLimitCycles) break;
     }
   }
   *abort_flag = 1;
@@ -180,12 +175,13 @@ struct TcSmem {
   static __host__ __device__ constexpr int weights(int stages) { return stages * L::STAGE_BYTES; }
   static __host__ __device__ constexpr int scale(int stages, int taps) { return weights(stages) + taps * L::W_TAP_BYTES; }
   static __host__ __device__ constexpr int bias(int stages, int taps) { return scale(stages, taps) + N * 4; }
-  static __host__ __device__ constexpr int bars(int stages, int taps) { return bias(stages, taps) + N * 4; }
+  static __host__ __device__ constexpr int staging(int stages, int taps) { return (bias(stages, taps) + N * 4 + 127) / 128 * 128; }
+  static __host__ __device__ constexpr int bars(int stages, int taps) { return staging(stages, taps) + 128 * 4 * N; }
   // barriers: full[stages], empty[stages], acc_full[2], acc_empty[2], wbar; then tmem ptr, abort flag
   static __host__ __device__ constexpr int total(int stages, int taps) { return bars(stages, taps) + (2 * stages + 5) * 8 + 16; }
 };
 
-template <int CS, int N>
+template <int CS, int N, int KS>
 __global__ void __launch_bounds__(kTcThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const LayerJob* __restrict__ jobs) {
   using L = TcLayout<CS, N>;
@@ -195,7 +191,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const LayerJob job = jobs[blockIdx.y];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int taps = p.ks * p.ks;
+  constexpr int taps = KS * KS;
+  constexpr int T_FIRST = KS == 3 ? 0 : 1, T_LAST = KS == 3 ? 2 : 1;   // horizontal / vertical tap range
   const int stages = p.n_stages;
 
   uint8_t* ring = smem;
@@ -284,14 +281,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
   alive = alive && (*s_abort == 0);            // the same answer in every thread
 
   // ---- roles ------------------------------------------------------------------------------
-  const int t_first = p.ks == 3 ? 0 : 1, t_last = p.ks == 3 ? 2 : 1;
   if (warp == 0) {
     if (lane == 0 && alive) {
       uint32_t stage = 0, phase = 0;
       uint32_t issued = 0, issued_phase = 0;       // per stage: a load was issued / parity of the last one
       for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
         const int rb = tile / n_cb, cb = tile - rb * n_cb;
-        for (int t = t_first; t <= t_last && alive; ++t) {
+        for (int t = T_FIRST; t <= T_LAST && alive; ++t) {
           alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
           if (!alive) break;
           issued |= 1u << stage;
@@ -310,14 +306,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       // at once; it matters when another role gave up.
       for (int i = 0; i < stages; ++i)
         if (issued & (1u << i)) {
-          const uint64_t t0 = global_timer_ns();
-          while (!mbar_try_wait(bar_full + 8 * i, (issued_phase >> i) & 1u) && global_timer_ns() - t0 < kWaitLimitNs) {}
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_full + 8 * i, (issued_phase >> i) & 1u) && clock64() - t0 < kWaitLimitCycles) {}
         }
     }
   } else if (warp == 1) {
     if (lane == 0 && alive) {
       // instruction descriptor: D float32, A and B bfloat16, both K-major, M = 128, N
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
+      // Shared-memory descriptors differ only in their start address, so the upper words are
+      // constants and every MMA costs one add per operand: the tiles are small (8-32 tensor
+      // cycles each), issue overhead would otherwise dominate.
+      constexpr uint32_t A_HI = (uint32_t)(L::GROUP_BYTES >> 4) | (1u << 14) | (L::A_LAYOUT << 29);
+      constexpr uint32_t B_HI = (uint32_t)((8 * L::W_ROW_BYTES) >> 4) | (1u << 14) | (L::W_LAYOUT << 29);
+      constexpr uint32_t LBO_FIELD = 1u << 16;
+      const uint32_t w_lo0 = (smem_u32(wsm) >> 4) | LBO_FIELD;
       uint32_t stage = 0, phase = 0;
       int it = 0;
       for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
@@ -326,26 +329,26 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
         if (!alive) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * N);
-        uint32_t accumulate = 0;
-        for (int t = t_first; t <= t_last && alive; ++t) {
+#pragma unroll
+        for (int t = T_FIRST; t <= T_LAST; ++t) {
+          if (!alive) break;
           alive = mbar_wait(bar_full + 8 * stage, phase, s_abort, p.error_flag);
           if (!alive) break;
           tc_fence_after();
-          const uint32_t a_stage = smem_u32(ring) + stage * L::STAGE_BYTES;
-          for (int r = t_first; r <= t_last; ++r) {
-            const int tap = p.ks == 3 ? r * 3 + t : 0;
-            const uint32_t w_tap = smem_u32(wsm) + tap * L::W_TAP_BYTES;
+          const uint32_t a_lo0 = ((smem_u32(ring) + stage * L::STAGE_BYTES) >> 4) | LBO_FIELD;
+#pragma unroll
+          for (int r = T_FIRST; r <= T_LAST; ++r) {
+            const int tap = KS == 3 ? r * 3 + t : 0;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
 #pragma unroll
               for (int kk = 0; kk < CS / 16; ++kk) {
                 const int byte = (part * CS + kk * 16) * 2;              // offset inside the pixel
-                const uint32_t a_addr = a_stage + (byte / L::CW_BYTES) * L::CHUNK_BYTES + r * L::GROUP_BYTES +
-                                        (byte % L::CW_BYTES);
-                const uint64_t adesc = smem_desc(a_addr, L::GROUP_BYTES, L::A_LAYOUT);
-                const uint64_t bdesc = smem_desc(w_tap + kk * 32, 8 * L::W_ROW_BYTES, L::W_LAYOUT);
+                const uint32_t a_off = (byte / L::CW_BYTES) * L::CHUNK_BYTES + r * L::GROUP_BYTES + (byte % L::CW_BYTES);
+                const uint64_t adesc = ((uint64_t)A_HI << 32) | (uint64_t)(a_lo0 + (a_off >> 4));
+                const uint64_t bdesc = ((uint64_t)B_HI << 32) | (uint64_t)(w_lo0 + ((tap * L::W_TAP_BYTES + kk * 32) >> 4));
+                const uint32_t accumulate = (t == T_FIRST && r == T_FIRST && part == 0 && kk == 0) ? 0u : 1u;
                 umma_bf16(d_tmem, adesc, bdesc, idesc, accumulate);
-                accumulate = 1;
               }
             }
           }
@@ -356,82 +359,140 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       }
     }
   } else {
-    // epilogue: warp q of the four owns TMEM lanes 32q .. 32q+31 (q = warp index mod 4)
+    // Epilogue: warp q of the four owns TMEM lanes 32q .. 32q+31 (q = warp index mod 4), i.e.
+    // tile rows 4q .. 4q+3 (8 pixels each).  A lane owns one pixel for the arithmetic, but a
+    // pixel is only 4N bytes, so per-lane global accesses would touch 32 cache lines per
+    // instruction.  Instead each warp stages its 32 pixels in shared memory: the residual rows
+    // are fetched into the staging buffer with coalesced 16-byte accesses *before* the
+    // accumulator is waited for, the result overwrites them in place, and the finished rows
+    // leave with coalesced stores (a row of 8 pixels is 32N contiguous bytes).  16-byte units
+    // are XOR-swizzled so that both access patterns are free of bank conflicts.
     const int q = warp & 3;
     const int m = q * 32 + lane;                       // row of the tile: pixel (g, wl)
     const int g = m >> 3, wl = m & 7;
+    constexpr int PIXB = 4 * N;                        // bytes of one output pixel
+    constexpr int UNITS = PIXB / 16;                   // 16-byte units per pixel (4, 8, 16)
+    constexpr int KEY_SHIFT = PIXB < 128 ? 1 : 0;      // N = 16: two pixels share a 128-byte window
+    constexpr int KEY_MASK = (UNITS < 8 ? UNITS : 8) - 1;
+    uint8_t* stg = smem + S::staging(stages, taps) + q * 32 * PIXB;
+    uint8_t* my_row = stg + lane * PIXB;
+    const int my_key = (lane >> KEY_SHIFT) & KEY_MASK;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
       const int buf = it & 1;
+      const int rb = tile / n_cb, cb = tile - rb * n_cb;
+      const bool coalesced = p.stride == 1;
+      // (1) residual rows -> staging (stride-1 layers; only they have a residual)
+      if (coalesced && job.res) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int jr = rb * kRowsPerTile + q * 4 + i;
+          if (jr < rows_total) {
+            const uint4* src = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(job.res) +
+                                                              ((size_t)jr * p.W + cb * kColsPerTile) * PIXB);
+#pragma unroll
+            for (int u = lane; u < 8 * UNITS; u += 32) {
+              const int pl = i * 8 + u / UNITS, uu = u % UNITS;
+              *reinterpret_cast<uint4*>(stg + pl * PIXB + ((uu ^ ((pl >> KEY_SHIFT) & KEY_MASK)) << 4)) = __ldg(src + u);
+            }
+          }
+        }
+        __syncwarp();
+      }
       alive = mbar_wait(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);
       alive = __all_sync(0xffffffffu, alive);     // the tensor-memory loads below need the whole warp
       if (!alive) break;
       tc_fence_after();
-      const int rb = tile / n_cb, cb = tile - rb * n_cb;
       const int j = rb * kRowsPerTile + g;             // padded input row (image, y')
       const int col = cb * kColsPerTile + wl;
       const int b = j / (p.H + 2);
       const int yp = j - b * (p.H + 2);
-      bool store = j < rows_total;
-      bool interior = yp >= 1 && yp <= p.H;
-      size_t out_pixel;
-      if (p.stride == 1) {
-        out_pixel = (size_t)j * p.W + col;
-      } else {
-        // keep even positions; padded border rows map to the output's border rows
+      const bool interior = yp >= 1 && yp <= p.H;
+      // stride 2: keep even positions; padded border rows map to the output's border rows
+      bool store2 = false;
+      size_t out_pixel2 = 0;
+      if (!coalesced) {
         int oyp;
+        store2 = j < rows_total && ((col & 1) == 0);
         if (yp == 0) oyp = 0;
         else if (yp == p.H + 1) oyp = p.Ho + 1;
-        else { oyp = ((yp - 1) >> 1) + 1; store = store && (((yp - 1) & 1) == 0); }
-        store = store && ((col & 1) == 0);
-        out_pixel = ((size_t)b * (p.Ho + 2) + oyp) * p.Wo + (col >> 1);
+        else { oyp = ((yp - 1) >> 1) + 1; store2 = store2 && (((yp - 1) & 1) == 0); }
+        out_pixel2 = ((size_t)b * (p.Ho + 2) + oyp) * p.Wo + (col >> 1);
       }
-      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(job.out) + out_pixel * (2 * N);
-      const __nv_bfloat16* res = job.res ? static_cast<const __nv_bfloat16*>(job.res) + out_pixel * (2 * N) : nullptr;
+      __nv_bfloat16* out2 = static_cast<__nv_bfloat16*>(job.out) + out_pixel2 * (2 * N);
+      const bool use_res = coalesced && job.res != nullptr && interior;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * N);
 #pragma unroll
       for (int c0 = 0; c0 < N; c0 += 16) {
         uint32_t v[16];
         tmem_ld16(taddr + c0, v);
         tmem_ld_wait();
-        if (store) {
-          uint32_t hi[8], lo[8];
-          uint32_t rh[8] = {0, 0, 0, 0, 0, 0, 0, 0}, rl[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-          if (res && interior) {
-            const uint4 a0 = __ldg(reinterpret_cast<const uint4*>(res + c0)), a1 = __ldg(reinterpret_cast<const uint4*>(res + c0) + 1);
-            const uint4 b0 = __ldg(reinterpret_cast<const uint4*>(res + N + c0)), b1 = __ldg(reinterpret_cast<const uint4*>(res + N + c0) + 1);
-            rh[0] = a0.x; rh[1] = a0.y; rh[2] = a0.z; rh[3] = a0.w; rh[4] = a1.x; rh[5] = a1.y; rh[6] = a1.z; rh[7] = a1.w;
-            rl[0] = b0.x; rl[1] = b0.y; rl[2] = b0.z; rl[3] = b0.w; rl[4] = b1.x; rl[5] = b1.y; rl[6] = b1.z; rl[7] = b1.w;
-          }
+        // 16-byte units of this pixel that hold columns c0 .. c0+15: two of hi, two of lo
+        const int uh = c0 / 8, ul = (N + c0) / 8;
+        uint4* ph0 = reinterpret_cast<uint4*>(my_row + (((uh) ^ my_key) << 4));
+        uint4* ph1 = reinterpret_cast<uint4*>(my_row + (((uh + 1) ^ my_key) << 4));
+        uint4* pl0 = reinterpret_cast<uint4*>(my_row + (((ul) ^ my_key) << 4));
+        uint4* pl1 = reinterpret_cast<uint4*>(my_row + (((ul + 1) ^ my_key) << 4));
+        uint32_t rh[8] = {0, 0, 0, 0, 0, 0, 0, 0}, rl[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        if (use_res) {
+          const uint4 a0 = *ph0, a1 = *ph1, b0 = *pl0, b1 = *pl1;
+          rh[0] = a0.x; rh[1] = a0.y; rh[2] = a0.z; rh[3] = a0.w; rh[4] = a1.x; rh[5] = a1.y; rh[6] = a1.z; rh[7] = a1.w;
+          rl[0] = b0.x; rl[1] = b0.y; rl[2] = b0.z; rl[3] = b0.w; rl[4] = b1.x; rl[5] = b1.y; rl[6] = b1.z; rl[7] = b1.w;
+        }
+        uint32_t hi[8], lo[8];
 #pragma unroll
-          for (int e = 0; e < 16; e += 2) {
-            float u0 = 0.f, u1 = 0.f;
-            if (interior) {
-              u0 = fmaf(__uint_as_float(v[e]), s_scale[c0 + e], s_bias[c0 + e]);
-              u1 = fmaf(__uint_as_float(v[e + 1]), s_scale[c0 + e + 1], s_bias[c0 + e + 1]);
-              // a bfloat16 is the upper half of a float: residual = hi + lo
-              u0 += __uint_as_float(rh[e >> 1] << 16) + __uint_as_float(rl[e >> 1] << 16);
-              u1 += __uint_as_float(rh[e >> 1] & 0xFFFF0000u) + __uint_as_float(rl[e >> 1] & 0xFFFF0000u);
-              u0 = apply_act(u0, p.act);
-              u1 = apply_act(u1, p.act);
-            }
-            __nv_bfloat16 h0, l0, h1, l1;
-            split_bf16(u0, h0, l0);
-            split_bf16(u1, h1, l1);
-            hi[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-            lo[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+        for (int e = 0; e < 16; e += 2) {
+          float u0 = 0.f, u1 = 0.f;
+          if (interior) {
+            u0 = fmaf(__uint_as_float(v[e]), s_scale[c0 + e], s_bias[c0 + e]);
+            u1 = fmaf(__uint_as_float(v[e + 1]), s_scale[c0 + e + 1], s_bias[c0 + e + 1]);
+            // a bfloat16 is the upper half of a float: residual = hi + lo
+            u0 += __uint_as_float(rh[e >> 1] << 16) + __uint_as_float(rl[e >> 1] << 16);
+            u1 += __uint_as_float(rh[e >> 1] & 0xFFFF0000u) + __uint_as_float(rl[e >> 1] & 0xFFFF0000u);
+            u0 = apply_act(u0, p.act);
+            u1 = apply_act(u1, p.act);
           }
-          uint4* oh = reinterpret_cast<uint4*>(out + c0);
-          uint4* ol = reinterpret_cast<uint4*>(out + N + c0);
+          __nv_bfloat16 h0, l0, h1, l1;
+          split_bf16(u0, h0, l0);
+          split_bf16(u1, h1, l1);
+          hi[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+          lo[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+        }
+        if (coalesced) {
+          *ph0 = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *ph1 = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+          *pl0 = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          *pl1 = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        } else if (store2) {
+          uint4* oh = reinterpret_cast<uint4*>(out2 + c0);
+          uint4* ol = reinterpret_cast<uint4*>(out2 + N + c0);
           oh[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
           oh[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
           ol[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
           ol[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
         }
       }
+      // the accumulator is drained: hand it back before the stores
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+      // (3) staging -> global, one row of 8 pixels (32N contiguous bytes) at a time
+      if (coalesced) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int jr = rb * kRowsPerTile + q * 4 + i;
+          if (jr < rows_total) {
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(job.out) +
+                                                  ((size_t)jr * p.W + cb * kColsPerTile) * PIXB);
+#pragma unroll
+            for (int u = lane; u < 8 * UNITS; u += 32) {
+              const int pl = i * 8 + u / UNITS, uu = u % UNITS;
+              dst[u] = *reinterpret_cast<const uint4*>(stg + pl * PIXB + ((uu ^ ((pl >> KEY_SHIFT) & KEY_MASK)) << 4));
+            }
+          }
+        }
+        __syncwarp();                                   // staging is reused by the next tile
+      }
     }
   }
 
@@ -461,7 +522,7 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-template <int CS, int N>
+template <int CS, int N, int KS>
 aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob* jobs_dev, int n_jobs,
                        int32_t* error_flag, double weight_bytes, cudaStream_t s) {
   using L = TcLayout<CS, N>;
@@ -474,18 +535,25 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
     AIQ_CUDA_TRY(cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     AIQ_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
   }
-  // as many ring stages as fit (two tiles in flight = 6), never fewer than 3
-  int stages = 6;
-  while (stages > 3 && S::total(stages, taps) + 1024 > smem_limit) --stages;
+  // Shared memory decides how many CTAs share an SM.  More resident CTAs hide the latency of
+  // a tile's load -> MMA -> epilogue chain better than a deeper ring does, so prefer two
+  // CTAs with at least 4 stages, then one with as many stages as fit (at most 6).
+  const int sm_budget = smem_limit + 1024;                 // per-SM capacity = opt-in block limit + 1 KB
+  int stages = 0;
+  for (int want = 2; want >= 1 && !stages; --want) {
+    const int per_cta = sm_budget / want - 1024;           // every block also reserves 1 KB
+    for (int st = 6; st >= (want > 1 ? 4 : 3); --st)
+      if (S::total(st, taps) + 1024 <= per_cta && S::total(st, taps) + 1024 <= smem_limit) { stages = st; break; }
+  }
+  if (!stages)
+    return set_error(AIQ_ERR_SHAPE, "conv_tc: shared memory for %d taps does not fit (%d bytes available)", taps, smem_limit);
   const int smem_bytes = S::total(stages, taps) + 1024;
-  if (smem_bytes > smem_limit)
-    return set_error(AIQ_ERR_SHAPE, "conv_tc: %d bytes of shared memory needed, %d available", smem_bytes, smem_limit);
   const int packed = N * (int)row_bytes(g.K, 8);
   if (packed > stages * L::STAGE_BYTES)
     return set_error(AIQ_ERR_SHAPE, "conv_tc: packed weights (%d bytes) exceed the staging ring", packed);
   static bool attr_set = false;
   if (!attr_set) {
-    AIQ_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<CS, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
+    AIQ_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<CS, N, KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
     attr_set = true;
   }
   TcParams p = {};
@@ -493,7 +561,13 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
   p.n_stages = stages; p.K = g.K; p.error_flag = error_flag;
   const int rows_total = g.B * (g.H + 2);
   const int n_tiles = ((rows_total + kRowsPerTile - 1) / kRowsPerTile) * (g.W / kColsPerTile);
-  int ctas = (n_sms + n_jobs - 1) / n_jobs;
+  // resident CTAs per SM: shared memory, and at most two (6 warps of ~110 registers fill the
+  // register file of an SM sub-partition after two CTAs)
+  int occ = sm_budget / (smem_bytes + 1024);
+  occ = occ > 2 ? 2 : (occ < 1 ? 1 : occ);
+  // All CTAs of the launch should be resident at once (a second wave would run nearly alone):
+  // split the resident capacity evenly over the jobs, rounding down.
+  int ctas = (n_sms * occ) / n_jobs;
   if (ctas > n_tiles) ctas = n_tiles;
   if (ctas < 1) ctas = 1;
   {
@@ -501,7 +575,7 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
                       2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
                       weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
                                                      (double)g.B * g.Ho * g.Wo * g.Cout));
-    conv_tc_kernel<CS, N><<<dim3(ctas, n_jobs), kTcThreads, smem_bytes, s>>>(map, p, jobs_dev);
+    conv_tc_kernel<CS, N, KS><<<dim3(ctas, n_jobs), kTcThreads, smem_bytes, s>>>(map, p, jobs_dev);
   }
   AIQ_LAUNCH_CHECK("conv_tc");
   return AIQ_OK;
@@ -542,8 +616,10 @@ aiq_status_t conv_tc_encode_map(const ConvGeom& g, const void* slot_base, int ba
 aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
                             int32_t* error_flag, double weight_bytes, cudaStream_t s) {
   const CUtensorMap& m = *static_cast<const CUtensorMap*>(map);
-#define AIQ_TC_CASE(CS_, N_) \
-  if (g.Cin == CS_ && g.Cout == N_) return launch_tc<CS_, N_>(g, m, jobs_dev, n_jobs, error_flag, weight_bytes, s);
+#define AIQ_TC_CASE(CS_, N_)                                                                              \
+  if (g.Cin == CS_ && g.Cout == N_)                                                                       \
+    return g.ks == 3 ? launch_tc<CS_, N_, 3>(g, m, jobs_dev, n_jobs, error_flag, weight_bytes, s)         \
+                     : launch_tc<CS_, N_, 1>(g, m, jobs_dev, n_jobs, error_flag, weight_bytes, s);
   AIQ_TC_CASE(16, 16) AIQ_TC_CASE(16, 32) AIQ_TC_CASE(16, 64)
   AIQ_TC_CASE(32, 16) AIQ_TC_CASE(32, 32) AIQ_TC_CASE(32, 64)
   AIQ_TC_CASE(64, 16) AIQ_TC_CASE(64, 32) AIQ_TC_CASE(64, 64)

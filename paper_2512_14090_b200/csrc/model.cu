@@ -697,7 +697,7 @@ extern "C" aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t
   t_launches = 0;
 
   // chunk: the requested (or default) size, shrunk until the layout fits the workspace
-  int B = g_opt_chunk > 0 ? g_opt_chunk : 256;
+  int B = g_opt_chunk > 0 ? g_opt_chunk : 1024;
   if (B > n_images) B = n_images;
   while (B > 1 && ws_layout(model, B, n_schemes).total > workspace_bytes) B = (B + 1) / 2;
   const WsLayout wl = ws_layout(model, B, n_schemes);
