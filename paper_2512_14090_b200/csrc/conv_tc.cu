@@ -19,8 +19,9 @@
 // memory, in the swizzled layout the MMA reads.  One thread issues the MMAs; four warps
 // drain the float32 accumulators from tensor memory, apply scale, bias, residual and
 // activation, split the result into two bfloat16 and store it.  Two accumulator buffers let
-// the epilogue of a tile overlap the MMAs of the next.  Stride-2 layers are computed at
-// input resolution and the epilogue keeps the even positions.
+// the epilogue of a tile overlap the MMAs of the next.  Stride-2 layers view the input as
+// (column parity, column pair, row parity, row pair), which makes every tap a dense TMA box;
+// they use one load and one ring stage per tap.
 //
 // Every wait is bounded: when a wait gives up the CTA raises an error word in global
 // memory, every role falls through, tensor memory is released and the kernel returns.
@@ -45,6 +46,7 @@ struct TcParams {
   int ks, stride, act;
   int n_stages;
   int K;                  // Cin * ks * ks (packed row length in elements)
+  int ver_pair_rows;      // stride 2: row pairs per version of the input slot = capacity * (H + 2) / 2
   int32_t* error_flag;    // device word, set to 1 when a bounded wait expired
 };
 
@@ -94,6 +96,13 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
       : "memory");
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -181,7 +190,7 @@ struct TcSmem {
   static __host__ __device__ constexpr int total(int stages, int taps) { return bars(stages, taps) + (2 * stages + 5) * 8 + 16; }
 };
 
-template <int CS, int N, int KS>
+template <int CS, int N, int KS, int STRIDE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const LayerJob* __restrict__ jobs) {
   using L = TcLayout<CS, N>;
@@ -208,9 +217,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * stages + 5);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
-  const int rows_total = p.B * (p.H + 2);
-  const int n_rb = (rows_total + kRowsPerTile - 1) / kRowsPerTile;
-  const int n_cb = p.W / kColsPerTile;
+  // Tiles.  Stride 1: 16 consecutive padded rows (image, y') x 8 columns, border rows included
+  // (they are written as zeros).  Stride 2: 16 interior output rows x 8 output columns, taken
+  // from IPT = 16 / Ho whole images when an image has fewer than 16 rows, or from one of the
+  // RBI = Ho / 16 row blocks of an image; the two border rows are zero-filled on the side.
+  const int rows_total = p.B * (p.H + 2);               // stride 1: padded rows of the batch
+  const int ipt = STRIDE == 2 && p.Ho < kRowsPerTile ? kRowsPerTile / p.Ho : 1;
+  const int rows_per_img = STRIDE == 2 ? (p.Ho < kRowsPerTile ? p.Ho : kRowsPerTile) : 0;
+  const int rbi = STRIDE == 2 && p.Ho > kRowsPerTile ? p.Ho / kRowsPerTile : 1;
+  const int n_rb = STRIDE == 2 ? ((p.B + ipt - 1) / ipt) * rbi : (rows_total + kRowsPerTile - 1) / kRowsPerTile;
+  const int n_cb = p.Wo / kColsPerTile;
   const int n_tiles = n_rb * n_cb;
 
   // ---- set-up -----------------------------------------------------------------------------
@@ -287,18 +303,45 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       uint32_t issued = 0, issued_phase = 0;       // per stage: a load was issued / parity of the last one
       for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
         const int rb = tile / n_cb, cb = tile - rb * n_cb;
-        for (int t = T_FIRST; t <= T_LAST && alive; ++t) {
-          alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
-          if (!alive) break;
-          issued |= 1u << stage;
-          issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
-          mbar_expect_tx(bar_full + 8 * stage, L::STAGE_BYTES);
+        if (STRIDE == 1) {
+          for (int t = T_FIRST; t <= T_LAST && alive; ++t) {
+            alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+            if (!alive) break;
+            issued |= 1u << stage;
+            issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
+            mbar_expect_tx(bar_full + 8 * stage, L::STAGE_BYTES);
 #pragma unroll
-          for (int ch = 0; ch < L::CHUNKS; ++ch)
-            tma_load_4d(smem_u32(ring) + stage * L::STAGE_BYTES + ch * L::CHUNK_BYTES, &in_map,
-                        bar_full + 8 * stage, ch * 64, cb * kColsPerTile + t - 1, rb * kRowsPerTile - 1,
-                        job.in_version);
-          if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+            for (int ch = 0; ch < L::CHUNKS; ++ch)
+              tma_load_4d(smem_u32(ring) + stage * L::STAGE_BYTES + ch * L::CHUNK_BYTES, &in_map,
+                          bar_full + 8 * stage, ch * 64, cb * kColsPerTile + t - 1, rb * kRowsPerTile - 1,
+                          job.in_version);
+            if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+          }
+        } else {
+          // One stage per tap: the map views the input as (channel, column parity, column pair,
+          // row parity, row pair), so tap (r, t) of a stride-2 window is a dense box.  Input
+          // padded row 2*oy + r = pair oy + (r >> 1), parity r & 1; input column 2*ox + t - 1 =
+          // pair ox + ((t - 1) >> 1), parity (t - 1) & 1 (pair -1 is out of range: zeros).
+          const int b0 = (rb / rbi) * ipt, oy0 = (rb % rbi) * kRowsPerTile;
+          for (int t = T_FIRST; t <= T_LAST && alive; ++t) {
+            for (int r = T_FIRST; r <= T_LAST && alive; ++r) {
+              alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+              if (!alive) break;
+              issued |= 1u << stage;
+              issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
+              mbar_expect_tx(bar_full + 8 * stage, L::CHUNKS * kRowsPerTile * L::GROUP_BYTES);
+              for (int img = 0; img < ipt; ++img) {
+                const int pair_row = job.in_version * p.ver_pair_rows + (b0 + img) * ((p.H + 2) >> 1) + oy0 + (r >> 1);
+#pragma unroll
+                for (int ch = 0; ch < L::CHUNKS; ++ch)
+                  tma_load_5d(smem_u32(ring) + stage * L::STAGE_BYTES + ch * L::CHUNK_BYTES +
+                                  img * rows_per_img * L::GROUP_BYTES,
+                              &in_map, bar_full + 8 * stage, ch * 64, (t - 1) & 1, cb * kColsPerTile + ((t - 1) >> 1),
+                              r & 1, pair_row);
+              }
+              if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+            }
+          }
         }
       }
       // copies in flight must land before the CTA exits: wait (bounded) for the last load
@@ -331,29 +374,46 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * N);
 #pragma unroll
         for (int t = T_FIRST; t <= T_LAST; ++t) {
-          if (!alive) break;
-          alive = mbar_wait(bar_full + 8 * stage, phase, s_abort, p.error_flag);
-          if (!alive) break;
-          tc_fence_after();
-          const uint32_t a_lo0 = ((smem_u32(ring) + stage * L::STAGE_BYTES) >> 4) | LBO_FIELD;
+          if (STRIDE == 1) {
+            if (!alive) break;
+            alive = mbar_wait(bar_full + 8 * stage, phase, s_abort, p.error_flag);
+            if (!alive) break;
+            tc_fence_after();
+          }
+          const uint32_t a_lo1 = ((smem_u32(ring) + stage * L::STAGE_BYTES) >> 4) | LBO_FIELD;
 #pragma unroll
           for (int r = T_FIRST; r <= T_LAST; ++r) {
+            uint32_t a_lo0 = a_lo1;
+            if (STRIDE == 2) {                     // every tap has a stage of its own
+              if (!alive) break;
+              alive = mbar_wait(bar_full + 8 * stage, phase, s_abort, p.error_flag);
+              if (!alive) break;
+              tc_fence_after();
+              a_lo0 = ((smem_u32(ring) + stage * L::STAGE_BYTES) >> 4) | LBO_FIELD;
+            }
             const int tap = KS == 3 ? r * 3 + t : 0;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
 #pragma unroll
               for (int kk = 0; kk < CS / 16; ++kk) {
                 const int byte = (part * CS + kk * 16) * 2;              // offset inside the pixel
-                const uint32_t a_off = (byte / L::CW_BYTES) * L::CHUNK_BYTES + r * L::GROUP_BYTES + (byte % L::CW_BYTES);
+                const uint32_t a_off = (byte / L::CW_BYTES) * L::CHUNK_BYTES + (STRIDE == 1 ? r * L::GROUP_BYTES : 0) +
+                                       (byte % L::CW_BYTES);
                 const uint64_t adesc = ((uint64_t)A_HI << 32) | (uint64_t)(a_lo0 + (a_off >> 4));
                 const uint64_t bdesc = ((uint64_t)B_HI << 32) | (uint64_t)(w_lo0 + ((tap * L::W_TAP_BYTES + kk * 32) >> 4));
                 const uint32_t accumulate = (t == T_FIRST && r == T_FIRST && part == 0 && kk == 0) ? 0u : 1u;
                 umma_bf16(d_tmem, adesc, bdesc, idesc, accumulate);
               }
             }
+            if (STRIDE == 2) {
+              umma_commit(bar_empty + 8 * stage);
+              if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+            }
           }
-          umma_commit(bar_empty + 8 * stage);        // the stage is free once these MMAs retire
-          if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+          if (STRIDE == 1) {
+            umma_commit(bar_empty + 8 * stage);        // the stage is free once these MMAs retire
+            if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+          }
         }
         if (alive) umma_commit(bar_acc_full + 8 * buf);
       }
@@ -381,15 +441,25 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
     for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
       const int buf = it & 1;
       const int rb = tile / n_cb, cb = tile - rb * n_cb;
-      const bool coalesced = p.stride == 1;
-      // (1) residual rows -> staging (stride-1 layers; only they have a residual)
-      if (coalesced && job.res) {
+      const int b0 = STRIDE == 2 ? (rb / rbi) * ipt : 0, oy0 = STRIDE == 2 ? (rb % rbi) * kRowsPerTile : 0;
+      // output row (image, padded y) of tile group gi, or -1 when the group is past the batch
+      auto out_row = [&](int gi) -> int {
+        if (STRIDE == 1) {
+          const int jr = rb * kRowsPerTile + gi;
+          return jr < rows_total ? jr : -1;
+        }
+        const int img = gi / rows_per_img;
+        const int bb = b0 + img;
+        return bb < p.B ? bb * (p.Ho + 2) + oy0 + (gi - img * rows_per_img) + 1 : -1;
+      };
+      // (1) residual rows -> staging
+      if (job.res) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int jr = rb * kRowsPerTile + q * 4 + i;
-          if (jr < rows_total) {
+          const int jr = out_row(q * 4 + i);
+          if (jr >= 0) {
             const uint4* src = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(job.res) +
-                                                              ((size_t)jr * p.W + cb * kColsPerTile) * PIXB);
+                                                              ((size_t)jr * p.Wo + cb * kColsPerTile) * PIXB);
 #pragma unroll
             for (int u = lane; u < 8 * UNITS; u += 32) {
               const int pl = i * 8 + u / UNITS, uu = u % UNITS;
@@ -403,24 +473,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       alive = __all_sync(0xffffffffu, alive);     // the tensor-memory loads below need the whole warp
       if (!alive) break;
       tc_fence_after();
-      const int j = rb * kRowsPerTile + g;             // padded input row (image, y')
-      const int col = cb * kColsPerTile + wl;
-      const int b = j / (p.H + 2);
-      const int yp = j - b * (p.H + 2);
-      const bool interior = yp >= 1 && yp <= p.H;
-      // stride 2: keep even positions; padded border rows map to the output's border rows
-      bool store2 = false;
-      size_t out_pixel2 = 0;
-      if (!coalesced) {
-        int oyp;
-        store2 = j < rows_total && ((col & 1) == 0);
-        if (yp == 0) oyp = 0;
-        else if (yp == p.H + 1) oyp = p.Ho + 1;
-        else { oyp = ((yp - 1) >> 1) + 1; store2 = store2 && (((yp - 1) & 1) == 0); }
-        out_pixel2 = ((size_t)b * (p.Ho + 2) + oyp) * p.Wo + (col >> 1);
+      bool interior = true;                       // stride 2 tiles hold interior rows only
+      if (STRIDE == 1) {
+        const int j = rb * kRowsPerTile + g;             // padded row (image, y')
+        const int yp = j % (p.H + 2);
+        interior = yp >= 1 && yp <= p.H;
       }
-      __nv_bfloat16* out2 = static_cast<__nv_bfloat16*>(job.out) + out_pixel2 * (2 * N);
-      const bool use_res = coalesced && job.res != nullptr && interior;
+      const bool use_res = job.res != nullptr && interior;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * N);
 #pragma unroll
       for (int c0 = 0; c0 < N; c0 += 16) {
@@ -435,9 +494,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
         uint4* pl1 = reinterpret_cast<uint4*>(my_row + (((ul + 1) ^ my_key) << 4));
         uint32_t rh[8] = {0, 0, 0, 0, 0, 0, 0, 0}, rl[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         if (use_res) {
-          const uint4 a0 = *ph0, a1 = *ph1, b0 = *pl0, b1 = *pl1;
+          const uint4 a0 = *ph0, a1 = *ph1, l0v = *pl0, l1v = *pl1;
           rh[0] = a0.x; rh[1] = a0.y; rh[2] = a0.z; rh[3] = a0.w; rh[4] = a1.x; rh[5] = a1.y; rh[6] = a1.z; rh[7] = a1.w;
-          rl[0] = b0.x; rl[1] = b0.y; rl[2] = b0.z; rl[3] = b0.w; rl[4] = b1.x; rl[5] = b1.y; rl[6] = b1.z; rl[7] = b1.w;
+          rl[0] = l0v.x; rl[1] = l0v.y; rl[2] = l0v.z; rl[3] = l0v.w; rl[4] = l1v.x; rl[5] = l1v.y; rl[6] = l1v.z; rl[7] = l1v.w;
         }
         uint32_t hi[8], lo[8];
 #pragma unroll
@@ -458,41 +517,45 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
           hi[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
           lo[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
         }
-        if (coalesced) {
-          *ph0 = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *ph1 = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-          *pl0 = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-          *pl1 = make_uint4(lo[4], lo[5], lo[6], lo[7]);
-        } else if (store2) {
-          uint4* oh = reinterpret_cast<uint4*>(out2 + c0);
-          uint4* ol = reinterpret_cast<uint4*>(out2 + N + c0);
-          oh[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          oh[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-          ol[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-          ol[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
-        }
+        *ph0 = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *ph1 = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+        *pl0 = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        *pl1 = make_uint4(lo[4], lo[5], lo[6], lo[7]);
       }
       // the accumulator is drained: hand it back before the stores
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
       // (3) staging -> global, one row of 8 pixels (32N contiguous bytes) at a time
-      if (coalesced) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int jr = rb * kRowsPerTile + q * 4 + i;
-          if (jr < rows_total) {
-            uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(job.out) +
-                                                  ((size_t)jr * p.W + cb * kColsPerTile) * PIXB);
+      for (int i = 0; i < 4; ++i) {
+        const int jr = out_row(q * 4 + i);
+        if (jr >= 0) {
+          uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(job.out) +
+                                                ((size_t)jr * p.Wo + cb * kColsPerTile) * PIXB);
 #pragma unroll
-            for (int u = lane; u < 8 * UNITS; u += 32) {
-              const int pl = i * 8 + u / UNITS, uu = u % UNITS;
-              dst[u] = *reinterpret_cast<const uint4*>(stg + pl * PIXB + ((uu ^ ((pl >> KEY_SHIFT) & KEY_MASK)) << 4));
-            }
+          for (int u = lane; u < 8 * UNITS; u += 32) {
+            const int pl = i * 8 + u / UNITS, uu = u % UNITS;
+            dst[u] = *reinterpret_cast<const uint4*>(stg + pl * PIXB + ((uu ^ ((pl >> KEY_SHIFT) & KEY_MASK)) << 4));
           }
         }
-        __syncwarp();                                   // staging is reused by the next tile
       }
+      if (STRIDE == 2) {
+        // zero border rows of the output images this tile touches (rows 0 and Ho + 1)
+        const bool top = oy0 == 0, bottom = oy0 + rows_per_img == p.Ho;
+        for (int img = q; img < ipt; img += 4) {
+          const int bb = b0 + img;
+          if (bb >= p.B) break;
+          for (int side = 0; side < 2; ++side) {
+            if (side == 0 ? !top : !bottom) continue;
+            const int jr = bb * (p.Ho + 2) + (side == 0 ? 0 : p.Ho + 1);
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(job.out) +
+                                                  ((size_t)jr * p.Wo + cb * kColsPerTile) * PIXB);
+            for (int u = lane; u < 8 * UNITS; u += 32) dst[u] = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+      }
+      __syncwarp();                                   // staging is reused by the next tile
     }
   }
 
@@ -522,9 +585,9 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-template <int CS, int N, int KS>
+template <int CS, int N, int KS, int STRIDE>
 aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob* jobs_dev, int n_jobs,
-                       int32_t* error_flag, double weight_bytes, cudaStream_t s) {
+                       int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s) {
   using L = TcLayout<CS, N>;
   using S = TcSmem<CS, N>;
   const int taps = g.ks * g.ks;
@@ -553,14 +616,21 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
     return set_error(AIQ_ERR_SHAPE, "conv_tc: packed weights (%d bytes) exceed the staging ring", packed);
   static bool attr_set = false;
   if (!attr_set) {
-    AIQ_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<CS, N, KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
+    AIQ_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<CS, N, KS, STRIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
     attr_set = true;
   }
   TcParams p = {};
   p.B = g.B; p.H = g.H; p.W = g.W; p.Ho = g.Ho; p.Wo = g.Wo; p.ks = g.ks; p.stride = g.stride; p.act = g.act;
   p.n_stages = stages; p.K = g.K; p.error_flag = error_flag;
-  const int rows_total = g.B * (g.H + 2);
-  const int n_tiles = ((rows_total + kRowsPerTile - 1) / kRowsPerTile) * (g.W / kColsPerTile);
+  p.ver_pair_rows = batch_capacity * (g.H + 2) / 2;
+  int n_tiles;
+  if (STRIDE == 1) {
+    n_tiles = ((g.B * (g.H + 2) + kRowsPerTile - 1) / kRowsPerTile) * (g.Wo / kColsPerTile);
+  } else {
+    const int ipt = g.Ho < kRowsPerTile ? kRowsPerTile / g.Ho : 1;
+    const int rbi = g.Ho > kRowsPerTile ? g.Ho / kRowsPerTile : 1;
+    n_tiles = ((g.B + ipt - 1) / ipt) * rbi * (g.Wo / kColsPerTile);
+  }
   // resident CTAs per SM: shared memory, and at most two (6 warps of ~110 registers fill the
   // register file of an SM sub-partition after two CTAs)
   int occ = sm_budget / (smem_bytes + 1024);
@@ -575,7 +645,7 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
                       2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
                       weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
                                                      (double)g.B * g.Ho * g.Wo * g.Cout));
-    conv_tc_kernel<CS, N, KS><<<dim3(ctas, n_jobs), kTcThreads, smem_bytes, s>>>(map, p, jobs_dev);
+    conv_tc_kernel<CS, N, KS, STRIDE><<<dim3(ctas, n_jobs), kTcThreads, smem_bytes, s>>>(map, p, jobs_dev);
   }
   AIQ_LAUNCH_CHECK("conv_tc");
   return AIQ_OK;
@@ -589,8 +659,12 @@ bool conv_tc_eligible(const ConvGeom& g) {
   if (g.stride != 1 && g.stride != 2) return false;
   if (g.Cin != 16 && g.Cin != 32 && g.Cin != 64) return false;
   if (g.Cout != 16 && g.Cout != 32 && g.Cout != 64) return false;
-  if (g.W % kColsPerTile != 0) return false;
-  if (g.stride == 2 && ((g.H & 1) || (g.W & 1))) return false;
+  if (g.Wo % kColsPerTile != 0) return false;
+  if (g.stride == 2) {
+    // whole images (or whole 16-row blocks of an image) must tile the 16 rows of a tile
+    if ((g.H & 1) || (g.W & 1)) return false;
+    if (!(g.Ho % kRowsPerTile == 0 || (g.Ho < kRowsPerTile && kRowsPerTile % g.Ho == 0))) return false;
+  }
   return true;
 }
 
@@ -600,30 +674,48 @@ aiq_status_t conv_tc_encode_map(const ConvGeom& g, const void* slot_base, int ba
   if (!enc) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
   const cuuint64_t pix_bytes = 4ull * g.Cs_in;
   const cuuint64_t rows = (cuuint64_t)batch_capacity * (g.H + 2);
-  cuuint64_t dims[4] = {(cuuint64_t)2 * g.Cs_in, (cuuint64_t)g.W, rows, (cuuint64_t)n_versions};
-  cuuint64_t strides[3] = {pix_bytes, pix_bytes * g.W, pix_bytes * g.W * rows};
   const cuuint32_t inner = pix_bytes < 128 ? (cuuint32_t)(2 * g.Cs_in) : 64u;
-  cuuint32_t box[4] = {inner, (cuuint32_t)kColsPerTile, (cuuint32_t)kBoxRows, 1u};
-  cuuint32_t estr[4] = {1, 1, 1, 1};
   const CUtensorMapSwizzle swz = pix_bytes < 128 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
-  CUresult r = enc(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(slot_base),
-                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r;
+  if (g.stride == 1) {
+    // (channel, column, padded row of the batch, version)
+    cuuint64_t dims[4] = {(cuuint64_t)2 * g.Cs_in, (cuuint64_t)g.W, rows, (cuuint64_t)n_versions};
+    cuuint64_t strides[3] = {pix_bytes, pix_bytes * g.W, pix_bytes * g.W * rows};
+    cuuint32_t box[4] = {inner, (cuuint32_t)kColsPerTile, (cuuint32_t)kBoxRows, 1u};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    r = enc(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(slot_base),
+            dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    // (channel, column parity, column pair, row parity, row pair over all versions): a tap of a
+    // stride-2 window is then a dense box.  Rows per image and per version are even.
+    const int rows_per_img = g.Ho < kRowsPerTile ? g.Ho : kRowsPerTile;
+    cuuint64_t dims[5] = {(cuuint64_t)2 * g.Cs_in, 2, (cuuint64_t)g.W / 2, 2, rows * n_versions / 2};
+    cuuint64_t strides[4] = {pix_bytes, 2 * pix_bytes, pix_bytes * g.W, 2 * pix_bytes * g.W};
+    cuuint32_t box[5] = {inner, 1u, (cuuint32_t)kColsPerTile, 1u, (cuuint32_t)rows_per_img};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    r = enc(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(slot_base),
+            dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
   if (r != CUDA_SUCCESS) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
   return AIQ_OK;
 }
 
 aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
-                            int32_t* error_flag, double weight_bytes, cudaStream_t s) {
+                            int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s) {
   const CUtensorMap& m = *static_cast<const CUtensorMap*>(map);
-#define AIQ_TC_CASE(CS_, N_)                                                                              \
-  if (g.Cin == CS_ && g.Cout == N_)                                                                       \
-    return g.ks == 3 ? launch_tc<CS_, N_, 3>(g, m, jobs_dev, n_jobs, error_flag, weight_bytes, s)         \
-                     : launch_tc<CS_, N_, 1>(g, m, jobs_dev, n_jobs, error_flag, weight_bytes, s);
+#define AIQ_TC_ARGS g, m, jobs_dev, n_jobs, batch_capacity, error_flag, weight_bytes, s
+#define AIQ_TC_CASE(CS_, N_)                                                                    \
+  if (g.Cin == CS_ && g.Cout == N_) {                                                           \
+    if (g.stride == 1) return g.ks == 3 ? launch_tc<CS_, N_, 3, 1>(AIQ_TC_ARGS) : launch_tc<CS_, N_, 1, 1>(AIQ_TC_ARGS); \
+    return g.ks == 3 ? launch_tc<CS_, N_, 3, 2>(AIQ_TC_ARGS) : launch_tc<CS_, N_, 1, 2>(AIQ_TC_ARGS);                    \
+  }
   AIQ_TC_CASE(16, 16) AIQ_TC_CASE(16, 32) AIQ_TC_CASE(16, 64)
   AIQ_TC_CASE(32, 16) AIQ_TC_CASE(32, 32) AIQ_TC_CASE(32, 64)
   AIQ_TC_CASE(64, 16) AIQ_TC_CASE(64, 32) AIQ_TC_CASE(64, 64)
 #undef AIQ_TC_CASE
+#undef AIQ_TC_ARGS
   return set_error(AIQ_ERR_SHAPE, "conv_tc: no kernel for Cin=%d Cout=%d", g.Cin, g.Cout);
 }
 

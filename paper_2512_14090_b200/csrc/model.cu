@@ -449,6 +449,7 @@ struct LayerPlan {
 };
 
 struct EvalPlan {
+  int batch_capacity = 0;               // images the plan's buffers are laid out for
   std::vector<LayerPlan> lp;            // per layer
   std::vector<LayerJob> jobs;           // host image of all job records
   std::vector<int> final_version;       // per scheme: version of the classifier output
@@ -468,6 +469,7 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
         return set_error(AIQ_ERR_UNSUPPORTED_BITS, "scheme %d, layer %d: bits=%d", s, l, (int)schemes[(size_t)s * n + l]);
   plan.lp.assign(n, LayerPlan());
   plan.jobs.clear();
+  plan.batch_capacity = B;
   std::vector<std::vector<int>> ver(n, std::vector<int>(S, 0));   // ver[l][s]
   auto slot_ptr = [&](int layer, int version) -> uint8_t* {
     const LayerInfo& li = m->layers[layer];
@@ -619,7 +621,7 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
       continue;
     }
     if (lp.n_tc > 0) {
-      st = launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, m->status_word, lp.weight_bytes_tc, stream);
+      st = launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream);
       if (st != AIQ_OK) return st;
     }
     if (lp.n_versions > lp.n_tc) {
