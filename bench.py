@@ -159,6 +159,85 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def run_kernel_sweep(args):
+    """Standalone memory-bound kernels against the HBM roofline: the quantized linear layer
+    (W [N][K] at 4/8/16/32 bits, M in {1,4,16,256}) and the quantize+pack kernel.  Operands
+    rotate over enough distinct copies to exceed twice the L2 capacity, so every launch
+    reads its weights from HBM.  One JSON line per case."""
+    import torch
+    from paper_2512_14090_b200 import build
+    build.build()
+    from paper_2512_14090_b200 import binding as aiq
+    from aiq_workloads import gen_linear_case
+    peaks = measured_peaks()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    L2_ROTATE = 300e6
+    reps = 20
+
+    def time_launches(fn, n):
+        """ms per launch of fn(i), i = 0..n-1, replayed from a CUDA graph so that host launch
+        overhead (about 10 us per call through ctypes) does not mask microsecond kernels."""
+        for i in range(min(n, 4)):
+            fn(i)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(n):
+                fn(i)
+        graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n          # ms per launch
+
+    shapes = [(4096, 4096), (8192, 8192), (1280, 320)]
+    if args.workload == "quantize":
+        for (N, K) in shapes[:2]:
+            w = torch.randn((N, K), device=dev) * 0.02
+            for bits in (4, 8, 16, 32):
+                rb = aiq.aiq_packed_row_bytes(K, bits)
+                packed = torch.empty((N, rb), dtype=torch.uint8, device=dev)
+                scales = torch.empty(N, dtype=torch.float32, device=dev)
+                nbytes = N * K * 4 + N * rb + N * 4
+                copies = max(2, int(np.ceil(L2_ROTATE / (N * K * 4))))
+                ws = [w] + [w.clone() for _ in range(copies - 1)]
+                ms = time_launches(lambda i: aiq.aiq_quantize_layer(ws[i % copies], bits, packed, scales), reps * copies)
+                gbs = nbytes / (ms * 1e-3) / 1e9
+                print(json.dumps(dict(workload="quantize", N=N, K=K, bits=bits, us=ms * 1e3, algorithmic_bytes=nbytes,
+                                      GBps=gbs, frac_of_measured_hbm=gbs / peaks["hbm_gbs"], frac_of_8TBps=gbs / 8000.0,
+                                      l2="input rotates over %d copies" % copies)), flush=True)
+        return
+    for (N, K) in shapes:
+        wh, _ = gen_linear_case(N, K, 1, 3234)
+        w = torch.from_numpy(wh).to(dev)
+        for bits in (4, 8, 16, 32):
+            rb = aiq.aiq_packed_row_bytes(K, bits)
+            packed0 = torch.empty((N, rb), dtype=torch.uint8, device=dev)
+            scales = torch.empty(N, dtype=torch.float32, device=dev)
+            aiq.aiq_quantize_layer(w, bits, packed0, scales)
+            copies = max(2, int(np.ceil(L2_ROTATE / (N * rb))))
+            packs = [packed0] + [packed0.clone() for _ in range(copies - 1)]
+            for M in (1, 4, 16, 256):
+                x = torch.randn((M, K), device=dev)
+                y = torch.empty((M, N), device=dev)
+                nbytes = N * rb + 4 * N + 4 * M * (K + N)
+                flops = 2.0 * M * N * K
+                n = reps * copies if M <= 16 else max(copies, 8)
+                wsb = aiq.aiq_qlinear_workspace_bytes(N, K, bits, M)
+                wsp = torch.empty(wsb, dtype=torch.uint8, device=dev) if wsb else None
+                ms = time_launches(lambda i: aiq.aiq_qlinear(packs[i % copies], scales, None, N, K, bits, x, y,
+                                                             workspace=wsp), n)
+                gbs = nbytes / (ms * 1e-3) / 1e9
+                print(json.dumps(dict(workload="qlinear", N=N, K=K, bits=bits, M=M, us=ms * 1e3,
+                                      algorithmic_bytes=nbytes, GBps=gbs, frac_of_measured_hbm=gbs / peaks["hbm_gbs"],
+                                      frac_of_8TBps=gbs / 8000.0, TFLOPs=flops / (ms * 1e-3) / 1e12,
+                                      l2="weights rotate over %d copies" % copies)), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -167,6 +246,9 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--chunk", type=int, default=0, help="images per evaluator pass (0 = library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="resnet20_step", choices=["resnet20_step", "qlinear", "quantize"],
+                    help="resnet20_step: the headline line (default).  qlinear / quantize: per-case lines for the "
+                         "standalone memory-bound kernels (1 GPU)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -174,6 +256,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+    if args.workload != "resnet20_step":
+        if rank == 0:
+            run_kernel_sweep(args)
         return
     if args.warmup < 3:
         args.warmup = 3
@@ -294,7 +380,20 @@ def main():
     p = prof[top]
     avg_ms = p["ms"] / max(p["launches"], 1)
     sm_mhz = clocks.get("sm_mhz") or peaks["sm_max_mhz"]
-    if top == "conv":
+    if top == "conv_tc":
+        # bf16 tensor-core implicit GEMM.  Algorithmic FLOPs = 2 per multiply-add of the
+        # convolution (the hi/lo split doubles the MMA work; that overhead is not counted).
+        peak = peaks["bf16_tflops_sustained"]
+        achieved = p["flops"] / (p["ms"] / 1000.0) / 1e12
+        roofline = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
+                        traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH, kernel="conv_tc_kernel (tcgen05 bf16, fp32 accumulate)",
+                        peak_source=f"dense bf16 GEMM, sustained, {peaks['source']}",
+                        launches=p["launches"], avg_launch_ms=avg_ms,
+                        algorithmic_flops_per_launch=p["flops"] / max(p["launches"], 1),
+                        algorithmic_bytes_per_launch=p["bytes"] / max(p["launches"], 1),
+                        note="N = Cout = 16..64 and K = 16 per MMA: operand reads from shared memory, not the "
+                             "tensor pipe, bound this kernel (see DESIGN.md)")
+    elif top == "conv":
         # float32 multiply-add path: 148 SMs x 128 lanes x 2 FLOP per clock
         peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12
         achieved = p["flops"] / (p["ms"] / 1000.0) / 1e12

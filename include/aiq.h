@@ -96,13 +96,23 @@ aiq_status_t aiq_quantize_layer(const float* W, int N, int K, int bits, void* pa
  * Small-batch quantized linear layer - the memory-bound case the method targets
  * (Abstract; Section 5, Roofline paragraph): weight bytes N*K*bits/8 dominate the traffic.
  *     y[m][n] = s_n * sum_k code[n][k] * x[m][k] + bias[n]
- * (16 / 32 bits: the stored element itself, s_n = 1).  float32 multiply-add, float32
- * accumulation.  packed / scales: as written by aiq_quantize_layer (device).  bias: device
- * [N] or NULL.  x: device float32 [M][K] row-major, 16-byte aligned; y: device float32
- * [M][N].  M >= 1.  Asynchronous on `stream`.
+ * (16 / 32 bits: the stored element itself, s_n = 1).  packed / scales: as written by
+ * aiq_quantize_layer (device).  bias: device [N] or NULL.  x: device float32 [M][K]
+ * row-major, 16-byte aligned; y: device float32 [M][N].  M >= 1.  Asynchronous on `stream`.
+ *
+ * Two kernels.  The plain one expands weights to float32 in registers and accumulates in
+ * float32 (any shape, any bit-width).  For 4- / 8-bit weights, M <= 16, K a multiple of 512
+ * and N*K >= 2^20 a faster one keeps the codes integer and uses the int8 tensor cores: the
+ * activations of each group of 512 k become three int8 digits with a shared exponent
+ * (21 bits below the group's largest |x|), the int32 sums are exact, and K-slices meet in y
+ * through float atomics (run-to-run differences in the last bit).  It needs scratch memory:
+ * pass `workspace` (device, 16-byte aligned) of at least aiq_qlinear_workspace_bytes(...)
+ * bytes; with workspace == NULL, or where that function returns 0, the plain kernel runs.
  */
+size_t aiq_qlinear_workspace_bytes(int N, int K, int bits, int M);
 aiq_status_t aiq_qlinear(const void* packed, const float* scales, const float* bias, int N,
-                         int K, int bits, const float* x, int M, float* y, void* stream);
+                         int K, int bits, const float* x, int M, float* y, void* workspace,
+                         size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------
  * Model description.  Layers are listed in scheme order: entry i of a scheme is the

@@ -21,7 +21,7 @@ ACT = {"none": 0, "relu": 1, "relu6": 2}
 
 EXPORTS = [
     "aiq_status_string", "aiq_last_error", "aiq_fold_bn", "aiq_packed_row_bytes",
-    "aiq_quantize_layer", "aiq_qlinear", "aiq_model_bytes", "aiq_model_create",
+    "aiq_quantize_layer", "aiq_qlinear", "aiq_qlinear_workspace_bytes", "aiq_model_bytes", "aiq_model_create",
     "aiq_model_destroy", "aiq_model_num_layers", "aiq_model_num_classes",
     "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
     "aiq_eval_schemes", "aiq_set_eval_options", "aiq_last_call_stats", "aiq_scheme_ai",
@@ -78,7 +78,9 @@ def _load():
     lib.aiq_quantize_layer.restype = i32
     lib.aiq_quantize_layer.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     lib.aiq_qlinear.restype = i32
-    lib.aiq_qlinear.argtypes = [vp, vp, vp, i32, i32, i32, vp, i32, vp, vp]
+    lib.aiq_qlinear.argtypes = [vp, vp, vp, i32, i32, i32, vp, i32, vp, vp, sz, vp]
+    lib.aiq_qlinear_workspace_bytes.restype = sz
+    lib.aiq_qlinear_workspace_bytes.argtypes = [i32, i32, i32, i32]
     lib.aiq_model_bytes.restype = sz
     lib.aiq_model_bytes.argtypes = [C.POINTER(ArchDesc)]
     lib.aiq_model_create.restype = i32
@@ -185,10 +187,15 @@ def aiq_quantize_layer(W, bits, packed_out, scales_out, nonfinite_flag=None, str
                                   _dev(nonfinite_flag), _stream(stream)))
 
 
-def aiq_qlinear(packed, scales, bias, N, K, bits, x, y, stream=None):
+def aiq_qlinear_workspace_bytes(N, K, bits, M):
+    return int(lib.aiq_qlinear_workspace_bytes(int(N), int(K), int(bits), int(M)))
+
+
+def aiq_qlinear(packed, scales, bias, N, K, bits, x, y, workspace=None, stream=None):
     M = x.shape[0]
     _check(lib.aiq_qlinear(_dev(packed), _dev(scales), _dev(bias), int(N), int(K), int(bits),
-                           _dev(x), int(M), _dev(y), _stream(stream)))
+                           _dev(x), int(M), _dev(y), _dev(workspace),
+                           workspace.numel() if workspace is not None else 0, _stream(stream)))
 
 
 def aiq_set_eval_options(chunk=0, share_prefix=True):

@@ -125,6 +125,10 @@ aiq_status_t launch_quantize(const float* W, int N, int K, int bits, void* packe
 // y[m][n] for every job: in = x [M][K], out = y [M][N]
 aiq_status_t launch_qlinear(const LayerJob* jobs_dev, const LayerJob* single_host, int n_jobs, int N,
                             int K, int M, cudaStream_t s);
+// warp-level tensor-core path of the linear layer (4- / 8-bit weights, M <= 16, large N*K)
+bool qlinear_mma_applicable(int N, int K, int bits, int M);
+size_t qlinear_mma_workspace_bytes(int K, int M);
+aiq_status_t launch_qlinear_mma(const LayerJob& job, int N, int K, int M, void* workspace, cudaStream_t s);
 // weight_bytes: packed weights + scales + biases of all jobs (for the profile's byte count)
 aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
                          const float* net_input, double weight_bytes, cudaStream_t s);

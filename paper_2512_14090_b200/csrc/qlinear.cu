@@ -180,8 +180,14 @@ aiq_status_t launch_qlinear(const LayerJob* jobs_dev, const LayerJob* single_hos
 
 }  // namespace aiq
 
+extern "C" size_t aiq_qlinear_workspace_bytes(int N, int K, int bits, int M) {
+  if (N <= 0 || K <= 0 || M <= 0 || !aiq::qlinear_mma_applicable(N, K, bits, M)) return 0;
+  return aiq::qlinear_mma_workspace_bytes(K, M);
+}
+
 extern "C" aiq_status_t aiq_qlinear(const void* packed, const float* scales, const float* bias, int N,
-                                    int K, int bits, const float* x, int M, float* y, void* stream) {
+                                    int K, int bits, const float* x, int M, float* y, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
   if (!aiq::bits_ok(bits)) return aiq::set_error(AIQ_ERR_UNSUPPORTED_BITS, "aiq_qlinear: bits=%d", bits);
   if (!packed || !scales || !x || !y) return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_qlinear: null pointer");
   if (N <= 0 || K <= 0 || M <= 0)
@@ -197,5 +203,12 @@ extern "C" aiq_status_t aiq_qlinear(const void* packed, const float* scales, con
   job.scale = scales;
   job.bias = bias;
   job.bits = bits;
+  // the integer tensor-core kernel needs scratch for the converted activations
+  if (workspace && aiq::qlinear_mma_applicable(N, K, bits, M)) {
+    if (((uintptr_t)workspace) & 15)
+      return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_qlinear: workspace not 16-byte aligned");
+    if (workspace_bytes >= aiq::qlinear_mma_workspace_bytes(K, M))
+      return aiq::launch_qlinear_mma(job, N, K, M, workspace, (cudaStream_t)stream);
+  }
   return aiq::launch_qlinear(nullptr, &job, 1, N, K, M, (cudaStream_t)stream);
 }

@@ -53,8 +53,12 @@ def test_host_side_argument_checks(aiq):
     assert "bits=3" in aiq.last_error()
     assert aiq.lib.aiq_quantize_layer(None, 4, 4, 8, one, one, None, None) == aiq.ERR_INVALID_ARG
     assert aiq.lib.aiq_quantize_layer(one, 0, 4, 8, one, one, None, None) == aiq.ERR_INVALID_ARG
-    assert aiq.lib.aiq_qlinear(one, one, None, 4, 4, 7, one, 1, one, None) == aiq.ERR_UNSUPPORTED_BITS
-    assert aiq.lib.aiq_qlinear(one, one, None, 4, 4, 8, one, 0, one, None) == aiq.ERR_INVALID_ARG
+    assert aiq.lib.aiq_qlinear(one, one, None, 4, 4, 7, one, 1, one, None, 0, None) == aiq.ERR_UNSUPPORTED_BITS
+    assert aiq.lib.aiq_qlinear(one, one, None, 4, 4, 8, one, 0, one, None, 0, None) == aiq.ERR_INVALID_ARG
+    assert aiq.aiq_qlinear_workspace_bytes(4096, 4096, 4, 1) > 0
+    assert aiq.aiq_qlinear_workspace_bytes(4096, 4096, 16, 1) == 0      # plain kernel only
+    assert aiq.aiq_qlinear_workspace_bytes(4096, 4000, 4, 1) == 0
+    assert aiq.aiq_qlinear_workspace_bytes(64, 512, 8, 1) == 0
     assert aiq.lib.aiq_fold_bn(None, one, one, one, one, 1, 1, 1e-5, one, one, None) == aiq.ERR_INVALID_ARG
     assert aiq.lib.aiq_forward(None, one, one, 1, one, one, 0, None) == aiq.ERR_INVALID_ARG
     assert aiq.lib.aiq_eval_schemes(None, one, 1, one, one, 1, one, None, None, one, 0, None) == aiq.ERR_INVALID_ARG
