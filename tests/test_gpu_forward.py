@@ -210,3 +210,32 @@ def test_forward_and_eval_errors():
     with pytest.raises(aiq.AiqError) as e:
         model.aiq_eval_schemes(np.full((1, model.n_layers), 8, np.uint8), x, labels, workspace=small)
     assert e.value.status == aiq.ERR_WORKSPACE_TOO_SMALL
+
+
+def test_full_size_greedy_step_sampled_against_oracle():
+    """The benchmark's configuration: 10,000 images, 21 candidate schemes, chunks of 1024,
+    tensor-core path.  The oracle cannot run 210,000 forwards, so predictions are compared on
+    a sample of images it computes one by one; over the whole set the counts must equal the
+    number of predictions that match the labels."""
+    import torch
+    aiq = binding()
+    arch = resnet20()
+    n = 10000
+    x = gen_images(n, 3, 32, 32, 5679)
+    sample = np.arange(0, n, 131)[:72]                      # 72 images spread over all chunks
+    params = balance_classifier(arch, gen_model(arch, 1234), x[sample])
+    model = aiq.Model(arch, params)
+    folded, bank = _oracle_bank(arch, params, (4, 8))
+    schemes = one_layer_lowered_schemes(22, conv_layer_indices(arch))
+    labels = np.random.default_rng(3).integers(0, 10, n).astype(np.int32)
+    labels[sample] = O.predict(O.forward_fp32_unquantized(arch, folded, x[sample]))
+    oacc, ocounts, opreds, omargins = O.eval_schemes(arch, bank, schemes, x[sample], labels[sample])
+    preds = torch.full((21, n), -1, dtype=torch.int32, device="cuda")
+    aiq.aiq_set_eval_options(0, True)
+    acc, counts = model.aiq_eval_schemes(schemes, to_dev(x), to_dev(labels), preds=preds)
+    p = preds.cpu().numpy()
+    assert p.min() >= 0 and p.max() <= 9
+    assert np.array_equal((p == labels[None, :]).sum(axis=1), counts)
+    assert np.allclose(acc, counts / float(n))
+    assert_preds_match(p[:, sample], opreds, omargins, "full size sample")
+    assert len(np.unique(p[0])) >= 5
