@@ -42,7 +42,7 @@ aiq_status_t launch_fold_bn(const float* W, const float* gamma, const float* bet
 // read from memory once.
 // ---------------------------------------------------------------------------------------
 template <int CACHE>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, CACHE == 1 ? 4 : 3)
 quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad, int bits,
                      uint8_t* __restrict__ packed, float* __restrict__ scales,
                      int32_t* __restrict__ nonfinite_flag) {
@@ -53,7 +53,7 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad, int bits,
 
   float v[CACHE][8];
   float amax = 0.0f;
-  bool bad = false;
+  float poison = 0.0f;           // stays 0 unless an element is NaN or infinite (x * 0 is then NaN)
 
   auto load_granule = [&](int gi, float* dstv) {
     const int k0 = gi << 3;
@@ -75,9 +75,8 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad, int bits,
       load_granule(gi, v[c]);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        const float a = fabsf(v[c][j]);
-        bad |= !(a <= 3.402823466e38f);          // false for NaN and for infinity
-        amax = fmaxf(amax, a);
+        poison = fmaf(v[c][j], 0.0f, poison);
+        amax = fmaxf(amax, fabsf(v[c][j]));
       }
     }
   }
@@ -87,9 +86,8 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad, int bits,
     load_granule(gi, t);
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const float a = fabsf(t[j]);
-      bad |= !(a <= 3.402823466e38f);
-      amax = fmaxf(amax, a);
+      poison = fmaf(t[j], 0.0f, poison);
+      amax = fmaxf(amax, fabsf(t[j]));
     }
   }
 
@@ -100,7 +98,7 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad, int bits,
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
   if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
-  if (bad) s_bad = 1;
+  if (poison != 0.0f) s_bad = 1;                 // NaN compares unequal to everything
   __syncthreads();
   amax = 0.0f;
   for (int w = 0; w < (int)(blockDim.x >> 5); ++w) amax = fmaxf(amax, s_max[w]);
@@ -120,24 +118,40 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad, int bits,
   if (threadIdx.x == 0) scales[n] = s;
 
   uint8_t* out_row = packed + (size_t)n * ((size_t)Kpad * bits / 8);
+  // code = rint(w / s) with the IEEE quotient.  A true division costs ~10 instructions, so the
+  // quotient is first estimated as w * (1/s): the estimate and the correctly rounded quotient
+  // differ by at most 1.5 * 2^-23 relative, hence they round to the same integer unless the
+  // estimate lies within that distance of a tie.  Only then (about one element in 10^4) is
+  // the exact division evaluated, so the result is bit-identical to always dividing.
+  const bool estimate_ok = s >= 1e-30f;        // a tiny scale would overflow the reciprocal: always divide
+  const float rs = estimate_ok ? __frcp_rn(s) : 0.f;
+  // Rounding without the conversion unit: adding 1.5 * 2^23 rounds the estimate to the nearest
+  // integer (ties to even) in the adder, and leaves that integer, in two's complement, in the
+  // low mantissa bits of the sum.  |estimate| <= 128, far inside the range where this holds.
+  // Codes cannot leave [-qmax, qmax]: |w| <= amax and s = fl(amax / qmax).
+  auto code_of = [&](float wv) -> uint32_t {
+    const float tq = wv * rs;
+    const float m = tq + 12582912.0f;
+    const float q = m - 12582912.0f;
+    uint32_t code = (uint32_t)__float_as_int(m);
+    if (!estimate_ok || fabsf(fabsf(tq - q) - 0.5f) <= fabsf(tq) * 4.8e-7f)   // 2^-21: near a tie
+      code = (uint32_t)(int)fminf(fmaxf(rintf(__fdiv_rn(wv, s)), lo), hi);
+    return code;
+  };
   auto store_granule = [&](int gi, const float* val) {
     if (bits == 4) {
       uint32_t word = 0;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        float q = rintf(__fdiv_rn(val[j], s));
-        q = fminf(fmaxf(q, lo), hi);
-        word |= ((uint32_t)((int)q) & 0xFu) << (4 * j);
+        word |= (code_of(val[j]) & 0xFu) << (4 * j);
       }
       reinterpret_cast<uint32_t*>(out_row)[gi] = word;
     } else if (bits == 8) {
       uint32_t w0 = 0, w1 = 0;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        float q = fminf(fmaxf(rintf(__fdiv_rn(val[j], s)), lo), hi);
-        w0 |= ((uint32_t)((int)q) & 0xFFu) << (8 * j);
-        float r = fminf(fmaxf(rintf(__fdiv_rn(val[j + 4], s)), lo), hi);
-        w1 |= ((uint32_t)((int)r) & 0xFFu) << (8 * j);
+        w0 |= (code_of(val[j]) & 0xFFu) << (8 * j);
+        w1 |= (code_of(val[j + 4]) & 0xFFu) << (8 * j);
       }
       reinterpret_cast<uint2*>(out_row)[gi] = make_uint2(w0, w1);
     } else if (bits == 16) {
