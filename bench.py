@@ -36,7 +36,9 @@ UNIT = "scheme-evals/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the
 # committed ncu summary under profiles/ (None until captured / after the kernel changed)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# conv_tc_kernel: 198.1 MB per launch measured at chunk 256 (profiles/conv_tc__resnet20_greedy_step.md),
+# scaled by 4 to the default chunk of 1024 images (traffic grows with the images of a launch)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 198.1e6
 
 
 def measured_peaks():
@@ -195,6 +197,37 @@ def run_kernel_sweep(args):
         return e0.elapsed_time(e1) / n          # ms per launch
 
     shapes = [(4096, 4096), (8192, 8192), (1280, 320)]
+    if args.workload == "forward":
+        # one scheme, one batch, through aiq_forward (host plan + launches included): images/s
+        from aiq_workloads import (resnet20, mobilenet_v2, gen_model, gen_images, gen_random_scheme,
+                                   mixed_int4_int8_scheme, conv_layer_indices)
+        cases = [("resnet20 (config 0)", resnet20(), 1234, [64], lambda a: gen_random_scheme(len(a["layers"]), 42)),
+                 ("mobilenet_v2_cifar (config 2)", mobilenet_v2("cifar"), 2234, [1, 256],
+                  lambda a: mixed_int4_int8_scheme(len(a["layers"]), conv_layer_indices(a), 10, 43)),
+                 ("mobilenet_v2_imagenet (config 4)", mobilenet_v2("imagenet"), 4234, [1, 32, 256],
+                  lambda a: np.full(len(a["layers"]), 8, np.uint8))]
+        for name, arch, seed, batches, mk in cases:
+            model = aiq.Model(arch, gen_model(arch, seed), device=dev)
+            scheme = mk(arch)
+            for B in batches:
+                xb = torch.randn((B, arch["in_c"], arch["in_h"], arch["in_w"]), device=dev)
+                logits = torch.empty((B, model.n_classes), device=dev)
+                wsb = torch.empty(model.aiq_workspace_bytes(B, 1), dtype=torch.uint8, device=dev)
+                for _ in range(3):
+                    model.aiq_forward(scheme, xb, logits=logits, workspace=wsb)
+                torch.cuda.synchronize()
+                n = 20 if B <= 32 else 5
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(n):
+                    model.aiq_forward(scheme, xb, logits=logits, workspace=wsb)
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / n
+                print(json.dumps(dict(workload="forward", model=name, batch=B, ms=ms, images_per_s=B / (ms * 1e-3),
+                                      launches=aiq.aiq_last_call_stats()["kernel_launches"])), flush=True)
+            model.close()
+        return
     if args.workload == "quantize":
         for (N, K) in shapes[:2]:
             w = torch.randn((N, K), device=dev) * 0.02
@@ -246,7 +279,7 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--chunk", type=int, default=0, help="images per evaluator pass (0 = library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="resnet20_step", choices=["resnet20_step", "qlinear", "quantize"],
+    ap.add_argument("--workload", default="resnet20_step", choices=["resnet20_step", "qlinear", "quantize", "forward"],
                     help="resnet20_step: the headline line (default).  qlinear / quantize: per-case lines for the "
                          "standalone memory-bound kernels (1 GPU)")
     args = ap.parse_args()
@@ -386,7 +419,8 @@ def main():
         peak = peaks["bf16_tflops_sustained"]
         achieved = p["flops"] / (p["ms"] / 1000.0) / 1e12
         roofline = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
-                        traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH, kernel="conv_tc_kernel (tcgen05 bf16, fp32 accumulate)",
+                        traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH if chunk == 1024 else None,
+                        kernel="conv_tc_kernel (tcgen05 bf16, fp32 accumulate)",
                         peak_source=f"dense bf16 GEMM, sustained, {peaks['source']}",
                         launches=p["launches"], avg_launch_ms=avg_ms,
                         algorithmic_flops_per_launch=p["flops"] / max(p["launches"], 1),
@@ -398,7 +432,7 @@ def main():
         peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12
         achieved = p["flops"] / (p["ms"] / 1000.0) / 1e12
         roofline = dict(bound="alu", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
-                        traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH, kernel="conv_igemm_kernel (float32 FMA)",
+                        traffic=None, kernel="conv_igemm_kernel (float32 FMA)",
                         peak_source=f"148 SMs x 128 FP32 lanes x 2 x {sm_mhz:.0f} MHz (median SM clock sampled during the run)",
                         launches=p["launches"], avg_launch_ms=avg_ms,
                         algorithmic_flops_per_launch=p["flops"] / max(p["launches"], 1),
@@ -406,7 +440,7 @@ def main():
     else:
         achieved = p["bytes"] / (p["ms"] / 1000.0) / 1e9
         roofline = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=achieved / peaks["hbm_gbs"], traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                        frac=achieved / peaks["hbm_gbs"], traffic=None,
                         kernel=top, peak_source=f"HBM copy bandwidth, {peaks['source']}",
                         launches=p["launches"], avg_launch_ms=avg_ms,
                         algorithmic_bytes_per_launch=p["bytes"] / max(p["launches"], 1))
