@@ -141,6 +141,13 @@ aiq_status_t conv_tc_encode_map(const ConvGeom& g, const void* slot_base, int ba
                                 void* map_out);
 aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
                             int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s);
+// Pointwise (1x1, stride 1) tensor-core convolution for any channel count that is a multiple
+// of 8 (conv_pw_tc.cuh).  `map`: CUtensorMap over the input slot, dims (Cs, 2, pixels of all versions).
+bool conv_pw_tc_eligible(const ConvGeom& g);
+aiq_status_t conv_pw_tc_encode_map(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
+                                   void* map_out);
+aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
+                               int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s);
 // pooled[b][c] = mean over the H x W interior of a split tensor, per job (in -> out float32 [B][C])
 aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int H, int W, int C, int act_format,
                             cudaStream_t s);

@@ -1,0 +1,285 @@
+// Pointwise (1x1, stride 1) convolution with many channels on the tcgen05 tensor cores.
+// Included by conv_tc.cu (shares its PTX wrappers); not a stand-alone translation unit.
+//
+// A 1x1 convolution over split activations is a plain GEMM over all (padded) pixels:
+//   D[128 pixels][Nt channels] += A[128][64 k] * B[Nt][64 k]^T   per chunk of 64 input channels,
+// once for the hi half and once for the lo half of the pixels (same B).  MobileNetV2's
+// expand / project / head layers have 16 .. 960 input and 16 .. 1280 output channels, so
+// neither operand fits in shared memory: both stream through a ring, one stage per chunk.
+//   warp 0      TMA producer: A tiles (hi and lo, 128 pixels x 64 channels each, 128-byte swizzle;
+//               channels past C arrive as zeros)
+//   warp 1      MMA issuer
+//   warps 2-5   epilogue (TMEM -> scale, bias, residual, activation -> split bfloat16 -> global)
+//   warps 6-9   weight expanders: packed 4 / 8-bit rows from global memory (L2) -> bfloat16 ->
+//               swizzled B tile in shared memory, made visible to the MMA with a proxy fence
+// A CTA owns one (job, tile of Nt output channels) and walks over pixel tiles.
+#pragma once
+
+namespace aiq {
+namespace {
+
+constexpr int kPwThreads = 320;
+constexpr int kPwChunk = 64;                         // input channels per stage
+constexpr int kPwATile = 128 * kPwChunk * 2;         // 16 KB: 128 pixels x 64 bfloat16
+
+struct PwParams {
+  int P;                    // padded pixels of the batch: B * (H + 2) * W
+  int H, W;                 // spatial size (rows 0 and H + 1 of every image are border rows)
+  int Cin, Cs_in, Cout, Cs_out;
+  int Nt;                   // output channels per CTA (multiple of 16, <= 128)
+  int n_ntiles;
+  int act, n_stages;
+  long long ver_pixels;     // pixels per version of the input slot (capacity * (H + 2) * W)
+  int32_t* error_flag;
+};
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+// shared memory: [stage: A_hi | A_lo | B] x n_stages, scale, bias, barriers, tmem ptr, abort flag
+__host__ __device__ inline int pw_stage_bytes(int Nt) { return 2 * kPwATile + Nt * kPwChunk * 2; }
+__host__ __device__ inline int pw_smem_bytes(int Nt, int stages) {
+  return stages * pw_stage_bytes(Nt) + 2 * 128 * 4 + (3 * stages + 4) * 8 + 16;
+}
+
+__global__ void __launch_bounds__(kPwThreads, 1)
+conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, PwParams p, const LayerJob* __restrict__ jobs) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int job_idx = blockIdx.y / p.n_ntiles, ntile = blockIdx.y - job_idx * p.n_ntiles;
+  const LayerJob job = jobs[job_idx];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int stages = p.n_stages, Nt = p.Nt, n0 = ntile * Nt;
+  const int stage_bytes = pw_stage_bytes(Nt);
+
+  float* s_scale = reinterpret_cast<float*>(smem + stages * stage_bytes);
+  float* s_bias = s_scale + 128;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_bias + 128);
+  const uint32_t bar_a_full = smem_u32(bars);               // TMA bytes of a stage have landed
+  const uint32_t bar_b_full = bar_a_full + 8 * stages;      // expanders finished the B tile of a stage
+  const uint32_t bar_empty = bar_b_full + 8 * stages;       // the MMAs that read a stage have retired
+  const uint32_t bar_acc_full = bar_empty + 8 * stages;
+  const uint32_t bar_acc_empty = bar_acc_full + 16;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 3 * stages + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  const int n_tiles = (p.P + 127) / 128;
+  const int n_chunks = (p.Cs_in + kPwChunk - 1) / kPwChunk;
+
+  if (tid == 0) {
+    for (int i = 0; i < stages; ++i) {
+      mbar_init(bar_a_full + 8 * i, 1);
+      mbar_init(bar_b_full + 8 * i, 4);          // one arrival per expander warp
+      mbar_init(bar_empty + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_acc_full + 8 * i, 1);
+      mbar_init(bar_acc_empty + 8 * i, 4);       // one arrival per epilogue warp
+    }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = tid; i < 128; i += kPwThreads) {
+    const int n = n0 + i;
+    s_scale[i] = (i < Nt && n < p.Cout) ? job.scale[n] : 0.f;   // padded channels come out as zeros
+    s_bias[i] = (i < Nt && n < p.Cout) ? job.bias[n] : 0.f;
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tmem_alloc(smem_u32(s_tmem), 256);           // two accumulator buffers of up to 128 columns
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  bool alive = true;
+
+  if (warp == 0) {
+    // ---- TMA producer -----------------------------------------------------------------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, issued = 0, issued_phase = 0;
+      for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
+        for (int c = 0; c < n_chunks && alive; ++c) {
+          alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+          if (!alive) break;
+          issued |= 1u << stage;
+          issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
+          mbar_expect_tx(bar_a_full + 8 * stage, 2 * kPwATile);
+          const uint32_t dst = smem_u32(smem) + stage * stage_bytes;
+          const int pix = (int)(job.in_version * p.ver_pixels) + tile * 128;
+          tma_load_3d(dst, &in_map, bar_a_full + 8 * stage, c * kPwChunk, 0, pix);             // hi
+          tma_load_3d(dst + kPwATile, &in_map, bar_a_full + 8 * stage, c * kPwChunk, 1, pix);  // lo
+          if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      for (int i = 0; i < stages; ++i)             // copies in flight must land before the CTA exits
+        if (issued & (1u << i)) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_a_full + 8 * i, (issued_phase >> i) & 1u) && clock64() - t0 < kWaitLimitCycles) {}
+        }
+    }
+  } else if (warp >= 6) {
+    // ---- weight expanders: packed codes -> bfloat16 B tile (Nt rows x 64 channels, 128-byte swizzle)
+    const int et = tid - 6 * 32;                                // 0 .. 127
+    const int kpad = (p.Cin + 31) / 32 * 32;
+    const size_t wrow = (size_t)kpad * job.bits / 8;
+    const int units_per_row = kPwChunk / 8;                     // 8 units of 8 channels (16 bytes of bfloat16)
+    uint32_t stage = 0, phase = 0;
+    for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
+      for (int c = 0; c < n_chunks && alive; ++c) {
+        alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+        alive = __all_sync(0xffffffffu, alive);
+        if (!alive) break;
+        uint8_t* btile = smem + stage * stage_bytes + 2 * kPwATile;
+        for (int u = et; u < Nt * units_per_row; u += 128) {
+          const int nl = u / units_per_row, cu = u - nl * units_per_row;
+          const int n = n0 + nl, ch = c * kPwChunk + cu * 8;
+          uint32_t out[4] = {0u, 0u, 0u, 0u};
+          if (n < p.Cout && ch < p.Cin) {                       // Cin is a multiple of 8 here
+            const uint8_t* src = job.w + (size_t)n * wrow;
+            int code[8];
+            if (job.bits == 8) {
+              const uint2 raw = __ldg(reinterpret_cast<const uint2*>(src + ch));
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                code[j] = (int)(int8_t)(raw.x >> (8 * j));
+                code[4 + j] = (int)(int8_t)(raw.y >> (8 * j));
+              }
+            } else {
+              const uint32_t raw = __ldg(reinterpret_cast<const uint32_t*>(src + ch / 2));
+#pragma unroll
+              for (int j = 0; j < 8; ++j) code[j] = (int)(((raw >> (4 * j)) & 0xFu) ^ 8u) - 8;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              out[j] = (uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code[2 * j])) |
+                       ((uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code[2 * j + 1])) << 16);
+          }
+          *reinterpret_cast<uint4*>(btile + swizzle_off((uint32_t)(nl * 128 + cu * 16), 7u)) =
+              make_uint4(out[0], out[1], out[2], out[3]);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_b_full + 8 * stage);
+        if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  }
+  else if (warp == 1) {
+    // ---- MMA issuer ---------------------------------------------------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(Nt >> 3) << 17) | ((128u >> 4) << 24);
+      constexpr uint32_t DESC_HI = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // SBO 1024, version 1, 128-byte swizzle
+      constexpr uint32_t LBO_FIELD = 1u << 16;
+      uint32_t stage = 0, phase = 0;
+      int it = 0;
+      for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
+        const int buf = it & 1;
+        alive = mbar_wait(bar_acc_empty + 8 * buf, ((it >> 1) & 1) ^ 1u, s_abort, p.error_flag);
+        if (!alive) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 128);
+        uint32_t accumulate = 0;
+        for (int c = 0; c < n_chunks && alive; ++c) {
+          alive = mbar_wait(bar_a_full + 8 * stage, phase, s_abort, p.error_flag) &&
+                  mbar_wait(bar_b_full + 8 * stage, phase, s_abort, p.error_flag);
+          if (!alive) break;
+          tc_fence_after();
+          const uint32_t a_lo = ((smem_u32(smem) + stage * stage_bytes) >> 4) | LBO_FIELD;
+          const uint32_t b_lo = a_lo + ((2 * kPwATile) >> 4);
+          const int kmax = min(4, (p.Cs_in - c * kPwChunk) / 16);      // 16-channel steps that hold data
+#pragma unroll
+          for (int part = 0; part < 2; ++part) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              if (kk < kmax) {
+                const uint64_t adesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(a_lo + ((part * kPwATile + kk * 32) >> 4));
+                const uint64_t bdesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + ((kk * 32) >> 4));
+                umma_bf16(d_tmem, adesc, bdesc, idesc, accumulate);
+                accumulate = 1;
+              }
+            }
+          }
+          umma_commit(bar_empty + 8 * stage);
+          if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+        }
+        if (alive) umma_commit(bar_acc_full + 8 * buf);
+      }
+    }
+  } else {
+    // ---- epilogue: warp q owns TMEM lanes 32q .. 32q+31 = pixels 32q .. 32q+31 of the tile -----
+    const int q = warp & 3;
+    int it = 0;
+    for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
+      const int buf = it & 1;
+      alive = mbar_wait(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);
+      alive = __all_sync(0xffffffffu, alive);
+      if (!alive) break;
+      tc_fence_after();
+      const int pix = tile * 128 + q * 32 + lane;
+      const int yp = (pix / p.W) % (p.H + 2);
+      const bool store = pix < p.P;
+      const bool interior = yp >= 1 && yp <= p.H;
+      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(job.out) + (size_t)pix * (2 * p.Cs_out);
+      const __nv_bfloat16* res = job.res ? static_cast<const __nv_bfloat16*>(job.res) + (size_t)pix * (2 * p.Cs_out) : nullptr;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 128);
+      for (int c0 = 0; c0 < Nt; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(taddr + c0, v);
+        tmem_ld_wait();
+        const int n = n0 + c0;
+        if (!store || n >= p.Cs_out) continue;
+        uint32_t rh[8] = {0, 0, 0, 0, 0, 0, 0, 0}, rl[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        if (res && interior) {
+          const uint4 a0 = __ldg(reinterpret_cast<const uint4*>(res + n)), a1 = __ldg(reinterpret_cast<const uint4*>(res + n) + 1);
+          const uint4 l0v = __ldg(reinterpret_cast<const uint4*>(res + p.Cs_out + n)), l1v = __ldg(reinterpret_cast<const uint4*>(res + p.Cs_out + n) + 1);
+          rh[0] = a0.x; rh[1] = a0.y; rh[2] = a0.z; rh[3] = a0.w; rh[4] = a1.x; rh[5] = a1.y; rh[6] = a1.z; rh[7] = a1.w;
+          rl[0] = l0v.x; rl[1] = l0v.y; rl[2] = l0v.z; rl[3] = l0v.w; rl[4] = l1v.x; rl[5] = l1v.y; rl[6] = l1v.z; rl[7] = l1v.w;
+        }
+        uint32_t hi[8], lo[8];
+#pragma unroll
+        for (int e = 0; e < 16; e += 2) {
+          float u0 = 0.f, u1 = 0.f;
+          if (interior) {
+            u0 = fmaf(__uint_as_float(v[e]), s_scale[c0 + e], s_bias[c0 + e]);
+            u1 = fmaf(__uint_as_float(v[e + 1]), s_scale[c0 + e + 1], s_bias[c0 + e + 1]);
+            u0 += __uint_as_float(rh[e >> 1] << 16) + __uint_as_float(rl[e >> 1] << 16);
+            u1 += __uint_as_float(rh[e >> 1] & 0xFFFF0000u) + __uint_as_float(rl[e >> 1] & 0xFFFF0000u);
+            u0 = apply_act(u0, p.act);
+            u1 = apply_act(u1, p.act);
+          }
+          __nv_bfloat16 h0, l0, h1, l1;
+          split_bf16(u0, h0, l0);
+          split_bf16(u1, h1, l1);
+          hi[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+          lo[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+        }
+        uint4* oh = reinterpret_cast<uint4*>(out + n);
+        uint4* ol = reinterpret_cast<uint4*>(out + p.Cs_out + n);
+        oh[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        oh[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+        ol[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        ol[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+    }
+  }
+
+  // ---- teardown -------------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 256);
+  }
+}
+
+}  // namespace
+}  // namespace aiq

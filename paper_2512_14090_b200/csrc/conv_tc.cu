@@ -653,6 +653,72 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
 
 }  // namespace
 
+}  // namespace aiq
+
+#include "conv_pw_tc.cuh"
+
+namespace aiq {
+
+bool conv_pw_tc_eligible(const ConvGeom& g) {
+  if (g.in_is_nchw || g.act_format != ACT_SPLIT) return false;
+  if (g.ks != 1 || g.pad != 0 || g.stride != 1) return false;
+  if (g.Cin % 8 != 0 || g.Cin < 16) return false;
+  return true;
+}
+
+aiq_status_t conv_pw_tc_encode_map(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
+                                   void* map_out) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  // (channel within a half, hi | lo, pixel over all versions)
+  const cuuint64_t pixels = (cuuint64_t)n_versions * batch_capacity * (g.H + 2) * g.W;
+  cuuint64_t dims[3] = {(cuuint64_t)g.Cs_in, 2, pixels};
+  cuuint64_t strides[2] = {2ull * g.Cs_in, 4ull * g.Cs_in};
+  cuuint32_t box[3] = {(cuuint32_t)kPwChunk, 1u, 128u};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(slot_base),
+                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled (pointwise) failed with code %d", (int)r);
+  return AIQ_OK;
+}
+
+aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
+                               int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s) {
+  static int smem_limit = 0, n_sms = 0;
+  if (!smem_limit) {
+    int dev = 0;
+    AIQ_CUDA_TRY(cudaGetDevice(&dev));
+    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
+    AIQ_CUDA_TRY(cudaFuncSetAttribute(conv_pw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
+  }
+  PwParams p = {};
+  p.P = g.B * (g.H + 2) * g.W; p.H = g.H; p.W = g.W;
+  p.Cin = g.Cin; p.Cs_in = g.Cs_in; p.Cout = g.Cout; p.Cs_out = g.Cs_out;
+  p.Nt = g.Cs_out < 128 ? g.Cs_out : 128;
+  p.n_ntiles = (g.Cs_out + p.Nt - 1) / p.Nt;
+  p.act = g.act;
+  p.ver_pixels = (long long)batch_capacity * (g.H + 2) * g.W;
+  p.error_flag = error_flag;
+  int stages = 4;
+  while (stages > 2 && pw_smem_bytes(p.Nt, stages) + 1024 > smem_limit) --stages;
+  p.n_stages = stages;
+  const int smem_bytes = pw_smem_bytes(p.Nt, stages) + 1024;
+  const int n_tiles = (p.P + 127) / 128;
+  int ctas = n_sms / (n_jobs * p.n_ntiles);
+  if (ctas > n_tiles) ctas = n_tiles;
+  if (ctas < 1) ctas = 1;
+  const CUtensorMap& m = *static_cast<const CUtensorMap*>(map);
+  {
+    LaunchScope scope(AIQ_KERNEL_CONV_TC, s, 2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)g.Cin * n_jobs,
+                      weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W + (double)g.B * g.Ho * g.Wo * g.Cout));
+    conv_pw_tc_kernel<<<dim3(ctas, n_jobs * p.n_ntiles), kPwThreads, smem_bytes, s>>>(m, p, jobs_dev);
+  }
+  AIQ_LAUNCH_CHECK("conv_pw_tc");
+  return AIQ_OK;
+}
+
 bool conv_tc_eligible(const ConvGeom& g) {
   if (g.in_is_nchw || g.act_format != ACT_SPLIT) return false;
   if (!((g.ks == 3 && g.pad == 1) || (g.ks == 1 && g.pad == 0))) return false;

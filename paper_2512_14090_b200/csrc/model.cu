@@ -206,9 +206,15 @@ static ConvGeom make_geom(const aiq_model* m, const LayerInfo& li, int B) {
   return g;
 }
 
-static bool layer_on_tensor_cores(const aiq_model* m, const LayerInfo& li) {
-  return li.d.kind == AIQ_LAYER_CONV && conv_tc_eligible(make_geom(m, li, 1));
+// 0: float32 kernels only; 1: small-channel 3x3 / 1x1 tensor-core kernel; 2: pointwise tensor-core kernel
+static int layer_tensor_kind(const aiq_model* m, const LayerInfo& li) {
+  if (li.d.kind != AIQ_LAYER_CONV) return 0;
+  const ConvGeom g = make_geom(m, li, 1);
+  if (conv_tc_eligible(g)) return 1;
+  if (conv_pw_tc_eligible(g)) return 2;
+  return 0;
 }
+static bool layer_on_tensor_cores(const aiq_model* m, const LayerInfo& li) { return layer_tensor_kind(m, li) != 0; }
 
 static void assign_slots(aiq_model* m) {
   const int n = (int)m->layers.size();
@@ -437,6 +443,7 @@ struct alignas(64) TensorMapBytes { uint8_t b[128]; };   // storage of one CUten
 struct LayerPlan {
   int n_versions = 0;
   int n_tc = 0;                         // leading jobs that run on the tensor-core kernel
+  int tc_kind = 0;                      // which tensor-core kernel (see layer_tensor_kind)
   double weight_bytes = 0.0;            // packed weights + scales + biases over all jobs
   double weight_bytes_tc = 0.0;
   TensorMapBytes in_map;                // over the input slot (tensor-core layers)
@@ -511,8 +518,10 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
         }
       if (tc_layer) {
         const LayerInfo& src = m->layers[li.d.input];
-        aiq_status_t st = conv_tc_encode_map(make_geom(m, li, B), ws + wl.slot_off[src.slot], B,
-                                             plan.lp[li.d.input].n_versions, &lp.in_map);
+        lp.tc_kind = layer_tensor_kind(m, li);
+        aiq_status_t st = lp.tc_kind == 1
+            ? conv_tc_encode_map(make_geom(m, li, B), ws + wl.slot_off[src.slot], B, plan.lp[li.d.input].n_versions, &lp.in_map)
+            : conv_pw_tc_encode_map(make_geom(m, li, B), ws + wl.slot_off[src.slot], B, plan.lp[li.d.input].n_versions, &lp.in_map);
         if (st != AIQ_OK) return st;
       }
       for (int v : vorder) {
@@ -621,7 +630,9 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
       continue;
     }
     if (lp.n_tc > 0) {
-      st = launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream);
+      st = lp.tc_kind == 1
+          ? launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream)
+          : launch_conv_pw_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream);
       if (st != AIQ_OK) return st;
     }
     if (lp.n_versions > lp.n_tc) {
