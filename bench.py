@@ -459,8 +459,11 @@ def main():
     if rank == 0:
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                     ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
-                    dtype="f32", data="synthetic",
+                    dtype="bf16", data="synthetic",
                     config=dict(workload=WORKLOAD, images_per_rank=N_IMAGES, schemes=S, layers=L,
+                                arithmetic="conv layers: bf16 tensor-core products of integer weight codes with "
+                                           "activations held as hi + lo bfloat16 pairs, float32 accumulation; stem, "
+                                           "pooling and classifier in float32",
                                 chunk=chunk, l2="flushed between timed steps (256 MiB write)",
                                 step="fold + quantize bank (4/8/16/32 bits) + eval 21 schemes + AI",
                                 labels="arg-max of the all-32-bit scheme, computed by the library",
