@@ -1,5 +1,5 @@
 // Forward kernels on the float32 multiply-add path: dense convolution as an implicit GEMM,
-// depthwise 3x3, global average pool, arg-max + agreement count.
+// global average pool, arg-max + agreement count (the depthwise kernel lives in depthwise.cu).
 //
 // Every kernel takes an array of LayerJob records and covers all of them in one launch
 // (gridDim.z = job), so one launch evaluates a layer for every distinct weight choice a
@@ -304,78 +304,6 @@ aiq_status_t launch_conv_tile(const ConvGeom& g, const LayerJob* jobs, int n_job
 }
 
 // ---------------------------------------------------------------------------------------
-// Depthwise 3x3 on split tensors.  A block owns a slice of up to 128 channels and a tile
-// of padded output pixels; a lane owns 4 consecutive channels.
-// ---------------------------------------------------------------------------------------
-constexpr int kDwPixPerBlock = 64;
-
-template <int FMT>
-__global__ void __launch_bounds__(256)
-depthwise3x3_kernel(ConvGeom g, const LayerJob* __restrict__ jobs) {
-  const LayerJob job = jobs[blockIdx.z];
-  const int c_base = blockIdx.y * 128;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  __shared__ __align__(16) float wsm[9][128];
-  __shared__ __align__(16) float ssm[128], bsm[128];
-  const int wrow_bytes = 32 * job.bits / 8;            // K = 9 pads to 32 elements
-  for (int i = threadIdx.x; i < 9 * 128; i += blockDim.x) {
-    const int tap = i / 128, cl = i - tap * 128;
-    const int c = c_base + cl;
-    wsm[tap][cl] = c < g.Cout ? load_element(job.w + (size_t)c * wrow_bytes, tap, job.bits) : 0.f;
-  }
-  for (int i = threadIdx.x; i < 128; i += blockDim.x) {
-    const int c = c_base + i;
-    ssm[i] = c < g.Cout ? job.scale[c] : 0.f;
-    bsm[i] = c < g.Cout ? job.bias[c] : 0.f;
-  }
-  __syncthreads();
-  const int c = c_base + lane * 4;
-  if (c >= g.Cs_out) return;
-  const int rows_out = g.Ho + 2;
-  const int M = g.B * rows_out * g.Wo;
-  const int Cs = g.Cs_out;                              // == Cs_in
-  const float4 sc = *reinterpret_cast<const float4*>(&ssm[lane * 4]);
-  const float4 bi = *reinterpret_cast<const float4*>(&bsm[lane * 4]);
-  const bool ok0 = c < g.Cout, ok1 = c + 1 < g.Cout, ok2 = c + 2 < g.Cout, ok3 = c + 3 < g.Cout;
-  for (int pi = warp; pi < kDwPixPerBlock; pi += 8) {
-    const int p = blockIdx.x * kDwPixPerBlock + pi;
-    if (p >= M) break;
-    const int b = p / (rows_out * g.Wo);
-    const int rem = p - b * (rows_out * g.Wo);
-    const int oyp = rem / g.Wo, ox = rem - (rem / g.Wo) * g.Wo;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (oyp >= 1 && oyp <= g.Ho) {
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int r = 0; r < 3; ++r) {
-        const int iy = (oyp - 1) * g.stride - 1 + r;
-        if (iy < 0 || iy >= g.H) continue;
-#pragma unroll
-        for (int t = 0; t < 3; ++t) {
-          const int ix = ox * g.stride - 1 + t;
-          if (ix < 0 || ix >= g.W) continue;
-          const float4 xv = act_load4<FMT>(job.in, (size_t)(b * (g.H + 2) + iy + 1) * g.W + ix, c, Cs);
-          const float4 wv = *reinterpret_cast<const float4*>(&wsm[r * 3 + t][lane * 4]);
-          acc.x = fmaf(xv.x, wv.x, acc.x);
-          acc.y = fmaf(xv.y, wv.y, acc.y);
-          acc.z = fmaf(xv.z, wv.z, acc.z);
-          acc.w = fmaf(xv.w, wv.w, acc.w);
-        }
-      }
-      float4 u = make_float4(fmaf(acc.x, sc.x, bi.x), fmaf(acc.y, sc.y, bi.y), fmaf(acc.z, sc.z, bi.z),
-                             fmaf(acc.w, sc.w, bi.w));
-      if (job.res) {
-        const float4 rr = act_load4<FMT>(job.res, (size_t)p, c, Cs);
-        u.x += rr.x; u.y += rr.y; u.z += rr.z; u.w += rr.w;
-      }
-      v = make_float4(ok0 ? apply_act(u.x, g.act) : 0.f, ok1 ? apply_act(u.y, g.act) : 0.f,
-                      ok2 ? apply_act(u.z, g.act) : 0.f, ok3 ? apply_act(u.w, g.act) : 0.f);
-    }
-    act_store4<FMT>(job.out, (size_t)p, c, Cs, v);
-  }
-}
-
-// ---------------------------------------------------------------------------------------
 // Global average pool over the interior of a split tensor: pooled[b][c] float32
 // ---------------------------------------------------------------------------------------
 template <int FMT>
@@ -446,19 +374,6 @@ aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs
   if (bn == 64) return launch_conv_tile<128, 64, 8, 4>(g, jobs_dev, n_jobs, net_input, in_mode, weight_bytes, s);
   if (bn == 32) return launch_conv_tile<128, 32, 4, 4>(g, jobs_dev, n_jobs, net_input, in_mode, weight_bytes, s);
   return launch_conv_tile<256, 16, 4, 4>(g, jobs_dev, n_jobs, net_input, in_mode, weight_bytes, s);
-}
-
-aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
-                              const float* /*net_input*/, double weight_bytes, cudaStream_t s) {
-  const int M = g.B * (g.Ho + 2) * g.Wo;
-  dim3 grid((M + kDwPixPerBlock - 1) / kDwPixPerBlock, (g.Cs_out + 127) / 128, n_jobs);
-  LaunchScope scope(AIQ_KERNEL_DEPTHWISE, s, 18.0 * g.B * g.Ho * g.Wo * g.Cout * n_jobs,
-                    weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
-                                                   (double)g.B * g.Ho * g.Wo * g.Cout));
-  if (g.act_format == ACT_SPLIT) depthwise3x3_kernel<ACT_SPLIT><<<grid, 256, 0, s>>>(g, jobs_dev);
-  else depthwise3x3_kernel<ACT_F32><<<grid, 256, 0, s>>>(g, jobs_dev);
-  AIQ_LAUNCH_CHECK("depthwise3x3");
-  return AIQ_OK;
 }
 
 aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int H, int W, int C, int act_format,
