@@ -224,8 +224,11 @@ def run_kernel_sweep(args):
                 e1.record()
                 torch.cuda.synchronize()
                 ms = e0.elapsed_time(e1) / n
+                aiq.aiq_profile_start()
+                model.aiq_forward(scheme, xb, logits=logits, workspace=wsb)
+                kinds = {k: round(v["ms"], 4) for k, v in aiq.aiq_profile_stop().items() if v["launches"]}
                 print(json.dumps(dict(workload="forward", model=name, batch=B, ms=ms, images_per_s=B / (ms * 1e-3),
-                                      launches=aiq.aiq_last_call_stats()["kernel_launches"])), flush=True)
+                                      launches=aiq.aiq_last_call_stats()["kernel_launches"], kernel_ms=kinds)), flush=True)
             model.close()
         return
     if args.workload == "quantize":

@@ -19,7 +19,7 @@ namespace aiq {
 namespace {
 
 constexpr int kDwThreads = 256;
-constexpr int kDwCols = 4;        // output columns per thread
+constexpr int kDwCols = 2;        // output columns per thread
 
 template <int FMT>
 __device__ __forceinline__ void load8(const void* __restrict__ base, size_t pixel, int c, int Cs, float* v) {
@@ -63,7 +63,7 @@ __device__ __forceinline__ void store8(void* __restrict__ base, size_t pixel, in
 }
 
 template <int FMT, int STRIDE>
-__global__ void __launch_bounds__(kDwThreads)
+__global__ void __launch_bounds__(kDwThreads, 4)
 depthwise3x3_kernel(ConvGeom g, const LayerJob* __restrict__ jobs) {
   extern __shared__ __align__(16) float dsm[];          // [9][Cs] weights, [Cs] scale, [Cs] bias
   const LayerJob job = jobs[blockIdx.y];
@@ -171,7 +171,7 @@ aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n
   if (smem > 48 * 1024) return set_error(AIQ_ERR_SHAPE, "depthwise: %d channels need %zu bytes of shared memory", g.Cout, smem);
   const long long n_items = (long long)g.B * (g.Ho + 2) * ((g.Wo + kDwCols - 1) / kDwCols) * (Cs / 8);
   long long blocks = (n_items + kDwThreads - 1) / kDwThreads;
-  const long long cap = (long long)n_sms * 8;                 // persistent: a few blocks per SM per job
+  const long long cap = (long long)n_sms * 4;                 // persistent: as many blocks as are resident (4 per SM)
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   dim3 grid((unsigned)blocks, n_jobs);
