@@ -105,7 +105,7 @@ struct LayerJob {
   int32_t bits;
   int32_t label_slot;   // head jobs: index of the count / prediction row
   int32_t in_version;   // index of `in` along the version dimension of its slot
-  int32_t pad_;
+  int32_t out_version;  // index of `out` along the version dimension of its slot
 };
 
 struct ConvGeom {
@@ -146,7 +146,10 @@ aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* 
 bool conv_pw_tc_eligible(const ConvGeom& g);
 aiq_status_t conv_pw_tc_encode_map(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
                                    void* map_out);
-aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
+// store map over the output slot: dims (Cs_out, 2, pixels per version, versions)
+aiq_status_t conv_pw_tc_encode_out_map(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
+                                       void* map_out);
+aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const void* out_map, const LayerJob* jobs_dev, int n_jobs,
                                int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s);
 // pooled[b][c] = mean over the H x W interior of a split tensor, per job (in -> out float32 [B][C])
 aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int H, int W, int C, int act_format,

@@ -42,12 +42,22 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 
 // shared memory: [stage: A_hi | A_lo | B] x n_stages, scale, bias, barriers, tmem ptr, abort flag
 __host__ __device__ inline int pw_stage_bytes(int Nt) { return 2 * kPwATile + Nt * kPwChunk * 2; }
+// output staging: per 64-channel group of the N tile one hi and one lo box of 128 pixels x 128 bytes
+__host__ __device__ inline int pw_out_groups(int Nt) { return (Nt + 63) / 64; }
+__host__ __device__ inline int pw_staging_bytes(int Nt) { return pw_out_groups(Nt) * 2 * kPwATile; }
 __host__ __device__ inline int pw_smem_bytes(int Nt, int stages) {
-  return stages * pw_stage_bytes(Nt) + 2 * 128 * 4 + (3 * stages + 4) * 8 + 16;
+  return stages * pw_stage_bytes(Nt) + pw_staging_bytes(Nt) + 2 * 128 * 4 + (3 * stages + 4) * 8 + 16;
+}
+
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+               : "memory");
 }
 
 __global__ void __launch_bounds__(kPwThreads, 1)
-conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, PwParams p, const LayerJob* __restrict__ jobs) {
+conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_constant__ CUtensorMap out_map, PwParams p,
+                  const LayerJob* __restrict__ jobs) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int job_idx = blockIdx.y / p.n_ntiles, ntile = blockIdx.y - job_idx * p.n_ntiles;
@@ -56,7 +66,8 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, PwParams p, const 
   const int stages = p.n_stages, Nt = p.Nt, n0 = ntile * Nt;
   const int stage_bytes = pw_stage_bytes(Nt);
 
-  float* s_scale = reinterpret_cast<float*>(smem + stages * stage_bytes);
+  uint8_t* staging = smem + stages * stage_bytes;            // 1024-aligned: every stage is a multiple of 2 KB
+  float* s_scale = reinterpret_cast<float*>(staging + pw_staging_bytes(Nt));
   float* s_bias = s_scale + 128;
   uint64_t* bars = reinterpret_cast<uint64_t*>(s_bias + 128);
   const uint32_t bar_a_full = smem_u32(bars);               // TMA bytes of a stage have landed
@@ -125,41 +136,66 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, PwParams p, const 
     }
   } else if (warp >= 6) {
     // ---- weight expanders: packed codes -> bfloat16 B tile (Nt rows x 64 channels, 128-byte swizzle)
+    // The packed words of a chunk are the same for every pixel tile and come from L2; they are
+    // fetched one chunk ahead into registers so that their latency hides behind the expansion of
+    // the current chunk and the wait for a free stage.
     const int et = tid - 6 * 32;                                // 0 .. 127
     const int kpad = (p.Cin + 31) / 32 * 32;
     const size_t wrow = (size_t)kpad * job.bits / 8;
-    const int units_per_row = kPwChunk / 8;                     // 8 units of 8 channels (16 bytes of bfloat16)
+    constexpr int UPR = kPwChunk / 8;                           // 8 units of 8 channels per row and chunk
+    constexpr int UPT = 128 * UPR / 128;                        // units per thread at Nt = 128: 8
+    const int n_units = Nt * UPR;
+    auto fetch = [&](int c, uint2* raw) {
+#pragma unroll
+      for (int i = 0; i < UPT; ++i) {
+        const int u = et + i * 128;
+        const int nl = u / UPR, cu = u - nl * UPR;
+        const int n = n0 + nl, ch = c * kPwChunk + cu * 8;
+        raw[i] = make_uint2(0u, 0u);
+        if (u < n_units && n < p.Cout && ch < p.Cin) {          // Cin is a multiple of 8 here
+          const uint8_t* src = job.w + (size_t)n * wrow;
+          if (job.bits == 8) raw[i] = __ldg(reinterpret_cast<const uint2*>(src + ch));
+          else raw[i].x = __ldg(reinterpret_cast<const uint32_t*>(src + ch / 2));
+        }
+      }
+    };
+    uint2 cur[UPT], nxt[UPT];
+    fetch(0, cur);
     uint32_t stage = 0, phase = 0;
     for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
       for (int c = 0; c < n_chunks && alive; ++c) {
+        fetch(c + 1 < n_chunks ? c + 1 : 0, nxt);               // next chunk (of this or the next tile)
         alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
         alive = __all_sync(0xffffffffu, alive);
         if (!alive) break;
         uint8_t* btile = smem + stage * stage_bytes + 2 * kPwATile;
-        for (int u = et; u < Nt * units_per_row; u += 128) {
-          const int nl = u / units_per_row, cu = u - nl * units_per_row;
-          const int n = n0 + nl, ch = c * kPwChunk + cu * 8;
-          uint32_t out[4] = {0u, 0u, 0u, 0u};
-          if (n < p.Cout && ch < p.Cin) {                       // Cin is a multiple of 8 here
-            const uint8_t* src = job.w + (size_t)n * wrow;
-            int code[8];
-            if (job.bits == 8) {
-              const uint2 raw = __ldg(reinterpret_cast<const uint2*>(src + ch));
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                code[j] = (int)(int8_t)(raw.x >> (8 * j));
-                code[4 + j] = (int)(int8_t)(raw.y >> (8 * j));
-              }
-            } else {
-              const uint32_t raw = __ldg(reinterpret_cast<const uint32_t*>(src + ch / 2));
+        for (int i = 0; i < UPT; ++i) {
+          const int u = et + i * 128;
+          if (u >= n_units) break;
+          const int nl = u / UPR, cu = u - nl * UPR;
+          int code[8];
+          if (job.bits == 8) {
 #pragma unroll
-              for (int j = 0; j < 8; ++j) code[j] = (int)(((raw >> (4 * j)) & 0xFu) ^ 8u) - 8;
+            for (int j = 0; j < 4; ++j) {
+              code[j] = (int)(int8_t)(cur[i].x >> (8 * j));
+              code[4 + j] = (int)(int8_t)(cur[i].y >> (8 * j));
             }
+          } else {
+            // a unit that was not fetched (padding) holds zero words, which must stay zero codes
+            const uint32_t raw = cur[i].x;
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              out[j] = (uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code[2 * j])) |
-                       ((uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code[2 * j + 1])) << 16);
+            for (int j = 0; j < 8; ++j) code[j] = (int)(((raw >> (4 * j)) & 0xFu) ^ 8u) - 8;
+            if (n0 + nl >= p.Cout || c * kPwChunk + cu * 8 >= p.Cin) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) code[j] = 0;
+            }
           }
+          uint32_t out[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            out[j] = (uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code[2 * j])) |
+                     ((uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code[2 * j + 1])) << 16);
           *reinterpret_cast<uint4*>(btile + swizzle_off((uint32_t)(nl * 128 + cu * 16), 7u)) =
               make_uint4(out[0], out[1], out[2], out[3]);
         }
@@ -167,6 +203,8 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, PwParams p, const 
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_b_full + 8 * stage);
         if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+#pragma unroll
+        for (int i = 0; i < UPT; ++i) cur[i] = nxt[i];
       }
     }
   }
@@ -217,25 +255,27 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, PwParams p, const 
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
       const int buf = it & 1;
-      alive = mbar_wait(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);
-      alive = __all_sync(0xffffffffu, alive);
+      alive = mbar_wait(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);   // false => *s_abort is set
+      // the previous tile's stores must have finished reading the staging tiles
+      if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      asm volatile("bar.sync 1, 128;" ::: "memory");     // every epilogue thread, unconditionally
+      alive = *s_abort == 0;                             // the same answer in all four warps
       if (!alive) break;
       tc_fence_after();
-      const int pix = tile * 128 + q * 32 + lane;
+      const int m = q * 32 + lane;                       // pixel row of the tile
+      const int pix = tile * 128 + m;
       const int yp = (pix / p.W) % (p.H + 2);
-      const bool store = pix < p.P;
-      const bool interior = yp >= 1 && yp <= p.H;
-      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(job.out) + (size_t)pix * (2 * p.Cs_out);
-      const __nv_bfloat16* res = job.res ? static_cast<const __nv_bfloat16*>(job.res) + (size_t)pix * (2 * p.Cs_out) : nullptr;
+      const bool interior = pix < p.P && yp >= 1 && yp <= p.H;
+      const __nv_bfloat16* res = (job.res && interior)
+          ? static_cast<const __nv_bfloat16*>(job.res) + (size_t)pix * (2 * p.Cs_out) : nullptr;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 128);
       for (int c0 = 0; c0 < Nt; c0 += 16) {
         uint32_t v[16];
         tmem_ld16(taddr + c0, v);
         tmem_ld_wait();
         const int n = n0 + c0;
-        if (!store || n >= p.Cs_out) continue;
         uint32_t rh[8] = {0, 0, 0, 0, 0, 0, 0, 0}, rl[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        if (res && interior) {
+        if (res && n < p.Cs_out) {
           const uint4 a0 = __ldg(reinterpret_cast<const uint4*>(res + n)), a1 = __ldg(reinterpret_cast<const uint4*>(res + n) + 1);
           const uint4 l0v = __ldg(reinterpret_cast<const uint4*>(res + p.Cs_out + n)), l1v = __ldg(reinterpret_cast<const uint4*>(res + p.Cs_out + n) + 1);
           rh[0] = a0.x; rh[1] = a0.y; rh[2] = a0.z; rh[3] = a0.w; rh[4] = a1.x; rh[5] = a1.y; rh[6] = a1.z; rh[7] = a1.w;
@@ -259,17 +299,35 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, PwParams p, const 
           hi[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
           lo[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
         }
-        uint4* oh = reinterpret_cast<uint4*>(out + n);
-        uint4* ol = reinterpret_cast<uint4*>(out + p.Cs_out + n);
-        oh[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        oh[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-        ol[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        ol[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        // staging tile (group, part): 128 rows x 128 bytes, 16-byte units XOR-swizzled by the row
+        // exactly as the 128-byte-swizzle tensor map expects
+        uint8_t* tile_hi = staging + (c0 >> 6) * 2 * kPwATile;
+        uint8_t* tile_lo = tile_hi + kPwATile;
+        const int u0i = (c0 & 63) >> 3;                  // first of the two units of these 16 channels
+        const uint32_t row = (uint32_t)m * 128u;
+        *reinterpret_cast<uint4*>(tile_hi + row + (((u0i) ^ (m & 7)) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(tile_hi + row + (((u0i + 1) ^ (m & 7)) << 4)) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+        *reinterpret_cast<uint4*>(tile_lo + row + (((u0i) ^ (m & 7)) << 4)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        *reinterpret_cast<uint4*>(tile_lo + row + (((u0i + 1) ^ (m & 7)) << 4)) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
       }
+      // the accumulator is drained: hand it back, then publish the staging tiles and store them
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (warp == 2 && lane == 0) {
+        for (int gi = 0; gi < pw_out_groups(Nt); ++gi) {
+          if (n0 + gi * 64 >= p.Cs_out) break;
+          // channels past Cs_out and pixels past the slot's capacity are clipped by the tensor map
+          tma_store_4d(&out_map, smem_u32(staging) + gi * 2 * kPwATile, n0 + gi * 64, 0, tile * 128, job.out_version);
+          tma_store_4d(&out_map, smem_u32(staging) + gi * 2 * kPwATile + kPwATile, n0 + gi * 64, 1, tile * 128, job.out_version);
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
     }
+    // all stores must have left shared memory (and be complete) before the CTA retires
+    if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   // ---- teardown -------------------------------------------------------------------------------

@@ -683,7 +683,25 @@ aiq_status_t conv_pw_tc_encode_map(const ConvGeom& g, const void* slot_base, int
   return AIQ_OK;
 }
 
-aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
+aiq_status_t conv_pw_tc_encode_out_map(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
+                                       void* map_out) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  // (channel within a half, hi | lo, pixel of a version, version): stores are clipped at the
+  // padded channel count and at the capacity of a version
+  const cuuint64_t pixels = (cuuint64_t)batch_capacity * (g.Ho + 2) * g.Wo;
+  cuuint64_t dims[4] = {(cuuint64_t)g.Cs_out, 2, pixels, (cuuint64_t)n_versions};
+  cuuint64_t strides[3] = {2ull * g.Cs_out, 4ull * g.Cs_out, 4ull * g.Cs_out * pixels};
+  cuuint32_t box[4] = {(cuuint32_t)kPwChunk, 1u, 128u, 1u};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = enc(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(slot_base),
+                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled (pointwise store) failed with code %d", (int)r);
+  return AIQ_OK;
+}
+
+aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const void* out_map, const LayerJob* jobs_dev, int n_jobs,
                                int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s) {
   static int smem_limit = 0, n_sms = 0;
   if (!smem_limit) {
@@ -703,6 +721,8 @@ aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const LayerJo
   p.error_flag = error_flag;
   int stages = 4;
   while (stages > 2 && pw_smem_bytes(p.Nt, stages) + 1024 > smem_limit) --stages;
+  if (pw_smem_bytes(p.Nt, stages) + 1024 > smem_limit)
+    return set_error(AIQ_ERR_SHAPE, "conv_pw_tc: %d bytes of shared memory needed", pw_smem_bytes(p.Nt, stages) + 1024);
   p.n_stages = stages;
   const int smem_bytes = pw_smem_bytes(p.Nt, stages) + 1024;
   const int n_tiles = (p.P + 127) / 128;
@@ -710,10 +730,11 @@ aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const LayerJo
   if (ctas > n_tiles) ctas = n_tiles;
   if (ctas < 1) ctas = 1;
   const CUtensorMap& m = *static_cast<const CUtensorMap*>(map);
+  const CUtensorMap& mo = *static_cast<const CUtensorMap*>(out_map);
   {
     LaunchScope scope(AIQ_KERNEL_CONV_TC, s, 2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)g.Cin * n_jobs,
                       weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W + (double)g.B * g.Ho * g.Wo * g.Cout));
-    conv_pw_tc_kernel<<<dim3(ctas, n_jobs * p.n_ntiles), kPwThreads, smem_bytes, s>>>(m, p, jobs_dev);
+    conv_pw_tc_kernel<<<dim3(ctas, n_jobs * p.n_ntiles), kPwThreads, smem_bytes, s>>>(m, mo, p, jobs_dev);
   }
   AIQ_LAUNCH_CHECK("conv_pw_tc");
   return AIQ_OK;

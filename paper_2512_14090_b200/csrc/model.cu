@@ -447,6 +447,7 @@ struct LayerPlan {
   double weight_bytes = 0.0;            // packed weights + scales + biases over all jobs
   double weight_bytes_tc = 0.0;
   TensorMapBytes in_map;                // over the input slot (tensor-core layers)
+  TensorMapBytes out_map;               // over the output slot (pointwise tensor-core layers)
   size_t job_first = 0;                 // index of the first job record of this layer
   // fc only
   int n_pool = 0;
@@ -523,6 +524,10 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
             ? conv_tc_encode_map(make_geom(m, li, B), ws + wl.slot_off[src.slot], B, plan.lp[li.d.input].n_versions, &lp.in_map)
             : conv_pw_tc_encode_map(make_geom(m, li, B), ws + wl.slot_off[src.slot], B, plan.lp[li.d.input].n_versions, &lp.in_map);
         if (st != AIQ_OK) return st;
+        if (lp.tc_kind == 2) {
+          st = conv_pw_tc_encode_out_map(make_geom(m, li, B), ws + wl.slot_off[li.slot], B, lp.n_versions, &lp.out_map);
+          if (st != AIQ_OK) return st;
+        }
       }
       for (int v : vorder) {
         LayerJob j = {};
@@ -532,6 +537,7 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
         j.res = li.d.residual >= 0 ? slot_ptr(li.d.residual, std::get<2>(keys[v])) : nullptr;
         j.out = slot_ptr(l, v);
         j.in_version = li.d.input >= 0 ? std::get<1>(keys[v]) : 0;
+        j.out_version = v;
         j.w = li.packed[bi];
         j.scale = li.scales[bi];
         j.bias = li.bias;
@@ -632,7 +638,7 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
     if (lp.n_tc > 0) {
       st = lp.tc_kind == 1
           ? launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream)
-          : launch_conv_pw_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream);
+          : launch_conv_pw_tc(g, &lp.in_map, &lp.out_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream);
       if (st != AIQ_OK) return st;
     }
     if (lp.n_versions > lp.n_tc) {
