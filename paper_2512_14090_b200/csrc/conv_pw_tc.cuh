@@ -209,8 +209,8 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
     }
   }
   else if (warp == 1) {
-    // ---- MMA issuer ---------------------------------------------------------------------------
-    if (lane == 0) {
+    // ---- MMA issuer: all 32 lanes converged, one elected lane issues (see umma_bf16) ----------
+    {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(Nt >> 3) << 17) | ((128u >> 4) << 24);
       constexpr uint32_t DESC_HI = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // SBO 1024, version 1, 128-byte swizzle
       constexpr uint32_t LBO_FIELD = 1u << 16;
@@ -218,14 +218,14 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
       int it = 0;
       for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
         const int buf = it & 1;
-        alive = mbar_wait(bar_acc_empty + 8 * buf, ((it >> 1) & 1) ^ 1u, s_abort, p.error_flag);
+        alive = mbar_wait_warp(bar_acc_empty + 8 * buf, ((it >> 1) & 1) ^ 1u, s_abort, p.error_flag);
         if (!alive) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 128);
         uint32_t accumulate = 0;
         for (int c = 0; c < n_chunks && alive; ++c) {
-          alive = mbar_wait(bar_a_full + 8 * stage, phase, s_abort, p.error_flag) &&
-                  mbar_wait(bar_b_full + 8 * stage, phase, s_abort, p.error_flag);
+          alive = mbar_wait_warp(bar_a_full + 8 * stage, phase, s_abort, p.error_flag) &&
+                  mbar_wait_warp(bar_b_full + 8 * stage, phase, s_abort, p.error_flag);
           if (!alive) break;
           tc_fence_after();
           const uint32_t a_lo = ((smem_u32(smem) + stage * stage_bytes) >> 4) | LBO_FIELD;

@@ -33,7 +33,7 @@ namespace aiq {
 
 namespace {
 
-constexpr int kTcThreads = 192;            // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
+constexpr int kTcThreads = 320;            // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
 constexpr int kRowsPerTile = 16;           // padded rows per tile
 constexpr int kColsPerTile = 8;
 constexpr int kBoxRows = kRowsPerTile + 2;
@@ -90,6 +90,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (error_flag) atomicExch(error_flag, 1);
   return false;
 }
+// bounded wait by a whole (converged) warp: the same answer in every lane
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               int32_t* error_flag) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, error_flag));
+}
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
                                             int c2, int c3) {
@@ -122,24 +127,48 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// The MMA-issuing warp runs its loop with all 32 lanes converged and lets one elected lane
+// issue each tensor-core instruction (elect.sync picks the same lane every time, so the
+// commits track the MMAs of that lane).  Converged code lets the compiler keep descriptors in
+// uniform registers; a loop inside `if (lane == 0)` measured 50 cycles per MMA issued, this
+// form 28 - 39, which matters here because the MMAs are small (8 - 32 cycles of math).
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "elect.sync _|q, 0xffffffff;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                           uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p, q;\n\t"
+      "elect.sync _|q, 0xffffffff;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
         "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* v) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr));
+}
+// v = hi + lo with hi = bf16_rn(v), lo = bf16_rn(v - hi), two values at a time (one packed
+// conversion per pair); the same roundings as split_bf16
+__device__ __forceinline__ void split_pair(float u0, float u1, uint32_t& hi2, uint32_t& lo2) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(u0, u1);
+  hi2 = *reinterpret_cast<const uint32_t*>(&h);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(u0 - __uint_as_float(hi2 << 16), u1 - __uint_as_float(hi2 & 0xFFFF0000u));
+  lo2 = *reinterpret_cast<const uint32_t*>(&l);
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -191,7 +220,7 @@ struct TcSmem {
 };
 
 template <int CS, int N, int KS, int STRIDE>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, (CS <= 32 && N <= 32) ? 2 : 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const LayerJob* __restrict__ jobs) {
   using L = TcLayout<CS, N>;
   using S = TcSmem<CS, N>;
@@ -237,7 +266,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_acc_full + 8 * i, 1);
-      mbar_init(bar_acc_empty + 8 * i, 4);     // one arrival per epilogue warp
+      mbar_init(bar_acc_empty + 8 * i, 8);     // one arrival per epilogue warp
     }
     mbar_init(bar_w, 1);
     *s_abort = 0;
@@ -354,7 +383,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
         }
     }
   } else if (warp == 1) {
-    if (lane == 0 && alive) {
+    if (alive) {                                   // all 32 lanes, converged (see umma_bf16)
       // instruction descriptor: D float32, A and B bfloat16, both K-major, M = 128, N
       constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
       // Shared-memory descriptors differ only in their start address, so the upper words are
@@ -368,7 +397,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       int it = 0;
       for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
         const int buf = it & 1;
-        alive = mbar_wait(bar_acc_empty + 8 * buf, ((it >> 1) & 1) ^ 1u, s_abort, p.error_flag);
+        alive = mbar_wait_warp(bar_acc_empty + 8 * buf, ((it >> 1) & 1) ^ 1u, s_abort, p.error_flag);
         if (!alive) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * N);
@@ -376,7 +405,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
         for (int t = T_FIRST; t <= T_LAST; ++t) {
           if (STRIDE == 1) {
             if (!alive) break;
-            alive = mbar_wait(bar_full + 8 * stage, phase, s_abort, p.error_flag);
+            alive = mbar_wait_warp(bar_full + 8 * stage, phase, s_abort, p.error_flag);
             if (!alive) break;
             tc_fence_after();
           }
@@ -386,7 +415,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
             uint32_t a_lo0 = a_lo1;
             if (STRIDE == 2) {                     // every tap has a stage of its own
               if (!alive) break;
-              alive = mbar_wait(bar_full + 8 * stage, phase, s_abort, p.error_flag);
+              alive = mbar_wait_warp(bar_full + 8 * stage, phase, s_abort, p.error_flag);
               if (!alive) break;
               tc_fence_after();
               a_lo0 = ((smem_u32(ring) + stage * L::STAGE_BYTES) >> 4) | LBO_FIELD;
@@ -419,24 +448,33 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       }
     }
   } else {
-    // Epilogue: warp q of the four owns TMEM lanes 32q .. 32q+31 (q = warp index mod 4), i.e.
-    // tile rows 4q .. 4q+3 (8 pixels each).  A lane owns one pixel for the arithmetic, but a
-    // pixel is only 4N bytes, so per-lane global accesses would touch 32 cache lines per
-    // instruction.  Instead each warp stages its 32 pixels in shared memory: the residual rows
-    // are fetched into the staging buffer with coalesced 16-byte accesses *before* the
-    // accumulator is waited for, the result overwrites them in place, and the finished rows
-    // leave with coalesced stores (a row of 8 pixels is 32N contiguous bytes).  16-byte units
-    // are XOR-swizzled so that both access patterns are free of bank conflicts.
+    // Epilogue: TMEM lanes 32q .. 32q+31 (tile rows 4q .. 4q+3, 8 pixels each) belong to the two
+    // warps with warp index mod 4 = q; warp h of the pair takes half of the output channels.
+    // The arithmetic of the epilogue (scale, bias, residual, activation, the split into two
+    // bfloat16) is a long dependent chain per tile, so it is spread over eight warps; with four
+    // the tensor cores waited for the epilogue more than half of the time.
+    // A lane owns one pixel for the arithmetic, but a pixel is only 4N bytes, so per-lane global
+    // accesses would touch 32 cache lines per instruction.  Instead the 32 pixels of a quarter
+    // are staged in shared memory: the residual rows are fetched into the staging buffer with
+    // coalesced 16-byte accesses *before* the accumulator is waited for, the result overwrites
+    // them in place, and the finished rows leave with coalesced stores (a row of 8 pixels is
+    // 32N contiguous bytes).  Each warp moves two of the quarter's four rows; two named-barrier
+    // syncs per tile order the pair (ids 1 .. 4, 64 threads).  16-byte units are XOR-swizzled
+    // so that both access patterns are free of bank conflicts.
     const int q = warp & 3;
+    const int h = (warp - 2) >> 2;
     const int m = q * 32 + lane;                       // row of the tile: pixel (g, wl)
-    const int g = m >> 3, wl = m & 7;
+    const int g = m >> 3;
     constexpr int PIXB = 4 * N;                        // bytes of one output pixel
     constexpr int UNITS = PIXB / 16;                   // 16-byte units per pixel (4, 8, 16)
     constexpr int KEY_SHIFT = PIXB < 128 ? 1 : 0;      // N = 16: two pixels share a 128-byte window
     constexpr int KEY_MASK = (UNITS < 8 ? UNITS : 8) - 1;
+    constexpr int CW = N >= 32 ? 16 : 8;               // accumulator columns per chunk
+    constexpr int NCH = N / (2 * CW);                  // chunks per warp (1, 1, 2)
     uint8_t* stg = smem + S::staging(stages, taps) + q * 32 * PIXB;
     uint8_t* my_row = stg + lane * PIXB;
     const int my_key = (lane >> KEY_SHIFT) & KEY_MASK;
+    const uint32_t pair_bar = 1u + (uint32_t)q;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
       const int buf = it & 1;
@@ -452,10 +490,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
         const int bb = b0 + img;
         return bb < p.B ? bb * (p.Ho + 2) + oy0 + (gi - img * rows_per_img) + 1 : -1;
       };
-      // (1) residual rows -> staging
+      // (1) residual rows -> staging (this warp's two rows of the quarter)
       if (job.res) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int ii = 0; ii < 2; ++ii) {
+          const int i = 2 * h + ii;
           const int jr = out_row(q * 4 + i);
           if (jr >= 0) {
             const uint4* src = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(job.res) +
@@ -467,10 +506,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
             }
           }
         }
-        __syncwarp();
       }
-      alive = mbar_wait(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);
-      alive = __all_sync(0xffffffffu, alive);     // the tensor-memory loads below need the whole warp
+      mbar_wait(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);   // false => *s_abort is set
+      // both warps of the pair, unconditionally: the partner's residual rows are in place and its
+      // stores of the previous tile have left the staging rows
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+      alive = *s_abort == 0;                      // the same answer in both warps of the pair
       if (!alive) break;
       tc_fence_after();
       bool interior = true;                       // stride 2 tiles hold interior rows only
@@ -481,54 +522,61 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       }
       const bool use_res = job.res != nullptr && interior;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * N);
+      uint32_t v[NCH][CW];
 #pragma unroll
-      for (int c0 = 0; c0 < N; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld16(taddr + c0, v);
-        tmem_ld_wait();
-        // 16-byte units of this pixel that hold columns c0 .. c0+15: two of hi, two of lo
-        const int uh = c0 / 8, ul = (N + c0) / 8;
-        uint4* ph0 = reinterpret_cast<uint4*>(my_row + (((uh) ^ my_key) << 4));
-        uint4* ph1 = reinterpret_cast<uint4*>(my_row + (((uh + 1) ^ my_key) << 4));
-        uint4* pl0 = reinterpret_cast<uint4*>(my_row + (((ul) ^ my_key) << 4));
-        uint4* pl1 = reinterpret_cast<uint4*>(my_row + (((ul + 1) ^ my_key) << 4));
-        uint32_t rh[8] = {0, 0, 0, 0, 0, 0, 0, 0}, rl[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        if (use_res) {
-          const uint4 a0 = *ph0, a1 = *ph1, l0v = *pl0, l1v = *pl1;
-          rh[0] = a0.x; rh[1] = a0.y; rh[2] = a0.z; rh[3] = a0.w; rh[4] = a1.x; rh[5] = a1.y; rh[6] = a1.z; rh[7] = a1.w;
-          rl[0] = l0v.x; rl[1] = l0v.y; rl[2] = l0v.z; rl[3] = l0v.w; rl[4] = l1v.x; rl[5] = l1v.y; rl[6] = l1v.z; rl[7] = l1v.w;
-        }
-        uint32_t hi[8], lo[8];
-#pragma unroll
-        for (int e = 0; e < 16; e += 2) {
-          float u0 = 0.f, u1 = 0.f;
-          if (interior) {
-            u0 = fmaf(__uint_as_float(v[e]), s_scale[c0 + e], s_bias[c0 + e]);
-            u1 = fmaf(__uint_as_float(v[e + 1]), s_scale[c0 + e + 1], s_bias[c0 + e + 1]);
-            // a bfloat16 is the upper half of a float: residual = hi + lo
-            u0 += __uint_as_float(rh[e >> 1] << 16) + __uint_as_float(rl[e >> 1] << 16);
-            u1 += __uint_as_float(rh[e >> 1] & 0xFFFF0000u) + __uint_as_float(rl[e >> 1] & 0xFFFF0000u);
-            u0 = apply_act(u0, p.act);
-            u1 = apply_act(u1, p.act);
-          }
-          __nv_bfloat16 h0, l0, h1, l1;
-          split_bf16(u0, h0, l0);
-          split_bf16(u1, h1, l1);
-          hi[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-          lo[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-        }
-        *ph0 = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *ph1 = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-        *pl0 = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        *pl1 = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+      for (int ch = 0; ch < NCH; ++ch) {
+        const int c0 = (2 * ch + h) * CW;
+        if (CW == 16) tmem_ld16(taddr + c0, v[ch]); else tmem_ld8(taddr + c0, v[ch]);
       }
-      // the accumulator is drained: hand it back before the stores
+      tmem_ld_wait();
+      // the accumulator values are in registers: hand the buffer back before the arithmetic
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+#pragma unroll
+      for (int ch = 0; ch < NCH; ++ch) {
+        const int c0 = (2 * ch + h) * CW;
+#pragma unroll
+        for (int u8 = 0; u8 < CW / 8; ++u8) {
+          // the 16-byte units of this pixel that hold columns c0 + 8 u8 .. + 7: one of hi, one of lo
+          const int cc = c0 + 8 * u8;
+          uint4* ph = reinterpret_cast<uint4*>(my_row + (((cc / 8) ^ my_key) << 4));
+          uint4* pl = reinterpret_cast<uint4*>(my_row + ((((N + cc) / 8) ^ my_key) << 4));
+          uint32_t rh[4] = {0, 0, 0, 0}, rl[4] = {0, 0, 0, 0};
+          if (use_res) {
+            const uint4 a = *ph, l = *pl;
+            rh[0] = a.x; rh[1] = a.y; rh[2] = a.z; rh[3] = a.w;
+            rl[0] = l.x; rl[1] = l.y; rl[2] = l.z; rl[3] = l.w;
+          }
+          const float4 sc0 = *reinterpret_cast<const float4*>(s_scale + cc), sc1 = *reinterpret_cast<const float4*>(s_scale + cc + 4);
+          const float4 bi0 = *reinterpret_cast<const float4*>(s_bias + cc), bi1 = *reinterpret_cast<const float4*>(s_bias + cc + 4);
+          const float sc[8] = {sc0.x, sc0.y, sc0.z, sc0.w, sc1.x, sc1.y, sc1.z, sc1.w};
+          const float bi[8] = {bi0.x, bi0.y, bi0.z, bi0.w, bi1.x, bi1.y, bi1.z, bi1.w};
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 8; e += 2) {
+            float u0 = 0.f, u1 = 0.f;
+            if (interior) {
+              u0 = fmaf(__uint_as_float(v[ch][8 * u8 + e]), sc[e], bi[e]);
+              u1 = fmaf(__uint_as_float(v[ch][8 * u8 + e + 1]), sc[e + 1], bi[e + 1]);
+              // a bfloat16 is the upper half of a float: residual = hi + lo
+              u0 += __uint_as_float(rh[e >> 1] << 16) + __uint_as_float(rl[e >> 1] << 16);
+              u1 += __uint_as_float(rh[e >> 1] & 0xFFFF0000u) + __uint_as_float(rl[e >> 1] & 0xFFFF0000u);
+              u0 = apply_act(u0, p.act);
+              u1 = apply_act(u1, p.act);
+            }
+            split_pair(u0, u1, hi[e >> 1], lo[e >> 1]);
+          }
+          *ph = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *pl = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+      }
+      // every column of the quarter's rows is final once the partner is here too
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
       // (3) staging -> global, one row of 8 pixels (32N contiguous bytes) at a time
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int ii = 0; ii < 2; ++ii) {
+        const int i = 2 * h + ii;
         const int jr = out_row(q * 4 + i);
         if (jr >= 0) {
           uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(job.out) +
@@ -543,7 +591,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       if (STRIDE == 2) {
         // zero border rows of the output images this tile touches (rows 0 and Ho + 1)
         const bool top = oy0 == 0, bottom = oy0 + rows_per_img == p.Ho;
-        for (int img = q; img < ipt; img += 4) {
+        for (int img = q + 4 * h; img < ipt; img += 8) {
           const int bb = b0 + img;
           if (bb >= p.B) break;
           for (int side = 0; side < 2; ++side) {
@@ -555,7 +603,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
           }
         }
       }
-      __syncwarp();                                   // staging is reused by the next tile
+      __syncwarp();                                   // this warp's staging rows are reused by the next tile
     }
   }
 
@@ -602,8 +650,9 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
   // a tile's load -> MMA -> epilogue chain better than a deeper ring does, so prefer two
   // CTAs with at least 4 stages, then one with as many stages as fit (at most 6).
   const int sm_budget = smem_limit + 1024;                 // per-SM capacity = opt-in block limit + 1 KB
+  constexpr int occ_cap = (CS <= 32 && N <= 32) ? 2 : 1;   // what __launch_bounds__ of the kernel allows
   int stages = 0;
-  for (int want = 2; want >= 1 && !stages; --want) {
+  for (int want = occ_cap; want >= 1 && !stages; --want) {
     const int per_cta = sm_budget / want - 1024;           // every block also reserves 1 KB
     for (int st = 6; st >= (want > 1 ? 4 : 3); --st)
       if (S::total(st, taps) + 1024 <= per_cta && S::total(st, taps) + 1024 <= smem_limit) { stages = st; break; }
@@ -631,10 +680,10 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
     const int rbi = g.Ho > kRowsPerTile ? g.Ho / kRowsPerTile : 1;
     n_tiles = ((g.B + ipt - 1) / ipt) * rbi * (g.Wo / kColsPerTile);
   }
-  // resident CTAs per SM: shared memory, and at most two (6 warps of ~110 registers fill the
-  // register file of an SM sub-partition after two CTAs)
+  // resident CTAs per SM: shared memory, and at most two where the kernel is compiled for two
+  // (10 warps of up to 96 registers each), else one
   int occ = sm_budget / (smem_bytes + 1024);
-  occ = occ > 2 ? 2 : (occ < 1 ? 1 : occ);
+  occ = occ > occ_cap ? occ_cap : (occ < 1 ? 1 : occ);
   // All CTAs of the launch should be resident at once (a second wave would run nearly alone):
   // split the resident capacity evenly over the jobs, rounding down.
   int ctas = (n_sms * occ) / n_jobs;
