@@ -36,14 +36,88 @@ aiq_status_t launch_fold_bn(const float* W, const float* gamma, const float* bet
 }
 
 // ---------------------------------------------------------------------------------------
-// quantize + pack: one block per row.  A thread owns granules of 8 consecutive elements
-// (two float4 loads); up to CACHE granules per thread stay in registers between the
-// max-abs pass and the rounding pass, so a row of up to blockDim * 8 * CACHE elements is
-// read from memory once.
+// quantize + pack
 // ---------------------------------------------------------------------------------------
-template <int CACHE>
+// code = rint(w / s) with the IEEE quotient, without dividing.  A true division costs ~10
+// instructions, so the quotient is estimated as e = w * (1/s) inside one fused multiply-add
+// with the constant 768: the sum lies in [512, 1024), where a float32 has 14 fraction bits,
+// so the adder rounds e to the nearest multiple of 2^-14 and leaves that fixed-point number
+// in the mantissa.  e and the correctly rounded quotient differ by at most 2^-23 relative
+// (< 1.6e-5 absolute, |e| <= 128), so both round to the same integer unless the fixed-point
+// value sits exactly on k + 1/2 (e within 2^-15 of a tie; one element in 2^14).  Only then is
+// the exact division evaluated, which makes the result bit-identical to always dividing.
+// Codes cannot leave [-qmax, qmax]: |w| <= amax and s = fl(amax / qmax).
+struct RowQuantizer {
+  float s, rs, lo, hi;
+  bool estimate_ok;
+  __device__ __forceinline__ RowQuantizer(float amax, int bits) {
+    s = 1.0f; lo = 0.f; hi = 0.f;
+    if (bits <= 8) {
+      const float qmax = (float)((1 << (bits - 1)) - 1);
+      if (amax != 0.0f) s = __fdiv_rn(amax, qmax);
+      lo = -(float)(1 << (bits - 1));
+      hi = qmax;
+    }
+    estimate_ok = s >= 1e-30f;           // a tiny scale would overflow the reciprocal: always divide
+    rs = estimate_ok ? __frcp_rn(s) : 0.f;
+  }
+  __device__ __forceinline__ uint32_t code(float wv) const {
+    // 768 = 1.5 * 2^9: bits = 0x44000000 + 0x400000 + round(2^14 e); u = round(2^14 e) + 2^13
+    const uint32_t u = (uint32_t)__float_as_int(fmaf(wv, rs, 768.0f)) - 0x443FE000u;
+    uint32_t c = (uint32_t)((int32_t)u >> 14);                      // floor(e + 1/2)
+    if (!estimate_ok || (u & 16383u) == 0u)                          // on (or too close to) a tie
+      c = (uint32_t)(int)fminf(fmaxf(rintf(__fdiv_rn(wv, s)), lo), hi);
+    return c;
+  }
+};
+
+// 8 consecutive elements -> packed output at granule index gi of the row
+template <int BITS>
+__device__ __forceinline__ void store_granule(uint8_t* out_row, int gi, const float* val, const RowQuantizer& rq) {
+  if (BITS == 4) {
+    uint32_t word = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) word |= (rq.code(val[j]) & 0xFu) << (4 * j);
+    reinterpret_cast<uint32_t*>(out_row)[gi] = word;
+  } else if (BITS == 8) {
+    uint32_t w0 = 0, w1 = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      w0 |= (rq.code(val[j]) & 0xFFu) << (8 * j);
+      w1 |= (rq.code(val[j + 4]) & 0xFFu) << (8 * j);
+    }
+    reinterpret_cast<uint2*>(out_row)[gi] = make_uint2(w0, w1);
+  } else if (BITS == 16) {
+    __half2 h0 = __floats2half2_rn(val[0], val[1]);
+    __half2 h1 = __floats2half2_rn(val[2], val[3]);
+    __half2 h2 = __floats2half2_rn(val[4], val[5]);
+    __half2 h3 = __floats2half2_rn(val[6], val[7]);
+    uint4 o;
+    o.x = *reinterpret_cast<uint32_t*>(&h0);
+    o.y = *reinterpret_cast<uint32_t*>(&h1);
+    o.z = *reinterpret_cast<uint32_t*>(&h2);
+    o.w = *reinterpret_cast<uint32_t*>(&h3);
+    reinterpret_cast<uint4*>(out_row)[gi] = o;
+  } else {
+    float4* o = reinterpret_cast<float4*>(out_row) + 2 * (size_t)gi;
+    o[0] = make_float4(val[0], val[1], val[2], val[3]);
+    o[1] = make_float4(val[4], val[5], val[6], val[7]);
+  }
+}
+
+// max |v| as an integer maximum of the sign-stripped bit patterns: NaN and infinity have
+// the largest patterns, so they survive the reduction and the row maximum itself tells
+// whether the row holds a non-finite element.
+__device__ __forceinline__ uint32_t absbits(float v) { return (uint32_t)__float_as_int(v) & 0x7FFFFFFFu; }
+constexpr uint32_t kInfBits = 0x7F800000u;
+
+// --- general kernel: one block per row.  A thread owns granules of 8 consecutive elements
+// (two float4 loads); up to CACHE granules per thread stay in registers between the max-abs
+// pass and the rounding pass, so a row of up to blockDim * 8 * CACHE elements is read from
+// memory once.
+template <int CACHE, int BITS>
 __global__ void __launch_bounds__(256, CACHE == 1 ? 4 : 3)
-quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad, int bits,
+quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad,
                      uint8_t* __restrict__ packed, float* __restrict__ scales,
                      int32_t* __restrict__ nonfinite_flag) {
   const int n = blockIdx.x;
@@ -52,8 +126,7 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad, int bits,
   const bool vec_ok = ((K & 3) == 0) && ((((uintptr_t)row) & 15) == 0);
 
   float v[CACHE][8];
-  float amax = 0.0f;
-  float poison = 0.0f;           // stays 0 unless an element is NaN or infinite (x * 0 is then NaN)
+  uint32_t amax_bits = 0;
 
   auto load_granule = [&](int gi, float* dstv) {
     const int k0 = gi << 3;
@@ -74,10 +147,7 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad, int bits,
     if (gi < n_gran) {
       load_granule(gi, v[c]);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        poison = fmaf(v[c][j], 0.0f, poison);
-        amax = fmaxf(amax, fabsf(v[c][j]));
-      }
+      for (int j = 0; j < 8; ++j) amax_bits = max(amax_bits, absbits(v[c][j]));
     }
   }
   // rows longer than the register cache: stream the remainder (re-read in pass 2)
@@ -85,123 +155,184 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad, int bits,
     float t[8];
     load_granule(gi, t);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      poison = fmaf(t[j], 0.0f, poison);
-      amax = fmaxf(amax, fabsf(t[j]));
-    }
+    for (int j = 0; j < 8; ++j) amax_bits = max(amax_bits, absbits(t[j]));
   }
 
-  __shared__ float s_max[8];
-  __shared__ int s_bad;
-  if (threadIdx.x == 0) s_bad = 0;
+  __shared__ uint32_t s_max[8];
+  amax_bits = __reduce_max_sync(0xffffffffu, amax_bits);
+  if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax_bits;
   __syncthreads();
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-  if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
-  if (poison != 0.0f) s_bad = 1;                 // NaN compares unequal to everything
-  __syncthreads();
-  amax = 0.0f;
-  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) amax = fmaxf(amax, s_max[w]);
-  if (s_bad) {
+  amax_bits = 0;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) amax_bits = max(amax_bits, s_max[w]);
+  if (amax_bits >= kInfBits) {
     if (threadIdx.x == 0 && nonfinite_flag) *nonfinite_flag = 1;
     return;
   }
+  const RowQuantizer rq(__uint_as_float(amax_bits), BITS);
+  if (threadIdx.x == 0) scales[n] = rq.s;
 
-  float s = 1.0f;
-  float lo = 0.f, hi = 0.f;
-  if (bits <= 8) {
-    const float qmax = (float)((1 << (bits - 1)) - 1);
-    if (amax != 0.0f) s = __fdiv_rn(amax, qmax);
-    lo = -(float)(1 << (bits - 1));
-    hi = qmax;
-  }
-  if (threadIdx.x == 0) scales[n] = s;
-
-  uint8_t* out_row = packed + (size_t)n * ((size_t)Kpad * bits / 8);
-  // code = rint(w / s) with the IEEE quotient.  A true division costs ~10 instructions, so the
-  // quotient is first estimated as w * (1/s): the estimate and the correctly rounded quotient
-  // differ by at most 1.5 * 2^-23 relative, hence they round to the same integer unless the
-  // estimate lies within that distance of a tie.  Only then (about one element in 10^4) is
-  // the exact division evaluated, so the result is bit-identical to always dividing.
-  const bool estimate_ok = s >= 1e-30f;        // a tiny scale would overflow the reciprocal: always divide
-  const float rs = estimate_ok ? __frcp_rn(s) : 0.f;
-  // Rounding without the conversion unit: adding 1.5 * 2^23 rounds the estimate to the nearest
-  // integer (ties to even) in the adder, and leaves that integer, in two's complement, in the
-  // low mantissa bits of the sum.  |estimate| <= 128, far inside the range where this holds.
-  // Codes cannot leave [-qmax, qmax]: |w| <= amax and s = fl(amax / qmax).
-  auto code_of = [&](float wv) -> uint32_t {
-    const float tq = wv * rs;
-    const float m = tq + 12582912.0f;
-    const float q = m - 12582912.0f;
-    uint32_t code = (uint32_t)__float_as_int(m);
-    if (!estimate_ok || fabsf(fabsf(tq - q) - 0.5f) <= fabsf(tq) * 4.8e-7f)   // 2^-21: near a tie
-      code = (uint32_t)(int)fminf(fmaxf(rintf(__fdiv_rn(wv, s)), lo), hi);
-    return code;
-  };
-  auto store_granule = [&](int gi, const float* val) {
-    if (bits == 4) {
-      uint32_t word = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        word |= (code_of(val[j]) & 0xFu) << (4 * j);
-      }
-      reinterpret_cast<uint32_t*>(out_row)[gi] = word;
-    } else if (bits == 8) {
-      uint32_t w0 = 0, w1 = 0;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        w0 |= (code_of(val[j]) & 0xFFu) << (8 * j);
-        w1 |= (code_of(val[j + 4]) & 0xFFu) << (8 * j);
-      }
-      reinterpret_cast<uint2*>(out_row)[gi] = make_uint2(w0, w1);
-    } else if (bits == 16) {
-      __half2 h0 = __floats2half2_rn(val[0], val[1]);
-      __half2 h1 = __floats2half2_rn(val[2], val[3]);
-      __half2 h2 = __floats2half2_rn(val[4], val[5]);
-      __half2 h3 = __floats2half2_rn(val[6], val[7]);
-      uint4 o;
-      o.x = *reinterpret_cast<uint32_t*>(&h0);
-      o.y = *reinterpret_cast<uint32_t*>(&h1);
-      o.z = *reinterpret_cast<uint32_t*>(&h2);
-      o.w = *reinterpret_cast<uint32_t*>(&h3);
-      reinterpret_cast<uint4*>(out_row)[gi] = o;
-    } else {
-      float4* o = reinterpret_cast<float4*>(out_row) + 2 * (size_t)gi;
-      o[0] = make_float4(val[0], val[1], val[2], val[3]);
-      o[1] = make_float4(val[4], val[5], val[6], val[7]);
-    }
-  };
-
+  uint8_t* out_row = packed + (size_t)n * ((size_t)Kpad * BITS / 8);
 #pragma unroll
   for (int c = 0; c < CACHE; ++c) {
     const int gi = threadIdx.x + c * blockDim.x;
-    if (gi < n_gran) store_granule(gi, v[c]);
+    if (gi < n_gran) store_granule<BITS>(out_row, gi, v[c], rq);
   }
   for (int gi = threadIdx.x + CACHE * blockDim.x; gi < n_gran; gi += blockDim.x) {
     float t[8];
     load_granule(gi, t);
-    store_granule(gi, t);
+    store_granule<BITS>(out_row, gi, t, rq);
   }
+}
+
+// --- streaming kernel for large matrices (the roofline case): persistent blocks, every row
+// arrives in shared memory by one bulk copy issued kStreamStages rows ahead, so the memory
+// system stays busy while a block reduces, rounds and packs.  A row goes from shared memory
+// into registers once (the stage is refilled right after), is reduced with one block-wide
+// barrier and leaves as packed words.  Needs K % 32 == 0, 16-byte aligned rows and
+// K <= 8192 (4 granules of 8 elements per thread).
+constexpr int kStreamThreads = 256;
+constexpr int kStreamCache = 4;
+
+__device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < (1u << 26); ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;                          // bounded: a copy that never lands must not hang the GPU
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kStreamThreads, 2)
+quantize_stream_kernel(const float* __restrict__ W, int N, int K, uint8_t* __restrict__ packed,
+                       float* __restrict__ scales, int32_t* __restrict__ nonfinite_flag, int stages) {
+  extern __shared__ __align__(128) uint8_t qs[];
+  const uint32_t row_bytes_in = (uint32_t)K * 4u;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(qs + (size_t)stages * row_bytes_in);
+  __shared__ uint32_t s_max[2][8];
+  const int tid = threadIdx.x;
+  const int n_gran = K >> 3;
+  const int n_mine = (N - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+  const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
+  const uint32_t buf0 = (uint32_t)__cvta_generic_to_shared(qs);
+
+  auto issue = [&](int i) {              // row i of this block -> stage i % stages (thread 0)
+    const int st = i % stages;
+    const float* src = W + (size_t)(blockIdx.x + (size_t)i * gridDim.x) * K;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar0 + 8 * st), "r"(row_bytes_in) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(buf0 + st * row_bytes_in), "l"(reinterpret_cast<uint64_t>(src)), "r"(row_bytes_in), "r"(bar0 + 8 * st)
+                 : "memory");
+  };
+  if (tid == 0) {
+    for (int i = 0; i < stages; ++i)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar0 + 8 * i), "r"(1) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    for (int i = 0; i < stages && i < n_mine; ++i) issue(i);
+  }
+  __syncthreads();
+
+  for (int i = 0; i < n_mine; ++i) {
+    const int st = i % stages;
+    const int n = blockIdx.x + i * gridDim.x;
+    if (!stream_wait(bar0 + 8 * st, (uint32_t)(i / stages) & 1u)) {
+      if (nonfinite_flag) *nonfinite_flag = 2;
+      return;
+    }
+    const float* row = reinterpret_cast<const float*>(qs + (size_t)st * row_bytes_in);
+    float v[kStreamCache][8];
+    uint32_t amax_bits = 0;
+#pragma unroll
+    for (int c = 0; c < kStreamCache; ++c) {
+      const int gi = tid + c * kStreamThreads;
+      if (gi < n_gran) {
+        const float4 a = *reinterpret_cast<const float4*>(row + 8 * gi);
+        const float4 b = *reinterpret_cast<const float4*>(row + 8 * gi + 4);
+        v[c][0] = a.x; v[c][1] = a.y; v[c][2] = a.z; v[c][3] = a.w;
+        v[c][4] = b.x; v[c][5] = b.y; v[c][6] = b.z; v[c][7] = b.w;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) amax_bits = max(amax_bits, absbits(v[c][j]));
+      }
+    }
+    amax_bits = __reduce_max_sync(0xffffffffu, amax_bits);
+    if ((tid & 31) == 0) s_max[i & 1][tid >> 5] = amax_bits;
+    __syncthreads();                     // every thread holds its part of the row in registers
+    if (tid == 0 && i + stages < n_mine) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the reads above before the copy's writes
+      issue(i + stages);
+    }
+    amax_bits = 0;
+#pragma unroll
+    for (int w = 0; w < kStreamThreads / 32; ++w) amax_bits = max(amax_bits, s_max[i & 1][w]);
+    if (amax_bits >= kInfBits) {         // uniform over the block: the row is skipped
+      if (tid == 0 && nonfinite_flag) *nonfinite_flag = 1;
+      continue;
+    }
+    const RowQuantizer rq(__uint_as_float(amax_bits), BITS);
+    if (tid == 0) scales[n] = rq.s;
+    uint8_t* out_row = packed + (size_t)n * ((size_t)K * BITS / 8);
+#pragma unroll
+    for (int c = 0; c < kStreamCache; ++c) {
+      const int gi = tid + c * kStreamThreads;
+      if (gi < n_gran) store_granule<BITS>(out_row, gi, v[c], rq);
+    }
+  }
+}
+
+template <int BITS>
+aiq_status_t launch_quantize_bits(const float* W, int N, int K, void* packed, float* scales,
+                                  int32_t* nonfinite_flag, cudaStream_t s) {
+  const int Kpad = padded_k(K);
+  const int n_gran = Kpad / 8;
+  uint8_t* p = static_cast<uint8_t*>(packed);
+  LaunchScope scope(AIQ_KERNEL_QUANTIZE, s, 2.0 * N * K,
+                    4.0 * N * K + (double)N * row_bytes(K, BITS) + 4.0 * N);
+  static int n_sms = 0, smem_limit = 0;
+  if (!n_sms) {
+    int dev = 0;
+    AIQ_CUDA_TRY(cudaGetDevice(&dev));
+    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
+    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    AIQ_CUDA_TRY(cudaFuncSetAttribute(quantize_stream_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      smem_limit - 1024));   // the kernel also has static shared memory
+  }
+  const bool stream_ok = K % 32 == 0 && K >= 2048 && K <= kStreamThreads * 8 * kStreamCache &&
+                         N >= 4 * n_sms && ((uintptr_t)W & 15) == 0;
+  if (stream_ok) {
+    // two blocks per SM: half of the shared memory each, minus the per-block reserve
+    const int per_block = (smem_limit + 1024) / 2 - 2048;
+    int stages = per_block / (K * 4);
+    if (stages > 8) stages = 8;
+    if (stages >= 2) {
+      const int smem = stages * K * 4 + stages * 8;
+      quantize_stream_kernel<BITS><<<2 * n_sms, kStreamThreads, smem, s>>>(W, N, K, p, scales, nonfinite_flag, stages);
+      AIQ_LAUNCH_CHECK("quantize_stream");
+      return AIQ_OK;
+    }
+  }
+  int threads = 32;
+  while (threads < 256 && threads < n_gran) threads <<= 1;
+  if (n_gran <= threads) {
+    quantize_rows_kernel<1, BITS><<<N, threads, 0, s>>>(W, K, Kpad, p, scales, nonfinite_flag);
+  } else {
+    quantize_rows_kernel<4, BITS><<<N, threads, 0, s>>>(W, K, Kpad, p, scales, nonfinite_flag);
+  }
+  AIQ_LAUNCH_CHECK("quantize_rows");
+  return AIQ_OK;
 }
 
 aiq_status_t launch_quantize(const float* W, int N, int K, int bits, void* packed, float* scales,
                              int32_t* nonfinite_flag, cudaStream_t s) {
-  const int Kpad = padded_k(K);
-  const int n_gran = Kpad / 8;
-  int threads = 32;
-  while (threads < 256 && threads < n_gran) threads <<= 1;
-  uint8_t* p = static_cast<uint8_t*>(packed);
-  {
-    LaunchScope scope(AIQ_KERNEL_QUANTIZE, s, 2.0 * N * K,
-                      4.0 * N * K + (double)N * row_bytes(K, bits) + 4.0 * N);
-    if (n_gran <= threads) {
-      quantize_rows_kernel<1><<<N, threads, 0, s>>>(W, K, Kpad, bits, p, scales, nonfinite_flag);
-    } else {
-      quantize_rows_kernel<4><<<N, threads, 0, s>>>(W, K, Kpad, bits, p, scales, nonfinite_flag);
-    }
+  switch (bits) {
+    case 4: return launch_quantize_bits<4>(W, N, K, packed, scales, nonfinite_flag, s);
+    case 8: return launch_quantize_bits<8>(W, N, K, packed, scales, nonfinite_flag, s);
+    case 16: return launch_quantize_bits<16>(W, N, K, packed, scales, nonfinite_flag, s);
+    default: return launch_quantize_bits<32>(W, N, K, packed, scales, nonfinite_flag, s);
   }
-  AIQ_LAUNCH_CHECK("quantize_rows");
-  return AIQ_OK;
 }
 
 }  // namespace aiq

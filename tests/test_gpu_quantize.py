@@ -41,6 +41,47 @@ def test_quantize_bit_exact(bits, shape):
         assert codes.min() >= -(2 ** (bits - 1)) and codes.max() <= 2 ** (bits - 1) - 1
 
 
+@pytest.mark.parametrize("bits", [4, 8, 16, 32])
+@pytest.mark.parametrize("shape", [(700, 2048), (1203, 4096), (600, 8192), (1500, 2080)])
+def test_quantize_streaming_kernel_bit_exact(bits, shape):
+    """Large matrices (K % 32 == 0, 2048 <= K <= 8192, many rows) take the persistent
+    streaming kernel: several rows per block, a ragged last round, zero rows, rows made of
+    near-ties of the rounding, and wide ranges of row magnitudes."""
+    aiq = binding()
+    N, K = shape
+    rng = np.random.default_rng(N * 7 + K)
+    W = (rng.standard_normal(shape) * np.exp(rng.uniform(-12, 6, (N, 1)))).astype(np.float32)
+    W[1, :] = 0.0
+    W[2, ::3] = 0.0
+    qmax = np.float32(2 ** (min(bits, 8) - 1) - 1)
+    for r in range(5, N, 97):            # rows of near-ties: (k + 1/2) * s and its neighbours
+        amax = np.float32(rng.uniform(0.1, 3.0))
+        s = amax / qmax
+        k = rng.integers(-int(qmax) + 1, int(qmax) - 1, K).astype(np.float32) + np.float32(0.5)
+        w = (k * s).astype(np.float32)
+        pick = rng.integers(0, 3, K)
+        w = np.where(pick == 0, np.nextafter(w, np.float32(0.0)), np.where(pick == 1, np.nextafter(w, np.float32(np.inf) * np.sign(w)), w))
+        w[0] = amax
+        W[r] = w.astype(np.float32)
+    packed, scales, flag = _quantize_gpu(aiq, W, bits)
+    v, s = O.quantize_rows(W, bits)
+    assert flag == 0
+    assert np.array_equal(scales.view(np.uint32), s.view(np.uint32))
+    assert np.array_equal(packed, O.pack_rows(v, bits))
+
+
+def test_streaming_kernel_flags_nonfinite_rows():
+    aiq = binding()
+    W = np.ones((800, 2048), np.float32)
+    W[700, 2047] = np.nan
+    assert _quantize_gpu(aiq, W, 8)[2] == 1
+    W[700, 2047] = -np.inf
+    assert _quantize_gpu(aiq, W, 4)[2] == 1
+    W[700, 2047] = 2.0
+    packed, scales, flag = _quantize_gpu(aiq, W, 4)
+    assert flag == 0 and scales[700] == np.float32(2.0) / np.float32(7.0)
+
+
 def test_quantize_near_ties_follow_division():
     aiq = binding()
     rng = np.random.default_rng(11)
