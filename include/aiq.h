@@ -100,14 +100,21 @@ aiq_status_t aiq_quantize_layer(const float* W, int N, int K, int bits, void* pa
  * aiq_quantize_layer (device).  bias: device [N] or NULL.  x: device float32 [M][K]
  * row-major, 16-byte aligned; y: device float32 [M][N].  M >= 1.  Asynchronous on `stream`.
  *
- * Two kernels.  The plain one expands weights to float32 in registers and accumulates in
- * float32 (any shape, any bit-width).  For 4- / 8-bit weights, M <= 16, K a multiple of 512
- * and N*K >= 2^20 a faster one keeps the codes integer and uses the int8 tensor cores: the
- * activations of each group of 512 k become three int8 digits with a shared exponent
- * (21 bits below the group's largest |x|), the int32 sums are exact, and K-slices meet in y
- * through float atomics (run-to-run differences in the last bit).  It needs scratch memory:
- * pass `workspace` (device, 16-byte aligned) of at least aiq_qlinear_workspace_bytes(...)
- * bytes; with workspace == NULL, or where that function returns 0, the plain kernel runs.
+ * Three kernels.  The plain one expands weights to float32 in registers and accumulates in
+ * float32 (any shape, any bit-width).  For 4- / 8-bit weights two faster ones exist:
+ *   M <= 8, K a multiple of 512, N*K >= 2^20: the codes stay integer and feed the int8
+ *     warp-level tensor cores; the activations of each group of 512 k become three int8
+ *     digits with a shared exponent (21 bits below the group's largest |x|), the int32 sums
+ *     are exact.
+ *   M >= 9, K a multiple of 8, K >= 64, N >= 32: a tcgen05 GEMM with the weight matrix as the
+ *     MMA's M operand (codes expanded to bfloat16 in shared memory, exact) and the batch as
+ *     its N operand; the activations enter as the sum of two bfloat16 (relative rounding
+ *     2^-17), accumulation is float32.
+ * Both split K over thread blocks where the matrix has too few rows to fill the GPU; the
+ * partial sums then meet in y through float atomics (run-to-run differences in the last
+ * bit).  Both need scratch memory: pass `workspace` (device, 16-byte aligned) of at least
+ * aiq_qlinear_workspace_bytes(...) bytes; with workspace == NULL, or where that function
+ * returns 0, the plain kernel runs.
  */
 size_t aiq_qlinear_workspace_bytes(int N, int K, int bits, int M);
 aiq_status_t aiq_qlinear(const void* packed, const float* scales, const float* bias, int N,

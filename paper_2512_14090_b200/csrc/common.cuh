@@ -129,6 +129,12 @@ aiq_status_t launch_qlinear(const LayerJob* jobs_dev, const LayerJob* single_hos
 bool qlinear_mma_applicable(int N, int K, int bits, int M);
 size_t qlinear_mma_workspace_bytes(int K, int M);
 aiq_status_t launch_qlinear_mma(const LayerJob& job, int N, int K, int M, void* workspace, cudaStream_t s);
+// tcgen05 path of the linear layer (4- / 8-bit weights, M >= 9): weights as the MMA's M operand,
+// the batch as its N operand; needs workspace for the activations as two bfloat16 planes
+bool qlinear_tc_applicable(int N, int K, int bits, int M);
+size_t qlinear_tc_workspace_bytes(int K, int M);
+aiq_status_t launch_qlinear_tc(const LayerJob& job, int N, int K, int M, void* workspace, int32_t* error_flag,
+                               cudaStream_t s);
 // weight_bytes: packed weights + scales + biases of all jobs (for the profile's byte count)
 aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
                          const float* net_input, double weight_bytes, cudaStream_t s);

@@ -174,28 +174,8 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
           const int u = et + i * 128;
           if (u >= n_units) break;
           const int nl = u / UPR, cu = u - nl * UPR;
-          int code[8];
-          if (job.bits == 8) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              code[j] = (int)(int8_t)(cur[i].x >> (8 * j));
-              code[4 + j] = (int)(int8_t)(cur[i].y >> (8 * j));
-            }
-          } else {
-            // a unit that was not fetched (padding) holds zero words, which must stay zero codes
-            const uint32_t raw = cur[i].x;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) code[j] = (int)(((raw >> (4 * j)) & 0xFu) ^ 8u) - 8;
-            if (n0 + nl >= p.Cout || c * kPwChunk + cu * 8 >= p.Cin) {
-#pragma unroll
-              for (int j = 0; j < 8; ++j) code[j] = 0;
-            }
-          }
           uint32_t out[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            out[j] = (uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code[2 * j])) |
-                     ((uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code[2 * j + 1])) << 16);
+          expand8_bf16(cur[i], job.bits, out);   // a unit that was not fetched holds zero words = zero codes
           *reinterpret_cast<uint4*>(btile + swizzle_off((uint32_t)(nl * 128 + cu * 16), 7u)) =
               make_uint4(out[0], out[1], out[2], out[3]);
         }

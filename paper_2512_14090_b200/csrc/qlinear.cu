@@ -181,8 +181,10 @@ aiq_status_t launch_qlinear(const LayerJob* jobs_dev, const LayerJob* single_hos
 }  // namespace aiq
 
 extern "C" size_t aiq_qlinear_workspace_bytes(int N, int K, int bits, int M) {
-  if (N <= 0 || K <= 0 || M <= 0 || !aiq::qlinear_mma_applicable(N, K, bits, M)) return 0;
-  return aiq::qlinear_mma_workspace_bytes(K, M);
+  if (N <= 0 || K <= 0 || M <= 0) return 0;
+  if (aiq::qlinear_tc_applicable(N, K, bits, M)) return aiq::qlinear_tc_workspace_bytes(K, M);
+  if (aiq::qlinear_mma_applicable(N, K, bits, M)) return aiq::qlinear_mma_workspace_bytes(K, M);
+  return 0;
 }
 
 extern "C" aiq_status_t aiq_qlinear(const void* packed, const float* scales, const float* bias, int N,
@@ -203,8 +205,13 @@ extern "C" aiq_status_t aiq_qlinear(const void* packed, const float* scales, con
   job.scale = scales;
   job.bias = bias;
   job.bits = bits;
-  // the integer tensor-core kernel needs scratch for the converted activations
-  if (workspace && aiq::qlinear_mma_applicable(N, K, bits, M)) {
+  // the tensor-core kernels need scratch for the converted activations
+  if (workspace && aiq::qlinear_tc_applicable(N, K, bits, M)) {
+    if (((uintptr_t)workspace) & 15)
+      return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_qlinear: workspace not 16-byte aligned");
+    if (workspace_bytes >= aiq::qlinear_tc_workspace_bytes(K, M))
+      return aiq::launch_qlinear_tc(job, N, K, M, workspace, nullptr, (cudaStream_t)stream);
+  } else if (workspace && aiq::qlinear_mma_applicable(N, K, bits, M)) {
     if (((uintptr_t)workspace) & 15)
       return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_qlinear: workspace not 16-byte aligned");
     if (workspace_bytes >= aiq::qlinear_mma_workspace_bytes(K, M))

@@ -31,7 +31,11 @@ def _run(aiq, W, x, bits, bias=None, use_workspace=True):
                                    (1000, 1280, 5), (37, 100, 3), (5, 27, 2), (4096, 4096, 1),
                                    (2048, 4096, 4), (300, 2052, 7), (1, 1, 1),
                                    # shapes on the warp-level tensor-core path (K % 512 == 0, N*K >= 2^20)
-                                   (4100, 512, 16), (1000, 1536, 3), (2050, 1024, 9), (8192, 8192, 2)])
+                                   (4100, 512, 16), (1000, 1536, 3), (2050, 1024, 9), (8192, 8192, 2),
+                                   # batches on the tcgen05 path (M >= 9, K % 8 == 0): ragged N, K and M tails,
+                                   # several batch blocks, K split over CTAs
+                                   (4096, 4096, 256), (1280, 320, 256), (1000, 1280, 37), (2050, 1024, 300),
+                                   (130, 72, 16), (33, 64, 9), (4100, 520, 64)])
 def test_qlinear_matches_oracle(bits, N, K, M):
     aiq = binding()
     W, x = gen_linear_case(N, K, M, seed=3234 + N + K + M)
@@ -50,7 +54,7 @@ def test_qlinear_exact_on_integers(bits):
     aiq = binding()
     rng = np.random.default_rng(1)
     qmax = 2 ** (bits - 1) - 1
-    for shape_w, m in (((96, 200), 4), ((2176, 512), 5)):      # plain kernel / tensor-core kernel
+    for shape_w, m in (((96, 200), 4), ((2176, 512), 5), ((300, 520), 20)):   # plain / int8 warp-level / tcgen05
         W = rng.integers(-qmax, qmax + 1, shape_w).astype(np.float32)
         W[:, 0] = qmax
         x = rng.integers(-8, 9, (m, shape_w[1])).astype(np.float32)
