@@ -165,8 +165,7 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
     for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
       for (int c = 0; c < n_chunks && alive; ++c) {
         fetch(c + 1 < n_chunks ? c + 1 : 0, nxt);               // next chunk (of this or the next tile)
-        alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
-        alive = __all_sync(0xffffffffu, alive);
+        alive = mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
         if (!alive) break;
         uint8_t* btile = smem + stage * stage_bytes + 2 * kPwATile;
 #pragma unroll
@@ -235,7 +234,7 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
       const int buf = it & 1;
-      alive = mbar_wait(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);   // false => *s_abort is set
+      alive = mbar_wait_warp(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);   // false => *s_abort is set
       // the previous tile's stores must have finished reading the staging tiles
       if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
       asm volatile("bar.sync 1, 128;" ::: "memory");     // every epilogue thread, unconditionally

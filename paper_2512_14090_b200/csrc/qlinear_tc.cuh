@@ -44,6 +44,7 @@ struct QtParams {
   int splits;
   int n_stages;
   int w_stages;             // packed weight tiles in flight
+  int stack;                // 1: hi and lo rows of B form one N = 2 Mt operand (Mt <= 128)
   int tmem_cols;
   int32_t* error_flag;      // optional
 };
@@ -167,8 +168,7 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
     for (int c = c_begin; c < c_end && alive; ++c) {
       const int sub = (c - c_begin) % cpw;                      // chunk inside the packed tile
       if (sub == 0) {
-        alive = mbar_wait(bar_w_full + 8 * wst, wphase, s_abort, p.error_flag);
-        alive = __all_sync(0xffffffffu, alive);
+        alive = mbar_wait_warp(bar_w_full + 8 * wst, wphase, s_abort, p.error_flag);
         if (!alive) break;
       }
       const uint8_t* wt = wring + wst * kQtWTile;
@@ -186,8 +186,7 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
         if (lane == 0) mbar_arrive(bar_w_empty + 8 * wst);
         if (++wst == (uint32_t)w_stages) { wst = 0; wphase ^= 1u; }
       }
-      alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
-      alive = __all_sync(0xffffffffu, alive);
+      alive = mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
       if (!alive) break;
       uint8_t* atile = smem + stage * stage_bytes;
 #pragma unroll
@@ -206,7 +205,11 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
     }
   } else if (warp == 1) {
     // ---- MMA issuer: all 32 lanes converged, one elected lane issues (see umma_bf16) ------------
-    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(Mt >> 3) << 17) | ((128u >> 4) << 24);
+    // Up to Mt = 128 the hi and the lo tile (adjacent in shared memory) are one B operand of
+    // 2 Mt rows: half as many MMAs, the two partial products land in separate accumulator
+    // columns and are added in the epilogue.  Small MMAs cost more to issue than to execute.
+    const int mma_n = p.stack ? 2 * Mt : Mt;
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mma_n >> 3) << 17) | ((128u >> 4) << 24);
     constexpr uint32_t DESC_HI = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // SBO 1024, version 1, 128-byte swizzle
     constexpr uint32_t LBO_FIELD = 1u << 16;
     const uint32_t tile_units = (uint32_t)(Mt * kQtChunk * 2) >> 4;
@@ -218,8 +221,8 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
       tc_fence_after();
       const uint32_t a_lo = ((smem_u32(smem) + stage * stage_bytes) >> 4) | LBO_FIELD;
       const uint32_t b_lo = a_lo + (kQtATile >> 4);
-#pragma unroll
-      for (int part = 0; part < 2; ++part) {
+      const int parts = p.stack ? 1 : 2;
+      for (int part = 0; part < parts; ++part) {
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
           const uint64_t adesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(a_lo + ((kk * 32) >> 4));
@@ -263,22 +266,23 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
     const bool n_ok = n < p.N;
     const float s = n_ok ? scale[n] : 0.f;
     const float b = (n_ok && bias && split == 0) ? bias[n] : 0.f;
-    alive = mbar_wait(bar_acc_full, 0, s_abort, p.error_flag);
-    alive = __all_sync(0xffffffffu, alive);
+    alive = mbar_wait_warp(bar_acc_full, 0, s_abort, p.error_flag);
     if (alive && c_begin < c_end) {
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
       for (int c0 = 0; c0 < Mt; c0 += 16) {
         if (m0 + c0 >= p.M) break;
-        uint32_t v[16];
+        uint32_t v[16], v2[16];
         tmem_ld16(taddr + c0, v);
+        if (p.stack) tmem_ld16(taddr + Mt + c0, v2);       // the lo half's partial products
         tmem_ld_wait();
         if (n_ok) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int m = m0 + c0 + j;
             if (m < p.M) {
-              const float val = fmaf(__uint_as_float(v[j]), s, b);
+              const float acc = p.stack ? __uint_as_float(v[j]) + __uint_as_float(v2[j]) : __uint_as_float(v[j]);
+              const float val = fmaf(acc, s, b);
               float* dst = y + (size_t)m * p.N + n;
               if (p.splits > 1) atomicAdd(dst, val); else *dst = val;
             }
@@ -341,8 +345,9 @@ aiq_status_t launch_qlinear_tc(const LayerJob& job, int N, int K, int M, void* w
   int w_stages = 3;
   while (w_stages < kQtMaxWStages && qt_smem_bytes(p.Mt, stages, w_stages + 1) + 1024 <= smem_limit) ++w_stages;
   p.w_stages = w_stages;
+  p.stack = p.Mt <= 128 ? 1 : 0;
   p.tmem_cols = 32;
-  while (p.tmem_cols < p.Mt) p.tmem_cols <<= 1;
+  while (p.tmem_cols < (p.stack ? 2 * p.Mt : p.Mt)) p.tmem_cols <<= 1;
 
   // activation planes in the workspace: (k, batch row, hi | lo)
   __nv_bfloat16* planes = static_cast<__nv_bfloat16*>(workspace);
