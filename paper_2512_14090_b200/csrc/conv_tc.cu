@@ -502,34 +502,55 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
     uint8_t* my_row = stg + lane * PIXB;
     const int my_key = (lane >> KEY_SHIFT) & KEY_MASK;
     const uint32_t pair_bar = 1u + (uint32_t)q;
+    // output row (image, padded y) of group gi of a tile, or -1 when the group is past the batch
+    auto tile_row = [&](int t, int gi) -> int {
+      const int trb = t / n_cb;
+      if (STRIDE == 1) {
+        const int jr = trb * kRowsPerTile + gi;
+        return jr < rows_total ? jr : -1;
+      }
+      const int rpi = STRIDE == 2 ? rows_per_img : 1;    // (stride 1 never gets here)
+      const int tb0 = (trb / rbi) * ipt, toy0 = (trb % rbi) * kRowsPerTile;
+      const int img = gi / rpi;
+      const int bb = tb0 + img;
+      return bb < p.B ? bb * (p.Ho + 2) + toy0 + (gi - img * rpi) + 1 : -1;
+    };
+    // The residual rows of the next tile are fetched into registers while the current tile is
+    // computed and stored, so their memory latency is off the critical path of the epilogue.
+    constexpr int RPL = (8 * UNITS + 31) / 32;         // 16-byte units per lane and row
+    uint4 rpre[2][RPL];
+    auto fetch_residual = [&](int t) {
+      const int tcb = t % n_cb;
+#pragma unroll
+      for (int ii = 0; ii < 2; ++ii) {
+        const int jr = tile_row(t, q * 4 + 2 * h + ii);
+        const uint4* src = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(job.res) +
+                                                          ((size_t)(jr < 0 ? 0 : jr) * p.Wo + tcb * kColsPerTile) * PIXB);
+#pragma unroll
+        for (int k = 0; k < RPL; ++k) {
+          const int u = lane + 32 * k;
+          rpre[ii][k] = (jr >= 0 && u < 8 * UNITS) ? __ldg(src + u) : make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+    };
+    if (job.res && (int)blockIdx.x < n_tiles && alive) fetch_residual(blockIdx.x);
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
       const int buf = it & 1;
       const int rb = tile / n_cb, cb = tile - rb * n_cb;
       const int b0 = STRIDE == 2 ? (rb / rbi) * ipt : 0, oy0 = STRIDE == 2 ? (rb % rbi) * kRowsPerTile : 0;
-      // output row (image, padded y) of tile group gi, or -1 when the group is past the batch
-      auto out_row = [&](int gi) -> int {
-        if (STRIDE == 1) {
-          const int jr = rb * kRowsPerTile + gi;
-          return jr < rows_total ? jr : -1;
-        }
-        const int img = gi / rows_per_img;
-        const int bb = b0 + img;
-        return bb < p.B ? bb * (p.Ho + 2) + oy0 + (gi - img * rows_per_img) + 1 : -1;
-      };
-      // (1) residual rows -> staging (this warp's two rows of the quarter)
+      auto out_row = [&](int gi) -> int { return tile_row(tile, gi); };
+      // (1) residual rows (fetched during the previous tile) -> staging: this warp's two rows
       if (job.res) {
 #pragma unroll
         for (int ii = 0; ii < 2; ++ii) {
           const int i = 2 * h + ii;
-          const int jr = out_row(q * 4 + i);
-          if (jr >= 0) {
-            const uint4* src = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(job.res) +
-                                                              ((size_t)jr * p.Wo + cb * kColsPerTile) * PIXB);
 #pragma unroll
-            for (int u = lane; u < 8 * UNITS; u += 32) {
+          for (int k = 0; k < RPL; ++k) {
+            const int u = lane + 32 * k;
+            if (u < 8 * UNITS) {
               const int pl = i * 8 + u / UNITS, uu = u % UNITS;
-              *reinterpret_cast<uint4*>(stg + pl * PIXB + ((uu ^ ((pl >> KEY_SHIFT) & KEY_MASK)) << 4)) = __ldg(src + u);
+              *reinterpret_cast<uint4*>(stg + pl * PIXB + ((uu ^ ((pl >> KEY_SHIFT) & KEY_MASK)) << 4)) = rpre[ii][k];
             }
           }
         }
@@ -540,6 +561,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
       alive = *s_abort == 0;                      // the same answer in both warps of the pair
       if (!alive) break;
+      if (job.res && tile + (int)gridDim.x < n_tiles) fetch_residual(tile + gridDim.x);
       tc_fence_after();
       bool interior = true;                       // stride 2 tiles hold interior rows only
       if (STRIDE == 1) {

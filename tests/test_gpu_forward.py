@@ -188,6 +188,43 @@ def test_eval_schemes_duplicates_fc_candidates_and_tiny_net():
     assert acc[-2] == 1.0
 
 
+def test_eval_schemes_coordinate_step_mobilenet_v2_imagenet():
+    """The coordinate-descent step on ImageNet-shaped MobileNetV2 at reduced size: candidates
+    that move one conv layer of an all-8 scheme to 32, 16 or 4 bits (so float32-kernel layers
+    sit inside a tensor-path model), evaluated with shared prefixes and a ragged last chunk.
+    Counts and predictions against the oracle; the chunk size must not change a count."""
+    import torch
+    aiq = binding()
+    arch = mobilenet_v2("imagenet")
+    x = gen_images(5, 3, 224, 224, 4236)
+    params = balance_classifier(arch, gen_model(arch, 4234), x)
+    model = aiq.Model(arch, params)
+    folded, bank = _oracle_bank(arch, params, (4, 8, 16, 32))
+    labels = O.predict(O.forward_fp32_unquantized(arch, folded, x))
+    all_schemes = coordinate_step_schemes(53, conv_layer_indices(arch))
+    assert all_schemes.shape == (52, 53)
+    schemes = all_schemes[[0, 1, 2, 10, 20, 31, 40, 47, 51]]
+    assert {int(b) for b in np.unique(schemes)} == {4, 8, 16, 32}
+    oacc, ocounts, opreds, omargins = O.eval_schemes(arch, bank, schemes, x, labels)
+    xd, ld = to_dev(x), to_dev(labels)
+    got = []
+    for chunk in (2, 5):
+        aiq.aiq_set_eval_options(chunk, True)
+        preds = torch.full((len(schemes), 5), -1, dtype=torch.int32, device="cuda")
+        acc, counts = model.aiq_eval_schemes(schemes, xd, ld, preds=preds, chunk=chunk)
+        got.append((counts.copy(), preds.cpu().numpy()))
+        assert np.allclose(acc, counts / 5.0)
+    aiq.aiq_set_eval_options(0, True)
+    assert np.array_equal(got[0][0], got[1][0]) and np.array_equal(got[0][1], got[1][1])
+    counts, p = got[0]
+    assert_preds_match(p, opreds, omargins, "coordinate step")
+    assert np.all(np.abs(counts - ocounts) <= (omargins <= 1e-2).sum(axis=1))
+    assert np.array_equal((p == labels[None, :]).sum(axis=1), counts)
+    ai = [model.aiq_scheme_ai(sc)[0] for sc in schemes]
+    oai = [O.scheme_ai(arch, sc)[0] for sc in schemes]
+    assert np.allclose(ai, oai, rtol=1e-12)
+
+
 def test_forward_and_eval_errors():
     import torch
     aiq = binding()
