@@ -42,16 +42,20 @@ struct QtParams {
   int n_chunks;             // ceil(K / 64)
   int chunks_per_split;
   int splits;
-  int n_stages;
+  int n_stages;             // A tiles (expanded weights) in flight
+  int b_stages;             // activation tile pairs in flight (a ring of its own: these are the
+                            // TMA loads with a long round trip, and at small batch they are small)
   int w_stages;             // packed weight tiles in flight
   int stack;                // 1: hi and lo rows of B form one N = 2 Mt operand (Mt <= 128)
   int tmem_cols;
   int32_t* error_flag;      // optional
 };
 
-__host__ __device__ inline int qt_stage_bytes(int Mt) { return kQtATile + 2 * Mt * kQtChunk * 2; }
-__host__ __device__ inline int qt_smem_bytes(int Mt, int stages, int w_stages) {
-  return stages * qt_stage_bytes(Mt) + w_stages * kQtWTile + (3 * stages + 2 * w_stages + 1) * 8 + 16;
+constexpr int kQtMaxBStages = 24;
+__host__ __device__ inline int qt_b_stage_bytes(int Mt) { return 2 * Mt * kQtChunk * 2; }   // hi tile + lo tile
+__host__ __device__ inline int qt_smem_bytes(int Mt, int stages, int b_stages, int w_stages) {
+  return stages * kQtATile + b_stages * qt_b_stage_bytes(Mt) + w_stages * kQtWTile +
+         (2 * stages + 2 * b_stages + 2 * w_stages + 1) * 8 + 16;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
@@ -88,29 +92,35 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n0 = blockIdx.x * 128, split = blockIdx.y, m0 = blockIdx.z * 256;
-  const int stages = p.n_stages, Mt = p.Mt, w_stages = p.w_stages;
-  const int stage_bytes = qt_stage_bytes(Mt);
+  const int stages = p.n_stages, b_stages = p.b_stages, Mt = p.Mt, w_stages = p.w_stages;
+  const int b_stage_bytes = qt_b_stage_bytes(Mt);
   const int c_begin = split * p.chunks_per_split;
   const int c_end = min(p.n_chunks, c_begin + p.chunks_per_split);
 
   // k chunks per packed tile: 128 bytes of a row are 256 (4 bits) or 128 (8 bits) elements
   const int cpw = p.bits == 4 ? 4 : 2;
-  uint8_t* wring = smem + stages * stage_bytes;             // packed weight tiles (1024-aligned)
+  // shared memory: A ring | B ring | packed weight ring | barriers (every tile 1024-aligned)
+  uint8_t* bring = smem + stages * kQtATile;
+  uint8_t* wring = bring + b_stages * b_stage_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(wring + w_stages * kQtWTile);
-  const uint32_t bar_a_full = smem_u32(bars);               // expanders finished the A tile of a stage
-  const uint32_t bar_b_full = bar_a_full + 8 * stages;      // TMA bytes of a stage have landed
-  const uint32_t bar_empty = bar_b_full + 8 * stages;       // the MMAs that read a stage have retired
-  const uint32_t bar_w_full = bar_empty + 8 * stages;       // a packed weight tile has landed
+  const uint32_t bar_a_full = smem_u32(bars);               // expanders finished an A tile
+  const uint32_t bar_a_empty = bar_a_full + 8 * stages;     // the MMAs that read an A tile have retired
+  const uint32_t bar_b_full = bar_a_empty + 8 * stages;     // TMA bytes of an activation tile pair have landed
+  const uint32_t bar_b_empty = bar_b_full + 8 * b_stages;   // the MMAs that read it have retired
+  const uint32_t bar_w_full = bar_b_empty + 8 * b_stages;   // a packed weight tile has landed
   const uint32_t bar_w_empty = bar_w_full + 8 * w_stages;   // the expanders are done with a packed tile
   const uint32_t bar_acc_full = bar_w_empty + 8 * w_stages;
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 3 * stages + 2 * w_stages + 1);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * stages + 2 * b_stages + 2 * w_stages + 1);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   if (tid == 0) {
     for (int i = 0; i < stages; ++i) {
       mbar_init(bar_a_full + 8 * i, kQtExpWarps);   // one arrival per expander warp
+      mbar_init(bar_a_empty + 8 * i, 1);
+    }
+    for (int i = 0; i < b_stages; ++i) {
       mbar_init(bar_b_full + 8 * i, 1);
-      mbar_init(bar_empty + 8 * i, 1);
+      mbar_init(bar_b_empty + 8 * i, 1);
     }
     for (int i = 0; i < w_stages; ++i) {
       mbar_init(bar_w_full + 8 * i, 1);
@@ -137,18 +147,18 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
       asm volatile("griddepcontrol.wait;" ::: "memory");
       uint32_t stage = 0, phase = 0, issued = 0, issued_phase = 0;
       for (int c = c_begin; c < c_end && alive; ++c) {
-        alive = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+        alive = mbar_wait(bar_b_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
         if (!alive) break;
         issued |= 1u << stage;
         issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
         const uint32_t tile_bytes = (uint32_t)Mt * kQtChunk * 2;
         mbar_expect_tx(bar_b_full + 8 * stage, 2 * tile_bytes);
-        const uint32_t dst = smem_u32(smem) + stage * stage_bytes + kQtATile;
+        const uint32_t dst = smem_u32(bring) + stage * b_stage_bytes;
         tma_load_3d(dst, &x_map, bar_b_full + 8 * stage, c * kQtChunk, m0, 0);                // hi
         tma_load_3d(dst + tile_bytes, &x_map, bar_b_full + 8 * stage, c * kQtChunk, m0, 1);   // lo
-        if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+        if (++stage == (uint32_t)b_stages) { stage = 0; phase ^= 1u; }
       }
-      for (int i = 0; i < stages; ++i)             // copies in flight must land before the CTA exits
+      for (int i = 0; i < b_stages; ++i)           // copies in flight must land before the CTA exits
         if (issued & (1u << i)) {
           const long long t0 = clock64();
           while (!mbar_try_wait(bar_b_full + 8 * i, (issued_phase >> i) & 1u) && clock64() - t0 < kWaitLimitCycles) {}
@@ -186,9 +196,9 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
         if (lane == 0) mbar_arrive(bar_w_empty + 8 * wst);
         if (++wst == (uint32_t)w_stages) { wst = 0; wphase ^= 1u; }
       }
-      alive = mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+      alive = mbar_wait_warp(bar_a_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
       if (!alive) break;
-      uint8_t* atile = smem + stage * stage_bytes;
+      uint8_t* atile = smem + stage * kQtATile;
 #pragma unroll
       for (int i = 0; i < UPT; ++i) {
         const int u = et + i * ET;
@@ -213,14 +223,14 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
     constexpr uint32_t DESC_HI = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // SBO 1024, version 1, 128-byte swizzle
     constexpr uint32_t LBO_FIELD = 1u << 16;
     const uint32_t tile_units = (uint32_t)(Mt * kQtChunk * 2) >> 4;
-    uint32_t stage = 0, phase = 0, accumulate = 0;
+    uint32_t stage = 0, phase = 0, bstage = 0, bphase = 0, accumulate = 0;
     for (int c = c_begin; c < c_end && alive; ++c) {
       alive = mbar_wait_warp(bar_a_full + 8 * stage, phase, s_abort, p.error_flag) &&
-              mbar_wait_warp(bar_b_full + 8 * stage, phase, s_abort, p.error_flag);
+              mbar_wait_warp(bar_b_full + 8 * bstage, bphase, s_abort, p.error_flag);
       if (!alive) break;
       tc_fence_after();
-      const uint32_t a_lo = ((smem_u32(smem) + stage * stage_bytes) >> 4) | LBO_FIELD;
-      const uint32_t b_lo = a_lo + (kQtATile >> 4);
+      const uint32_t a_lo = ((smem_u32(smem) + stage * kQtATile) >> 4) | LBO_FIELD;
+      const uint32_t b_lo = ((smem_u32(bring) + bstage * b_stage_bytes) >> 4) | LBO_FIELD;
       const int parts = p.stack ? 1 : 2;
       for (int part = 0; part < parts; ++part) {
 #pragma unroll
@@ -231,8 +241,10 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
           accumulate = 1;
         }
       }
-      umma_commit(bar_empty + 8 * stage);
+      umma_commit(bar_a_empty + 8 * stage);
+      umma_commit(bar_b_empty + 8 * bstage);
       if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+      if (++bstage == (uint32_t)b_stages) { bstage = 0; bphase ^= 1u; }
     }
     if (alive) umma_commit(bar_acc_full);
   } else {
@@ -334,16 +346,20 @@ aiq_status_t launch_qlinear_tc(const LayerJob& job, int N, int K, int M, void* w
   if (splits > p.n_chunks) splits = p.n_chunks;
   p.chunks_per_split = (p.n_chunks + splits - 1) / splits;
   p.splits = (p.n_chunks + p.chunks_per_split - 1) / p.chunks_per_split;
-  // shared memory: at least 2 operand stages and 3 packed weight tiles; then up to 6 operand
-  // stages, and whatever is left goes to weight tiles in flight (the stream that must not stall)
-  int stages = 6;
-  while (stages > 2 && qt_smem_bytes(p.Mt, stages, 3) + 1024 > smem_limit) --stages;
-  if (qt_smem_bytes(p.Mt, stages, 3) + 1024 > smem_limit)
-    return set_error(AIQ_ERR_SHAPE, "qlinear_tc: %d bytes of shared memory needed", qt_smem_bytes(p.Mt, stages, 3) + 1024);
-  if (stages > p.chunks_per_split) stages = p.chunks_per_split < 2 ? 2 : p.chunks_per_split;
+  // Shared memory: at least 2 A tiles, 2 activation tile pairs and 3 packed weight tiles.  Then
+  // up to 4 A tiles (they are produced on chip, a short ring suffices), as many activation
+  // stages as fit up to 24 (their TMA round trip is what a shallow ring would expose), and
+  // whatever is left goes to packed weight tiles in flight.
+  auto fits = [&](int a, int b, int w) { return qt_smem_bytes(p.Mt, a, b, w) + 1024 <= smem_limit; };
+  if (!fits(2, 2, 3))
+    return set_error(AIQ_ERR_SHAPE, "qlinear_tc: %d bytes of shared memory needed", qt_smem_bytes(p.Mt, 2, 2, 3) + 1024);
+  int stages = 2, b_stages = 2, w_stages = 3;
+  while (stages < 4 && fits(stages + 1, b_stages, w_stages)) ++stages;
+  while (w_stages < 4 && fits(stages, b_stages, w_stages + 1)) ++w_stages;
+  while (b_stages < kQtMaxBStages && b_stages < p.chunks_per_split && fits(stages, b_stages + 1, w_stages)) ++b_stages;
+  while (w_stages < kQtMaxWStages && fits(stages, b_stages, w_stages + 1)) ++w_stages;
   p.n_stages = stages;
-  int w_stages = 3;
-  while (w_stages < kQtMaxWStages && qt_smem_bytes(p.Mt, stages, w_stages + 1) + 1024 <= smem_limit) ++w_stages;
+  p.b_stages = b_stages;
   p.w_stages = w_stages;
   p.stack = p.Mt <= 128 ? 1 : 0;
   p.tmem_cols = 32;
@@ -388,7 +404,7 @@ aiq_status_t launch_qlinear_tc(const LayerJob& job, int N, int K, int M, void* w
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(row_blocks, p.splits, m_blocks);
   cfg.blockDim = dim3(kQtThreads);
-  cfg.dynamicSmemBytes = qt_smem_bytes(p.Mt, stages, w_stages) + 1024;
+  cfg.dynamicSmemBytes = qt_smem_bytes(p.Mt, stages, b_stages, w_stages) + 1024;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
