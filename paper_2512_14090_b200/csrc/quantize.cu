@@ -207,7 +207,7 @@ __device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity) {
 }
 
 template <int BITS>
-__global__ void __launch_bounds__(kStreamThreads, 2)
+__global__ void __launch_bounds__(kStreamThreads, 4)
 quantize_stream_kernel(const float* __restrict__ W, int N, int K, uint8_t* __restrict__ packed,
                        float* __restrict__ scales, int32_t* __restrict__ nonfinite_flag, int stages) {
   extern __shared__ __align__(128) uint8_t qs[];
@@ -303,13 +303,19 @@ aiq_status_t launch_quantize_bits(const float* W, int N, int K, void* packed, fl
   const bool stream_ok = K % 32 == 0 && K >= 2048 && K <= kStreamThreads * 8 * kStreamCache &&
                          N >= 4 * n_sms && ((uintptr_t)W & 15) == 0;
   if (stream_ok) {
-    // two blocks per SM: half of the shared memory each, minus the per-block reserve
-    const int per_block = (smem_limit + 1024) / 2 - 2048;
-    int stages = per_block / (K * 4);
+    // As many blocks per SM (up to 4) as leave each a ring of at least two rows: the rounding
+    // pass is a chain of dependent instructions, so resident warps matter as much as bytes in
+    // flight (ncu at two blocks per SM: 25 % of the warp slots, issue slots half used).
+    int blocks_per_sm = 4, stages = 0;
+    for (; blocks_per_sm >= 2; --blocks_per_sm) {
+      const int per_block = (smem_limit + 1024) / blocks_per_sm - 2048;   // minus the per-block reserve
+      stages = per_block / (K * 4);
+      if (stages >= 2) break;
+    }
     if (stages > 8) stages = 8;
     if (stages >= 2) {
       const int smem = stages * K * 4 + stages * 8;
-      quantize_stream_kernel<BITS><<<2 * n_sms, kStreamThreads, smem, s>>>(W, N, K, p, scales, nonfinite_flag, stages);
+      quantize_stream_kernel<BITS><<<blocks_per_sm * n_sms, kStreamThreads, smem, s>>>(W, N, K, p, scales, nonfinite_flag, stages);
       AIQ_LAUNCH_CHECK("quantize_stream");
       return AIQ_OK;
     }
