@@ -33,7 +33,10 @@ namespace aiq {
 
 namespace {
 
-constexpr int kTcThreads = 320;            // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
+// warp 0: TMA producer, warp 1: MMA issuer, then the epilogue warps: 2 per TMEM quarter, 4 where
+// N = 64 (those kernels run one CTA per SM, so registers allow it, and their epilogue is the longest)
+__host__ __device__ constexpr int tc_epilogue_warps_per_quarter(int n) { return n == 64 ? 4 : 2; }
+__host__ __device__ constexpr int tc_threads(int n) { return (2 + 4 * tc_epilogue_warps_per_quarter(n)) * 32; }
 constexpr int kRowsPerTile = 16;           // padded rows per tile
 constexpr int kColsPerTile = 8;
 constexpr int kBoxRows = kRowsPerTile + 2;
@@ -247,7 +250,7 @@ struct TcSmem {
 };
 
 template <int CS, int N, int KS, int STRIDE>
-__global__ void __launch_bounds__(kTcThreads, (CS <= 32 && N <= 32) ? 2 : 1)
+__global__ void __launch_bounds__(tc_threads(N), (CS <= 32 && N <= 32) ? 2 : 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const LayerJob* __restrict__ jobs) {
   using L = TcLayout<CS, N>;
   using S = TcSmem<CS, N>;
@@ -293,7 +296,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_acc_full + 8 * i, 1);
-      mbar_init(bar_acc_empty + 8 * i, 8);     // one arrival per epilogue warp
+      mbar_init(bar_acc_empty + 8 * i, 4 * tc_epilogue_warps_per_quarter(N));   // one arrival per epilogue warp
     }
     mbar_init(bar_w, 1);
     *s_abort = 0;
@@ -312,7 +315,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
     mbar_expect_tx(bar_w, packed_bytes);
     bulk_load(smem_u32(ring), job.w, packed_bytes, bar_w);
   }
-  for (int i = tid; i < N; i += kTcThreads) {
+  for (int i = tid; i < N; i += tc_threads(N)) {
     s_scale[i] = job.scale[i];
     s_bias[i] = job.bias[i];
   }
@@ -320,7 +323,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
   if (alive) {
     const int units_per_row = CS / 8;                         // 16-byte units of one weight row
     const int total_units = taps * N * units_per_row;
-    for (int u = tid; u < total_units; u += kTcThreads) {
+    for (int u = tid; u < total_units; u += tc_threads(N)) {
       const int c8 = u % units_per_row;
       const int n = (u / units_per_row) % N;
       const int tap = u / (units_per_row * N);
@@ -475,20 +478,22 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       }
     }
   } else {
-    // Epilogue: TMEM lanes 32q .. 32q+31 (tile rows 4q .. 4q+3, 8 pixels each) belong to the two
-    // warps with warp index mod 4 = q; warp h of the pair takes half of the output channels.
-    // The arithmetic of the epilogue (scale, bias, residual, activation, the split into two
-    // bfloat16) is a long dependent chain per tile, so it is spread over eight warps; with four
-    // the tensor cores waited for the epilogue more than half of the time.
+    // Epilogue: TMEM lanes 32q .. 32q+31 (tile rows 4q .. 4q+3, 8 pixels each) belong to the
+    // EPW (2, or 4 at N = 64) warps with warp index mod 4 = q; warp h of them takes 1/EPW of the
+    // output channels.  The arithmetic of the epilogue (scale, bias, residual, activation, the
+    // split into two bfloat16) is a long dependent chain per tile, so it is spread over many
+    // warps; with four in all the tensor cores waited for the epilogue more than half of the time.
     // A lane owns one pixel for the arithmetic, but a pixel is only 4N bytes, so per-lane global
     // accesses would touch 32 cache lines per instruction.  Instead the 32 pixels of a quarter
-    // are staged in shared memory: the residual rows are fetched into the staging buffer with
-    // coalesced 16-byte accesses *before* the accumulator is waited for, the result overwrites
-    // them in place, and the finished rows leave with coalesced stores (a row of 8 pixels is
-    // 32N contiguous bytes).  Each warp moves two of the quarter's four rows; two named-barrier
-    // syncs per tile order the pair (ids 1 .. 4, 64 threads).  16-byte units are XOR-swizzled
-    // so that both access patterns are free of bank conflicts.
+    // are staged in shared memory: the residual rows go into the staging buffer with coalesced
+    // 16-byte accesses, the result overwrites them in place, and the finished rows leave with
+    // coalesced stores (a row of 8 pixels is 32N contiguous bytes).  Each warp moves 4/EPW of
+    // the quarter's four rows; two named-barrier syncs per tile order the warps of a quarter
+    // (ids 1 .. 4).  16-byte units are XOR-swizzled so that both access patterns are free of
+    // bank conflicts.
     const int q = warp & 3;
+    constexpr int EPW = tc_epilogue_warps_per_quarter(N);   // warps that share a quarter
+    constexpr int RPW = 4 / EPW;                             // rows of the quarter each of them moves
     const int h = (warp - 2) >> 2;
     const int m = q * 32 + lane;                       // row of the tile: pixel (g, wl)
     const int g = m >> 3;
@@ -497,7 +502,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
     constexpr int KEY_SHIFT = PIXB < 128 ? 1 : 0;      // N = 16: two pixels share a 128-byte window
     constexpr int KEY_MASK = (UNITS < 8 ? UNITS : 8) - 1;
     constexpr int CW = N >= 32 ? 16 : 8;               // accumulator columns per chunk
-    constexpr int NCH = N / (2 * CW);                  // chunks per warp (1, 1, 2)
+    constexpr int NCH = N / (EPW * CW);                // chunks per warp (1)
     uint8_t* stg = smem + S::staging(stages, taps) + q * 32 * PIXB;
     uint8_t* my_row = stg + lane * PIXB;
     const int my_key = (lane >> KEY_SHIFT) & KEY_MASK;
@@ -518,12 +523,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
     // The residual rows of the next tile are fetched into registers while the current tile is
     // computed and stored, so their memory latency is off the critical path of the epilogue.
     constexpr int RPL = (8 * UNITS + 31) / 32;         // 16-byte units per lane and row
-    uint4 rpre[2][RPL];
+    uint4 rpre[RPW][RPL];
     auto fetch_residual = [&](int t) {
       const int tcb = t % n_cb;
 #pragma unroll
-      for (int ii = 0; ii < 2; ++ii) {
-        const int jr = tile_row(t, q * 4 + 2 * h + ii);
+      for (int ii = 0; ii < RPW; ++ii) {
+        const int jr = tile_row(t, q * 4 + RPW * h + ii);
         const uint4* src = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(job.res) +
                                                           ((size_t)(jr < 0 ? 0 : jr) * p.Wo + tcb * kColsPerTile) * PIXB);
 #pragma unroll
@@ -543,8 +548,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       // (1) residual rows (fetched during the previous tile) -> staging: this warp's two rows
       if (job.res) {
 #pragma unroll
-        for (int ii = 0; ii < 2; ++ii) {
-          const int i = 2 * h + ii;
+        for (int ii = 0; ii < RPW; ++ii) {
+          const int i = RPW * h + ii;
 #pragma unroll
           for (int k = 0; k < RPL; ++k) {
             const int u = lane + 32 * k;
@@ -556,10 +561,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
         }
       }
       mbar_wait_warp(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);   // false => *s_abort is set
-      // both warps of the pair, unconditionally: the partner's residual rows are in place and its
+      // all warps of the quarter, unconditionally: the partners' residual rows are in place and their
       // stores of the previous tile have left the staging rows
-      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-      alive = *s_abort == 0;                      // the same answer in both warps of the pair
+      asm volatile("bar.sync %0, %1;" ::"r"(pair_bar), "n"(32 * EPW) : "memory");
+      alive = *s_abort == 0;                      // the same answer in every warp of the quarter
       if (!alive) break;
       if (job.res && tile + (int)gridDim.x < n_tiles) fetch_residual(tile + gridDim.x);
       tc_fence_after();
@@ -574,7 +579,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       uint32_t v[NCH][CW];
 #pragma unroll
       for (int ch = 0; ch < NCH; ++ch) {
-        const int c0 = (2 * ch + h) * CW;
+        const int c0 = (EPW * ch + h) * CW;
         if (CW == 16) tmem_ld16(taddr + c0, v[ch]); else tmem_ld8(taddr + c0, v[ch]);
       }
       tmem_ld_wait();
@@ -584,7 +589,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
 #pragma unroll
       for (int ch = 0; ch < NCH; ++ch) {
-        const int c0 = (2 * ch + h) * CW;
+        const int c0 = (EPW * ch + h) * CW;
 #pragma unroll
         for (int u8 = 0; u8 < CW / 8; ++u8) {
           // the 16-byte units of this pixel that hold columns c0 + 8 u8 .. + 7: one of hi, one of lo
@@ -621,11 +626,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
         }
       }
       // every column of the quarter's rows is final once the partner is here too
-      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+      asm volatile("bar.sync %0, %1;" ::"r"(pair_bar), "n"(32 * EPW) : "memory");
       // (3) staging -> global, one row of 8 pixels (32N contiguous bytes) at a time
 #pragma unroll
-      for (int ii = 0; ii < 2; ++ii) {
-        const int i = 2 * h + ii;
+      for (int ii = 0; ii < RPW; ++ii) {
+        const int i = RPW * h + ii;
         const int jr = out_row(q * 4 + i);
         if (jr >= 0) {
           uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(job.out) +
@@ -640,7 +645,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       if (STRIDE == 2) {
         // zero border rows of the output images this tile touches (rows 0 and Ho + 1)
         const bool top = oy0 == 0, bottom = oy0 + rows_per_img == p.Ho;
-        for (int img = q + 4 * h; img < ipt; img += 8) {
+        for (int img = q + 4 * h; img < ipt; img += 4 * EPW) {
           const int bb = b0 + img;
           if (bb >= p.B) break;
           for (int side = 0; side < 2; ++side) {
@@ -743,7 +748,7 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
                       2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
                       weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
                                                      (double)g.B * g.Ho * g.Wo * g.Cout));
-    conv_tc_kernel<CS, N, KS, STRIDE><<<dim3(ctas, n_jobs), kTcThreads, smem_bytes, s>>>(map, p, jobs_dev);
+    conv_tc_kernel<CS, N, KS, STRIDE><<<dim3(ctas, n_jobs), tc_threads(N), smem_bytes, s>>>(map, p, jobs_dev);
   }
   AIQ_LAUNCH_CHECK("conv_tc");
   return AIQ_OK;
