@@ -1,8 +1,9 @@
 """CPU oracle for AIQ scheme evaluation (test infrastructure, not a product path).
 
 A plain, slow NumPy statement of what the hot path computes: batch-norm folding,
-the per-layer weight quantizer, the quantized CNN forward pass, top-1 agreement
-and the analytic global arithmetic intensity.  Only tests, the smoke check and
+the per-layer weight quantizer, the quantized CNN forward pass, top-1 agreement,
+the analytic global arithmetic intensity, and the two searches of Section 2.2 over the
+AIQ objective (the units inside the objective are a stated reading: parity unpinned).  Only tests, the smoke check and
 the benchmark's CPU-baseline leg may import this module; the CUDA library shares
 no code with it.
 
@@ -322,6 +323,100 @@ def scheme_ai(arch, scheme, batch=1):
         nbytes += layer["cout"] * K * int(bits) / 8.0
         nbytes += 4.0 * batch * (layer["cin"] * hi * wi + layer["cout"] * ho * wo)
     return flops / nbytes, flops, nbytes
+
+
+# ----------------------------------------------------------------------------
+# AIQ objective and the two searches (Section 2.1, Section 2.2)
+# ----------------------------------------------------------------------------
+def aiq_loss(ai, acc, acc_fp, lam):
+    """L(q; lambda) = -lambda * AI(q) + (1 - lambda) * AccLoss(q)   (Section 2.1).
+
+    The paper does not state the units of AccLoss nor a normalisation of AI.  Reading:
+    AccLoss(q) = 100 * (acc(q_FP) - acc(q)) in percentage points, AI in FLOP per byte,
+    neither normalised.  Parity unpinned for this choice of units (nothing printed in the
+    paper fixes it); the search logic around it is pinned by hand-worked tables.
+    """
+    return -lam * ai + (1.0 - lam) * 100.0 * (acc_fp - acc)
+
+
+def greedy_search(n_layers, acc_fn, ai_fn, lam, options=(8, 4), layers=None):
+    """Greedy search of Section 2.2.
+
+    Start from the all-FP32 scheme.  At each iteration the candidate moves are "lower the
+    bit-width of a still unquantized (32-bit) layer i to b", for every selectable layer i
+    and every b in `options`; the move with the smallest Delta L = L(candidate) - L(current)
+    is taken when that Delta L is negative.  As many iterations as there are selectable
+    layers.  Ties go to the first candidate in (layer, option) order.  When no move improves
+    the loss the scheme can no longer change and the remaining iterations are no-ops.
+    acc_fn(schemes [S][L] uint8) -> accuracies [S]; ai_fn(scheme) -> AI.
+    Returns (scheme, trace) with trace = list of (layer, bits, accepted, loss_after).
+    """
+    layers = list(range(n_layers)) if layers is None else list(layers)
+    q = np.full(n_layers, 32, np.uint8)
+    acc_fp = float(acc_fn(q[None, :])[0])
+    cur = aiq_loss(ai_fn(q), acc_fp, acc_fp, lam)
+    trace = []
+    for _ in range(len(layers)):
+        moves = [(i, b) for i in layers if q[i] == 32 for b in options if b < 32]
+        if not moves:
+            break
+        cands = np.repeat(q[None, :], len(moves), axis=0)
+        for r, (i, b) in enumerate(moves):
+            cands[r, i] = b
+        accs = acc_fn(cands)
+        best, best_delta = -1, 0.0
+        for r in range(len(moves)):
+            delta = aiq_loss(ai_fn(cands[r]), float(accs[r]), acc_fp, lam) - cur
+            if best < 0 or delta < best_delta:
+                best, best_delta = r, delta
+        i, b = moves[best]
+        if best_delta < 0:
+            q = cands[best].copy()
+            cur = cur + best_delta
+            trace.append((i, b, 1, cur))
+        else:
+            trace.append((i, b, 0, cur))
+            break
+    return q, trace
+
+
+def coordinate_descent(n_layers, acc_fn, ai_fn, lam, options=(32, 8, 4), layers=None, max_passes=8):
+    """Coordinate descent of Section 2.2.
+
+    Start from the all-FP32 scheme.  Visit the selectable layers in order; for each, hold
+    the others fixed and set q_i to the b in `options` with the smallest L (the current
+    value stays on ties; among strictly better values the first in option order wins).
+    Repeat passes until a pass changes nothing (or `max_passes`).
+    Returns (scheme, trace) with trace = list of (layer, bits, changed, loss_after).
+    """
+    layers = list(range(n_layers)) if layers is None else list(layers)
+    q = np.full(n_layers, 32, np.uint8)
+    acc_fp = float(acc_fn(q[None, :])[0])
+    cur = aiq_loss(ai_fn(q), acc_fp, acc_fp, lam)
+    trace = []
+    for _ in range(max_passes):
+        changed_any = False
+        for i in layers:
+            alts = [b for b in options if b != q[i]]
+            cands = np.repeat(q[None, :], len(alts), axis=0)
+            for r, b in enumerate(alts):
+                cands[r, i] = b
+            accs = acc_fn(cands)
+            best, best_loss = -1, cur
+            for r in range(len(alts)):
+                loss = aiq_loss(ai_fn(cands[r]), float(accs[r]), acc_fp, lam)
+                if loss < best_loss:
+                    best, best_loss = r, loss
+            if best >= 0:
+                q = cands[best].copy()
+                cur = best_loss
+                changed_any = True
+                trace.append((i, int(q[i]), 1, cur))
+            else:
+                trace.append((i, int(q[i]), 0, cur))
+        if not changed_any:
+            break
+    return q, trace
 
 
 # ----------------------------------------------------------------------------
