@@ -36,9 +36,9 @@ UNIT = "scheme-evals/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the
 # committed ncu summary under profiles/ (None until captured / after the kernel changed)
-# conv_tc_kernel: 198.1 MB per launch measured at chunk 256 (profiles/conv_tc__resnet20_greedy_step.md),
+# conv_tc_kernel: 197.6 MB per launch measured at chunk 256 (profiles/conv_tc__resnet20_greedy_step.md),
 # scaled by 4 to the default chunk of 1024 images (traffic grows with the images of a launch)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 198.1e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 197.6e6
 
 
 def measured_peaks():
@@ -197,6 +197,35 @@ def run_kernel_sweep(args):
         return e0.elapsed_time(e1) / n          # ms per launch
 
     shapes = [(4096, 4096), (8192, 8192), (1280, 320)]
+    if args.workload == "search":
+        # the two searches of Section 2.2 on ResNet-20 over the 10,000-image set (lambda = 0.9,
+        # the paper's value): wall time of the whole search, every candidate scored by the evaluator
+        from aiq_workloads import resnet20, gen_model, gen_images
+        arch = resnet20()
+        model = aiq.Model(arch, gen_model(arch, SEED_MODEL), device=dev)
+        L = model.n_layers
+        x = torch.from_numpy(gen_images(N_IMAGES, 3, 32, 32, SEED_IMAGES)).to(dev)
+        ws = torch.empty(model.aiq_workspace_bytes(1024, 3 * L), dtype=torch.uint8, device=dev)
+        preds = torch.empty((1, N_IMAGES), dtype=torch.int32, device=dev)
+        model.aiq_eval_schemes(np.full((1, L), 32, np.uint8), x, torch.zeros(N_IMAGES, dtype=torch.int32, device=dev),
+                               preds=preds, workspace=ws)
+        labels = preds[0].contiguous()
+        for name, fn in (("greedy", lambda: model.aiq_search_greedy(x, labels, 0.9, options=(8, 4), workspace=ws)),
+                         ("coordinate_descent", lambda: model.aiq_search_coordinate_descent(
+                             x, labels, 0.9, options=(32, 8, 4), max_passes=8, workspace=ws))):
+            fn()                                                     # warm-up
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            scheme, steps = fn()
+            torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+            evals = 1 + sum(st["candidates"] for st in steps)
+            print(json.dumps(dict(workload="search", algorithm=name, seconds=dt, scheme_evals=evals,
+                                  scheme_evals_per_s=evals / dt, iterations=len(steps), images=N_IMAGES,
+                                  final_scheme=[int(b) for b in scheme], final_ai=model.aiq_scheme_ai(scheme)[0],
+                                  final_acc=steps[-1]["acc"] if steps else None, lam=0.9)), flush=True)
+        model.close()
+        return
     if args.workload == "forward":
         # one scheme, one batch, through aiq_forward (host plan + launches included): images/s
         from aiq_workloads import (resnet20, mobilenet_v2, gen_model, gen_images, gen_random_scheme,
@@ -282,9 +311,10 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--chunk", type=int, default=0, help="images per evaluator pass (0 = library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="resnet20_step", choices=["resnet20_step", "qlinear", "quantize", "forward"],
+    ap.add_argument("--workload", default="resnet20_step", choices=["resnet20_step", "qlinear", "quantize", "forward", "search"],
                     help="resnet20_step: the headline line (default).  qlinear / quantize: per-case lines for the "
-                         "standalone memory-bound kernels (1 GPU)")
+                         "standalone memory-bound kernels; forward: one scheme, one batch; search: the two searches "
+                         "of Section 2.2 on ResNet-20 (all 1 GPU)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))

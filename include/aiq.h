@@ -15,6 +15,7 @@
  *   aiq_forward          logits of one scheme on one image batch
  *   aiq_eval_schemes     top-1 agreement of many schemes on an image set
  *   aiq_scheme_ai        AI(q), on the host
+ *   aiq_search_greedy / aiq_search_coordinate_descent   the searches of Section 2.2
  *
  * Conventions
  *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
@@ -295,6 +296,53 @@ void aiq_last_call_stats(int64_t* kernel_launches, int64_t* layer_evals, int64_t
  */
 aiq_status_t aiq_scheme_ai(const aiq_model_t* model, const uint8_t* scheme_bits, int ai_batch,
                            double* ai, double* flops, double* bytes);
+
+/* ------------------------------------------------------------------------------------
+ * The two searches of Section 2.2 over the AIQ objective of Section 2.1,
+ *     L(q; lambda) = -lambda * AI(q) + (1 - lambda) * AccLoss(q),
+ * as host loops over aiq_eval_schemes and aiq_scheme_ai (every candidate of an iteration is
+ * scored in one aiq_eval_schemes call).  The paper fixes neither the units of AccLoss nor a
+ * normalisation of AI; used here: AccLoss(q) = 100 * (acc(q_FP32) - acc(q)) (percentage
+ * points, both accuracies measured on the given images) and AI in FLOP per byte at batch 1.
+ *
+ * Both start from the all-32-bit scheme.  `layers`: host int32 list of the layers that may
+ * move (NULL = all L layers), visited in the given order.  `options`: host uint8 list of
+ * bit-widths, in the order in which ties are broken.  x, labels, workspace, stream: as for
+ * aiq_eval_schemes; the workspace must cover n_layers * n_options schemes.
+ *
+ * aiq_search_greedy: per iteration the candidate moves are "set a selectable layer that is
+ *   still at 32 bits to an option below 32"; the move with the smallest Delta L is applied
+ *   when Delta L < 0 (first candidate in (layer, option) order on ties); n_layers iterations
+ *   at most, ending early once no move lowers L (the scheme could not change any more).
+ * aiq_search_coordinate_descent: passes over the selectable layers; each layer takes the
+ *   option with the smallest L, the others held fixed (the current value stays unless an
+ *   option is strictly better); passes repeat until one changes nothing, max_passes at most.
+ *
+ * scheme_out: host uint8 [L].  trace (optional): one record per iteration (greedy) or per
+ * layer visit (coordinate descent), the first trace_capacity of them; *n_trace = how many
+ * there were.  Synchronous (every iteration reads accuracies back).
+ */
+typedef struct aiq_search_step {
+  int32_t layer;       /* layer of the best move of this iteration / the layer visited      */
+  int32_t bits;        /* its new bit-width (coordinate descent: its bit-width afterwards)   */
+  int32_t accepted;    /* 1 if the scheme changed                                            */
+  int32_t candidates;  /* schemes evaluated in this iteration                                */
+  double loss;         /* L of the scheme after the iteration                                */
+  double acc;          /* accuracy of the scheme after the iteration (greedy, rejected move: */
+                       /* of the rejected candidate)                                         */
+  double ai;           /* AI of that scheme                                                  */
+} aiq_search_step_t;
+aiq_status_t aiq_search_greedy(const aiq_model_t* model, const int32_t* layers, int n_layers,
+                               const uint8_t* options, int n_options, double lambda, const float* x,
+                               const int32_t* labels, int n_images, uint8_t* scheme_out,
+                               aiq_search_step_t* trace, int trace_capacity, int* n_trace,
+                               void* workspace, size_t workspace_bytes, void* stream);
+aiq_status_t aiq_search_coordinate_descent(const aiq_model_t* model, const int32_t* layers, int n_layers,
+                                           const uint8_t* options, int n_options, double lambda,
+                                           int max_passes, const float* x, const int32_t* labels,
+                                           int n_images, uint8_t* scheme_out, aiq_search_step_t* trace,
+                                           int trace_capacity, int* n_trace, void* workspace,
+                                           size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------
  * Per-kernel timing.  The paper measures throughput by wall clock (Section 3, experiment

@@ -26,7 +26,7 @@ EXPORTS = [
     "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
     "aiq_eval_schemes", "aiq_set_eval_options", "aiq_last_call_stats", "aiq_scheme_ai",
     "aiq_profile_start", "aiq_profile_stop", "aiq_forward_static",
-    "aiq_set_compute_path", "aiq_model_status",
+    "aiq_set_compute_path", "aiq_model_status", "aiq_search_greedy", "aiq_search_coordinate_descent",
 ]
 
 PATH_AUTO, PATH_FP32, PATH_TENSOR = 0, 1, 2
@@ -55,6 +55,11 @@ class ArchDesc(C.Structure):
 class KernelProfile(C.Structure):
     _fields_ = [("launches", C.c_int64), ("ms", C.c_double), ("flops", C.c_double),
                 ("bytes", C.c_double)]
+
+
+class SearchStep(C.Structure):
+    _fields_ = [("layer", C.c_int32), ("bits", C.c_int32), ("accepted", C.c_int32), ("candidates", C.c_int32),
+                ("loss", C.c_double), ("acc", C.c_double), ("ai", C.c_double)]
 
 
 class LayerWeights(C.Structure):
@@ -107,6 +112,12 @@ def _load():
     lib.aiq_set_eval_options.argtypes = [i32, i32]
     lib.aiq_last_call_stats.restype = None
     lib.aiq_last_call_stats.argtypes = [C.POINTER(C.c_int64)] * 3
+    lib.aiq_search_greedy.restype = i32
+    lib.aiq_search_greedy.argtypes = [vp, vp, i32, vp, i32, C.c_double, vp, vp, i32, vp,
+                                      C.POINTER(SearchStep), i32, C.POINTER(C.c_int), vp, sz, vp]
+    lib.aiq_search_coordinate_descent.restype = i32
+    lib.aiq_search_coordinate_descent.argtypes = [vp, vp, i32, vp, i32, C.c_double, i32, vp, vp, i32, vp,
+                                                  C.POINTER(SearchStep), i32, C.POINTER(C.c_int), vp, sz, vp]
     lib.aiq_scheme_ai.restype = i32
     lib.aiq_scheme_ai.argtypes = [vp, vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_double),
                                   C.POINTER(C.c_double)]
@@ -339,6 +350,37 @@ class Model:
                                     _host(acc), _host(counts), _dev(preds), _dev(ws), ws.numel(),
                                     _stream(stream)))
         return acc, counts
+
+    def _search(self, which, x, labels, lam, options, layers, max_passes, workspace, chunk, stream):
+        options = np.ascontiguousarray(options, dtype=np.uint8)
+        n_sel = self.n_layers if layers is None else len(layers)
+        lay = None if layers is None else np.ascontiguousarray(layers, dtype=np.int32)
+        N = x.shape[0]
+        ws = workspace if workspace is not None else self.workspace(min(chunk, N), max(1, n_sel * len(options)))
+        scheme = np.zeros(self.n_layers, dtype=np.uint8)
+        cap = 4 * (n_sel + 1) * max(1, max_passes)
+        trace = (SearchStep * cap)()
+        n_trace = C.c_int(0)
+        if which == "greedy":
+            _check(lib.aiq_search_greedy(self.handle, _host(lay), n_sel, _host(options), len(options), float(lam),
+                                         _dev(x), _dev(labels), N, _host(scheme), trace, cap, C.byref(n_trace),
+                                         _dev(ws), ws.numel(), _stream(stream)))
+        else:
+            _check(lib.aiq_search_coordinate_descent(self.handle, _host(lay), n_sel, _host(options), len(options),
+                                                     float(lam), int(max_passes), _dev(x), _dev(labels), N,
+                                                     _host(scheme), trace, cap, C.byref(n_trace), _dev(ws),
+                                                     ws.numel(), _stream(stream)))
+        steps = [dict(layer=t.layer, bits=t.bits, accepted=t.accepted, candidates=t.candidates, loss=t.loss,
+                      acc=t.acc, ai=t.ai) for t in trace[:min(n_trace.value, cap)]]
+        return scheme, steps
+
+    def aiq_search_greedy(self, x, labels, lam, options=(8, 4), layers=None, workspace=None, chunk=1024,
+                          stream=None):
+        return self._search("greedy", x, labels, lam, options, layers, 1, workspace, chunk, stream)
+
+    def aiq_search_coordinate_descent(self, x, labels, lam, options=(32, 8, 4), layers=None, max_passes=8,
+                                      workspace=None, chunk=1024, stream=None):
+        return self._search("cd", x, labels, lam, options, layers, max_passes, workspace, chunk, stream)
 
     def aiq_model_status(self, stream=None):
         _check(lib.aiq_model_status(self.handle, _stream(stream)))
