@@ -5,7 +5,8 @@ draws random arrays.  It holds none of the method's arithmetic (no folding, no
 quantizer, no convolution, no arithmetic-intensity formula), so both the CPU
 oracle's tests and the CUDA library's binding may consume its output as data.
 """
-from .archs import resnet20, mobilenet_v2, conv_layer_indices, tiny_net  # noqa: F401
+from .archs import (resnet20, mobilenet_v2, conv_layer_indices, tiny_net,  # noqa: F401
+                    heavy_early_resnet20, plain_convnet20)
 from .gen import (  # noqa: F401
     gen_model,
     gen_images,

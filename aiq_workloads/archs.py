@@ -32,16 +32,17 @@ def _fc(name, cin, cout, inp):
                 act="none", input=inp, residual=-1, has_bn=False)
 
 
-def resnet20(channels=(16, 32, 64), n_classes=10, in_hw=32, name="resnet20"):
+def resnet20(channels=(16, 32, 64), n_classes=10, in_hw=32, name="resnet20", stem=None):
     """CIFAR ResNet-20 with 1x1 projection shortcuts where shape changes.
 
-    Stem conv3x3, three stages of three basic blocks, global average pool,
-    linear classifier.  Scheme order: stem; per block conv1, conv2, then the
-    block's projection (if any); classifier last.
+    Stem conv3x3 (`stem` channels, default channels[0]), three stages of three basic
+    blocks, global average pool, linear classifier.  Scheme order: stem; per block conv1,
+    conv2, then the block's projection (if any); classifier last.
     """
-    layers = [_conv("stem", 3, channels[0], 3, 1, "relu", -1)]
+    stem = channels[0] if stem is None else stem
+    layers = [_conv("stem", 3, stem, 3, 1, "relu", -1)]
     prev = 0            # index of the layer producing the current block input
-    cin = channels[0]
+    cin = stem
     for si, c in enumerate(channels):
         for b in range(3):
             stride = 2 if (si > 0 and b == 0) else 1
@@ -58,6 +59,29 @@ def resnet20(channels=(16, 32, 64), n_classes=10, in_hw=32, name="resnet20"):
             cin = c
     layers.append(_fc("fc", cin, n_classes, prev))
     return dict(name=name, in_c=3, in_h=in_hw, in_w=in_hw, n_classes=n_classes, layers=layers)
+
+
+def heavy_early_resnet20(n_classes=10, in_hw=32):
+    """HeavyEarlyResNet20 (Section 4.5): ResNet-20 with the channel progression reversed,
+    channel groups (64, 32, 16, 16) for (stem, stage 1, stage 2, stage 3) instead of
+    (16, 16, 32, 64).  The first block of stage 1 then changes the width (64 -> 32) at
+    stride 1 and gets a projection shortcut like every other shape change."""
+    return resnet20(channels=(32, 16, 16), n_classes=n_classes, in_hw=in_hw, name="heavy_early_resnet20", stem=64)
+
+
+def plain_convnet20(n_classes=10, in_hw=32, width=64):
+    """PlainConvNet20 (Section 4.5): 20 convolution layers of 64 channels, no shortcuts, then
+    the classifier (21 weight tensors, as in Table 1).  The paper does not say where the
+    network reduces resolution; reading: stride 2 at layers 7 and 13, where ResNet-20 starts
+    its second and third stage, so that depth and cost stay comparable."""
+    layers = []
+    cin = 3
+    for i in range(20):
+        stride = 2 if i in (7, 13) else 1
+        layers.append(_conv(f"f{3 * i}", cin, width, 3, stride, "relu", i - 1))
+        cin = width
+    layers.append(_fc("cls", width, n_classes, 19))
+    return dict(name="plain_convnet20", in_c=3, in_h=in_hw, in_w=in_hw, n_classes=n_classes, layers=layers)
 
 
 _MBV2_CFG = [(1, 16, 1), (6, 24, 2), (6, 32, 3), (6, 64, 4), (6, 96, 3), (6, 160, 3), (6, 320, 1)]

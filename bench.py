@@ -197,6 +197,35 @@ def run_kernel_sweep(args):
         return e0.elapsed_time(e1) / n          # ms per launch
 
     shapes = [(4096, 4096), (8192, 8192), (1280, 320)]
+    if args.workload == "sensitivity":
+        # the paper's single-layer study (Section 3, experiment 1; the 8b / 4b columns of Table 1):
+        # every layer alone at 8 and at 4 bits, all others FP32, agreement with the FP32 model and AI
+        from aiq_workloads import resnet20, gen_model, gen_images, one_layer_lowered_schemes
+        arch = resnet20()
+        model = aiq.Model(arch, gen_model(arch, SEED_MODEL), device=dev)
+        L = model.n_layers
+        x = torch.from_numpy(gen_images(N_IMAGES, 3, 32, 32, SEED_IMAGES)).to(dev)
+        schemes = np.concatenate([np.full((1, L), 32, np.uint8),
+                                  one_layer_lowered_schemes(L, list(range(L)), base=32, low=8),
+                                  one_layer_lowered_schemes(L, list(range(L)), base=32, low=4)])
+        ws = torch.empty(model.aiq_workspace_bytes(1024, len(schemes)), dtype=torch.uint8, device=dev)
+        preds = torch.empty((len(schemes), N_IMAGES), dtype=torch.int32, device=dev)
+        zeros = torch.zeros(N_IMAGES, dtype=torch.int32, device=dev)
+        model.aiq_eval_schemes(schemes[:1], x, zeros, preds=preds[:1], workspace=ws)
+        labels = preds[0].contiguous()
+        model.aiq_eval_schemes(schemes, x, labels, workspace=ws)          # warm-up
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        acc, _ = model.aiq_eval_schemes(schemes, x, labels, workspace=ws)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        ai = [model.aiq_scheme_ai(sc)[0] for sc in schemes]
+        rows = [dict(layer=arch["layers"][i]["name"], acc_8b=float(acc[1 + i]), acc_4b=float(acc[1 + L + i]),
+                     ai_8b=ai[1 + i], ai_4b=ai[1 + L + i]) for i in range(L)]
+        print(json.dumps(dict(workload="sensitivity", model="resnet20", images=N_IMAGES, schemes=len(schemes),
+                              seconds=dt, scheme_evals_per_s=len(schemes) / dt, ai_fp32=ai[0], layers=rows)), flush=True)
+        model.close()
+        return
     if args.workload == "search":
         # the two searches of Section 2.2 on ResNet-20 over the 10,000-image set (lambda = 0.9,
         # the paper's value): wall time of the whole search, every candidate scored by the evaluator
@@ -311,10 +340,11 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--chunk", type=int, default=0, help="images per evaluator pass (0 = library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="resnet20_step", choices=["resnet20_step", "qlinear", "quantize", "forward", "search"],
+    ap.add_argument("--workload", default="resnet20_step", choices=["resnet20_step", "qlinear", "quantize", "forward", "search", "sensitivity"],
                     help="resnet20_step: the headline line (default).  qlinear / quantize: per-case lines for the "
                          "standalone memory-bound kernels; forward: one scheme, one batch; search: the two searches "
-                         "of Section 2.2 on ResNet-20 (all 1 GPU)")
+                         "of Section 2.2 on ResNet-20; sensitivity: every layer alone at 8 / 4 bits from an FP32 "
+                         "base (all 1 GPU)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))

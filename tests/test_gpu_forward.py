@@ -2,7 +2,8 @@
 import numpy as np
 import pytest
 
-from aiq_workloads import (resnet20, mobilenet_v2, tiny_net, gen_model, gen_images,
+from aiq_workloads import (resnet20, mobilenet_v2, tiny_net, heavy_early_resnet20, plain_convnet20,
+                           gen_model, gen_images,
                            gen_random_scheme, one_layer_lowered_schemes, coordinate_step_schemes,
                            mixed_int4_int8_scheme, conv_layer_indices)
 from oracle import aiq_oracle as O
@@ -223,6 +224,43 @@ def test_eval_schemes_coordinate_step_mobilenet_v2_imagenet():
     ai = [model.aiq_scheme_ai(sc)[0] for sc in schemes]
     oai = [O.scheme_ai(arch, sc)[0] for sc in schemes]
     assert np.allclose(ai, oai, rtol=1e-12)
+
+
+@pytest.mark.parametrize("path", ["fp32", "tensor"])
+@pytest.mark.parametrize("make", [heavy_early_resnet20, plain_convnet20])
+def test_structural_variants_of_section_4_5(make, path):
+    """HeavyEarlyResNet20 (wide layers first, width changes at stride 1, 64 -> 32 -> 16 channels)
+    and PlainConvNet20 (20 plain 64-channel convolutions): forward logits of mixed schemes and a
+    greedy step over every conv layer against the oracle."""
+    import torch
+    aiq = binding()
+    arch = make()
+    L = len(arch["layers"])
+    x = gen_images(40, 3, 32, 32, 4501)
+    params = balance_classifier(arch, gen_model(arch, 4500), x)
+    with compute_path(path):
+        model = aiq.Model(arch, params)
+    folded, bank = _oracle_bank(arch, params, (4, 8, 16, 32))
+    for seed in (1, 2):
+        scheme = gen_random_scheme(L, seed)
+        got = model.aiq_forward(scheme, to_dev(x[:9])).cpu().numpy()
+        ref = O.forward_scheme(arch, bank, scheme, x[:9])
+        if path == "fp32":
+            assert_logits_close(got, ref, f"{arch['name']} scheme seed {seed}")
+        else:
+            assert_logits_close_tensor(got, ref, f"{arch['name']} scheme seed {seed}")
+            assert_preds_match(O.predict(got), O.predict(ref), O.top2_margin(ref), arch["name"])
+    labels = O.predict(O.forward_fp32_unquantized(arch, folded, x))
+    schemes = one_layer_lowered_schemes(L, conv_layer_indices(arch))
+    oacc, ocounts, opreds, omargins = O.eval_schemes(arch, bank, schemes, x, labels)
+    preds = torch.full((len(schemes), 40), -1, dtype=torch.int32, device="cuda")
+    aiq.aiq_set_eval_options(16, True)
+    acc, counts = model.aiq_eval_schemes(schemes, to_dev(x), to_dev(labels), preds=preds, chunk=16)
+    aiq.aiq_set_eval_options(0, True)
+    p = preds.cpu().numpy()
+    assert_preds_match(p, opreds, omargins, arch["name"] + " greedy step")
+    assert np.all(np.abs(counts - ocounts) <= (omargins <= 1e-2).sum(axis=1))
+    assert abs(model.aiq_scheme_ai(schemes[3])[0] - O.scheme_ai(arch, schemes[3])[0]) < 1e-9
 
 
 def test_forward_and_eval_errors():

@@ -250,3 +250,18 @@ def test_mobilenet_shapes():
     assert O.layer_shapes(i)[-2][3:] == (7, 7) and O.layer_shapes(c)[-2][3:] == (8, 8)
     with pytest.raises(ValueError):
         O.scheme_ai(c, [5] * 53)
+
+
+def test_structural_variant_tables():
+    """Shapes of the Section 4.5 variants: HeavyEarlyResNet20 has channel groups (64, 32, 16, 16),
+    PlainConvNet20 has 20 convolutions of 64 channels plus the classifier (21 entries in Table 1)."""
+    from aiq_workloads import heavy_early_resnet20, plain_convnet20
+    h = heavy_early_resnet20()
+    assert h["layers"][0]["cout"] == 64
+    convs = [l for l in h["layers"] if l["kind"] == "conv" and l["k"] == 3]
+    assert [l["cout"] for l in convs[1:]] == [32] * 6 + [16] * 12
+    assert sum(1 for l in h["layers"] if l["k"] == 1 and l["kind"] == "conv") == 3      # every shape change
+    p = plain_convnet20()
+    assert len(p["layers"]) == 21 and p["layers"][-1]["kind"] == "fc"
+    assert all(l["cout"] == 64 and l["residual"] == -1 for l in p["layers"][:-1])
+    assert O.layer_shapes(p)[-2][3:] == (8, 8)
