@@ -86,8 +86,9 @@ aiq_status_t aiq_fold_bn(const float* W, const float* gamma, const float* beta,
  *
  * W: device float32 [N][K].  packed_out: device, N * row_bytes, 16-byte aligned.
  * scales_out: device float32 [N].  nonfinite_flag: optional device int32; set to 1 when a
- * NaN or infinity is met (outputs are then unspecified); never cleared by the call.
- * Asynchronous on `stream`.
+ * NaN or infinity is met (outputs are then unspecified), to 2 if a bounded wait inside the
+ * kernel for large matrices expired (should not happen; outputs invalid); never cleared by
+ * the call.  Asynchronous on `stream`.
  */
 size_t aiq_packed_row_bytes(int K, int bits);   /* 0 for an unsupported bits or K <= 0 */
 aiq_status_t aiq_quantize_layer(const float* W, int N, int K, int bits, void* packed_out,

@@ -360,6 +360,7 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
   CREATE_TRY(cudaMemcpyAsync(&host_flag, flag, 4, cudaMemcpyDeviceToHost, stream));
   CREATE_TRY(cudaStreamSynchronize(stream));
 #undef CREATE_TRY
+  if (host_flag == 2) return fail(set_error(AIQ_ERR_TIMEOUT, "a bounded wait inside the quantizer expired"));
   if (host_flag) return fail(set_error(AIQ_ERR_NONFINITE, "a weight is NaN or infinite"));
   *out = m;
   return AIQ_OK;
