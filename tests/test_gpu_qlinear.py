@@ -32,6 +32,7 @@ def _run(aiq, W, x, bits, bias=None, use_workspace=True):
                                    (2048, 4096, 4), (300, 2052, 7), (1, 1, 1),
                                    # shapes on the warp-level tensor-core path (K % 512 == 0, N*K >= 2^20)
                                    (4100, 512, 16), (1000, 1536, 3), (2050, 1024, 9), (8192, 8192, 2),
+                                   (1030, 1024, 1), (4100, 8192, 2), (2048, 3072, 2),
                                    # batches on the tcgen05 path (M >= 9, K % 8 == 0): ragged N, K and M tails,
                                    # several batch blocks, K split over CTAs
                                    (4096, 4096, 256), (1280, 320, 256), (1000, 1280, 37), (2050, 1024, 300),
@@ -54,7 +55,8 @@ def test_qlinear_exact_on_integers(bits):
     aiq = binding()
     rng = np.random.default_rng(1)
     qmax = 2 ** (bits - 1) - 1
-    for shape_w, m in (((96, 200), 4), ((2176, 512), 5), ((300, 520), 20)):   # plain / int8 warp-level / tcgen05
+    # plain / int8 warp-level (M = 5 and M = 2) / tcgen05
+    for shape_w, m in (((96, 200), 4), ((2176, 512), 5), ((2176, 2048), 2), ((300, 520), 20)):
         W = rng.integers(-qmax, qmax + 1, shape_w).astype(np.float32)
         W[:, 0] = qmax
         x = rng.integers(-8, 9, (m, shape_w[1])).astype(np.float32)
