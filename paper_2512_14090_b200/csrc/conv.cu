@@ -304,6 +304,103 @@ aiq_status_t launch_conv_tile(const ConvGeom& g, const LayerJob* jobs, int n_job
 }
 
 // ---------------------------------------------------------------------------------------
+// Stem convolution: 3x3, pad 1, a few input channels read straight from the float32 NCHW
+// network input.  K = 9 * Cin = 27 is too short for the tiled GEMM above (one 16-deep slice
+// and a half-empty one, two block barriers per 16 multiply-adds per thread), so a thread
+// owns one padded output pixel and all COUT channels: its 27 inputs sit in registers, the
+// expanded weights [k][COUT] in shared memory (read as warp-wide broadcasts), and the result
+// leaves as 16-byte stores.  Border rows are written as zeros.
+// ---------------------------------------------------------------------------------------
+constexpr int kStemThreads = 256;
+
+template <int COUT, int FMT>
+__global__ void __launch_bounds__(kStemThreads)
+conv_stem_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* __restrict__ net_input) {
+  extern __shared__ __align__(16) float stem_sm[];            // [Kt][COUT] weights, [COUT] scale, [COUT] bias
+  const LayerJob job = jobs[blockIdx.z];
+  const int Kt = 9 * g.Cin;
+  float* wsm = stem_sm;
+  float* ssm = wsm + Kt * COUT;
+  float* bsm = ssm + COUT;
+  const int wrow_bytes = ((g.K + 31) / 32 * 32) * job.bits / 8;
+  for (int i = threadIdx.x; i < Kt * COUT; i += kStemThreads) {
+    const int k = i / COUT, n = i - k * COUT;                // k = (tap, channel), channel fastest
+    const int tap = k / g.Cin, c = k - tap * g.Cin;
+    wsm[i] = n < g.Cout ? load_element(job.w + (size_t)n * wrow_bytes, c * 9 + tap, job.bits) : 0.f;
+  }
+  for (int n = threadIdx.x; n < COUT; n += kStemThreads) {
+    ssm[n] = n < g.Cout ? job.scale[n] : 0.f;
+    bsm[n] = n < g.Cout ? job.bias[n] : 0.f;
+  }
+  __syncthreads();
+
+  const int rows_out = g.Ho + 2;
+  const long long M = (long long)g.B * rows_out * g.Wo;      // padded output pixels
+  const long long p = (long long)blockIdx.x * kStemThreads + threadIdx.x;
+  if (p >= M) return;
+  const int b = (int)(p / (rows_out * g.Wo));
+  const int rem = (int)(p - (long long)b * rows_out * g.Wo);
+  const int oyp = rem / g.Wo, ox = rem - oyp * g.Wo;
+  float acc[COUT];
+#pragma unroll
+  for (int n = 0; n < COUT; ++n) acc[n] = 0.f;
+  const bool interior = oyp >= 1 && oyp <= g.Ho;
+  if (interior) {
+    const int iy0 = (oyp - 1) * g.stride - 1, ix0 = ox * g.stride - 1;
+    for (int c = 0; c < g.Cin; ++c) {
+      const float* plane = net_input + ((size_t)b * g.Cin + c) * g.H * g.W;
+#pragma unroll
+      for (int r = 0; r < 3; ++r) {
+        const int iy = iy0 + r;
+#pragma unroll
+        for (int t = 0; t < 3; ++t) {
+          const int ix = ix0 + t;
+          const float xv = (iy >= 0 && iy < g.H && ix >= 0 && ix < g.W) ? __ldg(plane + (size_t)iy * g.W + ix) : 0.f;
+          const float* wk = wsm + ((r * 3 + t) * g.Cin + c) * COUT;
+#pragma unroll
+          for (int n = 0; n < COUT; n += 4) {
+            const float4 wv = *reinterpret_cast<const float4*>(wk + n);
+            acc[n] = fmaf(xv, wv.x, acc[n]);
+            acc[n + 1] = fmaf(xv, wv.y, acc[n + 1]);
+            acc[n + 2] = fmaf(xv, wv.z, acc[n + 2]);
+            acc[n + 3] = fmaf(xv, wv.w, acc[n + 3]);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int n = 0; n < COUT; n += 4) {
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (interior) {
+      v.x = n < g.Cout ? apply_act(fmaf(acc[n], ssm[n], bsm[n]), g.act) : 0.f;
+      v.y = n + 1 < g.Cout ? apply_act(fmaf(acc[n + 1], ssm[n + 1], bsm[n + 1]), g.act) : 0.f;
+      v.z = n + 2 < g.Cout ? apply_act(fmaf(acc[n + 2], ssm[n + 2], bsm[n + 2]), g.act) : 0.f;
+      v.w = n + 3 < g.Cout ? apply_act(fmaf(acc[n + 3], ssm[n + 3], bsm[n + 3]), g.act) : 0.f;
+    }
+    act_store4<FMT>(job.out, (size_t)p, n, g.Cs_out, v);
+  }
+}
+
+template <int COUT>
+aiq_status_t launch_stem(const ConvGeom& g, const LayerJob* jobs, int n_jobs, const float* net_input,
+                         double weight_bytes, cudaStream_t s) {
+  const long long M = (long long)g.B * (g.Ho + 2) * g.Wo;
+  dim3 grid((unsigned)((M + kStemThreads - 1) / kStemThreads), 1, n_jobs);
+  const size_t smem = (size_t)(9 * g.Cin * COUT + 2 * COUT) * sizeof(float);
+  LaunchScope scope(AIQ_KERNEL_CONV, s,
+                    2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(9 * g.Cin) * n_jobs,
+                    weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
+                                                   (double)g.B * g.Ho * g.Wo * g.Cout));
+  if (g.act_format == ACT_SPLIT)
+    conv_stem_kernel<COUT, ACT_SPLIT><<<grid, kStemThreads, smem, s>>>(g, jobs, net_input);
+  else
+    conv_stem_kernel<COUT, ACT_F32><<<grid, kStemThreads, smem, s>>>(g, jobs, net_input);
+  AIQ_LAUNCH_CHECK("conv_stem");
+  return AIQ_OK;
+}
+
+// ---------------------------------------------------------------------------------------
 // Global average pool over the interior of a split tensor: pooled[b][c] float32
 // ---------------------------------------------------------------------------------------
 template <int FMT>
@@ -366,6 +463,11 @@ __global__ void argmax_count_kernel(const LayerJob* __restrict__ jobs, int B, in
 
 aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs, const float* net_input,
                          double weight_bytes, cudaStream_t s) {
+  if (g.in_is_nchw && g.ks == 3 && g.pad == 1 && g.Cin <= 4 && (g.stride == 1 || g.stride == 2)) {
+    if (g.Cs_out == 16) return launch_stem<16>(g, jobs_dev, n_jobs, net_input, weight_bytes, s);
+    if (g.Cs_out == 32) return launch_stem<32>(g, jobs_dev, n_jobs, net_input, weight_bytes, s);
+    if (g.Cs_out == 64) return launch_stem<64>(g, jobs_dev, n_jobs, net_input, weight_bytes, s);
+  }
   const int in_mode = g.in_is_nchw ? IN_NCHW : ((g.Cin % 4 == 0) ? IN_SPLIT_VEC : IN_SPLIT_SCALAR);
   auto waste = [&](int bn) { return (g.Cs_out + bn - 1) / bn * bn - g.Cs_out; };
   int bn = 64;
