@@ -403,17 +403,46 @@ aiq_status_t launch_stem(const ConvGeom& g, const LayerJob* jobs, int n_jobs, co
 // ---------------------------------------------------------------------------------------
 // Global average pool over the interior of a split tensor: pooled[b][c] float32
 // ---------------------------------------------------------------------------------------
+// One block per (image, job).  A thread owns 4 consecutive channels and every PL-th pixel
+// (8-byte loads of the hi and the lo half); the PL partial sums of a channel meet in shared
+// memory in a fixed order, so the result does not depend on timing.
+constexpr int kPoolThreads = 256;
+
 template <int FMT>
-__global__ void avgpool_kernel(const LayerJob* __restrict__ jobs, int H, int W, int C, int Cs) {
+__global__ void __launch_bounds__(kPoolThreads)
+avgpool_kernel(const LayerJob* __restrict__ jobs, int H, int W, int C, int Cs) {
+  __shared__ float4 s_sum[kPoolThreads];
   const LayerJob job = jobs[blockIdx.z];
   const int b = blockIdx.x;
   const float inv = 1.0f / (float)(H * W);
   float* __restrict__ out = static_cast<float*>(job.out);
   const size_t p0 = ((size_t)b * (H + 2) + 1) * W;       // first interior pixel of image b
-  for (int c = threadIdx.x; c < C; c += blockDim.x) {
-    float s = 0.f;
-    for (int i = 0; i < H * W; ++i) s += act_load1<FMT>(job.in, p0 + i, c, Cs);
-    out[(size_t)b * C + c] = s * inv;
+  const int quads = Cs / 4;                               // groups of 4 channels
+  const int qb = quads < kPoolThreads ? quads : kPoolThreads;   // quads handled per pass
+  const int PL = kPoolThreads / qb;                       // pixel lanes
+  const int ql = threadIdx.x % qb, pl = threadIdx.x / qb;
+  for (int q0 = 0; q0 < quads; q0 += qb) {
+    const int q = q0 + ql;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (q < quads && pl < PL)
+      for (int i = pl; i < H * W; i += PL) {
+        const float4 v = act_load4<FMT>(job.in, p0 + i, 4 * q, Cs);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+    s_sum[threadIdx.x] = acc;
+    __syncthreads();
+    if (pl == 0 && q < quads) {
+      float4 t = s_sum[ql];
+      for (int j = 1; j < PL; ++j) {
+        const float4 u = s_sum[j * qb + ql];
+        t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+      }
+      const float r[4] = {t.x * inv, t.y * inv, t.z * inv, t.w * inv};
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (4 * q + j < C) out[(size_t)b * C + 4 * q + j] = r[j];
+    }
+    __syncthreads();
   }
 }
 
@@ -480,7 +509,7 @@ aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs
 
 aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int H, int W, int C, int act_format,
                             cudaStream_t s) {
-  int threads = C >= 256 ? 256 : (C >= 128 ? 128 : 64);
+  const int threads = kPoolThreads;
   LaunchScope scope(AIQ_KERNEL_POOL, s, (double)n_jobs * B * H * W * C,
                     4.0 * n_jobs * B * ((double)H * W * C + C));
   if (act_format == ACT_SPLIT)
