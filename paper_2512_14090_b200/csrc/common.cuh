@@ -141,12 +141,16 @@ aiq_status_t launch_conv(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs
 aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
                               const float* net_input, double weight_bytes, cudaStream_t s);
 // Tensor-core convolution (conv_tc.cu).  `map` points to a 128-byte CUtensorMap over the input
-// slot: dims (2*Cs, W, batch_capacity*(H+2), versions).  Jobs must have 4- or 8-bit weights.
+// slot: dims (2*Cs, W, batch_capacity*(H+2), versions).
 bool conv_tc_eligible(const ConvGeom& g);
 aiq_status_t conv_tc_encode_map(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
                                 void* map_out);
+// All jobs of one launch have weights of one class: weight_bits = 8 (4- or 8-bit codes), 16 or 32.
+// 16- / 32-bit weights enter as 2 / 3 exact bfloat16 pieces; conv_tc_bits_ok says whether that fits.
+bool conv_tc_bits_ok(const ConvGeom& g, int bits);
 aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
-                            int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s);
+                            int batch_capacity, int32_t* error_flag, double weight_bytes, int weight_bits,
+                            cudaStream_t s);
 // Pointwise (1x1, stride 1) tensor-core convolution for any channel count that is a multiple
 // of 8 (conv_pw_tc.cuh).  `map`: CUtensorMap over the input slot, dims (Cs, 2, pixels of all versions).
 bool conv_pw_tc_eligible(const ConvGeom& g);

@@ -249,7 +249,8 @@ struct TcSmem {
   static __host__ __device__ constexpr int total(int stages, int taps) { return bars(stages, taps) + (2 * stages + 5) * 8 + 16; }
 };
 
-template <int CS, int N, int KS, int STRIDE>
+// PIECES: bfloat16 pieces per weight: 1 (4- / 8-bit codes), 2 (half), 3 (float32)
+template <int CS, int N, int KS, int STRIDE, int PIECES>
 __global__ void __launch_bounds__(tc_threads(N), (CS <= 32 && N <= 32) ? 2 : 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const LayerJob* __restrict__ jobs) {
   using L = TcLayout<CS, N>;
@@ -265,9 +266,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
 
   uint8_t* ring = smem;
   uint8_t* wsm = smem + S::weights(stages);
-  float* s_scale = reinterpret_cast<float*>(smem + S::scale(stages, taps));
-  float* s_bias = reinterpret_cast<float*>(smem + S::bias(stages, taps));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::bars(stages, taps));
+  // 16- and 32-bit weights are not exact in one bfloat16: they are held as the sum of 2 / 3
+  // bfloat16 pieces (8 + 8 (+ 8) significant bits: exact), one weight tile per piece and tap,
+  // and every MMA is issued once per piece into the same accumulator.
+  constexpr int pieces = PIECES;
+  constexpr int wtaps = taps * pieces;           // weight tiles in shared memory
+  float* s_scale = reinterpret_cast<float*>(smem + S::scale(stages, wtaps));
+  float* s_bias = reinterpret_cast<float*>(smem + S::bias(stages, wtaps));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::bars(stages, wtaps));
   const uint32_t bar_full = smem_u32(bars);
   const uint32_t bar_empty = bar_full + 8 * stages;
   const uint32_t bar_acc_full = bar_empty + 8 * stages;
@@ -328,6 +334,29 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       const int n = (u / units_per_row) % N;
       const int tap = u / (units_per_row * N);
       const uint8_t* row = ring + (size_t)n * wrow_bytes;
+      const uint32_t off = swizzle_off((uint32_t)(n * L::W_ROW_BYTES + c8 * 16), L::W_SWZ_MASK);
+      if (PIECES > 1) {
+        uint32_t pk[3][4];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int k = (c8 * 8 + j) * taps + tap;
+          float w = job.bits == 16 ? __half2float(reinterpret_cast<const __half*>(row)[k])
+                                   : reinterpret_cast<const float*>(row)[k];
+#pragma unroll
+          for (int pc = 0; pc < 3; ++pc) {
+            const __nv_bfloat16 h = __float2bfloat16_rn(w);
+            w -= __bfloat162float(h);                            // exact: the remainder of a rounding
+            const uint32_t hb = (uint32_t)__bfloat16_as_ushort(h);
+            if (j & 1) pk[pc][j >> 1] |= hb << 16; else pk[pc][j >> 1] = hb;
+          }
+        }
+#pragma unroll
+        for (int pc = 0; pc < 3; ++pc)
+          if (pc < pieces)
+            *reinterpret_cast<uint4*>(wsm + (size_t)(pc * taps + tap) * L::W_TAP_BYTES + off) =
+                make_uint4(pk[pc][0], pk[pc][1], pk[pc][2], pk[pc][3]);
+        continue;
+      }
       uint32_t packed[4];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -343,7 +372,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
         const uint32_t h = (uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code));
         if (j & 1) packed[j >> 1] |= h << 16; else packed[j >> 1] = h;
       }
-      const uint32_t off = swizzle_off((uint32_t)(n * L::W_ROW_BYTES + c8 * 16), L::W_SWZ_MASK);
       *reinterpret_cast<uint4*>(wsm + (size_t)tap * L::W_TAP_BYTES + off) =
           make_uint4(packed[0], packed[1], packed[2], packed[3]);
     }
@@ -459,9 +487,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
                 const uint32_t a_off = (byte / L::CW_BYTES) * L::CHUNK_BYTES + (STRIDE == 1 ? r * L::GROUP_BYTES : 0) +
                                        (byte % L::CW_BYTES);
                 const uint64_t adesc = ((uint64_t)A_HI << 32) | (uint64_t)(a_lo0 + (a_off >> 4));
-                const uint64_t bdesc = ((uint64_t)B_HI << 32) | (uint64_t)(w_lo0 + ((tap * L::W_TAP_BYTES + kk * 32) >> 4));
+                const uint32_t b_lo = w_lo0 + ((tap * L::W_TAP_BYTES + kk * 32) >> 4);
                 const uint32_t accumulate = (t == T_FIRST && r == T_FIRST && part == 0 && kk == 0) ? 0u : 1u;
-                umma_bf16(d_tmem, adesc, bdesc, idesc, accumulate);
+                umma_bf16(d_tmem, adesc, ((uint64_t)B_HI << 32) | (uint64_t)b_lo, idesc, accumulate);
+#pragma unroll
+                for (int pc = 1; pc < pieces; ++pc)             // further pieces of 16- / 32-bit weights
+                  umma_bf16(d_tmem, adesc,
+                            ((uint64_t)B_HI << 32) | (uint64_t)(b_lo + (uint32_t)((pc * taps * L::W_TAP_BYTES) >> 4)),
+                            idesc, 1u);
               }
             }
             if (STRIDE == 2) {
@@ -503,7 +536,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
     constexpr int KEY_MASK = (UNITS < 8 ? UNITS : 8) - 1;
     constexpr int CW = N >= 32 ? 16 : 8;               // accumulator columns per chunk
     constexpr int NCH = N / (EPW * CW);                // chunks per warp (1)
-    uint8_t* stg = smem + S::staging(stages, taps) + q * 32 * PIXB;
+    uint8_t* stg = smem + S::staging(stages, wtaps) + q * 32 * PIXB;
     uint8_t* my_row = stg + lane * PIXB;
     const int my_key = (lane >> KEY_SHIFT) & KEY_MASK;
     const uint32_t pair_bar = 1u + (uint32_t)q;
@@ -687,12 +720,12 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-template <int CS, int N, int KS, int STRIDE>
+template <int CS, int N, int KS, int STRIDE, int PIECES>
 aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob* jobs_dev, int n_jobs,
-                       int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s) {
+                       int batch_capacity, int32_t* error_flag, double weight_bytes, int weight_bits, cudaStream_t s) {
   using L = TcLayout<CS, N>;
   using S = TcSmem<CS, N>;
-  const int taps = g.ks * g.ks;
+  const int taps = g.ks * g.ks * PIECES;         // weight tiles held in shared memory
   static int smem_limit = 0, n_sms = 0;
   if (!smem_limit) {
     int dev = 0;
@@ -714,12 +747,12 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
   if (!stages)
     return set_error(AIQ_ERR_SHAPE, "conv_tc: shared memory for %d taps does not fit (%d bytes available)", taps, smem_limit);
   const int smem_bytes = S::total(stages, taps) + 1024;
-  const int packed = N * (int)row_bytes(g.K, 8);
+  const int packed = N * (int)row_bytes(g.K, weight_bits <= 8 ? 8 : weight_bits);
   if (packed > stages * L::STAGE_BYTES)
     return set_error(AIQ_ERR_SHAPE, "conv_tc: packed weights (%d bytes) exceed the staging ring", packed);
   static bool attr_set = false;
   if (!attr_set) {
-    AIQ_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<CS, N, KS, STRIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
+    AIQ_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<CS, N, KS, STRIDE, PIECES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
     attr_set = true;
   }
   TcParams p = {};
@@ -748,7 +781,7 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
                       2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
                       weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
                                                      (double)g.B * g.Ho * g.Wo * g.Cout));
-    conv_tc_kernel<CS, N, KS, STRIDE><<<dim3(ctas, n_jobs), tc_threads(N), smem_bytes, s>>>(map, p, jobs_dev);
+    conv_tc_kernel<CS, N, KS, STRIDE, PIECES><<<dim3(ctas, n_jobs), tc_threads(N), smem_bytes, s>>>(map, p, jobs_dev);
   }
   AIQ_LAUNCH_CHECK("conv_tc");
   return AIQ_OK;
@@ -893,18 +926,33 @@ aiq_status_t conv_tc_encode_map(const ConvGeom& g, const void* slot_base, int ba
   return AIQ_OK;
 }
 
+bool conv_tc_bits_ok(const ConvGeom& g, int bits) {
+  // 2 or 3 weight tiles per tap must fit shared memory beside the activation ring
+  return bits <= 8 || (g.Cin <= 32 && g.Cout <= 32);
+}
+
 aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
-                            int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s) {
+                            int batch_capacity, int32_t* error_flag, double weight_bytes, int weight_bits,
+                            cudaStream_t s) {
   const CUtensorMap& m = *static_cast<const CUtensorMap*>(map);
-#define AIQ_TC_ARGS g, m, jobs_dev, n_jobs, batch_capacity, error_flag, weight_bytes, s
+#define AIQ_TC_ARGS g, m, jobs_dev, n_jobs, batch_capacity, error_flag, weight_bytes, weight_bits, s
+#define AIQ_TC_KS(CS_, N_, P_)                                                                                   \
+  do {                                                                                                          \
+    if (g.stride == 1) return g.ks == 3 ? launch_tc<CS_, N_, 3, 1, P_>(AIQ_TC_ARGS) : launch_tc<CS_, N_, 1, 1, P_>(AIQ_TC_ARGS); \
+    return g.ks == 3 ? launch_tc<CS_, N_, 3, 2, P_>(AIQ_TC_ARGS) : launch_tc<CS_, N_, 1, 2, P_>(AIQ_TC_ARGS);    \
+  } while (0)
 #define AIQ_TC_CASE(CS_, N_)                                                                    \
-  if (g.Cin == CS_ && g.Cout == N_) {                                                           \
-    if (g.stride == 1) return g.ks == 3 ? launch_tc<CS_, N_, 3, 1>(AIQ_TC_ARGS) : launch_tc<CS_, N_, 1, 1>(AIQ_TC_ARGS); \
-    return g.ks == 3 ? launch_tc<CS_, N_, 3, 2>(AIQ_TC_ARGS) : launch_tc<CS_, N_, 1, 2>(AIQ_TC_ARGS);                    \
-  }
+  if (g.Cin == CS_ && g.Cout == N_ && pieces == 1) AIQ_TC_KS(CS_, N_, 1);
+#define AIQ_TC_CASE_WIDE(CS_, N_)                                                               \
+  if (g.Cin == CS_ && g.Cout == N_ && pieces == 2) AIQ_TC_KS(CS_, N_, 2);                       \
+  if (g.Cin == CS_ && g.Cout == N_ && pieces == 3) AIQ_TC_KS(CS_, N_, 3);
+  const int pieces = weight_bits <= 8 ? 1 : (weight_bits == 16 ? 2 : 3);
   AIQ_TC_CASE(16, 16) AIQ_TC_CASE(16, 32) AIQ_TC_CASE(16, 64)
   AIQ_TC_CASE(32, 16) AIQ_TC_CASE(32, 32) AIQ_TC_CASE(32, 64)
   AIQ_TC_CASE(64, 16) AIQ_TC_CASE(64, 32) AIQ_TC_CASE(64, 64)
+  AIQ_TC_CASE_WIDE(16, 16) AIQ_TC_CASE_WIDE(16, 32) AIQ_TC_CASE_WIDE(32, 16) AIQ_TC_CASE_WIDE(32, 32)
+#undef AIQ_TC_CASE_WIDE
+#undef AIQ_TC_KS
 #undef AIQ_TC_CASE
 #undef AIQ_TC_ARGS
   return set_error(AIQ_ERR_SHAPE, "conv_tc: no kernel for Cin=%d Cout=%d", g.Cin, g.Cout);

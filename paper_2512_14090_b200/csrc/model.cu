@@ -443,10 +443,11 @@ struct alignas(64) TensorMapBytes { uint8_t b[128]; };   // storage of one CUten
 
 struct LayerPlan {
   int n_versions = 0;
-  int n_tc = 0;                         // leading jobs that run on the tensor-core kernel
+  int n_tc = 0;                         // leading jobs that run on the tensor-core kernel (4- / 8-bit weights)
+  int n_tc16 = 0, n_tc32 = 0;           // then those with 16-bit and with 32-bit weights (tc_kind 1 only)
   int tc_kind = 0;                      // which tensor-core kernel (see layer_tensor_kind)
   double weight_bytes = 0.0;            // packed weights + scales + biases over all jobs
-  double weight_bytes_tc = 0.0;
+  double weight_bytes_tc = 0.0, weight_bytes_tc16 = 0.0, weight_bytes_tc32 = 0.0;
   TensorMapBytes in_map;                // over the input slot (tensor-core layers)
   TensorMapBytes out_map;               // over the output slot (pointwise tensor-core layers)
   size_t job_first = 0;                 // index of the first job record of this layer
@@ -510,14 +511,21 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
     plan.versions_total += lp.n_versions;
     if (li.d.kind != AIQ_LAYER_FC) {
       lp.job_first = plan.jobs.size();
-      // job order: versions the tensor-core kernel takes (4- / 8-bit weights) first
+      // job order: versions the tensor-core kernel takes first, grouped by weight class
+      // (4- / 8-bit codes, then 16-bit, then 32-bit where the kernel can hold their pieces)
       const bool tc_layer = layer_on_tensor_cores(m, li);
+      const bool tc_wide = tc_layer && layer_tensor_kind(m, li) == 1;
+      const ConvGeom g_cls = make_geom(m, li, B);
+      auto job_class = [&](int bits) -> int {      // 0: codes, 1: 16-bit, 2: 32-bit on tensor cores; 3: float32 kernel
+        if (tc_layer && bits <= 8) return 0;
+        if (tc_wide && bits == 16 && conv_tc_bits_ok(g_cls, 16)) return 1;
+        if (tc_wide && bits == 32 && conv_tc_bits_ok(g_cls, 32)) return 2;
+        return 3;
+      };
       std::vector<int> vorder;
-      for (int pass = 0; pass < 2; ++pass)
-        for (int v = 0; v < lp.n_versions; ++v) {
-          const bool tc = tc_layer && std::get<0>(keys[v]) <= 8;
-          if (tc == (pass == 0)) vorder.push_back(v);
-        }
+      for (int pass = 0; pass < 4; ++pass)
+        for (int v = 0; v < lp.n_versions; ++v)
+          if (job_class(std::get<0>(keys[v])) == pass) vorder.push_back(v);
       if (tc_layer) {
         const LayerInfo& src = m->layers[li.d.input];
         lp.tc_kind = layer_tensor_kind(m, li);
@@ -545,8 +553,12 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
         j.bits = bits;
         plan.jobs.push_back(j);
         const double wb = (double)li.d.cout * (row_bytes(li.K, bits) + 8.0);
-        if (tc_layer && bits <= 8) { lp.n_tc++; lp.weight_bytes_tc += wb; }
-        else lp.weight_bytes += wb;
+        switch (job_class(bits)) {
+          case 0: lp.n_tc++; lp.weight_bytes_tc += wb; break;
+          case 1: lp.n_tc16++; lp.weight_bytes_tc16 += wb; break;
+          case 2: lp.n_tc32++; lp.weight_bytes_tc32 += wb; break;
+          default: lp.weight_bytes += wb;
+        }
       }
       continue;
     }
@@ -638,12 +650,23 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
     }
     if (lp.n_tc > 0) {
       st = lp.tc_kind == 1
-          ? launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream)
+          ? launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, 8, stream)
           : launch_conv_pw_tc(g, &lp.in_map, &lp.out_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream);
       if (st != AIQ_OK) return st;
     }
-    if (lp.n_versions > lp.n_tc) {
-      st = launch_conv(g, jobs_dev + lp.job_first + lp.n_tc, lp.n_versions - lp.n_tc, x_chunk, lp.weight_bytes, stream);
+    int done = lp.n_tc;
+    if (lp.n_tc16 > 0) {
+      st = launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first + done, lp.n_tc16, plan.batch_capacity, m->status_word, lp.weight_bytes_tc16, 16, stream);
+      if (st != AIQ_OK) return st;
+      done += lp.n_tc16;
+    }
+    if (lp.n_tc32 > 0) {
+      st = launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first + done, lp.n_tc32, plan.batch_capacity, m->status_word, lp.weight_bytes_tc32, 32, stream);
+      if (st != AIQ_OK) return st;
+      done += lp.n_tc32;
+    }
+    if (lp.n_versions > done) {
+      st = launch_conv(g, jobs_dev + lp.job_first + done, lp.n_versions - done, x_chunk, lp.weight_bytes, stream);
       if (st != AIQ_OK) return st;
     }
   }
