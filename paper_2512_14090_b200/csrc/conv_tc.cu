@@ -50,6 +50,7 @@ struct TcParams {
   int n_stages;
   int K;                  // Cin * ks * ks (packed row length in elements)
   int ver_pair_rows;      // stride 2: row pairs per version of the input slot = capacity * (H + 2) / 2
+  int cs_out;             // multi-piece kernels: channels of an output pixel (N per blockIdx.z)
   int32_t* error_flag;    // device word, set to 1 when a bounded wait expired
 };
 
@@ -176,18 +177,6 @@ __device__ __forceinline__ void split_pair(float u0, float u1, uint32_t& hi2, ui
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptor, K-major, swizzled: rows of `swizzle bytes` pitch in groups
-// of 8; SBO = distance between groups.  layout: 2 = 128B, 4 = 64B, 6 = 32B swizzle.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t sbo_bytes, uint32_t layout) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr >> 4) & 0x3FFFu);
-  d |= (uint64_t)1 << 16;                               // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= (uint64_t)1 << 46;                               // descriptor version of sm_100
-  d |= (uint64_t)layout << 61;
-  return d;
-}
-
 // Eight packed codes (4 bits: raw.x; 8 bits: raw.x, raw.y; two's complement) -> eight
 // bfloat16, without the conversion unit: the offset-binary code is placed in the low
 // mantissa bits of 2^23, one subtraction gives the integer as a float, and because
@@ -271,6 +260,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
   // and every MMA is issued once per piece into the same accumulator.
   constexpr int pieces = PIECES;
   constexpr int wtaps = taps * pieces;           // weight tiles in shared memory
+  // The multi-piece kernels hold at most N = 32 output channels' weights: a layer of 2N output
+  // channels runs as two slices (blockIdx.z) that write their halves of every output pixel.
+  constexpr bool SLICED = PIECES > 1;
+  const int n_off = SLICED ? (int)blockIdx.z * N : 0;      // first output channel of this CTA
+  const int cs_out = SLICED ? p.cs_out : N;                // channels of an output pixel
   float* s_scale = reinterpret_cast<float*>(smem + S::scale(stages, wtaps));
   float* s_bias = reinterpret_cast<float*>(smem + S::bias(stages, wtaps));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::bars(stages, wtaps));
@@ -319,11 +313,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
   const uint32_t packed_bytes = wrow_bytes * N;
   if (tid == 0) {
     mbar_expect_tx(bar_w, packed_bytes);
-    bulk_load(smem_u32(ring), job.w, packed_bytes, bar_w);
+    bulk_load(smem_u32(ring), job.w + (size_t)n_off * wrow_bytes, packed_bytes, bar_w);
   }
   for (int i = tid; i < N; i += tc_threads(N)) {
-    s_scale[i] = job.scale[i];
-    s_bias[i] = job.bias[i];
+    s_scale[i] = job.scale[n_off + i];
+    s_bias[i] = job.bias[n_off + i];
   }
   bool alive = mbar_wait_warp(bar_w, 0, s_abort, p.error_flag);
   if (alive) {
@@ -335,7 +329,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       const int tap = u / (units_per_row * N);
       const uint8_t* row = ring + (size_t)n * wrow_bytes;
       const uint32_t off = swizzle_off((uint32_t)(n * L::W_ROW_BYTES + c8 * 16), L::W_SWZ_MASK);
-      if (PIECES > 1) {
+      if constexpr (PIECES > 1) {
         uint32_t pk[3][4];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -355,25 +349,25 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
           if (pc < pieces)
             *reinterpret_cast<uint4*>(wsm + (size_t)(pc * taps + tap) * L::W_TAP_BYTES + off) =
                 make_uint4(pk[pc][0], pk[pc][1], pk[pc][2], pk[pc][3]);
-        continue;
-      }
-      uint32_t packed[4];
+      } else {
+        uint32_t packed[4];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int k = (c8 * 8 + j) * taps + tap;             // element index in the (c, r, t) ordered row
-        int code;
-        if (job.bits == 8) {
-          code = (int)(int8_t)row[k];
-        } else {
-          const int byte = row[k >> 1];
-          const int nib = (k & 1) ? (byte >> 4) : (byte & 0xF);
-          code = (nib ^ 8) - 8;
+        for (int j = 0; j < 8; ++j) {
+          const int k = (c8 * 8 + j) * taps + tap;             // element index in the (c, r, t) ordered row
+          int code;
+          if (job.bits == 8) {
+            code = (int)(int8_t)row[k];
+          } else {
+            const int byte = row[k >> 1];
+            const int nib = (k & 1) ? (byte >> 4) : (byte & 0xF);
+            code = (nib ^ 8) - 8;
+          }
+          const uint32_t h = (uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code));
+          if (j & 1) packed[j >> 1] |= h << 16; else packed[j >> 1] = h;
         }
-        const uint32_t h = (uint32_t)__bfloat16_as_ushort(__int2bfloat16_rn(code));
-        if (j & 1) packed[j >> 1] |= h << 16; else packed[j >> 1] = h;
+        *reinterpret_cast<uint4*>(wsm + (size_t)tap * L::W_TAP_BYTES + off) =
+            make_uint4(packed[0], packed[1], packed[2], packed[3]);
       }
-      *reinterpret_cast<uint4*>(wsm + (size_t)tap * L::W_TAP_BYTES + off) =
-          make_uint4(packed[0], packed[1], packed[2], packed[3]);
     }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // expanded weights -> visible to the MMA
@@ -540,6 +534,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
     uint8_t* my_row = stg + lane * PIXB;
     const int my_key = (lane >> KEY_SHIFT) & KEY_MASK;
     const uint32_t pair_bar = 1u + (uint32_t)q;
+    // Global layout of a row of 8 output pixels: pixel pitch 4 cs_out bytes, [hi(cs_out) | lo(cs_out)].
+    // Staging unit u of the row (pixel u / UNITS, unit u % UNITS of [hi(N) | lo(N)]) lands at
+    // unit_off(u) bytes from the row's first pixel; without slices that is simply 16 u.
+    const size_t pix_pitch = SLICED ? (size_t)4 * cs_out : (size_t)PIXB;
+    auto unit_off = [&](int u) -> size_t {
+      if (!SLICED) return (size_t)u * 16;
+      const int px = u / UNITS, uu = u % UNITS;
+      const int half = uu >= UNITS / 2 ? 1 : 0;
+      return (size_t)px * pix_pitch + 2 * n_off + (half ? 2 * cs_out : 0) + (uu - half * (UNITS / 2)) * 16;
+    };
     // output row (image, padded y) of group gi of a tile, or -1 when the group is past the batch
     auto tile_row = [&](int t, int gi) -> int {
       const int trb = t / n_cb;
@@ -562,12 +566,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
 #pragma unroll
       for (int ii = 0; ii < RPW; ++ii) {
         const int jr = tile_row(t, q * 4 + RPW * h + ii);
-        const uint4* src = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(job.res) +
-                                                          ((size_t)(jr < 0 ? 0 : jr) * p.Wo + tcb * kColsPerTile) * PIXB);
+        const uint8_t* src = static_cast<const uint8_t*>(job.res) +
+                             ((size_t)(jr < 0 ? 0 : jr) * p.Wo + tcb * kColsPerTile) * pix_pitch;
 #pragma unroll
         for (int k = 0; k < RPL; ++k) {
           const int u = lane + 32 * k;
-          rpre[ii][k] = (jr >= 0 && u < 8 * UNITS) ? __ldg(src + u) : make_uint4(0u, 0u, 0u, 0u);
+          rpre[ii][k] = (jr >= 0 && u < 8 * UNITS) ? __ldg(reinterpret_cast<const uint4*>(src + unit_off(u)))
+                                                   : make_uint4(0u, 0u, 0u, 0u);
         }
       }
     };
@@ -666,12 +671,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
         const int i = RPW * h + ii;
         const int jr = out_row(q * 4 + i);
         if (jr >= 0) {
-          uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(job.out) +
-                                                ((size_t)jr * p.Wo + cb * kColsPerTile) * PIXB);
+          uint8_t* dst = static_cast<uint8_t*>(job.out) + ((size_t)jr * p.Wo + cb * kColsPerTile) * pix_pitch;
 #pragma unroll
           for (int u = lane; u < 8 * UNITS; u += 32) {
             const int pl = i * 8 + u / UNITS, uu = u % UNITS;
-            dst[u] = *reinterpret_cast<const uint4*>(stg + pl * PIXB + ((uu ^ ((pl >> KEY_SHIFT) & KEY_MASK)) << 4));
+            *reinterpret_cast<uint4*>(dst + unit_off(u)) =
+                *reinterpret_cast<const uint4*>(stg + pl * PIXB + ((uu ^ ((pl >> KEY_SHIFT) & KEY_MASK)) << 4));
           }
         }
       }
@@ -684,9 +689,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
           for (int side = 0; side < 2; ++side) {
             if (side == 0 ? !top : !bottom) continue;
             const int jr = bb * (p.Ho + 2) + (side == 0 ? 0 : p.Ho + 1);
-            uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(job.out) +
-                                                  ((size_t)jr * p.Wo + cb * kColsPerTile) * PIXB);
-            for (int u = lane; u < 8 * UNITS; u += 32) dst[u] = make_uint4(0u, 0u, 0u, 0u);
+            uint8_t* dst = static_cast<uint8_t*>(job.out) + ((size_t)jr * p.Wo + cb * kColsPerTile) * pix_pitch;
+            for (int u = lane; u < 8 * UNITS; u += 32)
+              *reinterpret_cast<uint4*>(dst + unit_off(u)) = make_uint4(0u, 0u, 0u, 0u);
           }
         }
       }
@@ -741,7 +746,7 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
   int stages = 0;
   for (int want = occ_cap; want >= 1 && !stages; --want) {
     const int per_cta = sm_budget / want - 1024;           // every block also reserves 1 KB
-    for (int st = 6; st >= (want > 1 ? 4 : 3); --st)
+    for (int st = 6; st >= (want > 1 ? 4 : (PIECES > 1 ? 2 : 3)); --st)
       if (S::total(st, taps) + 1024 <= per_cta && S::total(st, taps) + 1024 <= smem_limit) { stages = st; break; }
   }
   if (!stages)
@@ -759,6 +764,8 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
   p.B = g.B; p.H = g.H; p.W = g.W; p.Ho = g.Ho; p.Wo = g.Wo; p.ks = g.ks; p.stride = g.stride; p.act = g.act;
   p.n_stages = stages; p.K = g.K; p.error_flag = error_flag;
   p.ver_pair_rows = batch_capacity * (g.H + 2) / 2;
+  p.cs_out = g.Cout;
+  const int slices = g.Cout / N;                 // 1, or 2 output-channel slices (multi-piece kernels)
   int n_tiles;
   if (STRIDE == 1) {
     n_tiles = ((g.B * (g.H + 2) + kRowsPerTile - 1) / kRowsPerTile) * (g.Wo / kColsPerTile);
@@ -773,7 +780,7 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
   occ = occ > occ_cap ? occ_cap : (occ < 1 ? 1 : occ);
   // All CTAs of the launch should be resident at once (a second wave would run nearly alone):
   // split the resident capacity evenly over the jobs, rounding down.
-  int ctas = (n_sms * occ) / n_jobs;
+  int ctas = (n_sms * occ) / (n_jobs * slices);
   if (ctas > n_tiles) ctas = n_tiles;
   if (ctas < 1) ctas = 1;
   {
@@ -781,7 +788,7 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
                       2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
                       weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
                                                      (double)g.B * g.Ho * g.Wo * g.Cout));
-    conv_tc_kernel<CS, N, KS, STRIDE, PIECES><<<dim3(ctas, n_jobs), tc_threads(N), smem_bytes, s>>>(map, p, jobs_dev);
+    conv_tc_kernel<CS, N, KS, STRIDE, PIECES><<<dim3(ctas, n_jobs, slices), tc_threads(N), smem_bytes, s>>>(map, p, jobs_dev);
   }
   AIQ_LAUNCH_CHECK("conv_tc");
   return AIQ_OK;
@@ -927,8 +934,10 @@ aiq_status_t conv_tc_encode_map(const ConvGeom& g, const void* slot_base, int ba
 }
 
 bool conv_tc_bits_ok(const ConvGeom& g, int bits) {
-  // 2 or 3 weight tiles per tap must fit shared memory beside the activation ring
-  return bits <= 8 || (g.Cin <= 32 && g.Cout <= 32);
+  // 2 or 3 weight tiles per tap of a 32-channel output slice fit shared memory beside an
+  // activation ring of at least two stages for every eligible shape
+  (void)g;
+  return bits == 4 || bits == 8 || bits == 16 || bits == 32;
 }
 
 aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
@@ -944,13 +953,15 @@ aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* 
 #define AIQ_TC_CASE(CS_, N_)                                                                    \
   if (g.Cin == CS_ && g.Cout == N_ && pieces == 1) AIQ_TC_KS(CS_, N_, 1);
 #define AIQ_TC_CASE_WIDE(CS_, N_)                                                               \
-  if (g.Cin == CS_ && g.Cout == N_ && pieces == 2) AIQ_TC_KS(CS_, N_, 2);                       \
-  if (g.Cin == CS_ && g.Cout == N_ && pieces == 3) AIQ_TC_KS(CS_, N_, 3);
+  if (g.Cin == CS_ && (g.Cout == N_ || g.Cout == 2 * N_) && pieces == 2) AIQ_TC_KS(CS_, N_, 2); \
+  if (g.Cin == CS_ && (g.Cout == N_ || g.Cout == 2 * N_) && pieces == 3) AIQ_TC_KS(CS_, N_, 3);
   const int pieces = weight_bits <= 8 ? 1 : (weight_bits == 16 ? 2 : 3);
   AIQ_TC_CASE(16, 16) AIQ_TC_CASE(16, 32) AIQ_TC_CASE(16, 64)
   AIQ_TC_CASE(32, 16) AIQ_TC_CASE(32, 32) AIQ_TC_CASE(32, 64)
   AIQ_TC_CASE(64, 16) AIQ_TC_CASE(64, 32) AIQ_TC_CASE(64, 64)
-  AIQ_TC_CASE_WIDE(16, 16) AIQ_TC_CASE_WIDE(16, 32) AIQ_TC_CASE_WIDE(32, 16) AIQ_TC_CASE_WIDE(32, 32)
+  // 16- / 32-bit weights: at most 32 output channels per slice, 64 run as two slices of 32
+  AIQ_TC_CASE_WIDE(16, 32) AIQ_TC_CASE_WIDE(32, 32) AIQ_TC_CASE_WIDE(64, 32)
+  AIQ_TC_CASE_WIDE(16, 16) AIQ_TC_CASE_WIDE(32, 16) AIQ_TC_CASE_WIDE(64, 16)
 #undef AIQ_TC_CASE_WIDE
 #undef AIQ_TC_KS
 #undef AIQ_TC_CASE
