@@ -36,9 +36,9 @@ UNIT = "scheme-evals/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the
 # committed ncu summary under profiles/ (None until captured / after the kernel changed)
-# conv_tc_kernel: 197.6 MB per launch measured at chunk 256 (profiles/conv_tc__resnet20_greedy_step.md),
+# conv_tc_kernel: 197.9 MB per launch measured at chunk 256 (profiles/conv_tc__resnet20_greedy_step.md),
 # scaled by 4 to the default chunk of 1024 images (traffic grows with the images of a launch)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 197.6e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 197.9e6
 
 
 def measured_peaks():
