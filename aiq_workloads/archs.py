@@ -140,6 +140,21 @@ def tiny_net(in_c=3, hw=8, n_classes=5):
     return dict(name="tiny_net", in_c=in_c, in_h=hw, in_w=hw, n_classes=n_classes, layers=layers)
 
 
+def depthwise_stack(hw, channels=96, n_classes=7):
+    """A short network around two depthwise layers (test workload): stem 3x3, depthwise 3x3 at
+    stride 2, pointwise, depthwise 3x3 at stride 1 with a shortcut from its own input,
+    classifier.  `hw` sets the image size, so the depthwise layers see any output height."""
+    c = channels
+    layers = [
+        _conv("stem", 3, c, 3, 1, "relu6", -1),
+        _conv("dw.s2", c, c, 3, 2, "relu6", 0, kind="dw"),
+        _conv("pw", c, c, 1, 1, "none", 1),
+        _conv("dw.s1", c, c, 3, 1, "relu6", 2, residual=2, kind="dw"),
+        _fc("fc", c, n_classes, 3),
+    ]
+    return dict(name=f"depthwise_stack_{hw}", in_c=3, in_h=hw, in_w=hw, n_classes=n_classes, layers=layers)
+
+
 def conv_layer_indices(arch):
     """Indices of every layer that is not the classifier (the sweep candidates)."""
     return [i for i, l in enumerate(arch["layers"]) if l["kind"] != "fc"]

@@ -12,6 +12,12 @@
 //   - the 9 x C expanded weights, scales and biases sit in shared memory; blocks are
 //     persistent (grid-stride over items).
 // Rows 0 and Ho+1 of every output image (the physical padding rows) are written as zeros.
+//
+// Two kernels share this organisation.  depthwise3x3_kernel gives a thread one output row of
+// its columns: every output row re-reads its three input rows (from L1 / L2), which is fine
+// for small launches that need the parallelism.  depthwise3x3_walk_kernel gives a thread up to
+// 16 consecutive output rows: it walks down the input rows once, each row feeding the (up to
+// three) output rows it belongs to.
 #include "common.cuh"
 
 namespace aiq {
@@ -47,11 +53,12 @@ __device__ __forceinline__ void store8(void* __restrict__ base, size_t pixel, in
     uint32_t hw[4], lw[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      __nv_bfloat16 h0, l0, h1, l1;
-      split_bf16(v[2 * i], h0, l0);
-      split_bf16(v[2 * i + 1], h1, l1);
-      hw[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-      lw[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+      // hi = bf16_rn(v), lo = bf16_rn(v - hi), two values per packed conversion (the roundings of split_bf16)
+      const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      hw[i] = *reinterpret_cast<const uint32_t*>(&h);
+      const __nv_bfloat162 l = __floats2bfloat162_rn(v[2 * i] - __uint_as_float(hw[i] << 16),
+                                                     v[2 * i + 1] - __uint_as_float(hw[i] & 0xFFFF0000u));
+      lw[i] = *reinterpret_cast<const uint32_t*>(&l);
     }
     *reinterpret_cast<uint4*>(px + c) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
     *reinterpret_cast<uint4*>(px + Cs + c) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
@@ -59,6 +66,22 @@ __device__ __forceinline__ void store8(void* __restrict__ base, size_t pixel, in
     float* px = static_cast<float*>(base) + pixel * Cs + c;
     *reinterpret_cast<float4*>(px) = make_float4(v[0], v[1], v[2], v[3]);
     *reinterpret_cast<float4*>(px + 4) = make_float4(v[4], v[5], v[6], v[7]);
+  }
+}
+
+// Expanded weights [9][Cs], scales [Cs] and biases [Cs] of one job -> shared memory.  A thread
+// takes whole channels: the first tap brings the packed row (32 elements, 16 .. 128 bytes) into
+// L1 and the other eight taps hit it, and the channels of a thread are independent loads.
+__device__ __forceinline__ void stage_dw_params(const LayerJob& job, int Cout, int Cs, float* wsm, float* ssm, float* bsm) {
+  const int wrow_bytes = 32 * job.bits / 8;              // K = 9 pads to 32 elements
+#pragma unroll 4
+  for (int c = threadIdx.x; c < Cs; c += kDwThreads) {
+    const bool real = c < Cout;
+    const uint8_t* row = job.w + (size_t)(real ? c : 0) * wrow_bytes;
+#pragma unroll
+    for (int tap = 0; tap < 9; ++tap) wsm[tap * Cs + c] = real ? load_element(row, tap, job.bits) : 0.f;
+    ssm[c] = real ? job.scale[c] : 0.f;
+    bsm[c] = real ? job.bias[c] : 0.f;
   }
 }
 
@@ -71,15 +94,7 @@ depthwise3x3_kernel(ConvGeom g, const LayerJob* __restrict__ jobs) {
   float* wsm = dsm;
   float* ssm = dsm + 9 * Cs;
   float* bsm = ssm + Cs;
-  const int wrow_bytes = 32 * job.bits / 8;              // K = 9 pads to 32 elements
-  for (int i = threadIdx.x; i < 9 * Cs; i += kDwThreads) {
-    const int tap = i / Cs, c = i - tap * Cs;
-    wsm[i] = c < g.Cout ? load_element(job.w + (size_t)c * wrow_bytes, tap, job.bits) : 0.f;
-  }
-  for (int c = threadIdx.x; c < Cs; c += kDwThreads) {
-    ssm[c] = c < g.Cout ? job.scale[c] : 0.f;
-    bsm[c] = c < g.Cout ? job.bias[c] : 0.f;
-  }
+  stage_dw_params(job, g.Cout, Cs, wsm, ssm, bsm);
   __syncthreads();
 
   constexpr int IN_COLS = (kDwCols - 1) * STRIDE + 3;    // 6 or 9 input columns per thread
@@ -155,6 +170,195 @@ depthwise3x3_kernel(ConvGeom g, const LayerJob* __restrict__ jobs) {
   }
 }
 
+
+// Row-walking kernel.  A thread owns 8 channels x kDwCols output columns and walks down up to
+// `rb` consecutive output rows of one image, loading every input row once:
+//   stride 1: input row y feeds output rows y - 1 (tap row 2), y (tap row 1) and y + 1 (tap row
+//             0), held in three accumulator sets whose roles rotate from row to row;
+//   stride 2: output row j takes input rows 2j - 1, 2j, 2j + 1; row 2j + 1 is also the first
+//             tap row of output j + 1, whose product is carried over.
+// The row loop is a real loop (three rotated copies of the body at stride 1), so the code stays
+// small whatever `rb` is.
+template <int FMT, int STRIDE>
+__device__ __forceinline__ void dw_load_row(const void* __restrict__ in, size_t row_pix, int ix0, int W, int c, int Cs,
+                                            float (&v)[(kDwCols - 1) * STRIDE + 3][8]) {
+#pragma unroll
+  for (int xx = 0; xx < (kDwCols - 1) * STRIDE + 3; ++xx) {
+    const int ix = ix0 + xx;
+    if (ix >= 0 && ix < W) {
+      load8<FMT>(in, row_pix + ix, c, Cs, v[xx]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[xx][i] = 0.f;
+    }
+  }
+}
+
+// acc[x][i] (+)= sum_t in[x * STRIDE + t][i] * w[(r, t)][c + i]
+template <int STRIDE, bool ACCUMULATE>
+__device__ __forceinline__ void dw_tap_row(const float* __restrict__ wsm, int Cs, int c, int r,
+                                           const float (&in)[(kDwCols - 1) * STRIDE + 3][8], float (&acc)[kDwCols][8]) {
+#pragma unroll
+  for (int t = 0; t < 3; ++t) {
+    const float4 w0 = *reinterpret_cast<const float4*>(wsm + (r * 3 + t) * Cs + c);
+    const float4 w1 = *reinterpret_cast<const float4*>(wsm + (r * 3 + t) * Cs + c + 4);
+    const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+    for (int x = 0; x < kDwCols; ++x)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float prev = (ACCUMULATE || t > 0) ? acc[x][i] : 0.f;
+        acc[x][i] = fmaf(in[x * STRIDE + t][i], wv[i], prev);
+      }
+  }
+}
+
+template <int FMT, int STRIDE>
+__global__ void __launch_bounds__(kDwThreads, 2)
+depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) {
+  extern __shared__ __align__(16) float dsm[];          // [9][Cs] weights, [Cs] scale, [Cs] bias
+  const LayerJob job = jobs[blockIdx.y];
+  const int Cs = g.Cs_out;                               // == Cs_in
+  float* wsm = dsm;
+  float* ssm = dsm + 9 * Cs;
+  float* bsm = ssm + Cs;
+  stage_dw_params(job, g.Cout, Cs, wsm, ssm, bsm);
+  __syncthreads();
+
+  constexpr int IN_COLS = (kDwCols - 1) * STRIDE + 3;    // input columns per thread
+  const int octs = Cs / 8;
+  const int col_groups = (g.Wo + kDwCols - 1) / kDwCols;
+  const int row_blocks = (g.Ho + rb - 1) / rb;
+  const bool clamp = g.act != AIQ_ACT_NONE;              // relu: [0, inf), relu6: [0, 6]
+  const float act_hi = g.act == AIQ_ACT_RELU6 ? 6.0f : __int_as_float(0x7f800000);
+  const long long n_items = (long long)g.B * row_blocks * col_groups * octs;
+  for (long long item = (long long)blockIdx.x * kDwThreads + threadIdx.x; item < n_items;
+       item += (long long)gridDim.x * kDwThreads) {
+    const int oct = (int)(item % octs);
+    long long rest = item / octs;
+    const int cg = (int)(rest % col_groups);
+    rest /= col_groups;
+    const int rbk = (int)(rest % row_blocks);
+    const int b = (int)(rest / row_blocks);
+    const int c = oct * 8, ox0 = cg * kDwCols;
+    const int oy0 = rbk * rb;                            // first (unpadded) output row of the block
+    const int n_out = min(rb, g.Ho - oy0);               // output rows of this block
+    const size_t out_row0 = (size_t)b * (g.Ho + 2);      // padded output row 0 of the image
+    const size_t in_row0 = (size_t)b * (g.H + 2) + 1;    // padded input row of unpadded row 0
+    const int ix0 = ox0 * STRIDE - 1;
+
+    // finish and store output row oy (unpadded) from its accumulators
+    auto emit = [&](int oy, const float (&acc)[kDwCols][8]) {
+      const float4 s0 = *reinterpret_cast<const float4*>(ssm + c), s1 = *reinterpret_cast<const float4*>(ssm + c + 4);
+      const float4 b0 = *reinterpret_cast<const float4*>(bsm + c), b1 = *reinterpret_cast<const float4*>(bsm + c + 4);
+      const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+      const float bi[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+      for (int x = 0; x < kDwCols; ++x) {
+        const int ox = ox0 + x;
+        if (ox >= g.Wo) break;
+        const size_t opix = (out_row0 + oy + 1) * g.Wo + ox;
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = fmaf(acc[x][i], sc[i], bi[i]);
+        if (job.res) {
+          float rs[8];
+          load8<FMT>(job.res, opix, c, Cs, rs);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) v[i] += rs[i];
+        }
+        if (clamp) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) v[i] = fminf(fmaxf(v[i], 0.f), act_hi);
+        }
+        if (c + 8 > g.Cout) {                            // padding channels of the last octet stay zero
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            if (c + i >= g.Cout) v[i] = 0.f;
+        }
+        store8<FMT>(job.out, opix, c, Cs, v);
+      }
+    };
+
+    if (STRIDE == 1) {
+      // k-th input row of the block = unpadded row oy0 - 1 + k, k = 0 .. n_out + 1.  a0 / a1 / a2
+      // belong to output rows oy0 + k - 2 / k - 1 / k; a0 is complete after this row.
+      auto step = [&](int k, float (&a0)[kDwCols][8], float (&a1)[kDwCols][8], float (&a2)[kDwCols][8]) {
+        const int iy = oy0 - 1 + k;
+        const bool have = iy >= 0 && iy < g.H;
+        float in[IN_COLS][8];
+        if (have) dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, ix0, g.W, c, Cs, in);
+        if (have && k >= 2) dw_tap_row<STRIDE, true>(wsm, Cs, c, 2, in, a0);
+        if (have && k >= 1 && k <= n_out) dw_tap_row<STRIDE, true>(wsm, Cs, c, 1, in, a1);
+        if (have && k < n_out) {
+          dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, a2);
+        } else {
+#pragma unroll
+          for (int x = 0; x < kDwCols; ++x)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) a2[x][i] = 0.f;
+        }
+        if (k >= 2) emit(oy0 + k - 2, a0);
+      };
+      float A[kDwCols][8], B[kDwCols][8], C[kDwCols][8];
+#pragma unroll
+      for (int x = 0; x < kDwCols; ++x)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) A[x][i] = B[x][i] = 0.f;
+      const int n_rows = n_out + 2;
+      for (int k = 0; k < n_rows; k += 3) {
+        step(k, A, B, C);
+        if (k + 1 < n_rows) step(k + 1, B, C, A);
+        if (k + 2 < n_rows) step(k + 2, C, A, B);
+      }
+    } else {
+      // output row j of the block takes unpadded input rows 2 (oy0 + j) - 1, .., + 1
+      float acc[kDwCols][8], carry[kDwCols][8];
+      float in[IN_COLS][8];
+#pragma unroll
+      for (int x = 0; x < kDwCols; ++x)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) carry[x][i] = 0.f;
+      {
+        const int iy = 2 * oy0 - 1;
+        if (iy >= 0) {
+          dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, ix0, g.W, c, Cs, in);
+          dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, carry);
+        }
+      }
+      for (int j = 0; j < n_out; ++j) {
+        const int iy = 2 * (oy0 + j);
+#pragma unroll
+        for (int x = 0; x < kDwCols; ++x)
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { acc[x][i] = carry[x][i]; carry[x][i] = 0.f; }
+        if (iy < g.H) {
+          dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, ix0, g.W, c, Cs, in);
+          dw_tap_row<STRIDE, true>(wsm, Cs, c, 1, in, acc);
+        }
+        if (iy + 1 < g.H) {
+          dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy + 1) * g.W, ix0, g.W, c, Cs, in);
+          dw_tap_row<STRIDE, true>(wsm, Cs, c, 2, in, acc);
+          if (j + 1 < n_out) dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, carry);
+        }
+        emit(oy0 + j, acc);
+      }
+    }
+    // the two physical padding rows of the image, by the first and the last row block
+    if (rbk == 0 || rbk == row_blocks - 1) {
+      const float zero[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+      for (int side = 0; side < 2; ++side) {
+        if (side == 0 ? rbk != 0 : rbk != row_blocks - 1) continue;
+        const size_t jr = out_row0 + (side == 0 ? 0 : g.Ho + 1);
+#pragma unroll
+        for (int x = 0; x < kDwCols; ++x)
+          if (ox0 + x < g.Wo) store8<FMT>(job.out, jr * g.Wo + ox0 + x, c, Cs, zero);
+      }
+    }
+  }
+}
+
 }  // namespace
 
 aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n_jobs,
@@ -169,15 +373,31 @@ aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n
     AIQ_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
   }
   if (smem > 48 * 1024) return set_error(AIQ_ERR_SHAPE, "depthwise: %d channels need %zu bytes of shared memory", g.Cout, smem);
-  const long long n_items = (long long)g.B * (g.Ho + 2) * ((g.Wo + kDwCols - 1) / kDwCols) * (Cs / 8);
+  const int col_groups = (g.Wo + kDwCols - 1) / kDwCols;
+  // Rows per thread of the row-walking kernel: the image height cut into the fewest blocks of at
+  // most 16 rows, of equal height where it divides.  The kernel is used when it still gives
+  // every SM a block of threads; smaller launches need the parallelism of one row per thread.
+  const int n_blk = (g.Ho + 15) / 16;
+  const int rb = (g.Ho + n_blk - 1) / n_blk;
+  const long long items_rows = (long long)g.B * n_blk * col_groups * (Cs / 8);
+  const bool walk_rows = items_rows >= (long long)n_sms * kDwThreads;
+  const long long n_items = walk_rows ? items_rows : (long long)g.B * (g.Ho + 2) * col_groups * (Cs / 8);
   long long blocks = (n_items + kDwThreads - 1) / kDwThreads;
-  const long long cap = (long long)n_sms * 4;                 // persistent: as many blocks as are resident (4 per SM)
+  const long long cap = (long long)n_sms * (walk_rows ? 2 : 4);   // persistent: as many blocks as are resident
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   dim3 grid((unsigned)blocks, n_jobs);
   LaunchScope scope(AIQ_KERNEL_DEPTHWISE, s, 18.0 * g.B * g.Ho * g.Wo * g.Cout * n_jobs,
                     weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
                                                    (double)g.B * g.Ho * g.Wo * g.Cout));
+  if (walk_rows) {
+#define AIQ_DWR(FMT_, ST_) depthwise3x3_walk_kernel<FMT_, ST_><<<grid, kDwThreads, smem, s>>>(g, jobs_dev, rb)
+    if (g.act_format == ACT_SPLIT) { if (g.stride == 1) AIQ_DWR(ACT_SPLIT, 1); else AIQ_DWR(ACT_SPLIT, 2); }
+    else { if (g.stride == 1) AIQ_DWR(ACT_F32, 1); else AIQ_DWR(ACT_F32, 2); }
+#undef AIQ_DWR
+    AIQ_LAUNCH_CHECK("depthwise3x3_walk");
+    return AIQ_OK;
+  }
 #define AIQ_DW(FMT_, ST_) depthwise3x3_kernel<FMT_, ST_><<<grid, kDwThreads, smem, s>>>(g, jobs_dev)
   if (g.act_format == ACT_SPLIT) { if (g.stride == 1) AIQ_DW(ACT_SPLIT, 1); else AIQ_DW(ACT_SPLIT, 2); }
   else { if (g.stride == 1) AIQ_DW(ACT_F32, 1); else AIQ_DW(ACT_F32, 2); }
