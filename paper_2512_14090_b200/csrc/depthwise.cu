@@ -178,19 +178,17 @@ depthwise3x3_kernel(ConvGeom g, const LayerJob* __restrict__ jobs) {
 //   stride 2: output row j takes input rows 2j - 1, 2j, 2j + 1; row 2j + 1 is also the first
 //             tap row of output j + 1, whose product is carried over.
 // The row loop is a real loop (three rotated copies of the body at stride 1), so the code stays
-// small whatever `rb` is.
+// small whatever `rb` is.  Input rows -1 and H are the physical padding rows of the image, which
+// every kernel writes as zeros: they are loaded like any other row.
+// Input columns ix0 .. of one row.  A column outside the image reads `zero_pix`, a pixel of the
+// image's first physical padding row (always zeros), so no value has to be patched afterwards.
 template <int FMT, int STRIDE>
-__device__ __forceinline__ void dw_load_row(const void* __restrict__ in, size_t row_pix, int ix0, int W, int c, int Cs,
-                                            float (&v)[(kDwCols - 1) * STRIDE + 3][8]) {
+__device__ __forceinline__ void dw_load_row(const void* __restrict__ in, size_t row_pix, size_t zero_pix, int ix0, int W,
+                                            int c, int Cs, float (&v)[(kDwCols - 1) * STRIDE + 3][8]) {
 #pragma unroll
   for (int xx = 0; xx < (kDwCols - 1) * STRIDE + 3; ++xx) {
     const int ix = ix0 + xx;
-    if (ix >= 0 && ix < W) {
-      load8<FMT>(in, row_pix + ix, c, Cs, v[xx]);
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) v[xx][i] = 0.f;
-    }
+    load8<FMT>(in, (ix >= 0 && ix < W) ? row_pix + ix : zero_pix, c, Cs, v[xx]);
   }
 }
 
@@ -245,6 +243,7 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
     const int n_out = min(rb, g.Ho - oy0);               // output rows of this block
     const size_t out_row0 = (size_t)b * (g.Ho + 2);      // padded output row 0 of the image
     const size_t in_row0 = (size_t)b * (g.H + 2) + 1;    // padded input row of unpadded row 0
+    const size_t zero_pix = (in_row0 - 1) * g.W;         // a pixel of zeros (padding row)
     const int ix0 = ox0 * STRIDE - 1;
 
     // finish and store output row oy (unpadded) from its accumulators
@@ -284,20 +283,13 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
       // k-th input row of the block = unpadded row oy0 - 1 + k, k = 0 .. n_out + 1.  a0 / a1 / a2
       // belong to output rows oy0 + k - 2 / k - 1 / k; a0 is complete after this row.
       auto step = [&](int k, float (&a0)[kDwCols][8], float (&a1)[kDwCols][8], float (&a2)[kDwCols][8]) {
-        const int iy = oy0 - 1 + k;
-        const bool have = iy >= 0 && iy < g.H;
+        const int iy = oy0 - 1 + k;                      // -1 .. H
         float in[IN_COLS][8];
-        if (have) dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, ix0, g.W, c, Cs, in);
-        if (have && k >= 2) dw_tap_row<STRIDE, true>(wsm, Cs, c, 2, in, a0);
-        if (have && k >= 1 && k <= n_out) dw_tap_row<STRIDE, true>(wsm, Cs, c, 1, in, a1);
-        if (have && k < n_out) {
-          dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, a2);
-        } else {
-#pragma unroll
-          for (int x = 0; x < kDwCols; ++x)
-#pragma unroll
-            for (int i = 0; i < 8; ++i) a2[x][i] = 0.f;
-        }
+        dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, zero_pix, ix0, g.W, c, Cs, in);
+        // rows that belong to a neighbouring block are accumulated too and never stored
+        dw_tap_row<STRIDE, true>(wsm, Cs, c, 2, in, a0);
+        dw_tap_row<STRIDE, true>(wsm, Cs, c, 1, in, a1);
+        dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, a2);
         if (k >= 2) emit(oy0 + k - 2, a0);
       };
       float A[kDwCols][8], B[kDwCols][8], C[kDwCols][8];
@@ -319,28 +311,19 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
       for (int x = 0; x < kDwCols; ++x)
 #pragma unroll
         for (int i = 0; i < 8; ++i) carry[x][i] = 0.f;
-      {
-        const int iy = 2 * oy0 - 1;
-        if (iy >= 0) {
-          dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, ix0, g.W, c, Cs, in);
-          dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, carry);
-        }
-      }
+      dw_load_row<FMT, STRIDE>(job.in, (in_row0 + 2 * oy0 - 1) * g.W, zero_pix, ix0, g.W, c, Cs, in);
+      dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, carry);
       for (int j = 0; j < n_out; ++j) {
-        const int iy = 2 * (oy0 + j);
+        const int iy = 2 * (oy0 + j);                    // rows iy, iy + 1 <= H
+        dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, zero_pix, ix0, g.W, c, Cs, in);
 #pragma unroll
         for (int x = 0; x < kDwCols; ++x)
 #pragma unroll
-          for (int i = 0; i < 8; ++i) { acc[x][i] = carry[x][i]; carry[x][i] = 0.f; }
-        if (iy < g.H) {
-          dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, ix0, g.W, c, Cs, in);
-          dw_tap_row<STRIDE, true>(wsm, Cs, c, 1, in, acc);
-        }
-        if (iy + 1 < g.H) {
-          dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy + 1) * g.W, ix0, g.W, c, Cs, in);
-          dw_tap_row<STRIDE, true>(wsm, Cs, c, 2, in, acc);
-          if (j + 1 < n_out) dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, carry);
-        }
+          for (int i = 0; i < 8; ++i) acc[x][i] = carry[x][i];
+        dw_tap_row<STRIDE, true>(wsm, Cs, c, 1, in, acc);
+        dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy + 1) * g.W, zero_pix, ix0, g.W, c, Cs, in);
+        dw_tap_row<STRIDE, true>(wsm, Cs, c, 2, in, acc);
+        dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, carry);
         emit(oy0 + j, acc);
       }
     }
