@@ -26,6 +26,7 @@ namespace {
 
 constexpr int kDwThreads = 256;
 constexpr int kDwCols = 2;        // output columns per thread
+constexpr int kWalkCh = 4;        // channels per thread of the row-walking kernel
 
 template <int FMT>
 __device__ __forceinline__ void load8(const void* __restrict__ base, size_t pixel, int c, int Cs, float* v) {
@@ -171,7 +172,45 @@ depthwise3x3_kernel(ConvGeom g, const LayerJob* __restrict__ jobs) {
 }
 
 
-// Row-walking kernel.  A thread owns 8 channels x kDwCols output columns and walks down up to
+// Four channels of one pixel (the unit of the row-walking kernel)
+template <int FMT>
+__device__ __forceinline__ void load4(const void* __restrict__ base, size_t pixel, int c, int Cs, float* v) {
+  if (FMT == ACT_SPLIT) {
+    const __nv_bfloat16* px = static_cast<const __nv_bfloat16*>(base) + pixel * 2 * Cs;
+    const uint2 h = __ldg(reinterpret_cast<const uint2*>(px + c));
+    const uint2 l = __ldg(reinterpret_cast<const uint2*>(px + Cs + c));
+    v[0] = __uint_as_float(h.x << 16) + __uint_as_float(l.x << 16);            // a bfloat16 is the upper half of a float
+    v[1] = __uint_as_float(h.x & 0xFFFF0000u) + __uint_as_float(l.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(h.y << 16) + __uint_as_float(l.y << 16);
+    v[3] = __uint_as_float(h.y & 0xFFFF0000u) + __uint_as_float(l.y & 0xFFFF0000u);
+  } else {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(base) + pixel * Cs + c));
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  }
+}
+
+template <int FMT>
+__device__ __forceinline__ void store4(void* __restrict__ base, size_t pixel, int c, int Cs, const float* v) {
+  if (FMT == ACT_SPLIT) {
+    __nv_bfloat16* px = static_cast<__nv_bfloat16*>(base) + pixel * 2 * Cs;
+    uint32_t hw[2], lw[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      // hi = bf16_rn(v), lo = bf16_rn(v - hi), two values per packed conversion (the roundings of split_bf16)
+      const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      hw[i] = *reinterpret_cast<const uint32_t*>(&h);
+      const __nv_bfloat162 l = __floats2bfloat162_rn(v[2 * i] - __uint_as_float(hw[i] << 16),
+                                                     v[2 * i + 1] - __uint_as_float(hw[i] & 0xFFFF0000u));
+      lw[i] = *reinterpret_cast<const uint32_t*>(&l);
+    }
+    *reinterpret_cast<uint2*>(px + c) = make_uint2(hw[0], hw[1]);
+    *reinterpret_cast<uint2*>(px + Cs + c) = make_uint2(lw[0], lw[1]);
+  } else {
+    *reinterpret_cast<float4*>(static_cast<float*>(base) + pixel * Cs + c) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+}
+
+// Row-walking kernel.  A thread owns kWalkCh = 4 channels x kDwCols output columns and walks down up to
 // `rb` consecutive output rows of one image, loading every input row once:
 //   stride 1: input row y feeds output rows y - 1 (tap row 2), y (tap row 1) and y + 1 (tap row
 //             0), held in three accumulator sets whose roles rotate from row to row;
@@ -184,27 +223,26 @@ depthwise3x3_kernel(ConvGeom g, const LayerJob* __restrict__ jobs) {
 // image's first physical padding row (always zeros), so no value has to be patched afterwards.
 template <int FMT, int STRIDE>
 __device__ __forceinline__ void dw_load_row(const void* __restrict__ in, size_t row_pix, size_t zero_pix, int ix0, int W,
-                                            int c, int Cs, float (&v)[(kDwCols - 1) * STRIDE + 3][8]) {
+                                            int c, int Cs, float (&v)[(kDwCols - 1) * STRIDE + 3][kWalkCh]) {
 #pragma unroll
   for (int xx = 0; xx < (kDwCols - 1) * STRIDE + 3; ++xx) {
     const int ix = ix0 + xx;
-    load8<FMT>(in, (ix >= 0 && ix < W) ? row_pix + ix : zero_pix, c, Cs, v[xx]);
+    load4<FMT>(in, (ix >= 0 && ix < W) ? row_pix + ix : zero_pix, c, Cs, v[xx]);
   }
 }
 
 // acc[x][i] (+)= sum_t in[x * STRIDE + t][i] * w[(r, t)][c + i]
 template <int STRIDE, bool ACCUMULATE>
 __device__ __forceinline__ void dw_tap_row(const float* __restrict__ wsm, int Cs, int c, int r,
-                                           const float (&in)[(kDwCols - 1) * STRIDE + 3][8], float (&acc)[kDwCols][8]) {
+                                           const float (&in)[(kDwCols - 1) * STRIDE + 3][kWalkCh], float (&acc)[kDwCols][kWalkCh]) {
 #pragma unroll
   for (int t = 0; t < 3; ++t) {
     const float4 w0 = *reinterpret_cast<const float4*>(wsm + (r * 3 + t) * Cs + c);
-    const float4 w1 = *reinterpret_cast<const float4*>(wsm + (r * 3 + t) * Cs + c + 4);
-    const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+    const float wv[kWalkCh] = {w0.x, w0.y, w0.z, w0.w};
 #pragma unroll
     for (int x = 0; x < kDwCols; ++x)
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < kWalkCh; ++i) {
         const float prev = (ACCUMULATE || t > 0) ? acc[x][i] : 0.f;
         acc[x][i] = fmaf(in[x * STRIDE + t][i], wv[i], prev);
       }
@@ -212,7 +250,7 @@ __device__ __forceinline__ void dw_tap_row(const float* __restrict__ wsm, int Cs
 }
 
 template <int FMT, int STRIDE>
-__global__ void __launch_bounds__(kDwThreads, 2)
+__global__ void __launch_bounds__(kDwThreads, 3)
 depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) {
   extern __shared__ __align__(16) float dsm[];          // [9][Cs] weights, [Cs] scale, [Cs] bias
   const LayerJob job = jobs[blockIdx.y];
@@ -224,7 +262,7 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
   __syncthreads();
 
   constexpr int IN_COLS = (kDwCols - 1) * STRIDE + 3;    // input columns per thread
-  const int octs = Cs / 8;
+  const int octs = Cs / kWalkCh;                         // channel groups
   const int col_groups = (g.Wo + kDwCols - 1) / kDwCols;
   const int row_blocks = (g.Ho + rb - 1) / rb;
   const bool clamp = g.act != AIQ_ACT_NONE;              // relu: [0, inf), relu6: [0, 6]
@@ -238,7 +276,7 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
     rest /= col_groups;
     const int rbk = (int)(rest % row_blocks);
     const int b = (int)(rest / row_blocks);
-    const int c = oct * 8, ox0 = cg * kDwCols;
+    const int c = oct * kWalkCh, ox0 = cg * kDwCols;
     const int oy0 = rbk * rb;                            // first (unpadded) output row of the block
     const int n_out = min(rb, g.Ho - oy0);               // output rows of this block
     const size_t out_row0 = (size_t)b * (g.Ho + 2);      // padded output row 0 of the image
@@ -247,44 +285,44 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
     const int ix0 = ox0 * STRIDE - 1;
 
     // finish and store output row oy (unpadded) from its accumulators
-    auto emit = [&](int oy, const float (&acc)[kDwCols][8]) {
-      const float4 s0 = *reinterpret_cast<const float4*>(ssm + c), s1 = *reinterpret_cast<const float4*>(ssm + c + 4);
-      const float4 b0 = *reinterpret_cast<const float4*>(bsm + c), b1 = *reinterpret_cast<const float4*>(bsm + c + 4);
-      const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-      const float bi[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    auto emit = [&](int oy, const float (&acc)[kDwCols][kWalkCh]) {
+      const float4 s0 = *reinterpret_cast<const float4*>(ssm + c);
+      const float4 b0 = *reinterpret_cast<const float4*>(bsm + c);
+      const float sc[kWalkCh] = {s0.x, s0.y, s0.z, s0.w};
+      const float bi[kWalkCh] = {b0.x, b0.y, b0.z, b0.w};
 #pragma unroll
       for (int x = 0; x < kDwCols; ++x) {
         const int ox = ox0 + x;
         if (ox >= g.Wo) break;
         const size_t opix = (out_row0 + oy + 1) * g.Wo + ox;
-        float v[8];
+        float v[kWalkCh];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = fmaf(acc[x][i], sc[i], bi[i]);
+        for (int i = 0; i < kWalkCh; ++i) v[i] = fmaf(acc[x][i], sc[i], bi[i]);
         if (job.res) {
-          float rs[8];
-          load8<FMT>(job.res, opix, c, Cs, rs);
+          float rs[kWalkCh];
+          load4<FMT>(job.res, opix, c, Cs, rs);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) v[i] += rs[i];
+          for (int i = 0; i < kWalkCh; ++i) v[i] += rs[i];
         }
         if (clamp) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) v[i] = fminf(fmaxf(v[i], 0.f), act_hi);
+          for (int i = 0; i < kWalkCh; ++i) v[i] = fminf(fmaxf(v[i], 0.f), act_hi);
         }
-        if (c + 8 > g.Cout) {                            // padding channels of the last octet stay zero
+        if (c + kWalkCh > g.Cout) {                      // padding channels stay zero
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
+          for (int i = 0; i < kWalkCh; ++i)
             if (c + i >= g.Cout) v[i] = 0.f;
         }
-        store8<FMT>(job.out, opix, c, Cs, v);
+        store4<FMT>(job.out, opix, c, Cs, v);
       }
     };
 
     if (STRIDE == 1) {
       // k-th input row of the block = unpadded row oy0 - 1 + k, k = 0 .. n_out + 1.  a0 / a1 / a2
       // belong to output rows oy0 + k - 2 / k - 1 / k; a0 is complete after this row.
-      auto step = [&](int k, float (&a0)[kDwCols][8], float (&a1)[kDwCols][8], float (&a2)[kDwCols][8]) {
+      auto step = [&](int k, float (&a0)[kDwCols][kWalkCh], float (&a1)[kDwCols][kWalkCh], float (&a2)[kDwCols][kWalkCh]) {
         const int iy = oy0 - 1 + k;                      // -1 .. H
-        float in[IN_COLS][8];
+        float in[IN_COLS][kWalkCh];
         dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, zero_pix, ix0, g.W, c, Cs, in);
         // rows that belong to a neighbouring block are accumulated too and never stored
         dw_tap_row<STRIDE, true>(wsm, Cs, c, 2, in, a0);
@@ -292,11 +330,11 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
         dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, a2);
         if (k >= 2) emit(oy0 + k - 2, a0);
       };
-      float A[kDwCols][8], B[kDwCols][8], C[kDwCols][8];
+      float A[kDwCols][kWalkCh], B[kDwCols][kWalkCh], C[kDwCols][kWalkCh];
 #pragma unroll
       for (int x = 0; x < kDwCols; ++x)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) A[x][i] = B[x][i] = 0.f;
+        for (int i = 0; i < kWalkCh; ++i) A[x][i] = B[x][i] = 0.f;
       const int n_rows = n_out + 2;
       for (int k = 0; k < n_rows; k += 3) {
         step(k, A, B, C);
@@ -305,12 +343,12 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
       }
     } else {
       // output row j of the block takes unpadded input rows 2 (oy0 + j) - 1, .., + 1
-      float acc[kDwCols][8], carry[kDwCols][8];
-      float in[IN_COLS][8];
+      float acc[kDwCols][kWalkCh], carry[kDwCols][kWalkCh];
+      float in[IN_COLS][kWalkCh];
 #pragma unroll
       for (int x = 0; x < kDwCols; ++x)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) carry[x][i] = 0.f;
+        for (int i = 0; i < kWalkCh; ++i) carry[x][i] = 0.f;
       dw_load_row<FMT, STRIDE>(job.in, (in_row0 + 2 * oy0 - 1) * g.W, zero_pix, ix0, g.W, c, Cs, in);
       dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, carry);
       for (int j = 0; j < n_out; ++j) {
@@ -319,7 +357,7 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
 #pragma unroll
         for (int x = 0; x < kDwCols; ++x)
 #pragma unroll
-          for (int i = 0; i < 8; ++i) acc[x][i] = carry[x][i];
+          for (int i = 0; i < kWalkCh; ++i) acc[x][i] = carry[x][i];
         dw_tap_row<STRIDE, true>(wsm, Cs, c, 1, in, acc);
         dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy + 1) * g.W, zero_pix, ix0, g.W, c, Cs, in);
         dw_tap_row<STRIDE, true>(wsm, Cs, c, 2, in, acc);
@@ -329,14 +367,14 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
     }
     // the two physical padding rows of the image, by the first and the last row block
     if (rbk == 0 || rbk == row_blocks - 1) {
-      const float zero[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      const float zero[kWalkCh] = {0, 0, 0, 0};
 #pragma unroll
       for (int side = 0; side < 2; ++side) {
         if (side == 0 ? rbk != 0 : rbk != row_blocks - 1) continue;
         const size_t jr = out_row0 + (side == 0 ? 0 : g.Ho + 1);
 #pragma unroll
         for (int x = 0; x < kDwCols; ++x)
-          if (ox0 + x < g.Wo) store8<FMT>(job.out, jr * g.Wo + ox0 + x, c, Cs, zero);
+          if (ox0 + x < g.Wo) store4<FMT>(job.out, jr * g.Wo + ox0 + x, c, Cs, zero);
       }
     }
   }
@@ -362,11 +400,11 @@ aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n
   // every SM a block of threads; smaller launches need the parallelism of one row per thread.
   const int n_blk = (g.Ho + 15) / 16;
   const int rb = (g.Ho + n_blk - 1) / n_blk;
-  const long long items_rows = (long long)g.B * n_blk * col_groups * (Cs / 8);
+  const long long items_rows = (long long)g.B * n_blk * col_groups * (Cs / kWalkCh);
   const bool walk_rows = items_rows >= (long long)n_sms * kDwThreads;
   const long long n_items = walk_rows ? items_rows : (long long)g.B * (g.Ho + 2) * col_groups * (Cs / 8);
   long long blocks = (n_items + kDwThreads - 1) / kDwThreads;
-  const long long cap = (long long)n_sms * (walk_rows ? 2 : 4);   // persistent: as many blocks as are resident
+  const long long cap = (long long)n_sms * (walk_rows ? 3 : 4);   // persistent: as many blocks as are resident
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   dim3 grid((unsigned)blocks, n_jobs);
