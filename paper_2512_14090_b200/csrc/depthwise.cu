@@ -172,27 +172,26 @@ depthwise3x3_kernel(ConvGeom g, const LayerJob* __restrict__ jobs) {
 }
 
 
-// Four channels of one pixel (the unit of the row-walking kernel)
+// Four channels of one pixel (the unit of the row-walking kernel).  `p` points at the group's
+// first channel in the pixel (split format: in the hi half; the lo half is lo_off bytes on).
 template <int FMT>
-__device__ __forceinline__ void load4(const void* __restrict__ base, size_t pixel, int c, int Cs, float* v) {
+__device__ __forceinline__ void load4(const uint8_t* __restrict__ p, uint32_t lo_off, float* v) {
   if (FMT == ACT_SPLIT) {
-    const __nv_bfloat16* px = static_cast<const __nv_bfloat16*>(base) + pixel * 2 * Cs;
-    const uint2 h = __ldg(reinterpret_cast<const uint2*>(px + c));
-    const uint2 l = __ldg(reinterpret_cast<const uint2*>(px + Cs + c));
+    const uint2 h = __ldg(reinterpret_cast<const uint2*>(p));
+    const uint2 l = __ldg(reinterpret_cast<const uint2*>(p + lo_off));
     v[0] = __uint_as_float(h.x << 16) + __uint_as_float(l.x << 16);            // a bfloat16 is the upper half of a float
     v[1] = __uint_as_float(h.x & 0xFFFF0000u) + __uint_as_float(l.x & 0xFFFF0000u);
     v[2] = __uint_as_float(h.y << 16) + __uint_as_float(l.y << 16);
     v[3] = __uint_as_float(h.y & 0xFFFF0000u) + __uint_as_float(l.y & 0xFFFF0000u);
   } else {
-    const float4 a = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(base) + pixel * Cs + c));
+    const float4 a = __ldg(reinterpret_cast<const float4*>(p));
     v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
   }
 }
 
 template <int FMT>
-__device__ __forceinline__ void store4(void* __restrict__ base, size_t pixel, int c, int Cs, const float* v) {
+__device__ __forceinline__ void store4(uint8_t* __restrict__ p, uint32_t lo_off, const float* v) {
   if (FMT == ACT_SPLIT) {
-    __nv_bfloat16* px = static_cast<__nv_bfloat16*>(base) + pixel * 2 * Cs;
     uint32_t hw[2], lw[2];
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
@@ -203,10 +202,10 @@ __device__ __forceinline__ void store4(void* __restrict__ base, size_t pixel, in
                                                      v[2 * i + 1] - __uint_as_float(hw[i] & 0xFFFF0000u));
       lw[i] = *reinterpret_cast<const uint32_t*>(&l);
     }
-    *reinterpret_cast<uint2*>(px + c) = make_uint2(hw[0], hw[1]);
-    *reinterpret_cast<uint2*>(px + Cs + c) = make_uint2(lw[0], lw[1]);
+    *reinterpret_cast<uint2*>(p) = make_uint2(hw[0], hw[1]);
+    *reinterpret_cast<uint2*>(p + lo_off) = make_uint2(lw[0], lw[1]);
   } else {
-    *reinterpret_cast<float4*>(static_cast<float*>(base) + pixel * Cs + c) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
   }
 }
 
@@ -219,18 +218,6 @@ __device__ __forceinline__ void store4(void* __restrict__ base, size_t pixel, in
 // The row loop is a real loop (three rotated copies of the body at stride 1), so the code stays
 // small whatever `rb` is.  Input rows -1 and H are the physical padding rows of the image, which
 // every kernel writes as zeros: they are loaded like any other row.
-// Input columns ix0 .. of one row.  A column outside the image reads `zero_pix`, a pixel of the
-// image's first physical padding row (always zeros), so no value has to be patched afterwards.
-template <int FMT, int STRIDE>
-__device__ __forceinline__ void dw_load_row(const void* __restrict__ in, size_t row_pix, size_t zero_pix, int ix0, int W,
-                                            int c, int Cs, float (&v)[(kDwCols - 1) * STRIDE + 3][kWalkCh]) {
-#pragma unroll
-  for (int xx = 0; xx < (kDwCols - 1) * STRIDE + 3; ++xx) {
-    const int ix = ix0 + xx;
-    load4<FMT>(in, (ix >= 0 && ix < W) ? row_pix + ix : zero_pix, c, Cs, v[xx]);
-  }
-}
-
 // acc[x][i] (+)= sum_t in[x * STRIDE + t][i] * w[(r, t)][c + i]
 template <int STRIDE, bool ACCUMULATE>
 __device__ __forceinline__ void dw_tap_row(const float* __restrict__ wsm, int Cs, int c, int r,
@@ -265,6 +252,9 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
   const int octs = Cs / kWalkCh;                         // channel groups
   const int col_groups = (g.Wo + kDwCols - 1) / kDwCols;
   const int row_blocks = (g.Ho + rb - 1) / rb;
+  const size_t pix_bytes = (size_t)4 * Cs;               // a pixel: [hi(Cs) | lo(Cs)] bfloat16 or Cs floats
+  const uint32_t lo_off = 2u * Cs;                       // split format: bytes from the hi to the lo half
+  const uint32_t in_pitch = (uint32_t)(g.W * pix_bytes), out_pitch = (uint32_t)(g.Wo * pix_bytes);
   const bool clamp = g.act != AIQ_ACT_NONE;              // relu: [0, inf), relu6: [0, 6]
   const float act_hi = g.act == AIQ_ACT_RELU6 ? 6.0f : __int_as_float(0x7f800000);
   const long long n_items = (long long)g.B * row_blocks * col_groups * octs;
@@ -277,30 +267,54 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
     const int rbk = (int)(rest % row_blocks);
     const int b = (int)(rest / row_blocks);
     const int c = oct * kWalkCh, ox0 = cg * kDwCols;
+    const uint32_t ch_off = (uint32_t)c * (FMT == ACT_SPLIT ? 2u : 4u);   // bytes from a pixel to its channel c
     const int oy0 = rbk * rb;                            // first (unpadded) output row of the block
     const int n_out = min(rb, g.Ho - oy0);               // output rows of this block
     const size_t out_row0 = (size_t)b * (g.Ho + 2);      // padded output row 0 of the image
     const size_t in_row0 = (size_t)b * (g.H + 2) + 1;    // padded input row of unpadded row 0
-    const size_t zero_pix = (in_row0 - 1) * g.W;         // a pixel of zeros (padding row)
     const int ix0 = ox0 * STRIDE - 1;
 
-    // finish and store output row oy (unpadded) from its accumulators
-    auto emit = [&](int oy, const float (&acc)[kDwCols][kWalkCh]) {
+    // Addresses are kept as running pointers: one per input column, stepped by a row after every
+    // load (a column outside the image points at a pixel of the image's first padding row, which
+    // holds zeros, and does not move), one for the output row and one for the residual row.
+    const uint8_t* colp[IN_COLS];
+    uint32_t colstep[IN_COLS];
+    {
+      const uint8_t* in_base = static_cast<const uint8_t*>(job.in) + ch_off;
+      const size_t first_row = in_row0 + (size_t)(oy0 * STRIDE) - 1;      // padded row of m = 0 (>= in_row0 - 1)
+#pragma unroll
+      for (int xx = 0; xx < IN_COLS; ++xx) {
+        const int ix = ix0 + xx;
+        const bool inside = ix >= 0 && ix < g.W;
+        colp[xx] = in_base + (inside ? first_row * g.W + ix : (in_row0 - 1) * g.W) * pix_bytes;
+        colstep[xx] = inside ? in_pitch : 0u;
+      }
+    }
+    auto load_next_row = [&](float (&in)[IN_COLS][kWalkCh]) {
+#pragma unroll
+      for (int xx = 0; xx < IN_COLS; ++xx) {
+        load4<FMT>(colp[xx], lo_off, in[xx]);
+        colp[xx] += colstep[xx];
+      }
+    };
+    uint8_t* outp = static_cast<uint8_t*>(job.out) + ch_off + ((out_row0 + oy0 + 1) * g.Wo + ox0) * pix_bytes;
+    const uint8_t* resp = job.res ? static_cast<const uint8_t*>(job.res) + (outp - static_cast<uint8_t*>(job.out)) : nullptr;
+
+    // finish and store the next output row (rows are emitted in order) from its accumulators
+    auto emit = [&](const float (&acc)[kDwCols][kWalkCh]) {
       const float4 s0 = *reinterpret_cast<const float4*>(ssm + c);
       const float4 b0 = *reinterpret_cast<const float4*>(bsm + c);
       const float sc[kWalkCh] = {s0.x, s0.y, s0.z, s0.w};
       const float bi[kWalkCh] = {b0.x, b0.y, b0.z, b0.w};
 #pragma unroll
       for (int x = 0; x < kDwCols; ++x) {
-        const int ox = ox0 + x;
-        if (ox >= g.Wo) break;
-        const size_t opix = (out_row0 + oy + 1) * g.Wo + ox;
+        if (ox0 + x >= g.Wo) break;
         float v[kWalkCh];
 #pragma unroll
         for (int i = 0; i < kWalkCh; ++i) v[i] = fmaf(acc[x][i], sc[i], bi[i]);
-        if (job.res) {
+        if (resp) {
           float rs[kWalkCh];
-          load4<FMT>(job.res, opix, c, Cs, rs);
+          load4<FMT>(resp + x * pix_bytes, lo_off, rs);
 #pragma unroll
           for (int i = 0; i < kWalkCh; ++i) v[i] += rs[i];
         }
@@ -313,22 +327,23 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
           for (int i = 0; i < kWalkCh; ++i)
             if (c + i >= g.Cout) v[i] = 0.f;
         }
-        store4<FMT>(job.out, opix, c, Cs, v);
+        store4<FMT>(outp + x * pix_bytes, lo_off, v);
       }
+      outp += out_pitch;
+      if (resp) resp += out_pitch;
     };
 
     if (STRIDE == 1) {
       // k-th input row of the block = unpadded row oy0 - 1 + k, k = 0 .. n_out + 1.  a0 / a1 / a2
       // belong to output rows oy0 + k - 2 / k - 1 / k; a0 is complete after this row.
       auto step = [&](int k, float (&a0)[kDwCols][kWalkCh], float (&a1)[kDwCols][kWalkCh], float (&a2)[kDwCols][kWalkCh]) {
-        const int iy = oy0 - 1 + k;                      // -1 .. H
         float in[IN_COLS][kWalkCh];
-        dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, zero_pix, ix0, g.W, c, Cs, in);
+        load_next_row(in);                               // unpadded row oy0 - 1 + k (-1 .. H)
         // rows that belong to a neighbouring block are accumulated too and never stored
         dw_tap_row<STRIDE, true>(wsm, Cs, c, 2, in, a0);
         dw_tap_row<STRIDE, true>(wsm, Cs, c, 1, in, a1);
         dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, a2);
-        if (k >= 2) emit(oy0 + k - 2, a0);
+        if (k >= 2) emit(a0);
       };
       float A[kDwCols][kWalkCh], B[kDwCols][kWalkCh], C[kDwCols][kWalkCh];
 #pragma unroll
@@ -349,20 +364,19 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
       for (int x = 0; x < kDwCols; ++x)
 #pragma unroll
         for (int i = 0; i < kWalkCh; ++i) carry[x][i] = 0.f;
-      dw_load_row<FMT, STRIDE>(job.in, (in_row0 + 2 * oy0 - 1) * g.W, zero_pix, ix0, g.W, c, Cs, in);
+      load_next_row(in);                                 // unpadded row 2 oy0 - 1
       dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, carry);
       for (int j = 0; j < n_out; ++j) {
-        const int iy = 2 * (oy0 + j);                    // rows iy, iy + 1 <= H
-        dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy) * g.W, zero_pix, ix0, g.W, c, Cs, in);
+        load_next_row(in);                               // rows 2 (oy0 + j) and, below, + 1 (<= H)
 #pragma unroll
         for (int x = 0; x < kDwCols; ++x)
 #pragma unroll
           for (int i = 0; i < kWalkCh; ++i) acc[x][i] = carry[x][i];
         dw_tap_row<STRIDE, true>(wsm, Cs, c, 1, in, acc);
-        dw_load_row<FMT, STRIDE>(job.in, (in_row0 + iy + 1) * g.W, zero_pix, ix0, g.W, c, Cs, in);
+        load_next_row(in);
         dw_tap_row<STRIDE, true>(wsm, Cs, c, 2, in, acc);
         dw_tap_row<STRIDE, false>(wsm, Cs, c, 0, in, carry);
-        emit(oy0 + j, acc);
+        emit(acc);
       }
     }
     // the two physical padding rows of the image, by the first and the last row block
@@ -374,7 +388,8 @@ depthwise3x3_walk_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, int rb) 
         const size_t jr = out_row0 + (side == 0 ? 0 : g.Ho + 1);
 #pragma unroll
         for (int x = 0; x < kDwCols; ++x)
-          if (ox0 + x < g.Wo) store4<FMT>(job.out, jr * g.Wo + ox0 + x, c, Cs, zero);
+          if (ox0 + x < g.Wo)
+            store4<FMT>(static_cast<uint8_t*>(job.out) + ch_off + (jr * g.Wo + ox0 + x) * pix_bytes, lo_off, zero);
       }
     }
   }
