@@ -146,7 +146,7 @@ bool conv_tc_eligible(const ConvGeom& g);
 aiq_status_t conv_tc_encode_map(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
                                 void* map_out);
 // All jobs of one launch have weights of one class: weight_bits = 8 (4- or 8-bit codes), 16 or 32.
-// 16- / 32-bit weights enter as 2 / 3 exact bfloat16 pieces; conv_tc_bits_ok says whether that fits.
+// 16- / 32-bit weights enter as two bfloat16 pieces (hi + lo); conv_tc_bits_ok says whether the kernel takes them.
 bool conv_tc_bits_ok(const ConvGeom& g, int bits);
 aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
                             int batch_capacity, int32_t* error_flag, double weight_bytes, int weight_bits,

@@ -238,7 +238,7 @@ struct TcSmem {
   static __host__ __device__ constexpr int total(int stages, int taps) { return bars(stages, taps) + (2 * stages + 5) * 8 + 16; }
 };
 
-// PIECES: bfloat16 pieces per weight: 1 (4- / 8-bit codes), 2 (half), 3 (float32)
+// PIECES: bfloat16 pieces per weight: 1 (4- / 8-bit codes), 2 (half and float32 weights)
 template <int CS, int N, int KS, int STRIDE, int PIECES>
 __global__ void __launch_bounds__(tc_threads(N), (CS <= 32 && N <= 32) ? 2 : 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const LayerJob* __restrict__ jobs) {
@@ -255,9 +255,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
 
   uint8_t* ring = smem;
   uint8_t* wsm = smem + S::weights(stages);
-  // 16- and 32-bit weights are not exact in one bfloat16: they are held as the sum of 2 / 3
-  // bfloat16 pieces (8 + 8 (+ 8) significant bits: exact), one weight tile per piece and tap,
-  // and every MMA is issued once per piece into the same accumulator.
+  // 16- and 32-bit weights are not exact in one bfloat16: they are held as hi + lo, two bfloat16
+  // pieces (hi = bf16(w), lo = bf16(w - hi): 16 significant bits, exact for a half, within 2^-17
+  // of a float32 weight, the precision the activations are stored with), one weight tile per
+  // piece and tap, and every MMA is issued once per piece into the same accumulator.  A third
+  // piece does not pay: its products are 2^-16 of the sum and the float32 accumulation of the
+  // tensor cores drops most of them (measured: all of them when few weights are non-zero).
   constexpr int pieces = PIECES;
   constexpr int wtaps = taps * pieces;           // weight tiles in shared memory
   // The multi-piece kernels hold at most N = 32 output channels' weights: a layer of 2N output
@@ -330,25 +333,24 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
       const uint8_t* row = ring + (size_t)n * wrow_bytes;
       const uint32_t off = swizzle_off((uint32_t)(n * L::W_ROW_BYTES + c8 * 16), L::W_SWZ_MASK);
       if constexpr (PIECES > 1) {
-        uint32_t pk[3][4];
+        uint32_t pk[PIECES][4];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int k = (c8 * 8 + j) * taps + tap;
           float w = job.bits == 16 ? __half2float(reinterpret_cast<const __half*>(row)[k])
                                    : reinterpret_cast<const float*>(row)[k];
 #pragma unroll
-          for (int pc = 0; pc < 3; ++pc) {
+          for (int pc = 0; pc < PIECES; ++pc) {
             const __nv_bfloat16 h = __float2bfloat16_rn(w);
-            w -= __bfloat162float(h);                            // exact: the remainder of a rounding
+            w -= __bfloat162float(h);                            // exact: the remainder of the rounding
             const uint32_t hb = (uint32_t)__bfloat16_as_ushort(h);
             if (j & 1) pk[pc][j >> 1] |= hb << 16; else pk[pc][j >> 1] = hb;
           }
         }
 #pragma unroll
-        for (int pc = 0; pc < 3; ++pc)
-          if (pc < pieces)
-            *reinterpret_cast<uint4*>(wsm + (size_t)(pc * taps + tap) * L::W_TAP_BYTES + off) =
-                make_uint4(pk[pc][0], pk[pc][1], pk[pc][2], pk[pc][3]);
+        for (int pc = 0; pc < PIECES; ++pc)
+          *reinterpret_cast<uint4*>(wsm + (size_t)(pc * taps + tap) * L::W_TAP_BYTES + off) =
+              make_uint4(pk[pc][0], pk[pc][1], pk[pc][2], pk[pc][3]);
       } else {
         uint32_t packed[4];
 #pragma unroll
@@ -485,7 +487,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap in_map, TcParams p, const Lay
                 const uint32_t accumulate = (t == T_FIRST && r == T_FIRST && part == 0 && kk == 0) ? 0u : 1u;
                 umma_bf16(d_tmem, adesc, ((uint64_t)B_HI << 32) | (uint64_t)b_lo, idesc, accumulate);
 #pragma unroll
-                for (int pc = 1; pc < pieces; ++pc)             // further pieces of 16- / 32-bit weights
+                for (int pc = 1; pc < pieces; ++pc)             // the lo piece of 16- / 32-bit weights
                   umma_bf16(d_tmem, adesc,
                             ((uint64_t)B_HI << 32) | (uint64_t)(b_lo + (uint32_t)((pc * taps * L::W_TAP_BYTES) >> 4)),
                             idesc, 1u);
@@ -934,8 +936,8 @@ aiq_status_t conv_tc_encode_map(const ConvGeom& g, const void* slot_base, int ba
 }
 
 bool conv_tc_bits_ok(const ConvGeom& g, int bits) {
-  // 2 or 3 weight tiles per tap of a 32-channel output slice fit shared memory beside an
-  // activation ring of at least two stages for every eligible shape
+  // two weight tiles per tap of a 32-channel output slice fit shared memory beside the
+  // activation ring for every eligible shape
   (void)g;
   return bits == 4 || bits == 8 || bits == 16 || bits == 32;
 }
@@ -953,9 +955,8 @@ aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* 
 #define AIQ_TC_CASE(CS_, N_)                                                                    \
   if (g.Cin == CS_ && g.Cout == N_ && pieces == 1) AIQ_TC_KS(CS_, N_, 1);
 #define AIQ_TC_CASE_WIDE(CS_, N_)                                                               \
-  if (g.Cin == CS_ && (g.Cout == N_ || g.Cout == 2 * N_) && pieces == 2) AIQ_TC_KS(CS_, N_, 2); \
-  if (g.Cin == CS_ && (g.Cout == N_ || g.Cout == 2 * N_) && pieces == 3) AIQ_TC_KS(CS_, N_, 3);
-  const int pieces = weight_bits <= 8 ? 1 : (weight_bits == 16 ? 2 : 3);
+  if (g.Cin == CS_ && (g.Cout == N_ || g.Cout == 2 * N_) && pieces == 2) AIQ_TC_KS(CS_, N_, 2);
+  const int pieces = weight_bits <= 8 ? 1 : 2;
   AIQ_TC_CASE(16, 16) AIQ_TC_CASE(16, 32) AIQ_TC_CASE(16, 64)
   AIQ_TC_CASE(32, 16) AIQ_TC_CASE(32, 32) AIQ_TC_CASE(32, 64)
   AIQ_TC_CASE(64, 16) AIQ_TC_CASE(64, 32) AIQ_TC_CASE(64, 64)
