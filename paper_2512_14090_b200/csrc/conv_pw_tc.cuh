@@ -18,7 +18,7 @@
 namespace aiq {
 namespace {
 
-constexpr int kPwThreads = 320;
+constexpr int kPwThreads = 448;                      // producer, MMA, 4 epilogue, 4 expander, 4 more epilogue warps
 constexpr int kPwChunk = 64;                         // input channels per stage
 constexpr int kPwATile = 128 * kPwChunk * 2;         // 16 KB: 128 pixels x 64 bfloat16
 
@@ -89,7 +89,7 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_acc_full + 8 * i, 1);
-      mbar_init(bar_acc_empty + 8 * i, 4);       // one arrival per epilogue warp
+      mbar_init(bar_acc_empty + 8 * i, 8);       // one arrival per epilogue warp
     }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -134,7 +134,7 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
           while (!mbar_try_wait(bar_a_full + 8 * i, (issued_phase >> i) & 1u) && clock64() - t0 < kWaitLimitCycles) {}
         }
     }
-  } else if (warp >= 6) {
+  } else if (warp >= 6 && warp < 10) {
     // ---- weight expanders: packed codes -> bfloat16 B tile (Nt rows x 64 channels, 128-byte swizzle)
     // The packed words of a chunk are the same for every pixel tile and come from L2; they are
     // fetched one chunk ahead into registers so that their latency hides behind the expansion of
@@ -229,16 +229,19 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
       }
     }
   } else {
-    // ---- epilogue: warp q owns TMEM lanes 32q .. 32q+31 = pixels 32q .. 32q+31 of the tile -----
+    // ---- epilogue: warps 2 .. 5 and 10 .. 13.  TMEM lanes 32q .. 32q+31 = pixels 32q .. 32q+31 of
+    // the tile belong to the two warps with warp index mod 4 = q; they take alternate groups of
+    // 16 output channels (for layers that widen the channels the epilogue is most of the work).
     const int q = warp & 3;
+    const int h = warp >= 10 ? 1 : 0;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++it) {
       const int buf = it & 1;
       alive = mbar_wait_warp(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort, p.error_flag);   // false => *s_abort is set
       // the previous tile's stores must have finished reading the staging tiles
       if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-      asm volatile("bar.sync 1, 128;" ::: "memory");     // every epilogue thread, unconditionally
-      alive = *s_abort == 0;                             // the same answer in all four warps
+      asm volatile("bar.sync 1, 256;" ::: "memory");     // every epilogue thread, unconditionally
+      alive = *s_abort == 0;                             // the same answer in all eight warps
       if (!alive) break;
       tc_fence_after();
       const int m = q * 32 + lane;                       // pixel row of the tile
@@ -248,7 +251,7 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
       const __nv_bfloat16* res = (job.res && interior)
           ? static_cast<const __nv_bfloat16*>(job.res) + (size_t)pix * (2 * p.Cs_out) : nullptr;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 128);
-      for (int c0 = 0; c0 < Nt; c0 += 16) {
+      for (int c0 = 16 * h; c0 < Nt; c0 += 32) {
         uint32_t v[16];
         tmem_ld16(taddr + c0, v);
         tmem_ld_wait();
@@ -272,11 +275,7 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
             u0 = apply_act(u0, p.act);
             u1 = apply_act(u1, p.act);
           }
-          __nv_bfloat16 h0, l0, h1, l1;
-          split_bf16(u0, h0, l0);
-          split_bf16(u1, h1, l1);
-          hi[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-          lo[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+          split_pair(u0, u1, hi[e >> 1], lo[e >> 1]);
         }
         // staging tile (group, part): 128 rows x 128 bytes, 16-byte units XOR-swizzled by the row
         // exactly as the 128-byte-swizzle tensor map expects
@@ -294,7 +293,7 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
       if (warp == 2 && lane == 0) {
         for (int gi = 0; gi < pw_out_groups(Nt); ++gi) {
           if (n0 + gi * 64 >= p.Cs_out) break;
