@@ -860,7 +860,19 @@ aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const void* o
   PwParams p = {};
   p.P = g.B * (g.H + 2) * g.W; p.H = g.H; p.W = g.W;
   p.Cin = g.Cin; p.Cs_in = g.Cs_in; p.Cout = g.Cout; p.Cs_out = g.Cs_out;
-  p.Nt = g.Cs_out < 128 ? g.Cs_out : 128;
+  // Output-channel tiles of 128 or of 64 channels (the store box is 64 channels wide, so a tile
+  // is a whole number of boxes; only the last tile may be narrower).  A layer's CTAs are split
+  // evenly over its tiles, so its time goes with (tile width) / (CTAs per tile): 144 channels
+  // run as 64 + 64 + 16 rather than 128 + 16, 576 as 9 x 64 rather than 4 x 128 + 64.
+  if (g.Cs_out <= 128) {
+    p.Nt = g.Cs_out;
+  } else {
+    auto cost = [&](int nt) {
+      const int per_tile = n_sms / (n_jobs * ((g.Cs_out + nt - 1) / nt));
+      return (double)nt / (per_tile > 0 ? per_tile : 1);
+    };
+    p.Nt = cost(64) < cost(128) ? 64 : 128;
+  }
   p.n_ntiles = (g.Cs_out + p.Nt - 1) / p.Nt;
   p.act = g.act;
   p.ver_pixels = (long long)batch_capacity * (g.H + 2) * g.W;
