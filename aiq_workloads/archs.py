@@ -155,6 +155,18 @@ def depthwise_stack(hw, channels=96, n_classes=7):
     return dict(name=f"depthwise_stack_{hw}", in_c=3, in_h=hw, in_w=hw, n_classes=n_classes, layers=layers)
 
 
+def pointwise_stack(cin, cout, hw=8, n_classes=6):
+    """A short network around one pointwise (1x1) convolution (test workload): stem 3x3 to `cin`
+    channels, pointwise `cin` -> `cout`, classifier.  Lets a test reach any channel pair of the
+    pointwise layers of MobileNetV2 without the 50 layers around them."""
+    layers = [
+        _conv("stem", 3, cin, 3, 1, "relu6", -1),
+        _conv("pw", cin, cout, 1, 1, "relu6", 0),
+        _fc("fc", cout, n_classes, 1),
+    ]
+    return dict(name=f"pointwise_stack_{cin}_{cout}", in_c=3, in_h=hw, in_w=hw, n_classes=n_classes, layers=layers)
+
+
 def conv_layer_indices(arch):
     """Indices of every layer that is not the classifier (the sweep candidates)."""
     return [i for i, l in enumerate(arch["layers"]) if l["kind"] != "fc"]

@@ -34,10 +34,10 @@ WORKLOAD = "resnet20_cifar_greedy_step: 21 schemes (all-8, one conv layer -> 4 b
 METRIC = "scheme evals/sec (ResNet-20, 10k imgs)"
 UNIT = "scheme-evals/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the
-# committed ncu summary under profiles/ (None until captured / after the kernel changed)
-# conv_tc_kernel: 197.9 MB per launch measured at chunk 256 (profiles/conv_tc__resnet20_greedy_step.md),
-# scaled by 4 to the default chunk of 1024 images (traffic grows with the images of a launch)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from one ncu
+# capture (None until captured / after the kernel changed).
+# conv_tc_kernel: ncu DRAM byte count of 197.9 MB per launch at chunk 256, scaled by 4 to the
+# default chunk of 1024 images (traffic grows with the images of a launch)
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 197.9e6
 
 

@@ -40,8 +40,6 @@ def build(force=False, verbose=False):
     headers.append(os.path.join(ROOT, "include", "aiq.h"))
     if not force and not _stale(LIB_PATH, sources() + headers):
         return LIB_PATH
-    if not force and not _stale(LIB_PATH, sources() + headers):
-        return LIB_PATH
     nvcc = _nvcc()
     objs, todo = [], []
     for src in sources():

@@ -4,6 +4,7 @@
 #include "common.cuh"
 
 #include <algorithm>
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -810,8 +811,11 @@ extern "C" aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t
 static __device__ __align__(256) unsigned char g_static_workspace[AIQ_STATIC_WORKSPACE_BYTES];
 
 namespace aiq {
-static void* g_static_ws_ptr[64];        // per device; nullptr until the first call on it
-static bool g_static_ws_ready[64];
+// Device address of the array per device; nullptr until the first call on that device.  Two
+// host threads that make their first call at the same time both look the address up and
+// publish the same value, which is harmless; the atomic only makes sure that a reader never
+// sees a half-published pointer.
+static std::atomic<void*> g_static_ws_ptr[64];
 }  // namespace aiq
 
 extern "C" aiq_status_t aiq_forward_static(const aiq_model_t* model, const uint8_t* scheme_bits,
@@ -831,18 +835,17 @@ extern "C" aiq_status_t aiq_forward_static(const aiq_model_t* model, const uint8
   int dev = 0;
   AIQ_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return set_error(AIQ_ERR_INVALID_ARG, "aiq_forward_static: device %d", dev);
-  if (!g_static_ws_ready[dev]) {
+  void* ws_ptr = g_static_ws_ptr[dev].load(std::memory_order_acquire);
+  if (!ws_ptr) {
     // first call on this device (it is the current one): resolve the array's device address
-    void* ptr = nullptr;
-    cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_workspace);
-    if (e != cudaSuccess || !ptr)
+    cudaError_t e = cudaGetSymbolAddress(&ws_ptr, g_static_workspace);
+    if (e != cudaSuccess || !ws_ptr)
       return set_error(AIQ_ERR_CUDA, "cudaGetSymbolAddress(static workspace): %s", cudaGetErrorString(e));
-    g_static_ws_ptr[dev] = ptr;
-    g_static_ws_ready[dev] = true;
+    g_static_ws_ptr[dev].store(ws_ptr, std::memory_order_release);
   }
   // Nothing in the workspace has to start at zero for a forward pass: the job records are
   // copied in, and every activation, pooled value and logit is written before it is read.
-  return aiq_forward(model, scheme_bits, x, batch, logits, g_static_ws_ptr[dev],
+  return aiq_forward(model, scheme_bits, x, batch, logits, ws_ptr,
                      (size_t)AIQ_STATIC_WORKSPACE_BYTES, stream_);
 }
 

@@ -32,6 +32,16 @@ def test_every_declared_symbol_is_exported(aiq):
     assert sorted(aiq.EXPORTS) == declared
 
 
+def test_binding_constants_equal_the_header(aiq):
+    text = open(os.path.join(ROOT, "include", "aiq.h")).read()
+    m = re.search(r"#define\s+AIQ_STATIC_WORKSPACE_BYTES\s+\((\d+)u \* (\d+)u \* (\d+)u\)", text)
+    assert m and int(m.group(1)) * int(m.group(2)) * int(m.group(3)) == aiq.STATIC_WORKSPACE_BYTES
+    for name in ("OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED_BITS", "ERR_SHAPE", "ERR_WORKSPACE_TOO_SMALL",
+                 "ERR_CUDA", "ERR_NOT_SM100", "ERR_NONFINITE", "ERR_TIMEOUT"):
+        m = re.search(r"\bAIQ_%s = (\d+)" % name, text)
+        assert m and int(m.group(1)) == getattr(aiq, name), name
+
+
 def test_status_strings(aiq):
     seen = {aiq.status_string(i) for i in range(9)}
     assert len(seen) == 9 and "ok" in seen

@@ -265,3 +265,91 @@ def test_structural_variant_tables():
     assert len(p["layers"]) == 21 and p["layers"][-1]["kind"] == "fc"
     assert all(l["cout"] == 64 and l["residual"] == -1 for l in p["layers"][:-1])
     assert O.layer_shapes(p)[-2][3:] == (8, 8)
+
+
+# ---------------------------------------------------------------- standalone linear layer
+def _rows(text):
+    return np.asarray([[float(v) for v in row.split()] for row in text.split("/")])
+
+
+def test_qlinear_hand_table():
+    """y[m][n] = s_n * sum_k code[n][k] * x[m][k] + bias[n] on values worked out by hand: the
+    weight matrix is [N][K] with one scale per row, the bias is added once per output."""
+    g = _golden("qlinear_hand.txt")
+    codes = _rows(g["codes_2x3"][0]).astype(np.int8)
+    scales = _rows(g["scales_2"][0])[0].astype(np.float32)
+    bias = _rows(g["bias_2"][0])[0].astype(np.float32)
+    x = _rows(g["x_2x3"][0]).astype(np.float32)
+    y = O.qlinear(codes, scales, bias, 8, x)
+    assert y.dtype == np.float32 and y.tolist() == _rows(g["y_2x2"][0]).tolist()
+    # without a bias the outputs drop by exactly the bias
+    assert (O.qlinear(codes, scales, None, 8, x) + bias[None, :]).tolist() == y.tolist()
+    # 4-bit codes follow the same rule
+    assert O.qlinear(codes, scales, bias, 4, x).tolist() == y.tolist()
+    # square case: a transposed W or a scale per column would keep the shape but not the values
+    ysq = O.qlinear(_rows(g["codes_sq"][0]).astype(np.int8), _rows(g["scales_sq"][0])[0].astype(np.float32),
+                    None, 8, _rows(g["x_sq"][0]).astype(np.float32))
+    assert ysq.tolist() == _rows(g["y_sq"][0]).tolist()
+
+
+def test_qlinear_integer_inputs_are_exact_and_match_an_integer_matmul():
+    """With integer activations every product and partial sum is an integer below 2^53, so the
+    result must equal the int64 matrix product times the scale (a power of two here), exactly."""
+    rng = np.random.default_rng(7)
+    for bits, lim in ((4, 7), (8, 127)):
+        codes = rng.integers(-lim, lim + 1, (9, 40)).astype(np.int8)
+        x = rng.integers(-50, 51, (5, 40)).astype(np.float32)
+        scales = (2.0 ** rng.integers(-6, 3, 9)).astype(np.float32)
+        want = (x.astype(np.int64) @ codes.astype(np.int64).T).astype(np.float64) * scales[None, :].astype(np.float64)
+        got = O.qlinear(codes, scales, None, bits, x)
+        assert np.array_equal(got.astype(np.float64), want)
+    # 16 / 32 bits: the stored element itself, no scale
+    w = rng.integers(-8, 9, (6, 12)).astype(np.float32)
+    x = rng.integers(-8, 9, (3, 12)).astype(np.float32)
+    ones = np.ones(6, np.float32)
+    want = (x.astype(np.int64) @ w.astype(np.int64).T).astype(np.float64)
+    assert np.array_equal(O.qlinear(w.astype(np.float16), ones, None, 16, x).astype(np.float64), want)
+    assert np.array_equal(O.qlinear(w, ones, None, 32, x).astype(np.float64), want)
+
+
+def test_qlinear_is_the_classifier_of_a_one_layer_network():
+    """A network that is a single linear classifier on 1x1 images is the same computation
+    (the average pool of a 1x1 map is the identity): qlinear must equal forward() bit for bit."""
+    rng = np.random.default_rng(11)
+    N, K, M = 7, 20, 5
+    W = (rng.standard_normal((N, K)) * 0.3).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    arch = dict(name="lin", in_c=K, in_h=1, in_w=1, n_classes=N, layers=[
+        dict(name="fc", kind="fc", cin=K, cout=N, k=1, stride=1, pad=0, act="none", input=-1,
+             residual=-1, has_bn=False)])
+    for bits in (4, 8, 16, 32):
+        v, s = O.quantize_rows(W, bits)
+        y = O.qlinear(v, s, bias, bits, x)
+        ref = O.forward(arch, [(O.dequantize_rows(v, s, bits), bias)], x.reshape(M, K, 1, 1))
+        assert np.array_equal(y.view(np.uint32), ref.view(np.uint32))
+
+
+def test_eval_schemes_hand_table():
+    """Predictions, counts, accuracies and margins of three schemes on logits known by hand
+    (ties go to the lowest index; a count is the number of predictions equal to the label)."""
+    g = _golden("eval_schemes_hand.txt")
+    x = _rows(g["images"][0]).astype(np.float32).reshape(6, 3, 1, 1)
+    labels = _rows(g["labels"][0])[0].astype(np.int32)
+    arch = dict(name="lin", in_c=3, in_h=1, in_w=1, n_classes=3, layers=[
+        dict(name="fc", kind="fc", cin=3, cout=3, k=1, stride=1, pad=0, act="none", input=-1,
+             residual=-1, has_bn=False)])
+    zero = np.zeros(3, np.float32)
+    bank = [{32: (np.eye(3, dtype=np.float32), zero),
+             8: (np.asarray([[0, 1, 0], [0, 0, 1], [1, 0, 0]], np.float32), zero),
+             4: (np.asarray([[1, 0, 0], [1, 0, 0], [0, 0, 1]], np.float32), zero)}]
+    schemes = np.asarray([[32], [8], [4]], np.uint8)
+    acc, counts, preds, margins = O.eval_schemes(arch, bank, schemes, x, labels, chunk=4)
+    for row, bits in enumerate((32, 8, 4)):
+        assert preds[row].tolist() == [int(v) for v in g[f"pred_{bits}"][0].split()], bits
+        assert int(counts[row]) == int(g[f"count_{bits}"][0]), bits
+        assert acc[row] == int(g[f"count_{bits}"][0]) / 6.0
+        np.testing.assert_allclose(margins[row], [float(v) for v in g[f"margin_{bits}"][0].split()], atol=1e-6)
+    # the image whose margin is 0.01 (up to float32 rounding of 4.01) sits on the edge of the
+    # arg-max rule of the parity tests: it is the only one between 0.009 and 0.011
+    assert ((margins[0] > 0.009) & (margins[0] < 0.011)).sum() == 1

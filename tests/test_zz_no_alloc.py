@@ -6,7 +6,9 @@ budget was fixed and spent at start-up, or as a plug-in that only ever receives 
 output buffers.  aiq_forward_static serves them from a fixed workspace built into the
 library.  This test calls it through the C ABI twice in a row (the second call finds the
 first call's leftovers in the shared workspace) and checks each result against aiq_forward
-with an ordinary caller-provided workspace, at the tolerance the other forward tests use.
+with an ordinary caller-provided workspace and against the CPU oracle, at the tolerance the
+other forward tests use, and checks that a call leaves the amount of free device memory
+unchanged (it must not allocate).
 It lives in a file that sorts last so that a run stopping at the first failure has already
 executed every other test.
 """
@@ -14,38 +16,47 @@ import numpy as np
 import pytest
 
 from aiq_workloads import resnet20, tiny_net, gen_model, gen_images, gen_random_scheme
+from oracle import aiq_oracle as O
 from gpu_util import binding, to_dev, assert_logits_close
 
 pytestmark = pytest.mark.gpu
 
 
-def _compare_two_calls(aiq, model, cases):
+def _compare_two_calls(aiq, model, cases, arch, params):
     import torch
-    for scheme, x in cases:
+    bank = O.build_weight_bank(O.fold_model(arch, params))
+    for call, (scheme, x) in enumerate(cases):
         xd = to_dev(x)
         want = model.aiq_forward(scheme, xd).cpu().numpy()
         got = torch.full((x.shape[0], model.n_classes), float("nan"), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         model.aiq_forward_static(scheme, xd, got)
         torch.cuda.synchronize()
+        if call > 0:      # the first call may still load kernels of the library; later ones must not allocate
+            assert torch.cuda.mem_get_info()[0] == free_before, "aiq_forward_static changed the free device memory"
         assert_logits_close(got.cpu().numpy(), want, "aiq_forward_static vs aiq_forward")
+        assert_logits_close(got.cpu().numpy(), O.forward_scheme(arch, bank, scheme, x), "aiq_forward_static vs oracle")
 
 
 def test_static_workspace_matches_forward_on_two_calls_in_a_row():
     aiq = binding()
     arch = resnet20()
-    model = aiq.Model(arch, gen_model(arch, 1234))
+    params = gen_model(arch, 1234)
+    model = aiq.Model(arch, params)
     assert model.aiq_workspace_bytes(24, 1) <= aiq.STATIC_WORKSPACE_BYTES
     # the limit the header documents for this network
     assert model.aiq_workspace_bytes(40, 1) <= aiq.STATIC_WORKSPACE_BYTES < model.aiq_workspace_bytes(41, 1)
     cases = [(gen_random_scheme(model.n_layers, 42), gen_images(24, 3, 32, 32, 5678)),
              (gen_random_scheme(model.n_layers, 43), gen_images(7, 3, 32, 32, 5680))]
-    _compare_two_calls(aiq, model, cases)
+    _compare_two_calls(aiq, model, cases, arch, params)
     model.close()
     # another model through the same shared workspace, again twice
     arch = tiny_net()
-    model = aiq.Model(arch, gen_model(arch, 99))
+    params = gen_model(arch, 99)
+    model = aiq.Model(arch, params)
     cases = [(gen_random_scheme(model.n_layers, s), gen_images(11 + s, 3, 8, 8, 100 + s)) for s in (1, 2)]
-    _compare_two_calls(aiq, model, cases)
+    _compare_two_calls(aiq, model, cases, arch, params)
     model.close()
 
 
