@@ -117,6 +117,11 @@ aiq_status_t aiq_quantize_layer(const float* W, int N, int K, int bits, void* pa
  * bit).  Both need scratch memory: pass `workspace` (device, 16-byte aligned) of at least
  * aiq_qlinear_workspace_bytes(...) bytes; with workspace == NULL, or where that function
  * returns 0, the plain kernel runs.
+ * Device-side failure: the tcgen05 kernel bounds every wait on its copy / MMA pipeline (about
+ * 2 s of SM clocks).  Should one expire, the kernel stops early and y is invalid; the call has
+ * long returned AIQ_OK by then, so the record is on the device: the int32 at byte offset
+ * aiq_qlinear_workspace_bytes(...) - 16 of `workspace` is set to 0 by every call that uses the
+ * tcgen05 kernel and to 1 by a kernel whose wait expired.  Read it after synchronising.
  */
 size_t aiq_qlinear_workspace_bytes(int N, int K, int bits, int M);
 aiq_status_t aiq_qlinear(const void* packed, const float* scales, const float* bias, int N,
@@ -189,6 +194,14 @@ int aiq_model_num_classes(const aiq_model_t* model);  /* cout of the last layer 
  * asynchronous call on this model (AIQ_ERR_TIMEOUT: a bounded wait inside a kernel expired;
  * the outputs of that call are then invalid).  AIQ_OK otherwise.  Clears the record. */
 aiq_status_t aiq_model_status(const aiq_model_t* model, void* stream);
+
+/* Test aid for the failure path above (no counterpart in the paper).  Launches a one-thread
+ * kernel that waits, with the same bounded-wait routine as the tensor-core kernels, on a
+ * barrier nothing arrives at.  After `limit_cycles` SM clocks (0 < limit_cycles <= 2e9) the
+ * wait gives up, records the failure in the model's device status word and the kernel returns
+ * normally; the next aiq_model_status / aiq_eval_schemes on this model then reports
+ * AIQ_ERR_TIMEOUT and clears the record.  Asynchronous on `stream`. */
+aiq_status_t aiq_debug_expire_wait(const aiq_model_t* model, int64_t limit_cycles, void* stream);
 
 /* Device views into the model memory, for inspection: folded weights Wf [cout][K] and bias
  * [cout] of `layer`; packed rows and scales of (`layer`, `bits`) in the layout of

@@ -26,7 +26,7 @@ EXPORTS = [
     "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
     "aiq_eval_schemes", "aiq_set_eval_options", "aiq_last_call_stats", "aiq_scheme_ai",
     "aiq_profile_start", "aiq_profile_stop", "aiq_forward_static",
-    "aiq_set_compute_path", "aiq_model_status", "aiq_search_greedy", "aiq_search_coordinate_descent",
+    "aiq_set_compute_path", "aiq_model_status", "aiq_debug_expire_wait", "aiq_search_greedy", "aiq_search_coordinate_descent",
 ]
 
 PATH_AUTO, PATH_FP32, PATH_TENSOR = 0, 1, 2
@@ -125,6 +125,8 @@ def _load():
     lib.aiq_forward_static.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.aiq_model_status.restype = i32
     lib.aiq_model_status.argtypes = [vp, vp]
+    lib.aiq_debug_expire_wait.restype = i32
+    lib.aiq_debug_expire_wait.argtypes = [vp, C.c_int64, vp]
     lib.aiq_set_compute_path.restype = None
     lib.aiq_set_compute_path.argtypes = [i32]
     lib.aiq_profile_start.restype = i32
@@ -384,6 +386,9 @@ class Model:
 
     def aiq_model_status(self, stream=None):
         _check(lib.aiq_model_status(self.handle, _stream(stream)))
+
+    def aiq_debug_expire_wait(self, limit_cycles, stream=None):
+        _check(lib.aiq_debug_expire_wait(self.handle, int(limit_cycles), _stream(stream)))
 
     def aiq_scheme_ai(self, scheme_bits, ai_batch=1):
         scheme = np.ascontiguousarray(scheme_bits, dtype=np.uint8)

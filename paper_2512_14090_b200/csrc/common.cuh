@@ -7,6 +7,8 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <atomic>
+
 #include "../../include/aiq.h"
 
 namespace aiq {
@@ -29,6 +31,25 @@ void count_launch();                         // per-thread launch counter (aiq_l
     if (e__ != cudaSuccess)                                                             \
       return ::aiq::set_error(AIQ_ERR_CUDA, "launch %s: %s", what, cudaGetErrorString(e__)); \
     ::aiq::count_launch();                                                              \
+  } while (0)
+
+// Properties of the current device (looked up once per device, then cached).
+struct DeviceProps { int dev, n_sms, smem_optin; };
+aiq_status_t current_device_props(DeviceProps* out);
+
+// Opt-in of `kernel` to `bytes` of dynamic shared memory.  The attribute belongs to the
+// (kernel, device) pair, so the record of what has been set is kept per device; it is only
+// written after the runtime call succeeded.  `kernel` must name one kernel per call site.
+#define AIQ_ENSURE_DYNAMIC_SMEM(kernel, bytes)                                                   \
+  do {                                                                                           \
+    static std::atomic<int> set_bytes__[64];                                                     \
+    int dev__ = 0;                                                                               \
+    AIQ_CUDA_TRY(cudaGetDevice(&dev__));                                                         \
+    const bool cached__ = dev__ >= 0 && dev__ < 64;                                              \
+    if (!cached__ || set_bytes__[dev__].load(std::memory_order_acquire) < (int)(bytes)) {        \
+      AIQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(bytes))); \
+      if (cached__) set_bytes__[dev__].store((int)(bytes), std::memory_order_release);           \
+    }                                                                                            \
   } while (0)
 
 // Brackets one kernel launch with CUDA events while profiling is on (see aiq_profile_start),
@@ -161,6 +182,9 @@ aiq_status_t conv_pw_tc_encode_out_map(const ConvGeom& g, const void* slot_base,
                                        void* map_out);
 aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const void* out_map, const LayerJob* jobs_dev, int n_jobs,
                                int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s);
+// Test aid: a one-thread kernel whose bounded wait runs out after `limit_cycles` SM clocks; it sets
+// *error_flag to 1 and *observed (optional) to 2, then returns.
+aiq_status_t launch_expire_wait(int32_t* error_flag, long long limit_cycles, int32_t* observed, cudaStream_t s);
 // pooled[b][c] = mean over the H x W interior of a split tensor, per job (in -> out float32 [B][C])
 aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int H, int W, int C, int act_format,
                             cudaStream_t s);

@@ -77,22 +77,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false (and raises the abort flag) when the limit is hit or another
-// role has already aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* error_flag) {
+// Bounded wait.  Returns false (and raises the abort flag) when `limit_cycles` SM clocks have
+// passed, or another role has already aborted.
+__device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                              int32_t* error_flag, long long limit_cycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) break;
+      if (clock64() - t0 > limit_cycles) break;
     }
   }
   *abort_flag = 1;
   if (error_flag) atomicExch(error_flag, 1);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* error_flag) {
+  return mbar_wait_for(bar, parity, abort_flag, error_flag, kWaitLimitCycles);
 }
 // bounded wait by a whole (converged) warp: the same answer in every lane.  (Polling from
 // one elected lane and broadcasting the result was measured 40 % slower on the convolution.)
@@ -733,13 +737,9 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
   using L = TcLayout<CS, N>;
   using S = TcSmem<CS, N>;
   const int taps = g.ks * g.ks * PIECES;         // weight tiles held in shared memory
-  static int smem_limit = 0, n_sms = 0;
-  if (!smem_limit) {
-    int dev = 0;
-    AIQ_CUDA_TRY(cudaGetDevice(&dev));
-    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
-  }
+  DeviceProps props;
+  if (aiq_status_t st = current_device_props(&props)) return st;
+  const int smem_limit = props.smem_optin, n_sms = props.n_sms;
   // Shared memory decides how many CTAs share an SM.  More resident CTAs hide the latency of
   // a tile's load -> MMA -> epilogue chain better than a deeper ring does, so prefer two
   // CTAs with at least 4 stages, then one with as many stages as fit (at most 6).
@@ -757,11 +757,7 @@ aiq_status_t launch_tc(const ConvGeom& g, const CUtensorMap& map, const LayerJob
   const int packed = N * (int)row_bytes(g.K, weight_bits <= 8 ? 8 : weight_bits);
   if (packed > stages * L::STAGE_BYTES)
     return set_error(AIQ_ERR_SHAPE, "conv_tc: packed weights (%d bytes) exceed the staging ring", packed);
-  static bool attr_set = false;
-  if (!attr_set) {
-    AIQ_CUDA_TRY(cudaFuncSetAttribute(conv_tc_kernel<CS, N, KS, STRIDE, PIECES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
-    attr_set = true;
-  }
+  AIQ_ENSURE_DYNAMIC_SMEM((conv_tc_kernel<CS, N, KS, STRIDE, PIECES>), smem_limit);
   TcParams p = {};
   p.B = g.B; p.H = g.H; p.W = g.W; p.Ho = g.Ho; p.Wo = g.Wo; p.ks = g.ks; p.stride = g.stride; p.act = g.act;
   p.n_stages = stages; p.K = g.K; p.error_flag = error_flag;
@@ -849,14 +845,10 @@ aiq_status_t conv_pw_tc_encode_out_map(const ConvGeom& g, const void* slot_base,
 
 aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const void* out_map, const LayerJob* jobs_dev, int n_jobs,
                                int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s) {
-  static int smem_limit = 0, n_sms = 0;
-  if (!smem_limit) {
-    int dev = 0;
-    AIQ_CUDA_TRY(cudaGetDevice(&dev));
-    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
-    AIQ_CUDA_TRY(cudaFuncSetAttribute(conv_pw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
-  }
+  DeviceProps props;
+  if (aiq_status_t st = current_device_props(&props)) return st;
+  const int smem_limit = props.smem_optin, n_sms = props.n_sms;
+  AIQ_ENSURE_DYNAMIC_SMEM(conv_pw_tc_kernel, smem_limit);
   PwParams p = {};
   p.P = g.B * (g.H + 2) * g.W; p.H = g.H; p.W = g.W;
   p.Cin = g.Cin; p.Cs_in = g.Cs_in; p.Cout = g.Cout; p.Cs_out = g.Cs_out;
@@ -980,6 +972,30 @@ aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* 
 #undef AIQ_TC_CASE
 #undef AIQ_TC_ARGS
   return set_error(AIQ_ERR_SHAPE, "conv_tc: no kernel for Cin=%d Cout=%d", g.Cin, g.Cout);
+}
+
+// ---- the expiry path of the bounded waits, exercised on purpose ------------------------------
+// One thread waits, with the same helper the kernels above use, on a barrier that nothing ever
+// arrives at.  The wait gives up after `limit_cycles`, raises the error word and the kernel
+// returns normally: nothing traps, faults or hangs.
+namespace {
+__global__ void expire_wait_kernel(int32_t* error_flag, long long limit_cycles, int32_t* observed) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait_for(smem_u32(&bar), 0, &abort_flag, error_flag, limit_cycles);
+    if (observed) *observed = ok ? 0 : 1 + abort_flag;      // 2: gave up and raised the abort flag
+  }
+}
+}  // namespace
+
+aiq_status_t launch_expire_wait(int32_t* error_flag, long long limit_cycles, int32_t* observed, cudaStream_t s) {
+  expire_wait_kernel<<<1, 32, 0, s>>>(error_flag, limit_cycles, observed);
+  AIQ_LAUNCH_CHECK("expire_wait");
+  return AIQ_OK;
 }
 
 }  // namespace aiq

@@ -402,12 +402,9 @@ aiq_status_t launch_depthwise(const ConvGeom& g, const LayerJob* jobs_dev, int n
   if (g.stride != 1 && g.stride != 2) return set_error(AIQ_ERR_SHAPE, "depthwise: stride %d is not supported", g.stride);
   const int Cs = g.Cs_out;
   const size_t smem = (size_t)11 * Cs * sizeof(float);
-  static int n_sms = 0;
-  if (!n_sms) {
-    int dev = 0;
-    AIQ_CUDA_TRY(cudaGetDevice(&dev));
-    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
-  }
+  DeviceProps props;
+  if (aiq_status_t st = current_device_props(&props)) return st;
+  const int n_sms = props.n_sms;
   if (smem > 48 * 1024) return set_error(AIQ_ERR_SHAPE, "depthwise: %d channels need %zu bytes of shared memory", g.Cout, smem);
   const int col_groups = (g.Wo + kDwCols - 1) / kDwCols;
   // Rows per thread of the row-walking kernel: the image height cut into the fewest blocks of at

@@ -20,9 +20,11 @@ namespace aiq {
 // ---------------------------------------------------------------------------------------
 static thread_local char t_err[512] = "";
 static thread_local int64_t t_launches = 0, t_layer_evals = 0, t_layer_evals_unshared = 0;
-static int g_opt_chunk = 0;
-static int g_opt_share = 1;
-static int g_opt_path = AIQ_PATH_AUTO;
+// process-wide knobs (aiq_set_eval_options / aiq_set_compute_path): atomics, so a thread that
+// changes them while another evaluates gives that call either the old or the new value
+static std::atomic<int> g_opt_chunk{0};
+static std::atomic<int> g_opt_share{1};
+static std::atomic<int> g_opt_path{AIQ_PATH_AUTO};
 
 aiq_status_t set_error(aiq_status_t status, const char* fmt, ...) {
   va_list ap;
@@ -82,6 +84,20 @@ aiq_status_t check_device_sm100() {
   if (e != cudaSuccess) return set_error(AIQ_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
   if (dev >= 0 && dev < 64) cached[dev] = (major == 10) ? 1 : 2;
   if (major != 10) return set_error(AIQ_ERR_NOT_SM100, "device %d is compute capability %d.x, need 10.x", dev, major);
+  return AIQ_OK;
+}
+
+aiq_status_t current_device_props(DeviceProps* out) {
+  static std::atomic<int> ready[64];
+  static DeviceProps cache[64];
+  int dev = 0;
+  AIQ_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < 64 && ready[dev].load(std::memory_order_acquire)) { *out = cache[dev]; return AIQ_OK; }
+  DeviceProps p = {dev, 0, 0};
+  AIQ_CUDA_TRY(cudaDeviceGetAttribute(&p.n_sms, cudaDevAttrMultiProcessorCount, dev));
+  AIQ_CUDA_TRY(cudaDeviceGetAttribute(&p.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+  if (dev >= 0 && dev < 64) { cache[dev] = p; ready[dev].store(1, std::memory_order_release); }
+  *out = p;
   return AIQ_OK;
 }
 
@@ -306,7 +322,8 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
   m->act_format = ACT_SPLIT;                      // tentatively, to ask which layers would qualify
   bool any_tc = false;
   for (const LayerInfo& li : m->layers) any_tc = any_tc || layer_on_tensor_cores(m, li);
-  m->act_format = (g_opt_path == AIQ_PATH_TENSOR || (g_opt_path == AIQ_PATH_AUTO && any_tc)) ? ACT_SPLIT : ACT_F32;
+  const int opt_path = g_opt_path.load();
+  m->act_format = (opt_path == AIQ_PATH_TENSOR || (opt_path == AIQ_PATH_AUTO && any_tc)) ? ACT_SPLIT : ACT_F32;
   assign_slots(m);
   cudaStream_t stream = (cudaStream_t)stream_;
   uint8_t* base = static_cast<uint8_t*>(dev_mem);
@@ -380,6 +397,16 @@ extern "C" aiq_status_t aiq_model_status(const aiq_model_t* model, void* stream_
     return set_error(AIQ_ERR_TIMEOUT, "a bounded wait inside a kernel expired; outputs of that call are invalid");
   }
   return AIQ_OK;
+}
+
+extern "C" aiq_status_t aiq_debug_expire_wait(const aiq_model_t* model, int64_t limit_cycles, void* stream_) {
+  using namespace aiq;
+  if (!model) return set_error(AIQ_ERR_INVALID_ARG, "aiq_debug_expire_wait: null model");
+  if (limit_cycles <= 0 || limit_cycles > 2000000000ll)
+    return set_error(AIQ_ERR_INVALID_ARG, "aiq_debug_expire_wait: limit_cycles=%lld outside (0, 2e9]", (long long)limit_cycles);
+  aiq_status_t st = check_device_sm100();
+  if (st != AIQ_OK) return st;
+  return launch_expire_wait(model->status_word, limit_cycles, nullptr, (cudaStream_t)stream_);
 }
 
 extern "C" int aiq_model_num_layers(const aiq_model_t* model) { return model ? (int)model->layers.size() : -1; }
@@ -741,7 +768,8 @@ extern "C" aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t
   t_launches = 0;
 
   // chunk: the requested (or default) size, shrunk until the layout fits the workspace
-  int B = g_opt_chunk > 0 ? g_opt_chunk : 1024;
+  const int opt_chunk = g_opt_chunk.load();
+  int B = opt_chunk > 0 ? opt_chunk : 1024;
   if (B > n_images) B = n_images;
   while (B > 1 && ws_layout(model, B, n_schemes).total > workspace_bytes) B = (B + 1) / 2;
   const WsLayout wl = ws_layout(model, B, n_schemes);
@@ -750,7 +778,7 @@ extern "C" aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t
                      wl.total, workspace_bytes);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   EvalPlan plan;
-  st = build_plan(model, schemes, n_schemes, B, g_opt_share != 0, ws, wl, nullptr, plan);
+  st = build_plan(model, schemes, n_schemes, B, g_opt_share.load() != 0, ws, wl, nullptr, plan);
   if (st != AIQ_OK) return st;
   // Counts and predictions are indexed by a row in [0, n_schemes): the row of a final
   // version is the first scheme that maps to it; duplicate schemes are filled in afterwards.

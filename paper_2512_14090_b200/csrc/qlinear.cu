@@ -182,7 +182,7 @@ aiq_status_t launch_qlinear(const LayerJob* jobs_dev, const LayerJob* single_hos
 
 extern "C" size_t aiq_qlinear_workspace_bytes(int N, int K, int bits, int M) {
   if (N <= 0 || K <= 0 || M <= 0) return 0;
-  if (aiq::qlinear_tc_applicable(N, K, bits, M)) return aiq::qlinear_tc_workspace_bytes(K, M);
+  if (aiq::qlinear_tc_applicable(N, K, bits, M)) return aiq::qlinear_tc_workspace_bytes(K, M) + 16;   // + status word
   if (aiq::qlinear_mma_applicable(N, K, bits, M)) return aiq::qlinear_mma_workspace_bytes(K, M);
   return 0;
 }
@@ -209,8 +209,13 @@ extern "C" aiq_status_t aiq_qlinear(const void* packed, const float* scales, con
   if (workspace && aiq::qlinear_tc_applicable(N, K, bits, M)) {
     if (((uintptr_t)workspace) & 15)
       return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_qlinear: workspace not 16-byte aligned");
-    if (workspace_bytes >= aiq::qlinear_tc_workspace_bytes(K, M))
-      return aiq::launch_qlinear_tc(job, N, K, M, workspace, nullptr, (cudaStream_t)stream);
+    const size_t scratch = aiq::qlinear_tc_workspace_bytes(K, M);
+    if (workspace_bytes >= scratch + 16) {
+      // device status word behind the scratch: 0, or 1 once a bounded wait of the kernel expired
+      int32_t* status = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + scratch);
+      AIQ_CUDA_TRY(cudaMemsetAsync(status, 0, 16, (cudaStream_t)stream));
+      return aiq::launch_qlinear_tc(job, N, K, M, workspace, status, (cudaStream_t)stream);
+    }
   } else if (workspace && aiq::qlinear_mma_applicable(N, K, bits, M)) {
     if (((uintptr_t)workspace) & 15)
       return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_qlinear: workspace not 16-byte aligned");

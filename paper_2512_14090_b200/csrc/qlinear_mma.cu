@@ -358,12 +358,7 @@ aiq_status_t launch_qlinear_mma(const LayerJob& job, int N, int K, int M, void* 
 #define AIQ_QMMA(BITS_, NT_, GR_)                                                                           \
   do {                                                                                                      \
     const int smem = GR_ * kGroupFrags * NT_ * 32 * (int)sizeof(uint2) + kMmaWarps * kStages * kStageBytes; \
-    static bool attr_done = false;                                                                          \
-    if (!attr_done) {                                                                                       \
-      AIQ_CUDA_TRY(cudaFuncSetAttribute(qlinear_mma_kernel<BITS_, NT_, GR_>,                                \
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, smem));                \
-      attr_done = true;                                                                                     \
-    }                                                                                                       \
+    AIQ_ENSURE_DYNAMIC_SMEM((qlinear_mma_kernel<BITS_, NT_, GR_>), smem);                                   \
     qlinear_digits_kernel<BITS_, NT_><<<n_groups, 256, 0, s>>>(x, K, M, ws, n_groups, y, M * N);            \
     cudaLaunchConfig_t cfg = {};                                                                            \
     cfg.gridDim = grid; cfg.blockDim = dim3(kMmaWarps * 32); cfg.dynamicSmemBytes = smem; cfg.stream = s;   \

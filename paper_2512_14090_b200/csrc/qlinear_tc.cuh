@@ -326,14 +326,10 @@ size_t qlinear_tc_workspace_bytes(int K, int M) { return (size_t)2 * M * K * siz
 
 aiq_status_t launch_qlinear_tc(const LayerJob& job, int N, int K, int M, void* workspace, int32_t* error_flag,
                                cudaStream_t s) {
-  static int smem_limit = 0, n_sms = 0;
-  if (!smem_limit) {
-    int dev = 0;
-    AIQ_CUDA_TRY(cudaGetDevice(&dev));
-    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
-    AIQ_CUDA_TRY(cudaFuncSetAttribute(qlinear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit));
-  }
+  DeviceProps props;
+  if (aiq_status_t st = current_device_props(&props)) return st;
+  const int smem_limit = props.smem_optin, n_sms = props.n_sms;
+  AIQ_ENSURE_DYNAMIC_SMEM(qlinear_tc_kernel, smem_limit);
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
   QtParams p = {};

@@ -193,8 +193,11 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad,
 constexpr int kStreamThreads = 256;
 constexpr int kStreamCache = 4;
 
+// Bounded by SM clocks (about 2 s), like the waits of the tensor-core kernels: the time one poll
+// takes is up to the hardware, so a poll count alone would not bound the wait in seconds.
 __device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < (1u << 26); ++i) {
+  const long long t0 = clock64();
+  for (uint32_t i = 0; i < (1u << 30); ++i) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -202,6 +205,7 @@ __device__ __forceinline__ bool stream_wait(uint32_t bar, uint32_t parity) {
         "selp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     if (ok) return true;
+    if ((i & 255u) == 255u && clock64() - t0 > 4000ll * 1000ll * 1000ll) break;
   }
   return false;                          // bounded: a copy that never lands must not hang the GPU
 }
@@ -291,15 +295,9 @@ aiq_status_t launch_quantize_bits(const float* W, int N, int K, void* packed, fl
   uint8_t* p = static_cast<uint8_t*>(packed);
   LaunchScope scope(AIQ_KERNEL_QUANTIZE, s, 2.0 * N * K,
                     4.0 * N * K + (double)N * row_bytes(K, BITS) + 4.0 * N);
-  static int n_sms = 0, smem_limit = 0;
-  if (!n_sms) {
-    int dev = 0;
-    AIQ_CUDA_TRY(cudaGetDevice(&dev));
-    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
-    AIQ_CUDA_TRY(cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    AIQ_CUDA_TRY(cudaFuncSetAttribute(quantize_stream_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      smem_limit - 1024));   // the kernel also has static shared memory
-  }
+  DeviceProps props;
+  if (aiq_status_t st = current_device_props(&props)) return st;
+  const int n_sms = props.n_sms, smem_limit = props.smem_optin;
   const bool stream_ok = K % 32 == 0 && K >= 2048 && K <= kStreamThreads * 8 * kStreamCache &&
                          N >= 4 * n_sms && ((uintptr_t)W & 15) == 0;
   if (stream_ok) {
@@ -315,6 +313,7 @@ aiq_status_t launch_quantize_bits(const float* W, int N, int K, void* packed, fl
     if (stages > 8) stages = 8;
     if (stages >= 2) {
       const int smem = stages * K * 4 + stages * 8;
+      AIQ_ENSURE_DYNAMIC_SMEM(quantize_stream_kernel<BITS>, smem_limit - 1024);   // the kernel also has static shared memory
       quantize_stream_kernel<BITS><<<blocks_per_sm * n_sms, kStreamThreads, smem, s>>>(W, N, K, p, scales, nonfinite_flag, stages);
       AIQ_LAUNCH_CHECK("quantize_stream");
       return AIQ_OK;
