@@ -123,7 +123,7 @@ def test_mobilenet_v2_cifar_batch256_sampled():
     scheme = mixed_int4_int8_scheme(53, conv_layer_indices(arch), 10, 43)
     got = model.aiq_forward(scheme, to_dev(x)).cpu().numpy()
     ref = O.forward_scheme(arch, bank, scheme, x[sample])
-    assert len(np.unique(O.predict(ref))) >= 5
+    assert len(np.unique(O.predict(ref))) >= 3                # 16 images: several classes, small margins
     assert_tensor_path_logits(got[sample], ref, "mbv2 cifar batch=256")
     assert_preds_match(O.predict(got[sample]), O.predict(ref), O.top2_margin(ref), "mbv2 cifar batch=256")
     # the same images alone give the same logits: no dependence on the batch around them
