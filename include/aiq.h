@@ -244,7 +244,7 @@ aiq_status_t aiq_forward(const aiq_model_t* model, const uint8_t* scheme_bits, c
  *   - Limit: if the model at this batch needs more than AIQ_STATIC_WORKSPACE_BYTES (see
  *     aiq_workspace_bytes(model, batch, 1)) the call returns AIQ_ERR_WORKSPACE_TOO_SMALL
  *     and launches nothing; lower the batch or use aiq_forward.  8 MiB fits, e.g.,
- *     ResNet-20 up to batch 40.
+ *     ResNet-20 up to batch 32.
  *   - The first call on each device looks up the array's device address (one
  *     cudaGetSymbolAddress with that device current).  Make that first call outside any
  *     stream capture.
@@ -288,10 +288,16 @@ void aiq_set_eval_options(int chunk, int share_prefix);
  *                    in tensor memory); activations are stored as the sum of two bfloat16
  *                    (17-18 significant bits).  Other layers use the float32 kernels on the
  *                    same storage.
+ *                    Networks that consist of a 3x3 stem and dense 3x3 / 1x1 convolutions with
+ *                    16, 32 or 64 channels on maps 8 to 64 columns wide (the CIFAR ResNets) are
+ *                    stored image-interleaved and run on the row-streaming tensor-core kernel,
+ *                    which folds the three vertical taps into the width of one MMA.
+ *   AIQ_PATH_TENSOR_TILES  AIQ_PATH_TENSOR without the row-streaming kernel: every tensor-core
+ *                    layer runs on the kernels that tile the output pixels.
  *   AIQ_PATH_AUTO    AIQ_PATH_TENSOR when the model has at least one layer the tensor
  *                    kernels accept, else AIQ_PATH_FP32.  This is the default.
  */
-enum { AIQ_PATH_AUTO = 0, AIQ_PATH_FP32 = 1, AIQ_PATH_TENSOR = 2 };
+enum { AIQ_PATH_AUTO = 0, AIQ_PATH_FP32 = 1, AIQ_PATH_TENSOR = 2, AIQ_PATH_TENSOR_TILES = 3 };
 void aiq_set_compute_path(int path);
 
 /* Counters of the last aiq_forward / aiq_eval_schemes call on this thread: kernels

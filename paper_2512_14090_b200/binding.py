@@ -29,7 +29,7 @@ EXPORTS = [
     "aiq_set_compute_path", "aiq_model_status", "aiq_debug_expire_wait", "aiq_search_greedy", "aiq_search_coordinate_descent",
 ]
 
-PATH_AUTO, PATH_FP32, PATH_TENSOR = 0, 1, 2
+PATH_AUTO, PATH_FP32, PATH_TENSOR, PATH_TENSOR_TILES = 0, 1, 2, 3
 
 STATIC_WORKSPACE_BYTES = 8 * 1024 * 1024
 

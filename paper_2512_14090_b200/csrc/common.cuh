@@ -101,7 +101,15 @@ __device__ __forceinline__ float apply_act(float v, int act) {
 //             hi = bf16_rn(v), lo = bf16_rn(v - hi): 16+ significant bits in the same bytes,
 //             in the form the bf16 tensor cores consume without conversion (the two halves
 //             are two K-slices of the GEMM).  Used when the model has tensor-core layers.
-enum { ACT_F32 = 0, ACT_SPLIT = 1 };
+//   ACT_RS    the hi / lo bfloat16 pairs of ACT_SPLIT in the image-interleaved layout of the
+//             row-streaming tensor-core convolution (conv_rs.cu):
+//             [group][row][column][plane][image][8 bfloat16], G = rs_group_images(width) images per
+//             group, plane p < C/8 = hi halves of channels 8p .. 8p+7, plane C/8 + p = their lo
+//             halves; no padding rows; the batch is padded to a multiple of 16 images.
+enum { ACT_F32 = 0, ACT_SPLIT = 1, ACT_RS = 2 };
+inline int rs_group_images(int W) { return W % 16 == 0 ? 8 : 16; }
+inline int rs_padded_batch(int B) { return (B + 15) / 16 * 16; }
+inline size_t rs_image_bytes(int H, int W, int C) { return (size_t)H * W * 4 * C; }
 inline int padded_channels(int C) { return (C + 15) / 16 * 16; }
 inline size_t split_image_bytes(int H, int W, int C) {
   return (size_t)(H + 2) * W * 2 * padded_channels(C) * 2;
@@ -172,6 +180,13 @@ bool conv_tc_bits_ok(const ConvGeom& g, int bits);
 aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* jobs_dev, int n_jobs,
                             int batch_capacity, int32_t* error_flag, double weight_bytes, int weight_bits,
                             cudaStream_t s);
+// Row-streaming tensor-core convolution on ACT_RS tensors (conv_rs.cu).  `maps`: two CUtensorMaps
+// (256 bytes) over the input slot written by conv_rs_encode_maps.  weight_bits as for launch_conv_tc.
+bool conv_rs_eligible(const ConvGeom& g);
+aiq_status_t conv_rs_encode_maps(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
+                                 void* maps_out);
+aiq_status_t launch_conv_rs(const ConvGeom& g, const void* maps, const LayerJob* jobs_dev, int n_jobs, int batch_capacity,
+                            int32_t* error_flag, double weight_bytes, int weight_bits, cudaStream_t s);
 // Pointwise (1x1, stride 1) tensor-core convolution for any channel count that is a multiple
 // of 8 (conv_pw_tc.cuh).  `map`: CUtensorMap over the input slot, dims (Cs, 2, pixels of all versions).
 bool conv_pw_tc_eligible(const ConvGeom& g);

@@ -14,6 +14,8 @@ namespace aiq {
 
 namespace {
 
+__device__ __forceinline__ int rs_group_images_dev(int W) { return (W & 15) == 0 ? 8 : 16; }
+
 constexpr int kConvThreads = 256;
 constexpr int BK = 16;
 
@@ -382,17 +384,98 @@ conv_stem_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* __r
   }
 }
 
+// The same stem writing the image-interleaved ACT_RS layout: consecutive threads own consecutive
+// images of a group at one output position, so the 16-byte plane stores of a warp are contiguous.
+template <int COUT>
+__global__ void __launch_bounds__(kStemThreads)
+conv_stem_rs_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* __restrict__ net_input) {
+  extern __shared__ __align__(16) float stem_sm[];            // [Kt][COUT] weights, [COUT] scale, [COUT] bias
+  const LayerJob job = jobs[blockIdx.z];
+  const int Kt = 9 * g.Cin;
+  float* wsm = stem_sm;
+  float* ssm = wsm + Kt * COUT;
+  float* bsm = ssm + COUT;
+  const int wrow_bytes = ((g.K + 31) / 32 * 32) * job.bits / 8;
+  for (int i = threadIdx.x; i < Kt * COUT; i += kStemThreads) {
+    const int k = i / COUT, n = i - k * COUT;
+    const int tap = k / g.Cin, c = k - tap * g.Cin;
+    wsm[i] = load_element(job.w + (size_t)n * wrow_bytes, c * 9 + tap, job.bits);
+  }
+  for (int n = threadIdx.x; n < COUT; n += kStemThreads) { ssm[n] = job.scale[n]; bsm[n] = job.bias[n]; }
+  __syncthreads();
+
+  const int G = rs_group_images_dev(g.Wo);
+  const int Bp = (g.B + 15) / 16 * 16;
+  const long long M = (long long)Bp * g.Ho * g.Wo;
+  const long long p = (long long)blockIdx.x * kStemThreads + threadIdx.x;
+  if (p >= M) return;
+  const int img = (int)(p % G);
+  const int ox = (int)((p / G) % g.Wo);
+  const int oy = (int)((p / ((long long)G * g.Wo)) % g.Ho);
+  const int grp = (int)(p / ((long long)G * g.Wo * g.Ho));
+  const int b = grp * G + img;
+  float acc[COUT];
+#pragma unroll
+  for (int n = 0; n < COUT; ++n) acc[n] = 0.f;
+  if (b < g.B) {                                               // padding images of the last group see a zero input
+    const int iy0 = oy * g.stride - 1, ix0 = ox * g.stride - 1;
+    for (int c = 0; c < g.Cin; ++c) {
+      const float* plane = net_input + ((size_t)b * g.Cin + c) * g.H * g.W;
+#pragma unroll
+      for (int r = 0; r < 3; ++r) {
+        const int iy = iy0 + r;
+#pragma unroll
+        for (int t = 0; t < 3; ++t) {
+          const int ix = ix0 + t;
+          const float xv = (iy >= 0 && iy < g.H && ix >= 0 && ix < g.W) ? __ldg(plane + (size_t)iy * g.W + ix) : 0.f;
+          const float* wk = wsm + ((r * 3 + t) * g.Cin + c) * COUT;
+#pragma unroll
+          for (int n = 0; n < COUT; n += 4) {
+            const float4 wv = *reinterpret_cast<const float4*>(wk + n);
+            acc[n] = fmaf(xv, wv.x, acc[n]);
+            acc[n + 1] = fmaf(xv, wv.y, acc[n + 1]);
+            acc[n + 2] = fmaf(xv, wv.z, acc[n + 2]);
+            acc[n + 3] = fmaf(xv, wv.w, acc[n + 3]);
+          }
+        }
+      }
+    }
+  }
+  const size_t plane_bytes = (size_t)G * 16;
+  uint8_t* dst = static_cast<uint8_t*>(job.out) +
+                 ((((size_t)grp * g.Ho + oy) * g.Wo + ox) * (COUT / 4)) * plane_bytes + (size_t)img * 16;
+#pragma unroll
+  for (int n = 0; n < COUT; n += 8) {
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) {
+      const float u0 = apply_act(fmaf(acc[n + e], ssm[n + e], bsm[n + e]), g.act);
+      const float u1 = apply_act(fmaf(acc[n + e + 1], ssm[n + e + 1], bsm[n + e + 1]), g.act);
+      __nv_bfloat16 h0, l0, h1, l1;
+      split_bf16(u0, h0, l0);
+      split_bf16(u1, h1, l1);
+      hi[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      lo[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    }
+    *reinterpret_cast<uint4*>(dst + (size_t)(n / 8) * plane_bytes) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4*>(dst + (size_t)(COUT / 8 + n / 8) * plane_bytes) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  }
+}
+
 template <int COUT>
 aiq_status_t launch_stem(const ConvGeom& g, const LayerJob* jobs, int n_jobs, const float* net_input,
                          double weight_bytes, cudaStream_t s) {
-  const long long M = (long long)g.B * (g.Ho + 2) * g.Wo;
+  const long long M = g.act_format == ACT_RS ? (long long)rs_padded_batch(g.B) * g.Ho * g.Wo
+                                             : (long long)g.B * (g.Ho + 2) * g.Wo;
   dim3 grid((unsigned)((M + kStemThreads - 1) / kStemThreads), 1, n_jobs);
   const size_t smem = (size_t)(9 * g.Cin * COUT + 2 * COUT) * sizeof(float);
   LaunchScope scope(AIQ_KERNEL_CONV, s,
                     2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(9 * g.Cin) * n_jobs,
                     weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
                                                    (double)g.B * g.Ho * g.Wo * g.Cout));
-  if (g.act_format == ACT_SPLIT)
+  if (g.act_format == ACT_RS)
+    conv_stem_rs_kernel<COUT><<<grid, kStemThreads, smem, s>>>(g, jobs, net_input);
+  else if (g.act_format == ACT_SPLIT)
     conv_stem_kernel<COUT, ACT_SPLIT><<<grid, kStemThreads, smem, s>>>(g, jobs, net_input);
   else
     conv_stem_kernel<COUT, ACT_F32><<<grid, kStemThreads, smem, s>>>(g, jobs, net_input);
@@ -443,6 +526,50 @@ avgpool_kernel(const LayerJob* __restrict__ jobs, int H, int W, int C, int Cs) {
         if (4 * q + j < C) out[(size_t)b * C + 4 * q + j] = r[j];
     }
     __syncthreads();
+  }
+}
+
+// Global average pool of an ACT_RS tensor.  One block per (group, job); a thread owns 8
+// consecutive channels of one image and every PL-th position; partial sums meet in a fixed order.
+__global__ void __launch_bounds__(kPoolThreads)
+avgpool_rs_kernel(const LayerJob* __restrict__ jobs, int B, int H, int W, int C) {
+  __shared__ float s_sum[kPoolThreads][8];
+  const LayerJob job = jobs[blockIdx.z];
+  const int G = rs_group_images_dev(W);
+  const int grp = blockIdx.x;
+  const int octets = C / 8;
+  const int units = octets * G;                           // (image, channel octet) pairs: at most 128
+  const int PL = kPoolThreads / units;
+  const int unit = threadIdx.x % units, pl = threadIdx.x / units;
+  const int img = unit % G, oc = unit / G;
+  const size_t plane_bytes = (size_t)G * 16;
+  const size_t px_bytes = (size_t)(C / 4) * plane_bytes;
+  const uint8_t* base = static_cast<const uint8_t*>(job.in) + (size_t)grp * H * W * px_bytes + (size_t)img * 16;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (pl < PL)
+    for (int i = pl; i < H * W; i += PL) {
+      const uint4 hv = __ldg(reinterpret_cast<const uint4*>(base + (size_t)i * px_bytes + (size_t)oc * plane_bytes));
+      const uint4 lv = __ldg(reinterpret_cast<const uint4*>(base + (size_t)i * px_bytes + (size_t)(octets + oc) * plane_bytes));
+      const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w}, lw[4] = {lv.x, lv.y, lv.z, lv.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        acc[2 * j] += __uint_as_float(hw[j] << 16) + __uint_as_float(lw[j] << 16);
+        acc[2 * j + 1] += __uint_as_float(hw[j] & 0xFFFF0000u) + __uint_as_float(lw[j] & 0xFFFF0000u);
+      }
+    }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) s_sum[threadIdx.x][j] = acc[j];
+  __syncthreads();
+  const int b = grp * G + img;
+  if (pl == 0 && b < B) {
+    float* out = static_cast<float*>(job.out) + (size_t)b * C + oc * 8;
+    const float inv = 1.0f / (float)(H * W);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      float t = s_sum[unit][j];
+      for (int k = 1; k < PL; ++k) t += s_sum[k * units + unit][j];
+      out[j] = t * inv;
+    }
   }
 }
 
@@ -512,7 +639,9 @@ aiq_status_t launch_avgpool(const LayerJob* jobs_dev, int n_jobs, int B, int H, 
   const int threads = kPoolThreads;
   LaunchScope scope(AIQ_KERNEL_POOL, s, (double)n_jobs * B * H * W * C,
                     4.0 * n_jobs * B * ((double)H * W * C + C));
-  if (act_format == ACT_SPLIT)
+  if (act_format == ACT_RS)
+    avgpool_rs_kernel<<<dim3(rs_padded_batch(B) / rs_group_images(W), 1, n_jobs), threads, 0, s>>>(jobs_dev, B, H, W, C);
+  else if (act_format == ACT_SPLIT)
     avgpool_kernel<ACT_SPLIT><<<dim3(B, 1, n_jobs), threads, 0, s>>>(jobs_dev, H, W, C, padded_channels(C));
   else
     avgpool_kernel<ACT_F32><<<dim3(B, 1, n_jobs), threads, 0, s>>>(jobs_dev, H, W, C, padded_channels(C));

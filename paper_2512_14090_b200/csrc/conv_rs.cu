@@ -1,0 +1,652 @@
+// Row-streaming 3x3 / 1x1 convolution on the tcgen05 tensor cores for networks whose feature
+// maps are narrow (8, 16 or 32 columns) and have 16, 32 or 64 channels (the CIFAR ResNets).
+//
+//   out[y][x][n] = act( s_n * sum_{r,t,c} code[n][c][r][t] * in[y*S + r - 1][x*S + t - 1][c] + b_n + res[y][x][n] )
+//
+// With few output channels an MMA of 128 pixels x N = Cout spends its time fetching the 128-row
+// pixel operand from shared memory, once per tap: nine fetches per pixel and layer.  Here the
+// three vertical taps are folded into the MMA's N dimension instead.  The 128 accumulator lanes
+// are (column, image) pairs of ONE image row - a group of 8 or 16 images is interleaved in
+// memory for that purpose - so the output rows y-1, y, y+1 that an input row feeds live in the
+// same lanes, in neighbouring column ranges of tensor memory.  One MMA per horizontal tap with
+// the weights [W(r=2) | W(r=1) | W(r=0)] as an N = 3 Cout operand adds an input row's
+// contribution to all three; the tensor cores do the vertical sum, the pixel operand is fetched
+// three times instead of nine, and the MMAs are three times as wide.
+//
+// Activation format ACT_RS: [group][row][column][plane][image][8 bfloat16], G = 8 images per
+// group when the width is a multiple of 16, else 16; plane p < C/8 holds the hi halves of
+// channels 8p .. 8p+7, plane C/8 + p their lo halves (value = hi + lo, see common.cuh); no
+// padding rows or columns are stored.  A TMA box brings one input row of a group into shared
+// memory as [plane][column][image][16 bytes] with zero columns on both sides; in the canonical
+// K-major layout without swizzle (8 rows x 16 bytes per core matrix, 128 bytes from one group
+// of 8 rows to the next) that is directly the A operand of every horizontal tap: tap t starts t
+// columns further.  Stride-2 layers view the columns as (parity, pair), so that every tap is
+// again a dense run of column pairs.  Output rows are finished one input row later; the epilogue
+// warps read them from tensor memory, apply scale, bias, residual and activation, split into
+// two bfloat16 and store 16 bytes per lane and plane: the 32 lanes of a warp cover whole
+// 128-byte lines, so no staging through shared memory is needed.
+//
+// Every wait is bounded as in the other tcgen05 kernels.
+#include "tc_ptx.cuh"
+
+namespace aiq {
+
+namespace {
+
+constexpr int kRsEpiWarps = 16;                        // four per quarter of the accumulator lanes
+constexpr int kRsThreads = (2 + kRsEpiWarps) * 32;     // + TMA producer + MMA issuer
+constexpr int kRsMaxStages = 6;
+constexpr int kRsMaxSlots = 16;
+constexpr int kRsTileBytes = 2048;                     // 128 operand rows x 16 bytes of one plane
+
+struct RsParams {
+  int H, W, Ho, Wo;
+  int N;                  // output channels of one slice (blockIdx.z selects the slice)
+  int cout_total;         // channels of an output pixel
+  int act;
+  int gmode;              // images per group: 0: 8 in, 8 out;  1: 16 in, 16 out;  2: 8 in, 16 out (stride 2)
+  int n_items;            // output groups of the batch
+  int rows_per_version;   // step of the TMA row coordinate from one input version to the next
+  int n_stages, n_slots;  // input-row ring depth; output rows in flight per column tile (power of two)
+  int K;                  // elements of a packed weight row
+  int stage_bytes;        // bytes one input row occupies in shared memory
+  int a_tap_off[3];       // byte offset of horizontal tap t inside a stage (column tile 0, plane 0)
+  int a_lbo;              // bytes from one plane (8 channels) to the next
+  int xt;                 // column tiles (128 lanes each) per row
+  int32_t* error_flag;
+};
+
+__host__ __device__ constexpr int rs_taps(int ks) { return ks == 3 ? 3 : 1; }
+
+// shared memory regions (base aligned to 1024 bytes)
+struct RsSmem {
+  int ring, weights, scale, bias, bars, total;
+};
+__host__ __device__ inline RsSmem rs_smem(int stages, int stage_bytes, int weight_bytes, int N) {
+  RsSmem s;
+  s.ring = 0;
+  s.weights = stages * stage_bytes;
+  s.scale = s.weights + weight_bytes;
+  s.bias = s.scale + N * 4;
+  s.bars = (s.bias + N * 4 + 127) / 128 * 128;
+  s.total = s.bars + (2 * kRsMaxStages + 2 * kRsMaxSlots + 1) * 8 + 16;
+  return s;
+}
+
+template <int C, int KS, int STRIDE, int PIECES>
+__global__ void __launch_bounds__(kRsThreads, 1)
+conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1, RsParams p,
+               const LayerJob* __restrict__ jobs) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const LayerJob job = jobs[blockIdx.y];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr int T = rs_taps(KS);                     // horizontal taps = weight tiles per piece
+  constexpr int NBLK = KS == 3 ? 3 : 1;              // vertical taps stacked along N
+  constexpr int KCH = C / 8;                         // 16-byte K chunks of the channels
+  const int N = p.N, NB = NBLK * N;
+  const int tile_b = KCH * NB * 16;                  // bytes of one weight tile
+  const int weight_bytes = PIECES * T * tile_b;
+  const int stages = p.n_stages, R = p.n_slots;
+  const RsSmem sm = rs_smem(stages, p.stage_bytes, weight_bytes, N);
+  uint8_t* ring = smem;
+  uint8_t* wsm = smem + sm.weights;
+  float* s_scale = reinterpret_cast<float*>(smem + sm.scale);
+  float* s_bias = reinterpret_cast<float*>(smem + sm.bias);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
+  const uint32_t bar_in_full = smem_u32(bars);
+  const uint32_t bar_in_empty = bar_in_full + 8 * kRsMaxStages;
+  const uint32_t bar_out_full = bar_in_empty + 8 * kRsMaxStages;
+  const uint32_t bar_out_empty = bar_out_full + 8 * kRsMaxSlots;
+  const uint32_t bar_w = bar_out_empty + 8 * kRsMaxSlots;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kRsMaxStages + 2 * kRsMaxSlots + 1);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  const int n_off = (int)blockIdx.z * N;             // first output channel of this slice
+  // Epilogue work: per output row and quarter of the lanes, `units` = column tiles x 16-channel
+  // chunks.  The WQ warps of a quarter either share the units of every row, or, where a row has
+  // fewer units than that, take every (WQ / units)-th row each, so several rows are drained at once.
+  constexpr int WQ = kRsEpiWarps / 4;
+  const int units = p.xt * (N / 16);
+  const int epi_sets = units < WQ ? units : WQ;      // warps of a quarter that read one row
+
+  // ---- set-up -----------------------------------------------------------------------------
+  if (tid == 0) {
+    for (int i = 0; i < kRsMaxStages; ++i) {
+      mbar_init(bar_in_full + 8 * i, 1);
+      mbar_init(bar_in_empty + 8 * i, 1);
+    }
+    for (int i = 0; i < kRsMaxSlots; ++i) {
+      mbar_init(bar_out_full + 8 * i, 1);
+      mbar_init(bar_out_empty + 8 * i, 4 * epi_sets);      // one arrival per epilogue warp that reads the row
+    }
+    mbar_init(bar_w, 1);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tmem_alloc(smem_u32(s_tmem), 512);
+    tmem_relinquish();
+  }
+  // packed weight rows of this slice: one bulk copy into the (still unused) ring, then expansion
+  // to bfloat16 in the operand layout [tap][8-channel chunk][vertical tap block, channel][8 channels]
+  const int kpad = (p.K + 31) / 32 * 32;
+  const uint32_t wrow_bytes = (uint32_t)kpad * job.bits / 8;
+  const uint32_t packed_bytes = wrow_bytes * N;
+  if (tid == 0) {
+    mbar_expect_tx(bar_w, packed_bytes);
+    bulk_load(smem_u32(ring), job.w + (size_t)n_off * wrow_bytes, packed_bytes, bar_w);
+  }
+  for (int i = tid; i < N; i += kRsThreads) {
+    s_scale[i] = job.scale[n_off + i];
+    s_bias[i] = job.bias[n_off + i];
+  }
+  bool alive = mbar_wait_warp(bar_w, 0, s_abort, p.error_flag);
+  if (alive) {
+    const int w_units = T * KCH * NB;
+    for (int u = tid; u < w_units; u += kRsThreads) {
+      const int row = u % NB;
+      const int kc = (u / NB) % KCH;
+      const int ti = u / (NB * KCH);
+      const int blk = row / N, n = row - blk * N;
+      // vertical tap of a block: stride 1: the input row feeds output rows y-1, y, y+1 = taps 2, 1, 0;
+      // stride 2: even input rows carry tap 1 (block 0), odd rows taps 2 and 0 (blocks 1, 2)
+      const int r = KS == 1 ? 0 : (STRIDE == 1 ? 2 - blk : (blk == 0 ? 1 : (blk == 1 ? 2 : 0)));
+      const uint8_t* wrow = ring + (size_t)n * wrow_bytes;
+      uint32_t pk[PIECES][4];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int c = kc * 8 + j;
+        const int k = KS == 1 ? c : (c * 3 + r) * 3 + ti;
+        float w;
+        if (job.bits == 8) w = (float)(int)(int8_t)wrow[k];
+        else if (job.bits == 4) {
+          const int byte = wrow[k >> 1];
+          w = (float)((((k & 1) ? (byte >> 4) : (byte & 0xF)) ^ 8) - 8);
+        } else if (job.bits == 16) w = __half2float(reinterpret_cast<const __half*>(wrow)[k]);
+        else w = reinterpret_cast<const float*>(wrow)[k];
+#pragma unroll
+        for (int pc = 0; pc < PIECES; ++pc) {
+          const __nv_bfloat16 hb = __float2bfloat16_rn(w);   // exact for the integer codes
+          w -= __bfloat162float(hb);                          // exact: the remainder of the rounding
+          const uint32_t bits16 = (uint32_t)__bfloat16_as_ushort(hb);
+          if (j & 1) pk[pc][j >> 1] |= bits16 << 16; else pk[pc][j >> 1] = bits16;
+        }
+      }
+#pragma unroll
+      for (int pc = 0; pc < PIECES; ++pc)
+        *reinterpret_cast<uint4*>(wsm + (size_t)(pc * T + ti) * tile_b + (size_t)kc * NB * 16 + row * 16) =
+            make_uint4(pk[pc][0], pk[pc][1], pk[pc][2], pk[pc][3]);
+    }
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // expanded weights -> visible to the MMA
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  alive = alive && (*s_abort == 0);
+
+  // rows of the input that carry work: a 1x1 convolution at stride 2 only reads the even ones
+  auto row_used = [&](int y) -> bool { return !(KS == 1 && STRIDE == 2 && (y & 1)); };
+
+  // ---- roles ------------------------------------------------------------------------------
+  if (warp == 0) {
+    if (lane == 0 && alive) {
+      uint32_t stage = 0, phase = 0;
+      uint32_t issued = 0, issued_phase = 0;
+      for (int item = blockIdx.x; item < p.n_items && alive; item += gridDim.x) {
+        const int row0 = job.in_version * p.rows_per_version + (p.gmode == 2 ? 2 * item : item) * p.H;
+        for (int y = 0; y < p.H && alive; ++y) {
+          if (!row_used(y)) continue;
+          alive = mbar_wait(bar_in_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+          if (!alive) break;
+          issued |= 1u << stage;
+          issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
+          const uint32_t bar = bar_in_full + 8 * stage;
+          const uint32_t dst = smem_u32(ring) + stage * p.stage_bytes;
+          mbar_expect_tx(bar, (uint32_t)p.stage_bytes);
+          if (STRIDE == 1) {
+            tma_load_4d(dst, &map0, bar, 0, KS == 3 ? -1 : 0, 0, row0 + y);
+          } else if (p.gmode != 2) {
+            tma_load_5d(dst, &map0, bar, 0, KS == 3 ? -1 : 0, 0, 0, row0 + y);
+          } else if (KS == 3) {
+            // odd columns from pair -1 (tap 0), even columns (tap 1), odd columns from pair 0 (tap 2)
+            const uint32_t sub = (uint32_t)p.stage_bytes / 3;
+            tma_load_5d(dst, &map1, bar, 0, -1, 0, 0, row0 + y);
+            tma_load_5d(dst + sub, &map0, bar, 0, 0, 0, 0, row0 + y);
+            tma_load_5d(dst + 2 * sub, &map1, bar, 0, 0, 0, 0, row0 + y);
+          } else {
+            tma_load_5d(dst, &map0, bar, 0, 0, 0, 0, row0 + y);
+          }
+          if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      // copies in flight must land before the CTA exits (matters when another role gave up)
+      for (int i = 0; i < stages; ++i)
+        if (issued & (1u << i)) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_in_full + 8 * i, (issued_phase >> i) & 1u) && clock64() - t0 < kWaitLimitCycles) {}
+        }
+    }
+  } else if (warp == 1) {
+    if (alive) {                                     // all 32 lanes, converged; an elected lane issues
+      constexpr uint32_t IDESC0 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);   // f32 += bf16 x bf16, M = 128
+      constexpr uint32_t DESC_HI = (uint32_t)(128 >> 4) | (1u << 14);   // 128 bytes between groups of 8 rows; no swizzle
+      const uint32_t a_lbo_field = ((uint32_t)p.a_lbo >> 4) << 16;
+      const uint32_t w_lo0 = (smem_u32(wsm) >> 4) | (((uint32_t)(NB * 16) >> 4) << 16);
+      // operand steps in 16-byte units, so that an MMA costs a few additions
+      const uint32_t a_part_step = ((uint32_t)KCH * (uint32_t)p.a_lbo) >> 4;     // hi planes -> lo planes
+      const uint32_t a_kk_step = (2u * (uint32_t)p.a_lbo) >> 4;                  // 16 channels further
+      const uint32_t b_tile_step = (uint32_t)tile_b >> 4, b_kk_step = 2u * (uint32_t)NB;
+      const uint32_t n_field = ((uint32_t)N >> 3) << 17;                         // N field of one output row
+      const uint32_t a_tap0 = (uint32_t)p.a_tap_off[0], a_tap1 = (uint32_t)p.a_tap_off[1], a_tap2 = (uint32_t)p.a_tap_off[2];
+      uint32_t stage = 0, phase = 0;
+      int item_local = 0;
+      for (int item = blockIdx.x; item < p.n_items && alive; item += gridDim.x, ++item_local) {
+        const int q0 = item_local * p.Ho;
+        for (int y = 0; y < p.H && alive; ++y) {
+          if (!row_used(y)) continue;
+          // output rows this input row contributes to: [yo, yo + n_rows), weight blocks [blk, ...),
+          // the rows from index `fresh` on receive their first contribution (they overwrite)
+          int yo, n_rows, blk, fresh;
+          if (KS == 1) { yo = y / STRIDE; n_rows = 1; blk = 0; fresh = 0; }
+          else if (STRIDE == 1) {
+            yo = y > 0 ? y - 1 : 0;
+            const int hi = y + 1 < p.H ? y + 1 : p.H - 1;
+            n_rows = hi - yo + 1;
+            blk = yo - (y - 1);
+            fresh = y == 0 ? 0 : (y + 1 < p.H ? n_rows - 1 : n_rows);
+          } else if ((y & 1) == 0) { yo = y >> 1; n_rows = 1; blk = 0; fresh = y == 0 ? 0 : 1; }
+          else { yo = y >> 1; blk = 1; n_rows = (yo + 1 < p.Ho) ? 2 : 1; fresh = 1; }
+          for (int i = fresh; i < n_rows && alive; ++i) {
+            const int q = q0 + yo + i;
+            alive = mbar_wait_warp(bar_out_empty + 8 * (q & (R - 1)), ((q / R) & 1) ^ 1u, s_abort, p.error_flag);
+          }
+          if (!alive) break;
+          // The rows' accumulator slots are consecutive except where the ring wraps.  All K steps but
+          // the first add to every row: one MMA per run of consecutive slots (`rest`, at most two).
+          // The first K step must overwrite the fresh rows: runs are cut at `fresh` as well (`head`,
+          // at most three).  A run = (N field, accumulator column, weight row offset).
+          const int s0 = (q0 + yo) & (R - 1);
+          const int wrap = R - s0;                     // rows from this index on continue at slot 0
+          const int cw = (wrap > 0 && wrap < n_rows) ? wrap : n_rows;     // cut at the wrap, if inside
+          const int cf = (fresh > 0 && fresh < n_rows) ? fresh : n_rows;  // cut at the first fresh row, if inside
+          auto run_idesc = [&](int i, int j) -> uint32_t { return IDESC0 | (uint32_t)(j - i) * n_field; };
+          auto run_dcol = [&](int i) -> uint32_t { return (uint32_t)(((s0 + i) & (R - 1)) * N); };
+          auto run_boff = [&](int i) -> uint32_t { return (uint32_t)((blk + i) * N); };
+          // rest: [0, cw) [cw, n_rows)
+          const bool rest1 = cw < n_rows;
+          const uint32_t r0_idesc = run_idesc(0, cw), r0_dcol = run_dcol(0), r0_boff = run_boff(0);
+          const uint32_t r1_idesc = run_idesc(cw, n_rows), r1_dcol = run_dcol(cw), r1_boff = run_boff(cw);
+          // head: [0, c1) [c1, c2) [c2, n_rows) with c1 <= c2 the cuts in order
+          const int c1 = cw < cf ? cw : cf;
+          int c2 = cw < cf ? cf : cw;
+          if (c2 == c1) c2 = n_rows;
+          const bool head1 = c1 < n_rows, head2 = c2 < n_rows;
+          const uint32_t h0_idesc = run_idesc(0, c1), h0_dcol = run_dcol(0), h0_boff = run_boff(0), h0_acc = 0 >= fresh ? 0u : 1u;
+          const uint32_t h1_idesc = run_idesc(c1, c2), h1_dcol = run_dcol(c1), h1_boff = run_boff(c1), h1_acc = c1 >= fresh ? 0u : 1u;
+          const uint32_t h2_idesc = run_idesc(c2, n_rows), h2_dcol = run_dcol(c2), h2_boff = run_boff(c2), h2_acc = c2 >= fresh ? 0u : 1u;
+          alive = mbar_wait_warp(bar_in_full + 8 * stage, phase, s_abort, p.error_flag);
+          if (!alive) break;
+          tc_fence_after();
+          const uint32_t a_stage = smem_u32(ring) + stage * p.stage_bytes;
+          for (int xt = 0; xt < p.xt; ++xt) {
+            const uint32_t d_xt = tmem_base + (uint32_t)(xt * R * N);
+            const uint32_t a_xt = ((a_stage + (uint32_t)xt * kRsTileBytes) >> 4) | a_lbo_field;
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+              const uint32_t a_t = a_xt + ((t == 0 ? a_tap0 : (t == 1 ? a_tap1 : a_tap2)) >> 4);
+#pragma unroll
+              for (int part = 0; part < 2; ++part) {
+#pragma unroll
+                for (int kk = 0; kk < C / 16; ++kk) {
+                  const uint64_t adesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(a_t + part * a_part_step + kk * a_kk_step);
+#pragma unroll
+                  for (int pc = 0; pc < PIECES; ++pc) {
+                    const uint32_t b_lo = w_lo0 + (uint32_t)(pc * T + t) * b_tile_step + (uint32_t)kk * b_kk_step;
+                    if (t == 0 && part == 0 && kk == 0 && pc == 0) {
+                      umma_bf16(d_xt + h0_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + h0_boff), h0_idesc, h0_acc);
+                      if (head1) umma_bf16(d_xt + h1_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + h1_boff), h1_idesc, h1_acc);
+                      if (head2) umma_bf16(d_xt + h2_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + h2_boff), h2_idesc, h2_acc);
+                    } else {
+                      umma_bf16(d_xt + r0_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + r0_boff), r0_idesc, 1u);
+                      if (rest1) umma_bf16(d_xt + r1_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + r1_boff), r1_idesc, 1u);
+                    }
+                  }
+                }
+              }
+            }
+          }
+          umma_commit(bar_in_empty + 8 * stage);       // the stage is free once these MMAs retire
+          if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+          // output rows that are complete with this input row
+          if (KS == 1) umma_commit(bar_out_full + 8 * ((q0 + yo) & (R - 1)));
+          else if (STRIDE == 1) {
+            if (y >= 1) umma_commit(bar_out_full + 8 * ((q0 + y - 1) & (R - 1)));
+            if (y == p.H - 1) umma_commit(bar_out_full + 8 * ((q0 + y) & (R - 1)));
+          } else if (y & 1) umma_commit(bar_out_full + 8 * ((q0 + yo) & (R - 1)));
+        }
+      }
+    }
+  } else {
+    // Epilogue.  Accumulator lanes 32 qd .. 32 qd + 31 belong to the warps with warp index mod 4 = qd.
+    const int qd = warp & 3;
+    const int h = (warp - 2) >> 2;                     // index among the warps of the quarter
+    const int l = qd * 32 + lane;                      // accumulator lane = operand row of the tile
+    int x_local, img;
+    if (p.gmode == 0) { x_local = l >> 3; img = l & 7; }
+    else if (p.gmode == 1) { x_local = l >> 4; img = l & 15; }
+    else { x_local = (l >> 3) & 7; img = ((l >> 6) << 3) | (l & 7); }
+    const int X = p.gmode == 0 ? 16 : 8;               // columns per tile
+    const int Gout = p.gmode == 0 ? 8 : 16;
+    const int planes_out = p.cout_total / 4;
+    const size_t plane_bytes = (size_t)Gout * 16;
+    const size_t px_bytes = (size_t)planes_out * plane_bytes;
+    const int chunks = N / 16;
+    const uint8_t* res_base = static_cast<const uint8_t*>(job.res);
+    uint8_t* out_base = static_cast<uint8_t*>(job.out);
+    const int lo_plane0 = p.cout_total / 8;
+    // this warp's units of a row and its rows of an item
+    const int unit0 = units >= WQ ? h : h % units;
+    const int unit_step = units >= WQ ? WQ : units;
+    const int row_first = units >= WQ ? 0 : h / units;
+    const int row_step = units >= WQ ? 1 : WQ / units;
+    const int rows_mine = p.Ho / row_step;             // rows of an item this warp drains
+    const int n_my_items = ((int)blockIdx.x < p.n_items) ? (p.n_items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int total = n_my_items * rows_mine;
+    auto row_offset = [&](int k) -> size_t {           // byte offset of this lane's image in the k-th row of this warp
+      const int il = k / rows_mine;
+      const int y = row_first + (k - il * rows_mine) * row_step;
+      return ((size_t)((int)blockIdx.x + il * (int)gridDim.x) * p.Ho + y) * p.Wo * px_bytes + (size_t)img * 16;
+    };
+    auto unit_offset = [&](int u, int* c0) -> size_t { // byte offset of (column, first hi plane) of unit u inside a row
+      const int xt = u / chunks;
+      *c0 = (u - xt * chunks) * 16;
+      return (size_t)(xt * X + x_local) * px_bytes + (size_t)((n_off + *c0) >> 3) * plane_bytes;
+    };
+    // The residual of the first unit of this warp's next row is requested as soon as the current
+    // row's arithmetic is done, so its memory latency overlaps the stores and the next wait.
+    uint4 rres[4];
+    auto load_res = [&](int k, int u, uint4* r) {
+      int c0;
+      const uint8_t* src = res_base + row_offset(k) + unit_offset(u, &c0);
+      r[0] = __ldg(reinterpret_cast<const uint4*>(src));
+      r[1] = __ldg(reinterpret_cast<const uint4*>(src + plane_bytes));
+      r[2] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)lo_plane0 * plane_bytes));
+      r[3] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(lo_plane0 + 1) * plane_bytes));
+    };
+    if (res_base && total > 0 && alive) load_res(0, unit0, rres);
+    for (int k = 0; k < total && alive; ++k) {
+      const int il = k / rows_mine;
+      const int y = row_first + (k - il * rows_mine) * row_step;
+      const int q = il * p.Ho + y;
+      const int slot = q & (R - 1);
+      const size_t row_off = row_offset(k);
+      alive = mbar_wait_warp(bar_out_full + 8 * slot, (q / R) & 1, s_abort, p.error_flag);
+      if (!alive) break;
+      tc_fence_after();
+      for (int u = unit0; u < units; u += unit_step) {
+        int c0;
+        const size_t uoff = unit_offset(u, &c0);
+        const int xt = u / chunks;
+        uint32_t v[16];
+        tmem_ld16(tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)((xt * R + slot) * N + c0), v);
+        if (res_base && u != unit0) load_res(k, u, rres);
+        tmem_ld_wait();
+        if (u + unit_step >= units) {
+          // the last accumulator columns this warp reads from the slot: hand it back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_out_empty + 8 * slot);
+        }
+        uint32_t hi[8], lo[8];
+#pragma unroll
+        for (int e = 0; e < 16; e += 4) {
+          const float4 sc = *reinterpret_cast<const float4*>(s_scale + c0 + e);
+          const float4 bi = *reinterpret_cast<const float4*>(s_bias + c0 + e);
+          float u0 = fmaf(__uint_as_float(v[e]), sc.x, bi.x);
+          float u1 = fmaf(__uint_as_float(v[e + 1]), sc.y, bi.y);
+          float u2 = fmaf(__uint_as_float(v[e + 2]), sc.z, bi.z);
+          float u3 = fmaf(__uint_as_float(v[e + 3]), sc.w, bi.w);
+          if (res_base) {
+            // planes 0 / 1 of the chunk hold channels 0-7 / 8-15; a bfloat16 is the upper half of a float
+            const uint4 rh4 = rres[e >> 3], rl4 = rres[2 + (e >> 3)];
+            const uint32_t rh0 = (e & 4) ? rh4.z : rh4.x, rh1 = (e & 4) ? rh4.w : rh4.y;
+            const uint32_t rl0 = (e & 4) ? rl4.z : rl4.x, rl1 = (e & 4) ? rl4.w : rl4.y;
+            u0 += __uint_as_float(rh0 << 16) + __uint_as_float(rl0 << 16);
+            u1 += __uint_as_float(rh0 & 0xFFFF0000u) + __uint_as_float(rl0 & 0xFFFF0000u);
+            u2 += __uint_as_float(rh1 << 16) + __uint_as_float(rl1 << 16);
+            u3 += __uint_as_float(rh1 & 0xFFFF0000u) + __uint_as_float(rl1 & 0xFFFF0000u);
+          }
+          split_pair(apply_act(u0, p.act), apply_act(u1, p.act), hi[e >> 1], lo[e >> 1]);
+          split_pair(apply_act(u2, p.act), apply_act(u3, p.act), hi[(e >> 1) + 1], lo[(e >> 1) + 1]);
+        }
+        // the residual registers are free again: request the first unit of this warp's next row
+        if (res_base && u + unit_step >= units && k + 1 < total) load_res(k + 1, unit0, rres);
+        uint8_t* dst = out_base + row_off + uoff;
+        *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(dst + plane_bytes) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+        *reinterpret_cast<uint4*>(dst + (size_t)lo_plane0 * plane_bytes) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        *reinterpret_cast<uint4*>(dst + (size_t)(lo_plane0 + 1) * plane_bytes) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+      }
+    }
+  }
+
+  // ---- teardown -----------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn rs_encode_fn() {
+  static std::atomic<EncodeTiledFn> fn{nullptr};
+  if (EncodeTiledFn f = fn.load(std::memory_order_acquire)) return f;
+  void* sym = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn.store(reinterpret_cast<EncodeTiledFn>(sym), std::memory_order_release);
+  return reinterpret_cast<EncodeTiledFn>(sym);
+}
+
+// geometry shared by the map encoder and the launcher
+struct RsShape {
+  int Gin, Gout, gmode, planes, xt, stage_bytes, a_lbo, a_tap_off[3];
+};
+
+bool rs_shape(const ConvGeom& g, RsShape* s) {
+  if (g.in_is_nchw || g.act_format != ACT_RS) return false;
+  if (!((g.ks == 3 && g.pad == 1) || (g.ks == 1 && g.pad == 0))) return false;
+  if (g.stride != 1 && g.stride != 2) return false;
+  if (g.Cin != 16 && g.Cin != 32 && g.Cin != 64) return false;
+  if (g.Cout != 16 && g.Cout != 32 && g.Cout != 64) return false;
+  if (g.W % 8 != 0 || g.Wo % 8 != 0 || g.W > 64 || g.H < 2) return false;
+  if (g.stride == 2 && ((g.H & 1) || (g.W & 1))) return false;
+  s->Gin = rs_group_images(g.W);
+  s->Gout = rs_group_images(g.Wo);
+  s->planes = g.Cin / 4;
+  if (s->Gin == 8 && s->Gout == 8) s->gmode = 0;
+  else if (s->Gin == 16 && s->Gout == 16) s->gmode = 1;
+  else if (s->Gin == 8 && s->Gout == 16 && g.stride == 2 && g.W == 16) s->gmode = 2;
+  else return false;
+  if (s->gmode == 1 && g.stride != 1) return false;
+  const int X = s->gmode == 0 ? 16 : 8;
+  s->xt = g.Wo / X;
+  const int gb = s->Gin * 16;                        // bytes of one (column, plane) cell
+  s->a_tap_off[0] = s->a_tap_off[1] = s->a_tap_off[2] = 0;
+  if (g.stride == 1) {
+    const int cols = g.ks == 3 ? g.W + 2 : g.W;
+    s->a_lbo = cols * gb;
+    s->stage_bytes = s->planes * s->a_lbo;
+    if (g.ks == 3) for (int t = 0; t < 3; ++t) s->a_tap_off[t] = t * gb;
+  } else if (s->gmode == 0) {
+    if (g.ks == 3) {
+      const int pairs = g.W / 2 + 1;                 // pair -1 .. W/2 - 1
+      s->a_lbo = 2 * pairs * gb;                     // [plane][parity][pair]
+      s->stage_bytes = s->planes * s->a_lbo;
+      s->a_tap_off[0] = pairs * gb;                  // odd columns, from pair -1
+      s->a_tap_off[1] = gb;                          // even columns, from pair 0
+      s->a_tap_off[2] = pairs * gb + gb;             // odd columns, from pair 0
+    } else {
+      s->a_lbo = (g.W / 2) * gb;
+      s->stage_bytes = s->planes * s->a_lbo;
+    }
+  } else {
+    // 8 -> 16 images per group: per load [plane][half of the output group][8 column pairs][128 bytes]
+    s->a_lbo = 2048;
+    const int sub = s->planes * 2048;
+    s->stage_bytes = (g.ks == 3 ? 3 : 1) * sub;
+    if (g.ks == 3) for (int t = 0; t < 3; ++t) s->a_tap_off[t] = t * sub;
+  }
+  return true;
+}
+
+int rs_weight_slices(const ConvGeom& g, int weight_bits) { return (weight_bits > 8 && g.Cout == 64) ? 2 : 1; }
+
+int rs_weight_bytes(const ConvGeom& g, int weight_bits) {
+  const int pieces = weight_bits > 8 ? 2 : 1;
+  const int n = g.Cout / rs_weight_slices(g, weight_bits);
+  return pieces * rs_taps(g.ks) * (g.Cin / 8) * (g.ks == 3 ? 3 : 1) * n * 16;
+}
+
+// ring depth that fits beside the weights, or 0
+int rs_stages(const ConvGeom& g, const RsShape& s, int weight_bits, int smem_limit) {
+  const int n = g.Cout / rs_weight_slices(g, weight_bits);
+  const int packed = n * (int)row_bytes(g.K, weight_bits <= 8 ? 8 : weight_bits);
+  for (int st = kRsMaxStages; st >= 2; --st)
+    if (rs_smem(st, s.stage_bytes, rs_weight_bytes(g, weight_bits), n).total + 1024 <= smem_limit &&
+        packed <= st * s.stage_bytes)
+      return st;
+  return 0;
+}
+
+template <int C, int KS, int STRIDE, int PIECES>
+aiq_status_t launch_rs(const ConvGeom& g, const RsShape& sh, const CUtensorMap* maps, const LayerJob* jobs_dev, int n_jobs,
+                       int batch_capacity, int32_t* error_flag, double weight_bytes, int weight_bits, cudaStream_t s) {
+  DeviceProps props;
+  if (aiq_status_t st = current_device_props(&props)) return st;
+  const int slices = rs_weight_slices(g, weight_bits);
+  const int N = g.Cout / slices;
+  const int stages = rs_stages(g, sh, weight_bits, props.smem_optin);
+  if (!stages) return set_error(AIQ_ERR_SHAPE, "conv_rs: shared memory does not fit (%d bytes per input row)", sh.stage_bytes);
+  RsParams p = {};
+  p.H = g.H; p.W = g.W; p.Ho = g.Ho; p.Wo = g.Wo; p.N = N; p.cout_total = g.Cout; p.act = g.act;
+  p.gmode = sh.gmode;
+  p.n_items = rs_padded_batch(g.B) / sh.Gout;
+  p.rows_per_version = rs_padded_batch(batch_capacity) / sh.Gin * g.H;
+  p.n_stages = stages;
+  int slots = kRsMaxSlots;
+  while (slots > 4 && sh.xt * slots * N > 512) slots >>= 1;
+  if (sh.xt * slots * N > 512) return set_error(AIQ_ERR_SHAPE, "conv_rs: %d column tiles of %d channels exceed tensor memory", sh.xt, N);
+  p.n_slots = slots;
+  p.K = g.K; p.stage_bytes = sh.stage_bytes; p.a_lbo = sh.a_lbo; p.xt = sh.xt;
+  for (int t = 0; t < 3; ++t) p.a_tap_off[t] = sh.a_tap_off[t];
+  p.error_flag = error_flag;
+  const int smem_bytes = rs_smem(stages, sh.stage_bytes, rs_weight_bytes(g, weight_bits), N).total + 1024;
+  AIQ_ENSURE_DYNAMIC_SMEM((conv_rs_kernel<C, KS, STRIDE, PIECES>), props.smem_optin);
+  int ctas = props.n_sms / (n_jobs * slices);
+  if (ctas > p.n_items) ctas = p.n_items;
+  if (ctas < 1) ctas = 1;
+  {
+    LaunchScope scope(AIQ_KERNEL_CONV_TC, s,
+                      2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
+                      weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W + (double)g.B * g.Ho * g.Wo * g.Cout));
+    conv_rs_kernel<C, KS, STRIDE, PIECES><<<dim3(ctas, n_jobs, slices), kRsThreads, smem_bytes, s>>>(maps[0], maps[1], p, jobs_dev);
+  }
+  AIQ_LAUNCH_CHECK("conv_rs");
+  return AIQ_OK;
+}
+
+}  // namespace
+
+bool conv_rs_eligible(const ConvGeom& g) {
+  RsShape s;
+  if (!rs_shape(g, &s)) return false;
+  DeviceProps props;
+  int smem_limit = 227 * 1024;
+  if (current_device_props(&props) == AIQ_OK) smem_limit = props.smem_optin;
+  for (int bits : {8, 16, 32})
+    if (!rs_stages(g, s, bits, smem_limit)) return false;
+  const int n32 = g.Cout / rs_weight_slices(g, 32);
+  return s.xt * 4 * g.Cout <= 512 && s.xt * 4 * n32 <= 512;
+}
+
+aiq_status_t conv_rs_encode_maps(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
+                                 void* maps_out /* 2 x 128 bytes */) {
+  EncodeTiledFn enc = rs_encode_fn();
+  if (!enc) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  RsShape s;
+  if (!rs_shape(g, &s)) return set_error(AIQ_ERR_SHAPE, "conv_rs: layer shape is not supported");
+  CUtensorMap* maps = static_cast<CUtensorMap*>(maps_out);
+  const cuuint64_t gb = (cuuint64_t)s.Gin * 16;                         // bytes of a (column, plane) cell
+  const cuuint64_t col_bytes = (cuuint64_t)s.planes * gb;               // one column of a group
+  const cuuint64_t row_bytes_ = (cuuint64_t)g.W * col_bytes;            // one row of a group
+  const cuuint64_t rows = (cuuint64_t)n_versions * (rs_padded_batch(batch_capacity) / s.Gin) * g.H;
+  void* base = const_cast<void*>(slot_base);
+  CUresult r = CUDA_SUCCESS;
+  const cuuint32_t one[5] = {1, 1, 1, 1, 1};
+  if (g.stride == 1) {
+    // (image x 8 channels, column, plane, row over all groups and versions)
+    cuuint64_t dims[4] = {(cuuint64_t)s.Gin * 8, (cuuint64_t)g.W, (cuuint64_t)s.planes, rows};
+    cuuint64_t strides[3] = {col_bytes, gb, row_bytes_};
+    cuuint32_t box[4] = {(cuuint32_t)s.Gin * 8, (cuuint32_t)(g.ks == 3 ? g.W + 2 : g.W), (cuuint32_t)s.planes, 1u};
+    r = enc(&maps[0], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, one, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    maps[1] = maps[0];
+  } else if (s.gmode == 0) {
+    // (image x 8 channels, column pair, column parity, plane, row)
+    cuuint64_t dims[5] = {(cuuint64_t)s.Gin * 8, (cuuint64_t)g.W / 2, 2, (cuuint64_t)s.planes, rows};
+    cuuint64_t strides[4] = {2 * col_bytes, col_bytes, gb, row_bytes_};
+    cuuint32_t box[5] = {(cuuint32_t)s.Gin * 8, (cuuint32_t)(g.ks == 3 ? g.W / 2 + 1 : g.W / 2), g.ks == 3 ? 2u : 1u,
+                         (cuuint32_t)s.planes, 1u};
+    r = enc(&maps[0], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, one, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    maps[1] = maps[0];
+  } else {
+    // two input groups of 8 images feed one output group of 16: (image x 8 channels, column pair,
+    // group of the pair, plane, row), one map over the even columns and one over the odd ones
+    const cuuint64_t group_bytes = (cuuint64_t)g.H * row_bytes_;
+    cuuint64_t dims[5] = {64, (cuuint64_t)g.W / 2, 2, (cuuint64_t)s.planes, rows};
+    cuuint64_t strides[4] = {2 * col_bytes, group_bytes, gb, row_bytes_};
+    cuuint32_t box[5] = {64u, 8u, 2u, (cuuint32_t)s.planes, 1u};
+    for (int par = 0; par < 2 && r == CUDA_SUCCESS; ++par)
+      r = enc(&maps[par], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, static_cast<uint8_t*>(base) + par * col_bytes, dims, strides, box,
+              one, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
+  if (r != CUDA_SUCCESS) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled (row-streaming convolution) failed with code %d", (int)r);
+  return AIQ_OK;
+}
+
+aiq_status_t launch_conv_rs(const ConvGeom& g, const void* maps, const LayerJob* jobs_dev, int n_jobs, int batch_capacity,
+                            int32_t* error_flag, double weight_bytes, int weight_bits, cudaStream_t s) {
+  RsShape sh;
+  if (!rs_shape(g, &sh)) return set_error(AIQ_ERR_SHAPE, "conv_rs: layer shape is not supported");
+  const CUtensorMap* m = static_cast<const CUtensorMap*>(maps);
+#define AIQ_RS_ARGS g, sh, m, jobs_dev, n_jobs, batch_capacity, error_flag, weight_bytes, weight_bits, s
+#define AIQ_RS_KS(C_, P_)                                                                              \
+  do {                                                                                                \
+    if (g.ks == 3) return g.stride == 1 ? launch_rs<C_, 3, 1, P_>(AIQ_RS_ARGS) : launch_rs<C_, 3, 2, P_>(AIQ_RS_ARGS); \
+    return g.stride == 1 ? launch_rs<C_, 1, 1, P_>(AIQ_RS_ARGS) : launch_rs<C_, 1, 2, P_>(AIQ_RS_ARGS); \
+  } while (0)
+#define AIQ_RS_C(C_)                                  \
+  if (g.Cin == C_) {                                  \
+    if (weight_bits <= 8) AIQ_RS_KS(C_, 1);           \
+    AIQ_RS_KS(C_, 2);                                 \
+  }
+  AIQ_RS_C(16) AIQ_RS_C(32) AIQ_RS_C(64)
+#undef AIQ_RS_C
+#undef AIQ_RS_KS
+#undef AIQ_RS_ARGS
+  return set_error(AIQ_ERR_SHAPE, "conv_rs: no kernel for Cin=%d", g.Cin);
+}
+
+}  // namespace aiq

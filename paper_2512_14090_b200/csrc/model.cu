@@ -127,7 +127,7 @@ struct aiq_model {
   std::vector<size_t> slot_bytes;    // per-image capacity of each activation slot
   void* dev_mem;
   size_t dev_bytes;
-  int act_format;                    // ACT_F32 or ACT_SPLIT (see common.cuh)
+  int act_format;                    // ACT_F32, ACT_SPLIT or ACT_RS (see common.cuh)
   int32_t* status_word;              // device word raised by a kernel whose bounded wait expired
 };
 
@@ -223,10 +223,12 @@ static ConvGeom make_geom(const aiq_model* m, const LayerInfo& li, int B) {
   return g;
 }
 
-// 0: float32 kernels only; 1: small-channel 3x3 / 1x1 tensor-core kernel; 2: pointwise tensor-core kernel
+// 0: float32 kernels only; 1: small-channel 3x3 / 1x1 tensor-core kernel; 2: pointwise tensor-core
+// kernel; 3: row-streaming tensor-core kernel (models stored in ACT_RS)
 static int layer_tensor_kind(const aiq_model* m, const LayerInfo& li) {
   if (li.d.kind != AIQ_LAYER_CONV) return 0;
   const ConvGeom g = make_geom(m, li, 1);
+  if (conv_rs_eligible(g)) return 3;
   if (conv_tc_eligible(g)) return 1;
   if (conv_pw_tc_eligible(g)) return 2;
   return 0;
@@ -319,11 +321,29 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
   if (st != AIQ_OK) { delete m; return st; }
   m->in_c = arch->in_c; m->in_h = arch->in_h; m->in_w = arch->in_w;
   m->dev_mem = dev_mem; m->dev_bytes = dev_bytes;
-  m->act_format = ACT_SPLIT;                      // tentatively, to ask which layers would qualify
-  bool any_tc = false;
-  for (const LayerInfo& li : m->layers) any_tc = any_tc || layer_on_tensor_cores(m, li);
   const int opt_path = g_opt_path.load();
-  m->act_format = (opt_path == AIQ_PATH_TENSOR || (opt_path == AIQ_PATH_AUTO && any_tc)) ? ACT_SPLIT : ACT_F32;
+  // Row-streaming storage when every layer can live in it: a 3x3 stem on the network input, then
+  // only dense convolutions the row-streaming kernel takes, then the classifier.
+  m->act_format = ACT_RS;
+  bool all_rs = opt_path == AIQ_PATH_AUTO || opt_path == AIQ_PATH_TENSOR;
+  for (const LayerInfo& li : m->layers) {
+    if (!all_rs || li.d.kind == AIQ_LAYER_FC) continue;
+    if (li.d.input < 0)
+      all_rs = li.d.kind == AIQ_LAYER_CONV && li.d.ksize == 3 && li.d.pad == 1 && li.d.cin <= 4 && li.d.stride <= 2 &&
+               (li.d.cout == 16 || li.d.cout == 32 || li.d.cout == 64) && li.Wo % 8 == 0 && li.Wo <= 64;
+    else
+      all_rs = layer_tensor_kind(m, li) == 3;
+  }
+  if (!all_rs) {
+    m->act_format = ACT_SPLIT;                    // tentatively, to ask which layers would qualify
+    bool any_tc = false;
+    for (const LayerInfo& li : m->layers) any_tc = any_tc || layer_on_tensor_cores(m, li);
+    m->act_format = (opt_path == AIQ_PATH_TENSOR || opt_path == AIQ_PATH_TENSOR_TILES || (opt_path == AIQ_PATH_AUTO && any_tc))
+                        ? ACT_SPLIT : ACT_F32;
+  }
+  if (m->act_format == ACT_RS)
+    for (LayerInfo& li : m->layers)
+      if (li.d.kind != AIQ_LAYER_FC) li.out_bytes = rs_image_bytes(li.Ho, li.Wo, li.d.cout);
   assign_slots(m);
   cudaStream_t stream = (cudaStream_t)stream_;
   uint8_t* base = static_cast<uint8_t*>(dev_mem);
@@ -462,7 +482,8 @@ static WsLayout ws_layout(const aiq_model* m, int B, int S) {
   const LayerInfo& fc = m->layers.back();
   w.pooled_off = take((size_t)S * B * fc.d.cin * 4);
   w.logits_off = take((size_t)S * B * fc.d.cout * 4);
-  for (size_t e : m->slot_bytes) w.slot_off.push_back(take((size_t)S * B * e));
+  const size_t Bslot = m->act_format == ACT_RS ? (size_t)rs_padded_batch(B) : (size_t)B;   // images a version occupies
+  for (size_t e : m->slot_bytes) w.slot_off.push_back(take((size_t)S * Bslot * e));
   w.total = off;
   return w;
 }
@@ -476,8 +497,8 @@ struct LayerPlan {
   int tc_kind = 0;                      // which tensor-core kernel (see layer_tensor_kind)
   double weight_bytes = 0.0;            // packed weights + scales + biases over all jobs
   double weight_bytes_tc = 0.0, weight_bytes_tc16 = 0.0, weight_bytes_tc32 = 0.0;
-  TensorMapBytes in_map;                // over the input slot (tensor-core layers)
-  TensorMapBytes out_map;               // over the output slot (pointwise tensor-core layers)
+  TensorMapBytes maps[2];               // [0] over the input slot (tensor-core layers); [1] over the output slot
+                                        // (pointwise layers) or the second input map (row-streaming layers)
   size_t job_first = 0;                 // index of the first job record of this layer
   // fc only
   int n_pool = 0;
@@ -511,7 +532,8 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
   std::vector<std::vector<int>> ver(n, std::vector<int>(S, 0));   // ver[l][s]
   auto slot_ptr = [&](int layer, int version) -> uint8_t* {
     const LayerInfo& li = m->layers[layer];
-    return ws + wl.slot_off[li.slot] + (size_t)version * B * li.out_bytes;
+    const size_t Bslot = m->act_format == ACT_RS ? (size_t)rs_padded_batch(B) : (size_t)B;
+    return ws + wl.slot_off[li.slot] + (size_t)version * Bslot * li.out_bytes;
   };
   for (int l : m->order) {
     const LayerInfo& li = m->layers[l];
@@ -542,12 +564,13 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
       // job order: versions the tensor-core kernel takes first, grouped by weight class
       // (4- / 8-bit codes, then 16-bit, then 32-bit where the kernel can hold their pieces)
       const bool tc_layer = layer_on_tensor_cores(m, li);
-      const bool tc_wide = tc_layer && layer_tensor_kind(m, li) == 1;
+      const int tkind = layer_tensor_kind(m, li);
+      const bool tc_wide = tc_layer && (tkind == 1 || tkind == 3);
       const ConvGeom g_cls = make_geom(m, li, B);
       auto job_class = [&](int bits) -> int {      // 0: codes, 1: 16-bit, 2: 32-bit on tensor cores; 3: float32 kernel
         if (tc_layer && bits <= 8) return 0;
-        if (tc_wide && bits == 16 && conv_tc_bits_ok(g_cls, 16)) return 1;
-        if (tc_wide && bits == 32 && conv_tc_bits_ok(g_cls, 32)) return 2;
+        if (tc_wide && bits == 16 && (tkind == 3 || conv_tc_bits_ok(g_cls, 16))) return 1;
+        if (tc_wide && bits == 32 && (tkind == 3 || conv_tc_bits_ok(g_cls, 32))) return 2;
         return 3;
       };
       std::vector<int> vorder;
@@ -557,12 +580,14 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
       if (tc_layer) {
         const LayerInfo& src = m->layers[li.d.input];
         lp.tc_kind = layer_tensor_kind(m, li);
-        aiq_status_t st = lp.tc_kind == 1
-            ? conv_tc_encode_map(make_geom(m, li, B), ws + wl.slot_off[src.slot], B, plan.lp[li.d.input].n_versions, &lp.in_map)
-            : conv_pw_tc_encode_map(make_geom(m, li, B), ws + wl.slot_off[src.slot], B, plan.lp[li.d.input].n_versions, &lp.in_map);
+        aiq_status_t st = lp.tc_kind == 3
+            ? conv_rs_encode_maps(make_geom(m, li, B), ws + wl.slot_off[src.slot], B, plan.lp[li.d.input].n_versions, &lp.maps[0])
+            : lp.tc_kind == 1
+            ? conv_tc_encode_map(make_geom(m, li, B), ws + wl.slot_off[src.slot], B, plan.lp[li.d.input].n_versions, &lp.maps[0])
+            : conv_pw_tc_encode_map(make_geom(m, li, B), ws + wl.slot_off[src.slot], B, plan.lp[li.d.input].n_versions, &lp.maps[0]);
         if (st != AIQ_OK) return st;
         if (lp.tc_kind == 2) {
-          st = conv_pw_tc_encode_out_map(make_geom(m, li, B), ws + wl.slot_off[li.slot], B, lp.n_versions, &lp.out_map);
+          st = conv_pw_tc_encode_out_map(make_geom(m, li, B), ws + wl.slot_off[li.slot], B, lp.n_versions, &lp.maps[1]);
           if (st != AIQ_OK) return st;
         }
       }
@@ -676,20 +701,25 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
       if (st != AIQ_OK) return st;
       continue;
     }
+    auto launch_wide = [&](const LayerJob* jd, int n, double wb, int wbits) -> aiq_status_t {
+      return lp.tc_kind == 3
+          ? launch_conv_rs(g, &lp.maps[0], jd, n, plan.batch_capacity, m->status_word, wb, wbits, stream)
+          : launch_conv_tc(g, &lp.maps[0], jd, n, plan.batch_capacity, m->status_word, wb, wbits, stream);
+    };
     if (lp.n_tc > 0) {
-      st = lp.tc_kind == 1
-          ? launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, 8, stream)
-          : launch_conv_pw_tc(g, &lp.in_map, &lp.out_map, jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream);
+      st = lp.tc_kind != 2
+          ? launch_wide(jobs_dev + lp.job_first, lp.n_tc, lp.weight_bytes_tc, 8)
+          : launch_conv_pw_tc(g, &lp.maps[0], &lp.maps[1], jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream);
       if (st != AIQ_OK) return st;
     }
     int done = lp.n_tc;
     if (lp.n_tc16 > 0) {
-      st = launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first + done, lp.n_tc16, plan.batch_capacity, m->status_word, lp.weight_bytes_tc16, 16, stream);
+      st = launch_wide(jobs_dev + lp.job_first + done, lp.n_tc16, lp.weight_bytes_tc16, 16);
       if (st != AIQ_OK) return st;
       done += lp.n_tc16;
     }
     if (lp.n_tc32 > 0) {
-      st = launch_conv_tc(g, &lp.in_map, jobs_dev + lp.job_first + done, lp.n_tc32, plan.batch_capacity, m->status_word, lp.weight_bytes_tc32, 32, stream);
+      st = launch_wide(jobs_dev + lp.job_first + done, lp.n_tc32, lp.weight_bytes_tc32, 32);
       if (st != AIQ_OK) return st;
       done += lp.n_tc32;
     }
@@ -714,7 +744,7 @@ extern "C" void aiq_set_eval_options(int chunk, int share_prefix) {
 }
 
 extern "C" void aiq_set_compute_path(int path) {
-  aiq::g_opt_path = (path == AIQ_PATH_FP32 || path == AIQ_PATH_TENSOR) ? path : AIQ_PATH_AUTO;
+  aiq::g_opt_path = (path == AIQ_PATH_FP32 || path == AIQ_PATH_TENSOR || path == AIQ_PATH_TENSOR_TILES) ? path : AIQ_PATH_AUTO;
 }
 
 extern "C" void aiq_last_call_stats(int64_t* kernel_launches, int64_t* layer_evals, int64_t* layer_evals_unshared) {

@@ -49,7 +49,8 @@ class compute_path:
 
     def __enter__(self):
         b = binding()
-        b.aiq_set_compute_path({"auto": b.PATH_AUTO, "fp32": b.PATH_FP32, "tensor": b.PATH_TENSOR}[self.name])
+        b.aiq_set_compute_path({"auto": b.PATH_AUTO, "fp32": b.PATH_FP32, "tensor": b.PATH_TENSOR,
+                                "tiles": b.PATH_TENSOR_TILES}[self.name])
         return self
 
     def __exit__(self, *exc):

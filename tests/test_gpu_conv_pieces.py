@@ -45,8 +45,9 @@ SHAPES = [(16, 16, 3, 1), (16, 32, 3, 2), (16, 32, 1, 2), (32, 32, 3, 1), (32, 6
           (64, 64, 3, 1), (64, 32, 3, 1), (64, 16, 1, 1)]
 
 
+@pytest.mark.parametrize("path", ["tensor", "tiles"])
 @pytest.mark.parametrize("cin,cout,k,stride", SHAPES)
-def test_both_weight_pieces_count(cin, cout, k, stride):
+def test_both_weight_pieces_count(cin, cout, k, stride, path):
     aiq = binding()
     arch = _net(cin, cout, k, stride)
     rng = np.random.default_rng(100 * cin + cout + k + stride)
@@ -61,7 +62,7 @@ def test_both_weight_pieces_count(cin, cout, k, stride):
         dict(W=np.eye(cout, dtype=np.float32), bias=np.zeros(cout, np.float32)),
     ]
     x = rng.integers(1, 4, (4, 3, 16, 16)).astype(np.float32)      # stem outputs: integers <= 81
-    with compute_path("tensor"):
+    with compute_path(path):      # "tensor": the row-streaming kernel; "tiles": the pixel-tile kernel
         model = aiq.Model(arch, params)
     bank = O.build_weight_bank(O.fold_model(arch, params), (16, 32))
     w32, b32 = bank[1][32]

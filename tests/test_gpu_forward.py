@@ -47,7 +47,7 @@ def test_tiny_net_random_schemes(batch, path):
         assert_logits_close(got, ref, f"tiny batch={batch} seed={seed}")
 
 
-@pytest.mark.parametrize("path", ["fp32", "tensor"])
+@pytest.mark.parametrize("path", ["fp32", "tensor", "tiles"])
 def test_resnet20_batch64_mixed_scheme(path):
     """ResNet-20, batch 64, one bit-width per layer drawn from {32, 16, 8, 4}."""
     aiq = binding()
@@ -152,7 +152,7 @@ def test_mobilenet_v2_imagenet_shape(path):
             assert_preds_match(O.predict(got), O.predict(ref), O.top2_margin(ref), "mbv2 imagenet")
 
 
-@pytest.mark.parametrize("path", ["fp32", "tensor"])
+@pytest.mark.parametrize("path", ["fp32", "tensor", "tiles"])
 def test_eval_schemes_greedy_step_resnet20(path):
     """One greedy step: 21 candidates, each lowering one conv layer of an all-8 scheme to 4
     bits.  Counts, predictions and accuracies against the oracle; sharing on/off and the
@@ -261,7 +261,7 @@ def test_eval_schemes_coordinate_step_mobilenet_v2_imagenet():
     assert np.allclose(ai, oai, rtol=1e-12)
 
 
-@pytest.mark.parametrize("path", ["fp32", "tensor"])
+@pytest.mark.parametrize("path", ["fp32", "tensor", "tiles"])
 @pytest.mark.parametrize("make", [heavy_early_resnet20, plain_convnet20])
 def test_structural_variants_of_section_4_5(make, path):
     """HeavyEarlyResNet20 (wide layers first, width changes at stride 1, 64 -> 32 -> 16 channels)
