@@ -33,11 +33,34 @@ namespace aiq {
 
 namespace {
 
-constexpr int kRsEpiWarps = 16;                        // four per quarter of the accumulator lanes
-constexpr int kRsThreads = (2 + kRsEpiWarps) * 32;     // + TMA producer + MMA issuer
+// Warps: TMA producer, MMA issuer, then the epilogue warps, four per quarter of the accumulator
+// lanes where one CTA has an SM to itself, two per quarter where two CTAs share it (then each
+// CTA's issuing warp hides the other's per-row bookkeeping, and each takes half of tensor memory).
+constexpr int kRsMaxEpiWarps = 16;
+constexpr int kRsMaxThreads = (2 + kRsMaxEpiWarps) * 32;
 constexpr int kRsMaxStages = 6;
 constexpr int kRsMaxSlots = 16;
 constexpr int kRsTileBytes = 2048;                     // 128 operand rows x 16 bytes of one plane
+constexpr int kRsMaxRows = 64;                         // input rows of a feature map
+constexpr int kRsRowWords = 20;                        // words of one row program (see RowProgram)
+
+// What the MMA warp does for one input row: the runs of accumulator slots it feeds.  All K steps
+// but the first add to every output row the input row touches: one MMA per run of consecutive
+// slots (`rest`, at most two: the ring of slots may wrap).  The first K step must overwrite the
+// rows that receive their first contribution: its runs are cut there as well (`head`, at most
+// three).  A run = (instruction descriptor with its N, accumulator column, weight row offset in
+// 16-byte units).  The slots do not depend on the item because the ring depth divides the rows
+// of an item.
+struct RowProgram {
+  uint32_t head_idesc[3], head_dcol[3], head_boff[3];
+  uint32_t rest_idesc[2], rest_dcol[2], rest_boff[2];
+  uint32_t head_acc;        // bit i: run i of head accumulates (else overwrites)
+  uint32_t n_runs;          // head runs | rest runs << 4
+  uint32_t fresh;           // first output row that must be free before the MMAs | count << 8
+  uint32_t done;            // output rows complete after this input row: (row A + 1) | (row B + 1) << 8; 0 = none
+  uint32_t pad;
+};
+static_assert(sizeof(RowProgram) == kRsRowWords * 4, "row program size");
 
 struct RsParams {
   int H, W, Ho, Wo;
@@ -53,6 +76,7 @@ struct RsParams {
   int a_tap_off[3];       // byte offset of horizontal tap t inside a stage (column tile 0, plane 0)
   int a_lbo;              // bytes from one plane (8 channels) to the next
   int xt;                 // column tiles (128 lanes each) per row
+  int tmem_cols;          // tensor-memory columns this CTA allocates (512, or 256 with two CTAs per SM)
   int32_t* error_flag;
 };
 
@@ -60,7 +84,7 @@ __host__ __device__ constexpr int rs_taps(int ks) { return ks == 3 ? 3 : 1; }
 
 // shared memory regions (base aligned to 1024 bytes)
 struct RsSmem {
-  int ring, weights, scale, bias, bars, total;
+  int ring, weights, scale, bias, rows, bars, total;
 };
 __host__ __device__ inline RsSmem rs_smem(int stages, int stage_bytes, int weight_bytes, int N) {
   RsSmem s;
@@ -68,13 +92,14 @@ __host__ __device__ inline RsSmem rs_smem(int stages, int stage_bytes, int weigh
   s.weights = stages * stage_bytes;
   s.scale = s.weights + weight_bytes;
   s.bias = s.scale + N * 4;
-  s.bars = (s.bias + N * 4 + 127) / 128 * 128;
+  s.rows = (s.bias + N * 4 + 127) / 128 * 128;          // per input row: the MMA program (kRsRowWords words)
+  s.bars = s.rows + kRsMaxRows * kRsRowWords * 4;
   s.total = s.bars + (2 * kRsMaxStages + 2 * kRsMaxSlots + 1) * 8 + 16;
   return s;
 }
 
 template <int C, int KS, int STRIDE, int PIECES>
-__global__ void __launch_bounds__(kRsThreads, 1)
+__global__ void __launch_bounds__(kRsMaxThreads, 1)
 conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1, RsParams p,
                const LayerJob* __restrict__ jobs) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -93,6 +118,7 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   uint8_t* wsm = smem + sm.weights;
   float* s_scale = reinterpret_cast<float*>(smem + sm.scale);
   float* s_bias = reinterpret_cast<float*>(smem + sm.bias);
+  RowProgram* s_rows = reinterpret_cast<RowProgram*>(smem + sm.rows);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
   const uint32_t bar_in_full = smem_u32(bars);
   const uint32_t bar_in_empty = bar_in_full + 8 * kRsMaxStages;
@@ -105,7 +131,8 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   // Epilogue work: per output row and quarter of the lanes, `units` = column tiles x 16-channel
   // chunks.  The WQ warps of a quarter either share the units of every row, or, where a row has
   // fewer units than that, take every (WQ / units)-th row each, so several rows are drained at once.
-  constexpr int WQ = kRsEpiWarps / 4;
+  const int n_threads = (int)blockDim.x;
+  const int WQ = (n_threads / 32 - 2) / 4;           // epilogue warps per quarter: 4 or 2
   const int units = p.xt * (N / 16);
   const int epi_sets = units < WQ ? units : WQ;      // warps of a quarter that read one row
 
@@ -125,7 +152,7 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   }
   __syncthreads();
   if (warp == 1) {
-    tmem_alloc(smem_u32(s_tmem), 512);
+    tmem_alloc(smem_u32(s_tmem), (uint32_t)p.tmem_cols);
     tmem_relinquish();
   }
   // packed weight rows of this slice: one bulk copy into the (still unused) ring, then expansion
@@ -137,14 +164,67 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     mbar_expect_tx(bar_w, packed_bytes);
     bulk_load(smem_u32(ring), job.w + (size_t)n_off * wrow_bytes, packed_bytes, bar_w);
   }
-  for (int i = tid; i < N; i += kRsThreads) {
+  for (int i = tid; i < N; i += n_threads) {
     s_scale[i] = job.scale[n_off + i];
     s_bias[i] = job.bias[n_off + i];
+  }
+  // row programs (one thread per input row)
+  if (tid < p.H) {
+    constexpr uint32_t IDESC0 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);   // f32 += bf16 x bf16, M = 128
+    const uint32_t n_field = ((uint32_t)N >> 3) << 17;                                     // N field of one output row
+    const int y = tid;
+    // output rows this input row contributes to: [yo, yo + n_rows), weight blocks [blk, ...); the
+    // rows from index `fresh` on receive their first contribution; rows done_a / done_b are complete
+    int yo, n_rows, blk, fresh, done_a = -1, done_b = -1;
+    if (KS == 1) { yo = y / STRIDE; n_rows = 1; blk = 0; fresh = 0; done_a = yo; }
+    else if (STRIDE == 1) {
+      yo = y > 0 ? y - 1 : 0;
+      const int hi = y + 1 < p.H ? y + 1 : p.H - 1;
+      n_rows = hi - yo + 1;
+      blk = yo - (y - 1);
+      fresh = y == 0 ? 0 : (y + 1 < p.H ? n_rows - 1 : n_rows);
+      if (y >= 1) done_a = y - 1;
+      if (y == p.H - 1) done_b = y;
+    } else if ((y & 1) == 0) { yo = y >> 1; n_rows = 1; blk = 0; fresh = y == 0 ? 0 : 1; }
+    else { yo = y >> 1; blk = 1; n_rows = (yo + 1 < p.Ho) ? 2 : 1; fresh = 1; done_a = yo; }
+    const int s0 = yo & (R - 1);
+    const int wrap = R - s0;                       // rows from this index on continue at slot 0
+    const int cw = (wrap > 0 && wrap < n_rows) ? wrap : n_rows;
+    const int cf = (fresh > 0 && fresh < n_rows) ? fresh : n_rows;
+    RowProgram rp = {};
+    auto set_run = [&](uint32_t* idesc, uint32_t* dcol, uint32_t* boff, int k, int i, int j) {
+      idesc[k] = IDESC0 | (uint32_t)(j - i) * n_field;
+      dcol[k] = (uint32_t)(((s0 + i) & (R - 1)) * N);
+      boff[k] = (uint32_t)((blk + i) * N);
+    };
+    int n_rest = 1;
+    set_run(rp.rest_idesc, rp.rest_dcol, rp.rest_boff, 0, 0, cw);
+    if (cw < n_rows) { set_run(rp.rest_idesc, rp.rest_dcol, rp.rest_boff, 1, cw, n_rows); n_rest = 2; }
+    const int c1 = cw < cf ? cw : cf;
+    int c2 = cw < cf ? cf : cw;
+    if (c2 == c1) c2 = n_rows;
+    int n_head = 1;
+    set_run(rp.head_idesc, rp.head_dcol, rp.head_boff, 0, 0, c1);
+    rp.head_acc = 0 >= fresh ? 0u : 1u;
+    if (c1 < n_rows) {
+      set_run(rp.head_idesc, rp.head_dcol, rp.head_boff, 1, c1, c2);
+      rp.head_acc |= (c1 >= fresh ? 0u : 1u) << 1;
+      n_head = 2;
+      if (c2 < n_rows) {
+        set_run(rp.head_idesc, rp.head_dcol, rp.head_boff, 2, c2, n_rows);
+        rp.head_acc |= (c2 >= fresh ? 0u : 1u) << 2;
+        n_head = 3;
+      }
+    }
+    rp.n_runs = (uint32_t)n_head | ((uint32_t)n_rest << 4);
+    rp.fresh = (uint32_t)(yo + fresh) | ((uint32_t)(n_rows - fresh) << 8);
+    rp.done = (uint32_t)(done_a + 1) | ((uint32_t)(done_b + 1) << 8);
+    s_rows[y] = rp;
   }
   bool alive = mbar_wait_warp(bar_w, 0, s_abort, p.error_flag);
   if (alive) {
     const int w_units = T * KCH * NB;
-    for (int u = tid; u < w_units; u += kRsThreads) {
+    for (int u = tid; u < w_units; u += n_threads) {
       const int row = u % NB;
       const int kc = (u / NB) % KCH;
       const int ti = u / (NB * KCH);
@@ -246,46 +326,24 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         const int q0 = item_local * p.Ho;
         for (int y = 0; y < p.H && alive; ++y) {
           if (!row_used(y)) continue;
-          // output rows this input row contributes to: [yo, yo + n_rows), weight blocks [blk, ...),
-          // the rows from index `fresh` on receive their first contribution (they overwrite)
-          int yo, n_rows, blk, fresh;
-          if (KS == 1) { yo = y / STRIDE; n_rows = 1; blk = 0; fresh = 0; }
-          else if (STRIDE == 1) {
-            yo = y > 0 ? y - 1 : 0;
-            const int hi = y + 1 < p.H ? y + 1 : p.H - 1;
-            n_rows = hi - yo + 1;
-            blk = yo - (y - 1);
-            fresh = y == 0 ? 0 : (y + 1 < p.H ? n_rows - 1 : n_rows);
-          } else if ((y & 1) == 0) { yo = y >> 1; n_rows = 1; blk = 0; fresh = y == 0 ? 0 : 1; }
-          else { yo = y >> 1; blk = 1; n_rows = (yo + 1 < p.Ho) ? 2 : 1; fresh = 1; }
-          for (int i = fresh; i < n_rows && alive; ++i) {
-            const int q = q0 + yo + i;
+          const RowProgram& rp = s_rows[y];
+          const uint4 w0 = *reinterpret_cast<const uint4*>(&rp.head_idesc[0]);   // head_idesc[0..2], head_dcol[0]
+          const uint4 w1 = *reinterpret_cast<const uint4*>(&rp.head_dcol[1]);    // head_dcol[1..2], head_boff[0..1]
+          const uint4 w2 = *reinterpret_cast<const uint4*>(&rp.head_boff[2]);    // head_boff[2], rest_idesc[0..1], rest_dcol[0]
+          const uint4 w3 = *reinterpret_cast<const uint4*>(&rp.rest_dcol[1]);    // rest_dcol[1], rest_boff[0..1], head_acc
+          const uint4 w4 = *reinterpret_cast<const uint4*>(&rp.n_runs);          // n_runs, fresh, done, pad
+          const uint32_t h0_idesc = w0.x, h1_idesc = w0.y, h2_idesc = w0.z, h0_dcol = w0.w;
+          const uint32_t h1_dcol = w1.x, h2_dcol = w1.y, h0_boff = w1.z, h1_boff = w1.w;
+          const uint32_t h2_boff = w2.x, r0_idesc = w2.y, r1_idesc = w2.z, r0_dcol = w2.w;
+          const uint32_t r1_dcol = w3.x, r0_boff = w3.y, r1_boff = w3.z, head_acc = w3.w;
+          const bool head1 = (w4.x & 15u) > 1u, head2 = (w4.x & 15u) > 2u, rest1 = (w4.x >> 4) > 1u;
+          const uint32_t h0_acc = head_acc & 1u, h1_acc = (head_acc >> 1) & 1u, h2_acc = (head_acc >> 2) & 1u;
+          const int fresh_row = (int)(w4.y & 255u), n_fresh = (int)(w4.y >> 8);
+          for (int i = 0; i < n_fresh && alive; ++i) {
+            const int q = q0 + fresh_row + i;
             alive = mbar_wait_warp(bar_out_empty + 8 * (q & (R - 1)), ((q / R) & 1) ^ 1u, s_abort, p.error_flag);
           }
           if (!alive) break;
-          // The rows' accumulator slots are consecutive except where the ring wraps.  All K steps but
-          // the first add to every row: one MMA per run of consecutive slots (`rest`, at most two).
-          // The first K step must overwrite the fresh rows: runs are cut at `fresh` as well (`head`,
-          // at most three).  A run = (N field, accumulator column, weight row offset).
-          const int s0 = (q0 + yo) & (R - 1);
-          const int wrap = R - s0;                     // rows from this index on continue at slot 0
-          const int cw = (wrap > 0 && wrap < n_rows) ? wrap : n_rows;     // cut at the wrap, if inside
-          const int cf = (fresh > 0 && fresh < n_rows) ? fresh : n_rows;  // cut at the first fresh row, if inside
-          auto run_idesc = [&](int i, int j) -> uint32_t { return IDESC0 | (uint32_t)(j - i) * n_field; };
-          auto run_dcol = [&](int i) -> uint32_t { return (uint32_t)(((s0 + i) & (R - 1)) * N); };
-          auto run_boff = [&](int i) -> uint32_t { return (uint32_t)((blk + i) * N); };
-          // rest: [0, cw) [cw, n_rows)
-          const bool rest1 = cw < n_rows;
-          const uint32_t r0_idesc = run_idesc(0, cw), r0_dcol = run_dcol(0), r0_boff = run_boff(0);
-          const uint32_t r1_idesc = run_idesc(cw, n_rows), r1_dcol = run_dcol(cw), r1_boff = run_boff(cw);
-          // head: [0, c1) [c1, c2) [c2, n_rows) with c1 <= c2 the cuts in order
-          const int c1 = cw < cf ? cw : cf;
-          int c2 = cw < cf ? cf : cw;
-          if (c2 == c1) c2 = n_rows;
-          const bool head1 = c1 < n_rows, head2 = c2 < n_rows;
-          const uint32_t h0_idesc = run_idesc(0, c1), h0_dcol = run_dcol(0), h0_boff = run_boff(0), h0_acc = 0 >= fresh ? 0u : 1u;
-          const uint32_t h1_idesc = run_idesc(c1, c2), h1_dcol = run_dcol(c1), h1_boff = run_boff(c1), h1_acc = c1 >= fresh ? 0u : 1u;
-          const uint32_t h2_idesc = run_idesc(c2, n_rows), h2_dcol = run_dcol(c2), h2_boff = run_boff(c2), h2_acc = c2 >= fresh ? 0u : 1u;
           alive = mbar_wait_warp(bar_in_full + 8 * stage, phase, s_abort, p.error_flag);
           if (!alive) break;
           tc_fence_after();
@@ -320,11 +378,8 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           umma_commit(bar_in_empty + 8 * stage);       // the stage is free once these MMAs retire
           if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
           // output rows that are complete with this input row
-          if (KS == 1) umma_commit(bar_out_full + 8 * ((q0 + yo) & (R - 1)));
-          else if (STRIDE == 1) {
-            if (y >= 1) umma_commit(bar_out_full + 8 * ((q0 + y - 1) & (R - 1)));
-            if (y == p.H - 1) umma_commit(bar_out_full + 8 * ((q0 + y) & (R - 1)));
-          } else if (y & 1) umma_commit(bar_out_full + 8 * ((q0 + yo) & (R - 1)));
+          if (w4.z & 255u) umma_commit(bar_out_full + 8 * (((w4.z & 255u) - 1u) & (uint32_t)(R - 1)));
+          if (w4.z >> 8) umma_commit(bar_out_full + 8 * (((w4.z >> 8) - 1u) & (uint32_t)(R - 1)));
         }
       }
     }
@@ -437,7 +492,7 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
   }
 }
 
@@ -468,7 +523,7 @@ bool rs_shape(const ConvGeom& g, RsShape* s) {
   if (g.stride != 1 && g.stride != 2) return false;
   if (g.Cin != 16 && g.Cin != 32 && g.Cin != 64) return false;
   if (g.Cout != 16 && g.Cout != 32 && g.Cout != 64) return false;
-  if (g.W % 8 != 0 || g.Wo % 8 != 0 || g.W > 64 || g.H < 2) return false;
+  if (g.W % 8 != 0 || g.Wo % 8 != 0 || g.W > 64 || g.H < 2 || g.H > kRsMaxRows || g.Ho % 4 != 0) return false;
   if (g.stride == 2 && ((g.H & 1) || (g.W & 1))) return false;
   s->Gin = rs_group_images(g.W);
   s->Gout = rs_group_images(g.Wo);
@@ -542,24 +597,45 @@ aiq_status_t launch_rs(const ConvGeom& g, const RsShape& sh, const CUtensorMap* 
   p.gmode = sh.gmode;
   p.n_items = rs_padded_batch(g.B) / sh.Gout;
   p.rows_per_version = rs_padded_batch(batch_capacity) / sh.Gin * g.H;
-  p.n_stages = stages;
+  // Two CTAs per SM where two rings of at least three input rows and two copies of the weights fit
+  // (the 16- and 32-channel layers), else one.
+  const int wbytes = rs_weight_bytes(g, weight_bits);
+  int occ = 1, st2 = 0;
+  {
+    const int per_cta = (props.smem_optin + 1024) / 2 - 1024;      // an SM holds the opt-in limit + 1 KB; each CTA reserves 1 KB
+    const int packed = N * (int)row_bytes(g.K, weight_bits <= 8 ? 8 : weight_bits);
+    for (int st = kRsMaxStages; st >= 3 && !st2; --st)
+      if (rs_smem(st, sh.stage_bytes, wbytes, N).total + 1024 <= per_cta && packed <= st * sh.stage_bytes) st2 = st;
+    if (st2) occ = 2;
+  }
+  const int stages_used = occ == 2 ? st2 : stages;
+  p.n_stages = stages_used;
+  p.tmem_cols = 512 / occ;
+  // output rows in flight: a power of two that divides the rows of an item (the slot of a row then
+  // does not depend on the item) and fits the CTA's share of tensor memory
   int slots = kRsMaxSlots;
-  while (slots > 4 && sh.xt * slots * N > 512) slots >>= 1;
-  if (sh.xt * slots * N > 512) return set_error(AIQ_ERR_SHAPE, "conv_rs: %d column tiles of %d channels exceed tensor memory", sh.xt, N);
+  while (slots > 4 && (sh.xt * slots * N > p.tmem_cols || g.Ho % slots != 0)) slots >>= 1;
+  if (sh.xt * slots * N > p.tmem_cols && occ == 2) {             // too wide for half of tensor memory: one CTA per SM
+    occ = 1; p.n_stages = stages; p.tmem_cols = 512;
+    slots = kRsMaxSlots;
+    while (slots > 4 && (sh.xt * slots * N > 512 || g.Ho % slots != 0)) slots >>= 1;
+  }
+  if (sh.xt * slots * N > p.tmem_cols) return set_error(AIQ_ERR_SHAPE, "conv_rs: %d column tiles of %d channels exceed tensor memory", sh.xt, N);
   p.n_slots = slots;
   p.K = g.K; p.stage_bytes = sh.stage_bytes; p.a_lbo = sh.a_lbo; p.xt = sh.xt;
   for (int t = 0; t < 3; ++t) p.a_tap_off[t] = sh.a_tap_off[t];
   p.error_flag = error_flag;
-  const int smem_bytes = rs_smem(stages, sh.stage_bytes, rs_weight_bytes(g, weight_bits), N).total + 1024;
+  const int smem_bytes = rs_smem(p.n_stages, sh.stage_bytes, wbytes, N).total + 1024;
+  const int threads = (2 + (occ == 2 ? 8 : kRsMaxEpiWarps)) * 32;
   AIQ_ENSURE_DYNAMIC_SMEM((conv_rs_kernel<C, KS, STRIDE, PIECES>), props.smem_optin);
-  int ctas = props.n_sms / (n_jobs * slices);
+  int ctas = occ * props.n_sms / (n_jobs * slices);
   if (ctas > p.n_items) ctas = p.n_items;
   if (ctas < 1) ctas = 1;
   {
     LaunchScope scope(AIQ_KERNEL_CONV_TC, s,
                       2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
                       weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W + (double)g.B * g.Ho * g.Wo * g.Cout));
-    conv_rs_kernel<C, KS, STRIDE, PIECES><<<dim3(ctas, n_jobs, slices), kRsThreads, smem_bytes, s>>>(maps[0], maps[1], p, jobs_dev);
+    conv_rs_kernel<C, KS, STRIDE, PIECES><<<dim3(ctas, n_jobs, slices), threads, smem_bytes, s>>>(maps[0], maps[1], p, jobs_dev);
   }
   AIQ_LAUNCH_CHECK("conv_rs");
   return AIQ_OK;
