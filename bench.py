@@ -33,12 +33,38 @@ SEED_MODEL, SEED_IMAGES = 1234, 5679
 WORKLOAD = "resnet20_cifar_greedy_step: 21 schemes (all-8, one conv layer -> 4 bits) x 10000 images"
 METRIC = "scheme evals/sec (ResNet-20, 10k imgs)"
 UNIT = "scheme-evals/s"
+# images per evaluator pass of the headline workload: two passes over the 10,000 images (a pass
+# costs ~26 launches with their set-up; fewer, larger passes amortise it)
+DEFAULT_CHUNK = 5008
+
+
+def eval_workload(name):
+    """The two scheme-sweep workloads: what is evaluated, on what, and how the oracle samples it."""
+    from aiq_workloads import (resnet20, mobilenet_v2, one_layer_lowered_schemes, coordinate_step_schemes,
+                               conv_layer_indices)
+    if name == "resnet20_step":
+        arch = resnet20()
+        return dict(arch=arch, seed_model=SEED_MODEL, seed_images=SEED_IMAGES, n_images=N_IMAGES, image=(3, 32, 32),
+                    schemes=one_layer_lowered_schemes(len(arch["layers"]), conv_layer_indices(arch)),
+                    chunk=DEFAULT_CHUNK, workload=WORKLOAD, metric=METRIC, oracle_images=128, ref_images=16,
+                    tc_kernel="conv_rs_kernel (tcgen05 bf16, fp32 accumulate, row-streaming)")
+    if name == "mbv2_imagenet_cd_step":
+        # one coordinate-descent sweep slice (Section 2.2): 52 candidates, each moving one conv layer of
+        # an all-8 scheme to 32, 16 or 4 bits, on 2,048 ImageNet-shaped images
+        arch = mobilenet_v2("imagenet")
+        return dict(arch=arch, seed_model=4234, seed_images=4237, n_images=2048, image=(3, 224, 224),
+                    schemes=coordinate_step_schemes(len(arch["layers"]), conv_layer_indices(arch)),
+                    chunk=32, workload="mobilenet_v2_imagenet_coordinate_step: 52 schemes (all-8, one conv layer -> "
+                                       "32 / 16 / 4 bits) x 2048 images of 3x224x224",
+                    metric="scheme evals/sec (MobileNetV2-ImageNet, 2048 imgs)", oracle_images=2, ref_images=1,
+                    tc_kernel="conv_pw_tc_kernel / conv_tc_kernel (tcgen05 bf16, fp32 accumulate)")
+    raise ValueError(name)
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from one ncu
-# capture (None until captured / after the kernel changed).
-# conv_tc_kernel: ncu DRAM byte count of 197.9 MB per launch at chunk 256, scaled by 4 to the
-# default chunk of 1024 images (traffic grows with the images of a launch)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 197.9e6
+# capture, per image of the evaluator pass (traffic grows in proportion to the images of a launch;
+# the capture runs a smaller pass than the benchmark).  None until captured / after the kernel changed.
+NCU_TRAFFIC_BYTES_PER_LAUNCH_PER_IMAGE = None
+NCU_TRAFFIC_NOTE = None
 
 
 def measured_peaks():
@@ -107,9 +133,9 @@ class ClockSampler:
                     samples=len(sm))
 
 
-def oracle_sample_rate(n_sample_images, schemes, arch, params, x):
+def oracle_sample_rate(n_sample_images, schemes, arch, params, x, n_images=N_IMAGES):
     """Times the CPU oracle, as it stands, on `n_sample_images` images x all schemes and
-    scales linearly to the 10,000-image set.  Returns (scheme-evals/s, seconds, threads)."""
+    scales linearly to the `n_images`-image set.  Returns (scheme-evals/s, seconds, threads)."""
     from oracle import aiq_oracle as O
     threads = os.cpu_count() or 1
     try:
@@ -121,14 +147,14 @@ def oracle_sample_rate(n_sample_images, schemes, arch, params, x):
         pass
     t0 = time.perf_counter()
     folded = O.fold_model(arch, params)
-    bank = O.build_weight_bank(folded, bits_set=(4, 8))
+    bank = O.build_weight_bank(folded, bits_set=tuple(sorted({int(b) for b in np.unique(schemes)} | {8})))
     xs = x[:n_sample_images]
     labels = O.predict(O.forward_scheme(arch, bank, [8] * len(arch["layers"]), xs))
     O.eval_schemes(arch, bank, schemes, xs, labels)
     for s in schemes:
         O.scheme_ai(arch, s)
     dt = time.perf_counter() - t0
-    evals_per_s = len(schemes) / (dt * (N_IMAGES / float(n_sample_images)))
+    evals_per_s = len(schemes) / (dt * (n_images / float(n_sample_images)))
     return evals_per_s, dt, threads
 
 
@@ -136,29 +162,150 @@ def run_reference(args, rank, world):
     """--impl reference: the CPU oracle on the host cores, rank 0 only."""
     if rank != 0:
         return
-    from aiq_workloads import resnet20, gen_model, gen_images, one_layer_lowered_schemes, conv_layer_indices
-    arch = resnet20()
-    params = gen_model(arch, SEED_MODEL)
-    schemes = one_layer_lowered_schemes(len(arch["layers"]), conv_layer_indices(arch))
-    n_sample = 16
-    x = gen_images(n_sample, 3, 32, 32, SEED_IMAGES)
+    from aiq_workloads import gen_model, gen_images
+    wl = eval_workload(args.workload if args.workload == "mbv2_imagenet_cd_step" else "resnet20_step")
+    arch, schemes, n_images = wl["arch"], wl["schemes"], wl["n_images"]
+    params = gen_model(arch, wl["seed_model"])
+    n_sample = wl["ref_images"]
+    x = gen_images(n_sample, *wl["image"], wl["seed_images"])
     for _ in range(args.warmup):
-        oracle_sample_rate(4, schemes, arch, params, x)
+        oracle_sample_rate(min(4, n_sample), schemes[:2], arch, params, x, n_images)
     secs, threads = 0.0, 1
     for _ in range(args.steps):
-        _, dt, threads = oracle_sample_rate(n_sample, schemes, arch, params, x)
+        _, dt, threads = oracle_sample_rate(n_sample, schemes, arch, params, x, n_images)
         secs += dt
-    value = len(schemes) * args.steps / (secs * (N_IMAGES / float(n_sample)))
-    sample = (f"each step: all 21 schemes on the first {n_sample} of the 10000 images (fold, bank, "
-              f"labels, forward, count, AI), scaled linearly by 10000/{n_sample}")
-    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
-                warmup=args.warmup, ms_per_step=1000.0 * secs / args.steps * (N_IMAGES / float(n_sample)),
+    value = len(schemes) * args.steps / (secs * (n_images / float(n_sample)))
+    sample = (f"each step: all {len(schemes)} schemes on the first {n_sample} of the {n_images} images (fold, bank, "
+              f"labels, forward, count, AI), scaled linearly by {n_images}/{n_sample}")
+    line = dict(impl="reference", metric=wl["metric"], value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=1000.0 * secs / args.steps * (n_images / float(n_sample)),
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                config=dict(workload=WORKLOAD, note="CPU oracle (NumPy float64), extrapolated from a sample"),
+                config=dict(workload=wl["workload"], note="CPU oracle (NumPy float64), extrapolated from a sample"),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=threads, kind="oracle", sample=sample),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
                 gpu_launches=0)
     print(json.dumps(line), flush=True)
+
+
+def time_launches(torch, fn, n):
+    """ms per launch of fn(i), i = 0..n-1, replayed from a CUDA graph so that host launch
+    overhead (about 10 us per call through ctypes) does not mask microsecond kernels."""
+    for i in range(min(n, 4)):
+        fn(i)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(n):
+            fn(i)
+    graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / n          # ms per launch
+
+
+L2_ROTATE = 300e6       # operands rotate over copies totalling more than twice the L2 capacity
+
+
+def measure_qlinear(aiq, torch, peaks, dev, N, K, bits_list, M_list, reps=20):
+    """Standalone quantized linear layer against the HBM roofline (weights rotate through HBM)."""
+    from aiq_workloads import gen_linear_case
+    wh, _ = gen_linear_case(N, K, 1, 3234)
+    w = torch.from_numpy(wh).to(dev)
+    out = []
+    for bits in bits_list:
+        rb = aiq.aiq_packed_row_bytes(K, bits)
+        packed0 = torch.empty((N, rb), dtype=torch.uint8, device=dev)
+        scales = torch.empty(N, dtype=torch.float32, device=dev)
+        aiq.aiq_quantize_layer(w, bits, packed0, scales)
+        copies = max(2, int(np.ceil(L2_ROTATE / (N * rb))))
+        packs = [packed0] + [packed0.clone() for _ in range(copies - 1)]
+        for M in M_list:
+            x = torch.randn((M, K), device=dev)
+            y = torch.empty((M, N), device=dev)
+            nbytes = N * rb + 4 * N + 4 * M * (K + N)
+            flops = 2.0 * M * N * K
+            n = reps * copies if M <= 16 else max(copies, 8)
+            wsb = aiq.aiq_qlinear_workspace_bytes(N, K, bits, M)
+            wsp = torch.empty(wsb, dtype=torch.uint8, device=dev) if wsb else None
+            ms = time_launches(torch, lambda i: aiq.aiq_qlinear(packs[i % copies], scales, None, N, K, bits, x, y,
+                                                                workspace=wsp), n)
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            out.append(dict(workload="qlinear", N=N, K=K, bits=bits, M=M, us=ms * 1e3,
+                            algorithmic_bytes=nbytes, GBps=gbs, frac_of_measured_hbm=gbs / peaks["hbm_gbs"],
+                            frac_of_8TBps=gbs / 8000.0, TFLOPs=flops / (ms * 1e-3) / 1e12,
+                            l2="weights rotate over %d copies" % copies))
+    return out
+
+
+def measure_quantize(aiq, torch, peaks, dev, N, K, bits_list, reps=20):
+    """Quantize + pack kernel against the HBM roofline (the input rotates through HBM)."""
+    w = torch.randn((N, K), device=dev) * 0.02
+    copies = max(2, int(np.ceil(L2_ROTATE / (N * K * 4))))
+    ws = [w] + [w.clone() for _ in range(copies - 1)]
+    out = []
+    for bits in bits_list:
+        rb = aiq.aiq_packed_row_bytes(K, bits)
+        packed = torch.empty((N, rb), dtype=torch.uint8, device=dev)
+        scales = torch.empty(N, dtype=torch.float32, device=dev)
+        nbytes = N * K * 4 + N * rb + N * 4
+        ms = time_launches(torch, lambda i: aiq.aiq_quantize_layer(ws[i % copies], bits, packed, scales), reps * copies)
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out.append(dict(workload="quantize", N=N, K=K, bits=bits, us=ms * 1e3, algorithmic_bytes=nbytes,
+                        GBps=gbs, frac_of_measured_hbm=gbs / peaks["hbm_gbs"], frac_of_8TBps=gbs / 8000.0,
+                        l2="input rotates over %d copies" % copies))
+    return out
+
+
+def measure_mobilenet_layers(aiq, torch, peaks, dev, batch=256):
+    """Depthwise and pointwise layers of MobileNetV2-CIFAR at `batch` (10 conv layers at 4 bits, the
+    rest at 8): summed kernel time per kind from the library's per-launch events, against the
+    algorithmic activation + weight bytes of those launches."""
+    from aiq_workloads import mobilenet_v2, gen_model, mixed_int4_int8_scheme, conv_layer_indices
+    arch = mobilenet_v2("cifar")
+    model = aiq.Model(arch, gen_model(arch, 2234), device=dev)
+    scheme = mixed_int4_int8_scheme(len(arch["layers"]), conv_layer_indices(arch), 10, 43)
+    xb = torch.randn((batch, 3, 32, 32), device=dev)
+    logits = torch.empty((batch, model.n_classes), device=dev)
+    wsb = torch.empty(model.aiq_workspace_bytes(batch, 1), dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        model.aiq_forward(scheme, xb, logits=logits, workspace=wsb)
+    torch.cuda.synchronize()
+    agg = {}
+    reps = 5
+    for _ in range(reps):
+        aiq.aiq_profile_start()
+        model.aiq_forward(scheme, xb, logits=logits, workspace=wsb)
+        for k, v in aiq.aiq_profile_stop().items():
+            a = agg.setdefault(k, dict(launches=0, ms=0.0, bytes=0.0, flops=0.0))
+            for f in a:
+                a[f] += v[f]
+    model.close()
+    out = []
+    for kind, label in (("depthwise", "depthwise 3x3 layers (17)"), ("conv_tc", "pointwise 1x1 layers on tcgen05 (34)")):
+        a = agg.get(kind)
+        if not a or not a["launches"]:
+            continue
+        gbs = a["bytes"] / (a["ms"] * 1e-3) / 1e9
+        out.append(dict(workload="mobilenet_v2_cifar_b%d" % batch, kernels=label, launches_per_forward=a["launches"] // reps,
+                        us=a["ms"] * 1e3 / reps, algorithmic_bytes=a["bytes"] / reps, GBps=gbs,
+                        frac_of_measured_hbm=gbs / peaks["hbm_gbs"], TFLOPs=a["flops"] / (a["ms"] * 1e-3) / 1e12))
+    return out
+
+
+def standalone_kernel_lines(aiq, torch, peaks, dev):
+    """The `kernels` key of the headline line: the memory-bound kernels outside the headline step."""
+    lines = measure_qlinear(aiq, torch, peaks, dev, 8192, 8192, (4, 8), (1, 4, 16, 256), reps=10)
+    lines += measure_quantize(aiq, torch, peaks, dev, 8192, 8192, (4, 8, 16, 32), reps=5)
+    lines += measure_mobilenet_layers(aiq, torch, peaks, dev)
+    for ln in lines:
+        for k, v in list(ln.items()):
+            if isinstance(v, float):
+                ln[k] = float("%.5g" % v)
+    return lines
 
 
 def run_kernel_sweep(args):
@@ -174,28 +321,6 @@ def run_kernel_sweep(args):
     peaks = measured_peaks()
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
-    L2_ROTATE = 300e6
-    reps = 20
-
-    def time_launches(fn, n):
-        """ms per launch of fn(i), i = 0..n-1, replayed from a CUDA graph so that host launch
-        overhead (about 10 us per call through ctypes) does not mask microsecond kernels."""
-        for i in range(min(n, 4)):
-            fn(i)
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            for i in range(n):
-                fn(i)
-        graph.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        graph.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / n          # ms per launch
-
     shapes = [(4096, 4096), (8192, 8192), (1280, 320)]
     if args.workload == "sensitivity":
         # the paper's single-layer study (Section 3, experiment 1; the 8b / 4b columns of Table 1):
@@ -291,45 +416,12 @@ def run_kernel_sweep(args):
         return
     if args.workload == "quantize":
         for (N, K) in shapes[:2]:
-            w = torch.randn((N, K), device=dev) * 0.02
-            for bits in (4, 8, 16, 32):
-                rb = aiq.aiq_packed_row_bytes(K, bits)
-                packed = torch.empty((N, rb), dtype=torch.uint8, device=dev)
-                scales = torch.empty(N, dtype=torch.float32, device=dev)
-                nbytes = N * K * 4 + N * rb + N * 4
-                copies = max(2, int(np.ceil(L2_ROTATE / (N * K * 4))))
-                ws = [w] + [w.clone() for _ in range(copies - 1)]
-                ms = time_launches(lambda i: aiq.aiq_quantize_layer(ws[i % copies], bits, packed, scales), reps * copies)
-                gbs = nbytes / (ms * 1e-3) / 1e9
-                print(json.dumps(dict(workload="quantize", N=N, K=K, bits=bits, us=ms * 1e3, algorithmic_bytes=nbytes,
-                                      GBps=gbs, frac_of_measured_hbm=gbs / peaks["hbm_gbs"], frac_of_8TBps=gbs / 8000.0,
-                                      l2="input rotates over %d copies" % copies)), flush=True)
+            for ln in measure_quantize(aiq, torch, peaks, dev, N, K, (4, 8, 16, 32)):
+                print(json.dumps(ln), flush=True)
         return
     for (N, K) in shapes:
-        wh, _ = gen_linear_case(N, K, 1, 3234)
-        w = torch.from_numpy(wh).to(dev)
-        for bits in (4, 8, 16, 32):
-            rb = aiq.aiq_packed_row_bytes(K, bits)
-            packed0 = torch.empty((N, rb), dtype=torch.uint8, device=dev)
-            scales = torch.empty(N, dtype=torch.float32, device=dev)
-            aiq.aiq_quantize_layer(w, bits, packed0, scales)
-            copies = max(2, int(np.ceil(L2_ROTATE / (N * rb))))
-            packs = [packed0] + [packed0.clone() for _ in range(copies - 1)]
-            for M in (1, 4, 16, 256):
-                x = torch.randn((M, K), device=dev)
-                y = torch.empty((M, N), device=dev)
-                nbytes = N * rb + 4 * N + 4 * M * (K + N)
-                flops = 2.0 * M * N * K
-                n = reps * copies if M <= 16 else max(copies, 8)
-                wsb = aiq.aiq_qlinear_workspace_bytes(N, K, bits, M)
-                wsp = torch.empty(wsb, dtype=torch.uint8, device=dev) if wsb else None
-                ms = time_launches(lambda i: aiq.aiq_qlinear(packs[i % copies], scales, None, N, K, bits, x, y,
-                                                             workspace=wsp), n)
-                gbs = nbytes / (ms * 1e-3) / 1e9
-                print(json.dumps(dict(workload="qlinear", N=N, K=K, bits=bits, M=M, us=ms * 1e3,
-                                      algorithmic_bytes=nbytes, GBps=gbs, frac_of_measured_hbm=gbs / peaks["hbm_gbs"],
-                                      frac_of_8TBps=gbs / 8000.0, TFLOPs=flops / (ms * 1e-3) / 1e12,
-                                      l2="weights rotate over %d copies" % copies)), flush=True)
+        for ln in measure_qlinear(aiq, torch, peaks, dev, N, K, (4, 8, 16, 32), (1, 4, 16, 256)):
+            print(json.dumps(ln), flush=True)
 
 
 def main():
@@ -340,8 +432,11 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--chunk", type=int, default=0, help="images per evaluator pass (0 = library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="resnet20_step", choices=["resnet20_step", "qlinear", "quantize", "forward", "search", "sensitivity"],
-                    help="resnet20_step: the headline line (default).  qlinear / quantize: per-case lines for the "
+    ap.add_argument("--no-kernels", action="store_true", help="skip the standalone-kernel measurements of the headline line")
+    ap.add_argument("--workload", default="resnet20_step", choices=["resnet20_step", "mbv2_imagenet_cd_step", "qlinear", "quantize", "forward", "search", "sensitivity"],
+                    help="resnet20_step: the headline line (default).  mbv2_imagenet_cd_step: the coordinate-descent "
+                         "sweep slice on ImageNet-shaped MobileNetV2 (52 candidates x 2,048 images), same line format.  "
+                         "qlinear / quantize: per-case lines for the "
                          "standalone memory-bound kernels; forward: one scheme, one batch; search: the two searches "
                          "of Section 2.2 on ResNet-20; sensitivity: every layer alone at 8 / 4 bits from an FP32 "
                          "base (all 1 GPU)")
@@ -353,7 +448,7 @@ def main():
     if args.impl == "reference":
         run_reference(args, rank, world)
         return
-    if args.workload != "resnet20_step":
+    if args.workload not in ("resnet20_step", "mbv2_imagenet_cd_step"):
         if rank == 0:
             run_kernel_sweep(args)
         return
@@ -366,7 +461,7 @@ def main():
     build.build()
     from paper_2512_14090_b200 import binding as aiq          # fails loudly without libaiq.so
     from paper_2512_14090_b200.sharding import reduce_counts
-    from aiq_workloads import resnet20, gen_model, gen_images, one_layer_lowered_schemes, conv_layer_indices
+    from aiq_workloads import gen_model, gen_images
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -376,21 +471,21 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
 
-    arch = resnet20()
-    params = gen_model(arch, SEED_MODEL)
+    wl = eval_workload(args.workload)
+    arch, schemes, N_IMG = wl["arch"], wl["schemes"], wl["n_images"]
+    params = gen_model(arch, wl["seed_model"])
     L = len(arch["layers"])
-    schemes = one_layer_lowered_schemes(L, conv_layer_indices(arch))
     S = len(schemes)
-    x_host = torch.from_numpy(gen_images(N_IMAGES, 3, 32, 32, SEED_IMAGES + rank)).pin_memory()
+    x_host = torch.from_numpy(gen_images(N_IMG, *wl["image"], wl["seed_images"] + rank)).pin_memory()
     x_dev = x_host.to(dev)
     model = aiq.Model(arch, params, device=dev)
-    chunk = args.chunk if args.chunk > 0 else 1024
-    aiq.aiq_set_eval_options(args.chunk, True)
+    chunk = args.chunk if args.chunk > 0 else wl["chunk"]
+    aiq.aiq_set_eval_options(chunk, True)
     ws = torch.empty(model.aiq_workspace_bytes(chunk, S), dtype=torch.uint8, device=dev)
 
     # labels = arg-max of the FP32 model (the all-32 scheme), computed once by the library
-    preds32 = torch.empty((1, N_IMAGES), dtype=torch.int32, device=dev)
-    model.aiq_eval_schemes(np.full((1, L), 32, np.uint8), x_dev, torch.zeros(N_IMAGES, dtype=torch.int32, device=dev),
+    preds32 = torch.empty((1, N_IMG), dtype=torch.int32, device=dev)
+    model.aiq_eval_schemes(np.full((1, L), 32, np.uint8), x_dev, torch.zeros(N_IMG, dtype=torch.int32, device=dev),
                            preds=preds32, workspace=ws)
     labels_dev = preds32[0].contiguous()
     labels_host = labels_dev.cpu().pin_memory()
@@ -406,7 +501,7 @@ def main():
         launches[0] += aiq.aiq_last_call_stats()["kernel_launches"] + bank_launches
         ai = [m.aiq_scheme_ai(s)[0] for s in schemes]
         if world > 1:
-            counts, total, acc = reduce_counts(counts, N_IMAGES, device=dev)
+            counts, total, acc = reduce_counts(counts, N_IMG, device=dev)
         result.update(acc=np.asarray(acc, dtype=np.float64), ai=ai)
         m.close()
 
@@ -488,8 +583,11 @@ def main():
         tensor_frac = tensor_achieved / peaks["bf16_tflops_sustained"]
         hbm_achieved = p["bytes"] / t_s / 1e9
         hbm_frac = hbm_achieved / peaks["hbm_gbs"]
-        common = dict(traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH if chunk == 1024 else None,
-                      kernel="conv_tc_kernel (tcgen05 bf16, fp32 accumulate)",
+        traffic = None
+        if args.workload == "resnet20_step" and NCU_TRAFFIC_BYTES_PER_LAUNCH_PER_IMAGE is not None:
+            traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH_PER_IMAGE * min(chunk, N_IMG)
+        common = dict(traffic=traffic, traffic_note=NCU_TRAFFIC_NOTE if traffic is not None else None,
+                      kernel=wl["tc_kernel"],
                       launches=p["launches"], avg_launch_ms=avg_ms,
                       algorithmic_flops_per_launch=p["flops"] / max(p["launches"], 1),
                       algorithmic_bytes_per_launch=p["bytes"] / max(p["launches"], 1),
@@ -525,20 +623,29 @@ def main():
     # ---- CPU oracle beside it (rank 0, N = 1 only) ----------------------------------------
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_sample = 128
-        v, dt, threads = oracle_sample_rate(n_sample, schemes, arch, params, x_host[:n_sample].numpy())
+        n_sample = wl["oracle_images"]
+        v, dt, threads = oracle_sample_rate(n_sample, schemes, arch, params, x_host[:n_sample].numpy(), N_IMG)
         cpu_baseline = dict(value=v, unit=UNIT, cores=threads, kind="oracle", seconds=dt,
-                            sample=f"all 21 schemes on the first {n_sample} of the 10000 images (fold, bank, "
-                                   f"labels, forward, count, AI), scaled linearly by 10000/{n_sample}")
+                            sample=f"all {S} schemes on the first {n_sample} of the {N_IMG} images (fold, bank, "
+                                   f"labels, forward, count, AI), scaled linearly by {N_IMG}/{n_sample}")
+
+    # ---- the memory-bound kernels outside the headline step (rank 0, N = 1 only) ------------
+    kernels = None
+    if rank == 0 and world == 1 and not args.no_kernels and args.workload == "resnet20_step":
+        model.close()
+        del ws, x_dev_e2e
+        torch.cuda.empty_cache()
+        kernels = standalone_kernel_lines(aiq, torch, peaks, dev)
 
     if rank == 0:
-        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+        line = dict(metric=wl["metric"], value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                     ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype="bf16", data="synthetic",
-                    config=dict(workload=WORKLOAD, images_per_rank=N_IMAGES, schemes=S, layers=L,
-                                arithmetic="conv layers: bf16 tensor-core products of integer weight codes with "
-                                           "activations held as hi + lo bfloat16 pairs, float32 accumulation; stem, "
-                                           "pooling and classifier in float32",
+                    config=dict(workload=wl["workload"], images_per_rank=N_IMG, schemes=S, layers=L,
+                                arithmetic="dense conv layers: bf16 tensor-core products of weight codes (or of two "
+                                           "bfloat16 pieces of a 16-/32-bit weight) with activations held as hi + lo "
+                                           "bfloat16 pairs, float32 accumulation; stem, depthwise, pooling and "
+                                           "classifier in float32",
                                 chunk=chunk, l2="flushed between timed steps (256 MiB write)",
                                 step="fold + quantize bank (4/8/16/32 bits) + eval 21 schemes + AI",
                                 labels="arg-max of the all-32-bit scheme, computed by the library",
@@ -546,8 +653,8 @@ def main():
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                              ms_per_step=e2e_ms / args.steps),
                     gpu_launches=gpu_launches, clocks=clocks, roofline=roofline, cpu_baseline=cpu_baseline,
-                    kernel_time_share=kernel_share,
-                    images_per_s=world * S * N_IMAGES * args.steps / (total_ms / 1000.0),
+                    kernel_time_share=kernel_share, kernels=kernels,
+                    images_per_s=world * S * N_IMG * args.steps / (total_ms / 1000.0),
                     acc_min=float(result["acc"].min()), acc_max=float(result["acc"].max()),
                     ai_min=float(min(result["ai"])), ai_max=float(max(result["ai"])))
         print(json.dumps(line), flush=True)

@@ -261,6 +261,44 @@ def test_eval_schemes_coordinate_step_mobilenet_v2_imagenet():
     assert np.allclose(ai, oai, rtol=1e-12)
 
 
+def test_coordinate_step_all_52_candidates_mobilenet_v2_imagenet():
+    """The benchmark's second sweep workload at reduced image count: all 52 candidates of the
+    coordinate-descent slice on 3 images against the oracle, and the base (all-8) scheme on 24
+    images in the benchmark's pass size with 6 of them checked by the oracle."""
+    import torch
+    from bench import eval_workload
+    aiq = binding()
+    wl = eval_workload("mbv2_imagenet_cd_step")
+    arch, schemes = wl["arch"], wl["schemes"]
+    assert schemes.shape == (52, 53)
+    x = gen_images(24, 3, 224, 224, 4240)
+    sample = np.arange(0, 24, 4)
+    params = balance_classifier(arch, gen_model(arch, wl["seed_model"]), x[sample])
+    model = aiq.Model(arch, params)
+    folded, bank = _oracle_bank(arch, params, (4, 8, 16, 32))
+    labels = np.zeros(24, np.int32)
+    labels[sample] = O.predict(O.forward_fp32_unquantized(arch, folded, x[sample]))
+    # (a) every candidate on three images
+    sub = sample[:3]
+    oacc, ocounts, opreds, omargins = O.eval_schemes(arch, bank, schemes, x[sub], labels[sub])
+    preds = torch.full((52, 3), -1, dtype=torch.int32, device="cuda")
+    aiq.aiq_set_eval_options(wl["chunk"], True)
+    acc, counts = model.aiq_eval_schemes(schemes, to_dev(x[sub]), to_dev(labels[sub]), preds=preds, chunk=wl["chunk"])
+    p = preds.cpu().numpy()
+    assert_preds_match(p, opreds, omargins, "coordinate step, all candidates")
+    assert np.all(np.abs(counts - ocounts) <= (omargins <= 1e-2).sum(axis=1))
+    # (b) the base scheme over the larger set, sampled
+    base = np.full((1, 53), 8, np.uint8)
+    preds = torch.full((1, 24), -1, dtype=torch.int32, device="cuda")
+    acc, counts = model.aiq_eval_schemes(base, to_dev(x), to_dev(labels), preds=preds, chunk=wl["chunk"])
+    aiq.aiq_set_eval_options(0, True)
+    p = preds.cpu().numpy()
+    assert np.array_equal((p == labels[None, :]).sum(axis=1), counts)
+    oacc, ocounts, opreds, omargins = O.eval_schemes(arch, bank, base, x[sample], labels[sample])
+    assert_preds_match(p[:, sample], opreds, omargins, "coordinate step, base scheme")
+    model.close()
+
+
 @pytest.mark.parametrize("path", ["fp32", "tensor", "tiles"])
 @pytest.mark.parametrize("make", [heavy_early_resnet20, plain_convnet20])
 def test_structural_variants_of_section_4_5(make, path):
@@ -323,8 +361,8 @@ def test_forward_and_eval_errors():
 
 
 def test_full_size_greedy_step_sampled_against_oracle():
-    """The benchmark's configuration: 10,000 images, 21 candidate schemes, chunks of 1024,
-    tensor-core path.  The oracle cannot run 210,000 forwards, so predictions are compared on
+    """The benchmark's configuration: 10,000 images, 21 candidate schemes, the benchmark's pass
+    size, tensor-core path.  The oracle cannot run 210,000 forwards, so predictions are compared on
     a sample of images it computes one by one; over the whole set the counts must equal the
     number of predictions that match the labels."""
     import torch
@@ -341,8 +379,10 @@ def test_full_size_greedy_step_sampled_against_oracle():
     labels[sample] = O.predict(O.forward_fp32_unquantized(arch, folded, x[sample]))
     oacc, ocounts, opreds, omargins = O.eval_schemes(arch, bank, schemes, x[sample], labels[sample])
     preds = torch.full((21, n), -1, dtype=torch.int32, device="cuda")
+    from bench import DEFAULT_CHUNK
+    aiq.aiq_set_eval_options(DEFAULT_CHUNK, True)
+    acc, counts = model.aiq_eval_schemes(schemes, to_dev(x), to_dev(labels), preds=preds, chunk=DEFAULT_CHUNK)
     aiq.aiq_set_eval_options(0, True)
-    acc, counts = model.aiq_eval_schemes(schemes, to_dev(x), to_dev(labels), preds=preds)
     p = preds.cpu().numpy()
     assert p.min() >= 0 and p.max() <= 9
     assert np.array_equal((p == labels[None, :]).sum(axis=1), counts)
