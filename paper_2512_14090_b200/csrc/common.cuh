@@ -135,6 +135,13 @@ struct LayerJob {
   int32_t label_slot;   // head jobs: index of the count / prediction row
   int32_t in_version;   // index of `in` along the version dimension of its slot
   int32_t out_version;  // index of `out` along the version dimension of its slot
+  // fused basic block (conv_rs_block_kernel): the block's first convolution; `in` / `in_version` are
+  // then that convolution's input, which is also the shortcut
+  const uint8_t* w_pre;
+  const float* scale_pre;
+  const float* bias_pre;
+  int32_t bits_pre;
+  int32_t reserved;
 };
 
 struct ConvGeom {
@@ -187,6 +194,11 @@ aiq_status_t conv_rs_encode_maps(const ConvGeom& g, const void* slot_base, int b
                                  void* maps_out);
 aiq_status_t launch_conv_rs(const ConvGeom& g, const void* maps, const LayerJob* jobs_dev, int n_jobs, int batch_capacity,
                             int32_t* error_flag, double weight_bytes, int weight_bits, cudaStream_t s);
+// A whole identity-shortcut basic block (two 3x3 convolutions of C -> C channels) in one kernel; `g`
+// describes either convolution.  Jobs carry both weight sets (LayerJob::w_pre ...).
+bool conv_rs_block_eligible(const ConvGeom& g);
+aiq_status_t launch_conv_rs_block(const ConvGeom& g, const void* maps, const LayerJob* jobs_dev, int n_jobs, int batch_capacity,
+                                  int32_t* error_flag, double weight_bytes, cudaStream_t s);
 // Pointwise (1x1, stride 1) tensor-core convolution for any channel count that is a multiple
 // of 8 (conv_pw_tc.cuh).  `map`: CUtensorMap over the input slot, dims (Cs, 2, pixels of all versions).
 bool conv_pw_tc_eligible(const ConvGeom& g);

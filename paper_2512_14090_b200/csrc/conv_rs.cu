@@ -98,6 +98,184 @@ __host__ __device__ inline RsSmem rs_smem(int stages, int stage_bytes, int weigh
   return s;
 }
 
+// Row program of input row y (see RowProgram).  R = accumulator slots per column tile.
+template <int KS, int STRIDE>
+__device__ __forceinline__ RowProgram rs_row_program(int y, int H, int Ho, int N, int R) {
+  constexpr uint32_t IDESC0 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);   // f32 += bf16 x bf16, M = 128
+  const uint32_t n_field = ((uint32_t)N >> 3) << 17;                                     // N field of one output row
+  // output rows this input row contributes to: [yo, yo + n_rows), weight blocks [blk, ...); the
+  // rows from index `fresh` on receive their first contribution; rows done_a / done_b are complete
+  int yo, n_rows, blk, fresh, done_a = -1, done_b = -1;
+  if (KS == 1) { yo = y / STRIDE; n_rows = 1; blk = 0; fresh = 0; done_a = yo; }
+  else if (STRIDE == 1) {
+    yo = y > 0 ? y - 1 : 0;
+    const int hi = y + 1 < H ? y + 1 : H - 1;
+    n_rows = hi - yo + 1;
+    blk = yo - (y - 1);
+    fresh = y == 0 ? 0 : (y + 1 < H ? n_rows - 1 : n_rows);
+    if (y >= 1) done_a = y - 1;
+    if (y == H - 1) done_b = y;
+  } else if ((y & 1) == 0) { yo = y >> 1; n_rows = 1; blk = 0; fresh = y == 0 ? 0 : 1; }
+  else { yo = y >> 1; blk = 1; n_rows = (yo + 1 < Ho) ? 2 : 1; fresh = 1; done_a = yo; }
+  const int s0 = yo & (R - 1);
+  const int wrap = R - s0;                       // rows from this index on continue at slot 0
+  const int cw = (wrap > 0 && wrap < n_rows) ? wrap : n_rows;
+  const int cf = (fresh > 0 && fresh < n_rows) ? fresh : n_rows;
+  RowProgram rp = {};
+  auto set_run = [&](uint32_t* idesc, uint32_t* dcol, uint32_t* boff, int k, int i, int j) {
+    idesc[k] = IDESC0 | (uint32_t)(j - i) * n_field;
+    dcol[k] = (uint32_t)(((s0 + i) & (R - 1)) * N);
+    boff[k] = (uint32_t)((blk + i) * N);
+  };
+  int n_rest = 1;
+  set_run(rp.rest_idesc, rp.rest_dcol, rp.rest_boff, 0, 0, cw);
+  if (cw < n_rows) { set_run(rp.rest_idesc, rp.rest_dcol, rp.rest_boff, 1, cw, n_rows); n_rest = 2; }
+  const int c1 = cw < cf ? cw : cf;
+  int c2 = cw < cf ? cf : cw;
+  if (c2 == c1) c2 = n_rows;
+  int n_head = 1;
+  set_run(rp.head_idesc, rp.head_dcol, rp.head_boff, 0, 0, c1);
+  rp.head_acc = 0 >= fresh ? 0u : 1u;
+  if (c1 < n_rows) {
+    set_run(rp.head_idesc, rp.head_dcol, rp.head_boff, 1, c1, c2);
+    rp.head_acc |= (c1 >= fresh ? 0u : 1u) << 1;
+    n_head = 2;
+    if (c2 < n_rows) {
+      set_run(rp.head_idesc, rp.head_dcol, rp.head_boff, 2, c2, n_rows);
+      rp.head_acc |= (c2 >= fresh ? 0u : 1u) << 2;
+      n_head = 3;
+    }
+  }
+  rp.n_runs = (uint32_t)n_head | ((uint32_t)n_rest << 4);
+  rp.fresh = (uint32_t)(yo + fresh) | ((uint32_t)(n_rows - fresh) << 8);
+  rp.done = (uint32_t)(done_a + 1) | ((uint32_t)(done_b + 1) << 8);
+  return rp;
+}
+
+// Packed weight rows (staged in shared memory at `staged`, `wrow_bytes` apart, N rows) -> bfloat16
+// operand tiles at `wsm`: [piece][tap][8-channel chunk][vertical tap block, channel][8 channels].
+template <int C, int KS, int STRIDE, int PIECES>
+__device__ __forceinline__ void rs_expand_weights(const uint8_t* staged, uint32_t wrow_bytes, int bits, int N, uint8_t* wsm,
+                                                  int tid, int n_threads) {
+  constexpr int T = rs_taps(KS), NBLK = KS == 3 ? 3 : 1, KCH = C / 8;
+  const int NB = NBLK * N;
+  const int tile_b = KCH * NB * 16;
+  const int w_units = T * KCH * NB;
+  for (int u = tid; u < w_units; u += n_threads) {
+    const int row = u % NB;
+    const int kc = (u / NB) % KCH;
+    const int ti = u / (NB * KCH);
+    const int blk = row / N, n = row - blk * N;
+    // vertical tap of a block: stride 1: the input row feeds output rows y-1, y, y+1 = taps 2, 1, 0;
+    // stride 2: even input rows carry tap 1 (block 0), odd rows taps 2 and 0 (blocks 1, 2)
+    const int r = KS == 1 ? 0 : (STRIDE == 1 ? 2 - blk : (blk == 0 ? 1 : (blk == 1 ? 2 : 0)));
+    const uint8_t* wrow = staged + (size_t)n * wrow_bytes;
+    uint32_t pk[PIECES][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int c = kc * 8 + j;
+      const int k = KS == 1 ? c : (c * 3 + r) * 3 + ti;
+      float w;
+      if (bits == 8) w = (float)(int)(int8_t)wrow[k];
+      else if (bits == 4) {
+        const int byte = wrow[k >> 1];
+        w = (float)((((k & 1) ? (byte >> 4) : (byte & 0xF)) ^ 8) - 8);
+      } else if (bits == 16) w = __half2float(reinterpret_cast<const __half*>(wrow)[k]);
+      else w = reinterpret_cast<const float*>(wrow)[k];
+#pragma unroll
+      for (int pc = 0; pc < PIECES; ++pc) {
+        const __nv_bfloat16 hb = __float2bfloat16_rn(w);   // exact for the integer codes
+        w -= __bfloat162float(hb);                          // exact: the remainder of the rounding
+        const uint32_t bits16 = (uint32_t)__bfloat16_as_ushort(hb);
+        if (j & 1) pk[pc][j >> 1] |= bits16 << 16; else pk[pc][j >> 1] = bits16;
+      }
+    }
+#pragma unroll
+    for (int pc = 0; pc < PIECES; ++pc)
+      *reinterpret_cast<uint4*>(wsm + (size_t)(pc * T + ti) * tile_b + (size_t)kc * NB * 16 + row * 16) =
+          make_uint4(pk[pc][0], pk[pc][1], pk[pc][2], pk[pc][3]);
+  }
+}
+
+// A row program in registers.
+struct RowRegs { uint4 w0, w1, w2, w3, w4; };
+__device__ __forceinline__ RowRegs rs_load_row(const RowProgram& rp) {
+  RowRegs r;
+  r.w0 = *reinterpret_cast<const uint4*>(&rp.head_idesc[0]);   // head_idesc[0..2], head_dcol[0]
+  r.w1 = *reinterpret_cast<const uint4*>(&rp.head_dcol[1]);    // head_dcol[1..2], head_boff[0..1]
+  r.w2 = *reinterpret_cast<const uint4*>(&rp.head_boff[2]);    // head_boff[2], rest_idesc[0..1], rest_dcol[0]
+  r.w3 = *reinterpret_cast<const uint4*>(&rp.rest_dcol[1]);    // rest_dcol[1], rest_boff[0..1], head_acc
+  r.w4 = *reinterpret_cast<const uint4*>(&rp.n_runs);          // n_runs, fresh, done, pad
+  return r;
+}
+
+// All MMAs of one input row into one column tile: d_xt = accumulator base of the tile, a_xt = low
+// descriptor word of the tile's pixel operand (tap offset 0), operand steps in 16-byte units.
+// Called by a converged warp; an elected lane issues.
+template <int C, int T, int PIECES>
+__device__ __forceinline__ void rs_issue_row(const RowRegs& rr, uint32_t d_xt, uint32_t a_xt, uint32_t a_tap0, uint32_t a_tap1,
+                                             uint32_t a_tap2, uint32_t a_part_step, uint32_t a_kk_step, uint32_t w_lo0,
+                                             uint32_t b_tile_step, uint32_t b_kk_step) {
+  constexpr uint32_t DESC_HI = (uint32_t)(128 >> 4) | (1u << 14);   // 128 bytes between groups of 8 rows; no swizzle
+  const uint32_t h0_idesc = rr.w0.x, h1_idesc = rr.w0.y, h2_idesc = rr.w0.z, h0_dcol = rr.w0.w;
+  const uint32_t h1_dcol = rr.w1.x, h2_dcol = rr.w1.y, h0_boff = rr.w1.z, h1_boff = rr.w1.w;
+  const uint32_t h2_boff = rr.w2.x, r0_idesc = rr.w2.y, r1_idesc = rr.w2.z, r0_dcol = rr.w2.w;
+  const uint32_t r1_dcol = rr.w3.x, r0_boff = rr.w3.y, r1_boff = rr.w3.z, head_acc = rr.w3.w;
+  const bool head1 = (rr.w4.x & 15u) > 1u, head2 = (rr.w4.x & 15u) > 2u, rest1 = (rr.w4.x >> 4) > 1u;
+  const uint32_t h0_acc = head_acc & 1u, h1_acc = (head_acc >> 1) & 1u, h2_acc = (head_acc >> 2) & 1u;
+#pragma unroll
+  for (int t = 0; t < T; ++t) {
+    const uint32_t a_t = a_xt + ((t == 0 ? a_tap0 : (t == 1 ? a_tap1 : a_tap2)) >> 4);
+#pragma unroll
+    for (int part = 0; part < 2; ++part) {
+#pragma unroll
+      for (int kk = 0; kk < C / 16; ++kk) {
+        const uint64_t adesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(a_t + part * a_part_step + kk * a_kk_step);
+#pragma unroll
+        for (int pc = 0; pc < PIECES; ++pc) {
+          const uint32_t b_lo = w_lo0 + (uint32_t)(pc * T + t) * b_tile_step + (uint32_t)kk * b_kk_step;
+          if (t == 0 && part == 0 && kk == 0 && pc == 0) {
+            umma_bf16(d_xt + h0_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + h0_boff), h0_idesc, h0_acc);
+            if (head1) umma_bf16(d_xt + h1_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + h1_boff), h1_idesc, h1_acc);
+            if (head2) umma_bf16(d_xt + h2_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + h2_boff), h2_idesc, h2_acc);
+          } else {
+            umma_bf16(d_xt + r0_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + r0_boff), r0_idesc, 1u);
+            if (rest1) umma_bf16(d_xt + r1_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + r1_boff), r1_idesc, 1u);
+          }
+        }
+      }
+    }
+  }
+}
+
+// 16 accumulator values of one lane (a 16-channel chunk of one pixel) -> scale, bias, residual,
+// activation, split into hi / lo bfloat16 pairs: hi[0..3] / hi[4..7] are the two hi planes of
+// the chunk, lo likewise.  res: the four residual planes (hi, hi, lo, lo) of the same pixel.
+__device__ __forceinline__ void rs_finish_unit(const uint32_t* v, const float* scale, const float* bias, const uint4* res,
+                                               bool has_res, int act, uint32_t* hi, uint32_t* lo) {
+#pragma unroll
+  for (int e = 0; e < 16; e += 4) {
+    const float4 sc = *reinterpret_cast<const float4*>(scale + e);
+    const float4 bi = *reinterpret_cast<const float4*>(bias + e);
+    float u0 = fmaf(__uint_as_float(v[e]), sc.x, bi.x);
+    float u1 = fmaf(__uint_as_float(v[e + 1]), sc.y, bi.y);
+    float u2 = fmaf(__uint_as_float(v[e + 2]), sc.z, bi.z);
+    float u3 = fmaf(__uint_as_float(v[e + 3]), sc.w, bi.w);
+    if (has_res) {
+      // planes 0 / 1 of the chunk hold channels 0-7 / 8-15; a bfloat16 is the upper half of a float
+      const uint4 rh4 = res[e >> 3], rl4 = res[2 + (e >> 3)];
+      const uint32_t rh0 = (e & 4) ? rh4.z : rh4.x, rh1 = (e & 4) ? rh4.w : rh4.y;
+      const uint32_t rl0 = (e & 4) ? rl4.z : rl4.x, rl1 = (e & 4) ? rl4.w : rl4.y;
+      u0 += __uint_as_float(rh0 << 16) + __uint_as_float(rl0 << 16);
+      u1 += __uint_as_float(rh0 & 0xFFFF0000u) + __uint_as_float(rl0 & 0xFFFF0000u);
+      u2 += __uint_as_float(rh1 << 16) + __uint_as_float(rl1 << 16);
+      u3 += __uint_as_float(rh1 & 0xFFFF0000u) + __uint_as_float(rl1 & 0xFFFF0000u);
+    }
+    split_pair(apply_act(u0, act), apply_act(u1, act), hi[e >> 1], lo[e >> 1]);
+    split_pair(apply_act(u2, act), apply_act(u3, act), hi[(e >> 1) + 1], lo[(e >> 1) + 1]);
+  }
+}
+
 template <int C, int KS, int STRIDE, int PIECES>
 __global__ void __launch_bounds__(kRsMaxThreads, 1)
 conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1, RsParams p,
@@ -169,96 +347,9 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     s_bias[i] = job.bias[n_off + i];
   }
   // row programs (one thread per input row)
-  if (tid < p.H) {
-    constexpr uint32_t IDESC0 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);   // f32 += bf16 x bf16, M = 128
-    const uint32_t n_field = ((uint32_t)N >> 3) << 17;                                     // N field of one output row
-    const int y = tid;
-    // output rows this input row contributes to: [yo, yo + n_rows), weight blocks [blk, ...); the
-    // rows from index `fresh` on receive their first contribution; rows done_a / done_b are complete
-    int yo, n_rows, blk, fresh, done_a = -1, done_b = -1;
-    if (KS == 1) { yo = y / STRIDE; n_rows = 1; blk = 0; fresh = 0; done_a = yo; }
-    else if (STRIDE == 1) {
-      yo = y > 0 ? y - 1 : 0;
-      const int hi = y + 1 < p.H ? y + 1 : p.H - 1;
-      n_rows = hi - yo + 1;
-      blk = yo - (y - 1);
-      fresh = y == 0 ? 0 : (y + 1 < p.H ? n_rows - 1 : n_rows);
-      if (y >= 1) done_a = y - 1;
-      if (y == p.H - 1) done_b = y;
-    } else if ((y & 1) == 0) { yo = y >> 1; n_rows = 1; blk = 0; fresh = y == 0 ? 0 : 1; }
-    else { yo = y >> 1; blk = 1; n_rows = (yo + 1 < p.Ho) ? 2 : 1; fresh = 1; done_a = yo; }
-    const int s0 = yo & (R - 1);
-    const int wrap = R - s0;                       // rows from this index on continue at slot 0
-    const int cw = (wrap > 0 && wrap < n_rows) ? wrap : n_rows;
-    const int cf = (fresh > 0 && fresh < n_rows) ? fresh : n_rows;
-    RowProgram rp = {};
-    auto set_run = [&](uint32_t* idesc, uint32_t* dcol, uint32_t* boff, int k, int i, int j) {
-      idesc[k] = IDESC0 | (uint32_t)(j - i) * n_field;
-      dcol[k] = (uint32_t)(((s0 + i) & (R - 1)) * N);
-      boff[k] = (uint32_t)((blk + i) * N);
-    };
-    int n_rest = 1;
-    set_run(rp.rest_idesc, rp.rest_dcol, rp.rest_boff, 0, 0, cw);
-    if (cw < n_rows) { set_run(rp.rest_idesc, rp.rest_dcol, rp.rest_boff, 1, cw, n_rows); n_rest = 2; }
-    const int c1 = cw < cf ? cw : cf;
-    int c2 = cw < cf ? cf : cw;
-    if (c2 == c1) c2 = n_rows;
-    int n_head = 1;
-    set_run(rp.head_idesc, rp.head_dcol, rp.head_boff, 0, 0, c1);
-    rp.head_acc = 0 >= fresh ? 0u : 1u;
-    if (c1 < n_rows) {
-      set_run(rp.head_idesc, rp.head_dcol, rp.head_boff, 1, c1, c2);
-      rp.head_acc |= (c1 >= fresh ? 0u : 1u) << 1;
-      n_head = 2;
-      if (c2 < n_rows) {
-        set_run(rp.head_idesc, rp.head_dcol, rp.head_boff, 2, c2, n_rows);
-        rp.head_acc |= (c2 >= fresh ? 0u : 1u) << 2;
-        n_head = 3;
-      }
-    }
-    rp.n_runs = (uint32_t)n_head | ((uint32_t)n_rest << 4);
-    rp.fresh = (uint32_t)(yo + fresh) | ((uint32_t)(n_rows - fresh) << 8);
-    rp.done = (uint32_t)(done_a + 1) | ((uint32_t)(done_b + 1) << 8);
-    s_rows[y] = rp;
-  }
+  if (tid < p.H) s_rows[tid] = rs_row_program<KS, STRIDE>(tid, p.H, p.Ho, N, R);
   bool alive = mbar_wait_warp(bar_w, 0, s_abort, p.error_flag);
-  if (alive) {
-    const int w_units = T * KCH * NB;
-    for (int u = tid; u < w_units; u += n_threads) {
-      const int row = u % NB;
-      const int kc = (u / NB) % KCH;
-      const int ti = u / (NB * KCH);
-      const int blk = row / N, n = row - blk * N;
-      // vertical tap of a block: stride 1: the input row feeds output rows y-1, y, y+1 = taps 2, 1, 0;
-      // stride 2: even input rows carry tap 1 (block 0), odd rows taps 2 and 0 (blocks 1, 2)
-      const int r = KS == 1 ? 0 : (STRIDE == 1 ? 2 - blk : (blk == 0 ? 1 : (blk == 1 ? 2 : 0)));
-      const uint8_t* wrow = ring + (size_t)n * wrow_bytes;
-      uint32_t pk[PIECES][4];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int c = kc * 8 + j;
-        const int k = KS == 1 ? c : (c * 3 + r) * 3 + ti;
-        float w;
-        if (job.bits == 8) w = (float)(int)(int8_t)wrow[k];
-        else if (job.bits == 4) {
-          const int byte = wrow[k >> 1];
-          w = (float)((((k & 1) ? (byte >> 4) : (byte & 0xF)) ^ 8) - 8);
-        } else if (job.bits == 16) w = __half2float(reinterpret_cast<const __half*>(wrow)[k]);
-        else w = reinterpret_cast<const float*>(wrow)[k];
-#pragma unroll
-        for (int pc = 0; pc < PIECES; ++pc) {
-          const __nv_bfloat16 hb = __float2bfloat16_rn(w);   // exact for the integer codes
-          w -= __bfloat162float(hb);                          // exact: the remainder of the rounding
-          const uint32_t bits16 = (uint32_t)__bfloat16_as_ushort(hb);
-          if (j & 1) pk[pc][j >> 1] |= bits16 << 16; else pk[pc][j >> 1] = bits16;
-        }
-      }
-#pragma unroll
-      for (int pc = 0; pc < PIECES; ++pc)
-        *reinterpret_cast<uint4*>(wsm + (size_t)(pc * T + ti) * tile_b + (size_t)kc * NB * 16 + row * 16) =
-            make_uint4(pk[pc][0], pk[pc][1], pk[pc][2], pk[pc][3]);
-    }
-  }
+  if (alive) rs_expand_weights<C, KS, STRIDE, PIECES>(ring, wrow_bytes, job.bits, N, wsm, tid, n_threads);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // expanded weights -> visible to the MMA
   tc_fence_before();
   __syncthreads();
@@ -326,18 +417,8 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         const int q0 = item_local * p.Ho;
         for (int y = 0; y < p.H && alive; ++y) {
           if (!row_used(y)) continue;
-          const RowProgram& rp = s_rows[y];
-          const uint4 w0 = *reinterpret_cast<const uint4*>(&rp.head_idesc[0]);   // head_idesc[0..2], head_dcol[0]
-          const uint4 w1 = *reinterpret_cast<const uint4*>(&rp.head_dcol[1]);    // head_dcol[1..2], head_boff[0..1]
-          const uint4 w2 = *reinterpret_cast<const uint4*>(&rp.head_boff[2]);    // head_boff[2], rest_idesc[0..1], rest_dcol[0]
-          const uint4 w3 = *reinterpret_cast<const uint4*>(&rp.rest_dcol[1]);    // rest_dcol[1], rest_boff[0..1], head_acc
-          const uint4 w4 = *reinterpret_cast<const uint4*>(&rp.n_runs);          // n_runs, fresh, done, pad
-          const uint32_t h0_idesc = w0.x, h1_idesc = w0.y, h2_idesc = w0.z, h0_dcol = w0.w;
-          const uint32_t h1_dcol = w1.x, h2_dcol = w1.y, h0_boff = w1.z, h1_boff = w1.w;
-          const uint32_t h2_boff = w2.x, r0_idesc = w2.y, r1_idesc = w2.z, r0_dcol = w2.w;
-          const uint32_t r1_dcol = w3.x, r0_boff = w3.y, r1_boff = w3.z, head_acc = w3.w;
-          const bool head1 = (w4.x & 15u) > 1u, head2 = (w4.x & 15u) > 2u, rest1 = (w4.x >> 4) > 1u;
-          const uint32_t h0_acc = head_acc & 1u, h1_acc = (head_acc >> 1) & 1u, h2_acc = (head_acc >> 2) & 1u;
+          const RowRegs rr = rs_load_row(s_rows[y]);
+          const uint4 w4 = rr.w4;
           const int fresh_row = (int)(w4.y & 255u), n_fresh = (int)(w4.y >> 8);
           for (int i = 0; i < n_fresh && alive; ++i) {
             const int q = q0 + fresh_row + i;
@@ -348,33 +429,10 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           if (!alive) break;
           tc_fence_after();
           const uint32_t a_stage = smem_u32(ring) + stage * p.stage_bytes;
-          for (int xt = 0; xt < p.xt; ++xt) {
-            const uint32_t d_xt = tmem_base + (uint32_t)(xt * R * N);
-            const uint32_t a_xt = ((a_stage + (uint32_t)xt * kRsTileBytes) >> 4) | a_lbo_field;
-#pragma unroll
-            for (int t = 0; t < T; ++t) {
-              const uint32_t a_t = a_xt + ((t == 0 ? a_tap0 : (t == 1 ? a_tap1 : a_tap2)) >> 4);
-#pragma unroll
-              for (int part = 0; part < 2; ++part) {
-#pragma unroll
-                for (int kk = 0; kk < C / 16; ++kk) {
-                  const uint64_t adesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(a_t + part * a_part_step + kk * a_kk_step);
-#pragma unroll
-                  for (int pc = 0; pc < PIECES; ++pc) {
-                    const uint32_t b_lo = w_lo0 + (uint32_t)(pc * T + t) * b_tile_step + (uint32_t)kk * b_kk_step;
-                    if (t == 0 && part == 0 && kk == 0 && pc == 0) {
-                      umma_bf16(d_xt + h0_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + h0_boff), h0_idesc, h0_acc);
-                      if (head1) umma_bf16(d_xt + h1_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + h1_boff), h1_idesc, h1_acc);
-                      if (head2) umma_bf16(d_xt + h2_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + h2_boff), h2_idesc, h2_acc);
-                    } else {
-                      umma_bf16(d_xt + r0_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + r0_boff), r0_idesc, 1u);
-                      if (rest1) umma_bf16(d_xt + r1_dcol, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + r1_boff), r1_idesc, 1u);
-                    }
-                  }
-                }
-              }
-            }
-          }
+          for (int xt = 0; xt < p.xt; ++xt)
+            rs_issue_row<C, T, PIECES>(rr, tmem_base + (uint32_t)(xt * R * N),
+                                       ((a_stage + (uint32_t)xt * kRsTileBytes) >> 4) | a_lbo_field, a_tap0, a_tap1, a_tap2,
+                                       a_part_step, a_kk_step, w_lo0, b_tile_step, b_kk_step);
           umma_commit(bar_in_empty + 8 * stage);       // the stage is free once these MMAs retire
           if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
           // output rows that are complete with this input row
@@ -455,27 +513,7 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           if (lane == 0) mbar_arrive(bar_out_empty + 8 * slot);
         }
         uint32_t hi[8], lo[8];
-#pragma unroll
-        for (int e = 0; e < 16; e += 4) {
-          const float4 sc = *reinterpret_cast<const float4*>(s_scale + c0 + e);
-          const float4 bi = *reinterpret_cast<const float4*>(s_bias + c0 + e);
-          float u0 = fmaf(__uint_as_float(v[e]), sc.x, bi.x);
-          float u1 = fmaf(__uint_as_float(v[e + 1]), sc.y, bi.y);
-          float u2 = fmaf(__uint_as_float(v[e + 2]), sc.z, bi.z);
-          float u3 = fmaf(__uint_as_float(v[e + 3]), sc.w, bi.w);
-          if (res_base) {
-            // planes 0 / 1 of the chunk hold channels 0-7 / 8-15; a bfloat16 is the upper half of a float
-            const uint4 rh4 = rres[e >> 3], rl4 = rres[2 + (e >> 3)];
-            const uint32_t rh0 = (e & 4) ? rh4.z : rh4.x, rh1 = (e & 4) ? rh4.w : rh4.y;
-            const uint32_t rl0 = (e & 4) ? rl4.z : rl4.x, rl1 = (e & 4) ? rl4.w : rl4.y;
-            u0 += __uint_as_float(rh0 << 16) + __uint_as_float(rl0 << 16);
-            u1 += __uint_as_float(rh0 & 0xFFFF0000u) + __uint_as_float(rl0 & 0xFFFF0000u);
-            u2 += __uint_as_float(rh1 << 16) + __uint_as_float(rl1 << 16);
-            u3 += __uint_as_float(rh1 & 0xFFFF0000u) + __uint_as_float(rl1 & 0xFFFF0000u);
-          }
-          split_pair(apply_act(u0, p.act), apply_act(u1, p.act), hi[e >> 1], lo[e >> 1]);
-          split_pair(apply_act(u2, p.act), apply_act(u3, p.act), hi[(e >> 1) + 1], lo[(e >> 1) + 1]);
-        }
+        rs_finish_unit(v, s_scale + c0, s_bias + c0, rres, res_base != nullptr, p.act, hi, lo);
         // the residual registers are free again: request the first unit of this warp's next row
         if (res_base && u + unit_step >= units && k + 1 < total) load_res(k + 1, unit0, rres);
         uint8_t* dst = out_base + row_off + uoff;
@@ -493,6 +531,287 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// A whole basic block in one kernel:  out = relu( conv2( relu(conv1(x)) ) + x ),  both convolutions
+// 3x3 at stride 1 with C -> C channels (C = 16 or 32, 8 images per group, 4- / 8-bit weights).
+// The intermediate tensor never leaves the SM: the first epilogue writes each finished row of it
+// into a shared-memory ring in the layout the TMA gives input rows (zero columns on both sides
+// included), where the second convolution's MMAs read it; the shortcut x[y] is read from the input
+// ring, which keeps a row until the output row at the same height is finished.  Per block the
+// kernel reads x once and writes out once: 2 tensors instead of 5.
+//
+// Warps: 0 TMA producer, 1 MMA issuer of conv1, 2 MMA issuer of conv2 (each hides the other's
+// per-row bookkeeping), 3-10 first epilogue (accumulators -> shared memory), 11-18 second
+// epilogue (accumulators + shortcut -> global memory).  Tensor memory: columns 0-255 hold the
+// ring of conv1 rows, 256-511 the ring of conv2 rows.
+// ---------------------------------------------------------------------------------------------
+constexpr int kRbThreads = 19 * 32;
+constexpr int kRbSlots = 8;
+constexpr int kRbMaxIn = 6, kRbMaxMid = 4;
+
+struct RbParams {
+  int H, W;
+  int n_items;
+  int rows_per_version;
+  int in_stages, mid_stages;
+  int K;                  // elements of a packed weight row (9 C)
+  int stage_bytes, a_lbo, xt;
+  int32_t* error_flag;
+};
+
+struct RbSmem { int in_ring, mid_ring, w1, w2, coef, rows, bars, total; };
+__host__ __device__ inline RbSmem rb_smem(int in_stages, int mid_stages, int stage_bytes, int C) {
+  RbSmem s;
+  const int wbytes = 3 * (C / 8) * 3 * C * 16;
+  s.in_ring = 0;
+  s.mid_ring = in_stages * stage_bytes;
+  s.w1 = s.mid_ring + mid_stages * stage_bytes;
+  s.w2 = s.w1 + wbytes;
+  s.coef = s.w2 + wbytes;                                // scale1, bias1, scale2, bias2
+  s.rows = (s.coef + 4 * C * 4 + 127) / 128 * 128;
+  s.bars = s.rows + kRsMaxRows * kRsRowWords * 4;
+  s.total = s.bars + (2 * kRbMaxIn + 2 * kRbMaxMid + 4 * kRbSlots + 1) * 8 + 16;
+  return s;
+}
+
+template <int C>
+__global__ void __launch_bounds__(kRbThreads, 1)
+conv_rs_block_kernel(const __grid_constant__ CUtensorMap in_map, RbParams p, const LayerJob* __restrict__ jobs) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const LayerJob job = jobs[blockIdx.y];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr int N = C, NB = 3 * C, KCH = C / 8, R = kRbSlots;
+  constexpr int tile_b = KCH * NB * 16;
+  const int S_in = p.in_stages, S_mid = p.mid_stages;
+  const RbSmem sm = rb_smem(S_in, S_mid, p.stage_bytes, C);
+  uint8_t* in_ring = smem;
+  uint8_t* mid_ring = smem + sm.mid_ring;
+  uint8_t* w1 = smem + sm.w1;
+  uint8_t* w2 = smem + sm.w2;
+  float* s_coef = reinterpret_cast<float*>(smem + sm.coef);
+  RowProgram* s_rows = reinterpret_cast<RowProgram*>(smem + sm.rows);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
+  const uint32_t bar_in_full = smem_u32(bars);
+  const uint32_t bar_in_free = bar_in_full + 8 * kRbMaxIn;
+  const uint32_t bar_mid_full = bar_in_free + 8 * kRbMaxIn;
+  const uint32_t bar_mid_free = bar_mid_full + 8 * kRbMaxMid;
+  const uint32_t bar_a1_full = bar_mid_free + 8 * kRbMaxMid;
+  const uint32_t bar_a1_empty = bar_a1_full + 8 * R;
+  const uint32_t bar_a2_full = bar_a1_empty + 8 * R;
+  const uint32_t bar_a2_empty = bar_a2_full + 8 * R;
+  const uint32_t bar_w = bar_a2_empty + 8 * R;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kRbMaxIn + 2 * kRbMaxMid + 4 * R + 1);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  if (tid == 0) {
+    for (int i = 0; i < kRbMaxIn; ++i) {
+      mbar_init(bar_in_full + 8 * i, 1);
+      mbar_init(bar_in_free + 8 * i, 1 + 8);           // conv1's MMAs retired + the eight shortcut readers
+    }
+    for (int i = 0; i < kRbMaxMid; ++i) {
+      mbar_init(bar_mid_full + 8 * i, 8);              // the eight warps of the first epilogue
+      mbar_init(bar_mid_free + 8 * i, 1);
+    }
+    for (int i = 0; i < R; ++i) {
+      mbar_init(bar_a1_full + 8 * i, 1);
+      mbar_init(bar_a1_empty + 8 * i, 8);
+      mbar_init(bar_a2_full + 8 * i, 1);
+      mbar_init(bar_a2_empty + 8 * i, 8);
+    }
+    mbar_init(bar_w, 1);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tmem_alloc(smem_u32(s_tmem), 512);
+    tmem_relinquish();
+  }
+  // packed weights of both convolutions -> the (still unused) input ring, then expansion
+  const int kpad = (p.K + 31) / 32 * 32;
+  const uint32_t wrow1 = (uint32_t)kpad * job.bits_pre / 8, wrow2 = (uint32_t)kpad * job.bits / 8;
+  const uint32_t packed1 = wrow1 * N, packed2 = wrow2 * N;
+  if (tid == 0) {
+    mbar_expect_tx(bar_w, packed1 + packed2);
+    bulk_load(smem_u32(in_ring), job.w_pre, packed1, bar_w);
+    bulk_load(smem_u32(in_ring) + packed1, job.w, packed2, bar_w);
+  }
+  for (int i = tid; i < N; i += kRbThreads) {
+    s_coef[i] = job.scale_pre[i];
+    s_coef[N + i] = job.bias_pre[i];
+    s_coef[2 * N + i] = job.scale[i];
+    s_coef[3 * N + i] = job.bias[i];
+  }
+  if (tid < p.H) s_rows[tid] = rs_row_program<3, 1>(tid, p.H, p.H, N, R);
+  // the zero columns on both sides of every row of the intermediate ring are written once, here
+  for (int i = tid; i < S_mid * p.stage_bytes / 16; i += kRbThreads)
+    reinterpret_cast<uint4*>(mid_ring)[i] = make_uint4(0u, 0u, 0u, 0u);
+  bool alive = mbar_wait_warp(bar_w, 0, s_abort, p.error_flag);
+  if (alive) {
+    rs_expand_weights<C, 3, 1, 1>(in_ring, wrow1, job.bits_pre, N, w1, tid, kRbThreads);
+    rs_expand_weights<C, 3, 1, 1>(in_ring + packed1, wrow2, job.bits, N, w2, tid, kRbThreads);
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  alive = alive && (*s_abort == 0);
+
+  const int n_my_items = ((int)blockIdx.x < p.n_items) ? (p.n_items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  const int total = n_my_items * p.H;                  // rows this CTA streams, numbered g = item_local * H + y
+  // operand constants of the MMA issuers
+  const uint32_t a_lbo_field = ((uint32_t)p.a_lbo >> 4) << 16;
+  const uint32_t a_part_step = ((uint32_t)KCH * (uint32_t)p.a_lbo) >> 4, a_kk_step = (2u * (uint32_t)p.a_lbo) >> 4;
+  const uint32_t b_tile_step = (uint32_t)tile_b >> 4, b_kk_step = 2u * (uint32_t)NB;
+  const uint32_t b_lbo_field = ((uint32_t)(NB * 16) >> 4) << 16;
+  const uint32_t tap1 = 128u, tap2 = 256u;             // one column = 8 images x 16 bytes
+
+  if (warp == 0) {
+    if (lane == 0 && alive) {
+      uint32_t issued = 0, issued_phase = 0;
+      for (int g = 0; g < total && alive; ++g) {
+        const int il = g / p.H, y = g - il * p.H;
+        const uint32_t stage = (uint32_t)(g % S_in), phase = (uint32_t)((g / S_in) & 1);
+        alive = mbar_wait(bar_in_free + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+        if (!alive) break;
+        issued |= 1u << stage;
+        issued_phase = (issued_phase & ~(1u << stage)) | (phase << stage);
+        mbar_expect_tx(bar_in_full + 8 * stage, (uint32_t)p.stage_bytes);
+        const int item = (int)blockIdx.x + il * (int)gridDim.x;
+        tma_load_4d(smem_u32(in_ring) + stage * p.stage_bytes, &in_map, bar_in_full + 8 * stage, 0, -1, 0,
+                    job.in_version * p.rows_per_version + item * p.H + y);
+      }
+      for (int i = 0; i < S_in; ++i)
+        if (issued & (1u << i)) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar_in_full + 8 * i, (issued_phase >> i) & 1u) && clock64() - t0 < kWaitLimitCycles) {}
+        }
+    }
+  } else if (warp == 1 || warp == 2) {
+    // conv1 streams the input ring into accumulator ring 1; conv2 streams the intermediate ring into
+    // accumulator ring 2.  Same row programs: both are 3x3, stride 1, on H rows.
+    const bool second = warp == 2;
+    const uint32_t bar_src_full = second ? bar_mid_full : bar_in_full;
+    const uint32_t bar_src_free = second ? bar_mid_free : bar_in_free;
+    const uint32_t bar_acc_full = second ? bar_a2_full : bar_a1_full;
+    const uint32_t bar_acc_empty = second ? bar_a2_empty : bar_a1_empty;
+    const int S = second ? S_mid : S_in;
+    const uint32_t src_ring = smem_u32(second ? mid_ring : in_ring);
+    const uint32_t w_lo0 = (smem_u32(second ? w2 : w1) >> 4) | b_lbo_field;
+    const uint32_t d_base = tmem_base + (second ? 256u : 0u);
+    for (int g = 0; g < total && alive; ++g) {
+      const int il = g / p.H, y = g - il * p.H;
+      const RowRegs rr = rs_load_row(s_rows[y]);
+      const int fresh_row = (int)(rr.w4.y & 255u), n_fresh = (int)(rr.w4.y >> 8);
+      for (int i = 0; i < n_fresh && alive; ++i) {
+        const int q = il * p.H + fresh_row + i;
+        alive = mbar_wait_warp(bar_acc_empty + 8 * (q & (R - 1)), ((q / R) & 1) ^ 1u, s_abort, p.error_flag);
+      }
+      if (!alive) break;
+      const uint32_t stage = (uint32_t)(g % S), phase = (uint32_t)((g / S) & 1);
+      alive = mbar_wait_warp(bar_src_full + 8 * stage, phase, s_abort, p.error_flag);
+      if (!alive) break;
+      tc_fence_after();
+      const uint32_t a_stage = src_ring + stage * p.stage_bytes;
+      for (int xt = 0; xt < p.xt; ++xt)
+        rs_issue_row<C, 3, 1>(rr, d_base + (uint32_t)(xt * R * N), ((a_stage + (uint32_t)xt * kRsTileBytes) >> 4) | a_lbo_field,
+                              0u, tap1, tap2, a_part_step, a_kk_step, w_lo0, b_tile_step, b_kk_step);
+      umma_commit(bar_src_free + 8 * stage);
+      // rows complete with this one (H is a multiple of the ring depth, so the slot is the row's low bits)
+      if (rr.w4.z & 255u) umma_commit(bar_acc_full + 8 * (((rr.w4.z & 255u) - 1u) & (uint32_t)(R - 1)));
+      if (rr.w4.z >> 8) umma_commit(bar_acc_full + 8 * (((rr.w4.z >> 8) - 1u) & (uint32_t)(R - 1)));
+    }
+  } else {
+    const bool second = warp >= 11;
+    const int qd = warp & 3;
+    const int h = ((second ? warp - 11 : warp - 3) >> 2);       // 0 or 1: the unit of a row this warp takes
+    const int l = qd * 32 + lane;
+    const int x_local = l >> 3, img = l & 7;
+    constexpr int chunks = N / 16;
+    const int xt = h / chunks, c0 = (h - xt * chunks) * 16;
+    const int x = xt * 16 + x_local;
+    const int ph = c0 >> 3;                                      // first hi plane of the chunk
+    constexpr int lo_plane0 = C / 8;
+    const uint32_t bar_acc_full = second ? bar_a2_full : bar_a1_full;
+    const uint32_t bar_acc_empty = second ? bar_a2_empty : bar_a1_empty;
+    const uint32_t t_col = (second ? 256u : 0u) + (uint32_t)(xt * R * N + c0);
+    const float* scale = s_coef + (second ? 2 * N : 0) + c0;
+    const float* bias = s_coef + (second ? 3 * N : N) + c0;
+    // offset of this lane's (column, image) cell inside a ring stage, first hi plane of its chunk
+    const uint32_t cell = (uint32_t)ph * (uint32_t)p.a_lbo + (uint32_t)(x + 1) * 128u + (uint32_t)img * 16u;
+    const size_t plane_bytes = 128, px_bytes = (size_t)(C / 4) * 128;
+    uint8_t* out_base = static_cast<uint8_t*>(job.out);
+    for (int g = 0; g < total && alive; ++g) {
+      const int il = g / p.H, y = g - il * p.H;
+      const int slot = g & (R - 1);
+      uint32_t v[16];
+      uint32_t hi[8], lo[8];
+      if (!second) {
+        const uint32_t ms = (uint32_t)(g % S_mid), mphase = (uint32_t)((g / S_mid) & 1);
+        alive = mbar_wait_warp(bar_acc_full + 8 * slot, (g / R) & 1, s_abort, p.error_flag);
+        if (!alive) break;
+        tc_fence_after();
+        tmem_ld16(tmem_base + ((uint32_t)(qd * 32) << 16) + t_col + (uint32_t)(slot * N), v);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_acc_empty + 8 * slot);
+        rs_finish_unit(v, scale, bias, nullptr, false, AIQ_ACT_RELU, hi, lo);
+        // the stage of the intermediate ring must have been read by conv2's MMAs of its last occupant
+        alive = mbar_wait_warp(bar_mid_free + 8 * ms, mphase ^ 1u, s_abort, p.error_flag);
+        if (!alive) break;
+        uint8_t* dst = mid_ring + ms * p.stage_bytes + cell;
+        *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(dst + p.a_lbo) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+        *reinterpret_cast<uint4*>(dst + lo_plane0 * p.a_lbo) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        *reinterpret_cast<uint4*>(dst + (lo_plane0 + 1) * p.a_lbo) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_mid_full + 8 * ms);
+      } else {
+        const uint32_t is = (uint32_t)(g % S_in), iphase = (uint32_t)((g / S_in) & 1);
+        alive = mbar_wait_warp(bar_acc_full + 8 * slot, (g / R) & 1, s_abort, p.error_flag);
+        if (!alive) break;
+        tc_fence_after();
+        tmem_ld16(tmem_base + ((uint32_t)(qd * 32) << 16) + t_col + (uint32_t)(slot * N), v);
+        // shortcut: the block input at the same row, still in the input ring (its copy completed long
+        // ago; observing the barrier makes the data visible to this thread)
+        alive = mbar_wait_warp(bar_in_full + 8 * is, iphase, s_abort, p.error_flag);
+        uint4 rres[4];
+        const uint8_t* src = in_ring + is * p.stage_bytes + cell;
+        rres[0] = *reinterpret_cast<const uint4*>(src);
+        rres[1] = *reinterpret_cast<const uint4*>(src + p.a_lbo);
+        rres[2] = *reinterpret_cast<const uint4*>(src + lo_plane0 * p.a_lbo);
+        rres[3] = *reinterpret_cast<const uint4*>(src + (lo_plane0 + 1) * p.a_lbo);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(bar_acc_empty + 8 * slot);
+          mbar_arrive(bar_in_free + 8 * is);
+        }
+        if (!alive) break;
+        rs_finish_unit(v, scale, bias, rres, true, AIQ_ACT_RELU, hi, lo);
+        const int item = (int)blockIdx.x + il * (int)gridDim.x;
+        uint8_t* dst = out_base + (((size_t)item * p.H + y) * p.W + x) * px_bytes + (size_t)ph * plane_bytes + (size_t)img * 16;
+        *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(dst + plane_bytes) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+        *reinterpret_cast<uint4*>(dst + (size_t)lo_plane0 * plane_bytes) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        *reinterpret_cast<uint4*>(dst + (size_t)(lo_plane0 + 1) * plane_bytes) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -641,6 +960,49 @@ aiq_status_t launch_rs(const ConvGeom& g, const RsShape& sh, const CUtensorMap* 
   return AIQ_OK;
 }
 
+bool rb_shape_ok(const ConvGeom& g) {
+  if (g.in_is_nchw || g.act_format != ACT_RS) return false;
+  if (g.ks != 3 || g.pad != 1 || g.stride != 1 || g.Cin != g.Cout) return false;
+  if (!((g.Cin == 16 && g.W == 32) || (g.Cin == 32 && g.W == 16))) return false;   // two epilogue units per row
+  return g.H % kRbSlots == 0 && g.H <= kRsMaxRows && g.Ho == g.H && g.Wo == g.W;
+}
+
+template <int C>
+aiq_status_t launch_rb(const ConvGeom& g, const CUtensorMap* map, const LayerJob* jobs_dev, int n_jobs, int batch_capacity,
+                       int32_t* error_flag, double weight_bytes, cudaStream_t s) {
+  DeviceProps props;
+  if (aiq_status_t st = current_device_props(&props)) return st;
+  RbParams p = {};
+  p.H = g.H; p.W = g.W;
+  p.n_items = rs_padded_batch(g.B) / 8;
+  p.rows_per_version = rs_padded_batch(batch_capacity) / 8 * g.H;
+  p.K = g.K;
+  p.a_lbo = (g.W + 2) * 128;
+  p.stage_bytes = (C / 4) * p.a_lbo;
+  p.xt = g.W / 16;
+  p.error_flag = error_flag;
+  int in_stages = kRbMaxIn, mid_stages = kRbMaxMid;
+  while (rb_smem(in_stages, mid_stages, p.stage_bytes, C).total + 1024 > props.smem_optin && (in_stages > 4 || mid_stages > 3)) {
+    if (in_stages > 4 && in_stages - mid_stages >= 2) --in_stages; else if (mid_stages > 3) --mid_stages; else --in_stages;
+  }
+  const int smem_bytes = rb_smem(in_stages, mid_stages, p.stage_bytes, C).total + 1024;
+  const int packed = 2 * C * (int)row_bytes(g.K, 8);
+  if (smem_bytes > props.smem_optin || packed > in_stages * p.stage_bytes)
+    return set_error(AIQ_ERR_SHAPE, "conv_rs_block: %d bytes of shared memory needed", smem_bytes);
+  p.in_stages = in_stages; p.mid_stages = mid_stages;
+  AIQ_ENSURE_DYNAMIC_SMEM(conv_rs_block_kernel<C>, props.smem_optin);
+  int ctas = props.n_sms / n_jobs;
+  if (ctas > p.n_items) ctas = p.n_items;
+  if (ctas < 1) ctas = 1;
+  {
+    const double px = (double)g.B * g.H * g.W * C;
+    LaunchScope scope(AIQ_KERNEL_CONV_TC, s, 2.0 * 2.0 * px * (9.0 * C) * n_jobs, weight_bytes + 4.0 * n_jobs * 2.0 * px);
+    conv_rs_block_kernel<C><<<dim3(ctas, n_jobs), kRbThreads, smem_bytes, s>>>(map[0], p, jobs_dev);
+  }
+  AIQ_LAUNCH_CHECK("conv_rs_block");
+  return AIQ_OK;
+}
+
 }  // namespace
 
 bool conv_rs_eligible(const ConvGeom& g) {
@@ -723,6 +1085,16 @@ aiq_status_t launch_conv_rs(const ConvGeom& g, const void* maps, const LayerJob*
 #undef AIQ_RS_KS
 #undef AIQ_RS_ARGS
   return set_error(AIQ_ERR_SHAPE, "conv_rs: no kernel for Cin=%d", g.Cin);
+}
+
+bool conv_rs_block_eligible(const ConvGeom& g) { return rb_shape_ok(g); }
+
+aiq_status_t launch_conv_rs_block(const ConvGeom& g, const void* maps, const LayerJob* jobs_dev, int n_jobs, int batch_capacity,
+                                  int32_t* error_flag, double weight_bytes, cudaStream_t s) {
+  if (!rb_shape_ok(g)) return set_error(AIQ_ERR_SHAPE, "conv_rs_block: layer shape is not supported");
+  const CUtensorMap* m = static_cast<const CUtensorMap*>(maps);
+  if (g.Cin == 16) return launch_rb<16>(g, m, jobs_dev, n_jobs, batch_capacity, error_flag, weight_bytes, s);
+  return launch_rb<32>(g, m, jobs_dev, n_jobs, batch_capacity, error_flag, weight_bytes, s);
 }
 
 }  // namespace aiq

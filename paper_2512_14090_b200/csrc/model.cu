@@ -25,6 +25,7 @@ static thread_local int64_t t_launches = 0, t_layer_evals = 0, t_layer_evals_uns
 static std::atomic<int> g_opt_chunk{0};
 static std::atomic<int> g_opt_share{1};
 static std::atomic<int> g_opt_path{AIQ_PATH_AUTO};
+static std::atomic<int> g_opt_fuse{1};
 
 aiq_status_t set_error(aiq_status_t status, const char* fmt, ...) {
   va_list ap;
@@ -129,6 +130,8 @@ struct aiq_model {
   size_t dev_bytes;
   int act_format;                    // ACT_F32, ACT_SPLIT or ACT_RS (see common.cuh)
   int32_t* status_word;              // device word raised by a kernel whose bounded wait expired
+  std::vector<int> block_tail;       // per layer: the second convolution of the basic block this layer opens
+                                     // (the pair can run as one kernel), or -1
 };
 
 namespace aiq {
@@ -344,6 +347,27 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
   if (m->act_format == ACT_RS)
     for (LayerInfo& li : m->layers)
       if (li.d.kind != AIQ_LAYER_FC) li.out_bytes = rs_image_bytes(li.Ho, li.Wo, li.d.cout);
+  // identity-shortcut basic blocks that the fused block kernel takes: conv1 (3x3, ReLU) feeds only conv2
+  // (3x3, ReLU) and conv2 adds conv1's input
+  m->block_tail.assign(m->layers.size(), -1);
+  if (m->act_format == ACT_RS) {
+    const int n = (int)m->layers.size();
+    std::vector<int> uses(n, 0);
+    for (const LayerInfo& li : m->layers) {
+      if (li.d.input >= 0) uses[li.d.input]++;
+      if (li.d.residual >= 0) uses[li.d.residual]++;
+    }
+    for (int l1 = 0; l1 < n; ++l1) {
+      const LayerInfo& a = m->layers[l1];
+      if (a.d.kind != AIQ_LAYER_CONV || a.d.input < 0 || a.d.residual >= 0 || a.d.act != AIQ_ACT_RELU || uses[l1] != 1) continue;
+      for (int l2 = 0; l2 < n; ++l2) {
+        const LayerInfo& b = m->layers[l2];
+        if (b.d.kind == AIQ_LAYER_CONV && b.d.input == l1 && b.d.residual == a.d.input && b.d.act == AIQ_ACT_RELU &&
+            conv_rs_block_eligible(make_geom(m, a, 1)) && conv_rs_block_eligible(make_geom(m, b, 1)) && a.d.cin == b.d.cin)
+          m->block_tail[l1] = l2;
+      }
+    }
+  }
   assign_slots(m);
   cudaStream_t stream = (cudaStream_t)stream_;
   uint8_t* base = static_cast<uint8_t*>(dev_mem);
@@ -495,6 +519,8 @@ struct LayerPlan {
   int n_tc = 0;                         // leading jobs that run on the tensor-core kernel (4- / 8-bit weights)
   int n_tc16 = 0, n_tc32 = 0;           // then those with 16-bit and with 32-bit weights (tc_kind 1 only)
   int tc_kind = 0;                      // which tensor-core kernel (see layer_tensor_kind)
+  bool skipped = false;                 // first convolution of a fused block: evaluated inside its partner's kernel
+  int fused_head = -1;                  // second convolution of a fused block: the layer it absorbs
   double weight_bytes = 0.0;            // packed weights + scales + biases over all jobs
   double weight_bytes_tc = 0.0, weight_bytes_tc16 = 0.0, weight_bytes_tc32 = 0.0;
   TensorMapBytes maps[2];               // [0] over the input slot (tensor-core layers); [1] over the output slot
@@ -530,6 +556,17 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
   plan.jobs.clear();
   plan.batch_capacity = B;
   std::vector<std::vector<int>> ver(n, std::vector<int>(S, 0));   // ver[l][s]
+  std::vector<std::vector<std::tuple<int, int, int>>> all_keys(n);   // per layer and version: (bits, input version, residual version)
+  // a basic block runs as one kernel when every scheme gives both of its convolutions 4 or 8 bits
+  std::vector<int> fuse_head(n, -1);
+  if (g_opt_fuse.load())
+    for (int l1 = 0; l1 < n; ++l1) {
+      const int l2 = m->block_tail[l1];
+      if (l2 < 0) continue;
+      bool ok = true;
+      for (int s = 0; s < S && ok; ++s) ok = schemes[(size_t)s * n + l1] <= 8 && schemes[(size_t)s * n + l2] <= 8;
+      if (ok) fuse_head[l2] = l1;
+    }
   auto slot_ptr = [&](int layer, int version) -> uint8_t* {
     const LayerInfo& li = m->layers[layer];
     const size_t Bslot = m->act_format == ACT_RS ? (size_t)rs_padded_batch(B) : (size_t)B;
@@ -559,6 +596,46 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
     }
     lp.n_versions = (int)keys.size();
     plan.versions_total += lp.n_versions;
+    all_keys[l] = keys;
+    if (li.d.kind != AIQ_LAYER_FC && m->block_tail[l] >= 0 && fuse_head[m->block_tail[l]] == l) {
+      lp.skipped = true;                   // evaluated inside the kernel of the block's second convolution
+      continue;
+    }
+    if (li.d.kind != AIQ_LAYER_FC && fuse_head[l] >= 0) {
+      // fused block: one job per version of this (second) convolution, carrying the first one's weights
+      const int l1 = fuse_head[l];
+      const LayerInfo& head = m->layers[l1];
+      const LayerInfo& src = m->layers[head.d.input];
+      lp.fused_head = l1;
+      lp.job_first = plan.jobs.size();
+      aiq_status_t st = conv_rs_encode_maps(make_geom(m, head, B), ws + wl.slot_off[src.slot], B,
+                                            plan.lp[head.d.input].n_versions, &lp.maps[0]);
+      if (st != AIQ_OK) return st;
+      plan.versions_total += lp.n_versions - plan.lp[l1].n_versions;   // conv1 runs once per job of the block
+      for (int v = 0; v < lp.n_versions; ++v) {
+        const int bits = std::get<0>(keys[v]);
+        const std::tuple<int, int, int>& k1 = all_keys[l1][std::get<1>(keys[v])];
+        const int bits1 = std::get<0>(k1), vin = std::get<1>(k1);
+        LayerJob j = {};
+        j.in = slot_ptr(head.d.input, vin);
+        j.res = j.in;
+        j.out = slot_ptr(l, v);
+        j.in_version = vin;
+        j.out_version = v;
+        j.w = li.packed[bits_index(bits)];
+        j.scale = li.scales[bits_index(bits)];
+        j.bias = li.bias;
+        j.bits = bits;
+        j.w_pre = head.packed[bits_index(bits1)];
+        j.scale_pre = head.scales[bits_index(bits1)];
+        j.bias_pre = head.bias;
+        j.bits_pre = bits1;
+        plan.jobs.push_back(j);
+        lp.n_tc++;
+        lp.weight_bytes_tc += (double)li.d.cout * (row_bytes(li.K, bits) + 8.0) + (double)head.d.cout * (row_bytes(head.K, bits1) + 8.0);
+      }
+      continue;
+    }
     if (li.d.kind != AIQ_LAYER_FC) {
       lp.job_first = plan.jobs.size();
       // job order: versions the tensor-core kernel takes first, grouped by weight class
@@ -695,7 +772,14 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
       }
       continue;
     }
+    if (lp.skipped) continue;
     const ConvGeom g = make_geom(m, li, B);
+    if (lp.fused_head >= 0) {
+      st = launch_conv_rs_block(g, &lp.maps[0], jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word,
+                                lp.weight_bytes_tc, stream);
+      if (st != AIQ_OK) return st;
+      continue;
+    }
     if (li.d.kind == AIQ_LAYER_DEPTHWISE) {
       st = launch_depthwise(g, jobs_dev + lp.job_first, lp.n_versions, x_chunk, lp.weight_bytes, stream);
       if (st != AIQ_OK) return st;
@@ -742,6 +826,8 @@ extern "C" void aiq_set_eval_options(int chunk, int share_prefix) {
   aiq::g_opt_chunk = chunk > 0 ? chunk : 0;
   aiq::g_opt_share = share_prefix ? 1 : 0;
 }
+
+extern "C" void aiq_set_block_fusion(int on) { aiq::g_opt_fuse = on ? 1 : 0; }
 
 extern "C" void aiq_set_compute_path(int path) {
   aiq::g_opt_path = (path == AIQ_PATH_FP32 || path == AIQ_PATH_TENSOR || path == AIQ_PATH_TENSOR_TILES) ? path : AIQ_PATH_AUTO;

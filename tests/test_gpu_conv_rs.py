@@ -71,3 +71,53 @@ def test_row_streaming_convolution_single_layer(cin, cout, k, stride, hw, res):
             ref = O.forward_scheme(arch, bank, scheme, x)
             assert_logits_close(got, ref, f"{arch['name']} batch {batch} bits {bits}")
     model.close()
+
+
+def test_fused_basic_blocks_equal_the_layer_by_layer_path_bit_for_bit():
+    """ResNet-20: the identity-shortcut blocks of the 16- and 32-channel stages run as one kernel
+    each when every scheme gives them 4 or 8 bits.  The fused kernel does the same arithmetic in
+    the same order as the two layer kernels, so logits and predictions must be identical, and
+    both must match the oracle."""
+    import torch
+    from aiq_workloads import resnet20, one_layer_lowered_schemes, conv_layer_indices
+    aiq = binding()
+    arch = resnet20()
+    params = gen_model(arch, 1234)
+    model = aiq.Model(arch, params)
+    bank = O.build_weight_bank(O.fold_model(arch, params), (4, 8))
+    rng = np.random.default_rng(5)
+    for batch in (5, 40):
+        x = gen_images(batch, 3, 32, 32, 8200 + batch)
+        xd = to_dev(x)
+        for trial in range(3):
+            scheme = rng.choice(np.array([4, 8], np.uint8), 22)
+            aiq.aiq_set_block_fusion(True)
+            fused = model.aiq_forward(scheme, xd).cpu().numpy()
+            launches_fused = aiq.aiq_last_call_stats()["kernel_launches"]
+            aiq.aiq_set_block_fusion(False)
+            plain = model.aiq_forward(scheme, xd).cpu().numpy()
+            launches_plain = aiq.aiq_last_call_stats()["kernel_launches"]
+            aiq.aiq_set_block_fusion(True)
+            assert launches_fused == launches_plain - 5              # five blocks fold two launches into one
+            assert np.array_equal(fused.view(np.uint32), plain.view(np.uint32))
+            assert_logits_close(fused, O.forward_scheme(arch, bank, scheme, x), f"fused blocks batch {batch}")
+    # a scheme with a 16-bit layer inside a block: that block is not fused, the others are
+    scheme = np.full(22, 8, np.uint8)
+    scheme[2] = 16
+    x = gen_images(9, 3, 32, 32, 8300)
+    bank16 = O.build_weight_bank(O.fold_model(arch, params), (8, 16))
+    got = model.aiq_forward(scheme, to_dev(x)).cpu().numpy()
+    assert_logits_close(got, O.forward_scheme(arch, bank16, scheme, x), "one block unfused")
+    # evaluator: counts and predictions with and without fusion
+    x = gen_images(100, 3, 32, 32, 8400)
+    labels = O.predict(O.forward_scheme(arch, bank, np.full(22, 8, np.uint8), x))
+    schemes = one_layer_lowered_schemes(22, conv_layer_indices(arch))
+    res = []
+    for on in (True, False):
+        aiq.aiq_set_block_fusion(on)
+        preds = torch.full((21, 100), -1, dtype=torch.int32, device="cuda")
+        acc, counts = model.aiq_eval_schemes(schemes, to_dev(x), to_dev(labels), preds=preds, chunk=48)
+        res.append((counts.copy(), preds.cpu().numpy()))
+    aiq.aiq_set_block_fusion(True)
+    assert np.array_equal(res[0][0], res[1][0]) and np.array_equal(res[0][1], res[1][1])
+    model.close()
