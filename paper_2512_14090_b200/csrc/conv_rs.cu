@@ -610,17 +610,17 @@ conv_rs_block_kernel(const __grid_constant__ CUtensorMap in_map, RbParams p, con
   if (tid == 0) {
     for (int i = 0; i < kRbMaxIn; ++i) {
       mbar_init(bar_in_full + 8 * i, 1);
-      mbar_init(bar_in_free + 8 * i, 1 + 8);           // conv1's MMAs retired + the eight shortcut readers
+      mbar_init(bar_in_free + 8 * i, 1 + 4);           // conv1's MMAs retired + the four shortcut readers of the row
     }
     for (int i = 0; i < kRbMaxMid; ++i) {
-      mbar_init(bar_mid_full + 8 * i, 8);              // the eight warps of the first epilogue
+      mbar_init(bar_mid_full + 8 * i, 4);              // the four warps of the first epilogue that take the row
       mbar_init(bar_mid_free + 8 * i, 1);
     }
     for (int i = 0; i < R; ++i) {
       mbar_init(bar_a1_full + 8 * i, 1);
-      mbar_init(bar_a1_empty + 8 * i, 8);
+      mbar_init(bar_a1_empty + 8 * i, 4);
       mbar_init(bar_a2_full + 8 * i, 1);
-      mbar_init(bar_a2_empty + 8 * i, 8);
+      mbar_init(bar_a2_empty + 8 * i, 4);
     }
     mbar_init(bar_w, 1);
     *s_abort = 0;
@@ -727,67 +727,82 @@ conv_rs_block_kernel(const __grid_constant__ CUtensorMap in_map, RbParams p, con
       if (rr.w4.z >> 8) umma_commit(bar_acc_full + 8 * (((rr.w4.z >> 8) - 1u) & (uint32_t)(R - 1)));
     }
   } else {
+    // Each quarter of the accumulator lanes has two warps per epilogue; they take alternate rows, and
+    // a warp finishes both 16-channel units of its row, so two rows per epilogue are in flight.
     const bool second = warp >= 11;
     const int qd = warp & 3;
-    const int h = ((second ? warp - 11 : warp - 3) >> 2);       // 0 or 1: the unit of a row this warp takes
+    const int h = ((second ? warp - 11 : warp - 3) >> 2);       // 0 or 1: the parity of the rows this warp takes
     const int l = qd * 32 + lane;
     const int x_local = l >> 3, img = l & 7;
-    constexpr int chunks = N / 16;
-    const int xt = h / chunks, c0 = (h - xt * chunks) * 16;
-    const int x = xt * 16 + x_local;
-    const int ph = c0 >> 3;                                      // first hi plane of the chunk
+    constexpr int chunks = N / 16;                               // units of a row: (column tile, chunk), two in all
     constexpr int lo_plane0 = C / 8;
     const uint32_t bar_acc_full = second ? bar_a2_full : bar_a1_full;
     const uint32_t bar_acc_empty = second ? bar_a2_empty : bar_a1_empty;
-    const uint32_t t_col = (second ? 256u : 0u) + (uint32_t)(xt * R * N + c0);
-    const float* scale = s_coef + (second ? 2 * N : 0) + c0;
-    const float* bias = s_coef + (second ? 3 * N : N) + c0;
-    // offset of this lane's (column, image) cell inside a ring stage, first hi plane of its chunk
-    const uint32_t cell = (uint32_t)ph * (uint32_t)p.a_lbo + (uint32_t)(x + 1) * 128u + (uint32_t)img * 16u;
+    const float* scale = s_coef + (second ? 2 * N : 0);
+    const float* bias = s_coef + (second ? 3 * N : N);
     const size_t plane_bytes = 128, px_bytes = (size_t)(C / 4) * 128;
     uint8_t* out_base = static_cast<uint8_t*>(job.out);
-    for (int g = 0; g < total && alive; ++g) {
+    // per unit: accumulator column and offset of this lane's cell inside a ring stage (first hi plane of the chunk)
+    uint32_t t_col[2], cell[2];
+    int ux[2], uph[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int xt = u / chunks, c0 = (u - xt * chunks) * 16;
+      ux[u] = xt * 16 + x_local;
+      uph[u] = c0 >> 3;
+      t_col[u] = (second ? 256u : 0u) + (uint32_t)(xt * R * N + c0);
+      cell[u] = (uint32_t)uph[u] * (uint32_t)p.a_lbo + (uint32_t)(ux[u] + 1) * 128u + (uint32_t)img * 16u;
+    }
+    for (int g = h; g < total && alive; g += 2) {
       const int il = g / p.H, y = g - il * p.H;
       const int slot = g & (R - 1);
-      uint32_t v[16];
+      uint32_t v0[16], v1[16];
       uint32_t hi[8], lo[8];
+      alive = mbar_wait_warp(bar_acc_full + 8 * slot, (g / R) & 1, s_abort, p.error_flag);
+      if (!alive) break;
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(slot * N);
+      tmem_ld16(t_row + t_col[0], v0);
+      tmem_ld16(t_row + t_col[1], v1);
       if (!second) {
         const uint32_t ms = (uint32_t)(g % S_mid), mphase = (uint32_t)((g / S_mid) & 1);
-        alive = mbar_wait_warp(bar_acc_full + 8 * slot, (g / R) & 1, s_abort, p.error_flag);
-        if (!alive) break;
-        tc_fence_after();
-        tmem_ld16(tmem_base + ((uint32_t)(qd * 32) << 16) + t_col + (uint32_t)(slot * N), v);
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_acc_empty + 8 * slot);
-        rs_finish_unit(v, scale, bias, nullptr, false, AIQ_ACT_RELU, hi, lo);
         // the stage of the intermediate ring must have been read by conv2's MMAs of its last occupant
         alive = mbar_wait_warp(bar_mid_free + 8 * ms, mphase ^ 1u, s_abort, p.error_flag);
         if (!alive) break;
-        uint8_t* dst = mid_ring + ms * p.stage_bytes + cell;
-        *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(dst + p.a_lbo) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-        *reinterpret_cast<uint4*>(dst + lo_plane0 * p.a_lbo) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        *reinterpret_cast<uint4*>(dst + (lo_plane0 + 1) * p.a_lbo) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int c0 = (u % chunks) * 16;
+          rs_finish_unit(u == 0 ? v0 : v1, scale + c0, bias + c0, nullptr, false, AIQ_ACT_RELU, hi, lo);
+          uint8_t* dst = mid_ring + ms * p.stage_bytes + cell[u];
+          *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(dst + p.a_lbo) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+          *reinterpret_cast<uint4*>(dst + lo_plane0 * p.a_lbo) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          *reinterpret_cast<uint4*>(dst + (lo_plane0 + 1) * p.a_lbo) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_mid_full + 8 * ms);
       } else {
         const uint32_t is = (uint32_t)(g % S_in), iphase = (uint32_t)((g / S_in) & 1);
-        alive = mbar_wait_warp(bar_acc_full + 8 * slot, (g / R) & 1, s_abort, p.error_flag);
-        if (!alive) break;
-        tc_fence_after();
-        tmem_ld16(tmem_base + ((uint32_t)(qd * 32) << 16) + t_col + (uint32_t)(slot * N), v);
         // shortcut: the block input at the same row, still in the input ring (its copy completed long
         // ago; observing the barrier makes the data visible to this thread)
         alive = mbar_wait_warp(bar_in_full + 8 * is, iphase, s_abort, p.error_flag);
-        uint4 rres[4];
-        const uint8_t* src = in_ring + is * p.stage_bytes + cell;
-        rres[0] = *reinterpret_cast<const uint4*>(src);
-        rres[1] = *reinterpret_cast<const uint4*>(src + p.a_lbo);
-        rres[2] = *reinterpret_cast<const uint4*>(src + lo_plane0 * p.a_lbo);
-        rres[3] = *reinterpret_cast<const uint4*>(src + (lo_plane0 + 1) * p.a_lbo);
+        uint4 r0[4], r1[4];
+        {
+          const uint8_t* src = in_ring + is * p.stage_bytes;
+          r0[0] = *reinterpret_cast<const uint4*>(src + cell[0]);
+          r0[1] = *reinterpret_cast<const uint4*>(src + cell[0] + p.a_lbo);
+          r0[2] = *reinterpret_cast<const uint4*>(src + cell[0] + lo_plane0 * p.a_lbo);
+          r0[3] = *reinterpret_cast<const uint4*>(src + cell[0] + (lo_plane0 + 1) * p.a_lbo);
+          r1[0] = *reinterpret_cast<const uint4*>(src + cell[1]);
+          r1[1] = *reinterpret_cast<const uint4*>(src + cell[1] + p.a_lbo);
+          r1[2] = *reinterpret_cast<const uint4*>(src + cell[1] + lo_plane0 * p.a_lbo);
+          r1[3] = *reinterpret_cast<const uint4*>(src + cell[1] + (lo_plane0 + 1) * p.a_lbo);
+        }
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
@@ -796,13 +811,18 @@ conv_rs_block_kernel(const __grid_constant__ CUtensorMap in_map, RbParams p, con
           mbar_arrive(bar_in_free + 8 * is);
         }
         if (!alive) break;
-        rs_finish_unit(v, scale, bias, rres, true, AIQ_ACT_RELU, hi, lo);
         const int item = (int)blockIdx.x + il * (int)gridDim.x;
-        uint8_t* dst = out_base + (((size_t)item * p.H + y) * p.W + x) * px_bytes + (size_t)ph * plane_bytes + (size_t)img * 16;
-        *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(dst + plane_bytes) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-        *reinterpret_cast<uint4*>(dst + (size_t)lo_plane0 * plane_bytes) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        *reinterpret_cast<uint4*>(dst + (size_t)(lo_plane0 + 1) * plane_bytes) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        uint8_t* row_dst = out_base + ((size_t)item * p.H + y) * p.W * px_bytes + (size_t)img * 16;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int c0 = (u % chunks) * 16;
+          rs_finish_unit(u == 0 ? v0 : v1, scale + c0, bias + c0, u == 0 ? r0 : r1, true, AIQ_ACT_RELU, hi, lo);
+          uint8_t* dst = row_dst + (size_t)ux[u] * px_bytes + (size_t)uph[u] * plane_bytes;
+          *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(dst + plane_bytes) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+          *reinterpret_cast<uint4*>(dst + (size_t)lo_plane0 * plane_bytes) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          *reinterpret_cast<uint4*>(dst + (size_t)(lo_plane0 + 1) * plane_bytes) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        }
       }
     }
   }
