@@ -279,13 +279,16 @@ aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t* schemes, 
  * evaluates every scheme independently. */
 void aiq_set_eval_options(int chunk, int share_prefix);
 
-/* Block fusion (process-wide, default on; results never depend on it).  On networks stored for the
- * row-streaming kernel, a basic block out = relu(conv2(relu(conv1(x))) + x) with two 3x3
- * convolutions of 16 or 32 channels runs as one kernel whenever every scheme of the call gives both
- * convolutions 4 or 8 bits: the intermediate tensor then stays in shared memory (the paper's
- * searches only pay off if a candidate evaluation is cheap, Section 2.2).  0 runs every layer as a
- * kernel of its own. */
-void aiq_set_block_fusion(int on);
+/* Kernel fusion on networks stored for the row-streaming kernel (process-wide, both default on; the
+ * paper's searches only pay off if a candidate evaluation is cheap, Section 2.2).
+ *   blocks: a basic block out = relu(conv2(relu(conv1(x))) + x) with two 3x3 convolutions of 16 or 32
+ *           channels runs as one kernel whenever every scheme of the call gives both convolutions 4 or
+ *           8 bits: the intermediate tensor stays in shared memory.  Results are bit-identical to the
+ *           layer-by-layer path.
+ *   pool:   the classifier's global average pool is taken in the epilogue of the convolution that
+ *           produces its input; that tensor is then never stored.  Sums are formed in a fixed order
+ *           (run-to-run identical); they differ from the separate pooling kernel's in the last bits. */
+void aiq_set_fusion(int blocks, int pool);
 
 /* Compute path of models created after the call (process-wide; the paper has no kernels,
  * Section 3 runs stock PyTorch, so this is an implementation choice, not a step of AIQ):

@@ -24,7 +24,7 @@ EXPORTS = [
     "aiq_quantize_layer", "aiq_qlinear", "aiq_qlinear_workspace_bytes", "aiq_model_bytes", "aiq_model_create",
     "aiq_model_destroy", "aiq_model_num_layers", "aiq_model_num_classes",
     "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
-    "aiq_eval_schemes", "aiq_set_eval_options", "aiq_set_block_fusion", "aiq_last_call_stats", "aiq_scheme_ai",
+    "aiq_eval_schemes", "aiq_set_eval_options", "aiq_set_fusion", "aiq_last_call_stats", "aiq_scheme_ai",
     "aiq_profile_start", "aiq_profile_stop", "aiq_forward_static",
     "aiq_set_compute_path", "aiq_model_status", "aiq_debug_expire_wait", "aiq_search_greedy", "aiq_search_coordinate_descent",
 ]
@@ -110,8 +110,8 @@ def _load():
     lib.aiq_eval_schemes.argtypes = [vp, vp, i32, vp, vp, i32, vp, vp, vp, vp, sz, vp]
     lib.aiq_set_eval_options.restype = None
     lib.aiq_set_eval_options.argtypes = [i32, i32]
-    lib.aiq_set_block_fusion.restype = None
-    lib.aiq_set_block_fusion.argtypes = [i32]
+    lib.aiq_set_fusion.restype = None
+    lib.aiq_set_fusion.argtypes = [i32, i32]
     lib.aiq_last_call_stats.restype = None
     lib.aiq_last_call_stats.argtypes = [C.POINTER(C.c_int64)] * 3
     lib.aiq_search_greedy.restype = i32
@@ -217,8 +217,8 @@ def aiq_set_eval_options(chunk=0, share_prefix=True):
     lib.aiq_set_eval_options(int(chunk), int(bool(share_prefix)))
 
 
-def aiq_set_block_fusion(on=True):
-    lib.aiq_set_block_fusion(int(bool(on)))
+def aiq_set_fusion(blocks=True, pool=True):
+    lib.aiq_set_fusion(int(bool(blocks)), int(bool(pool)))
 
 
 def aiq_set_compute_path(path):

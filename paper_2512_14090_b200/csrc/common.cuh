@@ -142,6 +142,7 @@ struct LayerJob {
   const float* bias_pre;
   int32_t bits_pre;
   int32_t reserved;
+  float* pool;          // fused global average pool: float32 [batch][cout] written instead of `out`, or nullptr
 };
 
 struct ConvGeom {
@@ -192,8 +193,11 @@ aiq_status_t launch_conv_tc(const ConvGeom& g, const void* map, const LayerJob* 
 bool conv_rs_eligible(const ConvGeom& g);
 aiq_status_t conv_rs_encode_maps(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
                                  void* maps_out);
+// pool_jobs: the jobs carry LayerJob::pool; the kernel then writes the global average of its output
+// (float32 [batch][Cout]) instead of the output tensor.  Only where conv_rs_pool_fusable(g).
+bool conv_rs_pool_fusable(const ConvGeom& g);
 aiq_status_t launch_conv_rs(const ConvGeom& g, const void* maps, const LayerJob* jobs_dev, int n_jobs, int batch_capacity,
-                            int32_t* error_flag, double weight_bytes, int weight_bits, cudaStream_t s);
+                            int32_t* error_flag, double weight_bytes, int weight_bits, bool pool_jobs, cudaStream_t s);
 // A whole identity-shortcut basic block (two 3x3 convolutions of C -> C channels) in one kernel; `g`
 // describes either convolution.  Jobs carry both weight sets (LayerJob::w_pre ...).
 bool conv_rs_block_eligible(const ConvGeom& g);

@@ -77,6 +77,8 @@ struct RsParams {
   int a_lbo;              // bytes from one plane (8 channels) to the next
   int xt;                 // column tiles (128 lanes each) per row
   int tmem_cols;          // tensor-memory columns this CTA allocates (512, or 256 with two CTAs per SM)
+  int pool_bytes;         // shared memory for the fused average pool (0: the jobs of this launch do not pool)
+  int batch;              // images of the batch (the last group may hold fewer)
   int32_t* error_flag;
 };
 
@@ -84,17 +86,18 @@ __host__ __device__ constexpr int rs_taps(int ks) { return ks == 3 ? 3 : 1; }
 
 // shared memory regions (base aligned to 1024 bytes)
 struct RsSmem {
-  int ring, weights, scale, bias, rows, bars, total;
+  int ring, weights, scale, bias, rows, pool, bars, total;
 };
-__host__ __device__ inline RsSmem rs_smem(int stages, int stage_bytes, int weight_bytes, int N) {
+__host__ __device__ inline RsSmem rs_smem(int stages, int stage_bytes, int weight_bytes, int N, int pool_bytes = 0) {
   RsSmem s;
   s.ring = 0;
   s.weights = stages * stage_bytes;
   s.scale = s.weights + weight_bytes;
   s.bias = s.scale + N * 4;
   s.rows = (s.bias + N * 4 + 127) / 128 * 128;          // per input row: the MMA program (kRsRowWords words)
-  s.bars = s.rows + kRsMaxRows * kRsRowWords * 4;
-  s.total = s.bars + (2 * kRsMaxStages + 2 * kRsMaxSlots + 1) * 8 + 16;
+  s.pool = s.rows + kRsMaxRows * kRsRowWords * 4;       // partial sums of the fused average pool
+  s.bars = s.pool + pool_bytes;
+  s.total = s.bars + (2 * kRsMaxStages + 2 * kRsMaxSlots + 3) * 8 + 16;
   return s;
 }
 
@@ -291,19 +294,21 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   const int tile_b = KCH * NB * 16;                  // bytes of one weight tile
   const int weight_bytes = PIECES * T * tile_b;
   const int stages = p.n_stages, R = p.n_slots;
-  const RsSmem sm = rs_smem(stages, p.stage_bytes, weight_bytes, N);
+  const RsSmem sm = rs_smem(stages, p.stage_bytes, weight_bytes, N, p.pool_bytes);
   uint8_t* ring = smem;
   uint8_t* wsm = smem + sm.weights;
   float* s_scale = reinterpret_cast<float*>(smem + sm.scale);
   float* s_bias = reinterpret_cast<float*>(smem + sm.bias);
   RowProgram* s_rows = reinterpret_cast<RowProgram*>(smem + sm.rows);
+  float* s_pool = reinterpret_cast<float*>(smem + sm.pool);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
   const uint32_t bar_in_full = smem_u32(bars);
   const uint32_t bar_in_empty = bar_in_full + 8 * kRsMaxStages;
   const uint32_t bar_out_full = bar_in_empty + 8 * kRsMaxStages;
   const uint32_t bar_out_empty = bar_out_full + 8 * kRsMaxSlots;
   const uint32_t bar_w = bar_out_empty + 8 * kRsMaxSlots;
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kRsMaxStages + 2 * kRsMaxSlots + 1);
+  const uint32_t bar_pool = bar_w + 8;               // two rendezvous of the epilogue warps per pooled item
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kRsMaxStages + 2 * kRsMaxSlots + 3);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   const int n_off = (int)blockIdx.z * N;             // first output channel of this slice
   // Epilogue work: per output row and quarter of the lanes, `units` = column tiles x 16-channel
@@ -325,6 +330,8 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       mbar_init(bar_out_empty + 8 * i, 4 * epi_sets);      // one arrival per epilogue warp that reads the row
     }
     mbar_init(bar_w, 1);
+    mbar_init(bar_pool, 4 * WQ);
+    mbar_init(bar_pool + 8, 4 * WQ);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -346,6 +353,7 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     s_scale[i] = job.scale[n_off + i];
     s_bias[i] = job.bias[n_off + i];
   }
+  for (int i = tid; i < p.pool_bytes / 4; i += n_threads) s_pool[i] = 0.f;
   // row programs (one thread per input row)
   if (tid < p.H) s_rows[tid] = rs_row_program<KS, STRIDE>(tid, p.H, p.Ho, N, R);
   bool alive = mbar_wait_warp(bar_w, 0, s_abort, p.error_flag);
@@ -459,6 +467,8 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     const uint8_t* res_base = static_cast<const uint8_t*>(job.res);
     uint8_t* out_base = static_cast<uint8_t*>(job.out);
     const int lo_plane0 = p.cout_total / 8;
+    const bool pooling = p.pool_bytes > 0 && job.pool != nullptr;
+    const float pool_scale = 1.0f / (float)(p.Ho * p.Wo);
     // this warp's units of a row and its rows of an item
     const int unit0 = units >= WQ ? h : h % units;
     const int unit_step = units >= WQ ? WQ : units;
@@ -516,11 +526,57 @@ conv_rs_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         rs_finish_unit(v, s_scale + c0, s_bias + c0, rres, res_base != nullptr, p.act, hi, lo);
         // the residual registers are free again: request the first unit of this warp's next row
         if (res_base && u + unit_step >= units && k + 1 < total) load_res(k + 1, unit0, rres);
+        if (pooling) {
+          // Fused global average pool: the stored value hi + lo of each of the 16 channels, summed
+          // over the columns this warp holds (lanes that differ in the column bits), then added to
+          // this warp's partial sums [image][16 channels] in shared memory.  The tensor is not stored.
+          float* mine = s_pool + ((size_t)(warp - 2) * Gout + img) * 16;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            float a = __uint_as_float(hi[e] << 16) + __uint_as_float(lo[e] << 16);
+            float b = __uint_as_float(hi[e] & 0xFFFF0000u) + __uint_as_float(lo[e] & 0xFFFF0000u);
+            for (int o = Gout; o < 32; o <<= 1) {
+              a += __shfl_xor_sync(0xffffffffu, a, o);
+              b += __shfl_xor_sync(0xffffffffu, b, o);
+            }
+            // channel of word e of [hi plane 0 | hi plane 1]: words 0-3 = channels 0-7, 4-7 = channels 8-15
+            if (lane < Gout) { mine[2 * e] += a; mine[2 * e + 1] += b; }
+          }
+        } else {
         uint8_t* dst = out_base + row_off + uoff;
         *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
         *reinterpret_cast<uint4*>(dst + plane_bytes) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
         *reinterpret_cast<uint4*>(dst + (size_t)lo_plane0 * plane_bytes) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         *reinterpret_cast<uint4*>(dst + (size_t)(lo_plane0 + 1) * plane_bytes) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        }
+      }
+      if (pooling && (k + 1) % rows_mine == 0) {
+        // last row of an item for this warp: once all epilogue warps are here, the partial sums of the
+        // warps that hold a channel's chunk are added in a fixed order and the means leave for global memory
+        const int n_epi = n_threads - 64;
+        const uint32_t pool_parity = (uint32_t)(il & 1);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_pool);
+        alive = mbar_wait_warp(bar_pool, pool_parity, s_abort, p.error_flag);
+        if (!alive) break;
+        const int item = (int)blockIdx.x + il * (int)gridDim.x;
+        for (int i = tid - 64; i < Gout * N; i += n_epi) {
+          const int im = i / N, c = i - im * N;
+          float sum = 0.f;
+          for (int e = 0; e < 4 * WQ; ++e) {
+            const int eh = e >> 2;                                    // index of warp e among the warps of its quarter
+            const int eu = units >= WQ ? eh : eh % units;             // its unit
+            if ((eu % chunks) * 16 == (c & ~15)) sum += s_pool[((size_t)e * Gout + im) * 16 + (c & 15)];
+          }
+          const int b = item * Gout + im;
+          if (b < p.batch) job.pool[(size_t)b * p.cout_total + n_off + c] = sum * pool_scale;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_pool + 8);
+        alive = mbar_wait_warp(bar_pool + 8, pool_parity, s_abort, p.error_flag);
+        if (!alive) break;
+        for (int i = lane; i < Gout * 16; i += 32) s_pool[(size_t)(warp - 2) * Gout * 16 + i] = 0.f;
+        __syncwarp();
       }
     }
   }
@@ -911,70 +967,70 @@ int rs_weight_bytes(const ConvGeom& g, int weight_bits) {
   return pieces * rs_taps(g.ks) * (g.Cin / 8) * (g.ks == 3 ? 3 : 1) * n * 16;
 }
 
-// ring depth that fits beside the weights, or 0
-int rs_stages(const ConvGeom& g, const RsShape& s, int weight_bits, int smem_limit) {
-  const int n = g.Cout / rs_weight_slices(g, weight_bits);
-  const int packed = n * (int)row_bytes(g.K, weight_bits <= 8 ? 8 : weight_bits);
-  for (int st = kRsMaxStages; st >= 2; --st)
-    if (rs_smem(st, s.stage_bytes, rs_weight_bytes(g, weight_bits), n).total + 1024 <= smem_limit &&
-        packed <= st * s.stage_bytes)
-      return st;
-  return 0;
+// Launch configuration of one layer and weight class.
+struct RsConfig { int slices, N, occ, stages, slots, threads, tmem_cols, pool_bytes, smem_bytes; bool ok; };
+
+RsConfig rs_config(const ConvGeom& g, const RsShape& sh, int weight_bits, int smem_optin, bool pool) {
+  RsConfig c = {};
+  c.slices = rs_weight_slices(g, weight_bits);
+  c.N = g.Cout / c.slices;
+  const int wbytes = rs_weight_bytes(g, weight_bits);
+  const int packed = c.N * (int)row_bytes(g.K, weight_bits <= 8 ? 8 : weight_bits);
+  // Two CTAs per SM where two rings of at least three input rows and two copies of the weights fit
+  // (the 16- and 32-channel layers), else one CTA with as deep a ring as fits.
+  const int per_cta = (smem_optin + 1024) / 2 - 1024;   // an SM holds the opt-in limit + 1 KB; each CTA reserves 1 KB
+  auto fits = [&](int st, int limit, int pool_bytes) {
+    return rs_smem(st, sh.stage_bytes, wbytes, c.N, pool_bytes).total + 1024 <= limit && packed <= st * sh.stage_bytes;
+  };
+  for (int occ = 2; occ >= 1 && !c.stages; --occ) {
+    const int threads = (2 + (occ == 2 ? 8 : kRsMaxEpiWarps)) * 32;
+    const int pool_bytes = pool ? (threads / 32 - 2) * sh.Gout * 16 * 4 : 0;
+    // output rows in flight: a power of two that divides the rows of an item (the slot of a row then
+    // does not depend on the item) and fits the CTA's share of tensor memory
+    const int tmem_cols = 512 / occ;
+    int slots = kRsMaxSlots;
+    while (slots > 4 && (sh.xt * slots * c.N > tmem_cols || g.Ho % slots != 0)) slots >>= 1;
+    if (sh.xt * slots * c.N > tmem_cols || g.Ho % slots != 0) continue;
+    for (int st = kRsMaxStages; st >= (occ == 2 ? 3 : 2); --st)
+      if (fits(st, occ == 2 ? per_cta : smem_optin, pool_bytes)) {
+        c.occ = occ; c.stages = st; c.slots = slots; c.threads = threads; c.tmem_cols = tmem_cols; c.pool_bytes = pool_bytes;
+        c.smem_bytes = rs_smem(st, sh.stage_bytes, wbytes, c.N, pool_bytes).total + 1024;
+        break;
+      }
+  }
+  c.ok = c.stages > 0;
+  return c;
 }
 
 template <int C, int KS, int STRIDE, int PIECES>
 aiq_status_t launch_rs(const ConvGeom& g, const RsShape& sh, const CUtensorMap* maps, const LayerJob* jobs_dev, int n_jobs,
-                       int batch_capacity, int32_t* error_flag, double weight_bytes, int weight_bits, cudaStream_t s) {
+                       int batch_capacity, int32_t* error_flag, double weight_bytes, int weight_bits, bool pool_jobs,
+                       cudaStream_t s) {
   DeviceProps props;
   if (aiq_status_t st = current_device_props(&props)) return st;
-  const int slices = rs_weight_slices(g, weight_bits);
-  const int N = g.Cout / slices;
-  const int stages = rs_stages(g, sh, weight_bits, props.smem_optin);
-  if (!stages) return set_error(AIQ_ERR_SHAPE, "conv_rs: shared memory does not fit (%d bytes per input row)", sh.stage_bytes);
+  const RsConfig c = rs_config(g, sh, weight_bits, props.smem_optin, pool_jobs);
+  if (!c.ok) return set_error(AIQ_ERR_SHAPE, "conv_rs: shared or tensor memory does not fit (%d bytes per input row)", sh.stage_bytes);
   RsParams p = {};
-  p.H = g.H; p.W = g.W; p.Ho = g.Ho; p.Wo = g.Wo; p.N = N; p.cout_total = g.Cout; p.act = g.act;
+  p.H = g.H; p.W = g.W; p.Ho = g.Ho; p.Wo = g.Wo; p.N = c.N; p.cout_total = g.Cout; p.act = g.act;
   p.gmode = sh.gmode;
   p.n_items = rs_padded_batch(g.B) / sh.Gout;
   p.rows_per_version = rs_padded_batch(batch_capacity) / sh.Gin * g.H;
-  // Two CTAs per SM where two rings of at least three input rows and two copies of the weights fit
-  // (the 16- and 32-channel layers), else one.
-  const int wbytes = rs_weight_bytes(g, weight_bits);
-  int occ = 1, st2 = 0;
-  {
-    const int per_cta = (props.smem_optin + 1024) / 2 - 1024;      // an SM holds the opt-in limit + 1 KB; each CTA reserves 1 KB
-    const int packed = N * (int)row_bytes(g.K, weight_bits <= 8 ? 8 : weight_bits);
-    for (int st = kRsMaxStages; st >= 3 && !st2; --st)
-      if (rs_smem(st, sh.stage_bytes, wbytes, N).total + 1024 <= per_cta && packed <= st * sh.stage_bytes) st2 = st;
-    if (st2) occ = 2;
-  }
-  const int stages_used = occ == 2 ? st2 : stages;
-  p.n_stages = stages_used;
-  p.tmem_cols = 512 / occ;
-  // output rows in flight: a power of two that divides the rows of an item (the slot of a row then
-  // does not depend on the item) and fits the CTA's share of tensor memory
-  int slots = kRsMaxSlots;
-  while (slots > 4 && (sh.xt * slots * N > p.tmem_cols || g.Ho % slots != 0)) slots >>= 1;
-  if (sh.xt * slots * N > p.tmem_cols && occ == 2) {             // too wide for half of tensor memory: one CTA per SM
-    occ = 1; p.n_stages = stages; p.tmem_cols = 512;
-    slots = kRsMaxSlots;
-    while (slots > 4 && (sh.xt * slots * N > 512 || g.Ho % slots != 0)) slots >>= 1;
-  }
-  if (sh.xt * slots * N > p.tmem_cols) return set_error(AIQ_ERR_SHAPE, "conv_rs: %d column tiles of %d channels exceed tensor memory", sh.xt, N);
-  p.n_slots = slots;
+  p.n_stages = c.stages; p.n_slots = c.slots; p.tmem_cols = c.tmem_cols;
   p.K = g.K; p.stage_bytes = sh.stage_bytes; p.a_lbo = sh.a_lbo; p.xt = sh.xt;
   for (int t = 0; t < 3; ++t) p.a_tap_off[t] = sh.a_tap_off[t];
   p.error_flag = error_flag;
-  const int smem_bytes = rs_smem(p.n_stages, sh.stage_bytes, wbytes, N).total + 1024;
-  const int threads = (2 + (occ == 2 ? 8 : kRsMaxEpiWarps)) * 32;
+  p.batch = g.B;
+  p.pool_bytes = c.pool_bytes;
   AIQ_ENSURE_DYNAMIC_SMEM((conv_rs_kernel<C, KS, STRIDE, PIECES>), props.smem_optin);
-  int ctas = occ * props.n_sms / (n_jobs * slices);
+  int ctas = c.occ * props.n_sms / (n_jobs * c.slices);
   if (ctas > p.n_items) ctas = p.n_items;
   if (ctas < 1) ctas = 1;
   {
     LaunchScope scope(AIQ_KERNEL_CONV_TC, s,
                       2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(g.ks * g.ks * g.Cin) * n_jobs,
-                      weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W + (double)g.B * g.Ho * g.Wo * g.Cout));
-    conv_rs_kernel<C, KS, STRIDE, PIECES><<<dim3(ctas, n_jobs, slices), threads, smem_bytes, s>>>(maps[0], maps[1], p, jobs_dev);
+                      weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
+                                                     (pool_jobs ? 0.0 : (double)g.B * g.Ho * g.Wo * g.Cout)));
+    conv_rs_kernel<C, KS, STRIDE, PIECES><<<dim3(ctas, n_jobs, c.slices), c.threads, c.smem_bytes, s>>>(maps[0], maps[1], p, jobs_dev);
   }
   AIQ_LAUNCH_CHECK("conv_rs");
   return AIQ_OK;
@@ -1032,9 +1088,21 @@ bool conv_rs_eligible(const ConvGeom& g) {
   int smem_limit = 227 * 1024;
   if (current_device_props(&props) == AIQ_OK) smem_limit = props.smem_optin;
   for (int bits : {8, 16, 32})
-    if (!rs_stages(g, s, bits, smem_limit)) return false;
-  const int n32 = g.Cout / rs_weight_slices(g, 32);
-  return s.xt * 4 * g.Cout <= 512 && s.xt * 4 * n32 <= 512;
+    if (!rs_config(g, s, bits, smem_limit, false).ok) return false;
+  return true;
+}
+
+// The average pool can ride in the epilogue when every warp of the epilogue finishes one unit of a row.
+bool conv_rs_pool_fusable(const ConvGeom& g) {
+  RsShape s;
+  if (!rs_shape(g, &s) || s.gmode == 2) return false;
+  DeviceProps props;
+  if (current_device_props(&props) != AIQ_OK) return false;
+  for (int bits : {8, 16, 32}) {
+    const RsConfig c = rs_config(g, s, bits, props.smem_optin, true);
+    if (!c.ok || s.xt * (c.N / 16) > (c.threads / 32 - 2) / 4) return false;
+  }
+  return true;
 }
 
 aiq_status_t conv_rs_encode_maps(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
@@ -1085,11 +1153,11 @@ aiq_status_t conv_rs_encode_maps(const ConvGeom& g, const void* slot_base, int b
 }
 
 aiq_status_t launch_conv_rs(const ConvGeom& g, const void* maps, const LayerJob* jobs_dev, int n_jobs, int batch_capacity,
-                            int32_t* error_flag, double weight_bytes, int weight_bits, cudaStream_t s) {
+                            int32_t* error_flag, double weight_bytes, int weight_bits, bool pool_jobs, cudaStream_t s) {
   RsShape sh;
   if (!rs_shape(g, &sh)) return set_error(AIQ_ERR_SHAPE, "conv_rs: layer shape is not supported");
   const CUtensorMap* m = static_cast<const CUtensorMap*>(maps);
-#define AIQ_RS_ARGS g, sh, m, jobs_dev, n_jobs, batch_capacity, error_flag, weight_bytes, weight_bits, s
+#define AIQ_RS_ARGS g, sh, m, jobs_dev, n_jobs, batch_capacity, error_flag, weight_bytes, weight_bits, pool_jobs, s
 #define AIQ_RS_KS(C_, P_)                                                                              \
   do {                                                                                                \
     if (g.ks == 3) return g.stride == 1 ? launch_rs<C_, 3, 1, P_>(AIQ_RS_ARGS) : launch_rs<C_, 3, 2, P_>(AIQ_RS_ARGS); \

@@ -25,7 +25,8 @@ static thread_local int64_t t_launches = 0, t_layer_evals = 0, t_layer_evals_uns
 static std::atomic<int> g_opt_chunk{0};
 static std::atomic<int> g_opt_share{1};
 static std::atomic<int> g_opt_path{AIQ_PATH_AUTO};
-static std::atomic<int> g_opt_fuse{1};
+static std::atomic<int> g_opt_fuse{1};        // basic blocks as one kernel
+static std::atomic<int> g_opt_fuse_pool{1};   // average pool inside the last convolution's epilogue
 
 aiq_status_t set_error(aiq_status_t status, const char* fmt, ...) {
   va_list ap;
@@ -132,6 +133,7 @@ struct aiq_model {
   int32_t* status_word;              // device word raised by a kernel whose bounded wait expired
   std::vector<int> block_tail;       // per layer: the second convolution of the basic block this layer opens
                                      // (the pair can run as one kernel), or -1
+  int pool_layer;                    // the layer whose epilogue can do the classifier's average pool, or -1
 };
 
 namespace aiq {
@@ -350,6 +352,7 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
   // identity-shortcut basic blocks that the fused block kernel takes: conv1 (3x3, ReLU) feeds only conv2
   // (3x3, ReLU) and conv2 adds conv1's input
   m->block_tail.assign(m->layers.size(), -1);
+  m->pool_layer = -1;
   if (m->act_format == ACT_RS) {
     const int n = (int)m->layers.size();
     std::vector<int> uses(n, 0);
@@ -357,6 +360,11 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
       if (li.d.input >= 0) uses[li.d.input]++;
       if (li.d.residual >= 0) uses[li.d.residual]++;
     }
+    // the classifier's input: pooled inside its producer's epilogue when nothing else reads that tensor
+    const int last = m->layers.back().d.input;
+    if (uses[last] == 1 && m->layers[last].d.input >= 0 && layer_tensor_kind(m, m->layers[last]) == 3 &&
+        conv_rs_pool_fusable(make_geom(m, m->layers[last], 1)))
+      m->pool_layer = last;
     for (int l1 = 0; l1 < n; ++l1) {
       const LayerInfo& a = m->layers[l1];
       if (a.d.kind != AIQ_LAYER_CONV || a.d.input < 0 || a.d.residual >= 0 || a.d.act != AIQ_ACT_RELU || uses[l1] != 1) continue;
@@ -519,6 +527,7 @@ struct LayerPlan {
   int n_tc = 0;                         // leading jobs that run on the tensor-core kernel (4- / 8-bit weights)
   int n_tc16 = 0, n_tc32 = 0;           // then those with 16-bit and with 32-bit weights (tc_kind 1 only)
   int tc_kind = 0;                      // which tensor-core kernel (see layer_tensor_kind)
+  bool pools = false;                   // its jobs write the classifier's pooled input instead of the tensor
   bool skipped = false;                 // first convolution of a fused block: evaluated inside its partner's kernel
   int fused_head = -1;                  // second convolution of a fused block: the layer it absorbs
   double weight_bytes = 0.0;            // packed weights + scales + biases over all jobs
@@ -557,9 +566,10 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
   plan.batch_capacity = B;
   std::vector<std::vector<int>> ver(n, std::vector<int>(S, 0));   // ver[l][s]
   std::vector<std::vector<std::tuple<int, int, int>>> all_keys(n);   // per layer and version: (bits, input version, residual version)
+  const bool fuse = g_opt_fuse.load() != 0;
   // a basic block runs as one kernel when every scheme gives both of its convolutions 4 or 8 bits
   std::vector<int> fuse_head(n, -1);
-  if (g_opt_fuse.load())
+  if (fuse)
     for (int l1 = 0; l1 < n; ++l1) {
       const int l2 = m->block_tail[l1];
       if (l2 < 0) continue;
@@ -567,6 +577,7 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
       for (int s = 0; s < S && ok; ++s) ok = schemes[(size_t)s * n + l1] <= 8 && schemes[(size_t)s * n + l2] <= 8;
       if (ok) fuse_head[l2] = l1;
     }
+  float* const pooled_base = reinterpret_cast<float*>(ws + wl.pooled_off);
   auto slot_ptr = [&](int layer, int version) -> uint8_t* {
     const LayerInfo& li = m->layers[layer];
     const size_t Bslot = m->act_format == ACT_RS ? (size_t)rs_padded_batch(B) : (size_t)B;
@@ -681,6 +692,10 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
         j.scale = li.scales[bi];
         j.bias = li.bias;
         j.bits = bits;
+        if (g_opt_fuse_pool.load() && l == m->pool_layer && fuse_head[l] < 0) {
+          j.pool = pooled_base + (size_t)v * B * li.d.cout;      // the row the classifier reads for this version
+          lp.pools = true;
+        }
         plan.jobs.push_back(j);
         const double wb = (double)li.d.cout * (row_bytes(li.K, bits) + 8.0);
         switch (job_class(bits)) {
@@ -758,8 +773,10 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
     aiq_status_t st;
     if (li.d.kind == AIQ_LAYER_FC) {
       const LayerInfo& src = m->layers[li.d.input];
-      st = launch_avgpool(jobs_dev + lp.pool_first, lp.n_pool, B, src.Ho, src.Wo, src.d.cout, m->act_format, stream);
-      if (st != AIQ_OK) return st;
+      if (!plan.lp[li.d.input].pools) {           // else the producing layer's epilogue has written the pooled rows
+        st = launch_avgpool(jobs_dev + lp.pool_first, lp.n_pool, B, src.Ho, src.Wo, src.d.cout, m->act_format, stream);
+        if (st != AIQ_OK) return st;
+      }
       for (size_t gi = 0; gi < lp.bit_groups.size(); ++gi) {
         const size_t first = lp.job_first + lp.bit_groups[gi].first;
         st = launch_qlinear(jobs_dev + first, &plan.jobs[first], lp.bit_groups[gi].second, li.d.cout, li.K, B, stream);
@@ -787,7 +804,7 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
     }
     auto launch_wide = [&](const LayerJob* jd, int n, double wb, int wbits) -> aiq_status_t {
       return lp.tc_kind == 3
-          ? launch_conv_rs(g, &lp.maps[0], jd, n, plan.batch_capacity, m->status_word, wb, wbits, stream)
+          ? launch_conv_rs(g, &lp.maps[0], jd, n, plan.batch_capacity, m->status_word, wb, wbits, lp.pools, stream)
           : launch_conv_tc(g, &lp.maps[0], jd, n, plan.batch_capacity, m->status_word, wb, wbits, stream);
     };
     if (lp.n_tc > 0) {
@@ -827,7 +844,10 @@ extern "C" void aiq_set_eval_options(int chunk, int share_prefix) {
   aiq::g_opt_share = share_prefix ? 1 : 0;
 }
 
-extern "C" void aiq_set_block_fusion(int on) { aiq::g_opt_fuse = on ? 1 : 0; }
+extern "C" void aiq_set_fusion(int blocks, int pool) {
+  aiq::g_opt_fuse = blocks ? 1 : 0;
+  aiq::g_opt_fuse_pool = pool ? 1 : 0;
+}
 
 extern "C" void aiq_set_compute_path(int path) {
   aiq::g_opt_path = (path == AIQ_PATH_FP32 || path == AIQ_PATH_TENSOR || path == AIQ_PATH_TENSOR_TILES) ? path : AIQ_PATH_AUTO;

@@ -91,13 +91,13 @@ def test_fused_basic_blocks_equal_the_layer_by_layer_path_bit_for_bit():
         xd = to_dev(x)
         for trial in range(3):
             scheme = rng.choice(np.array([4, 8], np.uint8), 22)
-            aiq.aiq_set_block_fusion(True)
+            aiq.aiq_set_fusion(True, True)
             fused = model.aiq_forward(scheme, xd).cpu().numpy()
             launches_fused = aiq.aiq_last_call_stats()["kernel_launches"]
-            aiq.aiq_set_block_fusion(False)
+            aiq.aiq_set_fusion(False, True)
             plain = model.aiq_forward(scheme, xd).cpu().numpy()
             launches_plain = aiq.aiq_last_call_stats()["kernel_launches"]
-            aiq.aiq_set_block_fusion(True)
+            aiq.aiq_set_fusion(True, True)
             assert launches_fused == launches_plain - 5              # five blocks fold two launches into one
             assert np.array_equal(fused.view(np.uint32), plain.view(np.uint32))
             assert_logits_close(fused, O.forward_scheme(arch, bank, scheme, x), f"fused blocks batch {batch}")
@@ -114,10 +114,39 @@ def test_fused_basic_blocks_equal_the_layer_by_layer_path_bit_for_bit():
     schemes = one_layer_lowered_schemes(22, conv_layer_indices(arch))
     res = []
     for on in (True, False):
-        aiq.aiq_set_block_fusion(on)
+        aiq.aiq_set_fusion(on, True)
         preds = torch.full((21, 100), -1, dtype=torch.int32, device="cuda")
         acc, counts = model.aiq_eval_schemes(schemes, to_dev(x), to_dev(labels), preds=preds, chunk=48)
         res.append((counts.copy(), preds.cpu().numpy()))
-    aiq.aiq_set_block_fusion(True)
+    aiq.aiq_set_fusion(True, True)
     assert np.array_equal(res[0][0], res[1][0]) and np.array_equal(res[0][1], res[1][1])
     model.close()
+
+
+def test_average_pool_in_the_epilogue_matches_the_pooling_kernel():
+    """The classifier's average pool taken inside the last convolution's epilogue (the default) against
+    the separate pooling kernel and against the oracle; batches with a ragged last group."""
+    from aiq_workloads import resnet20, heavy_early_resnet20
+    aiq = binding()
+    for make, seed in ((resnet20, 1234), (heavy_early_resnet20, 4500)):
+        arch = make()
+        L = len(arch["layers"])
+        params = gen_model(arch, seed)
+        model = aiq.Model(arch, params)
+        bank = O.build_weight_bank(O.fold_model(arch, params), (4, 8, 32))
+        for batch, bits in ((1, 8), (19, 4), (48, 32)):
+            x = gen_images(batch, 3, 32, 32, 8500 + batch)
+            scheme = np.full(L, bits, np.uint8)
+            aiq.aiq_set_fusion(True, True)
+            fused = model.aiq_forward(scheme, to_dev(x)).cpu().numpy()
+            n_fused = aiq.aiq_last_call_stats()["kernel_launches"]
+            aiq.aiq_set_fusion(True, False)
+            plain = model.aiq_forward(scheme, to_dev(x)).cpu().numpy()
+            n_plain = aiq.aiq_last_call_stats()["kernel_launches"]
+            aiq.aiq_set_fusion(True, True)
+            assert n_fused == n_plain - 1                        # the pooling kernel is gone
+            ref = O.forward_scheme(arch, bank, scheme, x)
+            assert_logits_close(fused, ref, f"{arch['name']} pooled epilogue batch {batch}")
+            assert_logits_close(plain, ref, f"{arch['name']} pooling kernel batch {batch}")
+            assert np.abs(fused - plain).max() <= 1e-5 * (1.0 + np.abs(plain).max())
+        model.close()
