@@ -55,7 +55,7 @@ def fold_model(arch, params):
 # ----------------------------------------------------------------------------
 # Quantizer (Section 2.1: q_i in Q; Q = {FP32, INT8, INT4}, plus a 16-bit level)
 # ----------------------------------------------------------------------------
-def quantize_rows(W, bits):
+def quantize_rows(W, bits, per_tensor=False):
     """Quantize a folded weight matrix W [N][K] (one row per output channel).
 
     Section 2.1 assigns each layer a bit-width but prints no formula.  Reading:
@@ -65,6 +65,9 @@ def quantize_rows(W, bits):
                    code = clamp(rint(W[n,k] / s_n), -2^(bits-1), 2^(bits-1) - 1)
       bits 16:     IEEE half, round to nearest even; s_n = 1
       bits 32:     unchanged; s_n = 1
+    per_tensor=True is the variant with one scale for the whole tensor (the paper lists
+    per-channel effects as future work in Section 6, so its own experiments most likely used
+    this granularity): amax = max over all of W, every entry of `scales` holds amax / qmax.
     Returns (values, scales): values is int8 codes, float16 or float32; scales float32 [N].
     Non-finite weights raise ValueError.
     """
@@ -83,6 +86,8 @@ def quantize_rows(W, bits):
         return W.astype(np.float16), ones
     qmax = np.float32(2 ** (bits - 1) - 1)
     amax = np.max(np.abs(W), axis=1) if W.shape[1] else np.zeros(n, np.float32)
+    if per_tensor:
+        amax = np.full(n, np.max(amax) if n else 0.0, dtype=np.float32)
     s = (amax / qmax).astype(np.float32)
     s[amax == 0] = np.float32(1.0)
     q = np.rint(W / s[:, None])
@@ -230,13 +235,13 @@ def forward(arch, deq_layers, x):
     return outs[-1]
 
 
-def build_weight_bank(folded, bits_set=ALLOWED_BITS):
+def build_weight_bank(folded, bits_set=ALLOWED_BITS, per_tensor=False):
     """bank[i][bits] = (w_hat, b): a layer's quantized weights depend only on (layer, bits)."""
     bank = []
     for Wf, bf in folded:
         entry = {}
         for bits in bits_set:
-            v, s = quantize_rows(Wf, bits)
+            v, s = quantize_rows(Wf, bits, per_tensor)
             entry[bits] = (dequantize_rows(v, s, bits), bf)
         bank.append(entry)
     return bank

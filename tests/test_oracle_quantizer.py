@@ -204,3 +204,74 @@ def test_fold_identity_case():
                        np.asarray([0.125, 1.0], np.float32), var)
     assert np.array_equal(Wf, W)
     assert bf.tolist() == [0.375, -0.75]
+
+
+# ---------------------------------------------------------------- per-tensor-scale variant
+def _per_tensor_cases():
+    out = []
+    with open(os.path.join(GOLDEN, "quantizer_per_tensor_hand.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            bits, rows, scale, codes, row_codes = [p.strip() for p in line.split("|")]
+            parse = lambda t, conv: [[conv(v) for v in r.split()] for r in t.split("/")]
+            out.append((int(bits), parse(rows, float), float(scale), parse(codes, int), parse(row_codes, int)))
+    return out
+
+
+@pytest.mark.parametrize("bits,rows,scale,codes,row_codes", _per_tensor_cases())
+def test_per_tensor_hand_tables(bits, rows, scale, codes, row_codes):
+    W = np.asarray(rows, dtype=np.float32)
+    v, s = O.quantize_rows(W, bits, per_tensor=True)
+    assert v.tolist() == codes
+    assert s.tolist() == [scale] * len(rows)                 # the one scale, repeated for every row
+    v_row, _ = O.quantize_rows(W, bits)                      # the default granularity differs on these tensors
+    assert v_row.tolist() == row_codes
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_per_tensor_matches_exact_rational_arithmetic_and_bounds(bits):
+    """The tensor flattened to one long row is the per-channel rule applied once: same exact-rational
+    model.  Also: equal to the per-channel result when every row has the same maximum; codes in
+    range with the extremum attained somewhere; |w - s*code| <= s/2 (+ rounding of the product)."""
+    rng = np.random.default_rng(21)
+    W = (rng.standard_normal((9, 13)) * 0.2).astype(np.float32)
+    W[4] *= np.float32(0.01)
+    v, s = O.quantize_rows(W, bits, per_tensor=True)
+    codes, sc = quantize_row_exact(W.reshape(-1), bits)
+    assert all(f32_to_fraction(x) == sc for x in s)
+    assert v.reshape(-1).tolist() == codes
+    qmax = 2 ** (bits - 1) - 1
+    assert np.abs(v).max() == qmax and v.min() >= -(qmax + 1) and v.max() <= qmax
+    w_hat = O.dequantize_rows(v, s, bits)
+    assert np.all(np.abs(W.astype(np.float64) - w_hat.astype(np.float64)) <= float(s[0]) * (0.5 + 1e-6))
+    # rows with a common maximum: both granularities agree
+    W2 = W.copy()
+    W2[:, 0] = np.float32(3.0)
+    a, sa = O.quantize_rows(W2, bits, per_tensor=True)
+    b, sb = O.quantize_rows(W2, bits)
+    assert np.array_equal(a, b) and np.array_equal(sa, sb)
+    # 16 / 32 bits do not depend on the granularity
+    for wide in (16, 32):
+        a, sa = O.quantize_rows(W, wide, per_tensor=True)
+        b, sb = O.quantize_rows(W, wide)
+        assert np.array_equal(a, b) and np.array_equal(sa, sb)
+    # an all-zero tensor keeps scale 1
+    z, sz = O.quantize_rows(np.zeros((3, 5), np.float32), bits, per_tensor=True)
+    assert not z.any() and sz.tolist() == [1.0, 1.0, 1.0]
+
+
+def test_ai_does_not_depend_on_the_scale_granularity():
+    """AI counts weight bytes by bit-width only (Section 1 (i)); per-tensor and per-channel banks of
+    the same scheme have the same analytic intensity, while their accuracies may differ."""
+    from aiq_workloads import resnet20, gen_model, gen_images
+    arch = resnet20()
+    params = gen_model(arch, 1234)
+    folded = O.fold_model(arch, params)
+    x = gen_images(4, 3, 32, 32, 3)
+    bank_c = O.build_weight_bank(folded, (4,))
+    bank_t = O.build_weight_bank(folded, (4,), per_tensor=True)
+    scheme = [4] * 22
+    assert not np.array_equal(O.forward_scheme(arch, bank_c, scheme, x), O.forward_scheme(arch, bank_t, scheme, x))
+    assert O.scheme_ai(arch, scheme) == O.scheme_ai(arch, scheme)      # no bank argument at all: bytes follow q only
