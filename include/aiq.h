@@ -94,6 +94,22 @@ size_t aiq_packed_row_bytes(int K, int bits);   /* 0 for an unsupported bits or 
 aiq_status_t aiq_quantize_layer(const float* W, int N, int K, int bits, void* packed_out,
                                 float* scales_out, int32_t* nonfinite_flag, void* stream);
 
+/* The same quantizer with ONE scale for the whole tensor instead of one per output channel:
+ * amax = max |W[n][k]| over all n and k, s = amax / qmax, every entry of scales_out holds s (so the
+ * forward kernels need no second code path).  The paper prints no quantizer and lists per-channel
+ * effects as future work (Section 6), which makes this the granularity its own experiments most
+ * likely used; the per-channel rule above is this library's default.  16 and 32 bits do not
+ * depend on the granularity.  scratch: device, 4 bytes, 4-byte aligned (holds the tensor maximum
+ * during the call).  Otherwise as aiq_quantize_layer. */
+aiq_status_t aiq_quantize_layer_per_tensor(const float* W, int N, int K, int bits, void* packed_out,
+                                           float* scales_out, int32_t* nonfinite_flag, void* scratch,
+                                           void* stream);
+
+/* Scale granularity of the weight banks of models created after the call (process-wide; default
+ * AIQ_SCALE_PER_CHANNEL).  The analytic AI of a scheme does not depend on it. */
+enum { AIQ_SCALE_PER_CHANNEL = 0, AIQ_SCALE_PER_TENSOR = 1 };
+void aiq_set_scale_granularity(int granularity);
+
 /* ------------------------------------------------------------------------------------
  * Small-batch quantized linear layer - the memory-bound case the method targets
  * (Abstract; Section 5, Roofline paragraph): weight bytes N*K*bits/8 dominate the traffic.

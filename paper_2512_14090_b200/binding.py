@@ -24,7 +24,7 @@ EXPORTS = [
     "aiq_quantize_layer", "aiq_qlinear", "aiq_qlinear_workspace_bytes", "aiq_model_bytes", "aiq_model_create",
     "aiq_model_destroy", "aiq_model_num_layers", "aiq_model_num_classes",
     "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
-    "aiq_eval_schemes", "aiq_set_eval_options", "aiq_set_fusion", "aiq_last_call_stats", "aiq_scheme_ai",
+    "aiq_eval_schemes", "aiq_set_eval_options", "aiq_set_fusion", "aiq_quantize_layer_per_tensor", "aiq_set_scale_granularity", "aiq_last_call_stats", "aiq_scheme_ai",
     "aiq_profile_start", "aiq_profile_stop", "aiq_forward_static",
     "aiq_set_compute_path", "aiq_model_status", "aiq_debug_expire_wait", "aiq_search_greedy", "aiq_search_coordinate_descent",
 ]
@@ -110,6 +110,10 @@ def _load():
     lib.aiq_eval_schemes.argtypes = [vp, vp, i32, vp, vp, i32, vp, vp, vp, vp, sz, vp]
     lib.aiq_set_eval_options.restype = None
     lib.aiq_set_eval_options.argtypes = [i32, i32]
+    lib.aiq_quantize_layer_per_tensor.restype = i32
+    lib.aiq_quantize_layer_per_tensor.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.aiq_set_scale_granularity.restype = None
+    lib.aiq_set_scale_granularity.argtypes = [i32]
     lib.aiq_set_fusion.restype = None
     lib.aiq_set_fusion.argtypes = [i32, i32]
     lib.aiq_last_call_stats.restype = None
@@ -215,6 +219,19 @@ def aiq_qlinear(packed, scales, bias, N, K, bits, x, y, workspace=None, stream=N
 
 def aiq_set_eval_options(chunk=0, share_prefix=True):
     lib.aiq_set_eval_options(int(chunk), int(bool(share_prefix)))
+
+
+SCALE_PER_CHANNEL, SCALE_PER_TENSOR = 0, 1
+
+
+def aiq_set_scale_granularity(granularity):
+    lib.aiq_set_scale_granularity(int(granularity))
+
+
+def aiq_quantize_layer_per_tensor(W, bits, packed_out, scales_out, scratch, nonfinite_flag=None, stream=None):
+    N, K = W.shape
+    _check(lib.aiq_quantize_layer_per_tensor(_dev(W), int(N), int(K), int(bits), _dev(packed_out), _dev(scales_out),
+                                             _dev(nonfinite_flag), _dev(scratch), _stream(stream)))
 
 
 def aiq_set_fusion(blocks=True, pool=True):

@@ -157,8 +157,9 @@ struct ConvGeom {
 aiq_status_t launch_fold_bn(const float* W, const float* gamma, const float* beta, const float* mean,
                             const float* var, int N, int K, float eps, float* Wf, float* bf,
                             cudaStream_t s);
+// tensor_amax: nullptr = one scale per row; else device scratch word and one scale for the whole tensor
 aiq_status_t launch_quantize(const float* W, int N, int K, int bits, void* packed, float* scales,
-                             int32_t* nonfinite_flag, cudaStream_t s);
+                             int32_t* nonfinite_flag, uint32_t* tensor_amax, cudaStream_t s);
 // y[m][n] for every job: in = x [M][K], out = y [M][N]
 aiq_status_t launch_qlinear(const LayerJob* jobs_dev, const LayerJob* single_host, int n_jobs, int N,
                             int K, int M, cudaStream_t s);

@@ -25,6 +25,7 @@ static thread_local int64_t t_launches = 0, t_layer_evals = 0, t_layer_evals_uns
 static std::atomic<int> g_opt_chunk{0};
 static std::atomic<int> g_opt_share{1};
 static std::atomic<int> g_opt_path{AIQ_PATH_AUTO};
+static std::atomic<int> g_opt_per_tensor{0};  // scale granularity of models created afterwards
 static std::atomic<int> g_opt_fuse{1};        // basic blocks as one kernel
 static std::atomic<int> g_opt_fuse_pool{1};   // average pool inside the last convolution's epilogue
 
@@ -390,6 +391,7 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
       return fail(set_error(AIQ_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)));       \
   } while (0)
 
+  const bool per_tensor = g_opt_per_tensor.load() != 0;
   CREATE_TRY(cudaMemsetAsync(flag, 0, 256, stream));
   for (size_t i = 0; i < m->layers.size(); ++i) {
     LayerInfo& li = m->layers[i];
@@ -422,7 +424,8 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
       else CREATE_TRY(cudaMemsetAsync(li.bias, 0, n * 4, stream));
     }
     for (int b = 0; b < 4; ++b) {
-      st = launch_quantize(li.Wf, (int)n, (int)k, kBitsList[b], li.packed[b], li.scales[b], flag, stream);
+      st = launch_quantize(li.Wf, (int)n, (int)k, kBitsList[b], li.packed[b], li.scales[b], flag,
+                           per_tensor ? reinterpret_cast<uint32_t*>(flag + 2) : nullptr, stream);
       if (st != AIQ_OK) return fail(st);
     }
   }
@@ -842,6 +845,10 @@ extern "C" size_t aiq_workspace_bytes(const aiq_model_t* model, int max_batch, i
 extern "C" void aiq_set_eval_options(int chunk, int share_prefix) {
   aiq::g_opt_chunk = chunk > 0 ? chunk : 0;
   aiq::g_opt_share = share_prefix ? 1 : 0;
+}
+
+extern "C" void aiq_set_scale_granularity(int granularity) {
+  aiq::g_opt_per_tensor = granularity == AIQ_SCALE_PER_TENSOR ? 1 : 0;
 }
 
 extern "C" void aiq_set_fusion(int blocks, int pool) {

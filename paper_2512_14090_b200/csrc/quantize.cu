@@ -119,7 +119,7 @@ template <int CACHE, int BITS>
 __global__ void __launch_bounds__(256, CACHE == 1 ? 4 : 3)
 quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad,
                      uint8_t* __restrict__ packed, float* __restrict__ scales,
-                     int32_t* __restrict__ nonfinite_flag) {
+                     int32_t* __restrict__ nonfinite_flag, const uint32_t* __restrict__ tensor_amax) {
   const int n = blockIdx.x;
   const float* row = W + (size_t)n * K;
   const int n_gran = Kpad >> 3;
@@ -168,6 +168,8 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad,
     if (threadIdx.x == 0 && nonfinite_flag) *nonfinite_flag = 1;
     return;
   }
+  // per-tensor variant: the maximum over the whole tensor (computed by tensor_absmax_kernel) sets the scale
+  if (tensor_amax) amax_bits = *tensor_amax;
   const RowQuantizer rq(__uint_as_float(amax_bits), BITS);
   if (threadIdx.x == 0) scales[n] = rq.s;
 
@@ -287,9 +289,19 @@ quantize_stream_kernel(const float* __restrict__ W, int N, int K, uint8_t* __res
   }
 }
 
+// max |w| over a whole tensor, as the integer maximum of the sign-stripped bit patterns (order-free,
+// so atomics give a reproducible result).  *out must be zero before the launch.
+__global__ void tensor_absmax_kernel(const float* __restrict__ W, size_t n, uint32_t* __restrict__ out) {
+  uint32_t m = 0;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    m = max(m, absbits(__ldg(W + i)));
+  m = __reduce_max_sync(0xffffffffu, m);
+  if ((threadIdx.x & 31) == 0 && m) atomicMax(out, m);
+}
+
 template <int BITS>
 aiq_status_t launch_quantize_bits(const float* W, int N, int K, void* packed, float* scales,
-                                  int32_t* nonfinite_flag, cudaStream_t s) {
+                                  int32_t* nonfinite_flag, uint32_t* tensor_amax, cudaStream_t s) {
   const int Kpad = padded_k(K);
   const int n_gran = Kpad / 8;
   uint8_t* p = static_cast<uint8_t*>(packed);
@@ -298,7 +310,15 @@ aiq_status_t launch_quantize_bits(const float* W, int N, int K, void* packed, fl
   DeviceProps props;
   if (aiq_status_t st = current_device_props(&props)) return st;
   const int n_sms = props.n_sms, smem_limit = props.smem_optin;
-  const bool stream_ok = K % 32 == 0 && K >= 2048 && K <= kStreamThreads * 8 * kStreamCache &&
+  if (tensor_amax) {
+    AIQ_CUDA_TRY(cudaMemsetAsync(tensor_amax, 0, 4, s));
+    const size_t n = (size_t)N * K;
+    int blocks = (int)((n + 1023) / 1024);
+    if (blocks > 8 * n_sms) blocks = 8 * n_sms;
+    tensor_absmax_kernel<<<blocks, 256, 0, s>>>(W, n, tensor_amax);
+    AIQ_LAUNCH_CHECK("tensor_absmax");
+  }
+  const bool stream_ok = !tensor_amax && K % 32 == 0 && K >= 2048 && K <= kStreamThreads * 8 * kStreamCache &&
                          N >= 4 * n_sms && ((uintptr_t)W & 15) == 0;
   if (stream_ok) {
     // As many blocks per SM (up to 4) as leave each a ring of at least two rows: the rounding
@@ -322,21 +342,21 @@ aiq_status_t launch_quantize_bits(const float* W, int N, int K, void* packed, fl
   int threads = 32;
   while (threads < 256 && threads < n_gran) threads <<= 1;
   if (n_gran <= threads) {
-    quantize_rows_kernel<1, BITS><<<N, threads, 0, s>>>(W, K, Kpad, p, scales, nonfinite_flag);
+    quantize_rows_kernel<1, BITS><<<N, threads, 0, s>>>(W, K, Kpad, p, scales, nonfinite_flag, tensor_amax);
   } else {
-    quantize_rows_kernel<4, BITS><<<N, threads, 0, s>>>(W, K, Kpad, p, scales, nonfinite_flag);
+    quantize_rows_kernel<4, BITS><<<N, threads, 0, s>>>(W, K, Kpad, p, scales, nonfinite_flag, tensor_amax);
   }
   AIQ_LAUNCH_CHECK("quantize_rows");
   return AIQ_OK;
 }
 
 aiq_status_t launch_quantize(const float* W, int N, int K, int bits, void* packed, float* scales,
-                             int32_t* nonfinite_flag, cudaStream_t s) {
+                             int32_t* nonfinite_flag, uint32_t* tensor_amax, cudaStream_t s) {
   switch (bits) {
-    case 4: return launch_quantize_bits<4>(W, N, K, packed, scales, nonfinite_flag, s);
-    case 8: return launch_quantize_bits<8>(W, N, K, packed, scales, nonfinite_flag, s);
-    case 16: return launch_quantize_bits<16>(W, N, K, packed, scales, nonfinite_flag, s);
-    default: return launch_quantize_bits<32>(W, N, K, packed, scales, nonfinite_flag, s);
+    case 4: return launch_quantize_bits<4>(W, N, K, packed, scales, nonfinite_flag, tensor_amax, s);
+    case 8: return launch_quantize_bits<8>(W, N, K, packed, scales, nonfinite_flag, tensor_amax, s);
+    case 16: return launch_quantize_bits<16>(W, N, K, packed, scales, nonfinite_flag, nullptr, s);
+    default: return launch_quantize_bits<32>(W, N, K, packed, scales, nonfinite_flag, nullptr, s);
   }
 }
 
@@ -373,5 +393,22 @@ extern "C" aiq_status_t aiq_quantize_layer(const float* W, int N, int K, int bit
     return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_quantize_layer: packed_out not 16-byte aligned");
   aiq_status_t st = aiq::check_device_sm100();
   if (st != AIQ_OK) return st;
-  return aiq::launch_quantize(W, N, K, bits, packed_out, scales_out, nonfinite_flag, (cudaStream_t)stream);
+  return aiq::launch_quantize(W, N, K, bits, packed_out, scales_out, nonfinite_flag, nullptr, (cudaStream_t)stream);
+}
+
+extern "C" aiq_status_t aiq_quantize_layer_per_tensor(const float* W, int N, int K, int bits, void* packed_out,
+                                                      float* scales_out, int32_t* nonfinite_flag, void* scratch,
+                                                      void* stream) {
+  if (!aiq::bits_ok(bits))
+    return aiq::set_error(AIQ_ERR_UNSUPPORTED_BITS, "aiq_quantize_layer_per_tensor: bits=%d", bits);
+  if (!W || !packed_out || !scales_out || !scratch)
+    return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_quantize_layer_per_tensor: null pointer");
+  if (N <= 0 || K <= 0)
+    return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_quantize_layer_per_tensor: N=%d K=%d", N, K);
+  if ((((uintptr_t)packed_out) & 15) || (((uintptr_t)scratch) & 3))
+    return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_quantize_layer_per_tensor: packed_out must be 16-byte, scratch 4-byte aligned");
+  aiq_status_t st = aiq::check_device_sm100();
+  if (st != AIQ_OK) return st;
+  return aiq::launch_quantize(W, N, K, bits, packed_out, scales_out, nonfinite_flag, static_cast<uint32_t*>(scratch),
+                              (cudaStream_t)stream);
 }
