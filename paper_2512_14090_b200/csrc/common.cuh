@@ -212,8 +212,9 @@ aiq_status_t conv_pw_tc_encode_map(const ConvGeom& g, const void* slot_base, int
 // store map over the output slot: dims (Cs_out, 2, pixels per version, versions)
 aiq_status_t conv_pw_tc_encode_out_map(const ConvGeom& g, const void* slot_base, int batch_capacity, int n_versions,
                                        void* map_out);
+// weight_bits: 8 (4- or 8-bit codes), 16 or 32 (two bfloat16 pieces per weight); one class per launch
 aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const void* out_map, const LayerJob* jobs_dev, int n_jobs,
-                               int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s);
+                               int batch_capacity, int32_t* error_flag, double weight_bytes, int weight_bits, cudaStream_t s);
 // Test aid: a one-thread kernel whose bounded wait runs out after `limit_cycles` SM clocks; it sets
 // *error_flag to 1 and *observed (optional) to 2, then returns.
 aiq_status_t launch_expire_wait(int32_t* error_flag, long long limit_cycles, int32_t* observed, cudaStream_t s);

@@ -29,6 +29,7 @@ struct PwParams {
   int Nt;                   // output channels per CTA (multiple of 16, <= 128)
   int n_ntiles;
   int act, n_stages;
+  int pieces;               // bfloat16 pieces per weight: 1 (4- / 8-bit codes), 2 (16- / 32-bit weights as hi + lo)
   long long ver_pixels;     // pixels per version of the input slot (capacity * (H + 2) * W)
   int32_t* error_flag;
 };
@@ -40,13 +41,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
-// shared memory: [stage: A_hi | A_lo | B] x n_stages, scale, bias, barriers, tmem ptr, abort flag
-__host__ __device__ inline int pw_stage_bytes(int Nt) { return 2 * kPwATile + Nt * kPwChunk * 2; }
+// shared memory: [stage: A_hi | A_lo | B (one tile per weight piece)] x n_stages, scale, bias, barriers, tmem ptr, abort flag
+__host__ __device__ inline int pw_stage_bytes(int Nt, int pieces) { return 2 * kPwATile + pieces * Nt * kPwChunk * 2; }
 // output staging: per 64-channel group of the N tile one hi and one lo box of 128 pixels x 128 bytes
 __host__ __device__ inline int pw_out_groups(int Nt) { return (Nt + 63) / 64; }
 __host__ __device__ inline int pw_staging_bytes(int Nt) { return pw_out_groups(Nt) * 2 * kPwATile; }
-__host__ __device__ inline int pw_smem_bytes(int Nt, int stages) {
-  return stages * pw_stage_bytes(Nt) + pw_staging_bytes(Nt) + 2 * 128 * 4 + (3 * stages + 4) * 8 + 16;
+__host__ __device__ inline int pw_smem_bytes(int Nt, int stages, int pieces) {
+  return stages * pw_stage_bytes(Nt, pieces) + pw_staging_bytes(Nt) + 2 * 128 * 4 + (3 * stages + 4) * 8 + 16;
 }
 
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
@@ -64,7 +65,7 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
   const LayerJob job = jobs[job_idx];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int stages = p.n_stages, Nt = p.Nt, n0 = ntile * Nt;
-  const int stage_bytes = pw_stage_bytes(Nt);
+  const int stage_bytes = pw_stage_bytes(Nt, p.pieces);
 
   uint8_t* staging = smem + stages * stage_bytes;            // 1024-aligned: every stage is a multiple of 2 KB
   float* s_scale = reinterpret_cast<float*>(staging + pw_staging_bytes(Nt));
@@ -160,8 +161,50 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
       }
     };
     uint2 cur[UPT], nxt[UPT];
-    fetch(0, cur);
     uint32_t stage = 0, phase = 0;
+    if (p.pieces == 2) {
+      // 16- / 32-bit weights: w = hi + lo, hi = bf16(w), lo = bf16(w - hi) (exact for a half, within 2^-17 of
+      // a float32 weight): two B tiles per stage, the MMAs are issued once per piece.  The words come from
+      // L2 when they are needed (no register prefetch: a unit is 16 or 32 bytes here).
+      for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
+        for (int c = 0; c < n_chunks && alive; ++c) {
+          alive = mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+          if (!alive) break;
+          uint8_t* btile = smem + stage * stage_bytes + 2 * kPwATile;
+          for (int u = et; u < n_units; u += 128) {
+            const int nl = u / UPR, cu = u - nl * UPR;
+            const int n = n0 + nl, ch = c * kPwChunk + cu * 8;
+            float w[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[j] = 0.f;
+            if (n < p.Cout && ch < p.Cin) {
+              const uint8_t* src = job.w + (size_t)n * wrow;
+              if (job.bits == 16) {
+                const uint4 r = __ldg(reinterpret_cast<const uint4*>(src + (size_t)ch * 2));
+                const __half2* h2 = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { const float2 f = __half22float2(h2[j]); w[2 * j] = f.x; w[2 * j + 1] = f.y; }
+              } else {
+                const float4 r0 = __ldg(reinterpret_cast<const float4*>(src + (size_t)ch * 4));
+                const float4 r1 = __ldg(reinterpret_cast<const float4*>(src + (size_t)ch * 4) + 1);
+                w[0] = r0.x; w[1] = r0.y; w[2] = r0.z; w[3] = r0.w; w[4] = r1.x; w[5] = r1.y; w[6] = r1.z; w[7] = r1.w;
+              }
+            }
+            uint32_t hi4[4], lo4[4];
+#pragma unroll
+            for (int j = 0; j < 8; j += 2) split_pair(w[j], w[j + 1], hi4[j >> 1], lo4[j >> 1]);
+            const uint32_t off = swizzle_off((uint32_t)(nl * 128 + cu * 16), 7u);
+            *reinterpret_cast<uint4*>(btile + off) = make_uint4(hi4[0], hi4[1], hi4[2], hi4[3]);
+            *reinterpret_cast<uint4*>(btile + Nt * 128 + off) = make_uint4(lo4[0], lo4[1], lo4[2], lo4[3]);
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_b_full + 8 * stage);
+          if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    } else {
+    fetch(0, cur);
     for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
       for (int c = 0; c < n_chunks && alive; ++c) {
         fetch(c + 1 < n_chunks ? c + 1 : 0, nxt);               // next chunk (of this or the next tile)
@@ -185,6 +228,7 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
 #pragma unroll
         for (int i = 0; i < UPT; ++i) cur[i] = nxt[i];
       }
+    }
     }
   }
   else if (warp == 1) {
@@ -219,6 +263,8 @@ conv_pw_tc_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_const
                 const uint64_t bdesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + ((kk * 32) >> 4));
                 umma_bf16(d_tmem, adesc, bdesc, idesc, accumulate);
                 accumulate = 1;
+                if (p.pieces == 2)                  // the lo piece of 16- / 32-bit weights
+                  umma_bf16(d_tmem, adesc, ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + ((Nt * 128 + kk * 32) >> 4)), idesc, 1u);
               }
             }
           }

@@ -714,7 +714,7 @@ aiq_status_t conv_pw_tc_encode_out_map(const ConvGeom& g, const void* slot_base,
 }
 
 aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const void* out_map, const LayerJob* jobs_dev, int n_jobs,
-                               int batch_capacity, int32_t* error_flag, double weight_bytes, cudaStream_t s) {
+                               int batch_capacity, int32_t* error_flag, double weight_bytes, int weight_bits, cudaStream_t s) {
   DeviceProps props;
   if (aiq_status_t st = current_device_props(&props)) return st;
   const int smem_limit = props.smem_optin, n_sms = props.n_sms;
@@ -726,8 +726,11 @@ aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const void* o
   // is a whole number of boxes; only the last tile may be narrower).  A layer's CTAs are split
   // evenly over its tiles, so its time goes with (tile width) / (CTAs per tile): 144 channels
   // run as 64 + 64 + 16 rather than 128 + 16, 576 as 9 x 64 rather than 4 x 128 + 64.
-  if (g.Cs_out <= 128) {
+  p.pieces = weight_bits > 8 ? 2 : 1;
+  if (g.Cs_out <= 128 && !(p.pieces == 2 && g.Cs_out > 64)) {
     p.Nt = g.Cs_out;
+  } else if (p.pieces == 2) {
+    p.Nt = 64;                                   // two weight tiles per stage: narrower tiles keep three stages
   } else {
     auto cost = [&](int nt) {
       const int per_tile = n_sms / (n_jobs * ((g.Cs_out + nt - 1) / nt));
@@ -740,11 +743,11 @@ aiq_status_t launch_conv_pw_tc(const ConvGeom& g, const void* map, const void* o
   p.ver_pixels = (long long)batch_capacity * (g.H + 2) * g.W;
   p.error_flag = error_flag;
   int stages = 4;
-  while (stages > 2 && pw_smem_bytes(p.Nt, stages) + 1024 > smem_limit) --stages;
-  if (pw_smem_bytes(p.Nt, stages) + 1024 > smem_limit)
-    return set_error(AIQ_ERR_SHAPE, "conv_pw_tc: %d bytes of shared memory needed", pw_smem_bytes(p.Nt, stages) + 1024);
+  while (stages > 2 && pw_smem_bytes(p.Nt, stages, p.pieces) + 1024 > smem_limit) --stages;
+  if (pw_smem_bytes(p.Nt, stages, p.pieces) + 1024 > smem_limit)
+    return set_error(AIQ_ERR_SHAPE, "conv_pw_tc: %d bytes of shared memory needed", pw_smem_bytes(p.Nt, stages, p.pieces) + 1024);
   p.n_stages = stages;
-  const int smem_bytes = pw_smem_bytes(p.Nt, stages) + 1024;
+  const int smem_bytes = pw_smem_bytes(p.Nt, stages, p.pieces) + 1024;
   const int n_tiles = (p.P + 127) / 128;
   int ctas = n_sms / (n_jobs * p.n_ntiles);
   if (ctas > n_tiles) ctas = n_tiles;

@@ -656,12 +656,12 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
       // (4- / 8-bit codes, then 16-bit, then 32-bit where the kernel can hold their pieces)
       const bool tc_layer = layer_on_tensor_cores(m, li);
       const int tkind = layer_tensor_kind(m, li);
-      const bool tc_wide = tc_layer && (tkind == 1 || tkind == 3);
+      const bool tc_wide = tc_layer;            // every tensor-core kernel also takes 16- / 32-bit weights (two pieces)
       const ConvGeom g_cls = make_geom(m, li, B);
       auto job_class = [&](int bits) -> int {      // 0: codes, 1: 16-bit, 2: 32-bit on tensor cores; 3: float32 kernel
         if (tc_layer && bits <= 8) return 0;
-        if (tc_wide && bits == 16 && (tkind == 3 || conv_tc_bits_ok(g_cls, 16))) return 1;
-        if (tc_wide && bits == 32 && (tkind == 3 || conv_tc_bits_ok(g_cls, 32))) return 2;
+        if (tc_wide && bits == 16 && (tkind != 1 || conv_tc_bits_ok(g_cls, 16))) return 1;
+        if (tc_wide && bits == 32 && (tkind != 1 || conv_tc_bits_ok(g_cls, 32))) return 2;
         return 3;
       };
       std::vector<int> vorder;
@@ -808,12 +808,12 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
     auto launch_wide = [&](const LayerJob* jd, int n, double wb, int wbits) -> aiq_status_t {
       return lp.tc_kind == 3
           ? launch_conv_rs(g, &lp.maps[0], jd, n, plan.batch_capacity, m->status_word, wb, wbits, lp.pools, stream)
+          : lp.tc_kind == 2
+          ? launch_conv_pw_tc(g, &lp.maps[0], &lp.maps[1], jd, n, plan.batch_capacity, m->status_word, wb, wbits, stream)
           : launch_conv_tc(g, &lp.maps[0], jd, n, plan.batch_capacity, m->status_word, wb, wbits, stream);
     };
     if (lp.n_tc > 0) {
-      st = lp.tc_kind != 2
-          ? launch_wide(jobs_dev + lp.job_first, lp.n_tc, lp.weight_bytes_tc, 8)
-          : launch_conv_pw_tc(g, &lp.maps[0], &lp.maps[1], jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word, lp.weight_bytes_tc, stream);
+      st = launch_wide(jobs_dev + lp.job_first, lp.n_tc, lp.weight_bytes_tc, 8);
       if (st != AIQ_OK) return st;
     }
     int done = lp.n_tc;

@@ -42,7 +42,9 @@ def _net(cin, cout, k, stride, hw=16):
 # (Cin, Cout, kernel, stride): every instantiation family of the multi-piece kernel, the
 # two-slice case (64 output channels) included
 SHAPES = [(16, 16, 3, 1), (16, 32, 3, 2), (16, 32, 1, 2), (32, 32, 3, 1), (32, 64, 3, 2), (32, 64, 1, 2),
-          (64, 64, 3, 1), (64, 32, 3, 1), (64, 16, 1, 1)]
+          (64, 64, 3, 1), (64, 32, 3, 1), (64, 16, 1, 1),
+          # channel counts only the pointwise kernel takes: one and several K chunks, one and several output tiles
+          (96, 24, 1, 1), (48, 144, 1, 1), (160, 320, 1, 1)]
 
 
 @pytest.mark.parametrize("path", ["tensor", "tiles"])
