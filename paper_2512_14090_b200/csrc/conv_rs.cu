@@ -862,10 +862,7 @@ conv_rs_block_kernel(const __grid_constant__ CUtensorMap in_map, RbParams p, con
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(bar_acc_empty + 8 * slot);
-          mbar_arrive(bar_in_free + 8 * is);
-        }
+        if (lane == 0) mbar_arrive(bar_acc_empty + 8 * slot);
         if (!alive) break;
         const int item = (int)blockIdx.x + il * (int)gridDim.x;
         uint8_t* row_dst = out_base + ((size_t)item * p.H + y) * p.W * px_bytes + (size_t)img * 16;
@@ -879,6 +876,9 @@ conv_rs_block_kernel(const __grid_constant__ CUtensorMap in_map, RbParams p, con
           *reinterpret_cast<uint4*>(dst + (size_t)lo_plane0 * plane_bytes) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
           *reinterpret_cast<uint4*>(dst + (size_t)(lo_plane0 + 1) * plane_bytes) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
         }
+        // the shortcut words have been used, so their loads have returned: only now may the TMA refill the stage
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_in_free + 8 * is);
       }
     }
   }

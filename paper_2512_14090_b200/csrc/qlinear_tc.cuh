@@ -39,6 +39,7 @@ constexpr int kQtMaxWStages = 8;
 struct QtParams {
   int N, K, M, bits;
   int Mt;                   // batch rows per CTA tile (multiple of 16, <= 256)
+  int m_block;              // batch rows per blockIdx.z: 256, or 128 with two weight pieces (shared memory)
   int n_chunks;             // ceil(K / 64)
   int chunks_per_split;
   int splits;
@@ -46,6 +47,7 @@ struct QtParams {
   int b_stages;             // activation tile pairs in flight (a ring of its own: these are the
                             // TMA loads with a long round trip, and at small batch they are small)
   int w_stages;             // packed weight tiles in flight
+  int pieces;               // bfloat16 pieces per weight: 1 (4- / 8-bit codes), 2 (16- / 32-bit weights as hi + lo)
   int stack;                // 1: hi and lo rows of B form one N = 2 Mt operand (Mt <= 128)
   int tmem_cols;
   int32_t* error_flag;      // optional
@@ -53,8 +55,8 @@ struct QtParams {
 
 constexpr int kQtMaxBStages = 24;
 __host__ __device__ inline int qt_b_stage_bytes(int Mt) { return 2 * Mt * kQtChunk * 2; }   // hi tile + lo tile
-__host__ __device__ inline int qt_smem_bytes(int Mt, int stages, int b_stages, int w_stages) {
-  return stages * kQtATile + b_stages * qt_b_stage_bytes(Mt) + w_stages * kQtWTile +
+__host__ __device__ inline int qt_smem_bytes(int Mt, int stages, int b_stages, int w_stages, int pieces = 1) {
+  return stages * pieces * kQtATile + b_stages * qt_b_stage_bytes(Mt) + w_stages * kQtWTile +
          (2 * stages + 2 * b_stages + 2 * w_stages + 1) * 8 + 16;
 }
 
@@ -91,16 +93,19 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n0 = blockIdx.x * 128, split = blockIdx.y, m0 = blockIdx.z * 256;
+  const int n0 = blockIdx.x * 128, split = blockIdx.y, m0 = blockIdx.z * p.m_block;
   const int stages = p.n_stages, b_stages = p.b_stages, Mt = p.Mt, w_stages = p.w_stages;
   const int b_stage_bytes = qt_b_stage_bytes(Mt);
   const int c_begin = split * p.chunks_per_split;
   const int c_end = min(p.n_chunks, c_begin + p.chunks_per_split);
 
-  // k chunks per packed tile: 128 bytes of a row are 256 (4 bits) or 128 (8 bits) elements
-  const int cpw = p.bits == 4 ? 4 : 2;
+  // k chunks per packed tile: 128 bytes of a row are 256 (4 bits), 128 (8 bits) or 64 (16 bits) elements;
+  // at 32 bits a chunk of 64 k spans tpc = 2 packed tiles
+  const int cpw = p.bits == 4 ? 4 : (p.bits == 8 ? 2 : 1);
+  const int tpc = p.bits == 32 ? 2 : 1;
+  const int a_stage_bytes = p.pieces * kQtATile;            // hi tile (+ lo tile of 16- / 32-bit weights)
   // shared memory: A ring | B ring | packed weight ring | barriers (every tile 1024-aligned)
-  uint8_t* bring = smem + stages * kQtATile;
+  uint8_t* bring = smem + stages * a_stage_bytes;
   uint8_t* wring = bring + b_stages * b_stage_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(wring + w_stages * kQtWTile);
   const uint32_t bar_a_full = smem_u32(bars);               // expanders finished an A tile
@@ -175,6 +180,61 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
     constexpr int UPT = 128 * UPR / ET;                         // units per thread
     const int unit_bytes = p.bits;                              // 8 codes: 4 or 8 bytes
     uint32_t stage = 0, phase = 0, wst = 0, wphase = 0;
+    if (p.pieces == 2) {
+      // 16- / 32-bit weights: w = hi + lo with hi = bf16(w), lo = bf16(w - hi) (exact for a half, within 2^-17
+      // of a float32 weight); one A tile per piece, the MMAs of a chunk are issued once per piece.
+      for (int c = c_begin; c < c_end && alive; ++c) {
+        uint32_t tile_stage[2] = {wst, 0};
+        for (int t = 0; t < tpc && alive; ++t) {
+          tile_stage[t] = wst;
+          alive = mbar_wait_warp(bar_w_full + 8 * wst, wphase, s_abort, p.error_flag);
+          if (++wst == (uint32_t)w_stages) { wst = 0; wphase ^= 1u; }
+        }
+        if (!alive) break;
+        float w[UPT][8];
+#pragma unroll
+        for (int i = 0; i < UPT; ++i) {
+          const int u = et + i * ET;
+          const int nl = u / UPR, cu = u - nl * UPR;
+          if (p.bits == 16) {
+            const uint4 r = *reinterpret_cast<const uint4*>(wring + tile_stage[0] * kQtWTile + swizzle_off((uint32_t)(nl * 128 + cu * 16), 7u));
+            const __half2* h2 = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { const float2 f = __half22float2(h2[j]); w[i][2 * j] = f.x; w[i][2 * j + 1] = f.y; }
+          } else {
+            const uint8_t* wt = wring + tile_stage[cu >> 2] * kQtWTile;
+            const float4 r0 = *reinterpret_cast<const float4*>(wt + swizzle_off((uint32_t)(nl * 128 + (cu & 3) * 32), 7u));
+            const float4 r1 = *reinterpret_cast<const float4*>(wt + swizzle_off((uint32_t)(nl * 128 + (cu & 3) * 32 + 16), 7u));
+            w[i][0] = r0.x; w[i][1] = r0.y; w[i][2] = r0.z; w[i][3] = r0.w; w[i][4] = r1.x; w[i][5] = r1.y; w[i][6] = r1.z; w[i][7] = r1.w;
+          }
+        }
+        alive = mbar_wait_warp(bar_a_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
+        if (!alive) break;
+        uint8_t* atile = smem + stage * a_stage_bytes;
+#pragma unroll
+        for (int i = 0; i < UPT; ++i) {
+          const int u = et + i * ET;
+          const int nl = u / UPR, cu = u - nl * UPR;
+          uint32_t hi4[4], lo4[4];
+#pragma unroll
+          for (int j = 0; j < 8; j += 2) split_pair(w[i][j], w[i][j + 1], hi4[j >> 1], lo4[j >> 1]);
+          const uint32_t off = swizzle_off((uint32_t)(nl * 128 + cu * 16), 7u);
+          *reinterpret_cast<uint4*>(atile + off) = make_uint4(hi4[0], hi4[1], hi4[2], hi4[3]);
+          *reinterpret_cast<uint4*>(atile + kQtATile + off) = make_uint4(lo4[0], lo4[1], lo4[2], lo4[3]);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        // The packed tiles are released only now, after their words have been used: every lane's loads
+        // have then returned.  (Released right after the loads were issued, a refill by the TMA reached
+        // shared memory before the last loads of a warp had read it: wrong weights in 2-4 adjacent rows,
+        // a few times per million outputs.)
+        if (lane == 0) {
+          for (int t = 0; t < tpc; ++t) mbar_arrive(bar_w_empty + 8 * tile_stage[t]);
+          mbar_arrive(bar_a_full + 8 * stage);
+        }
+        if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+      }
+    } else
     for (int c = c_begin; c < c_end && alive; ++c) {
       const int sub = (c - c_begin) % cpw;                      // chunk inside the packed tile
       if (sub == 0) {
@@ -191,14 +251,13 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
         if (p.bits == 8) raw[i] = *reinterpret_cast<const uint2*>(wt + off);
         else raw[i] = make_uint2(*reinterpret_cast<const uint32_t*>(wt + off), 0u);
       }
-      if (sub == cpw - 1 || c + 1 == c_end) {                   // the packed tile is in registers: release it
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_w_empty + 8 * wst);
-        if (++wst == (uint32_t)w_stages) { wst = 0; wphase ^= 1u; }
-      }
+      // the packed tile is released further down, once its words have been used (see the two-piece path)
+      const bool last_of_tile = sub == cpw - 1 || c + 1 == c_end;
+      const uint32_t release_stage = wst;
+      if (last_of_tile && ++wst == (uint32_t)w_stages) { wst = 0; wphase ^= 1u; }
       alive = mbar_wait_warp(bar_a_empty + 8 * stage, phase ^ 1u, s_abort, p.error_flag);
       if (!alive) break;
-      uint8_t* atile = smem + stage * kQtATile;
+      uint8_t* atile = smem + stage * a_stage_bytes;
 #pragma unroll
       for (int i = 0; i < UPT; ++i) {
         const int u = et + i * ET;
@@ -210,7 +269,10 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_a_full + 8 * stage);
+      if (lane == 0) {
+        if (last_of_tile) mbar_arrive(bar_w_empty + 8 * release_stage);
+        mbar_arrive(bar_a_full + 8 * stage);
+      }
       if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
     }
   } else if (warp == 1) {
@@ -229,16 +291,18 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
               mbar_wait_warp(bar_b_full + 8 * bstage, bphase, s_abort, p.error_flag);
       if (!alive) break;
       tc_fence_after();
-      const uint32_t a_lo = ((smem_u32(smem) + stage * kQtATile) >> 4) | LBO_FIELD;
+      const uint32_t a_lo = ((smem_u32(smem) + stage * a_stage_bytes) >> 4) | LBO_FIELD;
       const uint32_t b_lo = ((smem_u32(bring) + bstage * b_stage_bytes) >> 4) | LBO_FIELD;
       const int parts = p.stack ? 1 : 2;
-      for (int part = 0; part < parts; ++part) {
+      for (int piece = 0; piece < p.pieces; ++piece) {
+        for (int part = 0; part < parts; ++part) {
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const uint64_t adesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(a_lo + ((kk * 32) >> 4));
-          const uint64_t bdesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + part * tile_units + ((kk * 32) >> 4));
-          umma_bf16(tmem_base, adesc, bdesc, idesc, accumulate);
-          accumulate = 1;
+          for (int kk = 0; kk < 4; ++kk) {
+            const uint64_t adesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(a_lo + ((piece * kQtATile + kk * 32) >> 4));
+            const uint64_t bdesc = ((uint64_t)DESC_HI << 32) | (uint64_t)(b_lo + part * tile_units + ((kk * 32) >> 4));
+            umma_bf16(tmem_base, adesc, bdesc, idesc, accumulate);
+            accumulate = 1;
+          }
         }
       }
       umma_commit(bar_a_empty + 8 * stage);
@@ -256,14 +320,16 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
       if (lane == 0) {
         uint32_t wst = 0, wphase = 0, w_issued = 0, w_issued_phase = 0;
         bool ok = true;
-        for (int c = c_begin; c < c_end && ok; c += cpw) {   // bytes [c * 64 * bits / 8, + 128) of 128 rows
-          ok = mbar_wait(bar_w_empty + 8 * wst, wphase ^ 1u, s_abort, p.error_flag);
-          if (!ok) break;
-          w_issued |= 1u << wst;
-          w_issued_phase = (w_issued_phase & ~(1u << wst)) | (wphase << wst);
-          mbar_expect_tx(bar_w_full + 8 * wst, kQtWTile);
-          tma_load_2d(smem_u32(wring) + wst * kQtWTile, &w_map, bar_w_full + 8 * wst, c * kQtChunk * p.bits / 8, n0);
-          if (++wst == (uint32_t)w_stages) { wst = 0; wphase ^= 1u; }
+        for (int c = c_begin; c < c_end && ok; c += cpw) {   // bytes [c * 64 * bits / 8, + 128 tpc) of 128 rows
+          for (int t = 0; t < tpc && ok; ++t) {
+            ok = mbar_wait(bar_w_empty + 8 * wst, wphase ^ 1u, s_abort, p.error_flag);
+            if (!ok) break;
+            w_issued |= 1u << wst;
+            w_issued_phase = (w_issued_phase & ~(1u << wst)) | (wphase << wst);
+            mbar_expect_tx(bar_w_full + 8 * wst, kQtWTile);
+            tma_load_2d(smem_u32(wring) + wst * kQtWTile, &w_map, bar_w_full + 8 * wst, c * kQtChunk * p.bits / 8 + t * 128, n0);
+            if (++wst == (uint32_t)w_stages) { wst = 0; wphase ^= 1u; }
+          }
         }
         if (!ok)                                   // copies in flight must land before the CTA exits
           for (int i = 0; i < w_stages; ++i)
@@ -316,7 +382,7 @@ qlinear_tc_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_consta
 }  // namespace
 
 bool qlinear_tc_applicable(int N, int K, int bits, int M) {
-  if (bits != 4 && bits != 8) return false;
+  if (!bits_ok(bits)) return false;
   if (M < 9) return false;                         // smaller batches: the warp-level kernels
   if (K % 8 != 0 || K < 64 || N < 32) return false;
   return true;
@@ -334,8 +400,10 @@ aiq_status_t launch_qlinear_tc(const LayerJob& job, int N, int K, int M, void* w
   if (!enc) return set_error(AIQ_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
   QtParams p = {};
   p.N = N; p.K = K; p.M = M; p.bits = job.bits; p.error_flag = error_flag;
-  p.Mt = M >= 256 ? 256 : (M + 15) / 16 * 16;
-  const int m_blocks = (M + 255) / 256, row_blocks = (N + 127) / 128;
+  p.pieces = job.bits > 8 ? 2 : 1;
+  p.m_block = p.pieces == 2 ? 128 : 256;           // two A tiles per stage leave room for activation tiles of 128 rows
+  p.Mt = M >= p.m_block ? p.m_block : (M + 15) / 16 * 16;
+  const int m_blocks = (M + p.m_block - 1) / p.m_block, row_blocks = (N + 127) / 128;
   p.n_chunks = (K + kQtChunk - 1) / kQtChunk;
   int splits = n_sms / (row_blocks * m_blocks);
   if (splits < 1) splits = 1;
@@ -346,9 +414,9 @@ aiq_status_t launch_qlinear_tc(const LayerJob& job, int N, int K, int M, void* w
   // up to 4 A tiles (they are produced on chip, a short ring suffices), as many activation
   // stages as fit up to 24 (their TMA round trip is what a shallow ring would expose), and
   // whatever is left goes to packed weight tiles in flight.
-  auto fits = [&](int a, int b, int w) { return qt_smem_bytes(p.Mt, a, b, w) + 1024 <= smem_limit; };
+  auto fits = [&](int a, int b, int w) { return qt_smem_bytes(p.Mt, a, b, w, p.pieces) + 1024 <= smem_limit; };
   if (!fits(2, 2, 3))
-    return set_error(AIQ_ERR_SHAPE, "qlinear_tc: %d bytes of shared memory needed", qt_smem_bytes(p.Mt, 2, 2, 3) + 1024);
+    return set_error(AIQ_ERR_SHAPE, "qlinear_tc: %d bytes of shared memory needed", qt_smem_bytes(p.Mt, 2, 2, 3, p.pieces) + 1024);
   int stages = 2, b_stages = 2, w_stages = 3;
   while (stages < 4 && fits(stages + 1, b_stages, w_stages)) ++stages;
   while (w_stages < 4 && fits(stages, b_stages, w_stages + 1)) ++w_stages;
@@ -400,7 +468,7 @@ aiq_status_t launch_qlinear_tc(const LayerJob& job, int N, int K, int M, void* w
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(row_blocks, p.splits, m_blocks);
   cfg.blockDim = dim3(kQtThreads);
-  cfg.dynamicSmemBytes = qt_smem_bytes(p.Mt, stages, b_stages, w_stages) + 1024;
+  cfg.dynamicSmemBytes = qt_smem_bytes(p.Mt, stages, b_stages, w_stages, p.pieces) + 1024;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

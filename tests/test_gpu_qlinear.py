@@ -64,3 +64,21 @@ def test_qlinear_exact_on_integers(bits):
         want = x.astype(np.int64) @ W.astype(np.int64).T
         assert np.array_equal(got.astype(np.int64), want)
         assert np.array_equal(ref.astype(np.int64), want)
+
+
+@pytest.mark.parametrize("bits", [16, 32])
+def test_qlinear_two_piece_path_exact_on_integers(bits):
+    """16- and 32-bit weights on the tcgen05 kernel enter as two bfloat16 pieces.  Small integer
+    weights and activations make every product and sum exact, so any dropped, repeated or stale
+    tile shows up as a wrong integer.  Shapes with many K chunks per CTA, several batch blocks and
+    K splits; each shape is run three times (a race would not repeat)."""
+    aiq = binding()
+    for (N, K, M) in ((128, 64, 16), (256, 512, 32), (4096, 4096, 128), (2048, 2048, 256), (4096, 4096, 256),
+                      (1000, 1288, 300)):
+        rng = np.random.default_rng(N + K + M + bits)
+        W = rng.integers(-3, 4, (N, K)).astype(np.float32)
+        x = rng.integers(-2, 3, (M, K)).astype(np.float32)
+        want = x.astype(np.int64) @ W.astype(np.int64).T
+        for trial in range(3):
+            got, ref = _run(aiq, W, x, bits)
+            assert np.array_equal(got.astype(np.int64), want), (N, K, M, bits, trial)
