@@ -7,7 +7,7 @@ oracle's tests and the CUDA library's binding may consume its output as data.
 """
 from .archs import (resnet20, mobilenet_v2, conv_layer_indices, tiny_net,  # noqa: F401
                     heavy_early_resnet20, plain_convnet20, depthwise_stack,
-                    pointwise_stack)
+                    pointwise_stack, inverted_residual_stack)
 from .gen import (  # noqa: F401
     gen_model,
     gen_images,

@@ -167,6 +167,22 @@ def pointwise_stack(cin, cout, hw=8, n_classes=6):
     return dict(name=f"pointwise_stack_{cin}_{cout}", in_c=3, in_h=hw, in_w=hw, n_classes=n_classes, layers=layers)
 
 
+def inverted_residual_stack(cin, cout, hw=8, stride=1, t=6, n_classes=6):
+    """A short network around one MobileNetV2 inverted-residual block (test workload): stem 3x3
+    to `cin` channels, expansion 1x1 to t * cin, depthwise 3x3 at `stride`, projection 1x1 to
+    `cout` with the shortcut from the block's input when stride is 1 and cin == cout, classifier."""
+    hid = cin * t
+    layers = [
+        _conv("stem", 3, cin, 3, 1, "relu6", -1),
+        _conv("b.expand", cin, hid, 1, 1, "relu6", 0),
+        _conv("b.dw", hid, hid, 3, stride, "relu6", 1, kind="dw"),
+        _conv("b.project", hid, cout, 1, 1, "none", 2, residual=0 if (stride == 1 and cin == cout) else -1),
+        _fc("fc", cout, n_classes, 3),
+    ]
+    return dict(name=f"inverted_residual_stack_{cin}_{cout}_{hw}_s{stride}", in_c=3, in_h=hw, in_w=hw,
+                n_classes=n_classes, layers=layers)
+
+
 def conv_layer_indices(arch):
     """Indices of every layer that is not the classifier (the sweep candidates)."""
     return [i for i, l in enumerate(arch["layers"]) if l["kind"] != "fc"]

@@ -141,7 +141,12 @@ struct LayerJob {
   const float* scale_pre;
   const float* bias_pre;
   int32_t bits_pre;
-  int32_t reserved;
+  int32_t bits_mid;
+  // fused inverted-residual block (mb_block_kernel): w_pre / scale_pre = operand images / coefficients of the
+  // expansion, scale_mid = coefficients of the depthwise layer, w = operand images of the projection
+  const uint8_t* w_mid;
+  const float* scale_mid;
+  const float* bias_mid;
   float* pool;          // fused global average pool: float32 [batch][cout] written instead of `out`, or nullptr
 };
 
@@ -201,6 +206,20 @@ aiq_status_t launch_conv_rs(const ConvGeom& g, const void* maps, const LayerJob*
                             int32_t* error_flag, double weight_bytes, int weight_bits, bool pool_jobs, cudaStream_t s);
 // A whole identity-shortcut basic block (two 3x3 convolutions of C -> C channels) in one kernel; `g`
 // describes either convolution.  Jobs carry both weight sets (LayerJob::w_pre ...).
+// fused MobileNetV2 inverted-residual block (expansion 1x1 -> depthwise 3x3 -> projection 1x1 [+ shortcut]) on split
+// activations; the three geometries are those of the block's layers
+// hidden channels per chunk (32 or 64) the kernel would use for this block on the current device, 0 = not eligible
+int mb_block_chunk_channels(const ConvGeom& ge, const ConvGeom& gd, const ConvGeom& gp);
+// bytes of one chunk's operand image: expansion (Cs_in / 8 planes of nh rows), projection (nh / 8 planes of Cs_out rows);
+// every plane carries 16 padding bytes
+__host__ __device__ inline size_t mb_etile_bytes(int cs_in, int nh) { return (size_t)(cs_in / 8) * (nh * 16 + 16); }
+__host__ __device__ inline size_t mb_ptile_bytes(int cs_out, int nh) { return (size_t)(nh / 8) * (cs_out * 16 + 16); }
+// role 0: expansion, 1: projection, 2: depthwise (coefficients only); see mb_block.cu
+aiq_status_t launch_mb_build_tiles(int role, const uint8_t* packed, const float* scale, const float* bias, int bits, int N,
+                                   int K, int nh, int cs, void* tile_out, float* coef_out, cudaStream_t s);
+// nh: the chunk width the jobs' operand images were built for
+aiq_status_t launch_mb_block(const ConvGeom& ge, const ConvGeom& gd, const ConvGeom& gp, int nh, const LayerJob* jobs_dev, int n_jobs,
+                             int32_t* error_flag, double weight_bytes, cudaStream_t s);
 bool conv_rs_block_eligible(const ConvGeom& g);
 aiq_status_t launch_conv_rs_block(const ConvGeom& g, const void* maps, const LayerJob* jobs_dev, int n_jobs, int batch_capacity,
                                   int32_t* error_flag, double weight_bytes, cudaStream_t s);

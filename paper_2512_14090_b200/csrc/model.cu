@@ -121,6 +121,12 @@ struct LayerInfo {
   uint8_t* packed[4];
   float* scales[4];
   int slot;                // activation slot of the output (-1: fc)
+  // layers of an inverted-residual block the fused kernel can take (see mb_block.cu): operand images of the
+  // 1x1 layers per 4- / 8-bit version, coefficient rows (expansion: 4 / 8 bits; depthwise: every bit-width),
+  // hidden channels per chunk the images were built for (0: none built)
+  uint8_t* mb_tile[2];
+  float* mb_coef[4];
+  int mb_nh;
 };
 
 struct aiq_model {
@@ -135,6 +141,8 @@ struct aiq_model {
   std::vector<int> block_tail;       // per layer: the second convolution of the basic block this layer opens
                                      // (the pair can run as one kernel), or -1
   int pool_layer;                    // the layer whose epilogue can do the classifier's average pool, or -1
+  std::vector<int> mb_mid, mb_tail;  // per layer: the depthwise and the projection layer of the inverted-residual
+                                     // block this (expansion) layer opens (the three can run as one kernel), or -1
 };
 
 namespace aiq {
@@ -270,7 +278,42 @@ static void assign_slots(aiq_model* m) {
   }
 }
 
-struct ModelLayout { size_t total, staging_off, flag_off; std::vector<size_t> wf, bias; std::vector<size_t> packed[4], scales[4]; };
+// Inverted-residual blocks by structure alone: an expansion 1x1 (no shortcut) that feeds only a depthwise 3x3
+// that feeds only a projection 1x1 whose shortcut (if any) is the expansion's input.  mid / tail: per
+// expansion layer the depthwise and the projection layer, else -1.
+static void find_mb_structure(const std::vector<LayerInfo>& L, std::vector<int>& mid, std::vector<int>& tail) {
+  const int n = (int)L.size();
+  mid.assign(n, -1);
+  tail.assign(n, -1);
+  std::vector<int> uses(n, 0);
+  for (const LayerInfo& li : L) {
+    if (li.d.input >= 0) uses[li.d.input]++;
+    if (li.d.residual >= 0) uses[li.d.residual]++;
+  }
+  for (int le = 0; le < n; ++le) {
+    const LayerInfo& e = L[le];
+    if (e.d.kind != AIQ_LAYER_CONV || e.d.ksize != 1 || e.d.input < 0 || e.d.residual >= 0 || uses[le] != 1) continue;
+    if (e.d.cin % 8 != 0 || e.d.cout % 16 != 0) continue;
+    for (int ld = 0; ld < n; ++ld) {
+      const LayerInfo& d = L[ld];
+      if (d.d.kind != AIQ_LAYER_DEPTHWISE || d.d.ksize != 3 || d.d.input != le || d.d.residual >= 0 || uses[ld] != 1) continue;
+      for (int lp = 0; lp < n; ++lp) {
+        const LayerInfo& pr = L[lp];
+        if (pr.d.kind != AIQ_LAYER_CONV || pr.d.ksize != 1 || pr.d.input != ld) continue;
+        if (pr.d.residual >= 0 && pr.d.residual != e.d.input) continue;
+        mid[le] = ld;
+        tail[le] = lp;
+      }
+    }
+  }
+}
+
+struct ModelLayout {
+  size_t total, staging_off, flag_off;
+  std::vector<size_t> wf, bias;
+  std::vector<size_t> packed[4], scales[4];
+  std::vector<size_t> mb_tile[2], mb_coef[4];       // 0: the layer has none
+};
 
 static ModelLayout model_layout(const std::vector<LayerInfo>& L) {
   ModelLayout lay;
@@ -288,6 +331,30 @@ static ModelLayout model_layout(const std::vector<LayerInfo>& L) {
     staging = std::max(staging, align_up(n * k * 4, 256) + 5 * align_up(n * 4, 256));
   }
   lay.staging_off = take(staging);
+  // operand images of inverted-residual blocks, sized for either chunk width the kernel may choose
+  for (int b = 0; b < 2; ++b) lay.mb_tile[b].assign(L.size(), 0);
+  for (int b = 0; b < 4; ++b) lay.mb_coef[b].assign(L.size(), 0);
+  std::vector<int> mid, tail;
+  find_mb_structure(L, mid, tail);
+  for (size_t le = 0; le < L.size(); ++le) {
+    if (tail[le] < 0) continue;
+    const int ld = mid[le], lp = tail[le];
+    const int ch = L[le].d.cout, cs_in = padded_channels(L[le].d.cin), cs_out = padded_channels(L[lp].d.cout);
+    size_t et = 0, pt = 0, ec = 0, dc = 0;
+    for (int nh = 32; nh <= 64; nh *= 2) {
+      const size_t chunks = (size_t)(ch + nh - 1) / nh;
+      et = std::max(et, chunks * mb_etile_bytes(cs_in, nh));
+      pt = std::max(pt, chunks * mb_ptile_bytes(cs_out, nh));
+      ec = std::max(ec, chunks * 2 * nh * 4);
+      dc = std::max(dc, chunks * 11 * nh * 4);
+    }
+    for (int b = 0; b < 2; ++b) {
+      lay.mb_tile[b][le] = take(et);
+      lay.mb_coef[b][le] = take(ec);
+      lay.mb_tile[b][lp] = take(pt);
+    }
+    for (int b = 0; b < 4; ++b) lay.mb_coef[b][ld] = take(dc);
+  }
   lay.total = off;
   return lay;
 }
@@ -377,6 +444,27 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
       }
     }
   }
+  // inverted-residual blocks that the fused block kernel takes (structure: find_mb_structure; shape and
+  // memory: mb_block_chunk_channels, on split activations with both 1x1 layers on the tensor cores)
+  m->mb_mid.assign(m->layers.size(), -1);
+  m->mb_tail.assign(m->layers.size(), -1);
+  for (LayerInfo& li : m->layers) li.mb_nh = 0;
+  if (m->act_format == ACT_SPLIT) {
+    std::vector<int> mid, tail;
+    find_mb_structure(m->layers, mid, tail);
+    for (size_t le = 0; le < m->layers.size(); ++le) {
+      if (tail[le] < 0) continue;
+      LayerInfo& e = m->layers[le];
+      LayerInfo& d = m->layers[mid[le]];
+      LayerInfo& pr = m->layers[tail[le]];
+      if (!layer_on_tensor_cores(m, e) || !layer_on_tensor_cores(m, pr)) continue;
+      const int nh = mb_block_chunk_channels(make_geom(m, e, 1), make_geom(m, d, 1), make_geom(m, pr, 1));
+      if (!nh) continue;
+      m->mb_mid[le] = mid[le];
+      m->mb_tail[le] = tail[le];
+      e.mb_nh = d.mb_nh = pr.mb_nh = nh;
+    }
+  }
   assign_slots(m);
   cudaStream_t stream = (cudaStream_t)stream_;
   uint8_t* base = static_cast<uint8_t*>(dev_mem);
@@ -426,6 +514,32 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
     for (int b = 0; b < 4; ++b) {
       st = launch_quantize(li.Wf, (int)n, (int)k, kBitsList[b], li.packed[b], li.scales[b], flag,
                            per_tensor ? reinterpret_cast<uint32_t*>(flag + 2) : nullptr, stream);
+      if (st != AIQ_OK) return fail(st);
+    }
+  }
+  // operand images of the fused inverted-residual blocks, from the packed codes just written
+  for (size_t le = 0; le < m->layers.size(); ++le) {
+    if (m->mb_tail[le] < 0) continue;
+    const int ld = m->mb_mid[le], lp = m->mb_tail[le];
+    LayerInfo& e = m->layers[le];
+    LayerInfo& d = m->layers[ld];
+    LayerInfo& pr = m->layers[lp];
+    const int nh = e.mb_nh;
+    for (int b = 0; b < 2; ++b) {
+      e.mb_tile[b] = base + lay.mb_tile[b][le];
+      e.mb_coef[b] = reinterpret_cast<float*>(base + lay.mb_coef[b][le]);
+      pr.mb_tile[b] = base + lay.mb_tile[b][lp];
+      st = launch_mb_build_tiles(0, e.packed[b], e.scales[b], e.bias, kBitsList[b], e.d.cout, e.K, nh,
+                                 padded_channels(e.d.cin), e.mb_tile[b], e.mb_coef[b], stream);
+      if (st != AIQ_OK) return fail(st);
+      st = launch_mb_build_tiles(1, pr.packed[b], pr.scales[b], pr.bias, kBitsList[b], pr.d.cout, pr.K, nh,
+                                 padded_channels(pr.d.cout), pr.mb_tile[b], nullptr, stream);
+      if (st != AIQ_OK) return fail(st);
+    }
+    for (int b = 0; b < 4; ++b) {
+      d.mb_coef[b] = reinterpret_cast<float*>(base + lay.mb_coef[b][ld]);
+      st = launch_mb_build_tiles(2, d.packed[b], d.scales[b], d.bias, kBitsList[b], d.d.cout, d.K, nh, 0, nullptr,
+                                 d.mb_coef[b], stream);
       if (st != AIQ_OK) return fail(st);
     }
   }
@@ -532,7 +646,8 @@ struct LayerPlan {
   int tc_kind = 0;                      // which tensor-core kernel (see layer_tensor_kind)
   bool pools = false;                   // its jobs write the classifier's pooled input instead of the tensor
   bool skipped = false;                 // first convolution of a fused block: evaluated inside its partner's kernel
-  int fused_head = -1;                  // second convolution of a fused block: the layer it absorbs
+  int fused_head = -1;                  // last layer of a fused block: the first layer it absorbs
+  int fused_mid = -1;                   // inverted-residual block: the depthwise layer between the two (else -1)
   double weight_bytes = 0.0;            // packed weights + scales + biases over all jobs
   double weight_bytes_tc = 0.0, weight_bytes_tc16 = 0.0, weight_bytes_tc32 = 0.0;
   TensorMapBytes maps[2];               // [0] over the input slot (tensor-core layers); [1] over the output slot
@@ -580,6 +695,17 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
       for (int s = 0; s < S && ok; ++s) ok = schemes[(size_t)s * n + l1] <= 8 && schemes[(size_t)s * n + l2] <= 8;
       if (ok) fuse_head[l2] = l1;
     }
+  // an inverted-residual block runs as one kernel when every scheme gives its two 1x1 layers 4 or 8 bits
+  std::vector<int> mb_head(n, -1);
+  std::vector<char> mb_absorbed(n, 0);
+  if (fuse)
+    for (int le = 0; le < n; ++le) {
+      const int lt = m->mb_tail[le];
+      if (lt < 0) continue;
+      bool ok = true;
+      for (int s = 0; s < S && ok; ++s) ok = schemes[(size_t)s * n + le] <= 8 && schemes[(size_t)s * n + lt] <= 8;
+      if (ok) { mb_head[lt] = le; mb_absorbed[le] = 1; mb_absorbed[m->mb_mid[le]] = 1; }
+    }
   float* const pooled_base = reinterpret_cast<float*>(ws + wl.pooled_off);
   auto slot_ptr = [&](int layer, int version) -> uint8_t* {
     const LayerInfo& li = m->layers[layer];
@@ -613,6 +739,47 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
     all_keys[l] = keys;
     if (li.d.kind != AIQ_LAYER_FC && m->block_tail[l] >= 0 && fuse_head[m->block_tail[l]] == l) {
       lp.skipped = true;                   // evaluated inside the kernel of the block's second convolution
+      continue;
+    }
+    if (li.d.kind != AIQ_LAYER_FC && mb_absorbed[l]) {
+      lp.skipped = true;                   // evaluated inside the kernel of the block's projection layer
+      continue;
+    }
+    if (li.d.kind != AIQ_LAYER_FC && mb_head[l] >= 0) {
+      // fused inverted-residual block: one job per version of the projection, carrying the weights of the
+      // expansion and depthwise versions it descends from
+      const int le = mb_head[l], ld = m->mb_mid[le];
+      const LayerInfo& ex = m->layers[le];
+      const LayerInfo& dw = m->layers[ld];
+      lp.fused_head = le;
+      lp.fused_mid = ld;
+      lp.job_first = plan.jobs.size();
+      plan.versions_total += 2 * lp.n_versions - plan.lp[le].n_versions - plan.lp[ld].n_versions;
+      for (int v = 0; v < lp.n_versions; ++v) {
+        const int bits = std::get<0>(keys[v]);
+        const std::tuple<int, int, int>& kd = all_keys[ld][std::get<1>(keys[v])];
+        const std::tuple<int, int, int>& ke = all_keys[le][std::get<1>(kd)];
+        const int bits_d = std::get<0>(kd), bits_e = std::get<0>(ke), vin = std::get<1>(ke);
+        LayerJob j = {};
+        j.in = slot_ptr(ex.d.input, vin);
+        j.res = li.d.residual >= 0 ? slot_ptr(li.d.residual, std::get<2>(keys[v])) : nullptr;
+        j.out = slot_ptr(l, v);
+        j.in_version = vin;
+        j.out_version = v;
+        j.w = li.mb_tile[bits_index(bits)];                  // operand images (see LayerJob)
+        j.scale = li.scales[bits_index(bits)];
+        j.bias = li.bias;
+        j.bits = bits;
+        j.w_pre = ex.mb_tile[bits_index(bits_e)];
+        j.scale_pre = ex.mb_coef[bits_index(bits_e)];
+        j.bits_pre = bits_e;
+        j.scale_mid = dw.mb_coef[bits_index(bits_d)];
+        j.bits_mid = bits_d;
+        plan.jobs.push_back(j);
+        lp.n_tc++;
+        lp.weight_bytes_tc += (double)li.d.cout * (row_bytes(li.K, bits) + 8.0) + (double)ex.d.cout * (row_bytes(ex.K, bits_e) + 8.0) +
+                              (double)dw.d.cout * (row_bytes(dw.K, bits_d) + 8.0);
+      }
       continue;
     }
     if (li.d.kind != AIQ_LAYER_FC && fuse_head[l] >= 0) {
@@ -794,6 +961,12 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
     }
     if (lp.skipped) continue;
     const ConvGeom g = make_geom(m, li, B);
+    if (lp.fused_head >= 0 && lp.fused_mid >= 0) {
+      st = launch_mb_block(make_geom(m, m->layers[lp.fused_head], B), make_geom(m, m->layers[lp.fused_mid], B), g, li.mb_nh,
+                           jobs_dev + lp.job_first, lp.n_tc, m->status_word, lp.weight_bytes_tc, stream);
+      if (st != AIQ_OK) return st;
+      continue;
+    }
     if (lp.fused_head >= 0) {
       st = launch_conv_rs_block(g, &lp.maps[0], jobs_dev + lp.job_first, lp.n_tc, plan.batch_capacity, m->status_word,
                                 lp.weight_bytes_tc, stream);

@@ -139,5 +139,31 @@ __device__ __forceinline__ void split_pair(float u0, float u1, uint32_t& hi2, ui
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Eight packed codes (4 bits: raw.x; 8 bits: raw.x, raw.y; two's complement) -> eight
+// bfloat16, without the conversion unit: the offset-binary code is placed in the low
+// mantissa bits of 2^23, one subtraction gives the integer as a float, and because
+// |code| <= 128 has at most 8 significant bits the upper half of that float is the exact
+// bfloat16.
+__device__ __forceinline__ void expand8_bf16(uint2 raw, int bits, uint32_t* out) {
+  float f[8];
+  if (bits == 8) {
+    const uint32_t w0 = raw.x ^ 0x80808080u, w1 = raw.y ^ 0x80808080u;
+    f[0] = __uint_as_float(__byte_perm(w0, 0x4B000000u, 0x7540)) - 8388736.0f;
+    f[1] = __uint_as_float(__byte_perm(w0, 0x4B000000u, 0x7541)) - 8388736.0f;
+    f[2] = __uint_as_float(__byte_perm(w0, 0x4B000000u, 0x7542)) - 8388736.0f;
+    f[3] = __uint_as_float(__byte_perm(w0, 0x4B000000u, 0x7543)) - 8388736.0f;
+    f[4] = __uint_as_float(__byte_perm(w1, 0x4B000000u, 0x7540)) - 8388736.0f;
+    f[5] = __uint_as_float(__byte_perm(w1, 0x4B000000u, 0x7541)) - 8388736.0f;
+    f[6] = __uint_as_float(__byte_perm(w1, 0x4B000000u, 0x7542)) - 8388736.0f;
+    f[7] = __uint_as_float(__byte_perm(w1, 0x4B000000u, 0x7543)) - 8388736.0f;
+  } else {
+    const uint32_t w = raw.x ^ 0x88888888u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(((w >> (4 * j)) & 0xFu) | 0x4B000000u) - 8388616.0f;
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) out[j] = __byte_perm(__float_as_uint(f[2 * j]), __float_as_uint(f[2 * j + 1]), 0x7632);
+}
+
 }  // namespace
 }  // namespace aiq
