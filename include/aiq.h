@@ -297,10 +297,14 @@ void aiq_set_eval_options(int chunk, int share_prefix);
 
 /* Kernel fusion on networks stored for the row-streaming kernel (process-wide, both default on; the
  * paper's searches only pay off if a candidate evaluation is cheap, Section 2.2).
- *   blocks: a basic block out = relu(conv2(relu(conv1(x))) + x) with two 3x3 convolutions of 16 or 32
- *           channels runs as one kernel whenever every scheme of the call gives both convolutions 4 or
- *           8 bits: the intermediate tensor stays in shared memory.  Results are bit-identical to the
- *           layer-by-layer path.
+ *   blocks: bit 0 (default on): a basic block out = relu(conv2(relu(conv1(x))) + x) with two 3x3
+ *           convolutions of 16 or 32 channels runs as one kernel whenever every scheme of the call gives
+ *           both convolutions 4 or 8 bits: the intermediate tensor stays in shared memory.  Results are
+ *           bit-identical to the layer-by-layer path.
+ *           bit 1 (default off): a MobileNetV2 inverted-residual block (expansion 1x1 -> depthwise 3x3 ->
+ *           projection 1x1, optional shortcut) runs as one kernel whenever every scheme gives both 1x1
+ *           layers 4 or 8 bits: the six-fold hidden tensor stays in shared memory (float32 there, so the
+ *           results differ from the layer-by-layer path by that path's rounding of the hidden tensor).
  *   pool:   the classifier's global average pool is taken in the epilogue of the convolution that
  *           produces its input; that tensor is then never stored.  Sums are formed in a fixed order
  *           (run-to-run identical); they differ from the separate pooling kernel's in the last bits. */

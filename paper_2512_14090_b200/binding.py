@@ -234,8 +234,8 @@ def aiq_quantize_layer_per_tensor(W, bits, packed_out, scales_out, scratch, nonf
                                              _dev(nonfinite_flag), _dev(scratch), _stream(stream)))
 
 
-def aiq_set_fusion(blocks=True, pool=True):
-    lib.aiq_set_fusion(int(bool(blocks)), int(bool(pool)))
+def aiq_set_fusion(blocks=True, pool=True, inverted_residual=False):
+    lib.aiq_set_fusion(int(bool(blocks)) | (2 if inverted_residual else 0), int(bool(pool)))
 
 
 def aiq_set_compute_path(path):

@@ -210,10 +210,9 @@ aiq_status_t launch_conv_rs(const ConvGeom& g, const void* maps, const LayerJob*
 // activations; the three geometries are those of the block's layers
 // hidden channels per chunk (32 or 64) the kernel would use for this block on the current device, 0 = not eligible
 int mb_block_chunk_channels(const ConvGeom& ge, const ConvGeom& gd, const ConvGeom& gp);
-// bytes of one chunk's operand image: expansion (Cs_in / 8 planes of nh rows), projection (nh / 8 planes of Cs_out rows);
-// every plane carries 16 padding bytes
-__host__ __device__ inline size_t mb_etile_bytes(int cs_in, int nh) { return (size_t)(cs_in / 8) * (nh * 16 + 16); }
-__host__ __device__ inline size_t mb_ptile_bytes(int cs_out, int nh) { return (size_t)(nh / 8) * (cs_out * 16 + 16); }
+// bytes of one chunk's operand image: expansion (Cs_in / 8 planes of nh rows), projection (nh / 8 planes of Cs_out rows)
+__host__ __device__ inline size_t mb_etile_bytes(int cs_in, int nh) { return (size_t)(cs_in / 8) * (nh * 16); }
+__host__ __device__ inline size_t mb_ptile_bytes(int cs_out, int nh) { return (size_t)(nh / 8) * (cs_out * 16); }
 // role 0: expansion, 1: projection, 2: depthwise (coefficients only); see mb_block.cu
 aiq_status_t launch_mb_build_tiles(int role, const uint8_t* packed, const float* scale, const float* bias, int bits, int N,
                                    int K, int nh, int cs, void* tile_out, float* coef_out, cudaStream_t s);

@@ -36,8 +36,9 @@ namespace aiq {
 
 namespace {
 
-constexpr int kMbThreads = 512;
-constexpr int kMbWarps = kMbThreads / 32;
+constexpr int kMbWorkers = 16;                      // warps that run the accumulator, depthwise and output passes
+constexpr int kMbThreads = (kMbWorkers + 1) * 32;   // + one warp that issues the MMAs and the bulk copies
+constexpr int kMbLeader = kMbWorkers * 32;          // its first thread
 
 struct MbParams {
   int H, W, Ho, Wo, stride;
@@ -48,6 +49,7 @@ struct MbParams {
   int NH;                   // hidden channels per chunk: 32 or 64
   int n_chunks;
   int tmem_cols;
+  int hid_px;               // pixels of a hidden plane: rows of a band x (W + 2): a zero column on both sides
   int act_e, act_d, act_p;
   int32_t* error_flag;
 };
@@ -56,22 +58,22 @@ struct MbParams {
 struct MbSmem {
   int a_in, a_lbo;          // input operand: 2 * Cs_in / 8 planes, a_lbo bytes apart
   int b1;                   // expansion operand image of the chunk (mb_etile_bytes)
-  int hid, hid_plane;       // hidden chunk, float32: NH / 4 planes of T1 * 128 pixels
+  int hid, hid_plane;       // hidden chunk, float32: NH / 4 planes of hid_px pixels (rows of W + 2 columns)
   int a2;                   // depthwise output, hi then lo planes of 128 pixels
   int b2;                   // projection operand image of the chunk (mb_ptile_bytes)
   int coef;                 // two buffers (chunk parity) of floats: s_e, b_e [NH]; w_d [9][NH]; s_d, b_d [NH]
   int proj;                 // floats: s_p, b_p [Cs_out]
   int bars, total;
 };
-__host__ __device__ inline MbSmem mb_smem(int Cs_in, int Cs_out, int T1, int NH) {
+__host__ __device__ inline MbSmem mb_smem(int Cs_in, int Cs_out, int T1, int NH, int hid_px) {
   MbSmem s;
   const int px = T1 * 128;
   s.a_in = 0;
-  s.a_lbo = px * 16 + 16;                         // +16: the planes of one pixel fall into different banks
+  s.a_lbo = px * 16;
   int off = (Cs_in / 4) * s.a_lbo;
   off = (off + 127) / 128 * 128;
   s.b1 = off;  off += (int)mb_etile_bytes(Cs_in, NH);
-  s.hid = off; s.hid_plane = px * 16; off += (NH / 4) * s.hid_plane;
+  s.hid = off; s.hid_plane = hid_px * 16; off += (NH / 4) * s.hid_plane;
   s.a2 = off;  off += (NH / 4) * 2048;
   s.b2 = off;  off += (int)mb_ptile_bytes(Cs_out, NH);
   s.coef = off; off += 2 * 13 * NH * 4;
@@ -85,6 +87,18 @@ __device__ __forceinline__ float4 act4(float4 v, int act) {
   return make_float4(apply_act(v.x, act), apply_act(v.y, act), apply_act(v.z, act), apply_act(v.w, act));
 }
 
+// acc += a * b on two float32 lanes with one instruction (same rounding as two fmaf)
+__device__ __forceinline__ void ffma2(float& acc0, float& acc1, float a0, float a1, float b0, float b1) {
+  asm("{\n\t.reg .b64 ra, rb, rc;\n\t"
+      "mov.b64 ra, {%2, %3};\n\t"
+      "mov.b64 rb, {%4, %5};\n\t"
+      "mov.b64 rc, {%0, %1};\n\t"
+      "fma.rn.f32x2 rc, ra, rb, rc;\n\t"
+      "mov.b64 {%0, %1}, rc;\n\t}"
+      : "+f"(acc0), "+f"(acc1)
+      : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
 __device__ __forceinline__ void mb_cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
@@ -96,7 +110,7 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
   const LayerJob job = jobs[blockIdx.y];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int NH = p.NH;
-  const MbSmem sm = mb_smem(p.Cs_in, p.Cs_out, p.T1, NH);
+  const MbSmem sm = mb_smem(p.Cs_in, p.Cs_out, p.T1, NH, p.hid_px);
   uint8_t* a_in = smem + sm.a_in;
   uint8_t* b1 = smem + sm.b1;
   uint8_t* hid = smem + sm.hid;
@@ -120,13 +134,31 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
   const int rows_in = (rb - 1) * p.stride + 3;
   const int Ph = rows_in * p.W;                      // hidden pixels of the band
   const int t1 = (Ph + 127) >> 7;
+  const int Wp = p.W + 2;                            // hidden rows carry a zero column on both sides
+  // Per lane, fixed over the chunks: where this lane's accumulator row of tile t goes in a hidden plane
+  // (-1: past the band; bit 30: the row lies outside the image and is stored as zeros), and where the
+  // 3x3 window of its it-th output pixel starts (-1: no such pixel)
+  int hoff[5], dbase[4];
+#pragma unroll
+  for (int t = 0; t < 5; ++t) {
+    const int ph = t * 128 + (warp & 3) * 32 + lane;
+    const int rr = ph / p.W, xx = ph - rr * p.W;
+    const int y_in = y_first + rr;
+    hoff[t] = ph < Ph ? (((rr * Wp + xx + 1) * 16) | ((y_in < 0 || y_in >= p.H) ? (1 << 30) : 0)) : -1;
+  }
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int o = it * 32 + lane;
+    const int yo = o / p.Wo, xo = o - yo * p.Wo;
+    dbase[it] = o < Po ? ((yo * p.stride) * Wp + xo * p.stride) * 16 : -1;
+  }
 
   if (tid == 0) {
     for (int i = 0; i < 6; ++i) mbar_init(bar1 + 8 * i, 1);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 0) {
+  if (warp == kMbWorkers) {
     tmem_alloc(smem_u32(s_tmem), (uint32_t)p.tmem_cols);
     tmem_relinquish();
   }
@@ -146,7 +178,7 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
   }
   // ---- operand images of a chunk: bulk copies issued by thread 0 ---------------------------------
   const int etile_bytes = (int)mb_etile_bytes(p.Cs_in, NH), ptile_bytes = (int)mb_ptile_bytes(p.Cs_out, NH);
-  const int b1_lbo = NH * 16 + 16, b2_lbo = p.Cs_out * 16 + 16;   // plane strides of the weight images
+  const int b1_lbo = NH * 16, b2_lbo = p.Cs_out * 16;   // plane strides of the weight images
   int n_w1 = 0, n_w2 = 0, n_cf0 = 0, n_cf1 = 0;      // copies issued per barrier (thread 0)
   auto load_expand = [&](int cc) {                   // expansion image of chunk cc -> b1
     mbar_expect_tx(bar_w1, (uint32_t)etile_bytes);
@@ -172,23 +204,22 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
   const uint32_t d1_col = (uint32_t)p.Cs_out;        // expansion accumulators behind the output accumulator
   const int n_halves = p.Cs_out > 256 ? 2 : 1;
   const int n_half = p.Cs_out / n_halves;
-  // expansion MMAs of chunk cc: all tiles of the band, hi and lo halves of the pixels (called by warp 0)
+  // expansion MMAs of chunk cc: all tiles of the band, hi and lo halves of the pixels (called by the issuing warp)
   auto issue_expand = [&](int cc, uint32_t tmem_base) {
     const int nh = min(NH, p.Ch - cc * NH);
     if (!mbar_wait_warp(bar_w1, (uint32_t)(cc & 1), s_abort, p.error_flag)) return;   // the chunk's image has landed
     const uint32_t idesc = IDESC0 | ((uint32_t)(nh >> 3) << 17);
-    const uint32_t a_lbo_field = ((uint32_t)sm.a_lbo >> 4) << 16;
-    const uint32_t b_lbo_field = ((uint32_t)b1_lbo >> 4) << 16;
-    const int planes = p.Cs_in / 8;
+    // low descriptor words (address and plane stride in 16-byte units) advance by constant steps
+    const uint32_t a_base = (smem_u32(a_in) >> 4) | (((uint32_t)sm.a_lbo >> 4) << 16);
+    const uint32_t b_base = (smem_u32(b1) >> 4) | (((uint32_t)b1_lbo >> 4) << 16);
+    const uint32_t a_kk = (uint32_t)(2 * sm.a_lbo) >> 4, a_part = (uint32_t)((p.Cs_in / 8) * sm.a_lbo) >> 4, b_kk = (uint32_t)(2 * b1_lbo) >> 4;
+    const int ksteps = p.Cs_in / 16;
     for (int t = 0; t < t1; ++t) {
+      const uint32_t d = tmem_base + d1_col + (uint32_t)(t * NH);
       for (int part = 0; part < 2; ++part) {
-        for (int kk = 0; kk < p.Cs_in / 16; ++kk) {
-          const uint32_t a_addr = smem_u32(a_in) + (uint32_t)(part * planes + 2 * kk) * (uint32_t)sm.a_lbo + (uint32_t)t * 2048u;
-          const uint32_t b_addr = smem_u32(b1) + (uint32_t)(2 * kk) * (uint32_t)b1_lbo;
-          umma_bf16(tmem_base + d1_col + (uint32_t)(t * NH),
-                    ((uint64_t)DESC_HI << 32) | (uint64_t)((a_addr >> 4) | a_lbo_field),
-                    ((uint64_t)DESC_HI << 32) | (uint64_t)((b_addr >> 4) | b_lbo_field), idesc, (part | kk) ? 1u : 0u);
-        }
+        uint32_t a_lo = a_base + (uint32_t)t * 128u + (uint32_t)part * a_part, b_lo = b_base;
+        for (int kk = 0; kk < ksteps; ++kk, a_lo += a_kk, b_lo += b_kk)
+          umma_bf16(d, ((uint64_t)DESC_HI << 32) | a_lo, ((uint64_t)DESC_HI << 32) | b_lo, idesc, (part | kk) ? 1u : 0u);
       }
     }
     umma_commit(bar1);
@@ -199,134 +230,142 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
     s_p[n] = n < p.Cout ? job.scale[n] : 0.f;
     b_p[n] = n < p.Cout ? job.bias[n] : 0.f;
   }
+  // the zero columns left and right of every hidden row: written once, no pass touches them again
+  for (int i = tid; i < (NH >> 2) * rows_in * 2; i += kMbThreads) {
+    const int pl = i / (rows_in * 2), r = (i >> 1) % rows_in, side = i & 1;
+    *reinterpret_cast<float4*>(hid + (size_t)pl * sm.hid_plane + (size_t)(r * Wp + side * (Wp - 1)) * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   tc_fence_before();
   __syncthreads();                                   // barriers initialised, band in place, tensor memory allocated
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  if (tid == 0) {
+  if (tid == kMbLeader) {
     load_expand(0);
     load_coef(0);
     load_project(0);
     if (p.n_chunks > 1) load_coef(1);
   }
-  if (warp == 0) issue_expand(0, tmem_base);
+  if (warp == kMbWorkers) issue_expand(0, tmem_base);
   bool alive = true;
 
   for (int c = 0; c < p.n_chunks; ++c) {
     const int nh = min(NH, p.Ch - c * NH);           // a multiple of 16
     // ---- A. expansion accumulators of chunk c -> hidden chunk (float32) ------------------------
     {
-      const bool ok = mbar_wait(bar1, (uint32_t)(c & 1), s_abort, p.error_flag) &&
-                      mbar_wait(bar_cf + 8 * (c & 1), (uint32_t)((c >> 1) & 1), s_abort, p.error_flag);
+      // one warp polls the barriers; the others wait at the block barrier, which costs neither issue slots nor
+      // shared-memory bandwidth (seventeen polling warps slowed the very MMAs they were waiting for)
+      bool ok = true;
+      if (warp == kMbWorkers)
+        ok = mbar_wait_warp(bar1, (uint32_t)(c & 1), s_abort, p.error_flag) &&
+             mbar_wait_warp(bar_cf + 8 * (c & 1), (uint32_t)((c >> 1) & 1), s_abort, p.error_flag);
       alive = __syncthreads_and(ok);
       if (!alive) break;
       tc_fence_after();
-      if (tid == 0 && c + 1 < p.n_chunks) load_expand(c + 1);   // chunk c's expansion MMAs are done: b1 is free
+      if (tid == kMbLeader && c + 1 < p.n_chunks) load_expand(c + 1);   // chunk c's expansion MMAs are done: b1 is free
       const int q = warp & 3, h = warp >> 2;
       const int groups = nh >> 4;
       const float* se = coef + (c & 1) * 13 * NH;
       const float* be = se + NH;
-      for (int g = h; g < t1 * groups; g += kMbWarps / 4) {
-        const int t = g / groups, cg = g - t * groups;
-        uint32_t v[16];
-        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + d1_col + (uint32_t)(t * NH + cg * 16), v);
-        tmem_ld_wait();
-        const int ph = t * 128 + q * 32 + lane;
-        const int y_in = y_first + ph / p.W;
-        const bool valid = ph < Ph && y_in >= 0 && y_in < p.H;
+      if (warp < kMbWorkers) {
 #pragma unroll
-        for (int e = 0; e < 16; e += 4) {
-          float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (valid) {
-            const float4 sc = *reinterpret_cast<const float4*>(se + cg * 16 + e);
-            const float4 bi = *reinterpret_cast<const float4*>(be + cg * 16 + e);
-            o = act4(make_float4(fmaf(__uint_as_float(v[e]), sc.x, bi.x), fmaf(__uint_as_float(v[e + 1]), sc.y, bi.y),
-                                 fmaf(__uint_as_float(v[e + 2]), sc.z, bi.z), fmaf(__uint_as_float(v[e + 3]), sc.w, bi.w)),
-                     p.act_e);
+        for (int t = 0; t < 5; ++t) {
+          if (t >= t1) break;
+          for (int cg = 0; cg < groups; ++cg) {
+            if (((t * groups + cg) & 3) != h) continue;      // the four warps of a lane quarter take turns
+            uint32_t v[16];
+            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + d1_col + (uint32_t)(t * NH + cg * 16), v);
+            tmem_ld_wait();
+            if (hoff[t] < 0) continue;
+            const bool outside = (hoff[t] >> 30) & 1;
+            uint8_t* dst = hid + (size_t)(cg * 4) * sm.hid_plane + (hoff[t] & 0xFFFFFF);
+#pragma unroll
+            for (int e = 0; e < 16; e += 4) {
+              const float4 sc = *reinterpret_cast<const float4*>(se + cg * 16 + e);
+              const float4 bi = *reinterpret_cast<const float4*>(be + cg * 16 + e);
+              float4 o = make_float4(bi.x, bi.y, bi.z, bi.w);
+              ffma2(o.x, o.y, __uint_as_float(v[e]), __uint_as_float(v[e + 1]), sc.x, sc.y);
+              ffma2(o.z, o.w, __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]), sc.z, sc.w);
+              o = act4(o, p.act_e);
+              if (outside) o = make_float4(0.f, 0.f, 0.f, 0.f);
+              *reinterpret_cast<float4*>(dst + (size_t)(e >> 2) * sm.hid_plane) = o;
+            }
           }
-          *reinterpret_cast<float4*>(hid + (size_t)((cg * 16 + e) >> 2) * sm.hid_plane + ph * 16) = o;
         }
       }
     }
     // ---- B. the projection of chunk c - 1 must have read a2 and b2 -----------------------------------
     if (c > 0) {
-      const bool ok = mbar_wait(bar2, (uint32_t)((c - 1) & 1), s_abort, p.error_flag);
+      bool ok = true;
+      if (warp == kMbWorkers) ok = mbar_wait_warp(bar2, (uint32_t)((c - 1) & 1), s_abort, p.error_flag);
       tc_fence_before();
       alive = __syncthreads_and(ok);                 // also: the hidden chunk is complete, the accumulators are read
       if (!alive) break;
-      if (tid == 0) load_project(c);
+      if (tid == kMbLeader) load_project(c);
     } else {
       tc_fence_before();
       __syncthreads();
     }
     // ---- C. expansion MMAs of the next chunk run behind the depthwise pass; next fetches ----------
-    if (warp == 0 && c + 1 < p.n_chunks) {
+    if (warp == kMbWorkers && c + 1 < p.n_chunks) {
       tc_fence_after();
       issue_expand(c + 1, tmem_base);
     }
     // ---- D. depthwise 3x3 on the hidden chunk -> A operand of the projection ---------------------
-    for (int pl = warp; pl < (nh >> 2); pl += kMbWarps) {
+    for (int pl = warp < kMbWorkers ? warp : (nh >> 2); pl < (nh >> 2); pl += kMbWorkers) {
       float4 wv[9];
-#pragma unroll
       const float* w_d = coef + (c & 1) * 13 * NH + 2 * NH;       // [9][NH], then s_d [NH], b_d [NH]
+#pragma unroll
       for (int t = 0; t < 9; ++t) wv[t] = *reinterpret_cast<const float4*>(w_d + t * NH + pl * 4);
       const float4 sc = *reinterpret_cast<const float4*>(w_d + 9 * NH + pl * 4);
       const float4 bi = *reinterpret_cast<const float4*>(w_d + 10 * NH + pl * 4);
       const uint8_t* hp = hid + (size_t)pl * sm.hid_plane;
       uint8_t* dst_hi = a2 + (size_t)(pl >> 1) * 2048 + (pl & 1) * 8;
       uint8_t* dst_lo = dst_hi + (size_t)(NH >> 3) * 2048;
-      for (int o = lane; o < Po; o += 32) {
-        const int yo = o / p.Wo, xo = o - yo * p.Wo;
-        // columns left and right of the image: the tap reads a clamped column and is weighted by zero
-        const int xc = xo * p.stride;
-        const int x0 = max(xc - 1, 0), x2 = min(xc + 1, p.W - 1);
-        const float m0 = xc >= 1 ? 1.f : 0.f, m2 = xc + 1 < p.W ? 1.f : 0.f;
-        const uint8_t* r0 = hp + (size_t)(yo * p.stride * p.W) * 16;
+#pragma unroll
+      for (int it = 0; it < 4; ++it) {
+        if (dbase[it] < 0) continue;
+        const uint8_t* r0 = hp + dbase[it];
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int dy = 0; dy < 3; ++dy) {
-          const uint8_t* rr = r0 + (size_t)(dy * p.W) * 16;
-          const float4 h0 = *reinterpret_cast<const float4*>(rr + x0 * 16);
-          const float4 h1 = *reinterpret_cast<const float4*>(rr + xc * 16);
-          const float4 h2 = *reinterpret_cast<const float4*>(rr + x2 * 16);
-          const float4 w0 = wv[dy * 3], w1 = wv[dy * 3 + 1], w2 = wv[dy * 3 + 2];
-          acc.x = fmaf(h0.x * m0, w0.x, acc.x); acc.y = fmaf(h0.y * m0, w0.y, acc.y);
-          acc.z = fmaf(h0.z * m0, w0.z, acc.z); acc.w = fmaf(h0.w * m0, w0.w, acc.w);
-          acc.x = fmaf(h1.x, w1.x, acc.x); acc.y = fmaf(h1.y, w1.y, acc.y);
-          acc.z = fmaf(h1.z, w1.z, acc.z); acc.w = fmaf(h1.w, w1.w, acc.w);
-          acc.x = fmaf(h2.x * m2, w2.x, acc.x); acc.y = fmaf(h2.y * m2, w2.y, acc.y);
-          acc.z = fmaf(h2.z * m2, w2.z, acc.z); acc.w = fmaf(h2.w * m2, w2.w, acc.w);
+#pragma unroll
+          for (int dx = 0; dx < 3; ++dx) {
+            const float4 hv = *reinterpret_cast<const float4*>(r0 + (size_t)(dy * Wp + dx) * 16);
+            const float4 w = wv[dy * 3 + dx];
+            ffma2(acc.x, acc.y, hv.x, hv.y, w.x, w.y);
+            ffma2(acc.z, acc.w, hv.z, hv.w, w.z, w.w);
+          }
         }
-        const float4 u = act4(make_float4(fmaf(acc.x, sc.x, bi.x), fmaf(acc.y, sc.y, bi.y), fmaf(acc.z, sc.z, bi.z),
-                                          fmaf(acc.w, sc.w, bi.w)), p.act_d);
+        float4 u = bi;
+        ffma2(u.x, u.y, acc.x, acc.y, sc.x, sc.y);
+        ffma2(u.z, u.w, acc.z, acc.w, sc.z, sc.w);
+        u = act4(u, p.act_d);
         uint2 hi, lo;
         split_pair(u.x, u.y, hi.x, lo.x);
         split_pair(u.z, u.w, hi.y, lo.y);
+        const int o = it * 32 + lane;
         *reinterpret_cast<uint2*>(dst_hi + o * 16) = hi;
         *reinterpret_cast<uint2*>(dst_lo + o * 16) = lo;
       }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
-    if (tid == 0 && c + 2 < p.n_chunks) load_coef(c + 2);        // this chunk's coefficient buffer is free
+    if (tid == kMbLeader && c + 2 < p.n_chunks) load_coef(c + 2);        // this chunk's coefficient buffer is free
     // ---- E. projection MMAs of the chunk (they run behind step A of the next chunk) ----------------
-    if (warp == 0 && mbar_wait_warp(bar_w2, (uint32_t)(c & 1), s_abort, p.error_flag)) {
+    if (warp == kMbWorkers && mbar_wait_warp(bar_w2, (uint32_t)(c & 1), s_abort, p.error_flag)) {
       tc_fence_after();
       const uint32_t idesc = IDESC0 | ((uint32_t)(n_half >> 3) << 17);
-      const uint32_t a_lbo_field = (2048u >> 4) << 16;
-      const uint32_t b_lbo_field = ((uint32_t)b2_lbo >> 4) << 16;
+      const uint32_t a_base = (smem_u32(a2) >> 4) | ((2048u >> 4) << 16);
+      const uint32_t b_base = (smem_u32(b2) >> 4) | (((uint32_t)b2_lbo >> 4) << 16);
+      const uint32_t b_kk = (uint32_t)(2 * b2_lbo) >> 4, b_half = (uint32_t)(n_half * 16) >> 4;
       for (int part = 0; part < 2; ++part) {
-        for (int kk = 0; kk < (nh >> 4); ++kk) {
-          const uint32_t a_addr = smem_u32(a2) + (uint32_t)(part * (NH >> 3) + 2 * kk) * 2048u;
-          for (int hf = 0; hf < n_halves; ++hf) {
-            const uint32_t b_addr = smem_u32(b2) + (uint32_t)(2 * kk) * (uint32_t)b2_lbo + (uint32_t)(hf * n_half * 16);
-            umma_bf16(tmem_base + (uint32_t)(hf * n_half),
-                      ((uint64_t)DESC_HI << 32) | (uint64_t)((a_addr >> 4) | a_lbo_field),
-                      ((uint64_t)DESC_HI << 32) | (uint64_t)((b_addr >> 4) | b_lbo_field), idesc, (c | part | kk) ? 1u : 0u);
-          }
-        }
+        uint32_t a_lo = a_base + (uint32_t)(part * (NH >> 3)) * 128u, b_lo = b_base;
+        for (int kk = 0; kk < (nh >> 4); ++kk, a_lo += 256u, b_lo += b_kk)
+          for (int hf = 0; hf < n_halves; ++hf)
+            umma_bf16(tmem_base + (uint32_t)(hf * n_half), ((uint64_t)DESC_HI << 32) | a_lo,
+                      ((uint64_t)DESC_HI << 32) | (b_lo + (uint32_t)hf * b_half), idesc, (c | part | kk) ? 1u : 0u);
       }
       umma_commit(bar2);
     }
@@ -334,7 +373,8 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
 
   // ---- output: accumulator -> scale, bias, shortcut, activation -> hi / lo pixels ------------------
   if (alive) {
-    const bool ok = mbar_wait(bar2, (uint32_t)((p.n_chunks - 1) & 1), s_abort, p.error_flag);
+    bool ok = true;
+    if (warp == kMbWorkers) ok = mbar_wait_warp(bar2, (uint32_t)((p.n_chunks - 1) & 1), s_abort, p.error_flag);
     alive = __syncthreads_and(ok);
   }
   if (alive) {
@@ -346,7 +386,7 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
     const size_t opix = ((size_t)img * (p.Ho + 2) + (size_t)(yo + 1)) * p.Wo + xo;   // shortcut: same geometry
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(job.out) + opix * (size_t)(2 * p.Cs_out);
     const __nv_bfloat16* res = job.res ? static_cast<const __nv_bfloat16*>(job.res) + opix * (size_t)(2 * p.Cs_out) : nullptr;
-    for (int cg = h; cg < (p.Cs_out >> 4); cg += kMbWarps / 4) {
+    for (int cg = warp < kMbWorkers ? h : (p.Cs_out >> 4); cg < (p.Cs_out >> 4); cg += kMbWorkers / 4) {
       uint32_t v[16];
       tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(cg * 16), v);
       tmem_ld_wait();
@@ -387,7 +427,7 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
   }
 
   // ---- teardown -------------------------------------------------------------------------------
-  if (!alive && tid == 0) {                          // copies in flight must land before the CTA exits
+  if (!alive && tid == kMbLeader) {                          // copies in flight must land before the CTA exits
     const uint32_t bars[4] = {bar_w1, bar_w2, bar_cf, bar_cf + 8};
     const int issued[4] = {n_w1, n_w2, n_cf0, n_cf1};
     for (int i = 0; i < 4; ++i) {
@@ -398,16 +438,16 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == kMbWorkers) {
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
   }
 }
 
 // Operand images of a block's layers, built once per weight version (see the file header):
-//   role 0, expansion  (N = Ch rows of K = Cin codes): per chunk [Cs_in / 8 planes][NH rows + 1][8 bfloat16];
+//   role 0, expansion  (N = Ch rows of K = Cin codes): per chunk [Cs_in / 8 planes][NH rows][8 bfloat16];
 //           coefficients per chunk: s_e [NH], b_e [NH]
-//   role 1, projection (N = Cout rows of K = Ch codes): per chunk [NH / 8 planes][Cs_out rows + 1][8 bfloat16]
+//   role 1, projection (N = Cout rows of K = Ch codes): per chunk [NH / 8 planes][Cs_out rows][8 bfloat16]
 //   role 2, depthwise  (N = Ch rows of 9 elements): coefficients per chunk: w [9][NH], s_d [NH], b_d [NH]
 // Rows, planes and channels past the layer's extent are zero.
 __global__ void mb_build_tiles_kernel(int role, const uint8_t* __restrict__ packed, const float* __restrict__ scale,
@@ -419,13 +459,13 @@ __global__ void mb_build_tiles_kernel(int role, const uint8_t* __restrict__ pack
   const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gsize = gridDim.x * blockDim.x;
   if (role == 0 || role == 1) {
     const int planes = role == 0 ? cs / 8 : NH / 8;
-    const int rows = (role == 0 ? NH : cs) + 1;      // + the 16 padding bytes of a plane
+    const int rows = role == 0 ? NH : cs;
     const int units = n_chunks * planes * rows;
     for (int u = gtid; u < units; u += gsize) {
       const int r = u % rows, j = (u / rows) % planes, c = u / (rows * planes);
       const int n = role == 0 ? c * NH + r : r;      // weight row
       const int k = role == 0 ? j * 8 : c * NH + j * 8;
-      const bool real = r < rows - 1 && n < N && k < K && (role == 0 ? r < NH : true);
+      const bool real = n < N && k < K;
       uint2 raw = make_uint2(0u, 0u);
       if (real) {
         const uint8_t* row = packed + (size_t)n * wrow;
@@ -468,7 +508,7 @@ MbConfig mb_config(const ConvGeom& ge, const ConvGeom& gd, const ConvGeom& gp, i
       const int nh = order[i][0], occ = order[i][1];
       int cols = 32;
       while (cols < cs_out + T1 * nh) cols <<= 1;
-      const int bytes = mb_smem(cs_in, cs_out, T1, nh).total + 128;
+      const int bytes = mb_smem(cs_in, cs_out, T1, nh, rows_in * (gd.W + 2)).total + 128;
       if (cols > 512 || bytes > smem_optin) continue;
       c.Rb = rb; c.bands = (gp.Ho + rb - 1) / rb; c.T1 = T1;
       c.NH = nh; c.occ = occ; c.tmem_cols = cols; c.smem_bytes = bytes; c.ok = true;
@@ -525,6 +565,7 @@ aiq_status_t launch_mb_block(const ConvGeom& ge, const ConvGeom& gd, const ConvG
   p.Cin = ge.Cin; p.Cs_in = padded_channels(ge.Cin); p.Ch = ge.Cout; p.Cout = gp.Cout; p.Cs_out = padded_channels(gp.Cout);
   p.Rb = c.Rb; p.bands = c.bands; p.T1 = c.T1; p.NH = c.NH; p.n_chunks = (p.Ch + c.NH - 1) / c.NH;
   p.tmem_cols = c.tmem_cols;
+  p.hid_px = ((c.Rb - 1) * gd.stride + 3) * (gd.W + 2);
   p.act_e = ge.act; p.act_d = gd.act; p.act_p = gp.act;
   p.error_flag = error_flag;
   AIQ_ENSURE_DYNAMIC_SMEM(mb_block_kernel, props.smem_optin);

@@ -26,7 +26,7 @@ static std::atomic<int> g_opt_chunk{0};
 static std::atomic<int> g_opt_share{1};
 static std::atomic<int> g_opt_path{AIQ_PATH_AUTO};
 static std::atomic<int> g_opt_per_tensor{0};  // scale granularity of models created afterwards
-static std::atomic<int> g_opt_fuse{1};        // basic blocks as one kernel
+static std::atomic<int> g_opt_fuse{1};        // bit 0: basic blocks as one kernel; bit 1: inverted-residual blocks as one kernel
 static std::atomic<int> g_opt_fuse_pool{1};   // average pool inside the last convolution's epilogue
 
 aiq_status_t set_error(aiq_status_t status, const char* fmt, ...) {
@@ -684,7 +684,8 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
   plan.batch_capacity = B;
   std::vector<std::vector<int>> ver(n, std::vector<int>(S, 0));   // ver[l][s]
   std::vector<std::vector<std::tuple<int, int, int>>> all_keys(n);   // per layer and version: (bits, input version, residual version)
-  const bool fuse = g_opt_fuse.load() != 0;
+  const bool fuse = (g_opt_fuse.load() & 1) != 0;
+  const bool fuse_mb = (g_opt_fuse.load() & 2) != 0;
   // a basic block runs as one kernel when every scheme gives both of its convolutions 4 or 8 bits
   std::vector<int> fuse_head(n, -1);
   if (fuse)
@@ -698,7 +699,7 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
   // an inverted-residual block runs as one kernel when every scheme gives its two 1x1 layers 4 or 8 bits
   std::vector<int> mb_head(n, -1);
   std::vector<char> mb_absorbed(n, 0);
-  if (fuse)
+  if (fuse_mb)
     for (int le = 0; le < n; ++le) {
       const int lt = m->mb_tail[le];
       if (lt < 0) continue;
@@ -1025,7 +1026,7 @@ extern "C" void aiq_set_scale_granularity(int granularity) {
 }
 
 extern "C" void aiq_set_fusion(int blocks, int pool) {
-  aiq::g_opt_fuse = blocks ? 1 : 0;
+  aiq::g_opt_fuse = blocks & 3;
   aiq::g_opt_fuse_pool = pool ? 1 : 0;
 }
 

@@ -37,15 +37,14 @@ def test_fused_block_tight_tolerance(cin, cout, hw, stride):
         for scheme in ([8, 8, 8, 8, 8], [8, 4, 8, 4, 8], [8, 8, 4, 8, 4]):
             scheme = np.array(scheme, np.uint8)
             ref = O.forward_scheme(arch, bank, scheme, x)
-            aiq.aiq_set_fusion(True, True)
-            got = model.aiq_forward(scheme, xd).cpu().numpy()
-            fused_launches = aiq.aiq_last_call_stats()["kernel_launches"]
-            aiq.aiq_set_fusion(False, True)
+            aiq.aiq_set_fusion(True, True, inverted_residual=True)
             try:
-                plain = model.aiq_forward(scheme, xd).cpu().numpy()
-                plain_launches = aiq.aiq_last_call_stats()["kernel_launches"]
+                got = model.aiq_forward(scheme, xd).cpu().numpy()
+                fused_launches = aiq.aiq_last_call_stats()["kernel_launches"]
             finally:
                 aiq.aiq_set_fusion(True, True)
+            plain = model.aiq_forward(scheme, xd).cpu().numpy()
+            plain_launches = aiq.aiq_last_call_stats()["kernel_launches"]
             what = f"block {cin}->{cout} {hw}x{hw} stride {stride} batch {batch} scheme {scheme.tolist()}"
             assert fused_launches == plain_launches - 2, what
             assert_logits_close(got, ref, what + " fused")
@@ -74,7 +73,42 @@ def test_fused_block_versions_share_one_launch():
                        np.uint8)
     oacc, ocounts, opreds, omargins = O.eval_schemes(arch, bank, schemes, x, labels)
     preds = torch.full((len(schemes), 40), -1, dtype=torch.int32, device="cuda")
-    acc, counts = model.aiq_eval_schemes(schemes, to_dev(x), to_dev(labels), preds=preds, chunk=40)
+    aiq.aiq_set_fusion(True, True, inverted_residual=True)
+    try:
+        acc, counts = model.aiq_eval_schemes(schemes, to_dev(x), to_dev(labels), preds=preds, chunk=40)
+        fused_launches = aiq.aiq_last_call_stats()["kernel_launches"]
+    finally:
+        aiq.aiq_set_fusion(True, True)
+    model.aiq_eval_schemes(schemes, to_dev(x), to_dev(labels), chunk=40)
+    assert fused_launches < aiq.aiq_last_call_stats()["kernel_launches"]
     assert_preds_match(preds.cpu().numpy(), opreds, omargins, "fused block, six candidates")
     assert np.all(np.abs(counts - ocounts) <= (omargins <= 1e-2).sum(axis=1))
+    model.close()
+
+
+@pytest.mark.parametrize("variant,hw,batch", [("cifar", 32, 24), ("imagenet", 224, 3)])
+def test_mobilenet_v2_with_fused_blocks(variant, hw, batch):
+    """The whole MobileNetV2 (16 of its 17 blocks fused, 10 seeded conv layers at 4 bits) against the
+    oracle at the tensor-path tolerance, with the classifier balanced so that the labels spread."""
+    from aiq_workloads import mobilenet_v2, mixed_int4_int8_scheme, conv_layer_indices
+    from gpu_util import assert_preds_match
+    from test_gpu_forward import balance_classifier, assert_tensor_path_logits
+    aiq = binding()
+    arch = mobilenet_v2(variant)
+    x = gen_images(batch, 3, hw, hw, 8624)
+    params = balance_classifier(arch, gen_model(arch, 2234), x)
+    model = aiq.Model(arch, params)
+    bank = O.build_weight_bank(O.fold_model(arch, params), (4, 8))
+    scheme = mixed_int4_int8_scheme(53, conv_layer_indices(arch), 10, 43)
+    ref = O.forward_scheme(arch, bank, scheme, x)
+    aiq.aiq_set_fusion(True, True, inverted_residual=True)
+    try:
+        got = model.aiq_forward(scheme, to_dev(x)).cpu().numpy()
+        fused_launches = aiq.aiq_last_call_stats()["kernel_launches"]
+    finally:
+        aiq.aiq_set_fusion(True, True)
+    model.aiq_forward(scheme, to_dev(x))
+    assert fused_launches <= aiq.aiq_last_call_stats()["kernel_launches"] - 2 * 15
+    assert_tensor_path_logits(got, ref, f"mbv2 {variant} fused blocks")
+    assert_preds_match(O.predict(got), O.predict(ref), O.top2_margin(ref), f"mbv2 {variant} fused blocks")
     model.close()
