@@ -318,6 +318,8 @@ def run_kernel_sweep(args):
     from paper_2512_14090_b200 import build
     build.build()
     from paper_2512_14090_b200 import binding as aiq
+    if args.fuse_inverted_residual:
+        aiq.aiq_set_fusion(True, True, inverted_residual=True)
     from aiq_workloads import gen_linear_case
     peaks = measured_peaks()
     dev = torch.device("cuda", 0)
@@ -441,6 +443,8 @@ def main():
                          "standalone memory-bound kernels; forward: one scheme, one batch; search: the two searches "
                          "of Section 2.2 on ResNet-20; sensitivity: every layer alone at 8 / 4 bits from an FP32 "
                          "base (all 1 GPU)")
+    ap.add_argument("--fuse-inverted-residual", action="store_true",
+                    help="run MobileNetV2's inverted-residual blocks as one kernel each (aiq_set_fusion bit 1)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -461,6 +465,8 @@ def main():
     from paper_2512_14090_b200 import build
     build.build()
     from paper_2512_14090_b200 import binding as aiq          # fails loudly without libaiq.so
+    if args.fuse_inverted_residual:
+        aiq.aiq_set_fusion(True, True, inverted_residual=True)
     from paper_2512_14090_b200.sharding import reduce_counts
     from aiq_workloads import gen_model, gen_images
 

@@ -79,7 +79,7 @@ __host__ __device__ inline MbSmem mb_smem(int Cs_in, int Cs_out, int T1, int NH,
   s.coef = off; off += 2 * 13 * NH * 4;
   s.proj = off; off += 2 * Cs_out * 4;
   s.bars = (off + 15) / 16 * 16;
-  s.total = s.bars + 6 * 8 + 16;
+  s.total = s.bars + 8 * 8 + 16;
   return s;
 }
 
@@ -120,9 +120,11 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
   float* s_p = reinterpret_cast<float*>(smem + sm.proj);
   float* b_p = s_p + p.Cs_out;
   // mbarriers: expansion MMAs done, projection MMAs done, expansion image landed, projection image
-  // landed, coefficients of an even / odd chunk landed
+  // landed, coefficients of an even / odd chunk landed, every worker warp has read the expansion
+  // accumulators, every worker warp has written its part of the projection operand
   const uint32_t bar1 = smem_u32(smem + sm.bars), bar2 = bar1 + 8, bar_w1 = bar1 + 16, bar_w2 = bar1 + 24, bar_cf = bar1 + 32;
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + sm.bars + 48);
+  const uint32_t bar_hid = bar1 + 48, bar_a2 = bar1 + 56;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + sm.bars + 64);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   // ---- this CTA's band ------------------------------------------------------------------------
@@ -155,6 +157,8 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
 
   if (tid == 0) {
     for (int i = 0; i < 6; ++i) mbar_init(bar1 + 8 * i, 1);
+    mbar_init(bar_hid, kMbWorkers);
+    mbar_init(bar_a2, kMbWorkers);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -249,21 +253,32 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
   }
   if (warp == kMbWorkers) issue_expand(0, tmem_base);
   bool alive = true;
+  // named barrier of the 16 worker warps; the issuing warp runs beside them and meets them only through mbarriers
+  // Whether to go on is decided by one thread before the barrier and read by all after it (two slots, used in
+  // turn), so that every worker warp leaves the loop at the same barrier.
+  volatile int* s_go = s_abort + 1;
+  int sync_k = 0;
+  auto workers_sync = [&]() -> bool {
+    if (tid == 0) s_go[sync_k & 1] = *s_abort == 0;
+    asm volatile("bar.sync 1, %0;" ::"n"(kMbWorkers * 32) : "memory");
+    const bool go = s_go[sync_k & 1] != 0;
+    ++sync_k;
+    return go;
+  };
 
-  for (int c = 0; c < p.n_chunks; ++c) {
-    const int nh = min(NH, p.Ch - c * NH);           // a multiple of 16
-    // ---- A. expansion accumulators of chunk c -> hidden chunk (float32) ------------------------
-    {
-      // one warp polls the barriers; the others wait at the block barrier, which costs neither issue slots nor
-      // shared-memory bandwidth (seventeen polling warps slowed the very MMAs they were waiting for)
-      bool ok = true;
-      if (warp == kMbWorkers)
-        ok = mbar_wait_warp(bar1, (uint32_t)(c & 1), s_abort, p.error_flag) &&
-             mbar_wait_warp(bar_cf + 8 * (c & 1), (uint32_t)((c >> 1) & 1), s_abort, p.error_flag);
-      alive = __syncthreads_and(ok);
-      if (!alive) break;
+  if (warp < kMbWorkers) {
+    // =================== worker warps: accumulators -> hidden chunk -> depthwise -> projection operand ===========
+    for (int c = 0; c < p.n_chunks; ++c) {
+      const int nh = min(NH, p.Ch - c * NH);         // a multiple of 16
+      // the chunk's expansion MMAs and coefficients: one warp polls, the others wait at the named barrier (which
+      // also ends the depthwise pass of the chunk before: the hidden tile may be overwritten)
+      if (warp == 0) {
+        mbar_wait_warp(bar1, (uint32_t)(c & 1), s_abort, p.error_flag);
+        mbar_wait_warp(bar_cf + 8 * (c & 1), (uint32_t)((c >> 1) & 1), s_abort, p.error_flag);
+      }
+      if (!workers_sync()) { alive = false; break; }
       tc_fence_after();
-      if (tid == kMbLeader && c + 1 < p.n_chunks) load_expand(c + 1);   // chunk c's expansion MMAs are done: b1 is free
+      // ---- A. expansion accumulators of chunk c -> hidden chunk (float32) ------------------------
       const int q = warp & 3, h = warp >> 2;
       const int groups = nh >> 4;
       const float* se = coef + (c & 1) * 13 * NH;
@@ -294,68 +309,82 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
           }
         }
       }
-    }
-    // ---- B. the projection of chunk c - 1 must have read a2 and b2 -----------------------------------
-    if (c > 0) {
-      bool ok = true;
-      if (warp == kMbWorkers) ok = mbar_wait_warp(bar2, (uint32_t)((c - 1) & 1), s_abort, p.error_flag);
       tc_fence_before();
-      alive = __syncthreads_and(ok);                 // also: the hidden chunk is complete, the accumulators are read
-      if (!alive) break;
-      if (tid == kMbLeader) load_project(c);
-    } else {
-      tc_fence_before();
-      __syncthreads();
-    }
-    // ---- C. expansion MMAs of the next chunk run behind the depthwise pass; next fetches ----------
-    if (warp == kMbWorkers && c + 1 < p.n_chunks) {
-      tc_fence_after();
-      issue_expand(c + 1, tmem_base);
-    }
-    // ---- D. depthwise 3x3 on the hidden chunk -> A operand of the projection ---------------------
-    for (int pl = warp < kMbWorkers ? warp : (nh >> 2); pl < (nh >> 2); pl += kMbWorkers) {
-      float4 wv[9];
-      const float* w_d = coef + (c & 1) * 13 * NH + 2 * NH;       // [9][NH], then s_d [NH], b_d [NH]
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_hid);           // this warp has read its accumulators
+      // the projection of chunk c - 1 must have read a2 before the depthwise pass overwrites it
+      if (warp == 0 && c > 0) mbar_wait_warp(bar2, (uint32_t)((c - 1) & 1), s_abort, p.error_flag);
+      if (!workers_sync()) { alive = false; break; }   // the hidden chunk is complete
+      // ---- D. depthwise 3x3 on the hidden chunk -> A operand of the projection ---------------------
+      for (int pl = warp < kMbWorkers ? warp : (nh >> 2); pl < (nh >> 2); pl += kMbWorkers) {
+        float4 wv[9];
+        const float* w_d = coef + (c & 1) * 13 * NH + 2 * NH;       // [9][NH], then s_d [NH], b_d [NH]
 #pragma unroll
-      for (int t = 0; t < 9; ++t) wv[t] = *reinterpret_cast<const float4*>(w_d + t * NH + pl * 4);
-      const float4 sc = *reinterpret_cast<const float4*>(w_d + 9 * NH + pl * 4);
-      const float4 bi = *reinterpret_cast<const float4*>(w_d + 10 * NH + pl * 4);
-      const uint8_t* hp = hid + (size_t)pl * sm.hid_plane;
-      uint8_t* dst_hi = a2 + (size_t)(pl >> 1) * 2048 + (pl & 1) * 8;
-      uint8_t* dst_lo = dst_hi + (size_t)(NH >> 3) * 2048;
+        for (int t = 0; t < 9; ++t) wv[t] = *reinterpret_cast<const float4*>(w_d + t * NH + pl * 4);
+        const float4 sc = *reinterpret_cast<const float4*>(w_d + 9 * NH + pl * 4);
+        const float4 bi = *reinterpret_cast<const float4*>(w_d + 10 * NH + pl * 4);
+        const uint8_t* hp = hid + (size_t)pl * sm.hid_plane;
+        uint8_t* dst_hi = a2 + (size_t)(pl >> 1) * 2048 + (pl & 1) * 8;
+        uint8_t* dst_lo = dst_hi + (size_t)(NH >> 3) * 2048;
 #pragma unroll
-      for (int it = 0; it < 4; ++it) {
-        if (dbase[it] < 0) continue;
-        const uint8_t* r0 = hp + dbase[it];
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int it = 0; it < 4; ++it) {
+          if (dbase[it] < 0) continue;
+          const uint8_t* r0 = hp + dbase[it];
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int dy = 0; dy < 3; ++dy) {
+          for (int dy = 0; dy < 3; ++dy) {
 #pragma unroll
-          for (int dx = 0; dx < 3; ++dx) {
-            const float4 hv = *reinterpret_cast<const float4*>(r0 + (size_t)(dy * Wp + dx) * 16);
-            const float4 w = wv[dy * 3 + dx];
-            ffma2(acc.x, acc.y, hv.x, hv.y, w.x, w.y);
-            ffma2(acc.z, acc.w, hv.z, hv.w, w.z, w.w);
+            for (int dx = 0; dx < 3; ++dx) {
+              const float4 hv = *reinterpret_cast<const float4*>(r0 + (size_t)(dy * Wp + dx) * 16);
+              const float4 w = wv[dy * 3 + dx];
+              ffma2(acc.x, acc.y, hv.x, hv.y, w.x, w.y);
+              ffma2(acc.z, acc.w, hv.z, hv.w, w.z, w.w);
+            }
           }
+          float4 u = bi;
+          ffma2(u.x, u.y, acc.x, acc.y, sc.x, sc.y);
+          ffma2(u.z, u.w, acc.z, acc.w, sc.z, sc.w);
+          u = act4(u, p.act_d);
+          uint2 hi, lo;
+          split_pair(u.x, u.y, hi.x, lo.x);
+          split_pair(u.z, u.w, hi.y, lo.y);
+          const int o = it * 32 + lane;
+          *reinterpret_cast<uint2*>(dst_hi + o * 16) = hi;
+          *reinterpret_cast<uint2*>(dst_lo + o * 16) = lo;
         }
-        float4 u = bi;
-        ffma2(u.x, u.y, acc.x, acc.y, sc.x, sc.y);
-        ffma2(u.z, u.w, acc.z, acc.w, sc.z, sc.w);
-        u = act4(u, p.act_d);
-        uint2 hi, lo;
-        split_pair(u.x, u.y, hi.x, lo.x);
-        split_pair(u.z, u.w, hi.y, lo.y);
-        const int o = it * 32 + lane;
-        *reinterpret_cast<uint2*>(dst_hi + o * 16) = hi;
-        *reinterpret_cast<uint2*>(dst_lo + o * 16) = lo;
       }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_a2);            // this warp's part of the projection operand is written
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncthreads();
-    if (tid == kMbLeader && c + 2 < p.n_chunks) load_coef(c + 2);        // this chunk's coefficient buffer is free
-    // ---- E. projection MMAs of the chunk (they run behind step A of the next chunk) ----------------
-    if (warp == kMbWorkers && mbar_wait_warp(bar_w2, (uint32_t)(c & 1), s_abort, p.error_flag)) {
+    // the last projection
+    if (alive) {
+      if (warp == 0) mbar_wait_warp(bar2, (uint32_t)((p.n_chunks - 1) & 1), s_abort, p.error_flag);
+      alive = workers_sync();
+    }
+  } else {
+    // =================== issuing warp: bulk copies and MMAs ===================================================
+    for (int c = 0; c < p.n_chunks && alive; ++c) {
+      const int nh = min(NH, p.Ch - c * NH);
+      // chunk c's expansion MMAs are done: b1 is free for the next image
+      alive = mbar_wait_warp(bar1, (uint32_t)(c & 1), s_abort, p.error_flag);
+      if (!alive) break;
+      if (lane == 0 && c + 1 < p.n_chunks) load_expand(c + 1);
+      // every worker has read the accumulators of chunk c: the expansion MMAs of the next chunk may overwrite them
+      alive = mbar_wait_warp(bar_hid, (uint32_t)(c & 1), s_abort, p.error_flag);
+      if (!alive) break;
+      if (c + 1 < p.n_chunks) {
+        tc_fence_after();
+        issue_expand(c + 1, tmem_base);
+      }
+      // the depthwise pass of chunk c is complete: its coefficient buffer is free, the projection can run
+      alive = mbar_wait_warp(bar_a2, (uint32_t)(c & 1), s_abort, p.error_flag);
+      if (!alive) break;
+      if (lane == 0 && c + 2 < p.n_chunks) load_coef(c + 2);
+      alive = mbar_wait_warp(bar_w2, (uint32_t)(c & 1), s_abort, p.error_flag);
+      if (!alive) break;
       tc_fence_after();
+      {
       const uint32_t idesc = IDESC0 | ((uint32_t)(n_half >> 3) << 17);
       const uint32_t a_base = (smem_u32(a2) >> 4) | ((2048u >> 4) << 16);
       const uint32_t b_base = (smem_u32(b2) >> 4) | (((uint32_t)b2_lbo >> 4) << 16);
@@ -367,16 +396,19 @@ mb_block_kernel(MbParams p, const LayerJob* __restrict__ jobs) {
             umma_bf16(tmem_base + (uint32_t)(hf * n_half), ((uint64_t)DESC_HI << 32) | a_lo,
                       ((uint64_t)DESC_HI << 32) | (b_lo + (uint32_t)hf * b_half), idesc, (c | part | kk) ? 1u : 0u);
       }
+      }
       umma_commit(bar2);
+      // the next projection image may land once these MMAs have read b2
+      if (c + 1 < p.n_chunks) {
+        alive = mbar_wait_warp(bar2, (uint32_t)(c & 1), s_abort, p.error_flag);
+        if (!alive) break;
+        if (lane == 0) load_project(c + 1);
+      }
     }
   }
 
   // ---- output: accumulator -> scale, bias, shortcut, activation -> hi / lo pixels ------------------
-  if (alive) {
-    bool ok = true;
-    if (warp == kMbWorkers) ok = mbar_wait_warp(bar2, (uint32_t)((p.n_chunks - 1) & 1), s_abort, p.error_flag);
-    alive = __syncthreads_and(ok);
-  }
+  alive = __syncthreads_and(alive);                  // every thread: the two roles meet again here
   if (alive) {
     tc_fence_after();
     const int q = warp & 3, h = warp >> 2;
