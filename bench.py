@@ -320,6 +320,7 @@ def run_kernel_sweep(args):
     from paper_2512_14090_b200 import binding as aiq
     if args.fuse_inverted_residual:
         aiq.aiq_set_fusion(True, True, inverted_residual=True)
+    aiq.aiq_set_compute_path({"auto": aiq.PATH_AUTO, "tiles": aiq.PATH_TENSOR_TILES, "fp32": aiq.PATH_FP32}[args.path])
     from aiq_workloads import gen_linear_case
     peaks = measured_peaks()
     dev = torch.device("cuda", 0)
@@ -443,6 +444,9 @@ def main():
                          "standalone memory-bound kernels; forward: one scheme, one batch; search: the two searches "
                          "of Section 2.2 on ResNet-20; sensitivity: every layer alone at 8 / 4 bits from an FP32 "
                          "base (all 1 GPU)")
+    ap.add_argument("--path", default="auto", choices=["auto", "tiles", "fp32"],
+                    help="compute path of models created by the kernel workloads: auto (row-streaming tensor-core "
+                         "kernels where the network allows), tiles (pixel-tile tensor-core kernels), fp32")
     ap.add_argument("--fuse-inverted-residual", action="store_true",
                     help="run MobileNetV2's inverted-residual blocks as one kernel each (aiq_set_fusion bit 1)")
     args = ap.parse_args()

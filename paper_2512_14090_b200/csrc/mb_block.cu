@@ -15,19 +15,31 @@
 // expansion for every tile of 128 pixels.  The weights of the two 1x1 layers are kept by the
 // model as ready bfloat16 operand images, one per chunk of hidden channels (built once from
 // the packed codes, exact: integer codes), the depthwise weights as float32 rows; a chunk's
-// images arrive by bulk copies while the chunk before is being computed.  Per chunk:
-//   A. all warps read the expansion accumulators, apply scale, bias and activation and park the
-//      chunk as float32 in shared memory ([4-channel plane][pixel][16 bytes]; rows outside the
-//      image are the depthwise layer's zero padding and are stored as zeros);
-//   C. one elected thread issues the expansion MMAs of the NEXT chunk (hi and lo halves of the
-//      pixels, all tiles of the band into separate accumulator columns); they run behind D;
-//   D. all warps run the depthwise 3x3 from the parked chunk (a lane per output pixel, four
-//      channels per lane, the nine weights of the plane in registers), apply scale, bias,
-//      activation and write the result as hi / lo bfloat16 planes: the A operand of the projection;
-//   E. the elected thread issues the projection MMAs of the chunk, which add to the block's
-//      output accumulator (128 pixels x Cout) in tensor memory; they run behind A of the next chunk.
-// After the last chunk the accumulator gets scale, bias and the shortcut and goes to global
-// memory.  Every wait is bounded as in the other tcgen05 kernels.
+// images arrive by bulk copies while the chunk before is being computed.
+//
+// Roles: 16 worker warps and one issuing warp, which meet only through mbarriers (the workers
+// among themselves through a named barrier).  Per chunk of hidden channels the workers
+//   A. read the expansion accumulators, apply scale, bias and activation and park the chunk as
+//      float32 in shared memory ([4-channel plane][row][W + 2 columns][16 bytes]: a zero column on
+//      both sides, written once; rows outside the image are the depthwise layer's zero padding and
+//      are stored as zeros),
+//   D. run the depthwise 3x3 from the parked chunk (a lane per output pixel, four channels per
+//      lane, the nine weights of the plane in registers; nine unconditional 16-byte loads), apply
+//      scale, bias, activation and write the result as hi / lo bfloat16 planes: the A operand of
+//      the projection;
+// the issuing warp
+//   - starts the bulk copy of the next expansion image as soon as the chunk's expansion MMAs are done,
+//   - issues the expansion MMAs of the NEXT chunk (hi and lo halves of the pixels, all tiles of the
+//     band into separate accumulator columns) once every worker has read the accumulators: they run
+//     behind D,
+//   - issues the projection MMAs of the chunk once every worker has written its part of the operand;
+//     they add to the block's output accumulator (128 pixels x Cout) in tensor memory and run behind
+//     A of the next chunk; then it fetches the next projection image.
+// After the last chunk the workers give the accumulator scale, bias and the shortcut and store it.
+// One warp polls an mbarrier on behalf of the workers (seventeen polling warps were measured to slow
+// the MMAs they wait for); whether to go on after a wait is decided by one thread before the named
+// barrier and read by all after it, so all workers leave at the same barrier.  Every wait is bounded
+// as in the other tcgen05 kernels.
 #include "tc_ptx.cuh"
 
 #include <algorithm>
