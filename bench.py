@@ -63,7 +63,7 @@ def eval_workload(name):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from one ncu
 # capture, per image of the evaluator pass (traffic grows in proportion to the images of a launch;
 # the capture runs a smaller pass than the benchmark).  None until captured / after the kernel changed.
-NCU_TRAFFIC_BYTES_PER_LAUNCH_PER_IMAGE = 0.637e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH_PER_IMAGE = 0.629e6
 NCU_TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum of the 15 row-streaming launches of one evaluator pass, "
                     "captured at 512 images per pass and scaled to this run's pass size by the images per launch")
 
