@@ -262,8 +262,9 @@ aiq_status_t aiq_forward(const aiq_model_t* model, const uint8_t* scheme_bits, c
  *     and launches nothing; lower the batch or use aiq_forward.  8 MiB fits, e.g.,
  *     ResNet-20 up to batch 32.
  *   - The first call on each device looks up the array's device address (one
- *     cudaGetSymbolAddress with that device current).  Make that first call outside any
- *     stream capture.
+ *     cudaGetSymbolAddress with that device current).  Like aiq_forward, the call plans on
+ *     the host and copies its job records from host memory: make no call of it while the
+ *     stream is being captured.
  *   - All calls on a device share the one array and it keeps whatever the previous call
  *     left there.  A forward pass needs nothing zeroed, so nothing is cleared; but two calls
  *     whose kernels overlap on the GPU (different streams, or different host threads) write
