@@ -462,6 +462,98 @@ conv_stem_rs_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* 
   }
 }
 
+// Stride-1 stem for ACT_RS with the input staged in shared memory.  A block owns kStemRows output
+// rows of one group of G images: the kStemRows + 2 input rows of every channel and image arrive
+// by coalesced 16-byte loads (the kernel above gathers 27 scattered words per thread) and are
+// held as [channel][row][image][column + 1 zero column on both sides], 4 words of slack per
+// row so that the 8 images x 4 columns of a warp read 32 different banks.  A thread owns one
+// (image, column) and walks down the rows.  Same arithmetic order as the gathering kernel.
+constexpr int kStemRows = 4;
+
+template <int COUT>
+__global__ void __launch_bounds__(256)
+conv_stem_rs_rows_kernel(ConvGeom g, const LayerJob* __restrict__ jobs, const float* __restrict__ net_input) {
+  extern __shared__ __align__(16) float stem_sm[];            // weights, scale, bias, input tile
+  const LayerJob job = jobs[blockIdx.z];
+  const int Kt = 9 * g.Cin;
+  float* wsm = stem_sm;
+  float* ssm = wsm + Kt * COUT;
+  float* bsm = ssm + COUT;
+  float* tile = bsm + COUT;
+  const int G = rs_group_images_dev(g.Wo);
+  const int RS = g.W + 4;                                      // words of a tile row
+  const int n_threads = blockDim.x;
+  const int wrow_bytes = ((g.K + 31) / 32 * 32) * job.bits / 8;
+  for (int i = threadIdx.x; i < Kt * COUT; i += n_threads) {
+    const int k = i / COUT, n = i - k * COUT;
+    const int tap = k / g.Cin, c = k - tap * g.Cin;
+    wsm[i] = load_element(job.w + (size_t)n * wrow_bytes, c * 9 + tap, job.bits);
+  }
+  for (int n = threadIdx.x; n < COUT; n += n_threads) { ssm[n] = job.scale[n]; bsm[n] = job.bias[n]; }
+  const int row_blocks = g.Ho / kStemRows;
+  const int grp = blockIdx.x / row_blocks, oy0 = (blockIdx.x - grp * row_blocks) * kStemRows;
+  // input rows oy0 - 1 .. oy0 + kStemRows of every channel and image of the group
+  const int W4 = g.W / 4;
+  const int n_quads = g.Cin * (kStemRows + 2) * G * W4;
+  for (int i = threadIdx.x; i < n_quads; i += n_threads) {
+    const int x4 = i % W4, img = (i / W4) % G, r = (i / (W4 * G)) % (kStemRows + 2), c = i / (W4 * G * (kStemRows + 2));
+    const int iy = oy0 - 1 + r, b = grp * G + img;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (iy >= 0 && iy < g.H && b < g.B)
+      v = __ldg(reinterpret_cast<const float4*>(net_input + (((size_t)b * g.Cin + c) * g.H + iy) * g.W) + x4);
+    float* dst = tile + ((size_t)(c * (kStemRows + 2) + r) * G + img) * RS + 1 + 4 * x4;
+    dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+  }
+  for (int i = threadIdx.x; i < g.Cin * (kStemRows + 2) * G * 2; i += n_threads)    // the zero columns
+    tile[(size_t)(i >> 1) * RS + ((i & 1) ? g.W + 1 : 0)] = 0.f;
+  __syncthreads();
+
+  const int img = threadIdx.x % G, ox = threadIdx.x / G;
+  const size_t plane_bytes = (size_t)G * 16;
+  for (int ry = 0; ry < kStemRows; ++ry) {
+    float acc[COUT];
+#pragma unroll
+    for (int n = 0; n < COUT; ++n) acc[n] = 0.f;
+    for (int c = 0; c < g.Cin; ++c) {
+#pragma unroll
+      for (int r = 0; r < 3; ++r) {
+        const float* row = tile + ((size_t)(c * (kStemRows + 2) + ry + r) * G + img) * RS + ox;
+#pragma unroll
+        for (int t = 0; t < 3; ++t) {
+          const float xv = row[t];
+          const float* wk = wsm + ((r * 3 + t) * g.Cin + c) * COUT;
+#pragma unroll
+          for (int n = 0; n < COUT; n += 4) {
+            const float4 wv = *reinterpret_cast<const float4*>(wk + n);
+            acc[n] = fmaf(xv, wv.x, acc[n]);
+            acc[n + 1] = fmaf(xv, wv.y, acc[n + 1]);
+            acc[n + 2] = fmaf(xv, wv.z, acc[n + 2]);
+            acc[n + 3] = fmaf(xv, wv.w, acc[n + 3]);
+          }
+        }
+      }
+    }
+    uint8_t* dst = static_cast<uint8_t*>(job.out) +
+                   ((((size_t)grp * g.Ho + oy0 + ry) * g.Wo + ox) * (COUT / 4)) * plane_bytes + (size_t)img * 16;
+#pragma unroll
+    for (int n = 0; n < COUT; n += 8) {
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int e = 0; e < 8; e += 2) {
+        const float u0 = apply_act(fmaf(acc[n + e], ssm[n + e], bsm[n + e]), g.act);
+        const float u1 = apply_act(fmaf(acc[n + e + 1], ssm[n + e + 1], bsm[n + e + 1]), g.act);
+        __nv_bfloat16 h0, l0, h1, l1;
+        split_bf16(u0, h0, l0);
+        split_bf16(u1, h1, l1);
+        hi[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+        lo[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+      }
+      *reinterpret_cast<uint4*>(dst + (size_t)(n / 8) * plane_bytes) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *reinterpret_cast<uint4*>(dst + (size_t)(COUT / 8 + n / 8) * plane_bytes) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    }
+  }
+}
+
 template <int COUT>
 aiq_status_t launch_stem(const ConvGeom& g, const LayerJob* jobs, int n_jobs, const float* net_input,
                          double weight_bytes, cudaStream_t s) {
@@ -473,7 +565,14 @@ aiq_status_t launch_stem(const ConvGeom& g, const LayerJob* jobs, int n_jobs, co
                     2.0 * g.B * g.Ho * g.Wo * g.Cout * (double)(9 * g.Cin) * n_jobs,
                     weight_bytes + 4.0 * n_jobs * ((double)g.B * g.Cin * g.H * g.W +
                                                    (double)g.B * g.Ho * g.Wo * g.Cout));
-  if (g.act_format == ACT_RS)
+  const int G = rs_group_images(g.Wo);
+  const size_t tile_bytes = (size_t)g.Cin * (kStemRows + 2) * G * (g.W + 4) * sizeof(float);
+  if (g.act_format == ACT_RS && g.stride == 1 && g.W == g.Wo && g.H == g.Ho && g.W % 4 == 0 && g.Ho % kStemRows == 0 &&
+      G * g.Wo <= 256 && (G * g.Wo) % 32 == 0 && smem + tile_bytes <= 100 * 1024) {
+    AIQ_ENSURE_DYNAMIC_SMEM((conv_stem_rs_rows_kernel<COUT>), 100 * 1024);
+    const dim3 rgrid((unsigned)(rs_padded_batch(g.B) / G * (g.Ho / kStemRows)), 1, n_jobs);
+    conv_stem_rs_rows_kernel<COUT><<<rgrid, G * g.Wo, smem + tile_bytes, s>>>(g, jobs, net_input);
+  } else if (g.act_format == ACT_RS)
     conv_stem_rs_kernel<COUT><<<grid, kStemThreads, smem, s>>>(g, jobs, net_input);
   else if (g.act_format == ACT_SPLIT)
     conv_stem_kernel<COUT, ACT_SPLIT><<<grid, kStemThreads, smem, s>>>(g, jobs, net_input);
