@@ -257,8 +257,8 @@ aiq_status_t aiq_forward(const aiq_model_t* model, const uint8_t* scheme_bits, c
  *
  * Same arguments, results and asynchrony as aiq_forward, minus the workspace.  The call
  * makes no cudaMalloc / cudaFree and uses no allocating library routine.
- *   - Limit: if the model at this batch needs more than AIQ_STATIC_WORKSPACE_BYTES (see
- *     aiq_workspace_bytes(model, batch, 1)) the call returns AIQ_ERR_WORKSPACE_TOO_SMALL
+ *   - Limit: if the model at this batch needs more than AIQ_STATIC_WORKSPACE_BYTES in its own
+ *     activation format (aiq_workspace_bytes(model, batch, 1) after aiq_set_small_pass_images(0)) the call returns AIQ_ERR_WORKSPACE_TOO_SMALL
  *     and launches nothing; lower the batch or use aiq_forward.  8 MiB fits, e.g.,
  *     ResNet-20 up to batch 32.
  *   - The first call on each device looks up the array's device address (one
@@ -310,6 +310,14 @@ void aiq_set_eval_options(int chunk, int share_prefix);
  *           produces its input; that tensor is then never stored.  Sums are formed in a fixed order
  *           (run-to-run identical); they differ from the separate pooling kernel's in the last bits. */
 void aiq_set_fusion(int blocks, int pool);
+
+/* Small passes (process-wide; evaluation cost, Section 2.2).  The row-streaming kernels work on groups of 8 or
+ * 16 images, so a pass of a few hundred images leaves most SMs idle.  A model created under
+ * AIQ_PATH_AUTO that stores its activations in the row-streaming format also keeps the pixel-tile view of
+ * the same weights; aiq_forward and aiq_eval_schemes run a pass of fewer than `image_schemes` (images of the
+ * pass x schemes; default 1024) on that view.  0: always the row-streaming kernels.  Both views meet the same
+ * tolerances; their logits differ in the last bits.  aiq_forward_static always uses the model's own format. */
+void aiq_set_small_pass_images(int image_schemes);
 
 /* Compute path of models created after the call (process-wide; the paper has no kernels,
  * Section 3 runs stock PyTorch, so this is an implementation choice, not a step of AIQ):

@@ -24,7 +24,7 @@ EXPORTS = [
     "aiq_quantize_layer", "aiq_qlinear", "aiq_qlinear_workspace_bytes", "aiq_model_bytes", "aiq_model_create",
     "aiq_model_destroy", "aiq_model_num_layers", "aiq_model_num_classes",
     "aiq_model_layer_folded", "aiq_model_layer_packed", "aiq_workspace_bytes", "aiq_forward",
-    "aiq_eval_schemes", "aiq_set_eval_options", "aiq_set_fusion", "aiq_quantize_layer_per_tensor", "aiq_set_scale_granularity", "aiq_last_call_stats", "aiq_scheme_ai",
+    "aiq_eval_schemes", "aiq_set_eval_options", "aiq_set_fusion", "aiq_set_small_pass_images", "aiq_quantize_layer_per_tensor", "aiq_set_scale_granularity", "aiq_last_call_stats", "aiq_scheme_ai",
     "aiq_profile_start", "aiq_profile_stop", "aiq_forward_static",
     "aiq_set_compute_path", "aiq_model_status", "aiq_debug_expire_wait", "aiq_search_greedy", "aiq_search_coordinate_descent",
 ]
@@ -116,6 +116,8 @@ def _load():
     lib.aiq_set_scale_granularity.argtypes = [i32]
     lib.aiq_set_fusion.restype = None
     lib.aiq_set_fusion.argtypes = [i32, i32]
+    lib.aiq_set_small_pass_images.restype = None
+    lib.aiq_set_small_pass_images.argtypes = [i32]
     lib.aiq_last_call_stats.restype = None
     lib.aiq_last_call_stats.argtypes = [C.POINTER(C.c_int64)] * 3
     lib.aiq_search_greedy.restype = i32
@@ -236,6 +238,10 @@ def aiq_quantize_layer_per_tensor(W, bits, packed_out, scales_out, scratch, nonf
 
 def aiq_set_fusion(blocks=True, pool=True, inverted_residual=False):
     lib.aiq_set_fusion(int(bool(blocks)) | (2 if inverted_residual else 0), int(bool(pool)))
+
+
+def aiq_set_small_pass_images(image_schemes):
+    lib.aiq_set_small_pass_images(int(image_schemes))
 
 
 def aiq_set_compute_path(path):

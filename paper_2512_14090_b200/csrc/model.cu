@@ -27,7 +27,8 @@ static std::atomic<int> g_opt_share{1};
 static std::atomic<int> g_opt_path{AIQ_PATH_AUTO};
 static std::atomic<int> g_opt_per_tensor{0};  // scale granularity of models created afterwards
 static std::atomic<int> g_opt_fuse{1};        // bit 0: basic blocks as one kernel; bit 1: inverted-residual blocks as one kernel
-static std::atomic<int> g_opt_fuse_pool{1};   // average pool inside the last convolution's epilogue
+static std::atomic<int> g_opt_fuse_pool{1};
+static std::atomic<int> g_opt_small_pass{1024};   // image-schemes per pass below which the small view runs   // average pool inside the last convolution's epilogue
 
 aiq_status_t set_error(aiq_status_t status, const char* fmt, ...) {
   va_list ap;
@@ -141,6 +142,8 @@ struct aiq_model {
   std::vector<int> block_tail;       // per layer: the second convolution of the basic block this layer opens
                                      // (the pair can run as one kernel), or -1
   int pool_layer;                    // the layer whose epilogue can do the classifier's average pool, or -1
+  aiq_model* small_view = nullptr;   // the same weights with split activations and the pixel-tile kernels, for passes
+                                     // too small to fill the row-streaming kernels (owned; else nullptr)
   std::vector<int> mb_mid, mb_tail;  // per layer: the depthwise and the projection layer of the inverted-residual
                                      // block this (expansion) layer opens (the three can run as one kernel), or -1
 };
@@ -359,42 +362,12 @@ static ModelLayout model_layout(const std::vector<LayerInfo>& L) {
   return lay;
 }
 
-}  // namespace aiq
-
-extern "C" size_t aiq_model_bytes(const aiq_arch_desc_t* arch) {
-  std::vector<LayerInfo> L;
-  std::vector<int> order;
-  if (aiq::infer_shapes(arch, L, order) != AIQ_OK) return 0;
-  return aiq::model_layout(L).total;
-}
-
-extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_layer_weights_t* weights,
-                                         void* dev_mem, size_t dev_bytes, void* stream_, aiq_model_t** out) {
-  using namespace aiq;
-  if (out) *out = nullptr;
-  if (!arch || !weights || !dev_mem || !out) return set_error(AIQ_ERR_INVALID_ARG, "aiq_model_create: null pointer");
-  if (((uintptr_t)dev_mem) & 255) return set_error(AIQ_ERR_INVALID_ARG, "aiq_model_create: dev_mem not 256-byte aligned");
-  aiq_model* m = new (std::nothrow) aiq_model();
-  if (!m) return set_error(AIQ_ERR_INVALID_ARG, "out of host memory");
-  aiq_status_t st = infer_shapes(arch, m->layers, m->order);
-  if (st != AIQ_OK) { delete m; return st; }
-  for (int i = 0; i < arch->n_layers; ++i) {
-    const aiq_layer_weights_t& w = weights[i];
-    if (!w.W || (m->layers[i].d.has_bn && (!w.gamma || !w.beta || !w.mean || !w.var))) {
-      delete m;
-      return set_error(AIQ_ERR_INVALID_ARG, "layer %d: missing weight pointers", i);
-    }
-  }
-  const ModelLayout lay = model_layout(m->layers);
-  if (dev_bytes < lay.total) {
-    delete m;
-    return set_error(AIQ_ERR_WORKSPACE_TOO_SMALL, "model needs %zu device bytes, got %zu", lay.total, dev_bytes);
-  }
-  st = check_device_sm100();
-  if (st != AIQ_OK) { delete m; return st; }
-  m->in_c = arch->in_c; m->in_h = arch->in_h; m->in_w = arch->in_w;
-  m->dev_mem = dev_mem; m->dev_bytes = dev_bytes;
-  const int opt_path = g_opt_path.load();
+// Everything about a model that depends on the activation format: the format itself (from the requested
+// compute path and what the layers allow), per-image tensor sizes, the fused blocks and pooled epilogue the
+// format's kernels can take, and the activation slots.
+static void derive_format(aiq_model* m, int opt_path) {
+  for (LayerInfo& li : m->layers)
+    if (li.d.kind != AIQ_LAYER_FC) li.out_bytes = split_image_bytes(li.Ho, li.Wo, li.d.cout);
   // Row-streaming storage when every layer can live in it: a 3x3 stem on the network input, then
   // only dense convolutions the row-streaming kernel takes, then the classifier.
   m->act_format = ACT_RS;
@@ -466,6 +439,44 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
     }
   }
   assign_slots(m);
+}
+
+}  // namespace aiq
+
+extern "C" size_t aiq_model_bytes(const aiq_arch_desc_t* arch) {
+  std::vector<LayerInfo> L;
+  std::vector<int> order;
+  if (aiq::infer_shapes(arch, L, order) != AIQ_OK) return 0;
+  return aiq::model_layout(L).total;
+}
+
+extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_layer_weights_t* weights,
+                                         void* dev_mem, size_t dev_bytes, void* stream_, aiq_model_t** out) {
+  using namespace aiq;
+  if (out) *out = nullptr;
+  if (!arch || !weights || !dev_mem || !out) return set_error(AIQ_ERR_INVALID_ARG, "aiq_model_create: null pointer");
+  if (((uintptr_t)dev_mem) & 255) return set_error(AIQ_ERR_INVALID_ARG, "aiq_model_create: dev_mem not 256-byte aligned");
+  aiq_model* m = new (std::nothrow) aiq_model();
+  if (!m) return set_error(AIQ_ERR_INVALID_ARG, "out of host memory");
+  aiq_status_t st = infer_shapes(arch, m->layers, m->order);
+  if (st != AIQ_OK) { delete m; return st; }
+  for (int i = 0; i < arch->n_layers; ++i) {
+    const aiq_layer_weights_t& w = weights[i];
+    if (!w.W || (m->layers[i].d.has_bn && (!w.gamma || !w.beta || !w.mean || !w.var))) {
+      delete m;
+      return set_error(AIQ_ERR_INVALID_ARG, "layer %d: missing weight pointers", i);
+    }
+  }
+  const ModelLayout lay = model_layout(m->layers);
+  if (dev_bytes < lay.total) {
+    delete m;
+    return set_error(AIQ_ERR_WORKSPACE_TOO_SMALL, "model needs %zu device bytes, got %zu", lay.total, dev_bytes);
+  }
+  st = check_device_sm100();
+  if (st != AIQ_OK) { delete m; return st; }
+  m->in_c = arch->in_c; m->in_h = arch->in_h; m->in_w = arch->in_w;
+  m->dev_mem = dev_mem; m->dev_bytes = dev_bytes;
+  derive_format(m, g_opt_path.load());
   cudaStream_t stream = (cudaStream_t)stream_;
   uint8_t* base = static_cast<uint8_t*>(dev_mem);
   int32_t* flag = reinterpret_cast<int32_t*>(base + lay.flag_off);
@@ -549,11 +560,24 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
 #undef CREATE_TRY
   if (host_flag == 2) return fail(set_error(AIQ_ERR_TIMEOUT, "a bounded wait inside the quantizer expired"));
   if (host_flag) return fail(set_error(AIQ_ERR_NONFINITE, "a weight is NaN or infinite"));
+  // Row-streaming kernels take a group of 8 or 16 images as their unit of work; a pass of a few hundred images
+  // leaves most SMs idle.  Under the automatic path the model also keeps the pixel-tile view of the same weights.
+  if (m->act_format == ACT_RS && g_opt_path.load() == AIQ_PATH_AUTO) {
+    aiq_model* v = new (std::nothrow) aiq_model(*m);
+    if (v) {
+      v->small_view = nullptr;
+      derive_format(v, AIQ_PATH_TENSOR_TILES);
+      m->small_view = v;
+    }
+  }
   *out = m;
   return AIQ_OK;
 }
 
-extern "C" void aiq_model_destroy(aiq_model_t* model) { delete model; }
+extern "C" void aiq_model_destroy(aiq_model_t* model) {
+  if (model) delete model->small_view;
+  delete model;
+}
 extern "C" aiq_status_t aiq_model_status(const aiq_model_t* model, void* stream_) {
   using namespace aiq;
   if (!model) return set_error(AIQ_ERR_INVALID_ARG, "aiq_model_status: null model");
@@ -1011,9 +1035,25 @@ static aiq_status_t run_chunk(const aiq_model* m, const EvalPlan& plan, const La
 
 }  // namespace aiq
 
+namespace aiq {
+// The view of the model a pass of `batch` images under `n_schemes` schemes runs on.
+static const aiq_model* pick_view(const aiq_model* m, int batch, int n_schemes) {
+  if (!m->small_view) return m;
+  return (long long)batch * n_schemes < (long long)g_opt_small_pass.load() ? m->small_view : m;
+}
+}  // namespace aiq
+
 extern "C" size_t aiq_workspace_bytes(const aiq_model_t* model, int max_batch, int max_schemes) {
   if (!model || max_batch <= 0 || max_schemes <= 0) return 0;
-  return aiq::ws_layout(model, max_batch, max_schemes).total;
+  size_t bytes = aiq::ws_layout(model, max_batch, max_schemes).total;
+  const int small_pass = aiq::g_opt_small_pass.load();     // the small view never sees a pass of this many images
+  if (model->small_view && small_pass > 0)
+    bytes = std::max(bytes, aiq::ws_layout(model->small_view, std::min(max_batch, small_pass), max_schemes).total);
+  return bytes;
+}
+
+extern "C" void aiq_set_small_pass_images(int image_schemes) {
+  aiq::g_opt_small_pass = image_schemes > 0 ? image_schemes : 0;
 }
 
 extern "C" void aiq_set_eval_options(int chunk, int share_prefix) {
@@ -1040,7 +1080,19 @@ extern "C" void aiq_last_call_stats(int64_t* kernel_launches, int64_t* layer_eva
   if (layer_evals_unshared) *layer_evals_unshared = aiq::t_layer_evals_unshared;
 }
 
+static aiq_status_t forward_on_view(const aiq_model_t* model, const uint8_t* scheme_bits, const float* x,
+                                    int batch, float* logits, void* workspace, size_t workspace_bytes,
+                                    void* stream_);
+
 extern "C" aiq_status_t aiq_forward(const aiq_model_t* model, const uint8_t* scheme_bits, const float* x,
+                                    int batch, float* logits, void* workspace, size_t workspace_bytes,
+                                    void* stream_) {
+  if (!model) return aiq::set_error(AIQ_ERR_INVALID_ARG, "aiq_forward: null pointer");
+  return forward_on_view(batch > 0 ? aiq::pick_view(model, batch, 1) : model, scheme_bits, x, batch, logits, workspace,
+                         workspace_bytes, stream_);
+}
+
+static aiq_status_t forward_on_view(const aiq_model_t* model, const uint8_t* scheme_bits, const float* x,
                                     int batch, float* logits, void* workspace, size_t workspace_bytes,
                                     void* stream_) {
   using namespace aiq;
@@ -1068,11 +1120,16 @@ extern "C" aiq_status_t aiq_forward(const aiq_model_t* model, const uint8_t* sch
   return st;
 }
 
-extern "C" aiq_status_t aiq_eval_schemes(const aiq_model_t* model, const uint8_t* schemes, int n_schemes,
+extern "C" aiq_status_t aiq_eval_schemes(const aiq_model_t* model_in, const uint8_t* schemes, int n_schemes,
                                          const float* x, const int32_t* labels, int n_images, float* acc,
                                          int32_t* correct_counts, int32_t* preds, void* workspace,
                                          size_t workspace_bytes, void* stream_) {
   using namespace aiq;
+  const aiq_model_t* model = model_in;
+  if (model_in && n_schemes > 0 && n_images > 0) {
+    const int want = g_opt_chunk.load() > 0 ? g_opt_chunk.load() : 1024;
+    model = pick_view(model_in, std::min(want, n_images), n_schemes);
+  }
   if (!model || !schemes || !x || !labels || !acc || !workspace)
     return set_error(AIQ_ERR_INVALID_ARG, "aiq_eval_schemes: null pointer");
   if (n_schemes <= 0 || n_images <= 0)
@@ -1190,7 +1247,7 @@ extern "C" aiq_status_t aiq_forward_static(const aiq_model_t* model, const uint8
   }
   // Nothing in the workspace has to start at zero for a forward pass: the job records are
   // copied in, and every activation, pooled value and logit is written before it is read.
-  return aiq_forward(model, scheme_bits, x, batch, logits, ws_ptr,
+  return forward_on_view(model, scheme_bits, x, batch, logits, ws_ptr,
                      (size_t)AIQ_STATIC_WORKSPACE_BYTES, stream_);
 }
 

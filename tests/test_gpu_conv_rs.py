@@ -16,6 +16,15 @@ from gpu_util import binding, to_dev, assert_logits_close, compute_path
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(autouse=True)
+def _row_streaming_kernels_at_any_batch():
+    """These tests are about the row-streaming kernels: keep small passes on them."""
+    aiq = binding()
+    aiq.aiq_set_small_pass_images(0)
+    yield
+    aiq.aiq_set_small_pass_images(1024)
+
+
 def _conv(name, cin, cout, k, stride, act, inp, residual=-1):
     return dict(name=name, kind="conv", cin=cin, cout=cout, k=k, stride=stride, pad=k // 2, act=act,
                 input=inp, residual=residual, has_bn=True)
