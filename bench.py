@@ -503,7 +503,7 @@ def main():
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # > L2 (126 MB)
     mem = model.mem
     launches = [0]
-    bank_launches = sum(1 for l in arch["layers"] if l["has_bn"]) + 4 * L   # fold + 4 quantize per layer
+    bank_launches = sum(1 for l in arch["layers"] if l["has_bn"]) + L   # per layer: fold, one quantizer launch for the four widths
     result = {}
 
     def step(x, labels):

@@ -165,6 +165,9 @@ aiq_status_t launch_fold_bn(const float* W, const float* gamma, const float* bet
 // tensor_amax: nullptr = one scale per row; else device scratch word and one scale for the whole tensor
 aiq_status_t launch_quantize(const float* W, int N, int K, int bits, void* packed, float* scales,
                              int32_t* nonfinite_flag, uint32_t* tensor_amax, cudaStream_t s);
+// all four widths (4, 8, 16, 32 bits, in that order) of one layer from one read of W; tensor_amax as above, for the 4- and 8-bit codes
+aiq_status_t launch_quantize_bank(const float* W, int N, int K, void* const* packed, float* const* scales,
+                                  int32_t* nonfinite_flag, uint32_t* tensor_amax, cudaStream_t s);
 // y[m][n] for every job: in = x [M][K], out = y [M][N]
 aiq_status_t launch_qlinear(const LayerJob* jobs_dev, const LayerJob* single_host, int n_jobs, int N,
                             int K, int M, cudaStream_t s);

@@ -522,9 +522,10 @@ extern "C" aiq_status_t aiq_model_create(const aiq_arch_desc_t* arch, const aiq_
       if (w.bias) CREATE_TRY(cudaMemcpyAsync(li.bias, w.bias, n * 4, cudaMemcpyHostToDevice, stream));
       else CREATE_TRY(cudaMemsetAsync(li.bias, 0, n * 4, stream));
     }
-    for (int b = 0; b < 4; ++b) {
-      st = launch_quantize(li.Wf, (int)n, (int)k, kBitsList[b], li.packed[b], li.scales[b], flag,
-                           per_tensor ? reinterpret_cast<uint32_t*>(flag + 2) : nullptr, stream);
+    {
+      void* packed4[4] = {li.packed[0], li.packed[1], li.packed[2], li.packed[3]};
+      st = launch_quantize_bank(li.Wf, (int)n, (int)k, packed4, li.scales, flag,
+                                per_tensor ? reinterpret_cast<uint32_t*>(flag + 2) : nullptr, stream);
       if (st != AIQ_OK) return fail(st);
     }
   }

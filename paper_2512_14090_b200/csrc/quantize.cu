@@ -6,6 +6,8 @@
 // intrinsics), so codes and scales are reproducible bit for bit.
 #include "common.cuh"
 
+#include <type_traits>
+
 namespace aiq {
 
 // ---------------------------------------------------------------------------------------
@@ -186,6 +188,81 @@ quantize_rows_kernel(const float* __restrict__ W, int K, int Kpad,
   }
 }
 
+// All four bit-widths of a layer from one read of its rows (the weight bank of a model: the
+// per-width kernel above would be launched four times on the same small matrix).  Same
+// quantizer and packing routines, so the bytes equal those of four separate calls.
+struct BankOut { uint8_t* packed[4]; float* scales[4]; };
+
+template <int CACHE>
+__global__ void __launch_bounds__(256, CACHE == 1 ? 4 : 3)
+quantize_bank_kernel(const float* __restrict__ W, int K, int Kpad, BankOut out, int32_t* __restrict__ nonfinite_flag,
+                     const uint32_t* __restrict__ tensor_amax) {
+  const int n = blockIdx.x;
+  const float* row = W + (size_t)n * K;
+  const int n_gran = Kpad >> 3;
+  const bool vec_ok = ((K & 3) == 0) && ((((uintptr_t)row) & 15) == 0);
+  float v[CACHE][8];
+  uint32_t amax_bits = 0;
+  auto load_granule = [&](int gi, float* dstv) {
+    const int k0 = gi << 3;
+    if (vec_ok && k0 + 8 <= K) {
+      const float4 a = __ldg(reinterpret_cast<const float4*>(row + k0));
+      const float4 b = __ldg(reinterpret_cast<const float4*>(row + k0 + 4));
+      dstv[0] = a.x; dstv[1] = a.y; dstv[2] = a.z; dstv[3] = a.w;
+      dstv[4] = b.x; dstv[5] = b.y; dstv[6] = b.z; dstv[7] = b.w;
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) dstv[j] = (k0 + j < K) ? __ldg(row + k0 + j) : 0.0f;
+    }
+  };
+#pragma unroll
+  for (int c = 0; c < CACHE; ++c) {
+    const int gi = threadIdx.x + c * blockDim.x;
+    if (gi < n_gran) {
+      load_granule(gi, v[c]);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) amax_bits = max(amax_bits, absbits(v[c][j]));
+    }
+  }
+  for (int gi = threadIdx.x + CACHE * blockDim.x; gi < n_gran; gi += blockDim.x) {
+    float t[8];
+    load_granule(gi, t);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) amax_bits = max(amax_bits, absbits(t[j]));
+  }
+  __shared__ uint32_t s_max[8];
+  amax_bits = __reduce_max_sync(0xffffffffu, amax_bits);
+  if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax_bits;
+  __syncthreads();
+  amax_bits = 0;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) amax_bits = max(amax_bits, s_max[w]);
+  if (amax_bits >= kInfBits) {
+    if (threadIdx.x == 0 && nonfinite_flag) *nonfinite_flag = 1;
+    return;
+  }
+  const uint32_t code_amax = tensor_amax ? *tensor_amax : amax_bits;   // per-tensor scales apply to the integer codes only
+  auto emit = [&](auto bits_tag, int slot, uint32_t amax) {
+    constexpr int BITS = decltype(bits_tag)::value;
+    const RowQuantizer rq(__uint_as_float(amax), BITS);
+    if (threadIdx.x == 0) out.scales[slot][n] = rq.s;
+    uint8_t* out_row = out.packed[slot] + (size_t)n * ((size_t)Kpad * BITS / 8);
+#pragma unroll
+    for (int c = 0; c < CACHE; ++c) {
+      const int gi = threadIdx.x + c * blockDim.x;
+      if (gi < n_gran) store_granule<BITS>(out_row, gi, v[c], rq);
+    }
+    for (int gi = threadIdx.x + CACHE * blockDim.x; gi < n_gran; gi += blockDim.x) {
+      float t[8];
+      load_granule(gi, t);
+      store_granule<BITS>(out_row, gi, t, rq);
+    }
+  };
+  emit(std::integral_constant<int, 4>(), 0, code_amax);
+  emit(std::integral_constant<int, 8>(), 1, code_amax);
+  emit(std::integral_constant<int, 16>(), 2, amax_bits);
+  emit(std::integral_constant<int, 32>(), 3, amax_bits);
+}
+
 // --- streaming kernel for large matrices (the roofline case): persistent blocks, every row
 // arrives in shared memory by one bulk copy issued kStreamStages rows ahead, so the memory
 // system stays busy while a block reduces, rounds and packs.  A row goes from shared memory
@@ -358,6 +435,41 @@ aiq_status_t launch_quantize(const float* W, int N, int K, int bits, void* packe
     case 16: return launch_quantize_bits<16>(W, N, K, packed, scales, nonfinite_flag, nullptr, s);
     default: return launch_quantize_bits<32>(W, N, K, packed, scales, nonfinite_flag, nullptr, s);
   }
+}
+
+// The four versions (4, 8, 16, 32 bits) of one layer of a model's weight bank.
+aiq_status_t launch_quantize_bank(const float* W, int N, int K, void* const* packed, float* const* scales,
+                                  int32_t* nonfinite_flag, uint32_t* tensor_amax, cudaStream_t s) {
+  static const int kBits[4] = {4, 8, 16, 32};
+  DeviceProps props;
+  if (aiq_status_t st = current_device_props(&props)) return st;
+  const int Kpad = padded_k(K), n_gran = Kpad / 8;
+  // large matrices take the streaming kernel, one launch per width
+  const bool stream_ok = !tensor_amax && K % 32 == 0 && K >= 2048 && N >= 4 * props.n_sms;
+  if (stream_ok) {
+    for (int b = 0; b < 4; ++b)
+      if (aiq_status_t st = launch_quantize(W, N, K, kBits[b], packed[b], scales[b], nonfinite_flag, nullptr, s)) return st;
+    return AIQ_OK;
+  }
+  double out_bytes = 0.0;
+  for (int b = 0; b < 4; ++b) out_bytes += (double)N * row_bytes(K, kBits[b]) + 4.0 * N;
+  LaunchScope scope(AIQ_KERNEL_QUANTIZE, s, 8.0 * N * K, 4.0 * N * K + out_bytes);
+  if (tensor_amax) {
+    AIQ_CUDA_TRY(cudaMemsetAsync(tensor_amax, 0, 4, s));
+    const size_t n = (size_t)N * K;
+    int blocks = (int)((n + 1023) / 1024);
+    if (blocks > 8 * props.n_sms) blocks = 8 * props.n_sms;
+    tensor_absmax_kernel<<<blocks, 256, 0, s>>>(W, n, tensor_amax);
+    AIQ_LAUNCH_CHECK("tensor_absmax");
+  }
+  BankOut out;
+  for (int b = 0; b < 4; ++b) { out.packed[b] = static_cast<uint8_t*>(packed[b]); out.scales[b] = scales[b]; }
+  int threads = 32;
+  while (threads < 256 && threads < n_gran) threads <<= 1;
+  if (n_gran <= threads) quantize_bank_kernel<1><<<N, threads, 0, s>>>(W, K, Kpad, out, nonfinite_flag, tensor_amax);
+  else quantize_bank_kernel<4><<<N, threads, 0, s>>>(W, K, Kpad, out, nonfinite_flag, tensor_amax);
+  AIQ_LAUNCH_CHECK("quantize_bank");
+  return AIQ_OK;
 }
 
 }  // namespace aiq
