@@ -318,8 +318,8 @@ def run_kernel_sweep(args):
     from paper_2512_14090_b200 import build
     build.build()
     from paper_2512_14090_b200 import binding as aiq
-    if args.fuse_inverted_residual:
-        aiq.aiq_set_fusion(True, True, inverted_residual=True)
+    if args.fuse_inverted_residual or args.no_fuse_inverted_residual:
+        aiq.aiq_set_fusion(True, True, inverted_residual=bool(args.fuse_inverted_residual))
     aiq.aiq_set_compute_path({"auto": aiq.PATH_AUTO, "tiles": aiq.PATH_TENSOR_TILES, "fp32": aiq.PATH_FP32}[args.path])
     from aiq_workloads import gen_linear_case
     peaks = measured_peaks()
@@ -448,7 +448,9 @@ def main():
                     help="compute path of models created by the kernel workloads: auto (row-streaming tensor-core "
                          "kernels where the network allows), tiles (pixel-tile tensor-core kernels), fp32")
     ap.add_argument("--fuse-inverted-residual", action="store_true",
-                    help="run MobileNetV2's inverted-residual blocks as one kernel each (aiq_set_fusion bit 1)")
+                    help="run every eligible inverted-residual block of MobileNetV2 as one kernel (aiq_set_fusion bit 1; "
+                         "the default fuses a block only where that was measured faster)")
+    ap.add_argument("--no-fuse-inverted-residual", action="store_true", help="never fuse inverted-residual blocks")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -469,8 +471,8 @@ def main():
     from paper_2512_14090_b200 import build
     build.build()
     from paper_2512_14090_b200 import binding as aiq          # fails loudly without libaiq.so
-    if args.fuse_inverted_residual:
-        aiq.aiq_set_fusion(True, True, inverted_residual=True)
+    if args.fuse_inverted_residual or args.no_fuse_inverted_residual:
+        aiq.aiq_set_fusion(True, True, inverted_residual=bool(args.fuse_inverted_residual))
     from paper_2512_14090_b200.sharding import reduce_counts
     from aiq_workloads import gen_model, gen_images
 

@@ -302,10 +302,13 @@ void aiq_set_eval_options(int chunk, int share_prefix);
  *           convolutions of 16 or 32 channels runs as one kernel whenever every scheme of the call gives
  *           both convolutions 4 or 8 bits: the intermediate tensor stays in shared memory.  Results are
  *           bit-identical to the layer-by-layer path.
- *           bit 1 (default off): a MobileNetV2 inverted-residual block (expansion 1x1 -> depthwise 3x3 ->
+ *           bit 2 (default on) / bit 1 (default off): a MobileNetV2 inverted-residual block (expansion 1x1 -> depthwise 3x3 ->
  *           projection 1x1, optional shortcut) runs as one kernel whenever every scheme gives both 1x1
  *           layers 4 or 8 bits: the six-fold hidden tensor stays in shared memory (float32 there, so the
  *           results differ from the layer-by-layer path by that path's rounding of the hidden tensor).
+ *           Bit 2 fuses a block only where the fused kernel was measured faster than the three layer kernels
+ *           (maps at most 8 columns wide, or stride 2 on maps up to 56 wide, and at least 128 bands of
+ *           128 output pixels in the pass); bit 1 fuses every eligible block.
  *   pool:   the classifier's global average pool is taken in the epilogue of the convolution that
  *           produces its input; that tensor is then never stored.  Sums are formed in a fixed order
  *           (run-to-run identical); they differ from the separate pooling kernel's in the last bits. */

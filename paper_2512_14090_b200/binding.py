@@ -236,8 +236,10 @@ def aiq_quantize_layer_per_tensor(W, bits, packed_out, scales_out, scratch, nonf
                                              _dev(nonfinite_flag), _dev(scratch), _stream(stream)))
 
 
-def aiq_set_fusion(blocks=True, pool=True, inverted_residual=False):
-    lib.aiq_set_fusion(int(bool(blocks)) | (2 if inverted_residual else 0), int(bool(pool)))
+def aiq_set_fusion(blocks=True, pool=True, inverted_residual="auto"):
+    """inverted_residual: "auto" (fuse where measured faster), True (every eligible block), False."""
+    ir = 4 if inverted_residual == "auto" else (2 if inverted_residual else 0)
+    lib.aiq_set_fusion(int(bool(blocks)) | ir, int(bool(pool)))
 
 
 def aiq_set_small_pass_images(image_schemes):

@@ -219,6 +219,8 @@ __host__ __device__ inline size_t mb_ptile_bytes(int cs_out, int nh) { return (s
 // role 0: expansion, 1: projection, 2: depthwise (coefficients only); see mb_block.cu
 aiq_status_t launch_mb_build_tiles(int role, const uint8_t* packed, const float* scale, const float* bias, int bits, int N,
                                    int K, int nh, int cs, void* tile_out, float* coef_out, cudaStream_t s);
+// whether the fused kernel is expected to beat the layer kernels for this block at this batch (measured policy)
+bool mb_block_pays(const ConvGeom& gd, const ConvGeom& gp);
 // nh: the chunk width the jobs' operand images were built for
 aiq_status_t launch_mb_block(const ConvGeom& ge, const ConvGeom& gd, const ConvGeom& gp, int nh, const LayerJob* jobs_dev, int n_jobs,
                              int32_t* error_flag, double weight_bytes, cudaStream_t s);

@@ -584,6 +584,19 @@ int mb_block_chunk_channels(const ConvGeom& ge, const ConvGeom& gd, const ConvGe
   return c.ok ? c.NH : 0;
 }
 
+// Where the fused kernel was measured faster than the three layer kernels (B200, both MobileNetV2 variants, batches
+// 32 and 256): blocks on maps at most 8 columns wide and stride-2 blocks on maps up to 56 wide, once the batch
+// gives at least 128 CTAs; elsewhere (wide maps: many waves of short CTAs; few CTAs: the chunks of a CTA run one
+// after the other) the layer kernels win.
+bool mb_block_pays(const ConvGeom& gd, const ConvGeom& gp) {
+  DeviceProps props;
+  if (current_device_props(&props) != AIQ_OK) return false;
+  const int rb = std::min(std::max(128 / gp.Wo, 1), gp.Ho);        // band height of mb_config's first choice
+  const long long ctas = (long long)gp.B * ((gp.Ho + rb - 1) / rb);
+  if (ctas < 128) return false;
+  return gd.W <= 8 || (gd.stride == 2 && gd.W <= 56);
+}
+
 aiq_status_t launch_mb_build_tiles(int role, const uint8_t* packed, const float* scale, const float* bias, int bits, int N,
                                    int K, int nh, int cs, void* tile_out, float* coef_out, cudaStream_t s) {
   if ((role == 0 || role == 1) && bits != 4 && bits != 8)

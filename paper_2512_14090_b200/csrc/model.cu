@@ -26,7 +26,8 @@ static std::atomic<int> g_opt_chunk{0};
 static std::atomic<int> g_opt_share{1};
 static std::atomic<int> g_opt_path{AIQ_PATH_AUTO};
 static std::atomic<int> g_opt_per_tensor{0};  // scale granularity of models created afterwards
-static std::atomic<int> g_opt_fuse{1};        // bit 0: basic blocks as one kernel; bit 1: inverted-residual blocks as one kernel
+static std::atomic<int> g_opt_fuse{5};        // bit 0: basic blocks as one kernel; inverted-residual blocks as one kernel:
+                                              // bit 1: wherever eligible, bit 2: where measured faster (mb_block_pays)
 static std::atomic<int> g_opt_fuse_pool{1};
 static std::atomic<int> g_opt_small_pass{1024};   // image-schemes per pass below which the small view runs   // average pool inside the last convolution's epilogue
 
@@ -710,7 +711,7 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
   std::vector<std::vector<int>> ver(n, std::vector<int>(S, 0));   // ver[l][s]
   std::vector<std::vector<std::tuple<int, int, int>>> all_keys(n);   // per layer and version: (bits, input version, residual version)
   const bool fuse = (g_opt_fuse.load() & 1) != 0;
-  const bool fuse_mb = (g_opt_fuse.load() & 2) != 0;
+  const bool fuse_mb_all = (g_opt_fuse.load() & 2) != 0, fuse_mb_auto = (g_opt_fuse.load() & 4) != 0;
   // a basic block runs as one kernel when every scheme gives both of its convolutions 4 or 8 bits
   std::vector<int> fuse_head(n, -1);
   if (fuse)
@@ -724,12 +725,14 @@ static aiq_status_t build_plan(const aiq_model* m, const uint8_t* schemes, int S
   // an inverted-residual block runs as one kernel when every scheme gives its two 1x1 layers 4 or 8 bits
   std::vector<int> mb_head(n, -1);
   std::vector<char> mb_absorbed(n, 0);
-  if (fuse_mb)
+  if (fuse_mb_all || fuse_mb_auto)
     for (int le = 0; le < n; ++le) {
       const int lt = m->mb_tail[le];
       if (lt < 0) continue;
       bool ok = true;
       for (int s = 0; s < S && ok; ++s) ok = schemes[(size_t)s * n + le] <= 8 && schemes[(size_t)s * n + lt] <= 8;
+      if (ok && !fuse_mb_all)
+        ok = mb_block_pays(make_geom(m, m->layers[m->mb_mid[le]], B), make_geom(m, m->layers[lt], B));
       if (ok) { mb_head[lt] = le; mb_absorbed[le] = 1; mb_absorbed[m->mb_mid[le]] = 1; }
     }
   float* const pooled_base = reinterpret_cast<float*>(ws + wl.pooled_off);
@@ -1067,7 +1070,7 @@ extern "C" void aiq_set_scale_granularity(int granularity) {
 }
 
 extern "C" void aiq_set_fusion(int blocks, int pool) {
-  aiq::g_opt_fuse = blocks & 3;
+  aiq::g_opt_fuse = blocks & 7;
   aiq::g_opt_fuse_pool = pool ? 1 : 0;
 }
 

@@ -126,9 +126,18 @@ def test_mobilenet_v2_cifar_batch256_sampled():
     assert len(np.unique(O.predict(ref))) >= 3                # 16 images: several classes, small margins
     assert_tensor_path_logits(got[sample], ref, "mbv2 cifar batch=256")
     assert_preds_match(O.predict(got[sample]), O.predict(ref), O.top2_margin(ref), "mbv2 cifar batch=256")
-    # the same images alone give the same logits: no dependence on the batch around them
+    # the same images alone give the same logits: no dependence on the batch around them (with the same
+    # kernels: the default policy fuses some inverted-residual blocks at batch 256 and none at batch 16)
     alone = model.aiq_forward(scheme, to_dev(x[sample])).cpu().numpy()
-    assert np.array_equal(alone, got[sample])
+    assert_tensor_path_logits(alone, ref, "mbv2 cifar, the sampled images alone")
+    aiq.aiq_set_fusion(True, True, inverted_residual=False)
+    try:
+        got_plain = model.aiq_forward(scheme, to_dev(x)).cpu().numpy()
+        alone_plain = model.aiq_forward(scheme, to_dev(x[sample])).cpu().numpy()
+    finally:
+        aiq.aiq_set_fusion(True, True)
+    assert np.array_equal(alone_plain, got_plain[sample])
+    assert np.array_equal(alone_plain, alone)
 
 
 @pytest.mark.parametrize("path", ["fp32", "tensor"])

@@ -112,3 +112,23 @@ def test_mobilenet_v2_with_fused_blocks(variant, hw, batch):
     assert_tensor_path_logits(got, ref, f"mbv2 {variant} fused blocks")
     assert_preds_match(O.predict(got), O.predict(ref), O.top2_margin(ref), f"mbv2 {variant} fused blocks")
     model.close()
+
+
+def test_default_policy_fuses_where_it_pays():
+    """Under the default setting a block on an 8-wide map is fused once the pass has 128 bands, and not
+    below; the fused pass follows the oracle on sampled images."""
+    aiq = binding()
+    arch = inverted_residual_stack(160, 160, 8, 1)
+    params = gen_model(arch, 8401)
+    model = aiq.Model(arch, params)
+    bank = O.build_weight_bank(O.fold_model(arch, params), (8,))
+    scheme = np.full(5, 8, np.uint8)
+    x = gen_images(128, 3, 8, 8, 8402)
+    got = model.aiq_forward(scheme, to_dev(x)).cpu().numpy()
+    launches_big = aiq.aiq_last_call_stats()["kernel_launches"]
+    model.aiq_forward(scheme, to_dev(x[:100]))
+    launches_small = aiq.aiq_last_call_stats()["kernel_launches"]
+    assert launches_big == launches_small - 2
+    sample = np.arange(3, 128, 16)
+    assert_logits_close(got[sample], O.forward_scheme(arch, bank, scheme, x[sample]), "default policy, fused pass")
+    model.close()
